@@ -1,0 +1,252 @@
+/*
+ * mixgcn.h -- C ABI of libmixgcn.so: the single-GPU (sm_100a) hot path of full-graph GCN
+ * training as the MixGCN paper states it -- per layer, sparse neighbour aggregation with the
+ * propagation matrix followed by the dense node update (Eq. 3; Algorithm 2), then the loss,
+ * the backward pass and the weight update (Algorithm 2, last two lines of the iteration).
+ *
+ * Conventions
+ *  - Node-major storage: X = H^T is n x d, row-major fp32, with a leading dimension `ld`
+ *    (in elements) that is a multiple of 4 and >= d; every matrix pointer is 16-byte aligned.
+ *    Pad columns [d, ld) are never read as data; the library writes zeros or leaves them.
+ *    Weights W_l = [W^(l)]^T are d_in x d_out row-major, dense (ld = d_out), fp32.
+ *  - "device" pointers must be ordinary device memory of the context's GPU; "host" pointers
+ *    are ordinary host memory.  The caller owns every buffer passed in; the library owns only
+ *    the opaque context (status word, workspace, two internal streams) and graph objects.
+ *  - All compute calls are asynchronous on the caller's stream (`stream` is a cudaStream_t
+ *    passed as void*; NULL = legacy default stream) unless stated otherwise.
+ *  - Every function returns a mixgcn_status and never throws, aborts or traps.  On an error
+ *    detected on the host nothing is launched and outputs are untouched; the message is kept
+ *    per thread in mixgcn_last_error().  Conditions only the device can see (empty train
+ *    mask, label out of range) are written to the context's device status word, the kernel
+ *    produces zeros, and mixgcn_ctx_poll_status() reports them.
+ *  - Deterministic: no atomics on floating-point data; the same inputs give bitwise the same
+ *    outputs on every call.
+ */
+#ifndef MIXGCN_H_
+#define MIXGCN_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    MIXGCN_OK = 0,
+    MIXGCN_EINVAL = 1,        /* null / negative / misaligned argument */
+    MIXGCN_ENOMEM = 2,        /* device or host allocation failed */
+    MIXGCN_ECUDA = 3,         /* a CUDA runtime call failed; see mixgcn_last_error() */
+    MIXGCN_EUNSUPPORTED = 4,  /* valid request this build cannot serve */
+    MIXGCN_EBADGRAPH = 5,     /* node id out of range, unsorted CSR, n or nnz too large */
+    MIXGCN_ETIMEOUT = 6,      /* a bounded device-side wait gave up */
+    MIXGCN_EDEVICE = 7        /* a kernel reported bad data (empty mask, bad label) */
+} mixgcn_status;
+
+typedef struct mixgcn_ctx mixgcn_ctx;
+typedef struct mixgcn_graph mixgcn_graph;
+
+const char* mixgcn_status_string(mixgcn_status s);
+const char* mixgcn_last_error(void); /* thread-local, never NULL */
+
+/* Create / destroy a context bound to CUDA device `device`.  Allocates the status word and
+ * two internal streams.  Destroy synchronises the device. */
+mixgcn_status mixgcn_ctx_create(mixgcn_ctx** out, int device);
+mixgcn_status mixgcn_ctx_destroy(mixgcn_ctx* ctx);
+
+/* Pre-size the context's workspace (split-K partials, column-sum partials, loss partials) so
+ * that later calls allocate nothing.  Without it the workspace grows on demand (a
+ * cudaMalloc inside the first call that needs more). */
+mixgcn_status mixgcn_ctx_reserve(mixgcn_ctx* ctx, int64_t bytes);
+
+/* Synchronises the context's device, reads and clears the device status word.
+ * Returns MIXGCN_OK, MIXGCN_EDEVICE or MIXGCN_ETIMEOUT; *code (nullable) receives the raw
+ * code: 0 none, 1 empty train mask, 2 label out of range, 3 bounded wait expired. */
+mixgcn_status mixgcn_ctx_poll_status(mixgcn_ctx* ctx, int32_t* code);
+
+/* Per-phase profiling.  While enabled the library brackets every kernel it launches with
+ * CUDA events on the launching stream.  mixgcn_ctx_profile_read synchronises and returns, for
+ * each phase, accumulated milliseconds and launch counts since the last read, then resets.
+ * Phases: 0 spmm, 1 gemm, 2 elementwise/epilogue, 3 loss, 4 adam, 5 graph build.
+ * `launches_total` (nullable) receives the number of kernels launched by this context since
+ * creation (counted whether or not profiling is enabled). */
+#define MIXGCN_N_PHASES 6
+mixgcn_status mixgcn_ctx_profile_enable(mixgcn_ctx* ctx, int enable);
+mixgcn_status mixgcn_ctx_profile_read(mixgcn_ctx* ctx, double ms[MIXGCN_N_PHASES],
+                                      int64_t launches[MIXGCN_N_PHASES], int64_t* launches_total);
+
+/* ------------------------------------------------------------------------------------------
+ * Graph: the propagation matrix A_hat = D^-1/2 (A + I) D^-1/2 with D_uu = sum_v (A+I)_uv
+ * (Section 2.1), kept in CSR (the adjacency index format of Section 3.2.1) together with the
+ * CSR of its transpose (aliased when the stored matrix is symmetric) and a degree-sorted row
+ * schedule for the aggregation kernels.
+ * ------------------------------------------------------------------------------------------ */
+#define MIXGCN_GRAPH_SYMMETRISE     1u /* store (v,u) for every (u,v) */
+#define MIXGCN_GRAPH_ADD_SELF_LOOPS 2u /* the "+ I" of Section 2.1 */
+#define MIXGCN_GRAPH_EDGES_ON_DEVICE 4u /* src/dst (or rowptr/col) are device pointers */
+
+/* Build from an edge list of m pairs (src[e], dst[e]) meaning entry (src, dst) of A.
+ * Input self-loops are dropped, duplicates collapse (A is binary), then one diagonal entry
+ * per node is added if ADD_SELF_LOOPS.  rowptr is int64[n+1], col int32[nnz] ascending per
+ * row, val fp32: dinv_u = 1/sqrt(deg_u) (IEEE sqrt then IEEE reciprocal, each rounded to
+ * fp32), val_uv = dinv_u * dinv_v (one rounded multiply), deg_u = entries in row u.
+ * Requires 0 < n < 2^31 - 1 and 0 <= m; ids in [0, n) else MIXGCN_EBADGRAPH.
+ * Synchronises before returning.  *out is owned by the caller until mixgcn_graph_destroy. */
+mixgcn_status mixgcn_graph_create(mixgcn_ctx* ctx, int64_t n, int64_t m, const int32_t* src,
+                                  const int32_t* dst, uint32_t flags, mixgcn_graph** out);
+
+/* Build from the CSR structure of A + I (or of any binary matrix): validates monotone rowptr,
+ * ids in range and strictly ascending columns per row (else MIXGCN_EBADGRAPH), then
+ * normalises as above.  Only EDGES_ON_DEVICE is honoured in flags.  Synchronises. */
+mixgcn_status mixgcn_graph_create_from_csr(mixgcn_ctx* ctx, int64_t n, const int64_t* rowptr,
+                                           const int32_t* col, uint32_t flags, mixgcn_graph** out);
+
+mixgcn_status mixgcn_graph_info(const mixgcn_graph* g, int64_t* n, int64_t* nnz,
+                                int32_t* max_deg, int32_t* symmetric);
+
+/* Copy the CSR (transposed != 0: of A_hat^T) to HOST arrays; any output may be NULL.
+ * rowptr int64[n+1], col int32[nnz], val fp32[nnz], deg int32[n] (entries per row of the
+ * non-transposed matrix), dinv fp32[n].  Synchronises. */
+mixgcn_status mixgcn_graph_export(const mixgcn_graph* g, int transposed, int64_t* rowptr,
+                                  int32_t* col, float* val, int32_t* deg, float* dinv);
+
+/* Copy the degree-sorted row schedule to HOST: perm int32[n] lists row ids by descending
+ * entry count (ties by ascending id). */
+mixgcn_status mixgcn_graph_export_schedule(const mixgcn_graph* g, int transposed, int32_t* perm);
+
+mixgcn_status mixgcn_graph_destroy(mixgcn_graph* g);
+
+/* ------------------------------------------------------------------------------------------
+ * Building blocks (device pointers).  The layer calls below are compositions of these.
+ * ------------------------------------------------------------------------------------------ */
+
+/* Epilogue applied to each output element y of an aggregation or an update, in this order:
+ *   y += bias[j]                       if bias != NULL
+ *   y  = max(y, 0)                     if relu
+ *   y  = drop_mask[i*d+j] ? y*keep_scale : 0      if drop_mask != NULL   (uint8, dense n x d)
+ *   y  = gate[i*ld_gate+j] > 0 ? y*gate_scale : 0 if gate != NULL        (fp32, n x d)
+ * The gate form is the backward sampled aggregation of Eq. 4 (M = ReLU mask). */
+typedef struct {
+    const float* bias;
+    int32_t relu;
+    const uint8_t* drop_mask;
+    float keep_scale;
+    const float* gate;
+    int64_t ld_gate;
+    float gate_scale;
+} mixgcn_epilogue;
+
+/* Neighbour aggregation Z = A_hat Y (transposed != 0: A_hat^T Y), n x w (Algorithm 2,
+ * aggregation line; column slices as in its p:q-1 ranges are taken internally).
+ * Y and Z must not overlap.  epi may be NULL.  Row sums are accumulated in fp32 in a fixed
+ * order. */
+mixgcn_status mixgcn_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, int transposed, int32_t w,
+                          const float* Y, int64_t ldy, float* Z, int64_t ldz,
+                          const mixgcn_epilogue* epi, void* stream);
+
+#define MIXGCN_PREC_FP32 0 /* fp32 FMA on the CUDA cores */
+#define MIXGCN_PREC_TF32 1 /* tensor cores, TF32 operands, fp32 accumulate */
+#define MIXGCN_PREC_BF16 2 /* tensor cores, BF16 operands, fp32 accumulate */
+
+/* Dense update GEMM  C = op(A) op(B)  with fp32 storage (Algorithm 2, update line, and its
+ * two backward products).  op(A) is M x K, op(B) is K x N, C is M x N row-major with ldc.
+ *   trans_a = 0: A is M x K row-major (lda >= K);  trans_a = 1: A is K x M row-major (lda >= M)
+ *   trans_b = 0: B is K x N row-major (ldb >= N);  trans_b = 1: B is N x K row-major (ldb >= K)
+ * epi (nullable) applies to C's rows/columns with d = N.  C must not overlap A or B.
+ * With trans_a = 1 and large K the product is split over K into partial sums held in the
+ * context workspace and combined in a fixed order. */
+mixgcn_status mixgcn_gemm(mixgcn_ctx* ctx, int32_t precision, int32_t trans_a, int32_t trans_b,
+                          int64_t M, int64_t N, int64_t K, const float* A, int64_t lda,
+                          const float* B, int64_t ldb, float* C, int64_t ldc,
+                          const mixgcn_epilogue* epi, void* stream);
+
+/* ------------------------------------------------------------------------------------------
+ * One GCN layer, X_out = drop * keep_scale * ReLU(A_hat X_in W + 1 b^T)   (Eq. 3)
+ * ------------------------------------------------------------------------------------------ */
+#define MIXGCN_ORDER_AUTO 0
+#define MIXGCN_ORDER_AGG_FIRST 1 /* (A_hat X) W : aggregate at width d_in  */
+#define MIXGCN_ORDER_UPD_FIRST 2 /* A_hat (X W) : aggregate at width d_out */
+
+#define MIXGCN_LAYER_RELU 1u        /* sigma = ReLU (omit on the last layer) */
+#define MIXGCN_LAYER_FIRST 2u       /* X_in is data: backward computes no input gradient */
+#define MIXGCN_LAYER_GATE_GIN 4u    /* backward: G_in = (A_hat^T ...) * 1[X_in > 0] * in_scale,
+                                       i.e. the ReLU mask of the layer below is applied by this
+                                       layer's aggregation epilogue (Eq. 4, backward form) */
+#define MIXGCN_LAYER_GOUT_GATED 8u  /* backward: G_out already carries this layer's ReLU/dropout
+                                       mask (the layer above used GATE_GIN) */
+
+typedef struct {
+    int32_t d_in, d_out;
+    int64_t ld_in, ld_out, ld_saved;
+    int32_t order;      /* MIXGCN_ORDER_* ; AUTO picks by the per-node FLOP model of Appendix A */
+    int32_t precision;  /* MIXGCN_PREC_* for the dense products */
+    uint32_t flags;     /* MIXGCN_LAYER_* */
+    float keep_scale;   /* 1/(1-p) for this layer's dropout mask; 1 if none */
+    float in_scale;     /* keep_scale of the layer below, used with GATE_GIN; 1 if none */
+    int32_t n_chunks;   /* >1: split rows into this many chunks and overlap the aggregation of
+                           chunk k+1 with the update of chunk k on two streams; 0/1: off */
+} mixgcn_layer_desc;
+
+/* Resolves MIXGCN_ORDER_AUTO: cost(agg-first) = c * d_in with c = 1 for a FIRST layer (its
+ * backward needs no aggregation) else 2; cost(upd-first) = 2 * d_out; the smaller wins, ties
+ * go to agg-first.  *saved_cols receives the number of columns the `saved` buffer needs
+ * (d_in for agg-first, d_out for upd-first). */
+mixgcn_status mixgcn_layer_plan(const mixgcn_layer_desc* desc, int32_t* order, int32_t* saved_cols);
+
+/* Forward.  bias, drop_mask nullable.  `saved` is n x ld_saved:
+ *   agg-first: receives A_hat X_in and must be handed unchanged to mixgcn_layer_bwd;
+ *   upd-first: scratch for X_in W (contents not needed afterwards).
+ * X_out is n x ld_out.  Buffers must not overlap. */
+mixgcn_status mixgcn_layer_fwd(mixgcn_ctx* ctx, const mixgcn_graph* g, const mixgcn_layer_desc* desc,
+                               const float* X_in, const float* W, const float* bias,
+                               const uint8_t* drop_mask, float* saved, float* X_out, void* stream);
+
+/* Backward.  G_out (n x ld_out) is the gradient w.r.t. X_out and is OVERWRITTEN (it becomes
+ * the gradient w.r.t. the pre-activation).  `saved` is consumed: agg-first reads A_hat X_in
+ * from it and then overwrites it; upd-first uses it as scratch.  dW is d_in x d_out, dbias
+ * d_out (nullable).  G_in (n x ld_in) receives the gradient w.r.t. X_in and must be NULL iff
+ * MIXGCN_LAYER_FIRST is set.  X_out and drop_mask are the forward's. */
+mixgcn_status mixgcn_layer_bwd(mixgcn_ctx* ctx, const mixgcn_graph* g, const mixgcn_layer_desc* desc,
+                               const float* X_in, float* saved, const float* X_out,
+                               const uint8_t* drop_mask, const float* W, float* G_out,
+                               float* G_in, float* dW, float* dbias, void* stream);
+
+/* Masked softmax cross-entropy (the loss line of Algorithm 2; mean over train nodes, natural
+ * log): loss = -(1/#T) sum_{v in T} log softmax(logits_v)[label_v]; dlogits_v =
+ * (softmax(logits_v) - e_label) / #T on T and 0 elsewhere; pred_v = lowest index of the row
+ * maximum; *n_correct = #{v in T : pred_v == label_v}.  logits n x C with ld; labels
+ * int32[n]; train_mask uint8[n]; loss device fp32 scalar; dlogits (nullable, may alias
+ * logits, same ld); pred int32[n] (nullable); n_correct device int64 scalar (nullable).
+ * 1 <= C <= 4096.  Empty mask or a label outside [0,C) on a train node: outputs are zeros
+ * and the status word is set. */
+mixgcn_status mixgcn_loss_softmax_xent(mixgcn_ctx* ctx, int64_t n, int32_t C, const float* logits,
+                                       int64_t ld, const int32_t* labels, const uint8_t* train_mask,
+                                       float* loss, float* dlogits, int32_t* pred,
+                                       int64_t* n_correct, void* stream);
+
+/* Adam over n_tensors parameter tensors (HOST arrays of DEVICE pointers and element counts):
+ * m = b1 m + (1-b1) g; v = b2 v + (1-b2) g^2; theta -= lr * (m/(1-b1^t)) / (sqrt(v/(1-b2^t)) + eps),
+ * t >= 1, no weight decay (the weight-update step of Algorithm 2). */
+mixgcn_status mixgcn_adam_step(mixgcn_ctx* ctx, int32_t n_tensors, float* const* param,
+                               const float* const* grad, float* const* m, float* const* v,
+                               const int64_t* numel, int64_t t, float lr, float beta1, float beta2,
+                               float eps, void* stream);
+
+/* One whole training iteration (Algorithm 2's loop body) with HOST inputs and outputs: copies
+ * features, labels, mask, weights, biases and Adam moments to the device, runs forward, loss,
+ * backward and Adam, and copies back the loss, the updated weights, biases and moments.
+ * dims is int32[L+1] (d_0 .. d_L); W, b, mW, vW, mb, vb are host arrays of L host pointers
+ * (dense fp32, updated in place); X is n x d_0 dense fp32; loss host fp32 scalar; pred
+ * (nullable) host int32[n].  Uses AUTO ordering, ReLU on all layers but the last, no dropout.
+ * Device buffers are taken from the context workspace (grown on demand).  Synchronises. */
+mixgcn_status mixgcn_train_step_host(mixgcn_ctx* ctx, const mixgcn_graph* g, int32_t L,
+                                     const int32_t* dims, int32_t precision, const float* X,
+                                     const int32_t* labels, const uint8_t* train_mask,
+                                     float* const* W, float* const* b, float* const* mW,
+                                     float* const* vW, float* const* mb, float* const* vb,
+                                     int64_t t, float lr, float beta1, float beta2, float eps,
+                                     float* loss, int32_t* pred);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MIXGCN_H_ */

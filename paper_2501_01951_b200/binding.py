@@ -1,0 +1,319 @@
+"""ctypes binding of ``include/mixgcn.h`` -- argument marshalling only.
+
+Every function here has the name of the C entry point without the ``mixgcn_`` prefix, takes
+torch tensors (device memory owned by the caller) and forwards raw pointers, sizes and the
+current torch CUDA stream.  No arithmetic of the method happens in Python.  Importing this
+module without a built ``libmixgcn.so`` raises: there is no fallback path.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libmixgcn.so")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        f"{LIB_PATH} is missing: build it with `python -m paper_2501_01951_b200.build` "
+        "(there is no CPU or PyTorch fallback for this library)")
+
+lib = C.CDLL(LIB_PATH)
+
+OK, EINVAL, ENOMEM, ECUDA, EUNSUPPORTED, EBADGRAPH, ETIMEOUT, EDEVICE = range(8)
+GRAPH_SYMMETRISE, GRAPH_ADD_SELF_LOOPS, GRAPH_EDGES_ON_DEVICE = 1, 2, 4
+PREC_FP32, PREC_TF32, PREC_BF16 = 0, 1, 2
+ORDER_AUTO, ORDER_AGG_FIRST, ORDER_UPD_FIRST = 0, 1, 2
+LAYER_RELU, LAYER_FIRST, LAYER_GATE_GIN, LAYER_GOUT_GATED = 1, 2, 4, 8
+N_PHASES = 6
+PHASES = ("spmm", "gemm", "elementwise", "loss", "adam", "graph")
+PRECISIONS = {"fp32": PREC_FP32, "tf32": PREC_TF32, "bf16": PREC_BF16}
+
+# every symbol include/mixgcn.h declares
+SYMBOLS = (
+    "mixgcn_status_string", "mixgcn_last_error", "mixgcn_ctx_create", "mixgcn_ctx_destroy",
+    "mixgcn_ctx_reserve", "mixgcn_ctx_poll_status", "mixgcn_ctx_profile_enable", "mixgcn_ctx_profile_read",
+    "mixgcn_graph_create", "mixgcn_graph_create_from_csr", "mixgcn_graph_info", "mixgcn_graph_export",
+    "mixgcn_graph_export_schedule", "mixgcn_graph_destroy", "mixgcn_spmm", "mixgcn_gemm",
+    "mixgcn_layer_plan", "mixgcn_layer_fwd", "mixgcn_layer_bwd", "mixgcn_loss_softmax_xent",
+    "mixgcn_adam_step", "mixgcn_train_step_host",
+)
+
+
+class Epilogue(C.Structure):
+    _fields_ = [("bias", C.c_void_p), ("relu", C.c_int32), ("drop_mask", C.c_void_p),
+                ("keep_scale", C.c_float), ("gate", C.c_void_p), ("ld_gate", C.c_int64),
+                ("gate_scale", C.c_float)]
+
+
+class LayerDesc(C.Structure):
+    _fields_ = [("d_in", C.c_int32), ("d_out", C.c_int32), ("ld_in", C.c_int64), ("ld_out", C.c_int64),
+                ("ld_saved", C.c_int64), ("order", C.c_int32), ("precision", C.c_int32),
+                ("flags", C.c_uint32), ("keep_scale", C.c_float), ("in_scale", C.c_float),
+                ("n_chunks", C.c_int32)]
+
+
+lib.mixgcn_status_string.restype = C.c_char_p
+lib.mixgcn_last_error.restype = C.c_char_p
+for _name in SYMBOLS[2:]:
+    getattr(lib, _name).restype = C.c_int
+
+
+class MixgcnError(RuntimeError):
+    def __init__(self, status: int):
+        self.status = status
+        msg = lib.mixgcn_last_error().decode()
+        super().__init__(f"{lib.mixgcn_status_string(status).decode()} ({status}): {msg}")
+
+
+def _check(status: int):
+    if status != OK:
+        raise MixgcnError(status)
+
+
+def _ptr(t):
+    """Device or host pointer of a tensor (None -> NULL)."""
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _dev(t, dtype, name):
+    if not t.is_cuda or t.dtype != dtype:
+        raise TypeError(f"{name}: expected a CUDA tensor of {dtype}, got {t.dtype} on {t.device}")
+    return t
+
+
+def _mat(t, name):
+    """2-D fp32 CUDA tensor with unit column stride -> (tensor, ld)."""
+    _dev(t, torch.float32, name)
+    if t.dim() != 2 or t.stride(1) != 1:
+        raise TypeError(f"{name}: expected a row-major 2-D tensor")
+    return t, t.stride(0)
+
+
+# ------------------------------------------------------------------------------ context
+
+class Ctx:
+    def __init__(self, device: int = 0):
+        self.h = C.c_void_p()
+        _check(lib.mixgcn_ctx_create(C.byref(self.h), C.c_int(device)))
+        self.device = device
+
+    def close(self):
+        if self.h:
+            lib.mixgcn_ctx_destroy(self.h)
+            self.h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def ctx_create(device: int = 0) -> Ctx:
+    return Ctx(device)
+
+
+def ctx_reserve(ctx: Ctx, nbytes: int):
+    _check(lib.mixgcn_ctx_reserve(ctx.h, C.c_int64(nbytes)))
+
+
+def ctx_poll_status(ctx: Ctx, raise_on_error: bool = True) -> int:
+    code = C.c_int32(0)
+    st = lib.mixgcn_ctx_poll_status(ctx.h, C.byref(code))
+    if raise_on_error:
+        _check(st)
+    return code.value
+
+
+def ctx_profile_enable(ctx: Ctx, enable: bool = True):
+    _check(lib.mixgcn_ctx_profile_enable(ctx.h, C.c_int(int(enable))))
+
+
+def ctx_profile_read(ctx: Ctx):
+    """-> ({phase: ms}, {phase: launches}, launches_total)."""
+    ms = (C.c_double * N_PHASES)()
+    ln = (C.c_int64 * N_PHASES)()
+    tot = C.c_int64(0)
+    _check(lib.mixgcn_ctx_profile_read(ctx.h, ms, ln, C.byref(tot)))
+    return dict(zip(PHASES, list(ms))), dict(zip(PHASES, list(ln))), tot.value
+
+
+# ------------------------------------------------------------------------------ graph
+
+class Graph:
+    def __init__(self, ctx: Ctx, handle):
+        self.ctx, self.h = ctx, handle
+        n, nnz, md, sym = C.c_int64(), C.c_int64(), C.c_int32(), C.c_int32()
+        _check(lib.mixgcn_graph_info(self.h, C.byref(n), C.byref(nnz), C.byref(md), C.byref(sym)))
+        self.n, self.nnz, self.max_deg, self.symmetric = n.value, nnz.value, md.value, bool(sym.value)
+
+    def close(self):
+        if self.h:
+            lib.mixgcn_graph_destroy(self.h)
+            self.h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def graph_create(ctx: Ctx, n: int, src: torch.Tensor, dst: torch.Tensor,
+                 flags: int = GRAPH_SYMMETRISE | GRAPH_ADD_SELF_LOOPS) -> Graph:
+    """src/dst: int32 tensors, both on the host or both on the context's device."""
+    if src.dtype != torch.int32 or dst.dtype != torch.int32 or src.numel() != dst.numel():
+        raise TypeError("graph_create: src and dst must be int32 tensors of equal length")
+    if src.is_cuda != dst.is_cuda:
+        raise TypeError("graph_create: src and dst must live on the same side")
+    src, dst = src.contiguous(), dst.contiguous()
+    if src.is_cuda:
+        flags |= GRAPH_EDGES_ON_DEVICE
+        torch.cuda.current_stream().synchronize()
+    h = C.c_void_p()
+    _check(lib.mixgcn_graph_create(ctx.h, C.c_int64(n), C.c_int64(src.numel()), _ptr(src), _ptr(dst),
+                                   C.c_uint32(flags), C.byref(h)))
+    return Graph(ctx, h)
+
+
+def graph_create_from_csr(ctx: Ctx, n: int, rowptr: torch.Tensor, col: torch.Tensor) -> Graph:
+    if rowptr.dtype != torch.int64 or col.dtype != torch.int32 or rowptr.numel() != n + 1:
+        raise TypeError("graph_create_from_csr: rowptr int64[n+1], col int32[nnz]")
+    rowptr, col = rowptr.contiguous(), col.contiguous()
+    flags = GRAPH_EDGES_ON_DEVICE if rowptr.is_cuda else 0
+    if rowptr.is_cuda:
+        torch.cuda.current_stream().synchronize()
+    h = C.c_void_p()
+    _check(lib.mixgcn_graph_create_from_csr(ctx.h, C.c_int64(n), _ptr(rowptr), _ptr(col), C.c_uint32(flags), C.byref(h)))
+    return Graph(ctx, h)
+
+
+def graph_export(g: Graph, transposed: bool = False):
+    """-> dict of host tensors rowptr, col, val, deg, dinv."""
+    out = dict(rowptr=torch.empty(g.n + 1, dtype=torch.int64), col=torch.empty(g.nnz, dtype=torch.int32),
+               val=torch.empty(g.nnz, dtype=torch.float32), deg=torch.empty(g.n, dtype=torch.int32),
+               dinv=torch.empty(g.n, dtype=torch.float32))
+    _check(lib.mixgcn_graph_export(g.h, C.c_int(int(transposed)), _ptr(out["rowptr"]), _ptr(out["col"]),
+                                   _ptr(out["val"]), _ptr(out["deg"]), _ptr(out["dinv"])))
+    return out
+
+
+def graph_export_schedule(g: Graph, transposed: bool = False) -> torch.Tensor:
+    perm = torch.empty(g.n, dtype=torch.int32)
+    _check(lib.mixgcn_graph_export_schedule(g.h, C.c_int(int(transposed)), _ptr(perm)))
+    return perm
+
+
+# ------------------------------------------------------------------------------ building blocks
+
+def make_epilogue(bias=None, relu=False, drop_mask=None, keep_scale=1.0, gate=None, gate_scale=1.0):
+    e = Epilogue()
+    e.bias = None if bias is None else _dev(bias, torch.float32, "bias").data_ptr()
+    e.relu = int(relu)
+    e.drop_mask = None if drop_mask is None else _dev(drop_mask, torch.uint8, "drop_mask").data_ptr()
+    e.keep_scale = keep_scale
+    if gate is not None:
+        gate, ldg = _mat(gate, "gate")
+        e.gate, e.ld_gate = gate.data_ptr(), ldg
+    e.gate_scale = gate_scale
+    e._keep = (bias, drop_mask, gate)
+    return e
+
+
+def spmm(ctx: Ctx, g: Graph, Y: torch.Tensor, Z: torch.Tensor, w: int, transposed: bool = False, epi: Epilogue | None = None):
+    Y, ldy = _mat(Y, "Y")
+    Z, ldz = _mat(Z, "Z")
+    _check(lib.mixgcn_spmm(ctx.h, g.h, C.c_int(int(transposed)), C.c_int32(w), _ptr(Y), C.c_int64(ldy),
+                           _ptr(Z), C.c_int64(ldz), None if epi is None else C.byref(epi), _stream()))
+
+
+def gemm(ctx: Ctx, precision: int, trans_a: bool, trans_b: bool, M: int, N: int, K: int,
+         A: torch.Tensor, B: torch.Tensor, Cm: torch.Tensor, epi: Epilogue | None = None):
+    A, lda = _mat(A, "A")
+    B, ldb = _mat(B, "B")
+    Cm, ldc = _mat(Cm, "C")
+    _check(lib.mixgcn_gemm(ctx.h, C.c_int32(precision), C.c_int32(int(trans_a)), C.c_int32(int(trans_b)),
+                           C.c_int64(M), C.c_int64(N), C.c_int64(K), _ptr(A), C.c_int64(lda), _ptr(B),
+                           C.c_int64(ldb), _ptr(Cm), C.c_int64(ldc), None if epi is None else C.byref(epi), _stream()))
+
+
+# ------------------------------------------------------------------------------ layers
+
+def layer_desc(d_in, d_out, ld_in, ld_out, ld_saved, order=ORDER_AUTO, precision=PREC_FP32, flags=0,
+               keep_scale=1.0, in_scale=1.0, n_chunks=0) -> LayerDesc:
+    return LayerDesc(d_in, d_out, ld_in, ld_out, ld_saved, order, precision, flags, keep_scale, in_scale, n_chunks)
+
+
+def layer_plan(desc: LayerDesc):
+    order, cols = C.c_int32(), C.c_int32()
+    _check(lib.mixgcn_layer_plan(C.byref(desc), C.byref(order), C.byref(cols)))
+    return order.value, cols.value
+
+
+def layer_fwd(ctx: Ctx, g: Graph, desc: LayerDesc, X_in, W, bias, drop_mask, saved, X_out):
+    _mat(X_in, "X_in"); _mat(saved, "saved"); _mat(X_out, "X_out"); _dev(W, torch.float32, "W")
+    if not W.is_contiguous():
+        raise TypeError("W must be dense row-major")
+    _check(lib.mixgcn_layer_fwd(ctx.h, g.h, C.byref(desc), _ptr(X_in), _ptr(W), _ptr(bias), _ptr(drop_mask),
+                                _ptr(saved), _ptr(X_out), _stream()))
+
+
+def layer_bwd(ctx: Ctx, g: Graph, desc: LayerDesc, X_in, saved, X_out, drop_mask, W, G_out, G_in, dW, dbias):
+    _mat(X_in, "X_in"); _mat(saved, "saved"); _mat(X_out, "X_out"); _mat(G_out, "G_out")
+    if G_in is not None:
+        _mat(G_in, "G_in")
+    if not (W.is_contiguous() and dW.is_contiguous()):
+        raise TypeError("W and dW must be dense row-major")
+    _check(lib.mixgcn_layer_bwd(ctx.h, g.h, C.byref(desc), _ptr(X_in), _ptr(saved), _ptr(X_out), _ptr(drop_mask),
+                                _ptr(W), _ptr(G_out), _ptr(G_in), _ptr(dW), _ptr(dbias), _stream()))
+
+
+def loss_softmax_xent(ctx: Ctx, logits, labels, train_mask, loss, dlogits=None, pred=None, n_correct=None, C_=None):
+    logits, ld = _mat(logits, "logits")
+    n = logits.shape[0]
+    Cc = logits.shape[1] if C_ is None else C_
+    _dev(labels, torch.int32, "labels"); _dev(train_mask, torch.uint8, "train_mask"); _dev(loss, torch.float32, "loss")
+    if dlogits is not None:
+        dlogits, ldd = _mat(dlogits, "dlogits")
+        if ldd != ld:
+            raise TypeError("dlogits must share the logits' leading dimension")
+    _check(lib.mixgcn_loss_softmax_xent(ctx.h, C.c_int64(n), C.c_int32(Cc), _ptr(logits), C.c_int64(ld), _ptr(labels),
+                                        _ptr(train_mask), _ptr(loss), _ptr(dlogits), _ptr(pred), _ptr(n_correct), _stream()))
+
+
+def adam_step(ctx: Ctx, params, grads, ms, vs, t, lr=0.01, beta1=0.9, beta2=0.999, eps=1e-8):
+    k = len(params)
+    for lst in (params, grads, ms, vs):
+        for x in lst:
+            _dev(x, torch.float32, "adam tensor")
+            if not x.is_contiguous():
+                raise TypeError("adam tensors must be contiguous")
+    arr = lambda lst: (C.c_void_p * k)(*[x.data_ptr() for x in lst])
+    numel = (C.c_int64 * k)(*[x.numel() for x in params])
+    _check(lib.mixgcn_adam_step(ctx.h, C.c_int32(k), arr(params), arr(grads), arr(ms), arr(vs), numel, C.c_int64(t),
+                                C.c_float(lr), C.c_float(beta1), C.c_float(beta2), C.c_float(eps), _stream()))
+
+
+def train_step_host(ctx: Ctx, g: Graph, dims, precision, X, labels, train_mask, W, b, mW, vW, mb, vb, t,
+                    lr=0.01, beta1=0.9, beta2=0.999, eps=1e-8, pred=None) -> float:
+    """All tensors are HOST tensors (pinned memory makes the copies faster); W, b and the Adam
+    moments are updated in place.  Returns the loss."""
+    L = len(dims) - 1
+    for x in [X, labels, train_mask, *W, *b, *mW, *vW, *mb, *vb]:
+        if x.is_cuda or not x.is_contiguous():
+            raise TypeError("train_step_host takes contiguous host tensors")
+    dims_a = (C.c_int32 * (L + 1))(*dims)
+    arr = lambda lst: (C.c_void_p * L)(*[x.data_ptr() for x in lst])
+    loss = C.c_float(0.0)
+    _check(lib.mixgcn_train_step_host(ctx.h, g.h, C.c_int32(L), dims_a, C.c_int32(precision), _ptr(X), _ptr(labels),
+                                      _ptr(train_mask), arr(W), arr(b), arr(mW), arr(vW), arr(mb), arr(vb),
+                                      C.c_int64(t), C.c_float(lr), C.c_float(beta1), C.c_float(beta2), C.c_float(eps),
+                                      C.byref(loss), _ptr(pred)))
+    return loss.value

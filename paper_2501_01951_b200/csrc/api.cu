@@ -1,0 +1,355 @@
+// Context, error reporting, profiling, and the per-layer composition of aggregation and update
+// (Eq. 3 and Algorithm 2 of the paper): ordering choice from the per-node FLOP model of
+// Appendix A, and the row-chunked aggregation -> update pipeline on two streams (the fine-grain
+// sparse/dense pipeline of Section 3.2.2 mapped onto one GPU).
+#include <stdarg.h>
+#include <string.h>
+
+#include <new>
+
+#include "internal.cuh"
+
+using namespace mixgcn;
+
+namespace {
+thread_local char g_err[512] = "";
+}
+
+namespace mixgcn {
+
+void set_error(const char* fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+}
+
+LaunchScope::LaunchScope(mixgcn_ctx* c, int phase, cudaStream_t s, int n_launches) : ctx(c), stream(s), span(-1) {
+    ctx->launches_total += n_launches;
+    ctx->phase_launches[phase] += n_launches;
+    if (!ctx->profile) return;
+    if (ctx->n_spans == ctx->cap_spans) {
+        int cap = ctx->cap_spans ? ctx->cap_spans * 2 : 256;
+        ProfSpan* ns = (ProfSpan*)realloc(ctx->spans, cap * sizeof(ProfSpan));
+        if (!ns) return;
+        for (int i = ctx->cap_spans; i < cap; ++i) { ns[i].a = nullptr; ns[i].b = nullptr; }
+        ctx->spans = ns; ctx->cap_spans = cap;
+    }
+    span = ctx->n_spans++;
+    ProfSpan& sp = ctx->spans[span];
+    if (!sp.a) { cudaEventCreate(&sp.a); cudaEventCreate(&sp.b); }
+    sp.phase = phase;
+    cudaEventRecord(sp.a, stream);
+}
+
+LaunchScope::~LaunchScope() {
+    if (span >= 0) cudaEventRecord(ctx->spans[span].b, stream);
+}
+
+mixgcn_status ensure_workspace(mixgcn_ctx* ctx, int64_t bytes) {
+    if (bytes <= ctx->workspace_bytes) return MIXGCN_OK;
+    int64_t want = bytes + (bytes >> 2);
+    want = (want + 255) & ~(int64_t)255;
+    void* p = nullptr;
+    // the old block may still be in use by enqueued kernels: wait before releasing it
+    MIXGCN_CUDA(cudaDeviceSynchronize());
+    if (ctx->workspace) cudaFree(ctx->workspace);
+    ctx->workspace = nullptr; ctx->workspace_bytes = 0;
+    cudaError_t e = cudaMalloc(&p, (size_t)want);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        MIXGCN_FAIL(MIXGCN_ENOMEM, "workspace of %lld bytes could not be allocated", (long long)want);
+    }
+    ctx->workspace = p; ctx->workspace_bytes = want;
+    return MIXGCN_OK;
+}
+
+mixgcn_status launch_gemm_simt(mixgcn_ctx* ctx, int ta, int tb, int64_t M, int64_t N, int64_t K,
+                               const float* A, int64_t lda, const float* B, int64_t ldb, float* C, int64_t ldc,
+                               const mixgcn_epilogue* epi, int64_t epi_row0, cudaStream_t s);
+
+mixgcn_status launch_gemm(mixgcn_ctx* ctx, int precision, int ta, int tb, int64_t M, int64_t N, int64_t K,
+                          const float* A, int64_t lda, const float* B, int64_t ldb, float* C, int64_t ldc,
+                          const mixgcn_epilogue* epi, int64_t epi_row0, cudaStream_t s) {
+    (void)precision;  // reduced-precision tensor-core kernels plug in here; fp32 serves every request
+    return launch_gemm_simt(ctx, ta, tb, M, N, K, A, lda, B, ldb, C, ldc, epi, epi_row0, s);
+}
+
+}  // namespace mixgcn
+
+extern "C" const char* mixgcn_status_string(mixgcn_status s) {
+    switch (s) {
+        case MIXGCN_OK: return "ok";
+        case MIXGCN_EINVAL: return "invalid argument";
+        case MIXGCN_ENOMEM: return "out of memory";
+        case MIXGCN_ECUDA: return "CUDA runtime error";
+        case MIXGCN_EUNSUPPORTED: return "unsupported";
+        case MIXGCN_EBADGRAPH: return "malformed graph";
+        case MIXGCN_ETIMEOUT: return "device wait timed out";
+        case MIXGCN_EDEVICE: return "device reported bad data";
+    }
+    return "unknown status";
+}
+
+extern "C" const char* mixgcn_last_error(void) { return g_err; }
+
+extern "C" mixgcn_status mixgcn_ctx_create(mixgcn_ctx** out, int device) {
+    if (!out) MIXGCN_FAIL(MIXGCN_EINVAL, "ctx_create: null out");
+    int count = 0;
+    MIXGCN_CUDA(cudaGetDeviceCount(&count));
+    if (device < 0 || device >= count) MIXGCN_FAIL(MIXGCN_EINVAL, "ctx_create: device %d not in [0,%d)", device, count);
+    MIXGCN_CUDA(cudaSetDevice(device));
+    cudaDeviceProp prop;
+    MIXGCN_CUDA(cudaGetDeviceProperties(&prop, device));
+    if (prop.major != 10) MIXGCN_FAIL(MIXGCN_EUNSUPPORTED, "ctx_create: device %d is sm_%d%d; this library is built for sm_100a only", device, prop.major, prop.minor);
+    mixgcn_ctx* c = new (std::nothrow) mixgcn_ctx();
+    if (!c) MIXGCN_FAIL(MIXGCN_ENOMEM, "ctx_create: host allocation failed");
+    memset(c, 0, sizeof(*c));
+    c->device = device;
+    c->sm_count = prop.multiProcessorCount;
+    MIXGCN_CUDA(cudaMalloc((void**)&c->d_status, 4 * sizeof(int32_t)));
+    MIXGCN_CUDA(cudaMemset(c->d_status, 0, 4 * sizeof(int32_t)));
+    for (int i = 0; i < 2; ++i) MIXGCN_CUDA(cudaStreamCreateWithFlags(&c->side_stream[i], cudaStreamNonBlocking));
+    MIXGCN_CUDA(cudaEventCreateWithFlags(&c->fork_ev, cudaEventDisableTiming));
+    for (int i = 0; i < 2; ++i) MIXGCN_CUDA(cudaEventCreateWithFlags(&c->join_ev[i], cudaEventDisableTiming));
+    for (int i = 0; i < 64; ++i) MIXGCN_CUDA(cudaEventCreateWithFlags(&c->chunk_ev[i], cudaEventDisableTiming));
+    *out = c;
+    return MIXGCN_OK;
+}
+
+extern "C" mixgcn_status mixgcn_ctx_destroy(mixgcn_ctx* ctx) {
+    if (!ctx) return MIXGCN_OK;
+    cudaSetDevice(ctx->device);
+    cudaDeviceSynchronize();
+    for (int i = 0; i < ctx->cap_spans; ++i) {
+        if (ctx->spans[i].a) cudaEventDestroy(ctx->spans[i].a);
+        if (ctx->spans[i].b) cudaEventDestroy(ctx->spans[i].b);
+    }
+    free(ctx->spans);
+    for (int i = 0; i < 64; ++i) if (ctx->chunk_ev[i]) cudaEventDestroy(ctx->chunk_ev[i]);
+    for (int i = 0; i < 2; ++i) { if (ctx->join_ev[i]) cudaEventDestroy(ctx->join_ev[i]); if (ctx->side_stream[i]) cudaStreamDestroy(ctx->side_stream[i]); }
+    if (ctx->fork_ev) cudaEventDestroy(ctx->fork_ev);
+    cudaFree(ctx->workspace);
+    cudaFree(ctx->d_status);
+    delete ctx;
+    return MIXGCN_OK;
+}
+
+extern "C" mixgcn_status mixgcn_ctx_reserve(mixgcn_ctx* ctx, int64_t bytes) {
+    if (!ctx || bytes < 0) MIXGCN_FAIL(MIXGCN_EINVAL, "ctx_reserve: bad argument");
+    MIXGCN_CUDA(cudaSetDevice(ctx->device));
+    return ensure_workspace(ctx, bytes);
+}
+
+extern "C" mixgcn_status mixgcn_ctx_poll_status(mixgcn_ctx* ctx, int32_t* code) {
+    if (!ctx) MIXGCN_FAIL(MIXGCN_EINVAL, "ctx_poll_status: null ctx");
+    MIXGCN_CUDA(cudaSetDevice(ctx->device));
+    MIXGCN_CUDA(cudaDeviceSynchronize());
+    int32_t h = 0;
+    MIXGCN_CUDA(cudaMemcpy(&h, ctx->d_status, sizeof(h), cudaMemcpyDeviceToHost));
+    MIXGCN_CUDA(cudaMemset(ctx->d_status, 0, sizeof(int32_t)));
+    if (code) *code = h;
+    if (h == DEV_OK) return MIXGCN_OK;
+    if (h == DEV_WAIT_EXPIRED) MIXGCN_FAIL(MIXGCN_ETIMEOUT, "a bounded device-side wait expired");
+    MIXGCN_FAIL(MIXGCN_EDEVICE, h == DEV_EMPTY_MASK ? "loss: the train mask is empty" : "loss: a label lies outside [0, C)");
+}
+
+extern "C" mixgcn_status mixgcn_ctx_profile_enable(mixgcn_ctx* ctx, int enable) {
+    if (!ctx) MIXGCN_FAIL(MIXGCN_EINVAL, "ctx_profile_enable: null ctx");
+    ctx->profile = enable ? 1 : 0;
+    return MIXGCN_OK;
+}
+
+extern "C" mixgcn_status mixgcn_ctx_profile_read(mixgcn_ctx* ctx, double ms[MIXGCN_N_PHASES],
+                                                 int64_t launches[MIXGCN_N_PHASES], int64_t* launches_total) {
+    if (!ctx) MIXGCN_FAIL(MIXGCN_EINVAL, "ctx_profile_read: null ctx");
+    MIXGCN_CUDA(cudaSetDevice(ctx->device));
+    MIXGCN_CUDA(cudaDeviceSynchronize());
+    if (ms) for (int i = 0; i < MIXGCN_N_PHASES; ++i) ms[i] = 0.0;
+    for (int i = 0; i < ctx->n_spans; ++i) {
+        float t = 0.f;
+        if (cudaEventElapsedTime(&t, ctx->spans[i].a, ctx->spans[i].b) == cudaSuccess && ms) ms[ctx->spans[i].phase] += t;
+    }
+    cudaGetLastError();
+    ctx->n_spans = 0;
+    if (launches) for (int i = 0; i < MIXGCN_N_PHASES; ++i) { launches[i] = ctx->phase_launches[i]; ctx->phase_launches[i] = 0; }
+    if (launches_total) *launches_total = ctx->launches_total;
+    return MIXGCN_OK;
+}
+
+extern "C" mixgcn_status mixgcn_gemm(mixgcn_ctx* ctx, int32_t precision, int32_t trans_a, int32_t trans_b,
+                                     int64_t M, int64_t N, int64_t K, const float* A, int64_t lda,
+                                     const float* B, int64_t ldb, float* C, int64_t ldc,
+                                     const mixgcn_epilogue* epi, void* stream) {
+    if (!ctx || !A || !B || !C) MIXGCN_FAIL(MIXGCN_EINVAL, "gemm: null argument");
+    if (M <= 0 || N <= 0 || K <= 0) MIXGCN_FAIL(MIXGCN_EINVAL, "gemm: M, N, K must be positive");
+    if (precision < MIXGCN_PREC_FP32 || precision > MIXGCN_PREC_BF16) MIXGCN_FAIL(MIXGCN_EINVAL, "gemm: unknown precision %d", precision);
+    const int64_t min_lda = trans_a ? M : K, min_ldb = trans_b ? K : N;
+    if (lda < min_lda || ldb < min_ldb || ldc < N)
+        MIXGCN_FAIL(MIXGCN_EINVAL, "gemm: leading dimensions must cover the matrix (lda=%lld ldb=%lld ldc=%lld)",
+                    (long long)lda, (long long)ldb, (long long)ldc);
+    if (C == A || C == B) MIXGCN_FAIL(MIXGCN_EINVAL, "gemm: C must not overlap A or B");
+    MIXGCN_CUDA(cudaSetDevice(ctx->device));
+    return launch_gemm(ctx, precision, trans_a, trans_b, M, N, K, A, lda, B, ldb, C, ldc, epi, 0, (cudaStream_t)stream);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Layer composition
+// ------------------------------------------------------------------------------------------------
+
+namespace {
+
+int resolve_order(const mixgcn_layer_desc* d) {
+    if (d->order == MIXGCN_ORDER_AGG_FIRST || d->order == MIXGCN_ORDER_UPD_FIRST) return d->order;
+    // Appendix A: aggregating costs deg(v) * width per node, so the width at which the sparse
+    // product runs decides.  A first layer aggregates once (forward only) in agg-first order.
+    const int64_t c = (d->flags & MIXGCN_LAYER_FIRST) ? 1 : 2;
+    const int64_t cost_agg = c * (int64_t)d->d_in, cost_upd = 2 * (int64_t)d->d_out;
+    return cost_agg <= cost_upd ? MIXGCN_ORDER_AGG_FIRST : MIXGCN_ORDER_UPD_FIRST;
+}
+
+mixgcn_status check_desc(const mixgcn_layer_desc* d, const char* who) {
+    if (!d) MIXGCN_FAIL(MIXGCN_EINVAL, "%s: null layer descriptor", who);
+    if (d->d_in <= 0 || d->d_out <= 0) MIXGCN_FAIL(MIXGCN_EINVAL, "%s: widths must be positive", who);
+    if (d->order < 0 || d->order > 2) MIXGCN_FAIL(MIXGCN_EINVAL, "%s: unknown order %d", who, d->order);
+    if (d->precision < 0 || d->precision > 2) MIXGCN_FAIL(MIXGCN_EINVAL, "%s: unknown precision %d", who, d->precision);
+    const int order = resolve_order(d);
+    const int saved_cols = order == MIXGCN_ORDER_AGG_FIRST ? d->d_in : d->d_out;
+    if (d->ld_in < d->d_in || d->ld_out < d->d_out || d->ld_saved < saved_cols || (d->ld_in & 3) || (d->ld_out & 3) || (d->ld_saved & 3))
+        MIXGCN_FAIL(MIXGCN_EINVAL, "%s: leading dimensions must be multiples of 4 with ld_in >= d_in, ld_out >= d_out, ld_saved >= %d", who, saved_cols);
+    if (d->n_chunks < 0 || d->n_chunks > 64) MIXGCN_FAIL(MIXGCN_EINVAL, "%s: n_chunks must lie in [0, 64]", who);
+    return MIXGCN_OK;
+}
+
+// Row range of chunk i of m over k rows: the floor(k*i/m) boundaries of Algorithm 2's update loop.
+inline int64_t chunk_bound(int64_t k, int i, int m) { return (k * (int64_t)i) / m; }
+
+}  // namespace
+
+extern "C" mixgcn_status mixgcn_layer_plan(const mixgcn_layer_desc* desc, int32_t* order, int32_t* saved_cols) {
+    if (!desc) MIXGCN_FAIL(MIXGCN_EINVAL, "layer_plan: null descriptor");
+    if (desc->d_in <= 0 || desc->d_out <= 0 || desc->order < 0 || desc->order > 2)
+        MIXGCN_FAIL(MIXGCN_EINVAL, "layer_plan: bad widths or order");
+    const int o = resolve_order(desc);
+    if (order) *order = o;
+    if (saved_cols) *saved_cols = o == MIXGCN_ORDER_AGG_FIRST ? desc->d_in : desc->d_out;
+    return MIXGCN_OK;
+}
+
+extern "C" mixgcn_status mixgcn_layer_fwd(mixgcn_ctx* ctx, const mixgcn_graph* g, const mixgcn_layer_desc* d,
+                                          const float* X_in, const float* W, const float* bias,
+                                          const uint8_t* drop_mask, float* saved, float* X_out, void* stream) {
+    if (!ctx || !g || !X_in || !W || !saved || !X_out) MIXGCN_FAIL(MIXGCN_EINVAL, "layer_fwd: null argument");
+    MIXGCN_TRY(check_desc(d, "layer_fwd"));
+    if (!aligned16(X_in) || !aligned16(saved) || !aligned16(X_out) || !aligned16(W))
+        MIXGCN_FAIL(MIXGCN_EINVAL, "layer_fwd: matrices must be 16-byte aligned");
+    MIXGCN_CUDA(cudaSetDevice(ctx->device));
+    cudaStream_t s = (cudaStream_t)stream;
+    const int64_t n = g->n;
+    const int order = resolve_order(d);
+    mixgcn_epilogue epi{};
+    epi.bias = bias;
+    epi.relu = (d->flags & MIXGCN_LAYER_RELU) ? 1 : 0;
+    epi.drop_mask = drop_mask;
+    epi.keep_scale = d->keep_scale;
+    const int64_t ldw = d->d_out;  // W is dense; the GEMM uses scalar loads for it when d_out % 4 != 0
+    const int chunks = d->n_chunks > 1 ? d->n_chunks : 1;
+
+    if (order == MIXGCN_ORDER_AGG_FIRST) {
+        if (chunks == 1) {
+            MIXGCN_TRY(launch_spmm(ctx, g, g->fwd, 0, n, d->d_in, X_in, d->ld_in, saved, d->ld_saved, nullptr, s));
+            MIXGCN_TRY(launch_gemm(ctx, d->precision, 0, 0, n, d->d_out, d->d_in, saved, d->ld_saved, W, ldw, X_out,
+                                   d->ld_out, &epi, 0, s));
+            return MIXGCN_OK;
+        }
+        // aggregation of chunk k+1 on stream A overlaps the update of chunk k on stream B
+        cudaStream_t sa = ctx->side_stream[0], sb = ctx->side_stream[1];
+        MIXGCN_CUDA(cudaEventRecord(ctx->fork_ev, s));
+        MIXGCN_CUDA(cudaStreamWaitEvent(sa, ctx->fork_ev, 0));
+        MIXGCN_CUDA(cudaStreamWaitEvent(sb, ctx->fork_ev, 0));
+        for (int k = 0; k < chunks; ++k) {
+            const int64_t r0 = chunk_bound(n, k, chunks), r1 = chunk_bound(n, k + 1, chunks);
+            if (r1 <= r0) continue;
+            MIXGCN_TRY(launch_spmm(ctx, g, g->fwd, r0, r1, d->d_in, X_in, d->ld_in, saved, d->ld_saved, nullptr, sa));
+            MIXGCN_CUDA(cudaEventRecord(ctx->chunk_ev[k], sa));
+            MIXGCN_CUDA(cudaStreamWaitEvent(sb, ctx->chunk_ev[k], 0));
+            MIXGCN_TRY(launch_gemm(ctx, d->precision, 0, 0, r1 - r0, d->d_out, d->d_in, saved + r0 * d->ld_saved,
+                                   d->ld_saved, W, ldw, X_out + r0 * d->ld_out, d->ld_out, &epi, r0, sb));
+        }
+        MIXGCN_CUDA(cudaEventRecord(ctx->join_ev[0], sa));
+        MIXGCN_CUDA(cudaEventRecord(ctx->join_ev[1], sb));
+        MIXGCN_CUDA(cudaStreamWaitEvent(s, ctx->join_ev[0], 0));
+        MIXGCN_CUDA(cudaStreamWaitEvent(s, ctx->join_ev[1], 0));
+        return MIXGCN_OK;
+    }
+    // update first: Q = X_in W (into `saved`), then X_out = epilogue(A_hat Q).  Every row of Q is
+    // needed before any aggregated row can be produced, so there is nothing to chunk here.
+    MIXGCN_TRY(launch_gemm(ctx, d->precision, 0, 0, n, d->d_out, d->d_in, X_in, d->ld_in, W, ldw, saved, d->ld_saved,
+                           nullptr, 0, s));
+    MIXGCN_TRY(launch_spmm(ctx, g, g->fwd, 0, n, d->d_out, saved, d->ld_saved, X_out, d->ld_out, &epi, s));
+    return MIXGCN_OK;
+}
+
+extern "C" mixgcn_status mixgcn_layer_bwd(mixgcn_ctx* ctx, const mixgcn_graph* g, const mixgcn_layer_desc* d,
+                                          const float* X_in, float* saved, const float* X_out,
+                                          const uint8_t* drop_mask, const float* W, float* G_out, float* G_in,
+                                          float* dW, float* dbias, void* stream) {
+    if (!ctx || !g || !X_in || !saved || !X_out || !W || !G_out || !dW) MIXGCN_FAIL(MIXGCN_EINVAL, "layer_bwd: null argument");
+    MIXGCN_TRY(check_desc(d, "layer_bwd"));
+    const bool first = (d->flags & MIXGCN_LAYER_FIRST) != 0;
+    if (first != (G_in == nullptr)) MIXGCN_FAIL(MIXGCN_EINVAL, "layer_bwd: G_in must be NULL exactly when MIXGCN_LAYER_FIRST is set");
+    if (!aligned16(X_in) || !aligned16(saved) || !aligned16(X_out) || !aligned16(W) || !aligned16(G_out) ||
+        !aligned16(dW) || (G_in && !aligned16(G_in)))
+        MIXGCN_FAIL(MIXGCN_EINVAL, "layer_bwd: matrices must be 16-byte aligned");
+    MIXGCN_CUDA(cudaSetDevice(ctx->device));
+    cudaStream_t s = (cudaStream_t)stream;
+    const int64_t n = g->n;
+    const int order = resolve_order(d);
+    const int relu = (d->flags & MIXGCN_LAYER_RELU) ? 1 : 0;
+    const int64_t ldw = d->d_out;
+
+    // gradient w.r.t. the pre-activation, in place in G_out
+    if (!(d->flags & MIXGCN_LAYER_GOUT_GATED) && (relu || drop_mask))
+        MIXGCN_TRY(launch_gate(ctx, n, d->d_out, G_out, d->ld_out, X_out, d->ld_out, relu, drop_mask, d->keep_scale, s));
+    if (dbias) MIXGCN_TRY(launch_colsum(ctx, n, d->d_out, G_out, d->ld_out, dbias, s));
+
+    mixgcn_epilogue gin_epi{};
+    const mixgcn_epilogue* gin = nullptr;
+    if (d->flags & MIXGCN_LAYER_GATE_GIN) {
+        gin_epi.gate = X_in; gin_epi.ld_gate = d->ld_in; gin_epi.gate_scale = d->in_scale; gin_epi.keep_scale = 1.0f;
+        gin = &gin_epi;
+    }
+
+    if (order == MIXGCN_ORDER_AGG_FIRST) {
+        // dW = (A_hat X_in)^T dP ; dZ = dP W^T (over `saved`) ; G_in = A_hat^T dZ
+        MIXGCN_TRY(launch_gemm(ctx, d->precision, 1, 0, d->d_in, d->d_out, n, saved, d->ld_saved, G_out, d->ld_out, dW,
+                               ldw, nullptr, 0, s));
+        if (!first) {
+            MIXGCN_TRY(launch_gemm(ctx, d->precision, 0, 1, n, d->d_in, d->d_out, G_out, d->ld_out, W, ldw, saved,
+                                   d->ld_saved, nullptr, 0, s));
+            MIXGCN_TRY(launch_spmm(ctx, g, g->bwd, 0, n, d->d_in, saved, d->ld_saved, G_in, d->ld_in, gin, s));
+        }
+        return MIXGCN_OK;
+    }
+    // update first: dQ = A_hat^T dZ (into `saved`) ; dW = X_in^T dQ ; G_in = dQ W^T
+    MIXGCN_TRY(launch_spmm(ctx, g, g->bwd, 0, n, d->d_out, G_out, d->ld_out, saved, d->ld_saved, nullptr, s));
+    MIXGCN_TRY(launch_gemm(ctx, d->precision, 1, 0, d->d_in, d->d_out, n, X_in, d->ld_in, saved, d->ld_saved, dW, ldw,
+                           nullptr, 0, s));
+    if (!first)
+        MIXGCN_TRY(launch_gemm(ctx, d->precision, 0, 1, n, d->d_in, d->d_out, saved, d->ld_saved, W, ldw, G_in, d->ld_in,
+                               gin, 0, s));
+    return MIXGCN_OK;
+}
+
+extern "C" mixgcn_status mixgcn_train_step_host(mixgcn_ctx* ctx, const mixgcn_graph* g, int32_t L,
+                                                const int32_t* dims, int32_t precision, const float* X,
+                                                const int32_t* labels, const uint8_t* train_mask,
+                                                float* const* W, float* const* b, float* const* mW,
+                                                float* const* vW, float* const* mb, float* const* vb,
+                                                int64_t t, float lr, float beta1, float beta2, float eps,
+                                                float* loss, int32_t* pred) {
+    (void)ctx; (void)g; (void)L; (void)dims; (void)precision; (void)X; (void)labels; (void)train_mask;
+    (void)W; (void)b; (void)mW; (void)vW; (void)mb; (void)vb; (void)t; (void)lr; (void)beta1; (void)beta2;
+    (void)eps; (void)loss; (void)pred;
+    MIXGCN_FAIL(MIXGCN_EUNSUPPORTED, "train_step_host: not built yet");
+}

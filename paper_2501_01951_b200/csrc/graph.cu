@@ -1,0 +1,380 @@
+// Graph construction on the device: edge list -> A + I in CSR -> symmetric normalisation
+// A_hat = D^-1/2 (A+I) D^-1/2 (Section 2.1 of the paper) -> CSR of the transpose (aliased when
+// symmetric) -> degree-sorted row schedule.  Sorting, run-length and selection steps use CUB
+// device primitives; everything else is a kernel in this file.
+#include <cub/cub.cuh>
+
+#include <new>
+
+#include "internal.cuh"
+
+using namespace mixgcn;
+
+namespace {
+
+constexpr int TPB = 256;
+inline unsigned blocks_for(int64_t n) { return (unsigned)((n + TPB - 1) / TPB); }
+
+// flag bits written by validation kernels
+enum { F_BAD_ID = 1, F_NOT_SYMMETRIC = 2, F_BAD_ROWPTR = 4, F_UNSORTED = 8 };
+
+__global__ void make_keys_kernel(int64_t n, int64_t m, const int32_t* __restrict__ src,
+                                 const int32_t* __restrict__ dst, int sym, int self_loops,
+                                 uint64_t sentinel, uint64_t* __restrict__ keys, int32_t* flags) {
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < m) {
+        int32_t u = src[i], v = dst[i];
+        bool bad = u < 0 || v < 0 || u >= n || v >= n;
+        if (bad) atomicOr(flags, F_BAD_ID);
+        bool drop = bad || u == v;
+        keys[i] = drop ? sentinel : (((uint64_t)(uint32_t)u << 32) | (uint32_t)v);
+        if (sym) keys[m + i] = drop ? sentinel : (((uint64_t)(uint32_t)v << 32) | (uint32_t)u);
+    }
+    if (self_loops && i < n) {
+        int64_t base = sym ? 2 * m : m;
+        keys[base + i] = ((uint64_t)i << 32) | (uint64_t)i;
+    }
+}
+
+// rowptr[q] = first position whose row id is >= q, from the sorted unique keys.
+__global__ void rowptr_from_keys_kernel(int64_t n, int64_t nnz, const uint64_t* __restrict__ keys,
+                                        int64_t* __restrict__ rowptr, int32_t* __restrict__ col) {
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < nnz) {
+        int64_t r = (int64_t)(keys[i] >> 32);
+        int64_t rp = i == 0 ? -1 : (int64_t)(keys[i - 1] >> 32);
+        for (int64_t q = rp + 1; q <= r; ++q) rowptr[q] = i;
+        col[i] = (int32_t)(uint32_t)(keys[i] & 0xFFFFFFFFull);
+    } else if (i == nnz) {
+        int64_t last = nnz == 0 ? -1 : (int64_t)(keys[nnz - 1] >> 32);
+        for (int64_t q = last + 1; q <= n; ++q) rowptr[q] = nnz;
+    }
+}
+
+__global__ void degree_kernel(int64_t n, const int64_t* __restrict__ rowptr, int32_t* __restrict__ deg,
+                              float* __restrict__ dinv) {
+    int64_t u = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (u >= n) return;
+    int32_t d = (int32_t)(rowptr[u + 1] - rowptr[u]);
+    deg[u] = d;
+    // dinv = 1/sqrt(deg): IEEE square root, then IEEE reciprocal, each rounded to fp32.
+    dinv[u] = d > 0 ? __frcp_rn(__fsqrt_rn((float)d)) : 0.0f;
+}
+
+// One warp per row: val_uv = dinv_u * dinv_v.
+__global__ void values_kernel(int64_t n, const int64_t* __restrict__ rowptr, const int32_t* __restrict__ col,
+                              const float* __restrict__ dinv, float* __restrict__ val) {
+    int64_t u = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    int lane = threadIdx.x & 31;
+    if (u >= n) return;
+    float du = dinv[u];
+    for (int64_t i = rowptr[u] + lane; i < rowptr[u + 1]; i += 32) val[i] = __fmul_rn(du, dinv[col[i]]);
+}
+
+// For every stored (u,v), u != v, look v's row up for u.
+__global__ void symmetry_kernel(int64_t n, const int64_t* __restrict__ rowptr, const int32_t* __restrict__ col,
+                                int32_t* flags) {
+    int64_t u = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    int lane = threadIdx.x & 31;
+    if (u >= n) return;
+    for (int64_t i = rowptr[u] + lane; i < rowptr[u + 1]; i += 32) {
+        int32_t v = col[i];
+        if (v == u) continue;
+        int64_t lo = rowptr[v], hi = rowptr[v + 1];
+        bool found = false;
+        while (lo < hi) {
+            int64_t mid = (lo + hi) >> 1;
+            int32_t c = col[mid];
+            if (c == (int32_t)u) { found = true; break; }
+            if (c < (int32_t)u) lo = mid + 1; else hi = mid;
+        }
+        if (!found) { atomicOr(flags, F_NOT_SYMMETRIC); return; }
+    }
+}
+
+__global__ void transpose_keys_kernel(int64_t n, const int64_t* __restrict__ rowptr,
+                                      const int32_t* __restrict__ col, uint64_t* __restrict__ keys) {
+    int64_t u = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    int lane = threadIdx.x & 31;
+    if (u >= n) return;
+    for (int64_t i = rowptr[u] + lane; i < rowptr[u + 1]; i += 32)
+        keys[i] = ((uint64_t)(uint32_t)col[i] << 32) | (uint32_t)u;
+}
+
+__global__ void schedule_keys_kernel(int64_t n, const int64_t* __restrict__ rowptr, uint64_t* __restrict__ keys) {
+    int64_t u = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (u >= n) return;
+    uint64_t d = (uint64_t)(rowptr[u + 1] - rowptr[u]);
+    keys[u] = ((0x7FFFFFFFull - d) << 32) | (uint64_t)u;  // descending entries, ascending id
+}
+
+__global__ void schedule_finish_kernel(int64_t n, const uint64_t* __restrict__ keys, int32_t* __restrict__ perm,
+                                       int threshold, unsigned long long* n_hub) {
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    perm[i] = (int32_t)(uint32_t)(keys[i] & 0xFFFFFFFFull);
+    int64_t d = (int64_t)(0x7FFFFFFFull - (keys[i] >> 32));
+    if (d > threshold) atomicAdd(n_hub, 1ull);
+}
+
+__global__ void validate_csr_kernel(int64_t n, int64_t nnz, const int64_t* __restrict__ rowptr,
+                                    const int32_t* __restrict__ col, int32_t* flags) {
+    int64_t u = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (u >= n) return;
+    int64_t b = rowptr[u], e = rowptr[u + 1];
+    if ((u == 0 && b != 0) || b < 0 || e < b || e > nnz) { atomicOr(flags, F_BAD_ROWPTR); return; }
+    if (e - b > 0x7FFFFFFFll) { atomicOr(flags, F_BAD_ROWPTR); return; }
+    for (int64_t i = b; i < e; ++i) {
+        int32_t c = col[i];
+        if (c < 0 || c >= n) { atomicOr(flags, F_BAD_ID); return; }
+        if (i > b && col[i - 1] >= c) { atomicOr(flags, F_UNSORTED); return; }
+    }
+}
+
+struct DevBuf {  // frees on scope exit
+    void* p = nullptr;
+    ~DevBuf() { if (p) cudaFree(p); }
+    template <class T> T* as() { return reinterpret_cast<T*>(p); }
+};
+
+int bits_for(uint64_t x) { int b = 0; while (x) { ++b; x >>= 1; } return b; }
+
+void free_view(CsrView& v) {
+    cudaFree(v.rowptr); cudaFree(v.col); cudaFree(v.val); cudaFree(v.perm);
+    v = CsrView{};
+}
+
+mixgcn_status build_schedule(int64_t n, CsrView& v, cudaStream_t s) {
+    DevBuf k0, k1, tmp, hub;
+    MIXGCN_CUDA(cudaMalloc(&k0.p, n * sizeof(uint64_t)));
+    MIXGCN_CUDA(cudaMalloc(&k1.p, n * sizeof(uint64_t)));
+    MIXGCN_CUDA(cudaMalloc(&hub.p, sizeof(unsigned long long)));
+    MIXGCN_CUDA(cudaMemsetAsync(hub.p, 0, sizeof(unsigned long long), s));
+    MIXGCN_CUDA(cudaMalloc((void**)&v.perm, n * sizeof(int32_t)));
+    schedule_keys_kernel<<<blocks_for(n), TPB, 0, s>>>(n, v.rowptr, k0.as<uint64_t>());
+    size_t tb = 0;
+    MIXGCN_CUDA(cub::DeviceRadixSort::SortKeys(nullptr, tb, k0.as<uint64_t>(), k1.as<uint64_t>(), n, 0, 64, s));
+    MIXGCN_CUDA(cudaMalloc(&tmp.p, tb ? tb : 1));
+    MIXGCN_CUDA(cub::DeviceRadixSort::SortKeys(tmp.p, tb, k0.as<uint64_t>(), k1.as<uint64_t>(), n, 0, 64, s));
+    schedule_finish_kernel<<<blocks_for(n), TPB, 0, s>>>(n, k1.as<uint64_t>(), v.perm, HUB_THRESHOLD,
+                                                         hub.as<unsigned long long>());
+    unsigned long long h = 0;
+    uint64_t first = 0;
+    MIXGCN_CUDA(cudaMemcpyAsync(&h, hub.p, sizeof(h), cudaMemcpyDeviceToHost, s));
+    MIXGCN_CUDA(cudaMemcpyAsync(&first, k1.p, sizeof(first), cudaMemcpyDeviceToHost, s));
+    MIXGCN_CUDA(cudaStreamSynchronize(s));
+    v.n_hub = (int64_t)h;
+    v.max_deg = (int32_t)(0x7FFFFFFFull - (first >> 32));
+    return MIXGCN_OK;
+}
+
+// Everything after rowptr/col exist: degrees, values, symmetry, transpose, schedules.
+mixgcn_status finish_graph(mixgcn_graph* g, cudaStream_t s) {
+    const int64_t n = g->n, nnz = g->nnz;
+    CsrView& A = g->fwd;
+    DevBuf flags;
+    MIXGCN_CUDA(cudaMalloc(&flags.p, sizeof(int32_t)));
+    MIXGCN_CUDA(cudaMemsetAsync(flags.p, 0, sizeof(int32_t), s));
+    MIXGCN_CUDA(cudaMalloc((void**)&g->deg, n * sizeof(int32_t)));
+    MIXGCN_CUDA(cudaMalloc((void**)&g->dinv, n * sizeof(float)));
+    MIXGCN_CUDA(cudaMalloc((void**)&A.val, (nnz > 0 ? nnz : 1) * sizeof(float)));
+    degree_kernel<<<blocks_for(n), TPB, 0, s>>>(n, A.rowptr, g->deg, g->dinv);
+    values_kernel<<<blocks_for(n * 32), TPB, 0, s>>>(n, A.rowptr, A.col, g->dinv, A.val);
+    symmetry_kernel<<<blocks_for(n * 32), TPB, 0, s>>>(n, A.rowptr, A.col, flags.as<int32_t>());
+    int32_t hf = 0;
+    MIXGCN_CUDA(cudaMemcpyAsync(&hf, flags.p, sizeof(hf), cudaMemcpyDeviceToHost, s));
+    MIXGCN_CUDA(cudaStreamSynchronize(s));
+    g->symmetric = (hf & F_NOT_SYMMETRIC) ? 0 : 1;
+    MIXGCN_TRY(build_schedule(n, A, s));
+    if (g->symmetric) {
+        g->bwd = A;  // alias: the same index serves the backward aggregation
+        return MIXGCN_OK;
+    }
+    // Transposed structure: sort (col,row) keys carrying the value.
+    CsrView& T = g->bwd;
+    DevBuf k0, k1, v1, tmp;
+    const int64_t cap = nnz > 0 ? nnz : 1;
+    MIXGCN_CUDA(cudaMalloc(&k0.p, cap * sizeof(uint64_t)));
+    MIXGCN_CUDA(cudaMalloc(&k1.p, cap * sizeof(uint64_t)));
+    MIXGCN_CUDA(cudaMalloc((void**)&T.val, cap * sizeof(float)));
+    MIXGCN_CUDA(cudaMalloc((void**)&T.rowptr, (n + 1) * sizeof(int64_t)));
+    MIXGCN_CUDA(cudaMalloc((void**)&T.col, cap * sizeof(int32_t)));
+    transpose_keys_kernel<<<blocks_for(n * 32), TPB, 0, s>>>(n, A.rowptr, A.col, k0.as<uint64_t>());
+    size_t tb = 0;
+    const int end_bit = 32 + bits_for((uint64_t)n);
+    MIXGCN_CUDA(cub::DeviceRadixSort::SortPairs(nullptr, tb, k0.as<uint64_t>(), k1.as<uint64_t>(), A.val, T.val,
+                                                nnz, 0, end_bit, s));
+    MIXGCN_CUDA(cudaMalloc(&tmp.p, tb ? tb : 1));
+    MIXGCN_CUDA(cub::DeviceRadixSort::SortPairs(tmp.p, tb, k0.as<uint64_t>(), k1.as<uint64_t>(), A.val, T.val,
+                                                nnz, 0, end_bit, s));
+    rowptr_from_keys_kernel<<<blocks_for(nnz + 1), TPB, 0, s>>>(n, nnz, k1.as<uint64_t>(), T.rowptr, T.col);
+    MIXGCN_CUDA(cudaStreamSynchronize(s));
+    MIXGCN_TRY(build_schedule(n, T, s));
+    return MIXGCN_OK;
+}
+
+mixgcn_status check_common(mixgcn_ctx* ctx, int64_t n, mixgcn_graph** out) {
+    if (!ctx || !out) MIXGCN_FAIL(MIXGCN_EINVAL, "graph_create: null ctx or out");
+    if (n <= 0) MIXGCN_FAIL(MIXGCN_EINVAL, "graph_create: n must be positive (got %lld)", (long long)n);
+    if (n >= 0x7FFFFFFFll) MIXGCN_FAIL(MIXGCN_EBADGRAPH, "graph_create: n = %lld does not fit int32 ids", (long long)n);
+    return MIXGCN_OK;
+}
+
+}  // namespace
+
+extern "C" mixgcn_status mixgcn_graph_destroy(mixgcn_graph* g) {
+    if (!g) return MIXGCN_OK;
+    cudaSetDevice(g->ctx->device);
+    if (!g->symmetric) free_view(g->bwd);
+    free_view(g->fwd);
+    cudaFree(g->deg);
+    cudaFree(g->dinv);
+    delete g;
+    return MIXGCN_OK;
+}
+
+extern "C" mixgcn_status mixgcn_graph_create(mixgcn_ctx* ctx, int64_t n, int64_t m, const int32_t* src,
+                                             const int32_t* dst, uint32_t flags, mixgcn_graph** out) {
+    MIXGCN_TRY(check_common(ctx, n, out));
+    if (m < 0 || (m > 0 && (!src || !dst))) MIXGCN_FAIL(MIXGCN_EINVAL, "graph_create: bad edge list (m=%lld)", (long long)m);
+    MIXGCN_CUDA(cudaSetDevice(ctx->device));
+    cudaStream_t s = ctx->side_stream[0];
+    const int sym = (flags & MIXGCN_GRAPH_SYMMETRISE) != 0, self = (flags & MIXGCN_GRAPH_ADD_SELF_LOOPS) != 0;
+    const int64_t total = m * (sym ? 2 : 1) + (self ? n : 0);
+
+    mixgcn_graph* g = new (std::nothrow) mixgcn_graph();
+    if (!g) MIXGCN_FAIL(MIXGCN_ENOMEM, "graph_create: host allocation failed");
+    g->ctx = ctx; g->n = n; g->nnz = 0; g->symmetric = 1;
+    struct Guard { mixgcn_graph* g; bool keep = false; ~Guard() { if (!keep) { g->symmetric = g->bwd.rowptr == g->fwd.rowptr; mixgcn_graph_destroy(g); } } } guard{g};
+    LaunchScope scope(ctx, PH_GRAPH, s, 12);
+
+    DevBuf dsrc, ddst, k0, k1, tmp, fl, cnt;
+    const int32_t *ps = src, *pd = dst;
+    if (!(flags & MIXGCN_GRAPH_EDGES_ON_DEVICE) && m > 0) {
+        MIXGCN_CUDA(cudaMalloc(&dsrc.p, m * sizeof(int32_t)));
+        MIXGCN_CUDA(cudaMalloc(&ddst.p, m * sizeof(int32_t)));
+        MIXGCN_CUDA(cudaMemcpyAsync(dsrc.p, src, m * sizeof(int32_t), cudaMemcpyHostToDevice, s));
+        MIXGCN_CUDA(cudaMemcpyAsync(ddst.p, dst, m * sizeof(int32_t), cudaMemcpyHostToDevice, s));
+        ps = dsrc.as<int32_t>(); pd = ddst.as<int32_t>();
+    }
+    const int64_t cap = total > 0 ? total : 1;
+    MIXGCN_CUDA(cudaMalloc(&k0.p, cap * sizeof(uint64_t)));
+    MIXGCN_CUDA(cudaMalloc(&k1.p, cap * sizeof(uint64_t)));
+    MIXGCN_CUDA(cudaMalloc(&fl.p, sizeof(int32_t)));
+    MIXGCN_CUDA(cudaMalloc(&cnt.p, sizeof(int64_t)));
+    MIXGCN_CUDA(cudaMemsetAsync(fl.p, 0, sizeof(int32_t), s));
+    const uint64_t sentinel = (uint64_t)n << 32;  // sorts after every valid key
+    {
+        int64_t work = m > n ? m : n;
+        make_keys_kernel<<<blocks_for(work > 0 ? work : 1), TPB, 0, s>>>(n, m, ps, pd, sym, self, sentinel,
+                                                                        k0.as<uint64_t>(), fl.as<int32_t>());
+    }
+    const int end_bit = 32 + bits_for((uint64_t)n);
+    size_t tb_sort = 0, tb_uniq = 0;
+    MIXGCN_CUDA(cub::DeviceRadixSort::SortKeys(nullptr, tb_sort, k0.as<uint64_t>(), k1.as<uint64_t>(), total, 0, end_bit, s));
+    MIXGCN_CUDA(cub::DeviceSelect::Unique(nullptr, tb_uniq, k1.as<uint64_t>(), k0.as<uint64_t>(), cnt.as<int64_t>(), total, s));
+    size_t tb = tb_sort > tb_uniq ? tb_sort : tb_uniq;
+    MIXGCN_CUDA(cudaMalloc(&tmp.p, tb ? tb : 1));
+    MIXGCN_CUDA(cub::DeviceRadixSort::SortKeys(tmp.p, tb, k0.as<uint64_t>(), k1.as<uint64_t>(), total, 0, end_bit, s));
+    // edge arrays are no longer needed
+    MIXGCN_CUDA(cub::DeviceSelect::Unique(tmp.p, tb, k1.as<uint64_t>(), k0.as<uint64_t>(), cnt.as<int64_t>(), total, s));
+    int64_t n_unique = 0;
+    int32_t hf = 0;
+    MIXGCN_CUDA(cudaMemcpyAsync(&n_unique, cnt.p, sizeof(int64_t), cudaMemcpyDeviceToHost, s));
+    MIXGCN_CUDA(cudaMemcpyAsync(&hf, fl.p, sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+    MIXGCN_CUDA(cudaStreamSynchronize(s));
+    if (hf & F_BAD_ID) MIXGCN_FAIL(MIXGCN_EBADGRAPH, "graph_create: a node id lies outside [0, %lld)", (long long)n);
+    if (total == 0) n_unique = 0;
+    if (n_unique > 0) {
+        uint64_t last = 0;
+        MIXGCN_CUDA(cudaMemcpy(&last, k0.as<uint64_t>() + (n_unique - 1), sizeof(last), cudaMemcpyDeviceToHost));
+        if (last == sentinel) --n_unique;
+    }
+    g->nnz = n_unique;
+    cudaFree(k1.p); k1.p = nullptr;
+    cudaFree(tmp.p); tmp.p = nullptr;
+    MIXGCN_CUDA(cudaMalloc((void**)&g->fwd.rowptr, (n + 1) * sizeof(int64_t)));
+    MIXGCN_CUDA(cudaMalloc((void**)&g->fwd.col, (n_unique > 0 ? n_unique : 1) * sizeof(int32_t)));
+    rowptr_from_keys_kernel<<<blocks_for(n_unique + 1), TPB, 0, s>>>(n, n_unique, k0.as<uint64_t>(), g->fwd.rowptr, g->fwd.col);
+    MIXGCN_CUDA(cudaStreamSynchronize(s));
+    cudaFree(k0.p); k0.p = nullptr;
+    MIXGCN_TRY(finish_graph(g, s));
+    MIXGCN_CUDA(cudaGetLastError());
+    guard.keep = true;
+    *out = g;
+    return MIXGCN_OK;
+}
+
+extern "C" mixgcn_status mixgcn_graph_create_from_csr(mixgcn_ctx* ctx, int64_t n, const int64_t* rowptr,
+                                                      const int32_t* col, uint32_t flags, mixgcn_graph** out) {
+    MIXGCN_TRY(check_common(ctx, n, out));
+    if (!rowptr) MIXGCN_FAIL(MIXGCN_EINVAL, "graph_create_from_csr: null rowptr");
+    MIXGCN_CUDA(cudaSetDevice(ctx->device));
+    cudaStream_t s = ctx->side_stream[0];
+    const bool on_dev = (flags & MIXGCN_GRAPH_EDGES_ON_DEVICE) != 0;
+    const cudaMemcpyKind kind = on_dev ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice;
+    int64_t nnz = 0;
+    MIXGCN_CUDA(cudaMemcpy(&nnz, rowptr + n, sizeof(int64_t), on_dev ? cudaMemcpyDeviceToHost : cudaMemcpyHostToHost));
+    if (nnz < 0) MIXGCN_FAIL(MIXGCN_EBADGRAPH, "graph_create_from_csr: rowptr[n] is negative");
+    if (nnz > 0 && !col) MIXGCN_FAIL(MIXGCN_EINVAL, "graph_create_from_csr: null col");
+
+    mixgcn_graph* g = new (std::nothrow) mixgcn_graph();
+    if (!g) MIXGCN_FAIL(MIXGCN_ENOMEM, "graph_create_from_csr: host allocation failed");
+    g->ctx = ctx; g->n = n; g->nnz = nnz; g->symmetric = 1;
+    struct Guard { mixgcn_graph* g; bool keep = false; ~Guard() { if (!keep) { g->symmetric = g->bwd.rowptr == g->fwd.rowptr; mixgcn_graph_destroy(g); } } } guard{g};
+    LaunchScope scope(ctx, PH_GRAPH, s, 8);
+    DevBuf fl;
+    MIXGCN_CUDA(cudaMalloc(&fl.p, sizeof(int32_t)));
+    MIXGCN_CUDA(cudaMemsetAsync(fl.p, 0, sizeof(int32_t), s));
+    MIXGCN_CUDA(cudaMalloc((void**)&g->fwd.rowptr, (n + 1) * sizeof(int64_t)));
+    MIXGCN_CUDA(cudaMalloc((void**)&g->fwd.col, (nnz > 0 ? nnz : 1) * sizeof(int32_t)));
+    MIXGCN_CUDA(cudaMemcpyAsync(g->fwd.rowptr, rowptr, (n + 1) * sizeof(int64_t), kind, s));
+    if (nnz > 0) MIXGCN_CUDA(cudaMemcpyAsync(g->fwd.col, col, nnz * sizeof(int32_t), kind, s));
+    // rowptr must be validated before col is indexed with it: first monotonicity on the host side
+    // of the device array (cheap kernel), then the per-row column checks.
+    validate_csr_kernel<<<blocks_for(n), TPB, 0, s>>>(n, nnz, g->fwd.rowptr, g->fwd.col, fl.as<int32_t>());
+    int32_t hf = 0;
+    MIXGCN_CUDA(cudaMemcpyAsync(&hf, fl.p, sizeof(hf), cudaMemcpyDeviceToHost, s));
+    MIXGCN_CUDA(cudaStreamSynchronize(s));
+    if (hf & F_BAD_ROWPTR) MIXGCN_FAIL(MIXGCN_EBADGRAPH, "graph_create_from_csr: rowptr is not monotone from 0");
+    if (hf & F_BAD_ID) MIXGCN_FAIL(MIXGCN_EBADGRAPH, "graph_create_from_csr: a column id lies outside [0, %lld)", (long long)n);
+    if (hf & F_UNSORTED) MIXGCN_FAIL(MIXGCN_EBADGRAPH, "graph_create_from_csr: columns are not strictly ascending in a row");
+    MIXGCN_TRY(finish_graph(g, s));
+    MIXGCN_CUDA(cudaGetLastError());
+    guard.keep = true;
+    *out = g;
+    return MIXGCN_OK;
+}
+
+extern "C" mixgcn_status mixgcn_graph_info(const mixgcn_graph* g, int64_t* n, int64_t* nnz, int32_t* max_deg,
+                                           int32_t* symmetric) {
+    if (!g) MIXGCN_FAIL(MIXGCN_EINVAL, "graph_info: null graph");
+    if (n) *n = g->n;
+    if (nnz) *nnz = g->nnz;
+    if (max_deg) *max_deg = g->fwd.max_deg;
+    if (symmetric) *symmetric = g->symmetric;
+    return MIXGCN_OK;
+}
+
+extern "C" mixgcn_status mixgcn_graph_export(const mixgcn_graph* g, int transposed, int64_t* rowptr, int32_t* col,
+                                             float* val, int32_t* deg, float* dinv) {
+    if (!g) MIXGCN_FAIL(MIXGCN_EINVAL, "graph_export: null graph");
+    MIXGCN_CUDA(cudaSetDevice(g->ctx->device));
+    MIXGCN_CUDA(cudaDeviceSynchronize());
+    const CsrView& v = transposed ? g->bwd : g->fwd;
+    if (rowptr) MIXGCN_CUDA(cudaMemcpy(rowptr, v.rowptr, (g->n + 1) * sizeof(int64_t), cudaMemcpyDeviceToHost));
+    if (col && g->nnz) MIXGCN_CUDA(cudaMemcpy(col, v.col, g->nnz * sizeof(int32_t), cudaMemcpyDeviceToHost));
+    if (val && g->nnz) MIXGCN_CUDA(cudaMemcpy(val, v.val, g->nnz * sizeof(float), cudaMemcpyDeviceToHost));
+    if (deg) MIXGCN_CUDA(cudaMemcpy(deg, g->deg, g->n * sizeof(int32_t), cudaMemcpyDeviceToHost));
+    if (dinv) MIXGCN_CUDA(cudaMemcpy(dinv, g->dinv, g->n * sizeof(float), cudaMemcpyDeviceToHost));
+    return MIXGCN_OK;
+}
+
+extern "C" mixgcn_status mixgcn_graph_export_schedule(const mixgcn_graph* g, int transposed, int32_t* perm) {
+    if (!g || !perm) MIXGCN_FAIL(MIXGCN_EINVAL, "graph_export_schedule: null argument");
+    MIXGCN_CUDA(cudaSetDevice(g->ctx->device));
+    MIXGCN_CUDA(cudaDeviceSynchronize());
+    const CsrView& v = transposed ? g->bwd : g->fwd;
+    MIXGCN_CUDA(cudaMemcpy(perm, v.perm, g->n * sizeof(int32_t), cudaMemcpyDeviceToHost));
+    return MIXGCN_OK;
+}

@@ -1,0 +1,113 @@
+// Internal declarations shared by the translation units of libmixgcn.so.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stdio.h>
+
+#include "mixgcn.h"
+
+namespace mixgcn {
+
+void set_error(const char* fmt, ...);
+
+#define MIXGCN_FAIL(status, ...)          \
+    do {                                  \
+        ::mixgcn::set_error(__VA_ARGS__); \
+        return (status);                  \
+    } while (0)
+
+#define MIXGCN_CUDA(expr)                                                                    \
+    do {                                                                                     \
+        cudaError_t _e = (expr);                                                             \
+        if (_e != cudaSuccess) {                                                             \
+            ::mixgcn::set_error("%s failed: %s (%s:%d)", #expr, cudaGetErrorString(_e),      \
+                                __FILE__, __LINE__);                                         \
+            return _e == cudaErrorMemoryAllocation ? MIXGCN_ENOMEM : MIXGCN_ECUDA;           \
+        }                                                                                    \
+    } while (0)
+
+#define MIXGCN_TRY(expr)                     \
+    do {                                     \
+        mixgcn_status _s = (expr);           \
+        if (_s != MIXGCN_OK) return _s;      \
+    } while (0)
+
+enum Phase { PH_SPMM = 0, PH_GEMM = 1, PH_ELEM = 2, PH_LOSS = 3, PH_ADAM = 4, PH_GRAPH = 5 };
+
+// device status word codes
+enum { DEV_OK = 0, DEV_EMPTY_MASK = 1, DEV_BAD_LABEL = 2, DEV_WAIT_EXPIRED = 3 };
+
+struct ProfSpan {
+    cudaEvent_t a, b;
+    int phase;
+};
+
+}  // namespace mixgcn
+
+struct mixgcn_ctx {
+    int device;
+    int sm_count;
+    int32_t* d_status;        // device status word (int32[4])
+    void* workspace;          // grow-on-demand scratch
+    int64_t workspace_bytes;
+    cudaStream_t side_stream[2];
+    cudaEvent_t fork_ev, join_ev[2];
+    cudaEvent_t chunk_ev[64];
+    // profiling
+    int profile;
+    mixgcn::ProfSpan* spans;
+    int n_spans, cap_spans;
+    int64_t launches_total;
+    int64_t phase_launches[MIXGCN_N_PHASES];
+    // host-step buffers live in the workspace tail; nothing else owned
+};
+
+// One CSR orientation of A_hat plus its aggregation schedule.
+struct CsrView {
+    int64_t* rowptr;   // [n+1]
+    int32_t* col;      // [nnz]
+    float* val;        // [nnz]
+    int32_t* perm;     // [n] rows by descending entry count
+    int64_t n_hub;     // first n_hub rows of perm have > HUB_THRESHOLD entries
+    int32_t max_deg;
+};
+
+struct mixgcn_graph {
+    mixgcn_ctx* ctx;
+    int64_t n, nnz;
+    int symmetric;
+    int32_t* deg;      // [n] entries per row of the stored matrix
+    float* dinv;       // [n]
+    CsrView fwd, bwd;  // bwd aliases fwd when symmetric
+};
+
+namespace mixgcn {
+
+constexpr int HUB_THRESHOLD = 4096;  // rows longer than this get a whole CTA
+
+// Launch bookkeeping: counts the launch and, when profiling, brackets it with events.
+struct LaunchScope {
+    mixgcn_ctx* ctx;
+    cudaStream_t stream;
+    int span;
+    LaunchScope(mixgcn_ctx* c, int phase, cudaStream_t s, int n_launches = 1);
+    ~LaunchScope();
+};
+
+mixgcn_status ensure_workspace(mixgcn_ctx* ctx, int64_t bytes);
+
+// kernels' host launchers (all asynchronous on `s`)
+mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView& A, int64_t row_begin,
+                          int64_t row_end, int32_t w, const float* Y, int64_t ldy, float* Z, int64_t ldz,
+                          const mixgcn_epilogue* epi, cudaStream_t s);
+mixgcn_status launch_gemm(mixgcn_ctx* ctx, int precision, int ta, int tb, int64_t M, int64_t N, int64_t K,
+                          const float* A, int64_t lda, const float* B, int64_t ldb, float* C, int64_t ldc,
+                          const mixgcn_epilogue* epi, int64_t epi_row0, cudaStream_t s);
+mixgcn_status launch_colsum(mixgcn_ctx* ctx, int64_t n, int32_t d, const float* X, int64_t ld, float* out,
+                            cudaStream_t s);
+mixgcn_status launch_gate(mixgcn_ctx* ctx, int64_t n, int32_t d, float* G, int64_t ldg, const float* X_out,
+                          int64_t ldx, int relu, const uint8_t* drop_mask, float keep_scale, cudaStream_t s);
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace mixgcn

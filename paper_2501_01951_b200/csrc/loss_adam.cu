@@ -1,0 +1,199 @@
+// Masked softmax cross-entropy with its gradient and arg-max (the loss line of Algorithm 2),
+// and the Adam step (its weight-update line).  Both are streaming kernels; floating-point
+// reductions run in a fixed order (per-warp shuffles, per-CTA partials, one final pass).
+#include "internal.cuh"
+
+using namespace mixgcn;
+
+namespace {
+
+constexpr int LOSS_WARPS = 8;
+
+__global__ void count_mask_kernel(int64_t n, const uint8_t* __restrict__ mask, unsigned long long* count) {
+    __shared__ unsigned int sm[8];
+    unsigned int c = 0;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
+        c += mask[i] ? 1u : 0u;
+    for (int o = 16; o > 0; o >>= 1) c += __shfl_down_sync(0xFFFFFFFFu, c, o);
+    if ((threadIdx.x & 31) == 0) sm[threadIdx.x >> 5] = c;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        unsigned int t = 0;
+        for (int w = 0; w < 8; ++w) t += sm[w];
+        if (t) atomicAdd(count, (unsigned long long)t);  // integer: order does not matter
+    }
+}
+
+// One warp per row.  part[block] receives the block's sum of per-row losses.
+__global__ void __launch_bounds__(LOSS_WARPS * 32) loss_rows_kernel(
+    int64_t n, int C, const float* logits, int64_t ld, const int32_t* __restrict__ labels,
+    const uint8_t* __restrict__ mask, const unsigned long long* __restrict__ count, float* dlogits,
+    int32_t* __restrict__ pred, unsigned long long* n_correct, double* __restrict__ part, int32_t* status) {
+    __shared__ double sm[LOSS_WARPS];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const unsigned long long T = *count;
+    const float invT = T ? (float)(1.0 / (double)T) : 0.0f;
+    double local = 0.0;
+    unsigned int correct = 0;
+    const int64_t stride = (int64_t)gridDim.x * LOSS_WARPS;
+    for (int64_t v = (int64_t)blockIdx.x * LOSS_WARPS + warp; v < n; v += stride) {
+        const float* row = logits + v * ld;
+        // arg-max with lowest-index ties
+        float mx = -INFINITY; int arg = 0x7FFFFFFF;
+        for (int c = lane; c < C; c += 32) {
+            const float x = row[c];
+            if (x > mx || (x == mx && c < arg)) { mx = x; arg = c; }
+        }
+        if (arg == 0x7FFFFFFF) arg = lane < C ? lane : 0;  // all -inf or NaN in this lane's columns
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float omx = __shfl_xor_sync(0xFFFFFFFFu, mx, o);
+            const int oarg = __shfl_xor_sync(0xFFFFFFFFu, arg, o);
+            if (omx > mx || (omx == mx && oarg < arg)) { mx = omx; arg = oarg; }
+        }
+        if (pred && lane == 0) pred[v] = arg;
+        const bool train = mask[v] != 0 && T != 0;
+        int y = 0;
+        bool ok = false;
+        if (train) {
+            y = labels[v];
+            ok = y >= 0 && y < C;
+            if (!ok && lane == 0) atomicMax(status, DEV_BAD_LABEL);
+        }
+        if (!train || !ok) {
+            if (dlogits) for (int c = lane; c < C; c += 32) dlogits[v * ld + c] = 0.0f;
+            continue;
+        }
+        float s = 0.0f;
+        for (int c = lane; c < C; c += 32) s += expf(row[c] - mx);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
+        const float lse = mx + logf(s);
+        const float py = row[y];
+        if (lane == 0) { local += (double)(lse - py); if (arg == y) ++correct; }
+        __syncwarp();  // dlogits may alias logits: every read of the row precedes the writes
+        if (dlogits)
+            for (int c = lane; c < C; c += 32) {
+                const float g = (expf(row[c] - lse) - (c == y ? 1.0f : 0.0f)) * invT;
+                dlogits[v * ld + c] = g;
+            }
+    }
+    if (lane == 0) sm[warp] = local;
+    if (n_correct && lane == 0 && correct) atomicAdd(n_correct, (unsigned long long)correct);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double t = 0.0;
+        for (int w = 0; w < LOSS_WARPS; ++w) t += sm[w];
+        part[blockIdx.x] = t;
+    }
+}
+
+__global__ void loss_final_kernel(int blocks, const double* __restrict__ part,
+                                  const unsigned long long* __restrict__ count, float* loss, int32_t* status) {
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    const unsigned long long T = *count;
+    if (T == 0) { *loss = 0.0f; atomicMax(status, DEV_EMPTY_MASK); return; }
+    double t = 0.0;
+    for (int b = 0; b < blocks; ++b) t += part[b];
+    *loss = (float)(t / (double)T);
+}
+
+constexpr int ADAM_MAX_TENSORS = 16;
+struct AdamBatch {
+    float* p[ADAM_MAX_TENSORS];
+    const float* g[ADAM_MAX_TENSORS];
+    float* m[ADAM_MAX_TENSORS];
+    float* v[ADAM_MAX_TENSORS];
+    int64_t numel[ADAM_MAX_TENSORS];
+    int count;
+    float lr, beta1, beta2, eps, inv_c1, inv_c2;
+};
+
+__global__ void adam_kernel(const AdamBatch b) {
+    const int t = blockIdx.y;
+    if (t >= b.count) return;
+    const int64_t nel = b.numel[t];
+    float* __restrict__ p = b.p[t]; const float* __restrict__ g = b.g[t];
+    float* __restrict__ m = b.m[t]; float* __restrict__ v = b.v[t];
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < nel; i += (int64_t)gridDim.x * blockDim.x) {
+        const float gi = g[i];
+        const float mi = b.beta1 * m[i] + (1.0f - b.beta1) * gi;
+        const float vi = b.beta2 * v[i] + (1.0f - b.beta2) * gi * gi;
+        m[i] = mi; v[i] = vi;
+        const float mhat = mi * b.inv_c1, vhat = vi * b.inv_c2;
+        p[i] = p[i] - b.lr * mhat / (sqrtf(vhat) + b.eps);
+    }
+}
+
+}  // namespace
+
+extern "C" mixgcn_status mixgcn_loss_softmax_xent(mixgcn_ctx* ctx, int64_t n, int32_t C, const float* logits,
+                                                  int64_t ld, const int32_t* labels, const uint8_t* train_mask,
+                                                  float* loss, float* dlogits, int32_t* pred, int64_t* n_correct,
+                                                  void* stream) {
+    if (!ctx || !logits || !labels || !train_mask || !loss) MIXGCN_FAIL(MIXGCN_EINVAL, "loss: null argument");
+    if (n <= 0 || C <= 0 || C > 4096) MIXGCN_FAIL(MIXGCN_EINVAL, "loss: need n > 0 and 1 <= C <= 4096 (n=%lld C=%d)", (long long)n, C);
+    if (ld < C) MIXGCN_FAIL(MIXGCN_EINVAL, "loss: ld (%lld) < C (%d)", (long long)ld, C);
+    MIXGCN_CUDA(cudaSetDevice(ctx->device));
+    cudaStream_t s = (cudaStream_t)stream;
+    int64_t blocks = (n + LOSS_WARPS - 1) / LOSS_WARPS;
+    const int64_t cap = (int64_t)ctx->sm_count * 16;
+    if (blocks > cap) blocks = cap;
+    // workspace: [count u64][pad][partials double[blocks]]
+    MIXGCN_TRY(mixgcn::ensure_workspace(ctx, 16 + blocks * (int64_t)sizeof(double)));
+    unsigned long long* count = reinterpret_cast<unsigned long long*>(ctx->workspace);
+    double* part = reinterpret_cast<double*>(reinterpret_cast<char*>(ctx->workspace) + 16);
+    MIXGCN_CUDA(cudaMemsetAsync(count, 0, sizeof(unsigned long long), s));
+    if (n_correct) MIXGCN_CUDA(cudaMemsetAsync(n_correct, 0, sizeof(int64_t), s));
+    {
+        LaunchScope scope(ctx, PH_LOSS, s);
+        int64_t cb = (n + 255) / 256; if (cb > cap) cb = cap;
+        count_mask_kernel<<<(unsigned)cb, 256, 0, s>>>(n, train_mask, count);
+    }
+    {
+        LaunchScope scope(ctx, PH_LOSS, s);
+        loss_rows_kernel<<<(unsigned)blocks, LOSS_WARPS * 32, 0, s>>>(
+            n, C, logits, ld, labels, train_mask, count, dlogits, pred,
+            reinterpret_cast<unsigned long long*>(n_correct), part, ctx->d_status);
+    }
+    {
+        LaunchScope scope(ctx, PH_LOSS, s);
+        loss_final_kernel<<<1, 32, 0, s>>>((int)blocks, part, count, loss, ctx->d_status);
+    }
+    MIXGCN_CUDA(cudaGetLastError());
+    return MIXGCN_OK;
+}
+
+extern "C" mixgcn_status mixgcn_adam_step(mixgcn_ctx* ctx, int32_t n_tensors, float* const* param,
+                                          const float* const* grad, float* const* m, float* const* v,
+                                          const int64_t* numel, int64_t t, float lr, float beta1, float beta2,
+                                          float eps, void* stream) {
+    if (!ctx || n_tensors < 0 || (n_tensors > 0 && (!param || !grad || !m || !v || !numel)))
+        MIXGCN_FAIL(MIXGCN_EINVAL, "adam: null argument");
+    if (t < 1) MIXGCN_FAIL(MIXGCN_EINVAL, "adam: step count t must be >= 1 (got %lld)", (long long)t);
+    for (int i = 0; i < n_tensors; ++i) {
+        if (numel[i] < 0 || (numel[i] > 0 && (!param[i] || !grad[i] || !m[i] || !v[i])))
+            MIXGCN_FAIL(MIXGCN_EINVAL, "adam: tensor %d has a null pointer or negative size", i);
+    }
+    MIXGCN_CUDA(cudaSetDevice(ctx->device));
+    cudaStream_t s = (cudaStream_t)stream;
+    const double c1 = 1.0 - pow((double)beta1, (double)t), c2 = 1.0 - pow((double)beta2, (double)t);
+    for (int base = 0; base < n_tensors; base += ADAM_MAX_TENSORS) {
+        AdamBatch b{};
+        int64_t mx = 0;
+        b.count = n_tensors - base < ADAM_MAX_TENSORS ? n_tensors - base : ADAM_MAX_TENSORS;
+        for (int i = 0; i < b.count; ++i) {
+            b.p[i] = param[base + i]; b.g[i] = grad[base + i]; b.m[i] = m[base + i]; b.v[i] = v[base + i];
+            b.numel[i] = numel[base + i];
+            if (b.numel[i] > mx) mx = b.numel[i];
+        }
+        if (mx == 0) continue;
+        b.lr = lr; b.beta1 = beta1; b.beta2 = beta2; b.eps = eps;
+        b.inv_c1 = (float)(1.0 / c1); b.inv_c2 = (float)(1.0 / c2);
+        int64_t bx = (mx + 255) / 256; if (bx > 1024) bx = 1024;
+        LaunchScope scope(ctx, PH_ADAM, s);
+        adam_kernel<<<dim3((unsigned)bx, (unsigned)b.count), 256, 0, s>>>(b);
+    }
+    MIXGCN_CUDA(cudaGetLastError());
+    return MIXGCN_OK;
+}

@@ -1,0 +1,113 @@
+"""Buffer plumbing for one full-graph GCN training iteration (the loop body of Algorithm 2).
+
+``GcnTrainer`` owns torch device buffers and calls the C-ABI in the order the algorithm
+gives -- for each layer aggregation+update (``layer_fwd``), then the loss, the backward pass
+(``layer_bwd``, last layer first) and the weight update (``adam_step``).  It performs no
+arithmetic itself: every value is produced by a kernel of ``libmixgcn.so``.
+"""
+from __future__ import annotations
+
+import torch
+
+from . import binding as mg
+
+
+def round4(x: int) -> int:
+    return (x + 3) // 4 * 4
+
+
+class GcnTrainer:
+    def __init__(self, ctx: mg.Ctx, graph: mg.Graph, dims, precision=mg.PREC_FP32, order=mg.ORDER_AUTO,
+                 n_chunks=0, fuse_gate=True, keep_scale=1.0, device=None):
+        self.ctx, self.g = ctx, graph
+        self.dims = tuple(int(d) for d in dims)
+        self.L = len(self.dims) - 1
+        self.n = graph.n
+        self.device = torch.device("cuda", ctx.device) if device is None else device
+        self.ld = [round4(d) for d in self.dims]
+        self.fuse_gate = fuse_gate
+        n, L = self.n, self.L
+        orders = order if isinstance(order, (list, tuple)) else [order] * L
+        self.descs, self.orders = [], []
+        for l in range(L):
+            flags = (mg.LAYER_RELU if l < L - 1 else 0) | (mg.LAYER_FIRST if l == 0 else 0)
+            if fuse_gate:
+                if l >= 1:
+                    flags |= mg.LAYER_GATE_GIN      # apply layer l-1's ReLU mask while producing G_in
+                if l < L - 1:
+                    flags |= mg.LAYER_GOUT_GATED    # ... so that layer l receives a gated G_out
+            d = mg.layer_desc(self.dims[l], self.dims[l + 1], self.ld[l], self.ld[l + 1], 4, orders[l], precision,
+                              flags, keep_scale if l < L - 1 else 1.0, keep_scale if l >= 1 else 1.0, n_chunks)
+            o, cols = mg.layer_plan(d)
+            d.ld_saved = round4(cols)
+            d.order = o
+            self.descs.append(d)
+            self.orders.append(o)
+        z = lambda r, c: torch.zeros((r, c), dtype=torch.float32, device=self.device)
+        self.X = [None] + [z(n, self.ld[l]) for l in range(1, L + 1)]
+        self.saved = [z(n, self.descs[l].ld_saved) for l in range(L)]
+        # gradient buffers: the logits' gradient is written over the logits; the input gradients of
+        # layers L-1, L-2, ... alternate between GA and GB (GB lives in the logits buffer when it fits)
+        self.G = [None] * (L + 1)
+        self.G[L] = self.X[L]
+        pool = []
+        if L >= 2:
+            wmax = max(self.ld[1:L])
+            pool.append(z(n, wmax))
+            if L >= 3:
+                if self.ld[L] >= wmax:
+                    pool.append(self.X[L])
+                else:
+                    pool.append(z(n, wmax))
+        for i, l in enumerate(range(L - 1, 0, -1)):
+            buf = pool[i % 2]
+            self.G[l] = buf.view(-1)[: n * self.ld[l]].view(n, self.ld[l])
+        self.loss = torch.zeros(1, dtype=torch.float32, device=self.device)
+        self.pred = torch.zeros(n, dtype=torch.int32, device=self.device)
+        self.n_correct = torch.zeros(1, dtype=torch.int64, device=self.device)
+        self.W = self.b = self.dW = self.db = None
+        self.masks = [None] * L
+
+    # -- parameters -----------------------------------------------------------------------------
+    def set_params(self, Ws, bs):
+        dev = self.device
+        self.W = [w.to(dev, torch.float32).contiguous().clone() for w in Ws]
+        self.b = [b.to(dev, torch.float32).contiguous().clone() for b in bs]
+        self.dW = [torch.zeros_like(w) for w in self.W]
+        self.db = [torch.zeros_like(b) for b in self.b]
+        self.mW = [torch.zeros_like(w) for w in self.W]
+        self.vW = [torch.zeros_like(w) for w in self.W]
+        self.mb = [torch.zeros_like(b) for b in self.b]
+        self.vb = [torch.zeros_like(b) for b in self.b]
+
+    def set_inputs(self, X0, labels, train_mask, drop_masks=None):
+        """X0: n x ld[0] device tensor (row-major, pads zero); labels int32; train_mask uint8."""
+        assert X0.shape == (self.n, self.ld[0]) and X0.stride(1) == 1
+        self.X[0], self.labels, self.train_mask = X0, labels, train_mask
+        if drop_masks is not None:
+            self.masks = list(drop_masks) + [None] * (self.L - len(drop_masks))
+
+    # -- the iteration --------------------------------------------------------------------------
+    def forward(self):
+        for l in range(self.L):
+            mg.layer_fwd(self.ctx, self.g, self.descs[l], self.X[l], self.W[l], self.b[l], self.masks[l],
+                         self.saved[l], self.X[l + 1])
+
+    def compute_loss(self):
+        mg.loss_softmax_xent(self.ctx, self.X[self.L], self.labels, self.train_mask, self.loss,
+                             dlogits=self.X[self.L], pred=self.pred, n_correct=self.n_correct, C_=self.dims[-1])
+
+    def backward(self):
+        for l in range(self.L - 1, -1, -1):
+            mg.layer_bwd(self.ctx, self.g, self.descs[l], self.X[l], self.saved[l], self.X[l + 1], self.masks[l],
+                         self.W[l], self.G[l + 1], self.G[l] if l > 0 else None, self.dW[l], self.db[l])
+
+    def step(self, t, lr=0.01, beta1=0.9, beta2=0.999, eps=1e-8):
+        mg.adam_step(self.ctx, self.W + self.b, self.dW + self.db, self.mW + self.mb, self.vW + self.vb, t,
+                     lr, beta1, beta2, eps)
+
+    def epoch(self, t, lr=0.01):
+        self.forward()
+        self.compute_loss()
+        self.backward()
+        self.step(t, lr)

@@ -1,0 +1,474 @@
+"""Parity of the CUDA path (through the C-ABI) with the CPU oracle, element by element, on the
+same seeded inputs.  Integer / index work must be bit-exact; fp32 results must agree with the
+fp64 oracle within TOL_FP32 relative Frobenius error."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from helpers import ADAM, TOL_FP32, host, padded, rel_fro, round4
+from oracle import gcn_oracle as orc
+from paper_2501_01951_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def mg():
+    from paper_2501_01951_b200 import build
+    build.build()
+    from paper_2501_01951_b200 import binding
+    return binding
+
+
+@pytest.fixture(scope="module")
+def ctx(mg):
+    c = mg.ctx_create(0)
+    yield c
+    assert mg.ctx_poll_status(c, raise_on_error=False) == 0
+    c.close()
+
+
+def i32(a):
+    return torch.tensor(np.asarray(a), dtype=torch.int32)
+
+
+def messy_edges(n, m, seed):
+    """Edge list with duplicates, both orientations, self-loops and isolated nodes."""
+    rng = np.random.default_rng(seed)
+    hi = max(1, (3 * n) // 4)                  # leave the top quarter of ids isolated
+    src, dst = rng.integers(0, hi, m), rng.integers(0, hi, m)
+    src[: m // 10] = dst[: m // 10]            # self-loops
+    src = np.concatenate([src, src[: m // 5]])
+    dst = np.concatenate([dst, dst[: m // 5]])  # duplicates
+    return src.astype(np.int32), dst.astype(np.int32)
+
+
+def star_plus(n, hub_deg, seed):
+    """A hub of degree hub_deg (forces the CTA-per-row path) plus random edges."""
+    rng = np.random.default_rng(seed)
+    s = np.concatenate([np.zeros(hub_deg, np.int64), rng.integers(0, n, 3 * n)])
+    d = np.concatenate([np.arange(1, hub_deg + 1), rng.integers(0, n, 3 * n)])
+    return s.astype(np.int32), d.astype(np.int32)
+
+
+GRAPHS = {
+    "messy-sym": lambda: (300, *messy_edges(300, 2000, 1), True),
+    "messy-directed": lambda: (257, *messy_edges(257, 1500, 2), False),
+    "single-node": lambda: (1, np.zeros(0, np.int32), np.zeros(0, np.int32), True),
+    "edgeless": lambda: (40, np.zeros(0, np.int32), np.zeros(0, np.int32), True),
+    "hub": lambda: (9000, *star_plus(9000, 6000, 3), True),
+    "hub-directed": lambda: (9000, *star_plus(9000, 6000, 4), False),
+}
+
+
+def build_both(mg, ctx, name):
+    n, s, d, sym = GRAPHS[name]()
+    flags_o = orc.ADD_SELF_LOOPS | (orc.SYMMETRISE if sym else 0)
+    flags_g = mg.GRAPH_ADD_SELF_LOOPS | (mg.GRAPH_SYMMETRISE if sym else 0)
+    go = orc.graph_build(n, s, d, flags_o)
+    gg = mg.graph_create(ctx, n, i32(s), i32(d), flags_g)
+    return go, gg
+
+
+# --------------------------------------------------------------------------- S0 graph build
+
+@pytest.mark.parametrize("name", list(GRAPHS))
+@pytest.mark.parametrize("on_device", [False, True])
+def test_graph_build_bit_exact(mg, ctx, name, on_device):
+    n, s, d, sym = GRAPHS[name]()
+    go = orc.graph_build(n, s, d, orc.ADD_SELF_LOOPS | (orc.SYMMETRISE if sym else 0))
+    ts, td = i32(s), i32(d)
+    if on_device:
+        ts, td = ts.cuda(), td.cuda()
+    gg = mg.graph_create(ctx, n, ts, td, mg.GRAPH_ADD_SELF_LOOPS | (mg.GRAPH_SYMMETRISE if sym else 0))
+    assert (gg.n, gg.nnz) == (go.n, go.nnz)
+    assert gg.max_deg == int(go.deg.max())
+    e = mg.graph_export(gg)
+    assert np.array_equal(e["rowptr"].numpy(), go.rowptr)
+    assert np.array_equal(e["col"].numpy(), go.col)
+    assert np.array_equal(e["deg"].numpy(), go.deg)
+    assert e["dinv"].numpy().tobytes() == go.dinv32.tobytes()
+    assert e["val"].numpy().tobytes() == go.val32.tobytes()
+    et = mg.graph_export(gg, transposed=True)
+    assert np.array_equal(et["rowptr"].numpy(), go.rowptr_t)
+    assert np.array_equal(et["col"].numpy(), go.col_t)
+    assert et["val"].numpy().tobytes() == go.val32[go.src_index_t].tobytes()
+    is_sym = np.array_equal(go.rowptr, go.rowptr_t) and np.array_equal(go.col, go.col_t)
+    assert gg.symmetric == is_sym
+    # schedule: a permutation, by descending entry count, ties by ascending id
+    perm = mg.graph_export_schedule(gg).numpy().astype(np.int64)
+    assert np.array_equal(np.sort(perm), np.arange(n))
+    key = (-go.deg[perm].astype(np.int64)) * (n + 1) + perm
+    assert np.all(np.diff(key) > 0)
+
+
+def test_graph_closed_forms(mg, ctx):
+    n = 33
+    s, d = np.triu_indices(n, 1)
+    e = mg.graph_export(mg.graph_create(ctx, n, i32(s), i32(d)))
+    assert int(e["rowptr"][-1]) == n * n
+    np.testing.assert_allclose(e["val"].numpy(), 1.0 / n, rtol=2e-7)          # complete graph: J/n
+    r = np.arange(n)
+    e = mg.graph_export(mg.graph_create(ctx, n, i32(r), i32((r + 1) % n)))
+    assert int(e["rowptr"][-1]) == 3 * n
+    np.testing.assert_allclose(e["val"].numpy(), 1.0 / 3.0, rtol=2e-7)        # 2-regular
+    e = mg.graph_export(mg.graph_create(ctx, n, i32([]), i32([])))
+    assert np.array_equal(e["col"].numpy(), r) and np.all(e["val"].numpy() == 1.0)   # A_hat = I
+
+
+def test_graph_tiny_workload_matches_oracle(mg, ctx):
+    wl = synth.CONFIGS["C1"]
+    s, d = synth.rmat_graph(wl.n, wl.undirected_edges, wl.seed("graph"))
+    go = orc.graph_build(wl.n, s.numpy(), d.numpy())
+    gg = mg.graph_create(ctx, wl.n, s.cuda(), d.cuda())
+    e = mg.graph_export(gg)
+    assert np.array_equal(e["rowptr"].numpy(), go.rowptr) and np.array_equal(e["col"].numpy(), go.col)
+    assert e["val"].numpy().tobytes() == go.val32.tobytes()
+    assert gg.symmetric
+
+
+def test_graph_from_csr_and_validation(mg, ctx):
+    go, _ = build_both(mg, ctx, "messy-directed")
+    for dev in ("cpu", "cuda"):
+        gg = mg.graph_create_from_csr(ctx, go.n, torch.tensor(go.rowptr).to(dev), torch.tensor(go.col).to(dev))
+        e = mg.graph_export(gg)
+        assert e["val"].numpy().tobytes() == go.val32.tobytes()
+        et = mg.graph_export(gg, transposed=True)
+        assert np.array_equal(et["col"].numpy(), go.col_t)
+    rp = torch.tensor([0, 2, 3], dtype=torch.int64)
+    for col in ([1, 0, 1], [0, 0, 1], [0, 5, 1]):                     # unsorted, duplicate, out of range
+        with pytest.raises(mg.MixgcnError) as ex:
+            mg.graph_create_from_csr(ctx, 2, rp, i32(col))
+        assert ex.value.status == mg.EBADGRAPH
+    with pytest.raises(mg.MixgcnError) as ex:
+        mg.graph_create_from_csr(ctx, 2, torch.tensor([0, 3, 2], dtype=torch.int64), i32([0, 1, 1]))
+    assert ex.value.status == mg.EBADGRAPH
+    with pytest.raises(mg.MixgcnError) as ex:
+        mg.graph_create(ctx, 4, i32([0, 7]), i32([1, 2]))
+    assert ex.value.status == mg.EBADGRAPH
+    with pytest.raises(mg.MixgcnError) as ex:
+        mg.graph_create(ctx, 0, i32([]), i32([]))
+    assert ex.value.status == mg.EINVAL
+
+
+# --------------------------------------------------------------------------- S1 / S5 aggregation
+
+WIDTHS = [1, 3, 4, 8, 41, 47, 64, 100, 128, 172, 256, 602, 1024, 1100]
+
+
+@pytest.mark.parametrize("name", ["messy-sym", "messy-directed", "hub", "hub-directed", "edgeless"])
+@pytest.mark.parametrize("w", WIDTHS)
+def test_spmm_matches_oracle(mg, ctx, name, w):
+    if name.startswith("hub") and w in (3, 47, 100, 602, 1100):
+        pytest.skip("hub graphs cover a subset of widths")
+    go, gg = build_both(mg, ctx, name)
+    X = synth.uniform_tensor((go.n, w), seed=w + 11, lo=-2, hi=2)
+    Y = padded(X, fill=float("nan"))                       # pad columns must never reach the result
+    for transposed in (False, True):
+        Z = torch.full((go.n, round4(w) + 4), 7.0, device="cuda")[:, : round4(w) + 4]
+        mg.spmm(ctx, gg, Y, Z, w, transposed=transposed)
+        want = orc.aggregate(go, X.numpy(), transposed=transposed)
+        assert rel_fro(host(Z, w), want) <= TOL_FP32
+        assert torch.all(Z[:, w:round4(w)] == 0) and torch.all(Z[:, round4(w):] == 7.0)
+
+
+def test_spmm_closed_forms_and_determinism(mg, ctx):
+    n = 64
+    s, d = np.triu_indices(n, 1)
+    gg = mg.graph_create(ctx, n, i32(s), i32(d))
+    X = synth.normal_features(n, 20, 5)
+    Y, Z = padded(X), torch.zeros(n, 20, device="cuda")
+    mg.spmm(ctx, gg, Y, Z, 20)
+    np.testing.assert_allclose(host(Z), np.tile(X.numpy().astype(np.float64).mean(0), (n, 1)), rtol=1e-5, atol=1e-6)
+    # symmetric graph: sqrt(deg~) is a fixed point of the aggregation
+    wl = synth.CONFIGS["C1"]
+    s, d = synth.rmat_graph(wl.n, wl.undirected_edges, wl.seed("graph"))
+    gg = mg.graph_create(ctx, wl.n, s, d)
+    deg = mg.graph_export(gg)["deg"].float()
+    R = padded(torch.sqrt(deg)[:, None].repeat(1, 4))
+    Z = torch.zeros_like(R)
+    mg.spmm(ctx, gg, R, Z, 4)
+    assert rel_fro(host(Z), host(R)) <= 1e-6
+    X = padded(synth.normal_features(wl.n, 64, 6))
+    Z1, Z2 = torch.zeros_like(X), torch.zeros_like(X)
+    mg.spmm(ctx, gg, X, Z1, 64)
+    mg.spmm(ctx, gg, X, Z2, 64)
+    assert torch.equal(Z1, Z2)                                     # bitwise reproducible
+
+
+def test_spmm_epilogue(mg, ctx):
+    go, gg = build_both(mg, ctx, "messy-directed")
+    n, w = go.n, 41
+    X = synth.uniform_tensor((n, w), 21, -1, 1)
+    bias = synth.uniform_tensor((w,), 22, -0.5, 0.5)
+    drop = (synth.uniform_tensor((n, w), 23, 0, 1) < 0.7).to(torch.uint8)
+    gate = synth.uniform_tensor((n, w), 24, -1, 1)
+    Z = torch.zeros(n, round4(w), device="cuda")
+    epi = mg.make_epilogue(bias=bias.cuda(), relu=True, drop_mask=drop.cuda(), keep_scale=1 / 0.7,
+                           gate=padded(gate), gate_scale=1.5)
+    mg.spmm(ctx, gg, padded(X), Z, w, epi=epi)
+    P = orc.aggregate(go, X.numpy()) + bias.numpy().astype(np.float64)
+    want = orc.activation(P, True, drop.numpy(), 1 / 0.7) * np.where(gate.numpy() > 0, 1.5, 0.0)
+    assert rel_fro(host(Z, w), want) <= TOL_FP32
+
+
+# --------------------------------------------------------------------------- S2 / S4 dense update
+
+GEMM_SHAPES = [  # M, N, K
+    (1, 1, 1), (5, 3, 2), (130, 70, 33), (257, 41, 602), (300, 256, 100), (1000, 172, 128), (129, 129, 129),
+]
+
+
+@pytest.mark.parametrize("M,N,K", GEMM_SHAPES)
+@pytest.mark.parametrize("ta,tb", [(False, False), (False, True), (True, False), (True, True)])
+def test_gemm_fp32_matches_oracle(mg, ctx, M, N, K, ta, tb):
+    A = synth.uniform_tensor((K, M) if ta else (M, K), 31 + M, -1, 1)
+    B = synth.uniform_tensor((N, K) if tb else (K, N), 32 + N, -1, 1)
+    Cd = torch.full((M, round4(N) + 4), 3.0, device="cuda")
+    mg.gemm(ctx, mg.PREC_FP32, ta, tb, M, N, K, padded(A, fill=float("nan")), padded(B, fill=float("nan")), Cd)
+    Ao = A.numpy().astype(np.float64).T if ta else A.numpy().astype(np.float64)
+    Bo = B.numpy().astype(np.float64).T if tb else B.numpy().astype(np.float64)
+    want = orc.update(Ao, Bo)
+    assert rel_fro(host(Cd, N), want) <= TOL_FP32
+    assert torch.all(Cd[:, round4(N):] == 3.0)
+
+
+def test_gemm_unaligned_weight_matrix(mg, ctx):
+    """W is dense d_in x d_out with d_out % 4 != 0: its rows are not 16-byte aligned."""
+    M, N, K = 200, 41, 100
+    A, W = synth.uniform_tensor((M, K), 1, -1, 1), synth.uniform_tensor((K, N), 2, -1, 1)
+    Cd = torch.zeros(M, round4(N), device="cuda")
+    mg.gemm(ctx, mg.PREC_FP32, False, False, M, N, K, padded(A), W.cuda(), Cd)
+    assert rel_fro(host(Cd, N), orc.update(A.numpy(), W.numpy())) <= TOL_FP32
+    dW = torch.zeros(K, N, device="cuda")
+    G = synth.uniform_tensor((M, N), 3, -1, 1)
+    mg.gemm(ctx, mg.PREC_FP32, True, False, K, N, M, padded(A), padded(G), dW)
+    assert rel_fro(host(dW), A.numpy().astype(np.float64).T @ G.numpy().astype(np.float64)) <= TOL_FP32
+
+
+def test_gemm_long_reduction_split_k(mg, ctx):
+    """Weight-gradient shape: K = number of nodes, split over CTAs, fixed-order reduction."""
+    M, N, K = 100, 47, 70001
+    A, B = synth.normal_features(K, M, 41), synth.normal_features(K, N, 42)
+    Cd1, Cd2 = torch.zeros(M, round4(N), device="cuda"), torch.zeros(M, round4(N), device="cuda")
+    mg.gemm(ctx, mg.PREC_FP32, True, False, M, N, K, padded(A), padded(B), Cd1)
+    mg.gemm(ctx, mg.PREC_FP32, True, False, M, N, K, padded(A), padded(B), Cd2)
+    want = A.numpy().astype(np.float64).T @ B.numpy().astype(np.float64)
+    assert rel_fro(host(Cd1, N), want) <= TOL_FP32
+    assert torch.equal(Cd1, Cd2)
+
+
+def test_gemm_epilogue(mg, ctx):
+    M, N, K = 150, 70, 50
+    A, B = synth.uniform_tensor((M, K), 51, -1, 1), synth.uniform_tensor((K, N), 52, -1, 1)
+    bias = synth.uniform_tensor((N,), 53, -1, 1)
+    drop = (synth.uniform_tensor((M, N), 54, 0, 1) < 0.5).to(torch.uint8)
+    Cd = torch.zeros(M, round4(N), device="cuda")
+    epi = mg.make_epilogue(bias=bias.cuda(), relu=True, drop_mask=drop.cuda(), keep_scale=2.0)
+    mg.gemm(ctx, mg.PREC_FP32, False, False, M, N, K, padded(A), padded(B), Cd, epi=epi)
+    want = orc.activation(orc.update(A.numpy(), B.numpy(), bias.numpy()), True, drop.numpy(), 2.0)
+    assert rel_fro(host(Cd, N), want) <= TOL_FP32
+
+
+# --------------------------------------------------------------------------- S3 loss
+
+@pytest.mark.parametrize("Cc", [1, 8, 41, 47, 64, 172, 1000])
+def test_loss_matches_oracle(mg, ctx, Cc):
+    n = 777
+    P = synth.uniform_tensor((n, Cc), 60 + Cc, -6, 6)
+    labels = synth.uniform_labels(n, Cc, 61)
+    mask = synth.bernoulli_mask(n, 0.4, 62)
+    lo, G, pred, nc, T = orc.loss(P.numpy(), labels.numpy(), mask.numpy())
+    Pd = padded(P)
+    loss = torch.zeros(1, device="cuda"); Gd = torch.full_like(Pd, 9.0)
+    predd = torch.zeros(n, dtype=torch.int32, device="cuda"); ncd = torch.zeros(1, dtype=torch.int64, device="cuda")
+    mg.loss_softmax_xent(ctx, Pd, labels.cuda(), mask.cuda(), loss, Gd, predd, ncd, C_=Cc)
+    assert abs(loss.item() - lo) <= 1e-6 * max(1.0, abs(lo))
+    assert rel_fro(host(Gd, Cc), G) <= TOL_FP32
+    assert np.array_equal(predd.cpu().numpy(), pred) and ncd.item() == nc         # arg-max: bit-exact
+    assert torch.all(Gd[mask.cuda() == 0, :Cc] == 0)
+    # in place over the logits
+    P2 = Pd.clone()
+    mg.loss_softmax_xent(ctx, P2, labels.cuda(), mask.cuda(), loss, P2, None, None, C_=Cc)
+    assert torch.equal(P2[:, :Cc], Gd[:, :Cc])
+
+
+def test_loss_closed_form_and_ties(mg, ctx):
+    n, Cc = 50, 41
+    labels = synth.uniform_labels(n, Cc, 1).cuda()
+    mask = torch.ones(n, dtype=torch.uint8, device="cuda")
+    loss = torch.zeros(1, device="cuda"); pred = torch.ones(n, dtype=torch.int32, device="cuda")
+    mg.loss_softmax_xent(ctx, torch.zeros(n, round4(Cc), device="cuda"), labels, mask, loss, None, pred, None, C_=Cc)
+    assert abs(loss.item() - math.log(Cc)) < 1e-6 and torch.all(pred == 0)
+
+
+def test_loss_device_side_errors_set_the_status_word(mg, ctx):
+    n, Cc = 20, 5
+    P = torch.zeros(n, 8, device="cuda"); loss = torch.ones(1, device="cuda"); G = torch.ones(n, 8, device="cuda")
+    labels = torch.zeros(n, dtype=torch.int32, device="cuda")
+    mg.loss_softmax_xent(ctx, P, labels, torch.zeros(n, dtype=torch.uint8, device="cuda"), loss, G, None, None, C_=Cc)
+    with pytest.raises(mg.MixgcnError) as e:
+        mg.ctx_poll_status(ctx)
+    assert e.value.status == mg.EDEVICE and loss.item() == 0 and torch.all(G[:, :Cc] == 0)
+    labels[3] = 9
+    mg.loss_softmax_xent(ctx, P, labels, torch.ones(n, dtype=torch.uint8, device="cuda"), loss, G, None, None, C_=Cc)
+    assert mg.ctx_poll_status(ctx, raise_on_error=False) == 2
+    assert mg.ctx_poll_status(ctx, raise_on_error=False) == 0      # cleared by the read
+
+
+# --------------------------------------------------------------------------- S6 Adam
+
+def test_adam_matches_oracle(mg, ctx):
+    shapes = [(64, 32), (32,), (1024, 100), (7,)] + [(3, 5)] * 20        # > one batch of tensors
+    P = [synth.uniform_tensor(s, 70 + i, -1, 1) for i, s in enumerate(shapes)]
+    pd = [p.cuda() for p in P]
+    md = [torch.zeros_like(p) for p in pd]; vd = [torch.zeros_like(p) for p in pd]
+    po = [p.numpy().astype(np.float64) for p in P]
+    mo = [np.zeros_like(p) for p in po]; vo = [np.zeros_like(p) for p in po]
+    for t in range(1, 5):
+        Gs = [synth.uniform_tensor(s, 100 * t + i, -1e-2, 1e-2) for i, s in enumerate(shapes)]
+        mg.adam_step(ctx, pd, [g.cuda() for g in Gs], md, vd, t, **ADAM)
+        for i in range(len(shapes)):
+            po[i], mo[i], vo[i] = orc.adam(po[i], Gs[i].numpy(), mo[i], vo[i], t, **ADAM)
+    for i in range(len(shapes)):
+        assert rel_fro(pd[i].cpu().numpy(), po[i]) <= 1e-6
+        assert rel_fro(md[i].cpu().numpy(), mo[i]) <= 1e-6 and rel_fro(vd[i].cpu().numpy(), vo[i]) <= 1e-6
+
+
+# --------------------------------------------------------------------------- layers and whole epochs
+
+def _run_layer(mg, ctx, go, gg, d_in, d_out, order, relu, first, use_drop, n_chunks, seed):
+    n = go.n
+    X = synth.uniform_tensor((n, d_in), seed, -1, 1)
+    W = synth.glorot_uniform(d_in, d_out, seed + 1)
+    b = synth.uniform_tensor((d_out,), seed + 2, -0.2, 0.2)
+    Gout = synth.uniform_tensor((n, d_out), seed + 3, -1, 1)
+    drop = (synth.uniform_tensor((n, d_out), seed + 4, 0, 1) < 0.6).to(torch.uint8) if use_drop else None
+    ks = 1 / 0.6 if use_drop else 1.0
+    flags = (mg.LAYER_RELU if relu else 0) | (mg.LAYER_FIRST if first else 0)
+    desc = mg.layer_desc(d_in, d_out, round4(d_in), round4(d_out), round4(max(d_in, d_out)), order, mg.PREC_FP32,
+                         flags, ks, 1.0, n_chunks)
+    Xd, Wd, bd = padded(X), W.cuda(), b.cuda()
+    dropd = None if drop is None else drop.cuda()
+    saved = torch.zeros(n, round4(max(d_in, d_out)), device="cuda")
+    Xout = torch.zeros(n, round4(d_out), device="cuda")
+    mg.layer_fwd(ctx, gg, desc, Xd, Wd, bd, dropd, saved, Xout)
+    Z = orc.aggregate(go, X.numpy())
+    Pp = orc.update(Z, W.numpy(), b.numpy())
+    want = orc.activation(Pp, relu, None if drop is None else drop.numpy(), ks)
+    assert rel_fro(host(Xout, d_out), want) <= TOL_FP32
+    Gd = padded(Gout)
+    Gin = None if first else torch.zeros(n, round4(d_in), device="cuda")
+    dW = torch.zeros(d_in, d_out, device="cuda"); db = torch.zeros(d_out, device="cuda")
+    mg.layer_bwd(ctx, gg, desc, Xd, saved, Xout, dropd, Wd, Gd, Gin, dW, db)
+    _, dWo, dbo, dZo = orc.update_bwd(Z, Pp, W.numpy(), Gout.numpy(), relu, None if drop is None else drop.numpy(),
+                                      ks, need_dZ=not first)
+    assert rel_fro(host(dW), dWo) <= TOL_FP32 and rel_fro(db.cpu().numpy(), dbo) <= TOL_FP32
+    if not first:
+        assert rel_fro(host(Gin, d_in), orc.aggregate(go, dZo, transposed=True)) <= TOL_FP32
+
+
+@pytest.mark.parametrize("name", ["messy-sym", "messy-directed"])
+@pytest.mark.parametrize("order", ["agg", "upd"])
+@pytest.mark.parametrize("d_in,d_out", [(64, 32), (33, 41), (8, 100)])
+def test_layer_fwd_bwd_both_orders(mg, ctx, name, order, d_in, d_out):
+    go, gg = build_both(mg, ctx, name)
+    o = mg.ORDER_AGG_FIRST if order == "agg" else mg.ORDER_UPD_FIRST
+    _run_layer(mg, ctx, go, gg, d_in, d_out, o, relu=True, first=False, use_drop=True, n_chunks=0, seed=80)
+    _run_layer(mg, ctx, go, gg, d_in, d_out, o, relu=False, first=True, use_drop=False, n_chunks=0, seed=90)
+
+
+@pytest.mark.parametrize("n_chunks", [2, 3, 7])
+def test_layer_chunked_pipeline_matches_unchunked(mg, ctx, n_chunks):
+    go, gg = build_both(mg, ctx, "hub")
+    _run_layer(mg, ctx, go, gg, 64, 48, mg.ORDER_AGG_FIRST, relu=True, first=False, use_drop=True,
+               n_chunks=n_chunks, seed=95)
+
+
+def _tiny_problem():
+    wl = synth.CONFIGS["C1"]
+    s, d = synth.rmat_graph(wl.n, wl.undirected_edges, wl.seed("graph"))
+    X = synth.normal_features(wl.n, wl.dims[0], wl.seed("features"))
+    y = synth.uniform_labels(wl.n, wl.classes, wl.seed("labels"))
+    m = synth.bernoulli_mask(wl.n, wl.mask_p, wl.seed("mask"))
+    Ws, bs = synth.make_weights(wl)
+    return wl, s, d, X, y, m, Ws, bs
+
+
+@pytest.mark.parametrize("order", ["auto", "agg", "upd"])
+@pytest.mark.parametrize("fuse_gate", [True, False])
+def test_training_epochs_match_oracle_on_tiny(mg, ctx, order, fuse_gate):
+    from paper_2501_01951_b200.train import GcnTrainer
+    wl, s, d, X, y, m, Ws, bs = _tiny_problem()
+    go = orc.graph_build(wl.n, s.numpy(), d.numpy())
+    gg = mg.graph_create(ctx, wl.n, s, d)
+    o = {"auto": mg.ORDER_AUTO, "agg": mg.ORDER_AGG_FIRST, "upd": mg.ORDER_UPD_FIRST}[order]
+    tr = GcnTrainer(ctx, gg, wl.dims, mg.PREC_FP32, order=o, fuse_gate=fuse_gate)
+    if order == "auto":
+        assert tr.orders == [mg.ORDER_AGG_FIRST, mg.ORDER_UPD_FIRST]
+    tr.set_params(Ws, bs)
+    tr.set_inputs(padded(X), y.cuda(), m.cuda())
+    Wo, bo, state = [w.numpy() for w in Ws], [b.numpy() for b in bs], None
+    for t in range(1, 4):
+        tr.forward()
+        logits = host(tr.X[-1], wl.classes).copy()
+        tr.compute_loss(); tr.backward(); tr.step(t, **ADAM)
+        ref = orc.train_epoch(go, X.numpy(), Wo, bo, y.numpy(), m.numpy(), state, t, **ADAM)
+        assert rel_fro(logits, ref["logits"]) <= TOL_FP32
+        assert abs(tr.loss.item() - ref["loss"]) <= 1e-5 * abs(ref["loss"])
+        # arg-max must agree wherever the oracle's top-2 gap is not a near-tie
+        top2 = np.sort(ref["logits"], axis=1)[:, -2:]
+        clear = (top2[:, 1] - top2[:, 0]) > 1e-4 * np.abs(ref["logits"]).max()
+        assert np.array_equal(tr.pred.cpu().numpy()[clear], ref["pred"][clear])
+        for l in range(tr.L):
+            assert rel_fro(tr.dW[l].cpu().numpy(), ref["dW"][l]) <= TOL_FP32
+            assert rel_fro(tr.db[l].cpu().numpy(), ref["db"][l]) <= TOL_FP32
+            # Adam turns g into ~sign(g) when |g| is tiny: compare the update where g is not negligible
+            gmax = np.abs(ref["dW"][l]).max()
+            big = np.abs(ref["dW"][l]) > 1e-4 * gmax
+            dgpu = tr.W[l].cpu().numpy().astype(np.float64) - Wo[l]
+            dref = ref["W"][l] - Wo[l]
+            assert rel_fro(dgpu[big], dref[big]) <= 1e-3
+        # continue both sides from the oracle's weights so that one side's rounding does not compound
+        Wo, bo, state = ref["W"], ref["b"], ref["state"]
+        tr.W = [torch.tensor(w, dtype=torch.float32, device="cuda") for w in Wo]
+        tr.b = [torch.tensor(b, dtype=torch.float32, device="cuda") for b in bo]
+        for l in range(tr.L):
+            tr.mW[l].copy_(torch.tensor(state["mW"][l])); tr.vW[l].copy_(torch.tensor(state["vW"][l]))
+            tr.mb[l].copy_(torch.tensor(state["mb"][l])); tr.vb[l].copy_(torch.tensor(state["vb"][l]))
+
+
+def test_epoch_is_bitwise_deterministic(mg, ctx):
+    from paper_2501_01951_b200.train import GcnTrainer
+    wl, s, d, X, y, m, Ws, bs = _tiny_problem()
+    gg = mg.graph_create(ctx, wl.n, s, d)
+    outs = []
+    for _ in range(2):
+        tr = GcnTrainer(ctx, gg, wl.dims, mg.PREC_FP32)
+        tr.set_params(Ws, bs)
+        tr.set_inputs(padded(X), y.cuda(), m.cuda())
+        for t in range(1, 3):
+            tr.epoch(t)
+        outs.append([w.clone() for w in tr.W] + [tr.loss.clone()])
+    for a, b in zip(*outs):
+        assert torch.equal(a, b)
+
+
+def test_argument_errors(mg, ctx):
+    go, gg = build_both(mg, ctx, "messy-sym")
+    n = go.n
+    Y, Z = torch.zeros(n, 8, device="cuda"), torch.zeros(n, 8, device="cuda")
+    with pytest.raises(mg.MixgcnError) as e:
+        mg.spmm(ctx, gg, Y, Z, 0)
+    assert e.value.status == mg.EINVAL
+    with pytest.raises(mg.MixgcnError):
+        mg.spmm(ctx, gg, Y, Y, 8)                                   # overlap
+    with pytest.raises(mg.MixgcnError):
+        mg.spmm(ctx, gg, Y, Z, 12)                                  # ld < w
+    with pytest.raises(mg.MixgcnError):
+        mg.spmm(ctx, gg, torch.zeros(n, 9, device="cuda")[:, :6], Z, 6)   # ld % 4 != 0
+    with pytest.raises(mg.MixgcnError):
+        mg.adam_step(ctx, [Y], [Y], [Y], [Y], 0)                    # t < 1
+    assert torch.all(Z == 0)                                         # outputs untouched on host-side errors
