@@ -130,6 +130,7 @@ extern "C" mixgcn_status mixgcn_ctx_destroy(mixgcn_ctx* ctx) {
     for (int i = 0; i < 2; ++i) { if (ctx->join_ev[i]) cudaEventDestroy(ctx->join_ev[i]); if (ctx->side_stream[i]) cudaStreamDestroy(ctx->side_stream[i]); }
     if (ctx->fork_ev) cudaEventDestroy(ctx->fork_ev);
     cudaFree(ctx->workspace);
+    cudaFree(ctx->arena);
     cudaFree(ctx->d_status);
     delete ctx;
     return MIXGCN_OK;
@@ -339,17 +340,4 @@ extern "C" mixgcn_status mixgcn_layer_bwd(mixgcn_ctx* ctx, const mixgcn_graph* g
         MIXGCN_TRY(launch_gemm(ctx, d->precision, 0, 1, n, d->d_in, d->d_out, saved, d->ld_saved, W, ldw, G_in, d->ld_in,
                                gin, 0, s));
     return MIXGCN_OK;
-}
-
-extern "C" mixgcn_status mixgcn_train_step_host(mixgcn_ctx* ctx, const mixgcn_graph* g, int32_t L,
-                                                const int32_t* dims, int32_t precision, const float* X,
-                                                const int32_t* labels, const uint8_t* train_mask,
-                                                float* const* W, float* const* b, float* const* mW,
-                                                float* const* vW, float* const* mb, float* const* vb,
-                                                int64_t t, float lr, float beta1, float beta2, float eps,
-                                                float* loss, int32_t* pred) {
-    (void)ctx; (void)g; (void)L; (void)dims; (void)precision; (void)X; (void)labels; (void)train_mask;
-    (void)W; (void)b; (void)mW; (void)vW; (void)mb; (void)vb; (void)t; (void)lr; (void)beta1; (void)beta2;
-    (void)eps; (void)loss; (void)pred;
-    MIXGCN_FAIL(MIXGCN_EUNSUPPORTED, "train_step_host: not built yet");
 }

@@ -1,0 +1,146 @@
+// One whole training iteration (the loop body of Algorithm 2) with host inputs and outputs:
+// host -> device copies, all layers forward, loss, backward, Adam, device -> host copies.
+// Device buffers come from an arena the context keeps between calls.
+#include <vector>
+
+#include "internal.cuh"
+
+using namespace mixgcn;
+
+namespace {
+
+inline int64_t round4(int64_t x) { return (x + 3) / 4 * 4; }
+
+struct Carver {
+    char* base; int64_t off = 0;
+    template <class T> T* take(int64_t count) {
+        T* p = base ? reinterpret_cast<T*>(base + off) : nullptr;
+        off += ((count * (int64_t)sizeof(T)) + 255) & ~(int64_t)255;
+        return p;
+    }
+};
+
+struct StepLayout {
+    std::vector<float*> X, saved, G, W, b, dW, db, mW, vW, mb, vb;
+    int32_t* labels; uint8_t* mask; float* loss; int32_t* pred;
+    std::vector<mixgcn_layer_desc> desc;
+    int64_t bytes;
+};
+
+// Pass base == nullptr to size the arena.
+mixgcn_status lay_out(char* base, int64_t n, int L, const int32_t* dims, int precision, StepLayout& lo) {
+    Carver c{base};
+    lo.desc.resize(L);
+    std::vector<int64_t> ld(L + 1);
+    for (int l = 0; l <= L; ++l) ld[l] = round4(dims[l]);
+    for (int l = 0; l < L; ++l) {
+        mixgcn_layer_desc& d = lo.desc[l];
+        d = mixgcn_layer_desc{};
+        d.d_in = dims[l]; d.d_out = dims[l + 1]; d.ld_in = ld[l]; d.ld_out = ld[l + 1]; d.ld_saved = 4;
+        d.order = MIXGCN_ORDER_AUTO; d.precision = precision; d.keep_scale = 1.0f; d.in_scale = 1.0f; d.n_chunks = 0;
+        d.flags = (l < L - 1 ? MIXGCN_LAYER_RELU : 0u) | (l == 0 ? MIXGCN_LAYER_FIRST : 0u) |
+                  (l >= 1 ? MIXGCN_LAYER_GATE_GIN : 0u) | (l < L - 1 ? MIXGCN_LAYER_GOUT_GATED : 0u);
+        int32_t order = 0, cols = 0;
+        MIXGCN_TRY(mixgcn_layer_plan(&d, &order, &cols));
+        d.order = order; d.ld_saved = round4(cols);
+    }
+    lo.X.resize(L + 1); lo.saved.resize(L); lo.G.assign(L + 1, nullptr);
+    for (int l = 0; l <= L; ++l) lo.X[l] = c.take<float>(n * ld[l]);
+    for (int l = 0; l < L; ++l) lo.saved[l] = c.take<float>(n * lo.desc[l].ld_saved);
+    int64_t wmax = 4;
+    for (int l = 1; l < L; ++l) wmax = ld[l] > wmax ? ld[l] : wmax;
+    float* pool[2] = {nullptr, nullptr};
+    if (L >= 2) pool[0] = c.take<float>(n * wmax);
+    if (L >= 3) pool[1] = ld[L] >= wmax ? lo.X[L] : c.take<float>(n * wmax);
+    lo.G[L] = lo.X[L];  // the logits' gradient overwrites the logits
+    for (int l = L - 1, i = 0; l >= 1; --l, ++i) lo.G[l] = pool[i % 2];
+    lo.labels = c.take<int32_t>(n); lo.mask = c.take<uint8_t>(n); lo.loss = c.take<float>(4); lo.pred = c.take<int32_t>(n);
+    auto each = [&](std::vector<float*>& v, bool weight) {
+        v.resize(L);
+        for (int l = 0; l < L; ++l) v[l] = c.take<float>(weight ? (int64_t)dims[l] * dims[l + 1] : dims[l + 1]);
+    };
+    each(lo.W, true); each(lo.dW, true); each(lo.mW, true); each(lo.vW, true);
+    each(lo.b, false); each(lo.db, false); each(lo.mb, false); each(lo.vb, false);
+    lo.bytes = c.off;
+    return MIXGCN_OK;
+}
+
+}  // namespace
+
+extern "C" mixgcn_status mixgcn_train_step_host(mixgcn_ctx* ctx, const mixgcn_graph* g, int32_t L,
+                                                const int32_t* dims, int32_t precision, const float* X,
+                                                const int32_t* labels, const uint8_t* train_mask,
+                                                float* const* W, float* const* b, float* const* mW,
+                                                float* const* vW, float* const* mb, float* const* vb,
+                                                int64_t t, float lr, float beta1, float beta2, float eps,
+                                                float* loss, int32_t* pred) {
+    if (!ctx || !g || !dims || !X || !labels || !train_mask || !W || !b || !mW || !vW || !mb || !vb || !loss)
+        MIXGCN_FAIL(MIXGCN_EINVAL, "train_step_host: null argument");
+    if (L < 1 || L > 64) MIXGCN_FAIL(MIXGCN_EINVAL, "train_step_host: need 1 <= L <= 64 (got %d)", L);
+    for (int l = 0; l <= L; ++l)
+        if (dims[l] <= 0) MIXGCN_FAIL(MIXGCN_EINVAL, "train_step_host: dims[%d] must be positive", l);
+    for (int l = 0; l < L; ++l)
+        if (!W[l] || !b[l] || !mW[l] || !vW[l] || !mb[l] || !vb[l]) MIXGCN_FAIL(MIXGCN_EINVAL, "train_step_host: null tensor in layer %d", l);
+    if (t < 1) MIXGCN_FAIL(MIXGCN_EINVAL, "train_step_host: t must be >= 1");
+    if (dims[L] > 4096) MIXGCN_FAIL(MIXGCN_EINVAL, "train_step_host: at most 4096 classes");
+    MIXGCN_CUDA(cudaSetDevice(ctx->device));
+    const int64_t n = g->n;
+    StepLayout lo;
+    MIXGCN_TRY(lay_out(nullptr, n, L, dims, precision, lo));
+    if (lo.bytes > ctx->arena_bytes) {
+        MIXGCN_CUDA(cudaDeviceSynchronize());
+        cudaFree(ctx->arena); ctx->arena = nullptr; ctx->arena_bytes = 0;
+        void* p = nullptr;
+        if (cudaMalloc(&p, (size_t)lo.bytes) != cudaSuccess) {
+            cudaGetLastError();
+            MIXGCN_FAIL(MIXGCN_ENOMEM, "train_step_host: %lld bytes of device memory could not be allocated", (long long)lo.bytes);
+        }
+        ctx->arena = p; ctx->arena_bytes = lo.bytes;
+        MIXGCN_CUDA(cudaMemset(p, 0, (size_t)lo.bytes));
+    }
+    MIXGCN_TRY(lay_out(reinterpret_cast<char*>(ctx->arena), n, L, dims, precision, lo));
+    cudaStream_t s = ctx->side_stream[0];
+    const cudaMemcpyKind H2D = cudaMemcpyHostToDevice, D2H = cudaMemcpyDeviceToHost;
+
+    // inputs
+    const int64_t d0 = dims[0], ld0 = round4(d0);
+    if (ld0 == d0) MIXGCN_CUDA(cudaMemcpyAsync(lo.X[0], X, (size_t)(n * d0) * sizeof(float), H2D, s));
+    else MIXGCN_CUDA(cudaMemcpy2DAsync(lo.X[0], ld0 * sizeof(float), X, d0 * sizeof(float), d0 * sizeof(float), (size_t)n, H2D, s));
+    MIXGCN_CUDA(cudaMemcpyAsync(lo.labels, labels, n * sizeof(int32_t), H2D, s));
+    MIXGCN_CUDA(cudaMemcpyAsync(lo.mask, train_mask, n * sizeof(uint8_t), H2D, s));
+    for (int l = 0; l < L; ++l) {
+        const size_t wb = (size_t)dims[l] * dims[l + 1] * sizeof(float), bb = (size_t)dims[l + 1] * sizeof(float);
+        MIXGCN_CUDA(cudaMemcpyAsync(lo.W[l], W[l], wb, H2D, s));
+        MIXGCN_CUDA(cudaMemcpyAsync(lo.mW[l], mW[l], wb, H2D, s));
+        MIXGCN_CUDA(cudaMemcpyAsync(lo.vW[l], vW[l], wb, H2D, s));
+        MIXGCN_CUDA(cudaMemcpyAsync(lo.b[l], b[l], bb, H2D, s));
+        MIXGCN_CUDA(cudaMemcpyAsync(lo.mb[l], mb[l], bb, H2D, s));
+        MIXGCN_CUDA(cudaMemcpyAsync(lo.vb[l], vb[l], bb, H2D, s));
+    }
+    // forward, loss, backward, update
+    for (int l = 0; l < L; ++l)
+        MIXGCN_TRY(mixgcn_layer_fwd(ctx, g, &lo.desc[l], lo.X[l], lo.W[l], lo.b[l], nullptr, lo.saved[l], lo.X[l + 1], s));
+    MIXGCN_TRY(mixgcn_loss_softmax_xent(ctx, n, dims[L], lo.X[L], round4(dims[L]), lo.labels, lo.mask, lo.loss, lo.X[L],
+                                        lo.pred, nullptr, s));
+    for (int l = L - 1; l >= 0; --l)
+        MIXGCN_TRY(mixgcn_layer_bwd(ctx, g, &lo.desc[l], lo.X[l], lo.saved[l], lo.X[l + 1], nullptr, lo.W[l], lo.G[l + 1],
+                                    l > 0 ? lo.G[l] : nullptr, lo.dW[l], lo.db[l], s));
+    std::vector<float*> P, M1, M2; std::vector<const float*> Gr; std::vector<int64_t> numel;
+    for (int l = 0; l < L; ++l) { P.push_back(lo.W[l]); Gr.push_back(lo.dW[l]); M1.push_back(lo.mW[l]); M2.push_back(lo.vW[l]); numel.push_back((int64_t)dims[l] * dims[l + 1]); }
+    for (int l = 0; l < L; ++l) { P.push_back(lo.b[l]); Gr.push_back(lo.db[l]); M1.push_back(lo.mb[l]); M2.push_back(lo.vb[l]); numel.push_back(dims[l + 1]); }
+    MIXGCN_TRY(mixgcn_adam_step(ctx, 2 * L, P.data(), Gr.data(), M1.data(), M2.data(), numel.data(), t, lr, beta1, beta2, eps, s));
+    // results
+    MIXGCN_CUDA(cudaMemcpyAsync(loss, lo.loss, sizeof(float), D2H, s));
+    if (pred) MIXGCN_CUDA(cudaMemcpyAsync(pred, lo.pred, n * sizeof(int32_t), D2H, s));
+    for (int l = 0; l < L; ++l) {
+        const size_t wb = (size_t)dims[l] * dims[l + 1] * sizeof(float), bb = (size_t)dims[l + 1] * sizeof(float);
+        MIXGCN_CUDA(cudaMemcpyAsync(W[l], lo.W[l], wb, D2H, s));
+        MIXGCN_CUDA(cudaMemcpyAsync(mW[l], lo.mW[l], wb, D2H, s));
+        MIXGCN_CUDA(cudaMemcpyAsync(vW[l], lo.vW[l], wb, D2H, s));
+        MIXGCN_CUDA(cudaMemcpyAsync(b[l], lo.b[l], bb, D2H, s));
+        MIXGCN_CUDA(cudaMemcpyAsync(mb[l], lo.mb[l], bb, D2H, s));
+        MIXGCN_CUDA(cudaMemcpyAsync(vb[l], lo.vb[l], bb, D2H, s));
+    }
+    MIXGCN_CUDA(cudaStreamSynchronize(s));
+    return MIXGCN_OK;
+}

@@ -59,7 +59,9 @@ struct mixgcn_ctx {
     int n_spans, cap_spans;
     int64_t launches_total;
     int64_t phase_launches[MIXGCN_N_PHASES];
-    // host-step buffers live in the workspace tail; nothing else owned
+    // device arena of mixgcn_train_step_host (activations, parameters, gradients), grown on demand
+    void* arena;
+    int64_t arena_bytes;
 };
 
 // One CSR orientation of A_hat plus its aggregation schedule.

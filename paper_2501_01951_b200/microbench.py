@@ -1,0 +1,82 @@
+"""Single-kernel runs through the C-ABI, sized by flags: for CUDA-event timing of one operation
+and as a small, self-ending target for profiler captures.
+
+    python -m paper_2501_01951_b200.microbench --op spmm --n 4000000 --edges 32000000 --w 128
+    python -m paper_2501_01951_b200.microbench --op gemm --M 1000000 --N 1024 --K 1024 --precision tf32
+
+Prints one JSON line with the median time and the derived algorithmic GB/s or TFLOP/s.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import statistics
+
+import torch
+
+from . import binding as mg
+from . import synth
+
+
+def _time(fn, iters, warmup):
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    ts = []
+    for _ in range(iters):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        fn()
+        b.record()
+        torch.cuda.synchronize()
+        ts.append(a.elapsed_time(b))
+    return statistics.median(ts), min(ts)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--op", required=True, choices=["spmm", "gemm"])
+    ap.add_argument("--n", type=int, default=1 << 20)
+    ap.add_argument("--edges", type=int, default=8 << 20, help="distinct undirected edges of the R-MAT graph")
+    ap.add_argument("--w", type=int, default=128)
+    ap.add_argument("--M", type=int, default=1 << 20)
+    ap.add_argument("--N", type=int, default=256)
+    ap.add_argument("--K", type=int, default=256)
+    ap.add_argument("--ta", type=int, default=0)
+    ap.add_argument("--tb", type=int, default=0)
+    ap.add_argument("--precision", default="fp32", choices=list(mg.PRECISIONS))
+    ap.add_argument("--iters", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=2)
+    ap.add_argument("--seed", type=int, default=1005)
+    args = ap.parse_args()
+
+    dev = torch.device("cuda", 0)
+    ctx = mg.ctx_create(0)
+    out = dict(op=args.op)
+    if args.op == "spmm":
+        s, d = synth.rmat_graph(args.n, args.edges, args.seed, device=dev)
+        g = mg.graph_create(ctx, args.n, s, d)
+        del s, d
+        ld = (args.w + 3) // 4 * 4
+        Y = synth.normal_features(args.n, args.w, 7, device=dev, ld=ld)
+        Z = torch.zeros_like(Y)
+        med, best = _time(lambda: mg.spmm(ctx, g, Y, Z, args.w), args.iters, args.warmup)
+        alg = 8 * (g.n + 1) + 8 * g.nnz + 8 * g.n * args.w
+        out.update(n=g.n, nnz=g.nnz, w=args.w, max_deg=g.max_deg, ms_median=round(med, 4), ms_best=round(best, 4),
+                   alg_bytes=alg, alg_gbs=round(alg / med / 1e6, 1), gather_gbs=round(4 * g.nnz * args.w / med / 1e6, 1))
+    else:
+        M, N, K = args.M, args.N, args.K
+        r4 = lambda x: (x + 3) // 4 * 4
+        A = synth.uniform_tensor((K, r4(M)) if args.ta else (M, r4(K)), 1, device=dev)
+        B = synth.uniform_tensor((N, r4(K)) if args.tb else (K, r4(N)), 2, device=dev)
+        Cm = torch.zeros((M, r4(N)), device=dev)
+        prec = mg.PRECISIONS[args.precision]
+        med, best = _time(lambda: mg.gemm(ctx, prec, bool(args.ta), bool(args.tb), M, N, K, A, B, Cm), args.iters, args.warmup)
+        out.update(M=M, N=N, K=K, ta=args.ta, tb=args.tb, precision=args.precision, ms_median=round(med, 4),
+                   ms_best=round(best, 4), tflops=round(2 * M * N * K / med / 1e9, 2),
+                   min_gbs=round(4 * (M * K + K * N + M * N) / med / 1e6, 1))
+    print(json.dumps(out), flush=True)
+
+
+if __name__ == "__main__":
+    main()

@@ -472,3 +472,31 @@ def test_argument_errors(mg, ctx):
     with pytest.raises(mg.MixgcnError):
         mg.adam_step(ctx, [Y], [Y], [Y], [Y], 0)                    # t < 1
     assert torch.all(Z == 0)                                         # outputs untouched on host-side errors
+
+
+def test_train_step_host_matches_oracle_and_device_path(mg, ctx):
+    """The host-buffer entry point runs the same kernels as the device-buffer calls."""
+    from paper_2501_01951_b200.train import GcnTrainer
+    wl, s, d, X, y, m, Ws, bs = _tiny_problem()
+    gg = mg.graph_create(ctx, wl.n, s, d)
+    W = [w.clone() for w in Ws]; b = [x.clone() for x in bs]
+    mW = [torch.zeros_like(w) for w in W]; vW = [torch.zeros_like(w) for w in W]
+    mb = [torch.zeros_like(x) for x in b]; vb = [torch.zeros_like(x) for x in b]
+    pred = torch.zeros(wl.n, dtype=torch.int32)
+    tr = GcnTrainer(ctx, gg, wl.dims, mg.PREC_FP32)
+    tr.set_params(Ws, bs)
+    tr.set_inputs(padded(X), y.cuda(), m.cuda())
+    for t in (1, 2):
+        loss = mg.train_step_host(ctx, gg, wl.dims, mg.PREC_FP32, X, y, m, W, b, mW, vW, mb, vb, t, pred=pred, **ADAM)
+        tr.forward(); tr.compute_loss(); tr.backward(); tr.step(t, **ADAM)
+        assert loss == tr.loss.item()
+        for l in range(tr.L):
+            assert torch.equal(W[l], tr.W[l].cpu()) and torch.equal(b[l], tr.b[l].cpu())
+            assert torch.equal(mW[l], tr.mW[l].cpu()) and torch.equal(vb[l], tr.vb[l].cpu())
+        assert torch.equal(pred, tr.pred.cpu())
+    go = orc.graph_build(wl.n, s.numpy(), d.numpy())
+    ref = orc.train_epoch(go, X.numpy(), [w.numpy() for w in Ws], [x.numpy() for x in bs], y.numpy(), m.numpy(), None, 1, **ADAM)
+    W1 = [w.clone() for w in Ws]; b1 = [x.clone() for x in bs]
+    z = lambda lst: [torch.zeros_like(x) for x in lst]
+    loss = mg.train_step_host(ctx, gg, wl.dims, mg.PREC_FP32, X, y, m, W1, b1, z(W1), z(W1), z(b1), z(b1), 1, **ADAM)
+    assert abs(loss - ref["loss"]) <= 1e-5 * abs(ref["loss"])
