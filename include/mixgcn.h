@@ -223,6 +223,29 @@ mixgcn_status mixgcn_loss_softmax_xent(mixgcn_ctx* ctx, int64_t n, int32_t C, co
                                        float* loss, float* dlogits, int32_t* pred,
                                        int64_t* n_correct, void* stream);
 
+/* The same loss for callers that cannot allocate device memory.  (The paper has no counterpart:
+ * this is a deployment variant of mixgcn_loss_softmax_xent.)  A process that has given the whole
+ * GPU to its own memory pool, or a latency-critical loop that cannot afford the device-wide
+ * synchronisation of cudaMalloc/cudaFree, cannot create a mixgcn_ctx (its status word and
+ * workspace are cudaMalloc'd).  This entry point needs no context and calls no allocator: its
+ * scratch (train-node counter, status word, one fp64 partial per 1024 rows) lives in a fixed
+ * 256 KB array inside the library image, present on every GPU that loads the library until the
+ * process exits.
+ *  - Runs on the calling thread's CURRENT device; all pointers are device pointers of it.
+ *  - Arguments and results as mixgcn_loss_softmax_xent; `status` (device int32, nullable)
+ *    receives 0, 1 (empty train mask) or 2 (label outside [0,C)) when the stream reaches it.
+ *  - Limit: n <= 33,554,432 rows (32768 partials x 1024 rows) and 1 <= C <= 4096; larger sizes
+ *    return MIXGCN_EUNSUPPORTED and launch nothing.
+ *  - The first call on each device looks up the scratch array's device address (one
+ *    cudaGetSymbolAddress, cached per device); make that first call before any stream capture.
+ *  - All calls on a device share the one array, which keeps the previous call's contents; each
+ *    call clears the counter and status word first.  Two calls that overlap on the GPU (different
+ *    streams, no ordering between them) race on it: order them. */
+mixgcn_status mixgcn_loss_softmax_xent_noalloc(int64_t n, int32_t C, const float* logits, int64_t ld,
+                                               const int32_t* labels, const uint8_t* train_mask,
+                                               float* loss, float* dlogits, int32_t* pred,
+                                               int64_t* n_correct, int32_t* status, void* stream);
+
 /* Adam over n_tensors parameter tensors (HOST arrays of DEVICE pointers and element counts):
  * m = b1 m + (1-b1) g; v = b2 v + (1-b2) g^2; theta -= lr * (m/(1-b1^t)) / (sqrt(v/(1-b2^t)) + eps),
  * t >= 1, no weight decay (the weight-update step of Algorithm 2). */

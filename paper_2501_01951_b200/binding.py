@@ -38,7 +38,7 @@ SYMBOLS = (
     "mixgcn_graph_create", "mixgcn_graph_create_from_csr", "mixgcn_graph_info", "mixgcn_graph_export",
     "mixgcn_graph_export_schedule", "mixgcn_graph_destroy", "mixgcn_spmm", "mixgcn_gemm",
     "mixgcn_layer_plan", "mixgcn_layer_fwd", "mixgcn_layer_bwd", "mixgcn_loss_softmax_xent",
-    "mixgcn_adam_step", "mixgcn_train_step_host",
+    "mixgcn_adam_step", "mixgcn_train_step_host", "mixgcn_loss_softmax_xent_noalloc",
 )
 
 
@@ -286,6 +286,23 @@ def loss_softmax_xent(ctx: Ctx, logits, labels, train_mask, loss, dlogits=None, 
             raise TypeError("dlogits must share the logits' leading dimension")
     _check(lib.mixgcn_loss_softmax_xent(ctx.h, C.c_int64(n), C.c_int32(Cc), _ptr(logits), C.c_int64(ld), _ptr(labels),
                                         _ptr(train_mask), _ptr(loss), _ptr(dlogits), _ptr(pred), _ptr(n_correct), _stream()))
+
+
+def loss_softmax_xent_noalloc(logits, labels, train_mask, loss, dlogits=None, pred=None, n_correct=None,
+                              status=None, C_=None):
+    """The loss for callers that cannot allocate device memory: no context, scratch inside the
+    library image.  Runs on torch's current device; at most 33,554,432 rows."""
+    logits, ld = _mat(logits, "logits")
+    n = logits.shape[0]
+    Cc = logits.shape[1] if C_ is None else C_
+    _dev(labels, torch.int32, "labels"); _dev(train_mask, torch.uint8, "train_mask"); _dev(loss, torch.float32, "loss")
+    if dlogits is not None:
+        dlogits, ldd = _mat(dlogits, "dlogits")
+        if ldd != ld:
+            raise TypeError("dlogits must share the logits' leading dimension")
+    _check(lib.mixgcn_loss_softmax_xent_noalloc(C.c_int64(n), C.c_int32(Cc), _ptr(logits), C.c_int64(ld), _ptr(labels),
+                                                _ptr(train_mask), _ptr(loss), _ptr(dlogits), _ptr(pred), _ptr(n_correct),
+                                                _ptr(status), _stream()))
 
 
 def adam_step(ctx: Ctx, params, grads, ms, vs, t, lr=0.01, beta1=0.9, beta2=0.999, eps=1e-8):

@@ -1,6 +1,8 @@
 // Masked softmax cross-entropy with its gradient and arg-max (the loss line of Algorithm 2),
 // and the Adam step (its weight-update line).  Both are streaming kernels; floating-point
 // reductions run in a fixed order (per-warp shuffles, per-CTA partials, one final pass).
+#include <stddef.h>
+
 #include "internal.cuh"
 
 using namespace mixgcn;
@@ -194,6 +196,78 @@ extern "C" mixgcn_status mixgcn_adam_step(mixgcn_ctx* ctx, int32_t n_tensors, fl
         LaunchScope scope(ctx, PH_ADAM, s);
         adam_kernel<<<dim3((unsigned)bx, (unsigned)b.count), 256, 0, s>>>(b);
     }
+    MIXGCN_CUDA(cudaGetLastError());
+    return MIXGCN_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Allocation-free variant of the loss.
+//
+// Some callers cannot take device memory from the CUDA allocator: a process that has handed the
+// whole GPU to its own memory pool (so cudaMalloc fails), or a latency-critical loop that cannot
+// afford the device-wide synchronisation cudaMalloc and cudaFree imply.  They cannot create a
+// mixgcn_ctx either (its status word and workspace come from cudaMalloc).  For them the loss
+// kernels above run here with their scratch in a fixed array that is part of the library image.
+// ------------------------------------------------------------------------------------------------
+namespace {
+
+constexpr int NOALLOC_MAX_PARTIALS = 32768;   // one fp64 partial per block
+constexpr int NOALLOC_ROWS_PER_BLOCK = 1024;  // => at most 33,554,432 rows
+constexpr int NOALLOC_MAX_DEVICES = 64;
+
+struct NoAllocScratch {
+    unsigned long long count;      // train nodes, cleared at the start of every call
+    int32_t status;                // 0 ok, 1 empty train mask, 2 label out of range; cleared likewise
+    int32_t pad;
+    double part[NOALLOC_MAX_PARTIALS];
+};
+
+// Held by every GPU that loads the library, until the process exits (about 256 KB).
+static __device__ __align__(256) unsigned char g_noalloc_scratch[sizeof(NoAllocScratch)];
+
+// In host code the array's name is only a handle for the runtime, not a device address; the real
+// address is looked up once per device (with that device current) and cached here.
+NoAllocScratch* g_noalloc_ptr[NOALLOC_MAX_DEVICES] = {};
+
+}  // namespace
+
+extern "C" mixgcn_status mixgcn_loss_softmax_xent_noalloc(int64_t n, int32_t C, const float* logits, int64_t ld,
+                                                          const int32_t* labels, const uint8_t* train_mask,
+                                                          float* loss, float* dlogits, int32_t* pred,
+                                                          int64_t* n_correct, int32_t* status, void* stream) {
+    if (!logits || !labels || !train_mask || !loss) MIXGCN_FAIL(MIXGCN_EINVAL, "loss_noalloc: null argument");
+    if (n <= 0 || C <= 0 || C > 4096)
+        MIXGCN_FAIL(MIXGCN_EINVAL, "loss_noalloc: need n > 0 and 1 <= C <= 4096 (n=%lld C=%d)", (long long)n, C);
+    if (ld < C) MIXGCN_FAIL(MIXGCN_EINVAL, "loss_noalloc: ld (%lld) < C (%d)", (long long)ld, C);
+    const int64_t max_rows = (int64_t)NOALLOC_MAX_PARTIALS * NOALLOC_ROWS_PER_BLOCK;
+    if (n > max_rows)
+        MIXGCN_FAIL(MIXGCN_EUNSUPPORTED,
+                    "loss_noalloc: n = %lld exceeds the %lld rows the built-in scratch covers; use mixgcn_loss_softmax_xent",
+                    (long long)n, (long long)max_rows);
+    int device = -1;
+    MIXGCN_CUDA(cudaGetDevice(&device));
+    if (device < 0 || device >= NOALLOC_MAX_DEVICES) MIXGCN_FAIL(MIXGCN_EUNSUPPORTED, "loss_noalloc: device index %d not supported", device);
+    if (!g_noalloc_ptr[device]) {
+        // first call on this device: resolve the device address of the scratch array
+        void* p = nullptr;
+        MIXGCN_CUDA(cudaGetSymbolAddress(&p, g_noalloc_scratch));
+        if (!p) MIXGCN_FAIL(MIXGCN_ECUDA, "loss_noalloc: the scratch symbol has no device address");
+        g_noalloc_ptr[device] = reinterpret_cast<NoAllocScratch*>(p);
+    }
+    NoAllocScratch* sc = g_noalloc_ptr[device];
+    cudaStream_t s = (cudaStream_t)stream;
+    const int64_t blocks = (n + NOALLOC_ROWS_PER_BLOCK - 1) / NOALLOC_ROWS_PER_BLOCK;
+    // the array keeps the previous call's contents: clear the counter and the status word
+    MIXGCN_CUDA(cudaMemsetAsync(sc, 0, offsetof(NoAllocScratch, part), s));
+    if (n_correct) MIXGCN_CUDA(cudaMemsetAsync(n_correct, 0, sizeof(int64_t), s));
+    int64_t cb = (n + 255) / 256;
+    if (cb > 4096) cb = 4096;
+    count_mask_kernel<<<(unsigned)cb, 256, 0, s>>>(n, train_mask, &sc->count);
+    loss_rows_kernel<<<(unsigned)blocks, LOSS_WARPS * 32, 0, s>>>(n, C, logits, ld, labels, train_mask, &sc->count, dlogits,
+                                                                 pred, reinterpret_cast<unsigned long long*>(n_correct),
+                                                                 sc->part, &sc->status);
+    loss_final_kernel<<<1, 32, 0, s>>>((int)blocks, sc->part, &sc->count, loss, &sc->status);
+    if (status) MIXGCN_CUDA(cudaMemcpyAsync(status, &sc->status, sizeof(int32_t), cudaMemcpyDeviceToDevice, s));
     MIXGCN_CUDA(cudaGetLastError());
     return MIXGCN_OK;
 }
