@@ -3,6 +3,7 @@
 // Appendix A, and the row-chunked aggregation -> update pipeline on two streams (the fine-grain
 // sparse/dense pipeline of Section 3.2.2 mapped onto one GPU).
 #include <stdarg.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <new>
@@ -68,10 +69,20 @@ mixgcn_status launch_gemm_simt(mixgcn_ctx* ctx, int ta, int tb, int64_t M, int64
                                const float* A, int64_t lda, const float* B, int64_t ldb, float* C, int64_t ldc,
                                const mixgcn_epilogue* epi, int64_t epi_row0, cudaStream_t s);
 
+mixgcn_status launch_gemm_tc(mixgcn_ctx* ctx, int ta, int tb, int64_t M, int64_t N, int64_t K, const float* A,
+                             int64_t lda, const float* B, int64_t ldb, float* C, int64_t ldc,
+                             const mixgcn_epilogue* epi, int64_t epi_row0, cudaStream_t s);
+
 mixgcn_status launch_gemm(mixgcn_ctx* ctx, int precision, int ta, int tb, int64_t M, int64_t N, int64_t K,
                           const float* A, int64_t lda, const float* B, int64_t ldb, float* C, int64_t ldc,
                           const mixgcn_epilogue* epi, int64_t epi_row0, cudaStream_t s) {
-    (void)precision;  // reduced-precision tensor-core kernels plug in here; fp32 serves every request
+    // TF32 / BF16 requests go to the tcgen05 kernels (TF32 operands serve both: at least the requested
+    // precision); shapes or alignments they do not take, and fp32 requests, use the FMA kernel.
+    static const bool disable_tc = getenv("MIXGCN_DISABLE_TC") != nullptr;
+    if (precision != MIXGCN_PREC_FP32 && !disable_tc) {
+        mixgcn_status st = launch_gemm_tc(ctx, ta, tb, M, N, K, A, lda, B, ldb, C, ldc, epi, epi_row0, s);
+        if (st != MIXGCN_EUNSUPPORTED) return st;
+    }
     return launch_gemm_simt(ctx, ta, tb, M, N, K, A, lda, B, ldb, C, ldc, epi, epi_row0, s);
 }
 

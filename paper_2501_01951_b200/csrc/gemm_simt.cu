@@ -329,6 +329,20 @@ mixgcn_status launch_gemm_simt(mixgcn_ctx* ctx, int ta, int tb, int64_t M, int64
     return MIXGCN_OK;
 }
 
+mixgcn_status launch_splitk_reduce(mixgcn_ctx* ctx, int64_t M, int64_t N, int splits, const float* part, float* C,
+                                   int64_t ldc, const mixgcn_epilogue* epi, cudaStream_t s) {
+    Epi e{};
+    if (epi) {
+        e.bias = epi->bias; e.relu = epi->relu; e.drop = epi->drop_mask; e.keep_scale = epi->keep_scale;
+        e.gate = epi->gate; e.ld_gate = epi->ld_gate; e.gate_scale = epi->gate_scale;
+    }
+    LaunchScope scope(ctx, PH_GEMM, s);
+    const int64_t total = M * N;
+    splitk_reduce_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(M, N, splits, part, C, ldc, e);
+    MIXGCN_CUDA(cudaGetLastError());
+    return MIXGCN_OK;
+}
+
 mixgcn_status launch_colsum(mixgcn_ctx* ctx, int64_t n, int32_t d, const float* X, int64_t ld, float* out,
                             cudaStream_t s) {
     int64_t rows_per_block = 2048;

@@ -1,0 +1,447 @@
+// Dense update products on the 5th-generation tensor cores (tcgen05) for sm_100a:
+// the update line of Algorithm 2 (P = Z W) and its two backward products (dZ = dP W^T,
+// dW = Z^T dP) with TF32 operands read straight from the fp32 activations and fp32 accumulation
+// in tensor memory.
+//
+//  * Operands reach shared memory by TMA (cp.async.bulk.tensor, 128-byte swizzle, out-of-bounds
+//    elements filled with zeros, so ragged M / N / K tails need no special code).
+//  * One elected thread issues tcgen05.mma (M = 128, N <= 256, K = 8 per instruction); the
+//    128 x N fp32 accumulator lives in TMEM and is read back by four warps with tcgen05.ld for the
+//    fused epilogue (bias, ReLU, dropout mask, gate) and the single store of C.
+//  * Warp roles: warps 0-3 epilogue (TMEM lane quarter = warp id), warp 4 TMA producer,
+//    warp 5 TMEM allocation + MMA issue.  Stages are handed over with mbarriers; every wait is
+//    bounded: on expiry the CTA records DEV_WAIT_EXPIRED in the status word, stops issuing work,
+//    frees its TMEM and returns.
+//  * Two operand forms.  "KK": A is M x K row-major (K contiguous) and B is N x K row-major -- the
+//    forward product and dZ, with the small weight matrix first packed (transposed if needed, zero
+//    padded) into the workspace.  "MM": A is K x M and B is K x N row-major (M / N contiguous,
+//    K = node count) -- the weight gradient, split over CTAs along K into partial tiles that the
+//    fixed-order fp64 reduction combines.
+#include <cuda.h>
+
+#include "internal.cuh"
+
+using namespace mixgcn;
+
+namespace {
+
+constexpr int TC_BM = 128;          // rows of D per CTA = UMMA M
+constexpr int TC_BK = 32;           // fp32 elements per stage along K (one 128-byte swizzle row / 32 k-rows)
+constexpr int TC_THREADS = 192;
+constexpr uint32_t WAIT_LIMIT = 1u << 22;
+
+struct TcEpi {
+    const float* bias; int relu;
+    const uint8_t* drop; float keep_scale;
+    const float* gate; int64_t ld_gate; float gate_scale;
+    int64_t row0;
+};
+
+struct TcParams {
+    int64_t M, N, K;
+    int bn;                 // UMMA N: multiple of 16, 16..256
+    int stages;
+    int64_t m_tiles, n_tiles;
+    int64_t k_per_split;    // MM form: multiple of TC_BK
+    int splits;
+    float* C; int64_t ldc; int vec_c;
+    int raw;                // 1: store the accumulator unchanged (split-K partial)
+    TcEpi epi;
+    int32_t* status;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait: false when the limit is reached (the caller then abandons the tile).
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+    for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 1023u) == 1023u && *abort_flag) return false;
+    }
+    return false;
+}
+__device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* map, int32_t c0, int32_t c1, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tc_mma_tf32(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor, 128-byte swizzle, version 1 (sm_100).
+//   K-major operand (rows of 128 bytes = 32 fp32 along K, 8-row groups of 1024 bytes):
+//     leading byte offset unused (1), stride byte offset = 1024.
+//   MN-major TF32 operand (k-rows of 128 bytes = 32 fp32 along M/N; one 32-wide chunk holds TC_BK
+//     k-rows): only the 128-byte swizzle with 32-byte atoms is defined for it (layout type 1; the
+//     TMA counterpart is SWIZZLE_128B_ATOM_32B); its K atom is 4 k-rows, so the stride byte offset
+//     is 512 and the leading byte offset is the distance between 32-wide chunks.
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint32_t layout_type) {
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+    d |= (uint64_t)1 << 46;   // descriptor version
+    d |= (uint64_t)layout_type << 61;   // 2 = SWIZZLE_128B, 1 = SWIZZLE_128B with 32-byte atoms
+    return d;
+}
+
+// Instruction descriptor: fp32 accumulate, TF32 x TF32, dense, M = 128.
+__host__ __device__ inline uint32_t make_idesc_tf32(int n, bool mn_major) {
+    uint32_t d = 0;
+    d |= 1u << 4;                       // D format F32
+    d |= 2u << 7;                       // A format TF32
+    d |= 2u << 10;                      // B format TF32
+    if (mn_major) d |= (1u << 15) | (1u << 16);
+    d |= (uint32_t)(n >> 3) << 17;
+    d |= (uint32_t)(TC_BM >> 4) << 24;
+    return d;
+}
+
+__device__ __forceinline__ float tc_apply_epi(const TcEpi& e, float y, int64_t m, int64_t n, int64_t N) {
+    if (e.bias) y += e.bias[n];
+    if (e.relu) y = fmaxf(y, 0.0f);
+    if (e.drop) y = e.drop[(e.row0 + m) * N + n] ? y * e.keep_scale : 0.0f;
+    if (e.gate) y = e.gate[(e.row0 + m) * e.ld_gate + n] > 0.0f ? y * e.gate_scale : 0.0f;
+    return y;
+}
+
+template <bool MN_MAJOR>
+__global__ void __launch_bounds__(TC_THREADS) gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a,
+                                                             const __grid_constant__ CUtensorMap map_b,
+                                                             const TcParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t full_bar[8], empty_bar[8], acc_bar;
+    __shared__ uint32_t tmem_holder;
+    __shared__ int abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int bn32 = (p.bn + 31) & ~31;
+    const uint32_t a_bytes = TC_BM * TC_BK * 4, b_bytes = (uint32_t)bn32 * TC_BK * 4;
+    const uint32_t stage_bytes = a_bytes + b_bytes;
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+
+    const int64_t tile = blockIdx.x;
+    const int64_t m0 = (tile / p.n_tiles) * TC_BM, n0 = (tile % p.n_tiles) * p.bn;
+    int64_t kb = 0, ke = p.K;
+    if (MN_MAJOR) {
+        kb = (int64_t)blockIdx.z * p.k_per_split;
+        ke = kb + p.k_per_split < p.K ? kb + p.k_per_split : p.K;
+    }
+    const int nk = (int)((ke - kb + TC_BK - 1) / TC_BK);
+    uint32_t tmem_cols = 32;
+    while ((int)tmem_cols < p.bn) tmem_cols <<= 1;
+
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        for (int s = 0; s < p.stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        mbar_init(&acc_bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 5) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_holder)), "r"(tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_holder;
+
+    if (warp == 4) {
+        if (lane == 0) {
+            // ---------------- TMA producer ----------------
+            for (int ks = 0; ks < nk; ++ks) {
+                const int s = ks % p.stages;
+                const uint32_t ph = ((ks / p.stages) & 1) ^ 1;
+                if (!mbar_wait(&empty_bar[s], ph, &abort_flag)) { abort_flag = 1; atomicMax(p.status, DEV_WAIT_EXPIRED); break; }
+                uint8_t* sa = smem + (size_t)s * stage_bytes;
+                uint8_t* sb = sa + a_bytes;
+                mbar_expect_tx(&full_bar[s], stage_bytes);
+                const int32_t k0 = (int32_t)(kb + (int64_t)ks * TC_BK);
+                if (!MN_MAJOR) {
+                    tma_load_2d(sa, &map_a, k0, (int32_t)m0, &full_bar[s]);                  // 128 rows x 32 k
+                    tma_load_2d(sb, &map_b, k0, (int32_t)n0, &full_bar[s]);                  // bn32 rows x 32 k
+                } else {
+                    for (int c = 0; c < TC_BM / 32; ++c)                                      // 32 k-rows x 32 m each
+                        tma_load_2d(sa + c * (TC_BK * 128), &map_a, (int32_t)(m0 + 32 * c), k0, &full_bar[s]);
+                    for (int c = 0; c < bn32 / 32; ++c)
+                        tma_load_2d(sb + c * (TC_BK * 128), &map_b, (int32_t)(n0 + 32 * c), k0, &full_bar[s]);
+                }
+            }
+        }
+    } else if (warp == 5) {
+        if (lane == 0) {
+            // ---------------- MMA issuer ----------------
+            const uint32_t idesc = make_idesc_tf32(p.bn, MN_MAJOR);
+            bool ok = true;
+            for (int ks = 0; ks < nk && ok; ++ks) {
+                const int s = ks % p.stages;
+                const uint32_t ph = (ks / p.stages) & 1;
+                if (!mbar_wait(&full_bar[s], ph, &abort_flag)) { abort_flag = 1; atomicMax(p.status, DEV_WAIT_EXPIRED); ok = false; break; }
+                tc_fence_after();
+                const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes), sb = sa + a_bytes;
+#pragma unroll
+                for (int k8 = 0; k8 < TC_BK / 8; ++k8) {
+                    uint64_t ad, bd;
+                    if (!MN_MAJOR) {
+                        ad = make_desc(sa + k8 * 32, 16, 1024, 2);
+                        bd = make_desc(sb + k8 * 32, 16, 1024, 2);
+                    } else {
+                        ad = make_desc(sa + k8 * 1024, TC_BK * 128, 512, 1);
+                        bd = make_desc(sb + k8 * 1024, TC_BK * 128, 512, 1);
+                    }
+                    tc_mma_tf32(tmem_base, ad, bd, idesc, (ks | k8) != 0 ? 1u : 0u);
+                }
+                tc_commit(&empty_bar[s]);     // the stage is free once these MMAs have read it
+            }
+            if (ok) tc_commit(&acc_bar);      // the accumulator is complete
+        }
+    } else {
+        // ---------------- epilogue: warps 0..3 own TMEM lanes 32*warp .. 32*warp+31 ----------------
+        bool ok = true;
+        if (nk > 0) {
+            if (lane == 0) ok = mbar_wait(&acc_bar, 0, &abort_flag);
+            ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
+            if (!ok && lane == 0) { abort_flag = 1; atomicMax(p.status, DEV_WAIT_EXPIRED); }
+        }
+        __syncwarp();
+        tc_fence_after();
+        if (ok) {
+            const int64_t m = m0 + warp * 32 + lane;
+            float* Cb = p.C + (MN_MAJOR && p.raw ? (int64_t)blockIdx.z * p.M * p.N : 0);
+            for (int c0 = 0; c0 < p.bn; c0 += 32) {
+                uint32_t r[32];
+                if (nk > 0) {
+                    tc_ld32(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, r);
+                    tc_wait_ld();
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) r[j] = 0u;
+                }
+                if (m < p.M) {
+                    const int64_t nb = n0 + c0;
+                    float* dst = Cb + m * p.ldc + nb;
+                    float v[32];
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        v[j] = __uint_as_float(r[j]);
+                        if (!p.raw && nb + j < p.N) v[j] = tc_apply_epi(p.epi, v[j], m, nb + j, p.N);
+                    }
+                    if (p.vec_c && nb + 31 < p.N && c0 + 31 < p.bn) {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4)
+                            *reinterpret_cast<float4*>(dst + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (nb + j < p.N && c0 + j < p.bn) dst[j] = v[j];
+                    }
+                }
+            }
+        }
+    }
+    if (threadIdx.x == 0 && abort_flag) {
+        // a wait expired: give copies that may still be in flight time to land before the CTA retires
+        for (int i = 0; i < 200; ++i) __nanosleep(1000);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 5) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
+    }
+}
+
+// dst[n][k] = trans ? src[k][n] : src[n][k] for n < N, k < K, zero elsewhere; dst is rows x kpad.
+__global__ void pack_b_kernel(const float* __restrict__ src, int64_t ld, int trans, int N, int K, int rows, int kpad,
+                              float* __restrict__ dst) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= (int64_t)rows * kpad) return;
+    const int n = (int)(i / kpad), k = (int)(i % kpad);
+    float v = 0.0f;
+    if (n < N && k < K) v = trans ? src[(int64_t)k * ld + n] : src[(int64_t)n * ld + k];
+    dst[i] = v;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+        else
+            cudaGetLastError();
+    }
+    return fn;
+}
+
+// 2-D fp32 tensor, `inner` contiguous elements per row, `outer` rows of `ld` elements; 128-byte swizzle.
+bool encode_2d(CUtensorMap* map, const float* base, int64_t inner, int64_t outer, int64_t ld, int box_inner, int box_outer,
+               CUtensorMapSwizzle swizzle = CU_TENSOR_MAP_SWIZZLE_128B) {
+    EncodeTiledFn fn = get_encode();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)outer};
+    cuuint64_t strides[1] = {(cuuint64_t)ld * sizeof(float)};
+    cuuint32_t box[2] = {(cuuint32_t)box_inner, (cuuint32_t)box_outer};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int pick_bn(int64_t N) {
+    int64_t bn = (N + 15) / 16 * 16;
+    if (bn > 256) {
+        // split N evenly into tiles that are multiples of 32 and <= 256
+        int64_t tiles = (N + 255) / 256;
+        bn = ((N + tiles - 1) / tiles + 31) / 32 * 32;
+    }
+    return (int)bn;
+}
+
+int pick_stages(int bn) {
+    const int bn32 = (bn + 31) & ~31;
+    const int stage = TC_BM * TC_BK * 4 + bn32 * TC_BK * 4;
+    int s = (96 * 1024) / stage;      // aim at two CTAs per SM
+    if (s < 2) s = 2;
+    if (s > 6) s = 6;
+    return s;
+}
+
+}  // namespace
+
+namespace mixgcn {
+
+mixgcn_status launch_splitk_reduce(mixgcn_ctx* ctx, int64_t M, int64_t N, int splits, const float* part, float* C,
+                                   int64_t ldc, const mixgcn_epilogue* epi, cudaStream_t s);
+
+// Returns MIXGCN_EUNSUPPORTED (without touching anything) when this shape / alignment is not
+// served by the tensor-core kernels; the caller then uses the fp32 kernel.
+mixgcn_status launch_gemm_tc(mixgcn_ctx* ctx, int ta, int tb, int64_t M, int64_t N, int64_t K, const float* A,
+                             int64_t lda, const float* B, int64_t ldb, float* C, int64_t ldc,
+                             const mixgcn_epilogue* epi, int64_t epi_row0, cudaStream_t s) {
+    if (M <= 0 || N <= 0 || K <= 0) return MIXGCN_EUNSUPPORTED;
+    if (ta && tb) return MIXGCN_EUNSUPPORTED;
+    if (!aligned16(A) || (lda & 3)) return MIXGCN_EUNSUPPORTED;
+    if (ta && (!aligned16(B) || (ldb & 3))) return MIXGCN_EUNSUPPORTED;
+    if (M >= (1ll << 31) || N >= (1ll << 31) || K >= (1ll << 31)) return MIXGCN_EUNSUPPORTED;
+    if (!get_encode()) return MIXGCN_EUNSUPPORTED;
+
+    TcParams p{};
+    p.M = M; p.N = N; p.K = K;
+    p.bn = pick_bn(N);
+    p.stages = pick_stages(p.bn);
+    p.m_tiles = (M + TC_BM - 1) / TC_BM;
+    p.n_tiles = (N + p.bn - 1) / p.bn;
+    p.C = C; p.ldc = ldc; p.vec_c = aligned16(C) && (ldc & 3) == 0;
+    p.status = ctx->d_status;
+    if (epi) {
+        p.epi.bias = epi->bias; p.epi.relu = epi->relu; p.epi.drop = epi->drop_mask; p.epi.keep_scale = epi->keep_scale;
+        p.epi.gate = epi->gate; p.epi.ld_gate = epi->ld_gate; p.epi.gate_scale = epi->gate_scale;
+    }
+    p.epi.row0 = epi_row0;
+    const int64_t tiles = p.m_tiles * p.n_tiles;
+    if (tiles > 0x7FFFFFFFll) return MIXGCN_EUNSUPPORTED;
+    const int bn32 = (p.bn + 31) & ~31;
+    const size_t smem = (size_t)p.stages * (TC_BM * TC_BK * 4 + bn32 * TC_BK * 4) + 1024;
+    CUtensorMap map_a, map_b;
+
+    if (!ta) {
+        // KK form: pack B as rows x kpad (K contiguous), rows = n_tiles * bn32
+        const int kpad = (int)((K + TC_BK - 1) / TC_BK * TC_BK);
+        const int rows = (int)(p.n_tiles * p.bn > bn32 ? p.n_tiles * p.bn : bn32);
+        MIXGCN_TRY(ensure_workspace(ctx, (int64_t)rows * kpad * (int64_t)sizeof(float)));
+        float* packed = reinterpret_cast<float*>(ctx->workspace);
+        if (!encode_2d(&map_a, A, K, M, lda, TC_BK, TC_BM)) return MIXGCN_EUNSUPPORTED;
+        if (!encode_2d(&map_b, packed, kpad, rows, kpad, TC_BK, bn32)) return MIXGCN_EUNSUPPORTED;
+        {
+            LaunchScope scope(ctx, PH_GEMM, s);
+            const int64_t total = (int64_t)rows * kpad;
+            pack_b_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(B, ldb, tb ? 0 : 1, (int)N, (int)K, rows, kpad, packed);
+        }
+        p.splits = 1; p.k_per_split = K; p.raw = 0;
+        MIXGCN_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        LaunchScope scope(ctx, PH_GEMM, s);
+        gemm_tc_kernel<false><<<dim3((unsigned)tiles, 1, 1), TC_THREADS, smem, s>>>(map_a, map_b, p);
+        MIXGCN_CUDA(cudaGetLastError());
+        return MIXGCN_OK;
+    }
+
+    // MM form (weight gradient): split K over CTAs
+    int splits = 1;
+    {
+        const int64_t want = (4 * (int64_t)ctx->sm_count + tiles - 1) / tiles;
+        const int64_t maxs = (K + 2047) / 2048;
+        splits = (int)(want < maxs ? want : maxs);
+        if (splits < 1) splits = 1;
+        if (splits > 2048) splits = 2048;
+    }
+    int64_t kps = (K + splits - 1) / splits;
+    kps = (kps + TC_BK - 1) / TC_BK * TC_BK;
+    splits = (int)((K + kps - 1) / kps);
+    p.k_per_split = kps; p.splits = splits;
+    if (!encode_2d(&map_a, A, M, K, lda, 32, TC_BK, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B)) return MIXGCN_EUNSUPPORTED;
+    if (!encode_2d(&map_b, B, N, K, ldb, 32, TC_BK, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B)) return MIXGCN_EUNSUPPORTED;
+    if (splits > 1) {
+        MIXGCN_TRY(ensure_workspace(ctx, (int64_t)splits * M * N * (int64_t)sizeof(float)));
+        p.C = reinterpret_cast<float*>(ctx->workspace); p.ldc = N; p.vec_c = (N & 3) == 0; p.raw = 1;
+    } else {
+        p.raw = 0;
+    }
+    MIXGCN_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    {
+        LaunchScope scope(ctx, PH_GEMM, s);
+        gemm_tc_kernel<true><<<dim3((unsigned)tiles, 1, (unsigned)splits), TC_THREADS, smem, s>>>(map_a, map_b, p);
+    }
+    MIXGCN_CUDA(cudaGetLastError());
+    if (splits > 1) MIXGCN_TRY(launch_splitk_reduce(ctx, M, N, splits, p.C, C, ldc, epi, s));
+    return MIXGCN_OK;
+}
+
+}  // namespace mixgcn

@@ -500,3 +500,81 @@ def test_train_step_host_matches_oracle_and_device_path(mg, ctx):
     z = lambda lst: [torch.zeros_like(x) for x in lst]
     loss = mg.train_step_host(ctx, gg, wl.dims, mg.PREC_FP32, X, y, m, W1, b1, z(W1), z(W1), z(b1), z(b1), 1, **ADAM)
     assert abs(loss - ref["loss"]) <= 1e-5 * abs(ref["loss"])
+
+
+# --------------------------------------------------------------------------- tensor-core products
+
+def _tf32_trunc(a):
+    """fp32 values with the 13 low mantissa bits cleared (what a TF32 operand read keeps)."""
+    b = np.ascontiguousarray(a, dtype=np.float32).view(np.uint32) & np.uint32(0xFFFFE000)
+    return b.view(np.float32).astype(np.float64)
+
+
+TC_SHAPES = [  # M, N, K
+    (128, 128, 32), (128, 16, 8), (300, 41, 100), (257, 256, 602), (1000, 172, 128), (640, 1024, 256), (513, 602, 47),
+]
+
+
+@pytest.mark.parametrize("M,N,K", TC_SHAPES)
+@pytest.mark.parametrize("tb", [False, True])
+def test_gemm_tf32_forward_forms(mg, ctx, M, N, K, tb):
+    from helpers import TOL_LOWP
+    A = synth.uniform_tensor((M, K), 131 + M, -1, 1)
+    B = synth.uniform_tensor((N, K) if tb else (K, N), 132 + N, -1, 1)
+    bias = synth.uniform_tensor((N,), 133, -1, 1)
+    Cd = torch.full((M, round4(N) + 4), 3.0, device="cuda")
+    epi = mg.make_epilogue(bias=bias.cuda(), relu=True)
+    mg.gemm(ctx, mg.PREC_TF32, False, tb, M, N, K, padded(A, fill=float("nan")), B.cuda().contiguous(), Cd, epi=epi)
+    Bo = B.numpy().T if tb else B.numpy()
+    want = orc.activation(orc.update(A.numpy(), Bo, bias.numpy()), True)
+    assert rel_fro(host(Cd, N), want) <= TOL_LOWP
+    assert torch.all(Cd[:, round4(N):] == 3.0)
+    # tighter: against the product of TF32-truncated operands the result is fp32-accurate
+    want_t = orc.activation(orc.update(_tf32_trunc(A.numpy()), _tf32_trunc(Bo), bias.numpy()), True)
+    assert rel_fro(host(Cd, N), want_t) <= 2e-5
+    assert mg.ctx_poll_status(ctx, raise_on_error=False) == 0
+
+
+@pytest.mark.parametrize("M,N,K", [(128, 128, 64), (64, 32, 4096), (100, 47, 70001), (602, 256, 9000), (1024, 64, 5000), (128, 172, 33333)])
+def test_gemm_tf32_weight_gradient_form(mg, ctx, M, N, K):
+    from helpers import TOL_LOWP
+    A, B = synth.normal_features(K, M, 141), synth.normal_features(K, N, 142)
+    Cd = torch.full((M, N), 3.0, device="cuda")
+    mg.gemm(ctx, mg.PREC_TF32, True, False, M, N, K, padded(A, fill=float("nan")), padded(B, fill=float("nan")), Cd)
+    want = A.numpy().astype(np.float64).T @ B.numpy().astype(np.float64)
+    assert rel_fro(host(Cd), want) <= TOL_LOWP
+    want_t = _tf32_trunc(A.numpy()).T @ _tf32_trunc(B.numpy())
+    assert rel_fro(host(Cd), want_t) <= 2e-5
+    Cd2 = torch.zeros_like(Cd)
+    mg.gemm(ctx, mg.PREC_TF32, True, False, M, N, K, padded(A, fill=float("nan")), padded(B, fill=float("nan")), Cd2)
+    assert torch.equal(Cd, Cd2)
+    assert mg.ctx_poll_status(ctx, raise_on_error=False) == 0
+
+
+def test_training_epoch_tf32_within_low_precision_bound(mg, ctx):
+    from helpers import TOL_LOWP
+    from paper_2501_01951_b200.train import GcnTrainer
+    wl, s, d, X, y, m, Ws, bs = _tiny_problem()
+    go = orc.graph_build(wl.n, s.numpy(), d.numpy())
+    gg = mg.graph_create(ctx, wl.n, s, d)
+    tr = GcnTrainer(ctx, gg, wl.dims, mg.PREC_TF32)
+    tr.set_params(Ws, bs)
+    tr.set_inputs(padded(X), y.cuda(), m.cuda())
+    tr.forward()
+    logits = host(tr.X[-1], wl.classes).copy()
+    tr.compute_loss(); tr.backward()
+    ref = orc.train_epoch(go, X.numpy(), [w.numpy() for w in Ws], [b.numpy() for b in bs], y.numpy(), m.numpy(), None, 1, **ADAM)
+    assert rel_fro(logits, ref["logits"]) <= TOL_LOWP
+    assert abs(tr.loss.item() - ref["loss"]) <= TOL_LOWP * abs(ref["loss"])
+    # Gradients are sums with heavy cancellation (softmax - onehot), so a relative bound on the result
+    # is not what reduced-precision operands can promise; the inner-product bound is: the error of
+    # sum_i a_i b_i is at most u * sum_i |a_i| |b_i|.  Measure the error against that scale.
+    Gout = ref["G"]
+    for l in range(tr.L - 1, -1, -1):
+        dP, dW, db, dZ = orc.update_bwd(ref["Zs"][l], ref["Ps"][l], Ws[l].numpy(), Gout, relu=l < tr.L - 1, need_dZ=l > 0)
+        scale_w = np.linalg.norm(np.abs(ref["Zs"][l]).T @ np.abs(dP))
+        scale_b = np.linalg.norm(np.abs(dP).sum(axis=0))
+        assert np.linalg.norm(tr.dW[l].cpu().numpy() - ref["dW"][l]) <= TOL_LOWP * scale_w
+        assert np.linalg.norm(tr.db[l].cpu().numpy() - ref["db"][l]) <= TOL_LOWP * scale_b
+        if l > 0:
+            Gout = orc.aggregate(go, dZ, transposed=True)
