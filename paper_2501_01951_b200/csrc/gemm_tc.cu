@@ -290,6 +290,217 @@ __global__ void __launch_bounds__(TC_THREADS) gemm_tc_kernel(const __grid_consta
     }
 }
 
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, const void* smem_src, int32_t c0, int32_t c1) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+                 ::"l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(smem_u32(smem_src)) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+constexpr int KK_EPI_WARPS = 8;                       // two per TMEM lane quarter, each takes every other 32-column chunk
+constexpr int KK_THREADS = (KK_EPI_WARPS + 2) * 32;    // + TMA producer warp + MMA warp
+constexpr int KK_BIAS_MAX = 1024;
+
+// Persistent K-major kernel for the tall products (M = node count): each CTA walks over output tiles
+// (n fastest, so consecutive tiles of a CTA share their A rows in L2).  The TMA producer runs ahead
+// through a ring of stages across tile boundaries, the accumulator is double-buffered in TMEM so the
+// epilogue of tile j overlaps the loads and MMAs of tile j+1, and when the packed weight matrix is
+// small enough it is loaded into shared memory once per CTA and stays there.  The epilogue (eight
+// warps) applies bias / ReLU from registers and shared memory, writes 32-row x 128-byte boxes in the
+// 128-byte swizzle and hands them to TMA stores, which also clip ragged M / N edges.
+__global__ void __launch_bounds__(KK_THREADS) gemm_tc_kk_kernel(const __grid_constant__ CUtensorMap map_a,
+                                                                const __grid_constant__ CUtensorMap map_b,
+                                                                const __grid_constant__ CUtensorMap map_c,
+                                                                const TcParams p, const int b_resident, const int tma_store) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t full_bar[8], empty_bar[8], acc_full[2], acc_empty[2], b_bar;
+    __shared__ __align__(16) float s_bias[KK_BIAS_MAX + 32];
+    __shared__ uint32_t tmem_holder;
+    __shared__ int abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int bn32 = (p.bn + 31) & ~31;
+    const uint32_t a_bytes = TC_BM * TC_BK * 4, b_bytes = (uint32_t)bn32 * TC_BK * 4;
+    const int nk = (int)((p.K + TC_BK - 1) / TC_BK);
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    // layout: [resident B: nk * b_bytes] [ring of stages: A (+ B when not resident)] [one output box per epilogue warp]
+    uint8_t* smem_b_res = smem;
+    uint8_t* smem_ring = smem + (b_resident ? (size_t)nk * b_bytes : 0);
+    const uint32_t stage_bytes = a_bytes + (b_resident ? 0u : b_bytes);
+    uint8_t* smem_out = smem_ring + (size_t)p.stages * stage_bytes;
+
+    const int64_t tiles = p.m_tiles * p.n_tiles;
+    uint32_t acc_stride = 32;
+    while ((int)acc_stride < p.bn) acc_stride <<= 1;
+    const uint32_t tmem_cols = acc_stride * 2;
+    const bool bias_in_smem = p.epi.bias != nullptr && p.N <= KK_BIAS_MAX;
+
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        for (int s = 0; s < p.stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], KK_EPI_WARPS); }
+        mbar_init(&b_bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (bias_in_smem)
+        for (int i = threadIdx.x; i < KK_BIAS_MAX + 32; i += KK_THREADS) s_bias[i] = i < p.N ? p.epi.bias[i] : 0.0f;
+    if (warp == KK_EPI_WARPS + 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_holder)), "r"(tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_holder;
+
+    if (warp == KK_EPI_WARPS) {
+        if (lane == 0) {
+            // ---------------- TMA producer ----------------
+            bool ok = true;
+            if (b_resident) {
+                mbar_expect_tx(&b_bar, (uint32_t)nk * b_bytes);
+                for (int ks = 0; ks < nk; ++ks) tma_load_2d(smem_b_res + (size_t)ks * b_bytes, &map_b, ks * TC_BK, 0, &b_bar);
+            }
+            uint32_t it = 0;
+            for (int64_t tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x) {
+                const int32_t m0 = (int32_t)((tile / p.n_tiles) * TC_BM), n0 = (int32_t)((tile % p.n_tiles) * p.bn);
+                for (int ks = 0; ks < nk; ++ks, ++it) {
+                    const int s = it % p.stages;
+                    const uint32_t ph = ((it / p.stages) & 1) ^ 1;
+                    if (!mbar_wait(&empty_bar[s], ph, &abort_flag)) { abort_flag = 1; atomicMax(p.status, DEV_WAIT_EXPIRED); ok = false; break; }
+                    uint8_t* sa = smem_ring + (size_t)s * stage_bytes;
+                    mbar_expect_tx(&full_bar[s], stage_bytes);
+                    tma_load_2d(sa, &map_a, ks * TC_BK, m0, &full_bar[s]);
+                    if (!b_resident) tma_load_2d(sa + a_bytes, &map_b, ks * TC_BK, n0, &full_bar[s]);
+                }
+            }
+        }
+    } else if (warp == KK_EPI_WARPS + 1) {
+        if (lane == 0) {
+            // ---------------- MMA issuer ----------------
+            const uint32_t idesc = make_idesc_tf32(p.bn, false);
+            bool ok = true;
+            if (b_resident) {
+                if (!mbar_wait(&b_bar, 0, &abort_flag)) { abort_flag = 1; atomicMax(p.status, DEV_WAIT_EXPIRED); ok = false; }
+            }
+            uint32_t it = 0, j = 0;
+            for (int64_t tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x, ++j) {
+                const uint32_t buf = j & 1;
+                if (!mbar_wait(&acc_empty[buf], ((j >> 1) & 1) ^ 1, &abort_flag)) { abort_flag = 1; atomicMax(p.status, DEV_WAIT_EXPIRED); ok = false; break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + buf * acc_stride;
+                for (int ks = 0; ks < nk; ++ks, ++it) {
+                    const int s = it % p.stages;
+                    const uint32_t ph = (it / p.stages) & 1;
+                    if (!mbar_wait(&full_bar[s], ph, &abort_flag)) { abort_flag = 1; atomicMax(p.status, DEV_WAIT_EXPIRED); ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t sa = smem_u32(smem_ring + (size_t)s * stage_bytes);
+                    const uint32_t sb = b_resident ? smem_u32(smem_b_res + (size_t)ks * b_bytes) : sa + a_bytes;
+#pragma unroll
+                    for (int k8 = 0; k8 < TC_BK / 8; ++k8)
+                        tc_mma_tf32(d_tmem, make_desc(sa + k8 * 32, 16, 1024, 2), make_desc(sb + k8 * 32, 16, 1024, 2), idesc,
+                                    (ks | k8) != 0 ? 1u : 0u);
+                    tc_commit(&empty_bar[s]);
+                }
+                if (ok) tc_commit(&acc_full[buf]);
+            }
+        }
+    } else {
+        // ---------------- epilogue: warp w reads TMEM lanes 32*(w&3).., 32-column chunks (w>>2), (w>>2)+2, ... ----------------
+        const int quarter = warp & 3, half = warp >> 2;
+        const bool generic = p.epi.drop != nullptr || p.epi.gate != nullptr || (p.epi.bias != nullptr && !bias_in_smem);
+        const bool add_bias = p.epi.bias != nullptr, relu = p.epi.relu != 0;
+        uint8_t* box = smem_out + (size_t)warp * 4096;
+        uint32_t j = 0;
+        bool ok = true;
+        for (int64_t tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x, ++j) {
+            const uint32_t buf = j & 1;
+            const int64_t m0 = (tile / p.n_tiles) * TC_BM;
+            const int n0 = (int)((tile % p.n_tiles) * p.bn);
+            if (lane == 0) ok = mbar_wait(&acc_full[buf], (j >> 1) & 1, &abort_flag);
+            ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
+            if (!ok) { if (lane == 0) { abort_flag = 1; atomicMax(p.status, DEV_WAIT_EXPIRED); } break; }
+            tc_fence_after();
+            const int64_t m = m0 + quarter * 32 + lane;
+            const bool row_ok = m < p.M;
+            for (int c0 = half * 32; c0 < p.bn; c0 += 64) {
+                uint32_t r[32];
+                tc_ld32(tmem_base + buf * acc_stride + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0, r);
+                tc_wait_ld();
+                const int nb = n0 + c0;
+                float v[32];
+#pragma unroll
+                for (int q = 0; q < 32; ++q) v[q] = __uint_as_float(r[q]);
+                if (!generic) {
+                    if (add_bias) {
+                        const float4* sb4 = reinterpret_cast<const float4*>(s_bias + nb);
+#pragma unroll
+                        for (int q = 0; q < 8; ++q) {
+                            const float4 b4 = sb4[q];
+                            v[4 * q] += b4.x; v[4 * q + 1] += b4.y; v[4 * q + 2] += b4.z; v[4 * q + 3] += b4.w;
+                        }
+                    }
+                    if (relu) {
+#pragma unroll
+                        for (int q = 0; q < 32; ++q) v[q] = fmaxf(v[q], 0.0f);
+                    }
+                } else if (row_ok) {
+#pragma unroll
+                    for (int q = 0; q < 32; ++q)
+                        if (nb + q < p.N) v[q] = tc_apply_epi(p.epi, v[q], m, nb + q, p.N);
+                }
+                if (tma_store) {
+                    // rows of 128 bytes in the 128-byte swizzle the tensor map expects: 16-byte chunk q of row r
+                    // lives at chunk position q ^ (r & 7).  The box is clipped to the matrix by the TMA unit.
+                    if (lane == 0) bulk_wait_read<0>();          // the store that last used this box has read it
+                    __syncwarp();
+#pragma unroll
+                    for (int q = 0; q < 8; ++q)
+                        *reinterpret_cast<float4*>(box + lane * 128 + ((q ^ (lane & 7)) << 4)) =
+                            make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0) {
+                        tma_store_2d(&map_c, box, nb, (int32_t)(m0 + quarter * 32));
+                        bulk_commit();
+                    }
+                } else if (row_ok) {
+                    float* dst = p.C + m * p.ldc + nb;
+                    if (p.vec_c && nb + 31 < p.N && c0 + 31 < p.bn) {
+#pragma unroll
+                        for (int q = 0; q < 32; q += 4)
+                            *reinterpret_cast<float4*>(dst + q) = make_float4(v[q], v[q + 1], v[q + 2], v[q + 3]);
+                    } else {
+#pragma unroll
+                        for (int q = 0; q < 32; ++q)
+                            if (nb + q < p.N && c0 + q < p.bn) dst[q] = v[q];
+                    }
+                }
+            }
+            // this warp is done reading the buffer: hand it back to the MMA issuer
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&acc_empty[buf]);
+        }
+        if (tma_store && lane == 0) bulk_wait_all();   // this warp's stores have completed before the CTA retires
+    }
+    if (threadIdx.x == 0 && abort_flag) {
+        for (int i = 0; i < 200; ++i) __nanosleep(1000);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == KK_EPI_WARPS + 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
+    }
+}
+
 // dst[n][k] = trans ? src[k][n] : src[n][k] for n < N, k < K, zero elsewhere; dst is rows x kpad.
 __global__ void pack_b_kernel(const float* __restrict__ src, int64_t ld, int trans, int N, int K, int rows, int kpad,
                               float* __restrict__ dst) {
@@ -406,9 +617,24 @@ mixgcn_status launch_gemm_tc(mixgcn_ctx* ctx, int ta, int tb, int64_t M, int64_t
             pack_b_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(B, ldb, tb ? 0 : 1, (int)N, (int)K, rows, kpad, packed);
         }
         p.splits = 1; p.k_per_split = K; p.raw = 0;
-        MIXGCN_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        // keep the packed weights resident in shared memory when they are small and there is one n-tile
+        const int nk = kpad / TC_BK;
+        const size_t b_all = (size_t)nk * bn32 * TC_BK * 4;
+        const int b_resident = (p.n_tiles == 1 && b_all <= 96 * 1024) ? 1 : 0;
+        const size_t stage = TC_BM * TC_BK * 4 + (b_resident ? 0 : (size_t)bn32 * TC_BK * 4);
+        const size_t budget = (b_resident ? 168 * 1024 - b_all : 160 * 1024);
+        int stages = (int)(budget / stage);
+        if (stages > 8) stages = 8;
+        if (stages < 2) stages = 2;
+        p.stages = stages;
+        const size_t smem_kk = (b_resident ? b_all : 0) + (size_t)stages * stage + 8 * 4096 + 1024;
+        const int tma_store = p.vec_c ? 1 : 0;
+        CUtensorMap map_c = map_a;
+        if (tma_store && !encode_2d(&map_c, C, N, M, ldc, 32, 32)) return MIXGCN_EUNSUPPORTED;
+        int64_t grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
+        MIXGCN_CUDA(cudaFuncSetAttribute(gemm_tc_kk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_kk));
         LaunchScope scope(ctx, PH_GEMM, s);
-        gemm_tc_kernel<false><<<dim3((unsigned)tiles, 1, 1), TC_THREADS, smem, s>>>(map_a, map_b, p);
+        gemm_tc_kk_kernel<<<dim3((unsigned)grid, 1, 1), KK_THREADS, smem_kk, s>>>(map_a, map_b, map_c, p, b_resident, tma_store);
         MIXGCN_CUDA(cudaGetLastError());
         return MIXGCN_OK;
     }

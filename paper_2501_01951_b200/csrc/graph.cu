@@ -108,13 +108,50 @@ __global__ void schedule_keys_kernel(int64_t n, const int64_t* __restrict__ rowp
     keys[u] = ((0x7FFFFFFFull - d) << 32) | (uint64_t)u;  // descending entries, ascending id
 }
 
+// perm from the sorted keys; counts[0] = rows longer than SPMM_SEG, counts[1..3] = rows longer than
+// SPMM_PACK_DEG[0..2] (one atomic per warp and counter; integers, so order does not matter).
 __global__ void schedule_finish_kernel(int64_t n, const uint64_t* __restrict__ keys, int32_t* __restrict__ perm,
-                                       int threshold, unsigned long long* n_hub) {
+                                       unsigned long long* counts) {
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    int64_t d = -1;
+    if (i < n) {
+        perm[i] = (int32_t)(uint32_t)(keys[i] & 0xFFFFFFFFull);
+        d = (int64_t)(0x7FFFFFFFull - (keys[i] >> 32));
+    }
+    const int thr[4] = {SPMM_SEG, SPMM_PACK_DEG[0], SPMM_PACK_DEG[1], SPMM_PACK_DEG[2]};
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        unsigned b = __ballot_sync(0xFFFFFFFFu, d > thr[q]);
+        if ((threadIdx.x & 31) == 0 && b) atomicAdd(counts + q, (unsigned long long)__popc(b));
+    }
+}
+
+__global__ void seg_count_kernel(int64_t n_long, const int32_t* __restrict__ perm, const int64_t* __restrict__ rowptr,
+                                 int64_t* __restrict__ cnt) {
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i > n_long) return;
+    if (i == n_long) { cnt[i] = 0; return; }
+    const int64_t u = perm[i];
+    cnt[i] = (rowptr[u + 1] - rowptr[u] + SPMM_SEG - 1) / SPMM_SEG;
+}
+
+__global__ void fill_records_kernel(int64_t n, int64_t n_long, int64_t total_segs, const int32_t* __restrict__ perm,
+                                    const int64_t* __restrict__ rowptr, const int64_t* __restrict__ seg_off,
+                                    SpmmRec* __restrict__ rec) {
     int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
-    perm[i] = (int32_t)(uint32_t)(keys[i] & 0xFFFFFFFFull);
-    int64_t d = (int64_t)(0x7FFFFFFFull - (keys[i] >> 32));
-    if (d > threshold) atomicAdd(n_hub, 1ull);
+    const int64_t u = perm[i];
+    const int64_t b = rowptr[u], e = rowptr[u + 1];
+    if (i < n_long) {
+        int64_t r = seg_off[i];
+        for (int64_t pos = b; pos < e; pos += SPMM_SEG, ++r) {
+            SpmmRec x; x.begin = pos; x.len = (int32_t)((e - pos) < SPMM_SEG ? (e - pos) : SPMM_SEG); x.row = (int32_t)i;
+            rec[r] = x;
+        }
+    } else {
+        SpmmRec x; x.begin = b; x.len = (int32_t)(e - b); x.row = (int32_t)u;
+        rec[total_segs + (i - n_long)] = x;
+    }
 }
 
 __global__ void validate_csr_kernel(int64_t n, int64_t nnz, const int64_t* __restrict__ rowptr,
@@ -140,7 +177,7 @@ struct DevBuf {  // frees on scope exit
 int bits_for(uint64_t x) { int b = 0; while (x) { ++b; x >>= 1; } return b; }
 
 void free_view(CsrView& v) {
-    cudaFree(v.rowptr); cudaFree(v.col); cudaFree(v.val); cudaFree(v.perm);
+    cudaFree(v.rowptr); cudaFree(v.col); cudaFree(v.val); cudaFree(v.perm); cudaFree(v.rec); cudaFree(v.seg_off);
     v = CsrView{};
 }
 
@@ -148,23 +185,40 @@ mixgcn_status build_schedule(int64_t n, CsrView& v, cudaStream_t s) {
     DevBuf k0, k1, tmp, hub;
     MIXGCN_CUDA(cudaMalloc(&k0.p, n * sizeof(uint64_t)));
     MIXGCN_CUDA(cudaMalloc(&k1.p, n * sizeof(uint64_t)));
-    MIXGCN_CUDA(cudaMalloc(&hub.p, sizeof(unsigned long long)));
-    MIXGCN_CUDA(cudaMemsetAsync(hub.p, 0, sizeof(unsigned long long), s));
+    MIXGCN_CUDA(cudaMalloc(&hub.p, 4 * sizeof(unsigned long long)));
+    MIXGCN_CUDA(cudaMemsetAsync(hub.p, 0, 4 * sizeof(unsigned long long), s));
     MIXGCN_CUDA(cudaMalloc((void**)&v.perm, n * sizeof(int32_t)));
     schedule_keys_kernel<<<blocks_for(n), TPB, 0, s>>>(n, v.rowptr, k0.as<uint64_t>());
     size_t tb = 0;
     MIXGCN_CUDA(cub::DeviceRadixSort::SortKeys(nullptr, tb, k0.as<uint64_t>(), k1.as<uint64_t>(), n, 0, 64, s));
     MIXGCN_CUDA(cudaMalloc(&tmp.p, tb ? tb : 1));
     MIXGCN_CUDA(cub::DeviceRadixSort::SortKeys(tmp.p, tb, k0.as<uint64_t>(), k1.as<uint64_t>(), n, 0, 64, s));
-    schedule_finish_kernel<<<blocks_for(n), TPB, 0, s>>>(n, k1.as<uint64_t>(), v.perm, HUB_THRESHOLD,
-                                                         hub.as<unsigned long long>());
-    unsigned long long h = 0;
+    schedule_finish_kernel<<<blocks_for(n), TPB, 0, s>>>(n, k1.as<uint64_t>(), v.perm, hub.as<unsigned long long>());
+    unsigned long long h[4] = {0, 0, 0, 0};
     uint64_t first = 0;
-    MIXGCN_CUDA(cudaMemcpyAsync(&h, hub.p, sizeof(h), cudaMemcpyDeviceToHost, s));
+    MIXGCN_CUDA(cudaMemcpyAsync(h, hub.p, sizeof(h), cudaMemcpyDeviceToHost, s));
     MIXGCN_CUDA(cudaMemcpyAsync(&first, k1.p, sizeof(first), cudaMemcpyDeviceToHost, s));
     MIXGCN_CUDA(cudaStreamSynchronize(s));
-    v.n_hub = (int64_t)h;
+    v.n_long = (int64_t)h[0];
+    for (int q = 0; q < 3; ++q) v.rows_above[q] = (int64_t)h[q + 1];
     v.max_deg = (int32_t)(0x7FFFFFFFull - (first >> 32));
+    // segment offsets of the long rows (exclusive scan of their segment counts)
+    DevBuf cnt, tmp2;
+    MIXGCN_CUDA(cudaMalloc(&cnt.p, (v.n_long + 1) * sizeof(int64_t)));
+    MIXGCN_CUDA(cudaMalloc((void**)&v.seg_off, (v.n_long + 1) * sizeof(int64_t)));
+    seg_count_kernel<<<blocks_for(v.n_long + 1), TPB, 0, s>>>(v.n_long, v.perm, v.rowptr, cnt.as<int64_t>());
+    size_t tb2 = 0;
+    MIXGCN_CUDA(cub::DeviceScan::ExclusiveSum(nullptr, tb2, cnt.as<int64_t>(), v.seg_off, v.n_long + 1, s));
+    MIXGCN_CUDA(cudaMalloc(&tmp2.p, tb2 ? tb2 : 1));
+    MIXGCN_CUDA(cub::DeviceScan::ExclusiveSum(tmp2.p, tb2, cnt.as<int64_t>(), v.seg_off, v.n_long + 1, s));
+    int64_t total = 0;
+    MIXGCN_CUDA(cudaMemcpyAsync(&total, v.seg_off + v.n_long, sizeof(int64_t), cudaMemcpyDeviceToHost, s));
+    MIXGCN_CUDA(cudaStreamSynchronize(s));
+    v.total_segs = total;
+    MIXGCN_CUDA(cudaMalloc((void**)&v.rec, (size_t)(total + n - v.n_long + 1) * sizeof(SpmmRec)));
+    fill_records_kernel<<<blocks_for(n), TPB, 0, s>>>(n, v.n_long, total, v.perm, v.rowptr, v.seg_off, v.rec);
+    MIXGCN_CUDA(cudaStreamSynchronize(s));
+    MIXGCN_CUDA(cudaGetLastError());
     return MIXGCN_OK;
 }
 

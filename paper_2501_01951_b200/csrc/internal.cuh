@@ -64,14 +64,28 @@ struct mixgcn_ctx {
     int64_t arena_bytes;
 };
 
+// One unit of aggregation work: `len` stored entries starting at `begin`.  For an ordinary row `row`
+// is the output row; for a segment of a long row it is the ordinal of that row among the long rows.
+struct __align__(16) SpmmRec {
+    int64_t begin;
+    int32_t len;
+    int32_t row;
+};
+
 // One CSR orientation of A_hat plus its aggregation schedule.
 struct CsrView {
     int64_t* rowptr;   // [n+1]
     int32_t* col;      // [nnz]
     float* val;        // [nnz]
     int32_t* perm;     // [n] rows by descending entry count
-    int64_t n_hub;     // first n_hub rows of perm have > HUB_THRESHOLD entries
     int32_t max_deg;
+    // schedule: rows longer than SPMM_SEG entries are cut into segments of SPMM_SEG (records
+    // [0, total_segs), long rows in perm order, segments in entry order); every other row is one
+    // record, in perm order (records [total_segs, total_segs + n - n_long)).
+    SpmmRec* rec;
+    int64_t n_long, total_segs;
+    int64_t* seg_off;          // [n_long+1] first segment record of each long row
+    int64_t rows_above[3];     // rows with more than SPMM_PACK_DEG[i] entries (bucket boundaries in perm order)
 };
 
 struct mixgcn_graph {
@@ -85,7 +99,8 @@ struct mixgcn_graph {
 
 namespace mixgcn {
 
-constexpr int HUB_THRESHOLD = 4096;  // rows longer than this get a whole CTA
+constexpr int SPMM_SEG = 512;                      // entries per segment of a long row
+constexpr int SPMM_PACK_DEG[3] = {12, 5, 2};       // rows up to these lengths share a warp 2-, 4-, 8-fold
 
 // Launch bookkeeping: counts the launch and, when profiling, brackets it with events.
 struct LaunchScope {

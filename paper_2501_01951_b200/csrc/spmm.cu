@@ -1,14 +1,19 @@
 // Neighbour aggregation Z = A_hat Y (Algorithm 2, aggregation line): deterministic, atomic-free,
 // row-wise CSR SpMM.
 //
-//  - A group of LPR lanes owns one output row; each lane owns VPL float4 column groups, so a
-//    gathered row of Y is read with coalesced 16-byte loads.
-//  - (col,val) of the row are fetched LPR at a time (one coalesced load per group) and handed
-//    round with warp shuffles; four gathered rows are in flight per lane before the FMAs.
-//  - Rows are taken in descending entry-count order (the graph's schedule), so the hardware
-//    block scheduler sees longest-first work; rows above HUB_THRESHOLD get a whole CTA whose
-//    warps split the row into contiguous segments and combine in fixed warp order.
-//  - Sums run over ascending column id inside a segment: the result is bit-reproducible.
+//  - A group of LPR lanes owns one output row (or one segment of a long row); each lane owns VPL
+//    float4 column groups, so a gathered row of Y is read with coalesced 16-byte loads.
+//  - The work list is the graph's schedule: one 16-byte record (first entry, length, row) per
+//    unit, longest first, so a unit starts after ONE dependent load instead of a chain through
+//    the permutation and the row pointers.
+//  - (col,val) of the unit are fetched LPR at a time (one coalesced load per group) and handed
+//    round with warp shuffles; U gathered rows (U * VPL = 8 float4 per lane) are in flight before
+//    the FMAs, with a predicated tail instead of a one-by-one remainder.
+//  - Degree buckets: rows of up to 12 / 5 / 2 entries share a warp 2- / 4- / 8-fold (fewer lanes per
+//    row, more float4 per lane), so short rows still keep eight loads per lane in flight.
+//  - Rows longer than SPMM_SEG entries are cut into segments that run as independent units and write
+//    partial rows to scratch; a second kernel adds the segments of each row in entry order and
+//    applies the epilogue.  Every sum has a fixed order: the result is bit-reproducible.
 //  - The epilogue (bias, ReLU, dropout mask, gate by another tensor's sign) is applied in
 //    registers before the single write of Z.
 #include "internal.cuh"
@@ -18,16 +23,18 @@ using namespace mixgcn;
 namespace {
 
 struct SpmmParams {
+    const SpmmRec* rec;    // schedule records, or null: unit idx is row idx of the CSR
     const int64_t* rowptr;
     const int32_t* col;
     const float* val;
-    const int32_t* perm;   // nullable: natural order
     int64_t idx_begin, idx_end;
     int32_t w;             // columns handled by this launch (slice width)
     int32_t j0;            // first column of the slice (multiple of 4)
     int32_t w_total;       // full width (for the dense drop-mask index)
     const float* Y; int64_t ldy;
     float* Z; int64_t ldz;
+    float* partial;        // non-null: unit idx writes its raw sums to partial[idx * ldp + ...]
+    int64_t ldp;
     // epilogue
     const float* bias; int relu;
     const uint8_t* drop; float keep_scale;
@@ -56,46 +63,45 @@ __device__ __forceinline__ void fma4(float4& acc, float a, const float4& y) {
     acc.z = fmaf(a, y.z, acc.z); acc.w = fmaf(a, y.w, acc.w);
 }
 
-// Accumulate entries [b, e) of one row into acc[] for the lane's column groups.
+template <int LPR, int VPL>
+struct Cfg {
+    static constexpr int U0 = 8 / VPL < 1 ? 1 : 8 / VPL;
+    static constexpr int U = U0 > LPR ? LPR : U0;   // gathered rows in flight per lane group
+};
+
+// Accumulate entries [b, e) into acc[] for the lane's column groups, ascending entry order.
 template <int LPR, int VPL>
 __device__ __forceinline__ void row_segment(const SpmmParams& p, int64_t b, int64_t e, int lig, unsigned mask,
                                             int w4, float4 (&acc)[VPL]) {
+    constexpr int U = Cfg<LPR, VPL>::U;
     const float* Yb = p.Y + p.j0;
     for (int64_t i0 = b; i0 < e; i0 += LPR) {
         int c = 0; float a = 0.0f;
         if (i0 + lig < e) { c = __ldg(p.col + i0 + lig); a = __ldg(p.val + i0 + lig); }
         const int cnt = (int)((e - i0) < LPR ? (e - i0) : LPR);
-        int k = 0;
-        for (; k + 4 <= cnt; k += 4) {
-            int ck[4]; float ak[4]; float4 y[4][VPL];
+        for (int k = 0; k < cnt; k += U) {
+            int ck[U]; float ak[U]; float4 y[U][VPL];
 #pragma unroll
-            for (int t = 0; t < 4; ++t) {
+            for (int t = 0; t < U; ++t) {
                 ck[t] = __shfl_sync(mask, c, k + t, LPR);
                 ak[t] = __shfl_sync(mask, a, k + t, LPR);
             }
 #pragma unroll
-            for (int t = 0; t < 4; ++t) {
+            for (int t = 0; t < U; ++t) {
                 const float4* yr = reinterpret_cast<const float4*>(Yb + (int64_t)ck[t] * p.ldy);
+                const bool live = k + t < cnt;
 #pragma unroll
                 for (int v = 0; v < VPL; ++v) {
                     const int c4 = lig + v * LPR;
-                    y[t][v] = (c4 < w4) ? __ldg(yr + c4) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    y[t][v] = (live && c4 < w4) ? __ldg(yr + c4) : make_float4(0.f, 0.f, 0.f, 0.f);
                 }
             }
 #pragma unroll
-            for (int t = 0; t < 4; ++t)
+            for (int t = 0; t < U; ++t)
+                if (k + t < cnt) {
 #pragma unroll
-                for (int v = 0; v < VPL; ++v) fma4(acc[v], ak[t], y[t][v]);
-        }
-        for (; k < cnt; ++k) {
-            const int c1 = __shfl_sync(mask, c, k, LPR);
-            const float a1 = __shfl_sync(mask, a, k, LPR);
-            const float4* yr = reinterpret_cast<const float4*>(Yb + (int64_t)c1 * p.ldy);
-#pragma unroll
-            for (int v = 0; v < VPL; ++v) {
-                const int c4 = lig + v * LPR;
-                if (c4 < w4) fma4(acc[v], a1, __ldg(yr + c4));
-            }
+                    for (int v = 0; v < VPL; ++v) fma4(acc[v], ak[t], y[t][v]);
+                }
         }
     }
 }
@@ -106,12 +112,31 @@ __global__ void __launch_bounds__(256) spmm_group_kernel(const SpmmParams p) {
     const int64_t idx = p.idx_begin + ((int64_t)blockIdx.x * 256 + threadIdx.x) / LPR;
     if (idx >= p.idx_end) return;  // the whole group leaves together
     const unsigned mask = LPR == 32 ? 0xFFFFFFFFu : (((1u << LPR) - 1u) << ((threadIdx.x & 31) & ~(LPR - 1)));
-    const int64_t u = p.perm ? (int64_t)__ldg(p.perm + idx) : idx;
+    int64_t b, e, u;
+    if (p.rec) {
+        const int4 r = __ldg(reinterpret_cast<const int4*>(p.rec + idx));
+        b = ((int64_t)(uint32_t)r.y << 32) | (uint32_t)r.x;
+        e = b + r.z;
+        u = r.w;
+    } else {
+        u = idx;
+        b = __ldg(p.rowptr + u);
+        e = __ldg(p.rowptr + u + 1);
+    }
     const int w4 = (p.w + 3) >> 2;
     float4 acc[VPL];
 #pragma unroll
     for (int v = 0; v < VPL; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
-    row_segment<LPR, VPL>(p, __ldg(p.rowptr + u), __ldg(p.rowptr + u + 1), lig, mask, w4, acc);
+    row_segment<LPR, VPL>(p, b, e, lig, mask, w4, acc);
+    if (p.partial) {
+        float4* dst = reinterpret_cast<float4*>(p.partial + idx * p.ldp);
+#pragma unroll
+        for (int v = 0; v < VPL; ++v) {
+            const int c4 = lig + v * LPR;
+            if (c4 < w4) dst[c4] = acc[v];
+        }
+        return;
+    }
 #pragma unroll
     for (int v = 0; v < VPL; ++v) {
         const int c4 = lig + v * LPR;
@@ -119,34 +144,21 @@ __global__ void __launch_bounds__(256) spmm_group_kernel(const SpmmParams p) {
     }
 }
 
-// One CTA (8 warps) per long row.
-template <int VPL>
-__global__ void __launch_bounds__(256) spmm_hub_kernel(const SpmmParams p) {
-    extern __shared__ float4 part[];  // [8][w4]
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int64_t idx = p.idx_begin + blockIdx.x;
-    const int64_t u = p.perm ? (int64_t)__ldg(p.perm + idx) : idx;
+// Long rows: add the segments' partial rows in entry order, apply the epilogue, write Z.
+// One group of 32 lanes per long row.
+__global__ void __launch_bounds__(256) spmm_combine_kernel(const SpmmParams p, int64_t n_long,
+                                                           const int64_t* __restrict__ seg_off,
+                                                           const int32_t* __restrict__ perm) {
+    const int lane = threadIdx.x & 31;
+    const int64_t i = ((int64_t)blockIdx.x * 256 + threadIdx.x) >> 5;
+    if (i >= n_long) return;
+    const int64_t s0 = seg_off[i], s1 = seg_off[i + 1];
+    const int64_t u = perm[i];
     const int w4 = (p.w + 3) >> 2;
-    const int64_t b = __ldg(p.rowptr + u), e = __ldg(p.rowptr + u + 1);
-    // contiguous segments, multiples of 32 entries so that every segment starts group-aligned
-    int64_t per = ((e - b + 8 * 32 - 1) / (8 * 32)) * 32;
-    int64_t sb = b + warp * per, se = sb + per;
-    if (sb > e) sb = e;
-    if (se > e) se = e;
-    float4 acc[VPL];
-#pragma unroll
-    for (int v = 0; v < VPL; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
-    row_segment<32, VPL>(p, sb, se, lane, 0xFFFFFFFFu, w4, acc);
-#pragma unroll
-    for (int v = 0; v < VPL; ++v) {
-        const int c4 = lane + v * 32;
-        if (c4 < w4) part[warp * w4 + c4] = acc[v];
-    }
-    __syncthreads();
-    for (int c4 = threadIdx.x; c4 < w4; c4 += 256) {
-        float4 s = part[c4];
-        for (int wq = 1; wq < 8; ++wq) {  // fixed order
-            float4 t = part[wq * w4 + c4];
+    for (int c4 = lane; c4 < w4; c4 += 32) {
+        float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int64_t q = s0; q < s1; ++q) {
+            const float4 t = __ldg(reinterpret_cast<const float4*>(p.partial + q * p.ldp) + c4);
             s.x += t.x; s.y += t.y; s.z += t.z; s.w += t.w;
         }
         store_row(p, u, c4, s);
@@ -155,52 +167,32 @@ __global__ void __launch_bounds__(256) spmm_hub_kernel(const SpmmParams p) {
 
 template <int LPR, int VPL>
 void launch_group(const SpmmParams& p, cudaStream_t s) {
-    const int64_t rows = p.idx_end - p.idx_begin;
-    if (rows <= 0) return;
-    const int rows_per_block = 256 / LPR;
-    const int64_t blocks = (rows + rows_per_block - 1) / rows_per_block;
+    const int64_t units = p.idx_end - p.idx_begin;
+    if (units <= 0) return;
+    const int per_block = 256 / LPR;
+    const int64_t blocks = (units + per_block - 1) / per_block;
     spmm_group_kernel<LPR, VPL><<<(unsigned)blocks, 256, 0, s>>>(p);
 }
 
-template <int VPL>
-void launch_hub(const SpmmParams& p, cudaStream_t s) {
-    const int64_t rows = p.idx_end - p.idx_begin;
-    if (rows <= 0) return;
+// Base configuration for a slice of w4 float4 columns, then packed `fold`-fold (fold in {1,2,4,8}):
+// fewer lanes per row, more float4 per lane.  Returns the fold actually used.
+int dispatch(const SpmmParams& p, int fold, cudaStream_t s) {
     const int w4 = (p.w + 3) >> 2;
-    spmm_hub_kernel<VPL><<<(unsigned)rows, 256, 8 * w4 * sizeof(float4), s>>>(p);
-}
-
-void dispatch_group(const SpmmParams& p, cudaStream_t s) {
-    const int w4 = (p.w + 3) >> 2;
-    if (w4 <= 1) return launch_group<1, 1>(p, s);
-    if (w4 <= 2) return launch_group<2, 1>(p, s);
-    if (w4 <= 4) return launch_group<4, 1>(p, s);
-    if (w4 <= 8) return launch_group<8, 1>(p, s);
-    if (w4 <= 16) return launch_group<16, 1>(p, s);
-    switch ((w4 + 31) / 32) {
-        case 1: return launch_group<32, 1>(p, s);
-        case 2: return launch_group<32, 2>(p, s);
-        case 3: return launch_group<32, 3>(p, s);
-        case 4: return launch_group<32, 4>(p, s);
-        case 5: return launch_group<32, 5>(p, s);
-        case 6: return launch_group<32, 6>(p, s);
-        case 7: return launch_group<32, 7>(p, s);
-        default: return launch_group<32, 8>(p, s);
-    }
-}
-
-void dispatch_hub(const SpmmParams& p, cudaStream_t s) {
-    const int w4 = (p.w + 3) >> 2;
-    switch ((w4 + 31) / 32) {
-        case 1: return launch_hub<1>(p, s);
-        case 2: return launch_hub<2>(p, s);
-        case 3: return launch_hub<3>(p, s);
-        case 4: return launch_hub<4>(p, s);
-        case 5: return launch_hub<5>(p, s);
-        case 6: return launch_hub<6>(p, s);
-        case 7: return launch_hub<7>(p, s);
-        default: return launch_hub<8>(p, s);
-    }
+    int lpr = 1;
+    while (lpr < 32 && lpr < w4) lpr <<= 1;
+    int vpl = (w4 + lpr - 1) / lpr;
+    while (fold > 1 && (lpr / fold < 1 || vpl * fold > 8)) fold >>= 1;
+    lpr /= fold; vpl *= fold;
+#define MIXGCN_SPMM_CASE(L, V) if (lpr == L && vpl == V) { launch_group<L, V>(p, s); return fold; }
+    MIXGCN_SPMM_CASE(32, 1) MIXGCN_SPMM_CASE(32, 2) MIXGCN_SPMM_CASE(32, 3) MIXGCN_SPMM_CASE(32, 4)
+    MIXGCN_SPMM_CASE(32, 5) MIXGCN_SPMM_CASE(32, 6) MIXGCN_SPMM_CASE(32, 7) MIXGCN_SPMM_CASE(32, 8)
+    MIXGCN_SPMM_CASE(16, 1) MIXGCN_SPMM_CASE(16, 2) MIXGCN_SPMM_CASE(16, 4) MIXGCN_SPMM_CASE(16, 6) MIXGCN_SPMM_CASE(16, 8)
+    MIXGCN_SPMM_CASE(8, 1) MIXGCN_SPMM_CASE(8, 2) MIXGCN_SPMM_CASE(8, 4) MIXGCN_SPMM_CASE(8, 8)
+    MIXGCN_SPMM_CASE(4, 1) MIXGCN_SPMM_CASE(4, 2) MIXGCN_SPMM_CASE(4, 4) MIXGCN_SPMM_CASE(4, 8)
+    MIXGCN_SPMM_CASE(2, 1) MIXGCN_SPMM_CASE(2, 2) MIXGCN_SPMM_CASE(2, 4) MIXGCN_SPMM_CASE(2, 8)
+    MIXGCN_SPMM_CASE(1, 1) MIXGCN_SPMM_CASE(1, 2) MIXGCN_SPMM_CASE(1, 4) MIXGCN_SPMM_CASE(1, 8)
+#undef MIXGCN_SPMM_CASE
+    return 0;
 }
 
 constexpr int MAX_SLICE = 1024;  // columns per launch: 8 float4 per lane
@@ -209,8 +201,9 @@ constexpr int MAX_SLICE = 1024;  // columns per launch: 8 float4 per lane
 
 namespace mixgcn {
 
-// Rows [row_begin, row_end): when the range is the whole matrix the degree-sorted schedule is
-// used (hub rows first); a partial range (pipeline chunk) runs in natural row order.
+// Rows [row_begin, row_end): when the range is the whole matrix the schedule is used (long rows as
+// segments, then rows longest first, short rows packed); a partial range (pipeline chunk) runs in
+// natural row order without scratch.
 mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView& A, int64_t row_begin,
                           int64_t row_end, int32_t w, const float* Y, int64_t ldy, float* Z, int64_t ldz,
                           const mixgcn_epilogue* epi, cudaStream_t s) {
@@ -226,22 +219,45 @@ mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView&
     for (int j0 = 0; j0 < w; j0 += MAX_SLICE) {
         p.j0 = j0;
         p.w = (w - j0) < MAX_SLICE ? (w - j0) : MAX_SLICE;
-        if (whole) {
-            p.perm = A.perm;
-            if (A.n_hub > 0) {
-                LaunchScope scope(ctx, PH_SPMM, s);
-                p.idx_begin = 0; p.idx_end = A.n_hub;
-                dispatch_hub(p, s);
-            }
-            if (A.n_hub < g->n) {
-                LaunchScope scope(ctx, PH_SPMM, s);
-                p.idx_begin = A.n_hub; p.idx_end = g->n;
-                dispatch_group(p, s);
-            }
-        } else {
+        if (!whole) {
             LaunchScope scope(ctx, PH_SPMM, s);
-            p.perm = nullptr; p.idx_begin = row_begin; p.idx_end = row_end;
-            dispatch_group(p, s);
+            p.rec = nullptr; p.partial = nullptr; p.idx_begin = row_begin; p.idx_end = row_end;
+            dispatch(p, 1, s);
+            continue;
+        }
+        p.rec = A.rec;
+        if (A.total_segs > 0) {
+            const int64_t ldp = ((int64_t)p.w + 3) / 4 * 4;
+            MIXGCN_TRY(ensure_workspace(ctx, A.total_segs * ldp * (int64_t)sizeof(float)));
+            p.partial = reinterpret_cast<float*>(ctx->workspace); p.ldp = ldp;
+            {
+                LaunchScope scope(ctx, PH_SPMM, s);
+                p.idx_begin = 0; p.idx_end = A.total_segs;
+                dispatch(p, 1, s);
+            }
+            {
+                LaunchScope scope(ctx, PH_SPMM, s);
+                const int64_t blocks = (A.n_long * 32 + 255) / 256;
+                spmm_combine_kernel<<<(unsigned)blocks, 256, 0, s>>>(p, A.n_long, A.seg_off, A.perm);
+            }
+            p.partial = nullptr;
+        }
+        // ordinary rows, in perm order: [n_long, n) -> records [total_segs, total_segs + n - n_long)
+        int64_t bound[5];
+        bound[0] = A.n_long;
+        for (int q = 0; q < 3; ++q) bound[q + 1] = A.rows_above[q] > A.n_long ? A.rows_above[q] : A.n_long;
+        bound[4] = g->n;
+        int64_t begin = bound[0];
+        int fold = 1;
+        for (int q = 0; q < 4; ++q, fold <<= 1) {
+            // a bucket whose fold is not available for this width is merged into the next launch range
+            int64_t end = bound[q + 1];
+            if (end <= begin) continue;
+            p.idx_begin = A.total_segs + (begin - A.n_long);
+            p.idx_end = A.total_segs + (end - A.n_long);
+            LaunchScope scope(ctx, PH_SPMM, s);
+            dispatch(p, fold, s);
+            begin = end;
         }
     }
     MIXGCN_CUDA(cudaGetLastError());
