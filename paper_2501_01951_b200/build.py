@@ -21,7 +21,7 @@ LIB = os.path.join(HERE, "libmixgcn.so")
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
 CFLAGS = ["-O3", "-std=c++17", "-lineinfo", "-Xcompiler", "-fPIC",
-          "-I", INCLUDE, "-I", CSRC, "--expt-relaxed-constexpr"]
+          "-I", INCLUDE, "-I", CSRC, "--expt-relaxed-constexpr"] + os.environ.get("MIXGCN_NVCC_FLAGS", "").split()
 
 
 def sources():

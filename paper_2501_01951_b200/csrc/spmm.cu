@@ -20,6 +20,13 @@
 
 using namespace mixgcn;
 
+#ifndef MIXGCN_SPMM_MINB
+#define MIXGCN_SPMM_MINB 1
+#endif
+#ifndef MIXGCN_SPMM_U
+#define MIXGCN_SPMM_U 8
+#endif
+
 namespace {
 
 struct SpmmParams {
@@ -65,7 +72,7 @@ __device__ __forceinline__ void fma4(float4& acc, float a, const float4& y) {
 
 template <int LPR, int VPL>
 struct Cfg {
-    static constexpr int U0 = 8 / VPL < 1 ? 1 : 8 / VPL;
+    static constexpr int U0 = MIXGCN_SPMM_U / VPL < 1 ? 1 : MIXGCN_SPMM_U / VPL;
     static constexpr int U = U0 > LPR ? LPR : U0;   // gathered rows in flight per lane group
 };
 
@@ -107,7 +114,7 @@ __device__ __forceinline__ void row_segment(const SpmmParams& p, int64_t b, int6
 }
 
 template <int LPR, int VPL>
-__global__ void __launch_bounds__(256) spmm_group_kernel(const SpmmParams p) {
+__global__ void __launch_bounds__(256, MIXGCN_SPMM_MINB) spmm_group_kernel(const SpmmParams p) {
     const int lig = threadIdx.x % LPR;
     const int64_t idx = p.idx_begin + ((int64_t)blockIdx.x * 256 + threadIdx.x) / LPR;
     if (idx >= p.idx_end) return;  // the whole group leaves together

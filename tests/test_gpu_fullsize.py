@@ -1,0 +1,208 @@
+"""Parity at the workloads' full sizes, in the launch configuration bench.py times.
+
+The oracle cannot run a whole epoch at these sizes in test time, so every operation is checked
+teacher-forced on sampled outputs the oracle computes one by one (the GPU's own input to that
+operation is copied to the host for the sampled rows), plus properties that hold at any size
+(A_hat sqrt(deg~) = sqrt(deg~); weight gradients probed with random vectors).  Expected values
+come from the oracle or from the definition evaluated with numpy on the generator's edge list."""
+import numpy as np
+import pytest
+import torch
+
+from helpers import TOL_FP32, TOL_LOWP, round4
+from oracle import gcn_oracle as orc
+from paper_2501_01951_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+N_SAMPLE = 192
+
+
+@pytest.fixture(scope="module")
+def mg():
+    from paper_2501_01951_b200 import build
+    build.build()
+    from paper_2501_01951_b200 import binding
+    return binding
+
+
+def _sample_rows(n, deg, seed):
+    """Random rows plus the longest rows and a few rows with a single entry."""
+    rng = np.random.default_rng(seed)
+    rows = set(rng.integers(0, n, N_SAMPLE).tolist())
+    order = np.argsort(deg)
+    rows.update(order[-4:].tolist())
+    rows.update(order[:4].tolist())
+    return np.array(sorted(rows), dtype=np.int64)
+
+
+def _sub_oracle_graph(n, src, dst, rows):
+    """Oracle rows of A_hat for `rows`, from the definition on the generator's unique undirected
+    edge list: neighbours of u are the endpoints of its edges plus u; deg~ = 1 + incident edges.
+    Returns a compact oracle Graph over the nodes involved and the map compact id -> node id."""
+    deg = (np.bincount(src, minlength=n) + np.bincount(dst, minlength=n) + 1).astype(np.int64)
+    sel = np.isin(src, rows) | np.isin(dst, rows)
+    s, d = src[sel], dst[sel]
+    nodes = np.unique(np.concatenate([rows, s, d]))
+    look = lambda x: np.searchsorted(nodes, x).astype(np.int64)       # nodes is sorted and contains every id looked up
+    g = orc.graph_build(len(nodes), look(s), look(d))
+    # the compact graph knows only the sampled rows' edges; overwrite its values with the full-graph degrees
+    r_of = np.repeat(np.arange(g.n), np.diff(g.rowptr))
+    g.val = 1.0 / np.sqrt(deg[nodes[r_of]].astype(np.float64) * deg[nodes[g.col]].astype(np.float64))
+    return g, nodes, look(rows), deg
+
+
+def _run_workload(mg, key, precision):
+    from paper_2501_01951_b200.train import GcnTrainer
+    wl = synth.CONFIGS[key]
+    dev = torch.device("cuda", 0)
+    ctx = mg.ctx_create(0)
+    src, dst = synth.rmat_graph(wl.n, wl.undirected_edges, wl.seed("graph"), device=dev)
+    g = mg.graph_create(ctx, wl.n, src, dst)
+    src_h, dst_h = src.cpu().numpy(), dst.cpu().numpy()
+    del src, dst
+    torch.cuda.empty_cache()
+    tr = GcnTrainer(ctx, g, wl.dims, precision)
+    X0 = synth.normal_features(wl.n, wl.dims[0], wl.seed("features"), device=dev, ld=round4(wl.dims[0]))
+    y = synth.uniform_labels(wl.n, wl.classes, wl.seed("labels"), device=dev)
+    m = synth.bernoulli_mask(wl.n, wl.mask_p, wl.seed("mask"), device=dev)
+    Ws, bs = synth.make_weights(wl, device=dev)
+    bs = [synth.uniform_tensor((b.numel(),), 77 + i, -0.1, 0.1, device=dev) for i, b in enumerate(bs)]   # exercise the bias path
+    tr.set_params(Ws, bs)
+    tr.set_inputs(X0, y, m)
+    return wl, ctx, g, tr, src_h, dst_h
+
+
+def _rel(a, b):
+    return float(np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-300))
+
+
+@pytest.mark.parametrize("key", ["C2", "C3", "C4", "C5"])
+def test_full_size_workload(mg, key):
+    wl = synth.CONFIGS[key]
+    free, _ = torch.cuda.mem_get_info()
+    dims = [round4(d) for d in wl.dims]
+    cols = sum(dims) + sum(max(dims[l], dims[l + 1]) for l in range(len(dims) - 1)) + max(dims[1:-1])
+    need = 4 * wl.n * cols + 36 * wl.undirected_edges
+    if free < need * 1.03:
+        pytest.skip(f"needs ~{need / 2**30:.0f} GiB of device memory")
+    prec = mg.PRECISIONS[wl.precision]
+    tol = TOL_FP32 if prec == mg.PREC_FP32 else TOL_LOWP
+    wl, ctx, g, tr, src_h, dst_h = _run_workload(mg, key, prec)
+    n, L = wl.n, tr.L
+    assert g.symmetric and g.n == n and g.nnz == 2 * len(src_h) + n
+
+    # ---- S0: sampled rows of the CSR, bit-exact, against the definition on the edge list
+    ex = mg.graph_export(g)
+    deg_gpu = ex["deg"].numpy()
+    rows = _sample_rows(n, deg_gpu, 1)
+    sub, nodes, crow, deg = _sub_oracle_graph(n, src_h, dst_h, rows)
+    assert np.array_equal(deg_gpu, deg.astype(np.int32)) and g.max_deg == int(deg.max())
+    dinv = (np.float32(1.0) / np.sqrt(deg.astype(np.float32))).astype(np.float32)
+    assert ex["dinv"].numpy().tobytes() == dinv.tobytes()
+    rp, col, val = ex["rowptr"].numpy(), ex["col"].numpy(), ex["val"].numpy()
+    for u, cu in zip(rows, crow):
+        want_cols = nodes[sub.col[sub.rowptr[cu]:sub.rowptr[cu + 1]]]
+        got = col[rp[u]:rp[u + 1]]
+        assert np.array_equal(got, want_cols)
+        assert np.array_equal(val[rp[u]:rp[u + 1]], (dinv[u] * dinv[got]).astype(np.float32))
+    del ex, rp, col, val
+
+    def rows_of(t, idx, d):
+        return t[torch.as_tensor(idx, device=t.device)][:, :d].cpu().numpy().astype(np.float64)
+
+    def check_spmm(Y, Z, w, what):
+        Ysub = rows_of(Y, nodes, w)                                  # the operation's own input, sampled
+        want = orc.aggregate_rows(sub, Ysub, crow)
+        assert _rel(rows_of(Z, rows, w), want) <= TOL_FP32, what
+
+    # ---- forward, layer by layer, teacher-forced on sampled rows
+    tr.forward()
+    torch.cuda.synchronize()
+    assert mg.ctx_poll_status(ctx, raise_on_error=False) == 0
+    for l in range(L):
+        d_in, d_out = wl.dims[l], wl.dims[l + 1]
+        W, b = tr.W[l].cpu().numpy(), tr.b[l].cpu().numpy()
+        last = l == L - 1
+        if tr.orders[l] == mg.ORDER_AGG_FIRST:
+            check_spmm(tr.X[l], tr.saved[l], d_in, f"layer {l} aggregation")
+            P = orc.update(rows_of(tr.saved[l], rows, d_in), W, b)
+            want = P if last else orc.activation(P)
+            assert _rel(rows_of(tr.X[l + 1], rows, d_out), want) <= tol, f"layer {l} update"
+        else:
+            Q = orc.update(rows_of(tr.X[l], rows, d_in), W)
+            assert _rel(rows_of(tr.saved[l], rows, d_out), Q) <= tol, f"layer {l} update (first)"
+            P = orc.aggregate_rows(sub, rows_of(tr.saved[l], nodes, d_out), crow) + b
+            want = P if last else orc.activation(P)
+            assert _rel(rows_of(tr.X[l + 1], rows, d_out), want) <= TOL_FP32, f"layer {l} aggregation (second)"
+
+    # ---- property at full scale: sqrt(deg~) is a fixed point of the aggregation (symmetric graph)
+    R = torch.zeros(n, 4, device="cuda")
+    R[:, 0] = torch.sqrt(torch.as_tensor(deg, device="cuda", dtype=torch.float32))
+    Zr = torch.zeros_like(R)
+    mg.spmm(ctx, g, R, Zr, 1)
+    assert float(torch.linalg.norm(Zr[:, 0] - R[:, 0]) / torch.linalg.norm(R[:, 0])) <= TOL_FP32
+    del R, Zr
+
+    # ---- loss on all train rows (they are few enough to copy), gradient on sampled rows
+    C = wl.classes
+    train_idx = torch.nonzero(tr.train_mask).flatten()
+    logits_train = tr.X[L][train_idx][:, :C].cpu().numpy().astype(np.float64)
+    labels_train = tr.labels[train_idx].cpu().numpy()
+    lo, Gt, pred_t, nc, T = orc.loss(logits_train, labels_train, np.ones(len(labels_train), np.uint8))
+    logits_rows = rows_of(tr.X[L], rows, C)
+    tr.compute_loss()
+    torch.cuda.synchronize()
+    assert abs(tr.loss.item() - lo) <= 2e-6 * abs(lo)
+    assert int(tr.n_correct.item()) == nc
+    assert np.array_equal(tr.pred[train_idx].cpu().numpy(), pred_t)                       # arg-max: bit-exact
+    assert np.array_equal(tr.pred[torch.as_tensor(rows, device="cuda")].cpu().numpy(), logits_rows.argmax(axis=1))
+    pick = np.random.default_rng(2).integers(0, len(train_idx), 64)
+    got = tr.X[L][train_idx[torch.as_tensor(pick, device="cuda")]][:, :C].cpu().numpy()
+    assert _rel(got, Gt[pick]) <= TOL_FP32
+    untrained = torch.nonzero(tr.train_mask == 0).flatten()[:1000]
+    assert float(tr.X[L][untrained][:, :C].abs().max()) == 0.0
+
+    # ---- backward of the last layer: dW, db probed with random vectors; input gradient on sampled rows
+    l = L - 1
+    d_in, d_out = wl.dims[l], wl.dims[l + 1]
+    agg_first = tr.orders[l] == mg.ORDER_AGG_FIRST
+    rng = np.random.default_rng(3)
+    a = torch.as_tensor(rng.standard_normal(d_in), device="cuda", dtype=torch.float64)
+    bv = torch.as_tensor(rng.standard_normal(d_out), device="cuda", dtype=torch.float64)
+
+    def probe(lhs, rhs):
+        """a^T (lhs^T rhs) b = sum_k (lhs a)_k (rhs b)_k and 1^T rhs b, in fp64 by chunks (torch, not this library)."""
+        val, colsum, scale = 0.0, 0.0, 0.0
+        step = 1 << 20
+        for r0 in range(0, n, step):
+            za = lhs[r0:r0 + step, :d_in].double() @ a
+            gb = rhs[r0:r0 + step, :d_out].double() @ bv
+            val += float(za @ gb); scale += float(za.abs() @ gb.abs()); colsum += float(gb.sum())
+        return val, colsum, scale
+
+    dP_nodes = rows_of(tr.G[L], nodes, d_out)                      # gradient w.r.t. the logits, rows the sample needs
+    if agg_first:
+        want_probe, want_db, scale = probe(tr.saved[l], tr.G[L])    # before the call: it consumes `saved`
+    tr.backward()
+    torch.cuda.synchronize()
+    assert mg.ctx_poll_status(ctx, raise_on_error=False) == 0
+    Wt = tr.W[l].cpu().numpy().T.copy()
+    gate = rows_of(tr.X[l], rows, d_in) > 0
+    if agg_first:
+        # G_in = gate(A_hat^T (dP W^T)); symmetric graph: A_hat^T = A_hat
+        want_gin = orc.aggregate_rows(sub, orc.update(dP_nodes, Wt), crow)
+        assert _rel(rows_of(tr.G[l], rows, d_in), want_gin * gate) <= tol
+    else:
+        # dQ = A_hat^T dP is left in `saved`; dW = X_in^T dQ; G_in = gate(dQ W^T)
+        want_dq = orc.aggregate_rows(sub, dP_nodes, crow)
+        assert _rel(rows_of(tr.saved[l], rows, d_out), want_dq) <= TOL_FP32
+        want_probe, _, scale = probe(tr.X[l], tr.saved[l])
+        _, want_db, _ = probe(tr.X[l], tr.G[L])
+        assert _rel(rows_of(tr.G[l], rows, d_in), orc.update(rows_of(tr.saved[l], rows, d_out), Wt) * gate) <= tol
+    assert abs(float(a @ tr.dW[l].double() @ bv) - want_probe) <= tol * scale
+    assert abs(float(tr.db[l].double() @ bv) - want_db) <= tol * scale + 1e-12
+    for t in tr.dW + tr.db:
+        assert bool(torch.isfinite(t).all())
+    g.close()
+    ctx.close()
