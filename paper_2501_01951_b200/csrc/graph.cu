@@ -126,32 +126,99 @@ __global__ void schedule_finish_kernel(int64_t n, const uint64_t* __restrict__ k
     }
 }
 
-__global__ void seg_count_kernel(int64_t n_long, const int32_t* __restrict__ perm, const int64_t* __restrict__ rowptr,
-                                 int64_t* __restrict__ cnt) {
-    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i > n_long) return;
-    if (i == n_long) { cnt[i] = 0; return; }
-    const int64_t u = perm[i];
-    cnt[i] = (rowptr[u + 1] - rowptr[u] + SPMM_SEG - 1) / SPMM_SEG;
+// Long rows are cut at dyadic column-block boundaries (and every SPMM_SEG entries): a row with d
+// entries uses 2^k blocks, the largest k <= SPMM_MAX_LOG_BLOCKS with d / 2^k >= SPMM_BLK_MIN_ENTRIES.
+__device__ __forceinline__ int row_log_blocks(int64_t d) {
+    int k = 0;
+    while (k < SPMM_MAX_LOG_BLOCKS && (d >> (k + 1)) >= SPMM_BLK_MIN_ENTRIES) ++k;
+    return k;
 }
 
-__global__ void fill_records_kernel(int64_t n, int64_t n_long, int64_t total_segs, const int32_t* __restrict__ perm,
-                                    const int64_t* __restrict__ rowptr, const int64_t* __restrict__ seg_off,
-                                    SpmmRec* __restrict__ rec) {
+__global__ void blk_count_kernel(int64_t n_long, const int32_t* __restrict__ perm, const int64_t* __restrict__ rowptr,
+                                 int64_t* __restrict__ nblk) {
     int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= n) return;
+    if (i > n_long) return;
+    if (i == n_long) { nblk[i] = 0; return; }
     const int64_t u = perm[i];
-    const int64_t b = rowptr[u], e = rowptr[u + 1];
-    if (i < n_long) {
-        int64_t r = seg_off[i];
-        for (int64_t pos = b; pos < e; pos += SPMM_SEG, ++r) {
-            SpmmRec x; x.begin = pos; x.len = (int32_t)((e - pos) < SPMM_SEG ? (e - pos) : SPMM_SEG); x.row = (int32_t)i;
-            rec[r] = x;
-        }
-    } else {
-        SpmmRec x; x.begin = b; x.len = (int32_t)(e - b); x.row = (int32_t)u;
-        rec[total_segs + (i - n_long)] = x;
+    nblk[i] = (int64_t)1 << row_log_blocks(rowptr[u + 1] - rowptr[u]);
+}
+
+__device__ __forceinline__ int64_t lower_bound_col(const int32_t* __restrict__ col, int64_t lo, int64_t hi, int64_t key) {
+    while (lo < hi) {
+        const int64_t mid = (lo + hi) >> 1;
+        if ((int64_t)col[mid] < key) lo = mid + 1; else hi = mid;
     }
+    return lo;
+}
+
+// largest i with off[i] <= t  (off is ascending, off[0] = 0, off[count] > t)
+__device__ __forceinline__ int64_t owner_of(const int64_t* __restrict__ off, int64_t count, int64_t t) {
+    int64_t lo = 0, hi = count;
+    while (hi - lo > 1) {
+        const int64_t mid = (lo + hi) >> 1;
+        if (off[mid] <= t) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+// One thread per (long row, column block) pair: the entries of the row inside the block and how many
+// segments they need.
+__global__ void pair_segments_kernel(int64_t n, int64_t n_long, int64_t total_pairs, const int32_t* __restrict__ perm,
+                                     const int64_t* __restrict__ rowptr, const int32_t* __restrict__ col,
+                                     const int64_t* __restrict__ blk_off, int64_t* __restrict__ pair_lo,
+                                     int64_t* __restrict__ pair_cnt, int64_t* __restrict__ pair_segs) {
+    int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t > total_pairs) return;
+    if (t == total_pairs) { pair_segs[t] = 0; return; }
+    const int64_t i = owner_of(blk_off, n_long, t);
+    const int64_t b = t - blk_off[i], nb = blk_off[i + 1] - blk_off[i];
+    const int64_t u = perm[i];
+    const int64_t rb = rowptr[u], re = rowptr[u + 1];
+    const int64_t width = (n + nb - 1) / nb;
+    const int64_t lo = lower_bound_col(col, rb, re, b * width);
+    const int64_t hi = lower_bound_col(col, lo, re, (b + 1) * width);
+    pair_lo[t] = lo;
+    pair_cnt[t] = hi - lo;
+    pair_segs[t] = (hi - lo + SPMM_SEG - 1) / SPMM_SEG;
+}
+
+__global__ void seg_fill_kernel(int64_t n_long, int64_t total_pairs, const int32_t* __restrict__ col,
+                                const int64_t* __restrict__ blk_off, const int64_t* __restrict__ pair_lo,
+                                const int64_t* __restrict__ pair_cnt, const int64_t* __restrict__ pair_seg_off,
+                                SpmmRec* __restrict__ rec_tmp, uint32_t* __restrict__ keys, uint32_t* __restrict__ ids,
+                                int64_t* __restrict__ seg_off) {
+    int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= total_pairs) return;
+    const int64_t i = owner_of(blk_off, n_long, t);
+    if (t == blk_off[i]) seg_off[i] = pair_seg_off[t];
+    if (t == total_pairs - 1) seg_off[n_long] = pair_seg_off[total_pairs];
+    int64_t q = pair_seg_off[t];
+    const int64_t lo = pair_lo[t], hi = lo + pair_cnt[t];
+    for (int64_t pos = lo; pos < hi; pos += SPMM_SEG, ++q) {
+        SpmmRec x; x.begin = pos; x.len = (int32_t)((hi - pos) < SPMM_SEG ? (hi - pos) : SPMM_SEG); x.row = (int32_t)i;
+        rec_tmp[q] = x;
+        keys[q] = (uint32_t)col[pos];      // segments run in order of their first column
+        ids[q] = (uint32_t)q;
+    }
+}
+
+__global__ void seg_place_kernel(int64_t total_segs, const uint32_t* __restrict__ order, const SpmmRec* __restrict__ rec_tmp,
+                                 SpmmRec* __restrict__ rec, int64_t* __restrict__ seg_pos) {
+    int64_t pos = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (pos >= total_segs) return;
+    const uint32_t q = order[pos];
+    rec[pos] = rec_tmp[q];
+    seg_pos[q] = pos;
+}
+
+// Ordinary rows: one record each, in perm order, after the segment records.
+__global__ void fill_records_kernel(int64_t n, int64_t n_long, int64_t total_segs, const int32_t* __restrict__ perm,
+                                    const int64_t* __restrict__ rowptr, SpmmRec* __restrict__ rec) {
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n || i < n_long) return;
+    const int64_t u = perm[i];
+    SpmmRec x; x.begin = rowptr[u]; x.len = (int32_t)(rowptr[u + 1] - rowptr[u]); x.row = (int32_t)u;
+    rec[total_segs + (i - n_long)] = x;
 }
 
 __global__ void validate_csr_kernel(int64_t n, int64_t nnz, const int64_t* __restrict__ rowptr,
@@ -177,7 +244,7 @@ struct DevBuf {  // frees on scope exit
 int bits_for(uint64_t x) { int b = 0; while (x) { ++b; x >>= 1; } return b; }
 
 void free_view(CsrView& v) {
-    cudaFree(v.rowptr); cudaFree(v.col); cudaFree(v.val); cudaFree(v.perm); cudaFree(v.rec); cudaFree(v.seg_off);
+    cudaFree(v.rowptr); cudaFree(v.col); cudaFree(v.val); cudaFree(v.perm); cudaFree(v.rec); cudaFree(v.seg_off); cudaFree(v.seg_pos);
     v = CsrView{};
 }
 
@@ -202,21 +269,61 @@ mixgcn_status build_schedule(int64_t n, CsrView& v, cudaStream_t s) {
     v.n_long = (int64_t)h[0];
     for (int q = 0; q < 3; ++q) v.rows_above[q] = (int64_t)h[q + 1];
     v.max_deg = (int32_t)(0x7FFFFFFFull - (first >> 32));
-    // segment offsets of the long rows (exclusive scan of their segment counts)
-    DevBuf cnt, tmp2;
-    MIXGCN_CUDA(cudaMalloc(&cnt.p, (v.n_long + 1) * sizeof(int64_t)));
-    MIXGCN_CUDA(cudaMalloc((void**)&v.seg_off, (v.n_long + 1) * sizeof(int64_t)));
-    seg_count_kernel<<<blocks_for(v.n_long + 1), TPB, 0, s>>>(v.n_long, v.perm, v.rowptr, cnt.as<int64_t>());
+    // long rows -> (row, column block) pairs -> segments, ordered by their first column
+    const int64_t nl = v.n_long;
+    DevBuf nblk, blk_off, tmp2;
+    MIXGCN_CUDA(cudaMalloc(&nblk.p, (nl + 1) * sizeof(int64_t)));
+    MIXGCN_CUDA(cudaMalloc(&blk_off.p, (nl + 1) * sizeof(int64_t)));
+    MIXGCN_CUDA(cudaMalloc((void**)&v.seg_off, (nl + 1) * sizeof(int64_t)));
+    MIXGCN_CUDA(cudaMemsetAsync(v.seg_off, 0, (nl + 1) * sizeof(int64_t), s));
+    blk_count_kernel<<<blocks_for(nl + 1), TPB, 0, s>>>(nl, v.perm, v.rowptr, nblk.as<int64_t>());
     size_t tb2 = 0;
-    MIXGCN_CUDA(cub::DeviceScan::ExclusiveSum(nullptr, tb2, cnt.as<int64_t>(), v.seg_off, v.n_long + 1, s));
+    MIXGCN_CUDA(cub::DeviceScan::ExclusiveSum(nullptr, tb2, nblk.as<int64_t>(), blk_off.as<int64_t>(), nl + 1, s));
     MIXGCN_CUDA(cudaMalloc(&tmp2.p, tb2 ? tb2 : 1));
-    MIXGCN_CUDA(cub::DeviceScan::ExclusiveSum(tmp2.p, tb2, cnt.as<int64_t>(), v.seg_off, v.n_long + 1, s));
-    int64_t total = 0;
-    MIXGCN_CUDA(cudaMemcpyAsync(&total, v.seg_off + v.n_long, sizeof(int64_t), cudaMemcpyDeviceToHost, s));
+    MIXGCN_CUDA(cub::DeviceScan::ExclusiveSum(tmp2.p, tb2, nblk.as<int64_t>(), blk_off.as<int64_t>(), nl + 1, s));
+    int64_t total_pairs = 0;
+    MIXGCN_CUDA(cudaMemcpyAsync(&total_pairs, blk_off.as<int64_t>() + nl, sizeof(int64_t), cudaMemcpyDeviceToHost, s));
     MIXGCN_CUDA(cudaStreamSynchronize(s));
+    int64_t total = 0;
+    DevBuf pair_lo, pair_cnt, pair_segs, pair_seg_off, tmp3, rec_tmp, keys0, keys1, ids0, ids1, tmp4;
+    if (total_pairs > 0) {
+        MIXGCN_CUDA(cudaMalloc(&pair_lo.p, total_pairs * sizeof(int64_t)));
+        MIXGCN_CUDA(cudaMalloc(&pair_cnt.p, total_pairs * sizeof(int64_t)));
+        MIXGCN_CUDA(cudaMalloc(&pair_segs.p, (total_pairs + 1) * sizeof(int64_t)));
+        MIXGCN_CUDA(cudaMalloc(&pair_seg_off.p, (total_pairs + 1) * sizeof(int64_t)));
+        pair_segments_kernel<<<blocks_for(total_pairs + 1), TPB, 0, s>>>(n, nl, total_pairs, v.perm, v.rowptr, v.col,
+                                                                        blk_off.as<int64_t>(), pair_lo.as<int64_t>(),
+                                                                        pair_cnt.as<int64_t>(), pair_segs.as<int64_t>());
+        size_t tb3 = 0;
+        MIXGCN_CUDA(cub::DeviceScan::ExclusiveSum(nullptr, tb3, pair_segs.as<int64_t>(), pair_seg_off.as<int64_t>(), total_pairs + 1, s));
+        MIXGCN_CUDA(cudaMalloc(&tmp3.p, tb3 ? tb3 : 1));
+        MIXGCN_CUDA(cub::DeviceScan::ExclusiveSum(tmp3.p, tb3, pair_segs.as<int64_t>(), pair_seg_off.as<int64_t>(), total_pairs + 1, s));
+        MIXGCN_CUDA(cudaMemcpyAsync(&total, pair_seg_off.as<int64_t>() + total_pairs, sizeof(int64_t), cudaMemcpyDeviceToHost, s));
+        MIXGCN_CUDA(cudaStreamSynchronize(s));
+    }
+    if (total >= 0xFFFFFFFFll) MIXGCN_FAIL(MIXGCN_EUNSUPPORTED, "graph schedule: too many long-row segments (%lld)", (long long)total);
     v.total_segs = total;
-    MIXGCN_CUDA(cudaMalloc((void**)&v.rec, (size_t)(total + n - v.n_long + 1) * sizeof(SpmmRec)));
-    fill_records_kernel<<<blocks_for(n), TPB, 0, s>>>(n, v.n_long, total, v.perm, v.rowptr, v.seg_off, v.rec);
+    MIXGCN_CUDA(cudaMalloc((void**)&v.rec, (size_t)(total + n - nl + 1) * sizeof(SpmmRec)));
+    MIXGCN_CUDA(cudaMalloc((void**)&v.seg_pos, (size_t)(total + 1) * sizeof(int64_t)));
+    if (total > 0) {
+        MIXGCN_CUDA(cudaMalloc(&rec_tmp.p, total * sizeof(SpmmRec)));
+        MIXGCN_CUDA(cudaMalloc(&keys0.p, total * sizeof(uint32_t)));
+        MIXGCN_CUDA(cudaMalloc(&keys1.p, total * sizeof(uint32_t)));
+        MIXGCN_CUDA(cudaMalloc(&ids0.p, total * sizeof(uint32_t)));
+        MIXGCN_CUDA(cudaMalloc(&ids1.p, total * sizeof(uint32_t)));
+        seg_fill_kernel<<<blocks_for(total_pairs), TPB, 0, s>>>(nl, total_pairs, v.col, blk_off.as<int64_t>(), pair_lo.as<int64_t>(),
+                                                               pair_cnt.as<int64_t>(), pair_seg_off.as<int64_t>(),
+                                                               rec_tmp.as<SpmmRec>(), keys0.as<uint32_t>(), ids0.as<uint32_t>(),
+                                                               v.seg_off);
+        size_t tb4 = 0;
+        MIXGCN_CUDA(cub::DeviceRadixSort::SortPairs(nullptr, tb4, keys0.as<uint32_t>(), keys1.as<uint32_t>(), ids0.as<uint32_t>(),
+                                                    ids1.as<uint32_t>(), total, 0, 32, s));
+        MIXGCN_CUDA(cudaMalloc(&tmp4.p, tb4 ? tb4 : 1));
+        MIXGCN_CUDA(cub::DeviceRadixSort::SortPairs(tmp4.p, tb4, keys0.as<uint32_t>(), keys1.as<uint32_t>(), ids0.as<uint32_t>(),
+                                                    ids1.as<uint32_t>(), total, 0, 32, s));
+        seg_place_kernel<<<blocks_for(total), TPB, 0, s>>>(total, ids1.as<uint32_t>(), rec_tmp.as<SpmmRec>(), v.rec, v.seg_pos);
+    }
+    fill_records_kernel<<<blocks_for(n), TPB, 0, s>>>(n, nl, total, v.perm, v.rowptr, v.rec);
     MIXGCN_CUDA(cudaStreamSynchronize(s));
     MIXGCN_CUDA(cudaGetLastError());
     return MIXGCN_OK;

@@ -79,12 +79,15 @@ struct CsrView {
     float* val;        // [nnz]
     int32_t* perm;     // [n] rows by descending entry count
     int32_t max_deg;
-    // schedule: rows longer than SPMM_SEG entries are cut into segments of SPMM_SEG (records
-    // [0, total_segs), long rows in perm order, segments in entry order); every other row is one
-    // record, in perm order (records [total_segs, total_segs + n - n_long)).
+    // schedule: rows longer than SPMM_SEG entries are cut into segments at dyadic column-block
+    // boundaries and every SPMM_SEG entries; the segment records [0, total_segs) run in order of
+    // their first column, so that segments of different long rows that gather the same rows of Y run
+    // close in time (those rows are then served by the L2).  Every other row is one record, in perm
+    // order (records [total_segs, total_segs + n - n_long)).
     SpmmRec* rec;
     int64_t n_long, total_segs;
-    int64_t* seg_off;          // [n_long+1] first segment record of each long row
+    int64_t* seg_off;          // [n_long+1] segments of long row i are numbered seg_off[i] .. seg_off[i+1]-1 in entry order
+    int64_t* seg_pos;          // [total_segs] record position (= partial-row slot) of segment number q
     int64_t rows_above[3];     // rows with more than SPMM_PACK_DEG[i] entries (bucket boundaries in perm order)
 };
 
@@ -99,7 +102,18 @@ struct mixgcn_graph {
 
 namespace mixgcn {
 
-constexpr int SPMM_SEG = 512;                      // entries per segment of a long row
+#ifndef MIXGCN_SPMM_SEG
+#define MIXGCN_SPMM_SEG 512
+#endif
+#ifndef MIXGCN_SPMM_BLK_MIN
+#define MIXGCN_SPMM_BLK_MIN 64
+#endif
+#ifndef MIXGCN_SPMM_LOG_BLOCKS
+#define MIXGCN_SPMM_LOG_BLOCKS 8
+#endif
+constexpr int SPMM_SEG = MIXGCN_SPMM_SEG;                 // rows longer than this are cut into segments of at most this many entries
+constexpr int SPMM_BLK_MIN_ENTRIES = MIXGCN_SPMM_BLK_MIN; // a long row uses 2^k column blocks while it keeps >= this many entries per block
+constexpr int SPMM_MAX_LOG_BLOCKS = MIXGCN_SPMM_LOG_BLOCKS; // at most 2^this column blocks per row
 constexpr int SPMM_PACK_DEG[3] = {12, 5, 2};       // rows up to these lengths share a warp 2-, 4-, 8-fold
 
 // Launch bookkeeping: counts the launch and, when profiling, brackets it with events.

@@ -11,9 +11,11 @@
 //    the FMAs, with a predicated tail instead of a one-by-one remainder.
 //  - Degree buckets: rows of up to 12 / 5 / 2 entries share a warp 2- / 4- / 8-fold (fewer lanes per
 //    row, more float4 per lane), so short rows still keep eight loads per lane in flight.
-//  - Rows longer than SPMM_SEG entries are cut into segments that run as independent units and write
-//    partial rows to scratch; a second kernel adds the segments of each row in entry order and
-//    applies the epilogue.  Every sum has a fixed order: the result is bit-reproducible.
+//  - Rows longer than SPMM_SEG entries are cut (at column-block boundaries and every SPMM_SEG
+//    entries) into segments that run as independent units, in order of their first column, and
+//    write partial rows to scratch: hub rows that gather the same rows of Y do so close in time
+//    and share them through the L2.  A second kernel adds the segments of each row in entry order
+//    and applies the epilogue.  Every sum has a fixed order: the result is bit-reproducible.
 //  - The epilogue (bias, ReLU, dropout mask, gate by another tensor's sign) is applied in
 //    registers before the single write of Z.
 #include "internal.cuh"
@@ -155,6 +157,7 @@ __global__ void __launch_bounds__(256, MIXGCN_SPMM_MINB) spmm_group_kernel(const
 // One group of 32 lanes per long row.
 __global__ void __launch_bounds__(256) spmm_combine_kernel(const SpmmParams p, int64_t n_long,
                                                            const int64_t* __restrict__ seg_off,
+                                                           const int64_t* __restrict__ seg_pos,
                                                            const int32_t* __restrict__ perm) {
     const int lane = threadIdx.x & 31;
     const int64_t i = ((int64_t)blockIdx.x * 256 + threadIdx.x) >> 5;
@@ -165,7 +168,7 @@ __global__ void __launch_bounds__(256) spmm_combine_kernel(const SpmmParams p, i
     for (int c4 = lane; c4 < w4; c4 += 32) {
         float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
         for (int64_t q = s0; q < s1; ++q) {
-            const float4 t = __ldg(reinterpret_cast<const float4*>(p.partial + q * p.ldp) + c4);
+            const float4 t = __ldg(reinterpret_cast<const float4*>(p.partial + __ldg(seg_pos + q) * p.ldp) + c4);
             s.x += t.x; s.y += t.y; s.z += t.z; s.w += t.w;
         }
         store_row(p, u, c4, s);
@@ -245,7 +248,7 @@ mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView&
             {
                 LaunchScope scope(ctx, PH_SPMM, s);
                 const int64_t blocks = (A.n_long * 32 + 255) / 256;
-                spmm_combine_kernel<<<(unsigned)blocks, 256, 0, s>>>(p, A.n_long, A.seg_off, A.perm);
+                spmm_combine_kernel<<<(unsigned)blocks, 256, 0, s>>>(p, A.n_long, A.seg_off, A.seg_pos, A.perm);
             }
             p.partial = nullptr;
         }

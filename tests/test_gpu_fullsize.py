@@ -80,6 +80,7 @@ def _rel(a, b):
 @pytest.mark.parametrize("key", ["C2", "C3", "C4", "C5"])
 def test_full_size_workload(mg, key):
     wl = synth.CONFIGS[key]
+    torch.cuda.empty_cache()
     free, _ = torch.cuda.mem_get_info()
     dims = [round4(d) for d in wl.dims]
     cols = sum(dims) + sum(max(dims[l], dims[l + 1]) for l in range(len(dims) - 1)) + max(dims[1:-1])
