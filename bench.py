@@ -34,6 +34,11 @@ import torch
 
 from paper_2501_01951_b200 import synth
 
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of ONE aggregation call at the workload's
+# size and width, from the ncu capture summarised in profiles/spmm_C5_dram_traffic.md (every
+# aggregation of C5 has width 128 and the same graph, so the figure holds for each of its calls).
+NCU_SPMM_CALL_DRAM_BYTES = {"C5": 136767976704}
+
 METRIC = "full-graph GCN train epochs/s"
 UNIT = "epochs/s"
 
@@ -203,7 +208,7 @@ def run_ours(args, rank, world, local_rank):
     achieved = alg_bytes / (spmm_ms / 1e3) / 1e9 if spmm_ms > 0 else 0.0
     roofline = dict(bound="hbm", kernel="spmm (aggregation)", achieved=round(achieved, 1), peak=peaks["hbm_gbs"],
                     unit="GB/s", frac=round(achieved / peaks["hbm_gbs"], 4), peak_source=peaks["source"],
-                    traffic=None, calls=spmm_calls, avg_call_ms=round(spmm_ms / max(spmm_calls, 1), 4),
+                    traffic=NCU_SPMM_CALL_DRAM_BYTES.get(args.workload), calls=spmm_calls, avg_call_ms=round(spmm_ms / max(spmm_calls, 1), 4),
                     alg_bytes_per_call=int(alg_bytes / max(spmm_calls, 1)),
                     gather_gbs=round(sum(4 * nnz * w * k for w, k in plan) * args.steps / (spmm_ms / 1e3) / 1e9, 1) if spmm_ms > 0 else 0.0)
     flops = gemm_flops(n, wl.dims, tr.orders) * args.steps
