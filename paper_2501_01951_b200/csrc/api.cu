@@ -65,6 +65,22 @@ mixgcn_status ensure_workspace(mixgcn_ctx* ctx, int64_t bytes) {
     return MIXGCN_OK;
 }
 
+mixgcn_status ensure_workspace_spmm(mixgcn_ctx* ctx, int64_t bytes) {
+    if (bytes <= ctx->workspace_spmm_bytes) return MIXGCN_OK;
+    int64_t want = bytes + (bytes >> 2);
+    want = (want + 255) & ~(int64_t)255;
+    void* p = nullptr;
+    MIXGCN_CUDA(cudaDeviceSynchronize());
+    if (ctx->workspace_spmm) cudaFree(ctx->workspace_spmm);
+    ctx->workspace_spmm = nullptr; ctx->workspace_spmm_bytes = 0;
+    if (cudaMalloc(&p, (size_t)want) != cudaSuccess) {
+        cudaGetLastError();
+        MIXGCN_FAIL(MIXGCN_ENOMEM, "aggregation workspace of %lld bytes could not be allocated", (long long)want);
+    }
+    ctx->workspace_spmm = p; ctx->workspace_spmm_bytes = want;
+    return MIXGCN_OK;
+}
+
 mixgcn_status launch_gemm_simt(mixgcn_ctx* ctx, int ta, int tb, int64_t M, int64_t N, int64_t K,
                                const float* A, int64_t lda, const float* B, int64_t ldb, float* C, int64_t ldc,
                                const mixgcn_epilogue* epi, int64_t epi_row0, cudaStream_t s);
@@ -141,6 +157,7 @@ extern "C" mixgcn_status mixgcn_ctx_destroy(mixgcn_ctx* ctx) {
     for (int i = 0; i < 2; ++i) { if (ctx->join_ev[i]) cudaEventDestroy(ctx->join_ev[i]); if (ctx->side_stream[i]) cudaStreamDestroy(ctx->side_stream[i]); }
     if (ctx->fork_ev) cudaEventDestroy(ctx->fork_ev);
     cudaFree(ctx->workspace);
+    cudaFree(ctx->workspace_spmm);
     cudaFree(ctx->arena);
     cudaFree(ctx->d_status);
     delete ctx;
@@ -269,12 +286,13 @@ extern "C" mixgcn_status mixgcn_layer_fwd(mixgcn_ctx* ctx, const mixgcn_graph* g
 
     if (order == MIXGCN_ORDER_AGG_FIRST) {
         if (chunks == 1) {
-            MIXGCN_TRY(launch_spmm(ctx, g, g->fwd, 0, n, d->d_in, X_in, d->ld_in, saved, d->ld_saved, nullptr, s));
+            MIXGCN_TRY(launch_spmm(ctx, g, g->fwd, 1, 0, d->d_in, X_in, d->ld_in, saved, d->ld_saved, nullptr, s));
             MIXGCN_TRY(launch_gemm(ctx, d->precision, 0, 0, n, d->d_out, d->d_in, saved, d->ld_saved, W, ldw, X_out,
                                    d->ld_out, &epi, 0, s));
             return MIXGCN_OK;
         }
         // aggregation of chunk k+1 on stream A overlaps the update of chunk k on stream B
+        MIXGCN_TRY(ensure_chunk_schedules(g, g->fwd, chunks));
         cudaStream_t sa = ctx->side_stream[0], sb = ctx->side_stream[1];
         MIXGCN_CUDA(cudaEventRecord(ctx->fork_ev, s));
         MIXGCN_CUDA(cudaStreamWaitEvent(sa, ctx->fork_ev, 0));
@@ -282,7 +300,7 @@ extern "C" mixgcn_status mixgcn_layer_fwd(mixgcn_ctx* ctx, const mixgcn_graph* g
         for (int k = 0; k < chunks; ++k) {
             const int64_t r0 = chunk_bound(n, k, chunks), r1 = chunk_bound(n, k + 1, chunks);
             if (r1 <= r0) continue;
-            MIXGCN_TRY(launch_spmm(ctx, g, g->fwd, r0, r1, d->d_in, X_in, d->ld_in, saved, d->ld_saved, nullptr, sa));
+            MIXGCN_TRY(launch_spmm(ctx, g, g->fwd, chunks, k, d->d_in, X_in, d->ld_in, saved, d->ld_saved, nullptr, sa));
             MIXGCN_CUDA(cudaEventRecord(ctx->chunk_ev[k], sa));
             MIXGCN_CUDA(cudaStreamWaitEvent(sb, ctx->chunk_ev[k], 0));
             MIXGCN_TRY(launch_gemm(ctx, d->precision, 0, 0, r1 - r0, d->d_out, d->d_in, saved + r0 * d->ld_saved,
@@ -298,7 +316,7 @@ extern "C" mixgcn_status mixgcn_layer_fwd(mixgcn_ctx* ctx, const mixgcn_graph* g
     // needed before any aggregated row can be produced, so there is nothing to chunk here.
     MIXGCN_TRY(launch_gemm(ctx, d->precision, 0, 0, n, d->d_out, d->d_in, X_in, d->ld_in, W, ldw, saved, d->ld_saved,
                            nullptr, 0, s));
-    MIXGCN_TRY(launch_spmm(ctx, g, g->fwd, 0, n, d->d_out, saved, d->ld_saved, X_out, d->ld_out, &epi, s));
+    MIXGCN_TRY(launch_spmm(ctx, g, g->fwd, 1, 0, d->d_out, saved, d->ld_saved, X_out, d->ld_out, &epi, s));
     return MIXGCN_OK;
 }
 
@@ -339,12 +357,12 @@ extern "C" mixgcn_status mixgcn_layer_bwd(mixgcn_ctx* ctx, const mixgcn_graph* g
         if (!first) {
             MIXGCN_TRY(launch_gemm(ctx, d->precision, 0, 1, n, d->d_in, d->d_out, G_out, d->ld_out, W, ldw, saved,
                                    d->ld_saved, nullptr, 0, s));
-            MIXGCN_TRY(launch_spmm(ctx, g, g->bwd, 0, n, d->d_in, saved, d->ld_saved, G_in, d->ld_in, gin, s));
+            MIXGCN_TRY(launch_spmm(ctx, g, g->bwd, 1, 0, d->d_in, saved, d->ld_saved, G_in, d->ld_in, gin, s));
         }
         return MIXGCN_OK;
     }
     // update first: dQ = A_hat^T dZ (into `saved`) ; dW = X_in^T dQ ; G_in = dQ W^T
-    MIXGCN_TRY(launch_spmm(ctx, g, g->bwd, 0, n, d->d_out, G_out, d->ld_out, saved, d->ld_saved, nullptr, s));
+    MIXGCN_TRY(launch_spmm(ctx, g, g->bwd, 1, 0, d->d_out, G_out, d->ld_out, saved, d->ld_saved, nullptr, s));
     MIXGCN_TRY(launch_gemm(ctx, d->precision, 1, 0, d->d_in, d->d_out, n, X_in, d->ld_in, saved, d->ld_saved, dW, ldw,
                            nullptr, 0, s));
     if (!first)

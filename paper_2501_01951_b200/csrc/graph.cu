@@ -101,11 +101,13 @@ __global__ void transpose_keys_kernel(int64_t n, const int64_t* __restrict__ row
         keys[i] = ((uint64_t)(uint32_t)col[i] << 32) | (uint32_t)u;
 }
 
-__global__ void schedule_keys_kernel(int64_t n, const int64_t* __restrict__ rowptr, uint64_t* __restrict__ keys) {
-    int64_t u = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (u >= n) return;
+__global__ void schedule_keys_kernel(int64_t row0, int64_t n_rows, const int64_t* __restrict__ rowptr,
+                                     uint64_t* __restrict__ keys) {
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n_rows) return;
+    const int64_t u = row0 + i;
     uint64_t d = (uint64_t)(rowptr[u + 1] - rowptr[u]);
-    keys[u] = ((0x7FFFFFFFull - d) << 32) | (uint64_t)u;  // descending entries, ascending id
+    keys[i] = ((0x7FFFFFFFull - d) << 32) | (uint64_t)u;  // descending entries, ascending id
 }
 
 // perm from the sorted keys; counts[0] = rows longer than SPMM_SEG, counts[1..3] = rows longer than
@@ -243,19 +245,32 @@ struct DevBuf {  // frees on scope exit
 
 int bits_for(uint64_t x) { int b = 0; while (x) { ++b; x >>= 1; } return b; }
 
+void free_schedule(SpmmSchedule& v) {
+    cudaFree(v.perm); cudaFree(v.rec); cudaFree(v.seg_off); cudaFree(v.seg_pos);
+    v = SpmmSchedule{};
+}
+
 void free_view(CsrView& v) {
-    cudaFree(v.rowptr); cudaFree(v.col); cudaFree(v.val); cudaFree(v.perm); cudaFree(v.rec); cudaFree(v.seg_off); cudaFree(v.seg_pos);
+    cudaFree(v.rowptr); cudaFree(v.col); cudaFree(v.val);
+    free_schedule(v.full);
+    for (int k = 0; k < v.n_chunk; ++k) free_schedule(v.chunk[k]);
+    delete[] v.chunk;
     v = CsrView{};
 }
 
-mixgcn_status build_schedule(int64_t n, CsrView& v, cudaStream_t s) {
+// Schedule of rows [row0, row0 + n) of the CSR (rowptr, col) of a matrix with n_total columns.
+mixgcn_status build_schedule(int64_t n_total, const int64_t* rowptr, const int32_t* col, int64_t row0, int64_t n,
+                             SpmmSchedule& v, cudaStream_t s) {
+    v = SpmmSchedule{};
+    v.row0 = row0; v.n_rows = n;
+    if (n <= 0) return MIXGCN_OK;
     DevBuf k0, k1, tmp, hub;
     MIXGCN_CUDA(cudaMalloc(&k0.p, n * sizeof(uint64_t)));
     MIXGCN_CUDA(cudaMalloc(&k1.p, n * sizeof(uint64_t)));
     MIXGCN_CUDA(cudaMalloc(&hub.p, 4 * sizeof(unsigned long long)));
     MIXGCN_CUDA(cudaMemsetAsync(hub.p, 0, 4 * sizeof(unsigned long long), s));
     MIXGCN_CUDA(cudaMalloc((void**)&v.perm, n * sizeof(int32_t)));
-    schedule_keys_kernel<<<blocks_for(n), TPB, 0, s>>>(n, v.rowptr, k0.as<uint64_t>());
+    schedule_keys_kernel<<<blocks_for(n), TPB, 0, s>>>(row0, n, rowptr, k0.as<uint64_t>());
     size_t tb = 0;
     MIXGCN_CUDA(cub::DeviceRadixSort::SortKeys(nullptr, tb, k0.as<uint64_t>(), k1.as<uint64_t>(), n, 0, 64, s));
     MIXGCN_CUDA(cudaMalloc(&tmp.p, tb ? tb : 1));
@@ -276,7 +291,7 @@ mixgcn_status build_schedule(int64_t n, CsrView& v, cudaStream_t s) {
     MIXGCN_CUDA(cudaMalloc(&blk_off.p, (nl + 1) * sizeof(int64_t)));
     MIXGCN_CUDA(cudaMalloc((void**)&v.seg_off, (nl + 1) * sizeof(int64_t)));
     MIXGCN_CUDA(cudaMemsetAsync(v.seg_off, 0, (nl + 1) * sizeof(int64_t), s));
-    blk_count_kernel<<<blocks_for(nl + 1), TPB, 0, s>>>(nl, v.perm, v.rowptr, nblk.as<int64_t>());
+    blk_count_kernel<<<blocks_for(nl + 1), TPB, 0, s>>>(nl, v.perm, rowptr, nblk.as<int64_t>());
     size_t tb2 = 0;
     MIXGCN_CUDA(cub::DeviceScan::ExclusiveSum(nullptr, tb2, nblk.as<int64_t>(), blk_off.as<int64_t>(), nl + 1, s));
     MIXGCN_CUDA(cudaMalloc(&tmp2.p, tb2 ? tb2 : 1));
@@ -291,7 +306,7 @@ mixgcn_status build_schedule(int64_t n, CsrView& v, cudaStream_t s) {
         MIXGCN_CUDA(cudaMalloc(&pair_cnt.p, total_pairs * sizeof(int64_t)));
         MIXGCN_CUDA(cudaMalloc(&pair_segs.p, (total_pairs + 1) * sizeof(int64_t)));
         MIXGCN_CUDA(cudaMalloc(&pair_seg_off.p, (total_pairs + 1) * sizeof(int64_t)));
-        pair_segments_kernel<<<blocks_for(total_pairs + 1), TPB, 0, s>>>(n, nl, total_pairs, v.perm, v.rowptr, v.col,
+        pair_segments_kernel<<<blocks_for(total_pairs + 1), TPB, 0, s>>>(n_total, nl, total_pairs, v.perm, rowptr, col,
                                                                         blk_off.as<int64_t>(), pair_lo.as<int64_t>(),
                                                                         pair_cnt.as<int64_t>(), pair_segs.as<int64_t>());
         size_t tb3 = 0;
@@ -311,7 +326,7 @@ mixgcn_status build_schedule(int64_t n, CsrView& v, cudaStream_t s) {
         MIXGCN_CUDA(cudaMalloc(&keys1.p, total * sizeof(uint32_t)));
         MIXGCN_CUDA(cudaMalloc(&ids0.p, total * sizeof(uint32_t)));
         MIXGCN_CUDA(cudaMalloc(&ids1.p, total * sizeof(uint32_t)));
-        seg_fill_kernel<<<blocks_for(total_pairs), TPB, 0, s>>>(nl, total_pairs, v.col, blk_off.as<int64_t>(), pair_lo.as<int64_t>(),
+        seg_fill_kernel<<<blocks_for(total_pairs), TPB, 0, s>>>(nl, total_pairs, col, blk_off.as<int64_t>(), pair_lo.as<int64_t>(),
                                                                pair_cnt.as<int64_t>(), pair_seg_off.as<int64_t>(),
                                                                rec_tmp.as<SpmmRec>(), keys0.as<uint32_t>(), ids0.as<uint32_t>(),
                                                                v.seg_off);
@@ -323,7 +338,7 @@ mixgcn_status build_schedule(int64_t n, CsrView& v, cudaStream_t s) {
                                                     ids1.as<uint32_t>(), total, 0, 32, s));
         seg_place_kernel<<<blocks_for(total), TPB, 0, s>>>(total, ids1.as<uint32_t>(), rec_tmp.as<SpmmRec>(), v.rec, v.seg_pos);
     }
-    fill_records_kernel<<<blocks_for(n), TPB, 0, s>>>(n, nl, total, v.perm, v.rowptr, v.rec);
+    fill_records_kernel<<<blocks_for(n), TPB, 0, s>>>(n, nl, total, v.perm, rowptr, v.rec);
     MIXGCN_CUDA(cudaStreamSynchronize(s));
     MIXGCN_CUDA(cudaGetLastError());
     return MIXGCN_OK;
@@ -346,7 +361,7 @@ mixgcn_status finish_graph(mixgcn_graph* g, cudaStream_t s) {
     MIXGCN_CUDA(cudaMemcpyAsync(&hf, flags.p, sizeof(hf), cudaMemcpyDeviceToHost, s));
     MIXGCN_CUDA(cudaStreamSynchronize(s));
     g->symmetric = (hf & F_NOT_SYMMETRIC) ? 0 : 1;
-    MIXGCN_TRY(build_schedule(n, A, s));
+    MIXGCN_TRY(build_schedule(n, A.rowptr, A.col, 0, n, A.full, s));
     if (g->symmetric) {
         g->bwd = A;  // alias: the same index serves the backward aggregation
         return MIXGCN_OK;
@@ -370,7 +385,7 @@ mixgcn_status finish_graph(mixgcn_graph* g, cudaStream_t s) {
                                                 nnz, 0, end_bit, s));
     rowptr_from_keys_kernel<<<blocks_for(nnz + 1), TPB, 0, s>>>(n, nnz, k1.as<uint64_t>(), T.rowptr, T.col);
     MIXGCN_CUDA(cudaStreamSynchronize(s));
-    MIXGCN_TRY(build_schedule(n, T, s));
+    MIXGCN_TRY(build_schedule(n, T.rowptr, T.col, 0, n, T.full, s));
     return MIXGCN_OK;
 }
 
@@ -382,6 +397,35 @@ mixgcn_status check_common(mixgcn_ctx* ctx, int64_t n, mixgcn_graph** out) {
 }
 
 }  // namespace
+
+namespace mixgcn {
+
+mixgcn_status ensure_chunk_schedules(const mixgcn_graph* g, const CsrView& A_const, int chunks) {
+    // a cache inside the graph object; a symmetric graph keeps one set (in fwd) and mirrors it into the alias
+    CsrView& A = const_cast<CsrView&>(g->symmetric ? g->fwd : A_const);
+    if (chunks <= 1 || A.n_chunk == chunks) return MIXGCN_OK;
+    MIXGCN_CUDA(cudaDeviceSynchronize());         // earlier launches may still read the schedules being replaced
+    for (int k = 0; k < A.n_chunk; ++k) free_schedule(A.chunk[k]);
+    delete[] A.chunk;
+    A.chunk = nullptr; A.n_chunk = 0;
+    SpmmSchedule* sc = new (std::nothrow) SpmmSchedule[chunks]();
+    if (!sc) MIXGCN_FAIL(MIXGCN_ENOMEM, "chunk schedules: host allocation failed");
+    cudaStream_t s = g->ctx->side_stream[0];
+    for (int k = 0; k < chunks; ++k) {
+        const int64_t r0 = (g->n * (int64_t)k) / chunks, r1 = (g->n * (int64_t)(k + 1)) / chunks;
+        mixgcn_status st = build_schedule(g->n, A.rowptr, A.col, r0, r1 - r0, sc[k], s);
+        if (st != MIXGCN_OK) {
+            for (int q = 0; q <= k; ++q) free_schedule(sc[q]);
+            delete[] sc;
+            return st;
+        }
+    }
+    A.chunk = sc; A.n_chunk = chunks;
+    if (g->symmetric) const_cast<mixgcn_graph*>(g)->bwd = g->fwd;   // keep the alias in step
+    return MIXGCN_OK;
+}
+
+}  // namespace mixgcn
 
 extern "C" mixgcn_status mixgcn_graph_destroy(mixgcn_graph* g) {
     if (!g) return MIXGCN_OK;
@@ -512,7 +556,7 @@ extern "C" mixgcn_status mixgcn_graph_info(const mixgcn_graph* g, int64_t* n, in
     if (!g) MIXGCN_FAIL(MIXGCN_EINVAL, "graph_info: null graph");
     if (n) *n = g->n;
     if (nnz) *nnz = g->nnz;
-    if (max_deg) *max_deg = g->fwd.max_deg;
+    if (max_deg) *max_deg = g->fwd.full.max_deg;
     if (symmetric) *symmetric = g->symmetric;
     return MIXGCN_OK;
 }
@@ -536,6 +580,6 @@ extern "C" mixgcn_status mixgcn_graph_export_schedule(const mixgcn_graph* g, int
     MIXGCN_CUDA(cudaSetDevice(g->ctx->device));
     MIXGCN_CUDA(cudaDeviceSynchronize());
     const CsrView& v = transposed ? g->bwd : g->fwd;
-    MIXGCN_CUDA(cudaMemcpy(perm, v.perm, g->n * sizeof(int32_t), cudaMemcpyDeviceToHost));
+    MIXGCN_CUDA(cudaMemcpy(perm, v.full.perm, g->n * sizeof(int32_t), cudaMemcpyDeviceToHost));
     return MIXGCN_OK;
 }

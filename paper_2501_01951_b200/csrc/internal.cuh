@@ -48,8 +48,10 @@ struct mixgcn_ctx {
     int device;
     int sm_count;
     int32_t* d_status;        // device status word (int32[4])
-    void* workspace;          // grow-on-demand scratch
+    void* workspace;          // grow-on-demand scratch of the dense products, column sums and the loss
     int64_t workspace_bytes;
+    void* workspace_spmm;     // scratch of the aggregation (partial rows of long-row segments); separate so
+    int64_t workspace_spmm_bytes;  // that an aggregation and a dense product may overlap on two streams
     cudaStream_t side_stream[2];
     cudaEvent_t fork_ev, join_ev[2];
     cudaEvent_t chunk_ev[64];
@@ -72,23 +74,32 @@ struct __align__(16) SpmmRec {
     int32_t row;
 };
 
-// One CSR orientation of A_hat plus its aggregation schedule.
-struct CsrView {
-    int64_t* rowptr;   // [n+1]
-    int32_t* col;      // [nnz]
-    float* val;        // [nnz]
-    int32_t* perm;     // [n] rows by descending entry count
+// Aggregation schedule of the rows [row0, row0 + n_rows) of one CSR orientation.
+// Rows longer than SPMM_SEG entries are cut into segments at dyadic column-block boundaries and
+// every SPMM_SEG entries; the segment records [0, total_segs) run in order of their first column, so
+// that segments of different long rows that gather the same rows of Y run close in time (those rows
+// are then served by the L2).  Every other row is one record, in perm order (records
+// [total_segs, total_segs + n_rows - n_long)).
+struct SpmmSchedule {
+    int64_t row0, n_rows;
+    int32_t* perm;             // [n_rows] row ids by descending entry count (ties by ascending id)
     int32_t max_deg;
-    // schedule: rows longer than SPMM_SEG entries are cut into segments at dyadic column-block
-    // boundaries and every SPMM_SEG entries; the segment records [0, total_segs) run in order of
-    // their first column, so that segments of different long rows that gather the same rows of Y run
-    // close in time (those rows are then served by the L2).  Every other row is one record, in perm
-    // order (records [total_segs, total_segs + n - n_long)).
     SpmmRec* rec;
     int64_t n_long, total_segs;
     int64_t* seg_off;          // [n_long+1] segments of long row i are numbered seg_off[i] .. seg_off[i+1]-1 in entry order
     int64_t* seg_pos;          // [total_segs] record position (= partial-row slot) of segment number q
     int64_t rows_above[3];     // rows with more than SPMM_PACK_DEG[i] entries (bucket boundaries in perm order)
+};
+
+// One CSR orientation of A_hat plus its aggregation schedules: one over all rows, and (built on
+// first use) one per row chunk of the two-stream pipeline.
+struct CsrView {
+    int64_t* rowptr;   // [n+1]
+    int32_t* col;      // [nnz]
+    float* val;        // [nnz]
+    SpmmSchedule full;
+    SpmmSchedule* chunk;   // [n_chunk] schedules of the chunks floor(n*k/n_chunk) .. floor(n*(k+1)/n_chunk)
+    int n_chunk;
 };
 
 struct mixgcn_graph {
@@ -126,10 +137,14 @@ struct LaunchScope {
 };
 
 mixgcn_status ensure_workspace(mixgcn_ctx* ctx, int64_t bytes);
+mixgcn_status ensure_workspace_spmm(mixgcn_ctx* ctx, int64_t bytes);
+// Builds (once) the schedules of the `chunks` row chunks of this orientation.  Synchronises on first use.
+mixgcn_status ensure_chunk_schedules(const mixgcn_graph* g, const CsrView& A, int chunks);
 
 // kernels' host launchers (all asynchronous on `s`)
-mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView& A, int64_t row_begin,
-                          int64_t row_end, int32_t w, const float* Y, int64_t ldy, float* Z, int64_t ldz,
+// Aggregation over all rows (chunks <= 1) or over chunk k of `chunks` row chunks.
+mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView& A, int chunks, int k,
+                          int32_t w, const float* Y, int64_t ldy, float* Z, int64_t ldz,
                           const mixgcn_epilogue* epi, cudaStream_t s);
 mixgcn_status launch_gemm(mixgcn_ctx* ctx, int precision, int ta, int tb, int64_t M, int64_t N, int64_t K,
                           const float* A, int64_t lda, const float* B, int64_t ldb, float* C, int64_t ldc,

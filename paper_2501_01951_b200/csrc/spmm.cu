@@ -211,14 +211,18 @@ constexpr int MAX_SLICE = 1024;  // columns per launch: 8 float4 per lane
 
 namespace mixgcn {
 
-// Rows [row_begin, row_end): when the range is the whole matrix the schedule is used (long rows as
-// segments, then rows longest first, short rows packed); a partial range (pipeline chunk) runs in
-// natural row order without scratch.
-mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView& A, int64_t row_begin,
-                          int64_t row_end, int32_t w, const float* Y, int64_t ldy, float* Z, int64_t ldz,
+// Aggregation of all rows (chunks <= 1) or of row chunk k of `chunks` (the pipeline's chunks), each
+// with its own schedule: long rows as column-ordered segments, then rows longest first, short rows packed.
+mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView& A, int chunks, int k,
+                          int32_t w, const float* Y, int64_t ldy, float* Z, int64_t ldz,
                           const mixgcn_epilogue* epi, cudaStream_t s) {
-    if (row_end <= row_begin || w <= 0) return MIXGCN_OK;
-    const bool whole = row_begin == 0 && row_end == g->n;
+    if (w <= 0) return MIXGCN_OK;
+    if (chunks > 1) {
+        MIXGCN_TRY(ensure_chunk_schedules(g, A, chunks));
+        if (k < 0 || k >= A.n_chunk) MIXGCN_FAIL(MIXGCN_EINVAL, "spmm: chunk %d of %d does not exist", k, chunks);
+    }
+    const SpmmSchedule& S = chunks > 1 ? A.chunk[k] : A.full;
+    if (S.n_rows <= 0) return MIXGCN_OK;
     SpmmParams p{};
     p.rowptr = A.rowptr; p.col = A.col; p.val = A.val;
     p.Y = Y; p.ldy = ldy; p.Z = Z; p.ldz = ldz; p.w_total = w;
@@ -226,45 +230,38 @@ mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView&
         p.bias = epi->bias; p.relu = epi->relu; p.drop = epi->drop_mask; p.keep_scale = epi->keep_scale;
         p.gate = epi->gate; p.ld_gate = epi->ld_gate; p.gate_scale = epi->gate_scale;
     }
+    p.rec = S.rec;
     for (int j0 = 0; j0 < w; j0 += MAX_SLICE) {
         p.j0 = j0;
         p.w = (w - j0) < MAX_SLICE ? (w - j0) : MAX_SLICE;
-        if (!whole) {
-            LaunchScope scope(ctx, PH_SPMM, s);
-            p.rec = nullptr; p.partial = nullptr; p.idx_begin = row_begin; p.idx_end = row_end;
-            dispatch(p, 1, s);
-            continue;
-        }
-        p.rec = A.rec;
-        if (A.total_segs > 0) {
+        if (S.total_segs > 0) {
             const int64_t ldp = ((int64_t)p.w + 3) / 4 * 4;
-            MIXGCN_TRY(ensure_workspace(ctx, A.total_segs * ldp * (int64_t)sizeof(float)));
-            p.partial = reinterpret_cast<float*>(ctx->workspace); p.ldp = ldp;
+            MIXGCN_TRY(ensure_workspace_spmm(ctx, S.total_segs * ldp * (int64_t)sizeof(float)));
+            p.partial = reinterpret_cast<float*>(ctx->workspace_spmm); p.ldp = ldp;
             {
                 LaunchScope scope(ctx, PH_SPMM, s);
-                p.idx_begin = 0; p.idx_end = A.total_segs;
+                p.idx_begin = 0; p.idx_end = S.total_segs;
                 dispatch(p, 1, s);
             }
             {
                 LaunchScope scope(ctx, PH_SPMM, s);
-                const int64_t blocks = (A.n_long * 32 + 255) / 256;
-                spmm_combine_kernel<<<(unsigned)blocks, 256, 0, s>>>(p, A.n_long, A.seg_off, A.seg_pos, A.perm);
+                const int64_t blocks = (S.n_long * 32 + 255) / 256;
+                spmm_combine_kernel<<<(unsigned)blocks, 256, 0, s>>>(p, S.n_long, S.seg_off, S.seg_pos, S.perm);
             }
             p.partial = nullptr;
         }
-        // ordinary rows, in perm order: [n_long, n) -> records [total_segs, total_segs + n - n_long)
+        // ordinary rows, in perm order: [n_long, n_rows) -> records [total_segs, total_segs + n_rows - n_long)
         int64_t bound[5];
-        bound[0] = A.n_long;
-        for (int q = 0; q < 3; ++q) bound[q + 1] = A.rows_above[q] > A.n_long ? A.rows_above[q] : A.n_long;
-        bound[4] = g->n;
+        bound[0] = S.n_long;
+        for (int q = 0; q < 3; ++q) bound[q + 1] = S.rows_above[q] > S.n_long ? S.rows_above[q] : S.n_long;
+        bound[4] = S.n_rows;
         int64_t begin = bound[0];
         int fold = 1;
         for (int q = 0; q < 4; ++q, fold <<= 1) {
-            // a bucket whose fold is not available for this width is merged into the next launch range
             int64_t end = bound[q + 1];
             if (end <= begin) continue;
-            p.idx_begin = A.total_segs + (begin - A.n_long);
-            p.idx_end = A.total_segs + (end - A.n_long);
+            p.idx_begin = S.total_segs + (begin - S.n_long);
+            p.idx_end = S.total_segs + (end - S.n_long);
             LaunchScope scope(ctx, PH_SPMM, s);
             dispatch(p, fold, s);
             begin = end;
@@ -288,5 +285,5 @@ extern "C" mixgcn_status mixgcn_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, int
     if (Y == Z) MIXGCN_FAIL(MIXGCN_EINVAL, "spmm: Y and Z must not overlap");
     if (epi && epi->gate && epi->ld_gate < w) MIXGCN_FAIL(MIXGCN_EINVAL, "spmm: gate leading dimension < w");
     MIXGCN_CUDA(cudaSetDevice(ctx->device));
-    return launch_spmm(ctx, g, transposed ? g->bwd : g->fwd, 0, g->n, w, Y, ldy, Z, ldz, epi, (cudaStream_t)stream);
+    return launch_spmm(ctx, g, transposed ? g->bwd : g->fwd, 1, 0, w, Y, ldy, Z, ldz, epi, (cudaStream_t)stream);
 }
