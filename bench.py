@@ -137,6 +137,17 @@ def build_problem(wl, device):
     return src, dst
 
 
+def replicas_throughput(ms_local, steps, world, device):
+    """Whole-job throughput of `world` independent replicas: the slowest rank's time (max over ranks)
+    bounds the job, and every rank completed `steps` epochs in it.  Returns (max ms, epochs/s)."""
+    ms = float(ms_local)
+    if world > 1:
+        tt = torch.tensor([ms], dtype=torch.float64, device=device)
+        torch.distributed.all_reduce(tt, op=torch.distributed.ReduceOp.MAX)
+        ms = float(tt.item())
+    return ms, world * steps / (ms / 1e3)
+
+
 def run_ours(args, rank, world, local_rank):
     from paper_2501_01951_b200 import binding as mg
     from paper_2501_01951_b200.train import GcnTrainer, round4
@@ -193,12 +204,8 @@ def run_ours(args, rank, world, local_rank):
     loss_val = tr.loss.item()
     n_train = int(m.sum().item())
 
-    if world > 1:
-        tt = torch.tensor([ms_total], device=dev)
-        torch.distributed.all_reduce(tt, op=torch.distributed.ReduceOp.MAX)
-        ms_total = tt.item()
+    ms_total, value = replicas_throughput(ms_total, args.steps, world, dev)
     ms_per_step = ms_total / args.steps
-    value = world * args.steps / (ms_total / 1e3)
 
     # roofline of the aggregation kernels over the timed steps
     plan = spmm_plan(wl, tr.orders)

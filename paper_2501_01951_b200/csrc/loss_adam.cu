@@ -90,6 +90,134 @@ __global__ void __launch_bounds__(LOSS_WARPS * 32) loss_rows_kernel(
     }
 }
 
+// Same computation for C <= 128 * VPL with the row held in registers: one float4-vectorised read of the
+// logits, one float4 write of the gradient (requires ld % 4 == 0 and 16-byte aligned pointers).
+template <int VPL>
+__global__ void __launch_bounds__(LOSS_WARPS * 32) loss_rows_vec_kernel(
+    int64_t n, int C, const float* logits, int64_t ld, const int32_t* __restrict__ labels,
+    const uint8_t* __restrict__ mask, const unsigned long long* __restrict__ count, float* dlogits,
+    int32_t* __restrict__ pred, unsigned long long* n_correct, double* __restrict__ part, int32_t* status) {
+    __shared__ double sm[LOSS_WARPS];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const unsigned long long T = *count;
+    const float invT = T ? (float)(1.0 / (double)T) : 0.0f;
+    const int C4 = (C + 3) >> 2;
+    double local = 0.0;
+    unsigned int correct = 0;
+    const int64_t stride = (int64_t)gridDim.x * LOSS_WARPS;
+    // the next row's loads are issued before the current row is reduced, so two rows per warp are in flight
+    auto load_row = [&](int64_t v, float4 (&t)[VPL]) {
+        const float4* row4 = reinterpret_cast<const float4*>(logits + v * ld);
+#pragma unroll
+        for (int q = 0; q < VPL; ++q) {
+            const int g = lane + 32 * q;
+            t[q] = (v < n && g < C4) ? row4[g] : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+        }
+    };
+    float4 nxt[VPL];
+    load_row((int64_t)blockIdx.x * LOSS_WARPS + warp, nxt);
+    for (int64_t v = (int64_t)blockIdx.x * LOSS_WARPS + warp; v < n; v += stride) {
+        float x[VPL][4];
+#pragma unroll
+        for (int q = 0; q < VPL; ++q) {
+            const int g = lane + 32 * q;
+            x[q][0] = nxt[q].x; x[q][1] = nxt[q].y; x[q][2] = nxt[q].z; x[q][3] = nxt[q].w;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) if (g * 4 + e >= C) x[q][e] = -INFINITY;   // pad columns are not data
+        }
+        load_row(v + stride, nxt);
+        float mx = -INFINITY; int arg = 0x7FFFFFFF;
+#pragma unroll
+        for (int q = 0; q < VPL; ++q)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int c = (lane + 32 * q) * 4 + e;
+                if (c < C && (x[q][e] > mx || (x[q][e] == mx && c < arg))) { mx = x[q][e]; arg = c; }
+            }
+        if (arg == 0x7FFFFFFF) arg = lane * 4 < C ? lane * 4 : 0;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float omx = __shfl_xor_sync(0xFFFFFFFFu, mx, o);
+            const int oarg = __shfl_xor_sync(0xFFFFFFFFu, arg, o);
+            if (omx > mx || (omx == mx && oarg < arg)) { mx = omx; arg = oarg; }
+        }
+        if (pred && lane == 0) pred[v] = arg;
+        const bool train = mask[v] != 0 && T != 0;
+        int y = 0;
+        bool ok = false;
+        if (train) {
+            y = labels[v];
+            ok = y >= 0 && y < C;
+            if (!ok && lane == 0) atomicMax(status, DEV_BAD_LABEL);
+        }
+        float4* out4 = dlogits ? reinterpret_cast<float4*>(dlogits + v * ld) : nullptr;
+        if (!train || !ok) {
+            if (out4) {
+#pragma unroll
+                for (int q = 0; q < VPL; ++q) {
+                    const int g = lane + 32 * q;
+                    if (g < C4) out4[g] = make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+            }
+            continue;
+        }
+        float s = 0.0f;
+#pragma unroll
+        for (int q = 0; q < VPL; ++q)
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+                if ((lane + 32 * q) * 4 + e < C) s += expf(x[q][e] - mx);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
+        const float lse = mx + logf(s);
+        // the label's logit lives in lane (y/4) % 32, slot (y/4) / 32, element y % 4
+        float py = 0.0f;
+#pragma unroll
+        for (int q = 0; q < VPL; ++q)
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+                if ((lane + 32 * q) * 4 + e == y) py = x[q][e];
+        py = __shfl_sync(0xFFFFFFFFu, py, (y >> 2) & 31);
+        if (lane == 0) { local += (double)(lse - py); if (arg == y) ++correct; }
+        if (out4) {
+#pragma unroll
+            for (int q = 0; q < VPL; ++q) {
+                const int g = lane + 32 * q;
+                if (g < C4) {
+                    float r[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const int c = g * 4 + e;
+                        r[e] = c < C ? (expf(x[q][e] - lse) - (c == y ? 1.0f : 0.0f)) * invT : 0.0f;
+                    }
+                    out4[g] = make_float4(r[0], r[1], r[2], r[3]);
+                }
+            }
+        }
+    }
+    if (lane == 0) sm[warp] = local;
+    if (n_correct && lane == 0 && correct) atomicAdd(n_correct, (unsigned long long)correct);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double t = 0.0;
+        for (int w = 0; w < LOSS_WARPS; ++w) t += sm[w];
+        part[blockIdx.x] = t;
+    }
+}
+
+// Picks the register-resident kernel when the row fits (C <= 256) and the layout allows float4 access.
+void launch_loss_rows(unsigned blocks, cudaStream_t s, int64_t n, int C, const float* logits, int64_t ld,
+                      const int32_t* labels, const uint8_t* mask, const unsigned long long* count, float* dlogits,
+                      int32_t* pred, unsigned long long* n_correct, double* part, int32_t* status) {
+    const bool vec = (ld & 3) == 0 && aligned16(logits) && (!dlogits || aligned16(dlogits));
+    if (vec && C <= 128)
+        loss_rows_vec_kernel<1><<<blocks, LOSS_WARPS * 32, 0, s>>>(n, C, logits, ld, labels, mask, count, dlogits, pred, n_correct, part, status);
+    else if (vec && C <= 256)
+        loss_rows_vec_kernel<2><<<blocks, LOSS_WARPS * 32, 0, s>>>(n, C, logits, ld, labels, mask, count, dlogits, pred, n_correct, part, status);
+    else
+        loss_rows_kernel<<<blocks, LOSS_WARPS * 32, 0, s>>>(n, C, logits, ld, labels, mask, count, dlogits, pred, n_correct, part, status);
+}
+
 __global__ void loss_final_kernel(int blocks, const double* __restrict__ part,
                                   const unsigned long long* __restrict__ count, float* loss, int32_t* status) {
     if (threadIdx.x != 0 || blockIdx.x != 0) return;
@@ -154,9 +282,8 @@ extern "C" mixgcn_status mixgcn_loss_softmax_xent(mixgcn_ctx* ctx, int64_t n, in
     }
     {
         LaunchScope scope(ctx, PH_LOSS, s);
-        loss_rows_kernel<<<(unsigned)blocks, LOSS_WARPS * 32, 0, s>>>(
-            n, C, logits, ld, labels, train_mask, count, dlogits, pred,
-            reinterpret_cast<unsigned long long*>(n_correct), part, ctx->d_status);
+        launch_loss_rows((unsigned)blocks, s, n, C, logits, ld, labels, train_mask, count, dlogits, pred,
+                         reinterpret_cast<unsigned long long*>(n_correct), part, ctx->d_status);
     }
     {
         LaunchScope scope(ctx, PH_LOSS, s);
@@ -263,9 +390,8 @@ extern "C" mixgcn_status mixgcn_loss_softmax_xent_noalloc(int64_t n, int32_t C, 
     int64_t cb = (n + 255) / 256;
     if (cb > 4096) cb = 4096;
     count_mask_kernel<<<(unsigned)cb, 256, 0, s>>>(n, train_mask, &sc->count);
-    loss_rows_kernel<<<(unsigned)blocks, LOSS_WARPS * 32, 0, s>>>(n, C, logits, ld, labels, train_mask, &sc->count, dlogits,
-                                                                 pred, reinterpret_cast<unsigned long long*>(n_correct),
-                                                                 sc->part, &sc->status);
+    launch_loss_rows((unsigned)blocks, s, n, C, logits, ld, labels, train_mask, &sc->count, dlogits, pred,
+                     reinterpret_cast<unsigned long long*>(n_correct), sc->part, &sc->status);
     loss_final_kernel<<<1, 32, 0, s>>>((int)blocks, sc->part, &sc->count, loss, &sc->status);
     if (status) MIXGCN_CUDA(cudaMemcpyAsync(status, &sc->status, sizeof(int32_t), cudaMemcpyDeviceToDevice, s));
     MIXGCN_CUDA(cudaGetLastError());
