@@ -103,8 +103,9 @@ class ClockSampler:
 
 # ------------------------------------------------------------------------------------ workload
 
-def spmm_plan(wl, orders):
-    """Widths of the aggregation calls of one epoch: (width, count) per layer, from the ordering."""
+def spmm_plan(wl, orders, sparse_levels=0):
+    """Widths of the DENSE-input aggregation calls of one epoch: (width, count) per layer, from the
+    ordering; the backward aggregations of the top `sparse_levels` layers run row-sparse and are not counted."""
     from paper_2501_01951_b200 import binding as mg
     calls = []
     L = len(wl.dims) - 1
@@ -112,6 +113,8 @@ def spmm_plan(wl, orders):
         agg = orders[l] == mg.ORDER_AGG_FIRST
         w = wl.dims[l] if agg else wl.dims[l + 1]
         k = 1 + (0 if (l == 0 and agg) else 1)          # forward, plus backward unless first layer agg-first
+        if l >= L - sparse_levels and k == 2:
+            k = 1                                        # this layer's backward aggregation takes the row-sparse path
         calls.append((w, k))
     return calls
 
@@ -164,7 +167,8 @@ def run_ours(args, rank, world, local_rank):
     del src, dst
     torch.cuda.empty_cache()
     n, nnz = g.n, g.nnz
-    tr = GcnTrainer(ctx, g, wl.dims, prec, n_chunks=args.chunks)
+    tr = GcnTrainer(ctx, g, wl.dims, prec, n_chunks=args.chunks,
+                    row_sparse=args.row_sparse if args.row_sparse == "auto" else int(args.row_sparse))
     X0 = synth.normal_features(n, wl.dims[0], wl.seed("features"), device=dev, ld=round4(wl.dims[0]))
     y = synth.uniform_labels(n, wl.classes, wl.seed("labels"), device=dev)
     m = synth.bernoulli_mask(n, wl.mask_p, wl.seed("mask"), device=dev)
@@ -208,7 +212,7 @@ def run_ours(args, rank, world, local_rank):
     ms_per_step = ms_total / args.steps
 
     # roofline of the aggregation kernels over the timed steps
-    plan = spmm_plan(wl, tr.orders)
+    plan = spmm_plan(wl, tr.orders, tr.row_sparse_levels)
     spmm_calls = sum(k for _, k in plan) * args.steps
     alg_bytes = sum(spmm_alg_bytes(n, nnz, w) * k for w, k in plan) * args.steps
     spmm_ms = phase_ms["spmm"]
@@ -230,7 +234,7 @@ def run_ours(args, rank, world, local_rank):
                dtype={mg.PREC_FP32: "f32", mg.PREC_TF32: "tf32", mg.PREC_BF16: "bf16"}[prec], data="synthetic",
                config=dict(workload=wl.name, n=n, nnz=nnz, dims=list(wl.dims), train_nodes=n_train,
                            orders=["agg-first" if o == mg.ORDER_AGG_FIRST else "upd-first" for o in tr.orders],
-                           chunks=args.chunks, l2="inputs larger than L2" if 4 * n * wl.dims[0] > 126e6 else "inputs fit L2 (no flush)",
+                           chunks=args.chunks, row_sparse_levels=tr.row_sparse_levels, l2="inputs larger than L2" if 4 * n * wl.dims[0] > 126e6 else "inputs fit L2 (no flush)",
                            parallelism=f"replicas x{world}" if world > 1 else "single GPU", setup_s=round(setup_s, 1)),
                clocks=clk, gpu_launches=int(launches_after - launches_before),
                roofline=roofline, gemm=gemm, phase_ms_per_epoch=breakdown, loss=round(loss_val, 6), device_status=status)
@@ -357,6 +361,7 @@ def main():
     ap.add_argument("--workload", default=os.environ.get("MIXGCN_WORKLOAD", "C5"), choices=list(synth.CONFIGS))
     ap.add_argument("--precision", default=None, choices=["fp32", "tf32", "bf16"])
     ap.add_argument("--chunks", type=int, default=0)
+    ap.add_argument("--row-sparse", default="auto", help="layers (from the top) whose backward gets a row mask: auto, 0, 1, 2, ...")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-seconds", type=float, default=20.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -60,16 +60,18 @@ mixgcn_status mixgcn_ctx_reserve(mixgcn_ctx* ctx, int64_t bytes);
 
 /* Synchronises the context's device, reads and clears the device status word.
  * Returns MIXGCN_OK, MIXGCN_EDEVICE or MIXGCN_ETIMEOUT; *code (nullable) receives the raw
- * code: 0 none, 1 empty train mask, 2 label out of range, 3 bounded wait expired. */
+ * code: 0 none, 1 empty train mask, 2 label out of range, 3 bounded wait expired,
+ * 4 gout_row_count does not match gout_row_mask. */
 mixgcn_status mixgcn_ctx_poll_status(mixgcn_ctx* ctx, int32_t* code);
 
 /* Per-phase profiling.  While enabled the library brackets every kernel it launches with
  * CUDA events on the launching stream.  mixgcn_ctx_profile_read synchronises and returns, for
  * each phase, accumulated milliseconds and launch counts since the last read, then resets.
- * Phases: 0 spmm, 1 gemm, 2 elementwise/epilogue, 3 loss, 4 adam, 5 graph build.
+ * Phases: 0 spmm (dense input), 1 gemm, 2 elementwise/epilogue, 3 loss, 4 adam, 5 graph build,
+ * 6 spmm with a row-sparse input.
  * `launches_total` (nullable) receives the number of kernels launched by this context since
  * creation (counted whether or not profiling is enabled). */
-#define MIXGCN_N_PHASES 6
+#define MIXGCN_N_PHASES 7
 mixgcn_status mixgcn_ctx_profile_enable(mixgcn_ctx* ctx, int enable);
 mixgcn_status mixgcn_ctx_profile_read(mixgcn_ctx* ctx, double ms[MIXGCN_N_PHASES],
                                       int64_t launches[MIXGCN_N_PHASES], int64_t* launches_total);
@@ -184,6 +186,19 @@ typedef struct {
     float in_scale;     /* keep_scale of the layer below, used with GATE_GIN; 1 if none */
     int32_t n_chunks;   /* >1: split rows into this many chunks and overlap the aggregation of
                            chunk k+1 with the update of chunk k on two streams; 0/1: off */
+    /* Row-sparse backward (all optional; NULL / 0 = dense).  The gradient of a masked loss is non-zero
+     * on train rows only, and one aggregation later on their neighbours only; telling the library
+     * which rows may be non-zero lets it skip the rest -- the sampled form of Eq. 4 applied to the
+     * rows of the operand instead of the elements of the output.  Results are those of the dense
+     * computation with its exactly-zero terms left out.
+     *   gout_row_mask   device uint8[n]: rows of G_out whose byte is 0 ARE exactly zero (caller's promise)
+     *   gout_row_count  number of non-zero bytes in gout_row_mask if known, else 0; when it is below
+     *                   n/4 (agg-first order) the dense products run on the compacted rows; a wrong
+     *                   count is reported through the status word (code 4), never a memory fault
+     *   gin_row_mask    device uint8[n], written: 0 for rows of G_in that are exactly zero */
+    const uint8_t* gout_row_mask;
+    int64_t gout_row_count;
+    uint8_t* gin_row_mask;
 } mixgcn_layer_desc;
 
 /* Resolves MIXGCN_ORDER_AUTO: cost(agg-first) = c * d_in with c = 1 for a FIRST layer (its

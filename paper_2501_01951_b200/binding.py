@@ -27,8 +27,8 @@ GRAPH_SYMMETRISE, GRAPH_ADD_SELF_LOOPS, GRAPH_EDGES_ON_DEVICE = 1, 2, 4
 PREC_FP32, PREC_TF32, PREC_BF16 = 0, 1, 2
 ORDER_AUTO, ORDER_AGG_FIRST, ORDER_UPD_FIRST = 0, 1, 2
 LAYER_RELU, LAYER_FIRST, LAYER_GATE_GIN, LAYER_GOUT_GATED = 1, 2, 4, 8
-N_PHASES = 6
-PHASES = ("spmm", "gemm", "elementwise", "loss", "adam", "graph")
+N_PHASES = 7
+PHASES = ("spmm", "gemm", "elementwise", "loss", "adam", "graph", "spmm_sparse")
 PRECISIONS = {"fp32": PREC_FP32, "tf32": PREC_TF32, "bf16": PREC_BF16}
 
 # every symbol include/mixgcn.h declares
@@ -52,7 +52,8 @@ class LayerDesc(C.Structure):
     _fields_ = [("d_in", C.c_int32), ("d_out", C.c_int32), ("ld_in", C.c_int64), ("ld_out", C.c_int64),
                 ("ld_saved", C.c_int64), ("order", C.c_int32), ("precision", C.c_int32),
                 ("flags", C.c_uint32), ("keep_scale", C.c_float), ("in_scale", C.c_float),
-                ("n_chunks", C.c_int32)]
+                ("n_chunks", C.c_int32), ("gout_row_mask", C.c_void_p), ("gout_row_count", C.c_int64),
+                ("gin_row_mask", C.c_void_p)]
 
 
 lib.mixgcn_status_string.restype = C.c_char_p
@@ -248,7 +249,8 @@ def gemm(ctx: Ctx, precision: int, trans_a: bool, trans_b: bool, M: int, N: int,
 
 def layer_desc(d_in, d_out, ld_in, ld_out, ld_saved, order=ORDER_AUTO, precision=PREC_FP32, flags=0,
                keep_scale=1.0, in_scale=1.0, n_chunks=0) -> LayerDesc:
-    return LayerDesc(d_in, d_out, ld_in, ld_out, ld_saved, order, precision, flags, keep_scale, in_scale, n_chunks)
+    return LayerDesc(d_in, d_out, ld_in, ld_out, ld_saved, order, precision, flags, keep_scale, in_scale, n_chunks,
+                     None, 0, None)
 
 
 def layer_plan(desc: LayerDesc):

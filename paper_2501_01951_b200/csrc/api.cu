@@ -158,6 +158,7 @@ extern "C" mixgcn_status mixgcn_ctx_destroy(mixgcn_ctx* ctx) {
     if (ctx->fork_ev) cudaEventDestroy(ctx->fork_ev);
     cudaFree(ctx->workspace);
     cudaFree(ctx->workspace_spmm);
+    cudaFree(ctx->workspace_rows);
     cudaFree(ctx->arena);
     cudaFree(ctx->d_status);
     delete ctx;
@@ -180,7 +181,7 @@ extern "C" mixgcn_status mixgcn_ctx_poll_status(mixgcn_ctx* ctx, int32_t* code) 
     if (code) *code = h;
     if (h == DEV_OK) return MIXGCN_OK;
     if (h == DEV_WAIT_EXPIRED) MIXGCN_FAIL(MIXGCN_ETIMEOUT, "a bounded device-side wait expired");
-    MIXGCN_FAIL(MIXGCN_EDEVICE, h == DEV_EMPTY_MASK ? "loss: the train mask is empty" : "loss: a label lies outside [0, C)");
+    MIXGCN_FAIL(MIXGCN_EDEVICE, h == DEV_EMPTY_MASK ? "loss: the train mask is empty" : h == DEV_BAD_LABEL ? "loss: a label lies outside [0, C)" : "layer_bwd: gout_row_count does not match gout_row_mask");
 }
 
 extern "C" mixgcn_status mixgcn_ctx_profile_enable(mixgcn_ctx* ctx, int enable) {
@@ -341,7 +342,6 @@ extern "C" mixgcn_status mixgcn_layer_bwd(mixgcn_ctx* ctx, const mixgcn_graph* g
     // gradient w.r.t. the pre-activation, in place in G_out
     if (!(d->flags & MIXGCN_LAYER_GOUT_GATED) && (relu || drop_mask))
         MIXGCN_TRY(launch_gate(ctx, n, d->d_out, G_out, d->ld_out, X_out, d->ld_out, relu, drop_mask, d->keep_scale, s));
-    if (dbias) MIXGCN_TRY(launch_colsum(ctx, n, d->d_out, G_out, d->ld_out, dbias, s));
 
     mixgcn_epilogue gin_epi{};
     const mixgcn_epilogue* gin = nullptr;
@@ -349,20 +349,44 @@ extern "C" mixgcn_status mixgcn_layer_bwd(mixgcn_ctx* ctx, const mixgcn_graph* g
         gin_epi.gate = X_in; gin_epi.ld_gate = d->ld_in; gin_epi.gate_scale = d->in_scale; gin_epi.keep_scale = 1.0f;
         gin = &gin_epi;
     }
+    const uint8_t* rmask = d->gout_row_mask;
+    SpmmRowSparse sp{rmask, nullptr, d->gin_row_mask};
+    const SpmmRowSparse* spp = rmask ? &sp : nullptr;
 
     if (order == MIXGCN_ORDER_AGG_FIRST) {
+        const int64_t cnt = d->gout_row_count;
+        if (rmask && cnt > 0 && cnt * 4 < n) {
+            // Few non-zero rows: dW, db and dZ from the compacted rows, then a row-sparse aggregation.
+            RowSet rs;
+            const int64_t lda = (d->d_in + 3) / 4 * 4, ldb = (d->d_out + 3) / 4 * 4;
+            MIXGCN_TRY(build_row_set(ctx, n, rmask, cnt, lda, ldb, &rs, s));
+            MIXGCN_TRY(launch_gather_rows(ctx, cnt, d->d_in, rs.idx, saved, d->ld_saved, rs.a, lda, s));     // Z_T
+            MIXGCN_TRY(launch_gather_rows(ctx, cnt, d->d_out, rs.idx, G_out, d->ld_out, rs.b, ldb, s));      // dP_T
+            if (dbias) MIXGCN_TRY(launch_colsum(ctx, cnt, d->d_out, rs.b, ldb, dbias, s));
+            MIXGCN_TRY(launch_gemm(ctx, d->precision, 1, 0, d->d_in, d->d_out, cnt, rs.a, lda, rs.b, ldb, dW, ldw, nullptr, 0, s));
+            if (!first) {
+                MIXGCN_TRY(launch_gemm(ctx, d->precision, 0, 1, cnt, d->d_in, d->d_out, rs.b, ldb, W, ldw, rs.a, lda, nullptr, 0, s));
+                sp.in_pos = rs.pos;                                                                             // dZ_T is compact
+                MIXGCN_TRY(launch_spmm(ctx, g, g->bwd, 1, 0, d->d_in, rs.a, lda, G_in, d->ld_in, gin, s, &sp));
+            }
+            return MIXGCN_OK;
+        }
         // dW = (A_hat X_in)^T dP ; dZ = dP W^T (over `saved`) ; G_in = A_hat^T dZ
+        if (dbias) MIXGCN_TRY(launch_colsum(ctx, n, d->d_out, G_out, d->ld_out, dbias, s));
         MIXGCN_TRY(launch_gemm(ctx, d->precision, 1, 0, d->d_in, d->d_out, n, saved, d->ld_saved, G_out, d->ld_out, dW,
                                ldw, nullptr, 0, s));
         if (!first) {
             MIXGCN_TRY(launch_gemm(ctx, d->precision, 0, 1, n, d->d_in, d->d_out, G_out, d->ld_out, W, ldw, saved,
                                    d->ld_saved, nullptr, 0, s));
-            MIXGCN_TRY(launch_spmm(ctx, g, g->bwd, 1, 0, d->d_in, saved, d->ld_saved, G_in, d->ld_in, gin, s));
+            MIXGCN_TRY(launch_spmm(ctx, g, g->bwd, 1, 0, d->d_in, saved, d->ld_saved, G_in, d->ld_in, gin, s, spp));
         }
         return MIXGCN_OK;
     }
     // update first: dQ = A_hat^T dZ (into `saved`) ; dW = X_in^T dQ ; G_in = dQ W^T
-    MIXGCN_TRY(launch_spmm(ctx, g, g->bwd, 1, 0, d->d_out, G_out, d->ld_out, saved, d->ld_saved, nullptr, s));
+    // (rows of dQ that received no contribution are zero, and so are those rows of G_in: the mask the
+    // aggregation reports is G_in's row mask as well)
+    if (dbias) MIXGCN_TRY(launch_colsum(ctx, n, d->d_out, G_out, d->ld_out, dbias, s));
+    MIXGCN_TRY(launch_spmm(ctx, g, g->bwd, 1, 0, d->d_out, G_out, d->ld_out, saved, d->ld_saved, nullptr, s, spp));
     MIXGCN_TRY(launch_gemm(ctx, d->precision, 1, 0, d->d_in, d->d_out, n, X_in, d->ld_in, saved, d->ld_saved, dW, ldw,
                            nullptr, 0, s));
     if (!first)

@@ -23,6 +23,7 @@ struct Carver {
 struct StepLayout {
     std::vector<float*> X, saved, G, W, b, dW, db, mW, vW, mb, vb;
     int32_t* labels; uint8_t* mask; float* loss; int32_t* pred;
+    std::vector<uint8_t*> rowmask;   // [L] byte masks the row-sparse backward fills (layer l's input-gradient rows)
     std::vector<mixgcn_layer_desc> desc;
     int64_t bytes;
 };
@@ -55,6 +56,8 @@ mixgcn_status lay_out(char* base, int64_t n, int L, const int32_t* dims, int pre
     lo.G[L] = lo.X[L];  // the logits' gradient overwrites the logits
     for (int l = L - 1, i = 0; l >= 1; --l, ++i) lo.G[l] = pool[i % 2];
     lo.labels = c.take<int32_t>(n); lo.mask = c.take<uint8_t>(n); lo.loss = c.take<float>(4); lo.pred = c.take<int32_t>(n);
+    lo.rowmask.resize(L);
+    for (int l = 0; l < L; ++l) lo.rowmask[l] = c.take<uint8_t>(n);
     auto each = [&](std::vector<float*>& v, bool weight) {
         v.resize(L);
         for (int l = 0; l < L; ++l) v[l] = c.take<float>(weight ? (int64_t)dims[l] * dims[l + 1] : dims[l + 1]);
@@ -99,6 +102,22 @@ extern "C" mixgcn_status mixgcn_train_step_host(mixgcn_ctx* ctx, const mixgcn_gr
         MIXGCN_CUDA(cudaMemset(p, 0, (size_t)lo.bytes));
     }
     MIXGCN_TRY(lay_out(reinterpret_cast<char*>(ctx->arena), n, L, dims, precision, lo));
+    // Row sparsity of the backward pass: the loss gradient is non-zero on train rows only, and one
+    // aggregation later on their neighbours only (same rule as the device-buffer trainer).
+    int64_t n_train = 0;
+    for (int64_t i = 0; i < n; ++i) n_train += train_mask[i] ? 1 : 0;
+    {
+        const double frac = (double)n_train / (double)n, mean_entries = (double)g->nnz / (double)n;
+        int levels = frac >= 0.25 ? 0 : (frac * mean_entries < 0.5 ? 2 : 1);
+        if (levels > L) levels = L;
+        const uint8_t* in_mask = lo.mask;
+        for (int i = 0; i < levels; ++i) {
+            const int l = L - 1 - i;
+            lo.desc[l].gout_row_mask = in_mask;
+            lo.desc[l].gout_row_count = i == 0 ? n_train : 0;
+            if (l > 0 && i + 1 < levels) { lo.desc[l].gin_row_mask = lo.rowmask[l]; in_mask = lo.rowmask[l]; }
+        }
+    }
     cudaStream_t s = ctx->side_stream[0];
     const cudaMemcpyKind H2D = cudaMemcpyHostToDevice, D2H = cudaMemcpyDeviceToHost;
 

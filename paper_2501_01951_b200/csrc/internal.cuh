@@ -32,10 +32,10 @@ void set_error(const char* fmt, ...);
         if (_s != MIXGCN_OK) return _s;      \
     } while (0)
 
-enum Phase { PH_SPMM = 0, PH_GEMM = 1, PH_ELEM = 2, PH_LOSS = 3, PH_ADAM = 4, PH_GRAPH = 5 };
+enum Phase { PH_SPMM = 0, PH_GEMM = 1, PH_ELEM = 2, PH_LOSS = 3, PH_ADAM = 4, PH_GRAPH = 5, PH_SPMM_SPARSE = 6 };
 
 // device status word codes
-enum { DEV_OK = 0, DEV_EMPTY_MASK = 1, DEV_BAD_LABEL = 2, DEV_WAIT_EXPIRED = 3 };
+enum { DEV_OK = 0, DEV_EMPTY_MASK = 1, DEV_BAD_LABEL = 2, DEV_WAIT_EXPIRED = 3, DEV_BAD_ROW_COUNT = 4 };
 
 struct ProfSpan {
     cudaEvent_t a, b;
@@ -50,6 +50,8 @@ struct mixgcn_ctx {
     int32_t* d_status;        // device status word (int32[4])
     void* workspace;          // grow-on-demand scratch of the dense products, column sums and the loss
     int64_t workspace_bytes;
+    void* workspace_rows;     // scratch of the row-sparse backward (row list, positions, compact operands)
+    int64_t workspace_rows_bytes;
     void* workspace_spmm;     // scratch of the aggregation (partial rows of long-row segments); separate so
     int64_t workspace_spmm_bytes;  // that an aggregation and a dense product may overlap on two streams
     cudaStream_t side_stream[2];
@@ -141,11 +143,20 @@ mixgcn_status ensure_workspace_spmm(mixgcn_ctx* ctx, int64_t bytes);
 // Builds (once) the schedules of the `chunks` row chunks of this orientation.  Synchronises on first use.
 mixgcn_status ensure_chunk_schedules(const mixgcn_graph* g, const CsrView& A, int chunks);
 
+// Row-sparse input of an aggregation: rows v with in_mask[v] == 0 are exactly zero and skipped; a
+// kept row v is read from row in_pos[v] of Y (null: row v); out_mask (nullable) receives which
+// output rows received a contribution.
+struct SpmmRowSparse {
+    const uint8_t* in_mask;
+    const int32_t* in_pos;
+    uint8_t* out_mask;
+};
+
 // kernels' host launchers (all asynchronous on `s`)
 // Aggregation over all rows (chunks <= 1) or over chunk k of `chunks` row chunks.
 mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView& A, int chunks, int k,
                           int32_t w, const float* Y, int64_t ldy, float* Z, int64_t ldz,
-                          const mixgcn_epilogue* epi, cudaStream_t s);
+                          const mixgcn_epilogue* epi, cudaStream_t s, const SpmmRowSparse* sparse = nullptr);
 mixgcn_status launch_gemm(mixgcn_ctx* ctx, int precision, int ta, int tb, int64_t M, int64_t N, int64_t K,
                           const float* A, int64_t lda, const float* B, int64_t ldb, float* C, int64_t ldc,
                           const mixgcn_epilogue* epi, int64_t epi_row0, cudaStream_t s);
@@ -153,6 +164,19 @@ mixgcn_status launch_colsum(mixgcn_ctx* ctx, int64_t n, int32_t d, const float* 
                             cudaStream_t s);
 mixgcn_status launch_gate(mixgcn_ctx* ctx, int64_t n, int32_t d, float* G, int64_t ldg, const float* X_out,
                           int64_t ldx, int relu, const uint8_t* drop_mask, float keep_scale, cudaStream_t s);
+
+// Row set of a row-sparse backward call, carved from the context's row workspace.
+struct RowSet {
+    int32_t* idx;    // [count] kept rows, ascending
+    int32_t* pos;    // [n] position of a kept row in idx, -1 otherwise
+    float* a;        // count x ld_a compact operand
+    float* b;        // count x ld_b compact operand
+    int64_t count;
+};
+mixgcn_status build_row_set(mixgcn_ctx* ctx, int64_t n, const uint8_t* mask, int64_t count, int64_t ld_a, int64_t ld_b,
+                            RowSet* rs, cudaStream_t s);
+mixgcn_status launch_gather_rows(mixgcn_ctx* ctx, int64_t count, int32_t d, const int32_t* idx, const float* src,
+                                 int64_t ld_src, float* dst, int64_t ld_dst, cudaStream_t s);
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 

@@ -1,0 +1,88 @@
+// Helpers of the row-sparse backward pass: when the gradient that enters a layer has only a few
+// non-zero rows (the masked loss gives non-zero rows on train nodes only), the dense products
+// run on the compacted rows and the aggregation skips the zero rows.
+#include <cub/cub.cuh>
+
+#include "internal.cuh"
+
+using namespace mixgcn;
+
+namespace {
+
+__global__ void pos_scatter_kernel(int64_t count, const int32_t* __restrict__ idx, int32_t* __restrict__ pos) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < count) pos[idx[i]] = (int32_t)i;
+}
+
+__global__ void check_count_kernel(const int64_t* selected, int64_t expected, int32_t* status) {
+    if (threadIdx.x == 0 && blockIdx.x == 0 && *selected != expected) atomicMax(status, DEV_BAD_ROW_COUNT);
+}
+
+// dst[i, :] = src[idx[i], :], float4 wide (ld multiples of 4, 16-byte aligned), d4 = ceil(d/4) groups per row
+__global__ void gather_rows_kernel(int64_t count, int d4, const int32_t* __restrict__ idx, const float* __restrict__ src,
+                                   int64_t ld_src, float* __restrict__ dst, int64_t ld_dst) {
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= count * d4) return;
+    const int64_t i = t / d4; const int c = (int)(t % d4);
+    reinterpret_cast<float4*>(dst + i * ld_dst)[c] = __ldg(reinterpret_cast<const float4*>(src + (int64_t)idx[i] * ld_src) + c);
+}
+
+}  // namespace
+
+namespace mixgcn {
+
+mixgcn_status ensure_workspace_rows(mixgcn_ctx* ctx, int64_t bytes) {
+    if (bytes <= ctx->workspace_rows_bytes) return MIXGCN_OK;
+    int64_t want = bytes + (bytes >> 3);
+    want = (want + 255) & ~(int64_t)255;
+    void* p = nullptr;
+    MIXGCN_CUDA(cudaDeviceSynchronize());
+    if (ctx->workspace_rows) cudaFree(ctx->workspace_rows);
+    ctx->workspace_rows = nullptr; ctx->workspace_rows_bytes = 0;
+    if (cudaMalloc(&p, (size_t)want) != cudaSuccess) {
+        cudaGetLastError();
+        MIXGCN_FAIL(MIXGCN_ENOMEM, "row-sparse workspace of %lld bytes could not be allocated", (long long)want);
+    }
+    ctx->workspace_rows = p; ctx->workspace_rows_bytes = want;
+    return MIXGCN_OK;
+}
+
+// Carves the row-sparse workspace and fills the row list and the position map of `mask`.
+// idx has capacity n (memory-safe whatever the mask holds); if the number of set rows differs from
+// `count` the device status word receives DEV_BAD_ROW_COUNT.
+mixgcn_status build_row_set(mixgcn_ctx* ctx, int64_t n, const uint8_t* mask, int64_t count, int64_t ld_a, int64_t ld_b,
+                            RowSet* rs, cudaStream_t s) {
+    size_t tb = 0;
+    cub::CountingInputIterator<int32_t> ids(0);
+    MIXGCN_CUDA(cub::DeviceSelect::Flagged(nullptr, tb, ids, mask, (int32_t*)nullptr, (int64_t*)nullptr, n, s));
+    auto up = [](int64_t x) { return (x + 255) & ~(int64_t)255; };
+    const int64_t o_pos = 0, o_idx = o_pos + up(n * 4), o_sel = o_idx + up(n * 4), o_tmp = o_sel + 256,
+                  o_a = o_tmp + up((int64_t)tb), o_b = o_a + up(count * ld_a * 4), total = o_b + up(count * ld_b * 4);
+    MIXGCN_TRY(ensure_workspace_rows(ctx, total));
+    char* base = reinterpret_cast<char*>(ctx->workspace_rows);
+    rs->pos = reinterpret_cast<int32_t*>(base + o_pos);
+    rs->idx = reinterpret_cast<int32_t*>(base + o_idx);
+    int64_t* selected = reinterpret_cast<int64_t*>(base + o_sel);
+    rs->a = reinterpret_cast<float*>(base + o_a);
+    rs->b = reinterpret_cast<float*>(base + o_b);
+    rs->count = count;
+    LaunchScope scope(ctx, PH_ELEM, s, 4);
+    MIXGCN_CUDA(cub::DeviceSelect::Flagged(base + o_tmp, tb, ids, mask, rs->idx, selected, n, s));
+    check_count_kernel<<<1, 32, 0, s>>>(selected, count, ctx->d_status);
+    MIXGCN_CUDA(cudaMemsetAsync(rs->pos, 0xFF, (size_t)n * 4, s));       // -1 everywhere
+    if (count > 0) pos_scatter_kernel<<<(unsigned)((count + 255) / 256), 256, 0, s>>>(count, rs->idx, rs->pos);
+    MIXGCN_CUDA(cudaGetLastError());
+    return MIXGCN_OK;
+}
+
+mixgcn_status launch_gather_rows(mixgcn_ctx* ctx, int64_t count, int32_t d, const int32_t* idx, const float* src,
+                                 int64_t ld_src, float* dst, int64_t ld_dst, cudaStream_t s) {
+    if (count <= 0) return MIXGCN_OK;
+    const int d4 = (d + 3) / 4;
+    LaunchScope scope(ctx, PH_ELEM, s);
+    gather_rows_kernel<<<(unsigned)((count * d4 + 255) / 256), 256, 0, s>>>(count, d4, idx, src, ld_src, dst, ld_dst);
+    MIXGCN_CUDA(cudaGetLastError());
+    return MIXGCN_OK;
+}
+
+}  // namespace mixgcn

@@ -44,6 +44,11 @@ struct SpmmParams {
     float* Z; int64_t ldz;
     float* partial;        // non-null: unit idx writes its raw sums to partial[idx * ldp + ...]
     int64_t ldp;
+    // row-sparse input (spmm_sparse_kernel): rows v of the input with in_mask[v] == 0 are exactly zero
+    // and are skipped; a kept row v is read from Y row in_pos[v] (in_pos == null: row v itself)
+    const uint8_t* in_mask;
+    const int32_t* in_pos;
+    uint8_t* out_mask;     // nullable: receives 1 for output rows that received a contribution, else 0
     // epilogue
     const float* bias; int relu;
     const uint8_t* drop; float keep_scale;
@@ -153,6 +158,85 @@ __global__ void __launch_bounds__(256, MIXGCN_SPMM_MINB) spmm_group_kernel(const
     }
 }
 
+// Row-sparse input: most rows of Y are exactly zero (gradients of a masked loss and what they
+// propagate to).  A unit scans its column ids, tests the row mask (one byte per entry, L2-resident)
+// and gathers only the kept rows, four at a time, in entry order -- the same sum as the dense kernel
+// with its zero terms left out.  Values are read for kept entries only.
+template <int LPR, int VPL>
+__global__ void __launch_bounds__(256) spmm_sparse_kernel(const SpmmParams p) {
+    const int lig = threadIdx.x % LPR;
+    const int64_t idx = p.idx_begin + ((int64_t)blockIdx.x * 256 + threadIdx.x) / LPR;
+    if (idx >= p.idx_end) return;
+    const int group_base = (threadIdx.x & 31) & ~(LPR - 1);
+    const unsigned mask = LPR == 32 ? 0xFFFFFFFFu : (((1u << LPR) - 1u) << group_base);
+    const int4 rc = __ldg(reinterpret_cast<const int4*>(p.rec + idx));
+    const int64_t b = ((int64_t)(uint32_t)rc.y << 32) | (uint32_t)rc.x, e = b + rc.z;
+    const int64_t u = rc.w;
+    const int w4 = (p.w + 3) >> 2;
+    const float* Yb = p.Y + p.j0;
+    float4 acc[VPL];
+#pragma unroll
+    for (int v = 0; v < VPL; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+    bool any = false;
+    for (int64_t i0 = b; i0 < e; i0 += LPR) {
+        int r = -1; float a = 0.0f;
+        if (i0 + lig < e) {
+            const int c = __ldg(p.col + i0 + lig);
+            if (__ldg(p.in_mask + c)) {
+                r = p.in_pos ? __ldg(p.in_pos + c) : c;
+                a = __ldg(p.val + i0 + lig);
+            }
+        }
+        unsigned hits = __ballot_sync(mask, r >= 0) & mask;
+        any |= hits != 0;
+        constexpr int HB = VPL >= 4 ? 1 : 4 / VPL;     // kept rows gathered per batch
+        while (hits) {
+            int src[HB], nh = 0;
+#pragma unroll
+            for (int t = 0; t < HB; ++t) {
+                src[t] = 0;
+                if (hits) { src[t] = __ffs(hits) - 1 - group_base; hits &= hits - 1; ++nh; }
+            }
+            int rk[HB]; float ak[HB]; float4 y[HB][VPL];
+#pragma unroll
+            for (int t = 0; t < HB; ++t) {
+                rk[t] = __shfl_sync(mask, r, src[t], LPR);
+                ak[t] = __shfl_sync(mask, a, src[t], LPR);
+            }
+#pragma unroll
+            for (int t = 0; t < HB; ++t) {
+                const float4* yr = reinterpret_cast<const float4*>(Yb + (int64_t)(rk[t] < 0 ? 0 : rk[t]) * p.ldy);
+#pragma unroll
+                for (int v = 0; v < VPL; ++v) {
+                    const int c4 = lig + v * LPR;
+                    y[t][v] = (t < nh && c4 < w4) ? __ldg(yr + c4) : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+            }
+#pragma unroll
+            for (int t = 0; t < HB; ++t)
+                if (t < nh) {
+#pragma unroll
+                    for (int v = 0; v < VPL; ++v) fma4(acc[v], ak[t], y[t][v]);
+                }
+        }
+    }
+    if (p.partial) {
+        float4* dst = reinterpret_cast<float4*>(p.partial + idx * p.ldp);
+#pragma unroll
+        for (int v = 0; v < VPL; ++v) {
+            const int c4 = lig + v * LPR;
+            if (c4 < w4) dst[c4] = acc[v];
+        }
+        return;
+    }
+    if (p.out_mask && lig == 0 && p.j0 == 0) p.out_mask[u] = any ? 1 : 0;
+#pragma unroll
+    for (int v = 0; v < VPL; ++v) {
+        const int c4 = lig + v * LPR;
+        if (c4 < w4) store_row(p, u, c4, acc[v]);
+    }
+}
+
 // Long rows: add the segments' partial rows in entry order, apply the epilogue, write Z.
 // One group of 32 lanes per long row.
 __global__ void __launch_bounds__(256) spmm_combine_kernel(const SpmmParams p, int64_t n_long,
@@ -165,6 +249,7 @@ __global__ void __launch_bounds__(256) spmm_combine_kernel(const SpmmParams p, i
     const int64_t s0 = seg_off[i], s1 = seg_off[i + 1];
     const int64_t u = perm[i];
     const int w4 = (p.w + 3) >> 2;
+    if (p.out_mask && lane == 0) p.out_mask[u] = 1;    // long rows are kept without looking (conservative)
     for (int c4 = lane; c4 < w4; c4 += 32) {
         float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
         for (int64_t q = s0; q < s1; ++q) {
@@ -205,6 +290,32 @@ int dispatch(const SpmmParams& p, int fold, cudaStream_t s) {
     return 0;
 }
 
+template <int LPR, int VPL>
+void launch_sparse(const SpmmParams& p, cudaStream_t s) {
+    const int64_t units = p.idx_end - p.idx_begin;
+    if (units <= 0) return;
+    const int per_block = 256 / LPR;
+    spmm_sparse_kernel<LPR, VPL><<<(unsigned)((units + per_block - 1) / per_block), 256, 0, s>>>(p);
+}
+
+void dispatch_sparse(const SpmmParams& p, int fold, cudaStream_t s) {
+    const int w4 = (p.w + 3) >> 2;
+    int lpr = 1;
+    while (lpr < 32 && lpr < w4) lpr <<= 1;
+    int vpl = (w4 + lpr - 1) / lpr;
+    while (fold > 1 && (lpr / fold < 1 || vpl * fold > 8)) fold >>= 1;
+    lpr /= fold; vpl *= fold;
+#define MIXGCN_SPMM_CASE(L, V) if (lpr == L && vpl == V) { launch_sparse<L, V>(p, s); return; }
+    MIXGCN_SPMM_CASE(32, 1) MIXGCN_SPMM_CASE(32, 2) MIXGCN_SPMM_CASE(32, 3) MIXGCN_SPMM_CASE(32, 4)
+    MIXGCN_SPMM_CASE(32, 5) MIXGCN_SPMM_CASE(32, 6) MIXGCN_SPMM_CASE(32, 7) MIXGCN_SPMM_CASE(32, 8)
+    MIXGCN_SPMM_CASE(16, 1) MIXGCN_SPMM_CASE(16, 2) MIXGCN_SPMM_CASE(16, 4) MIXGCN_SPMM_CASE(16, 6) MIXGCN_SPMM_CASE(16, 8)
+    MIXGCN_SPMM_CASE(8, 1) MIXGCN_SPMM_CASE(8, 2) MIXGCN_SPMM_CASE(8, 4) MIXGCN_SPMM_CASE(8, 8)
+    MIXGCN_SPMM_CASE(4, 1) MIXGCN_SPMM_CASE(4, 2) MIXGCN_SPMM_CASE(4, 4) MIXGCN_SPMM_CASE(4, 8)
+    MIXGCN_SPMM_CASE(2, 1) MIXGCN_SPMM_CASE(2, 2) MIXGCN_SPMM_CASE(2, 4) MIXGCN_SPMM_CASE(2, 8)
+    MIXGCN_SPMM_CASE(1, 1) MIXGCN_SPMM_CASE(1, 2) MIXGCN_SPMM_CASE(1, 4) MIXGCN_SPMM_CASE(1, 8)
+#undef MIXGCN_SPMM_CASE
+}
+
 constexpr int MAX_SLICE = 1024;  // columns per launch: 8 float4 per lane
 
 }  // namespace
@@ -215,7 +326,7 @@ namespace mixgcn {
 // with its own schedule: long rows as column-ordered segments, then rows longest first, short rows packed.
 mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView& A, int chunks, int k,
                           int32_t w, const float* Y, int64_t ldy, float* Z, int64_t ldz,
-                          const mixgcn_epilogue* epi, cudaStream_t s) {
+                          const mixgcn_epilogue* epi, cudaStream_t s, const SpmmRowSparse* sparse) {
     if (w <= 0) return MIXGCN_OK;
     if (chunks > 1) {
         MIXGCN_TRY(ensure_chunk_schedules(g, A, chunks));
@@ -231,9 +342,48 @@ mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView&
         p.gate = epi->gate; p.ld_gate = epi->ld_gate; p.gate_scale = epi->gate_scale;
     }
     p.rec = S.rec;
+    if (sparse) { p.in_mask = sparse->in_mask; p.in_pos = sparse->in_pos; p.out_mask = sparse->out_mask; }
     for (int j0 = 0; j0 < w; j0 += MAX_SLICE) {
         p.j0 = j0;
         p.w = (w - j0) < MAX_SLICE ? (w - j0) : MAX_SLICE;
+        if (sparse) {
+            // same units, sparse-input kernel: long-row segments to scratch + combine, then every other row
+            if (S.total_segs > 0) {
+                const int64_t ldp = ((int64_t)p.w + 3) / 4 * 4;
+                MIXGCN_TRY(ensure_workspace_spmm(ctx, S.total_segs * ldp * (int64_t)sizeof(float)));
+                p.partial = reinterpret_cast<float*>(ctx->workspace_spmm); p.ldp = ldp;
+                {
+                    LaunchScope scope(ctx, PH_SPMM_SPARSE, s);
+                    p.idx_begin = 0; p.idx_end = S.total_segs;
+                    dispatch_sparse(p, 1, s);
+                }
+                {
+                    LaunchScope scope(ctx, PH_SPMM_SPARSE, s);
+                    const int64_t blocks = (S.n_long * 32 + 255) / 256;
+                    spmm_combine_kernel<<<(unsigned)blocks, 256, 0, s>>>(p, S.n_long, S.seg_off, S.seg_pos, S.perm);
+                }
+                p.partial = nullptr;
+            }
+            {
+                // ordinary rows by degree bucket, short rows packed 2/4/8 per warp as in the dense path
+                int64_t bnd[5];
+                bnd[0] = S.n_long;
+                for (int q = 0; q < 3; ++q) bnd[q + 1] = S.rows_above[q] > S.n_long ? S.rows_above[q] : S.n_long;
+                bnd[4] = S.n_rows;
+                int64_t begin = bnd[0];
+                int fold = 1;
+                for (int q = 0; q < 4; ++q, fold <<= 1) {
+                    const int64_t end = bnd[q + 1];
+                    if (end <= begin) continue;
+                    p.idx_begin = S.total_segs + (begin - S.n_long);
+                    p.idx_end = S.total_segs + (end - S.n_long);
+                    LaunchScope scope(ctx, PH_SPMM_SPARSE, s);
+                    dispatch_sparse(p, fold, s);
+                    begin = end;
+                }
+            }
+            continue;
+        }
         if (S.total_segs > 0) {
             const int64_t ldp = ((int64_t)p.w + 3) / 4 * 4;
             MIXGCN_TRY(ensure_workspace_spmm(ctx, S.total_segs * ldp * (int64_t)sizeof(float)));

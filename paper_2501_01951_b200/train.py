@@ -18,7 +18,7 @@ def round4(x: int) -> int:
 
 class GcnTrainer:
     def __init__(self, ctx: mg.Ctx, graph: mg.Graph, dims, precision=mg.PREC_FP32, order=mg.ORDER_AUTO,
-                 n_chunks=0, fuse_gate=True, keep_scale=1.0, device=None):
+                 n_chunks=0, fuse_gate=True, keep_scale=1.0, device=None, row_sparse="auto"):
         self.ctx, self.g = ctx, graph
         self.dims = tuple(int(d) for d in dims)
         self.L = len(self.dims) - 1
@@ -26,6 +26,8 @@ class GcnTrainer:
         self.device = torch.device("cuda", ctx.device) if device is None else device
         self.ld = [round4(d) for d in self.dims]
         self.fuse_gate = fuse_gate
+        self.row_sparse = row_sparse          # "auto" | number of layers (from the top) whose backward gets a row mask
+        self.row_masks = None
         n, L = self.n, self.L
         orders = order if isinstance(order, (list, tuple)) else [order] * L
         self.descs, self.orders = [], []
@@ -86,6 +88,35 @@ class GcnTrainer:
         self.X[0], self.labels, self.train_mask = X0, labels, train_mask
         if drop_masks is not None:
             self.masks = list(drop_masks) + [None] * (self.L - len(drop_masks))
+        self._plan_row_sparsity()
+
+    def _plan_row_sparsity(self):
+        """The loss gradient is non-zero on train rows only; one aggregation later on their neighbours
+        only.  Hand those row masks to layer_bwd for the top `levels` layers (plumbing: the masks are
+        the train mask and byte arrays the library fills)."""
+        n, L = self.n, self.L
+        n_train = int(self.train_mask.sum().item())
+        frac = n_train / max(n, 1)
+        levels = self.row_sparse
+        if levels == "auto":
+            mean_entries = self.g.nnz / max(n, 1)
+            levels = 0 if frac >= 0.25 else (2 if frac * mean_entries < 0.5 else 1)
+        levels = max(0, min(int(levels), L))
+        self.row_sparse_levels = levels
+        self.row_masks = [None] * (L + 1)
+        for d in self.descs:
+            d.gout_row_mask, d.gout_row_count, d.gin_row_mask = None, 0, None
+        if levels == 0:
+            return
+        self.row_masks[L] = self.train_mask
+        for i in range(levels):
+            l = L - 1 - i                                 # layer whose backward receives row_masks[l + 1]
+            d = self.descs[l]
+            d.gout_row_mask = self.row_masks[l + 1].data_ptr()
+            d.gout_row_count = n_train if i == 0 else 0
+            if l > 0 and i + 1 < levels:
+                self.row_masks[l] = torch.zeros(n, dtype=torch.uint8, device=self.device)
+                d.gin_row_mask = self.row_masks[l].data_ptr()
 
     # -- the iteration --------------------------------------------------------------------------
     def forward(self):

@@ -578,3 +578,84 @@ def test_training_epoch_tf32_within_low_precision_bound(mg, ctx):
         assert np.linalg.norm(tr.db[l].cpu().numpy() - ref["db"][l]) <= TOL_LOWP * scale_b
         if l > 0:
             Gout = orc.aggregate(go, dZ, transposed=True)
+
+
+# --------------------------------------------------------------------------- row-sparse backward
+
+@pytest.mark.parametrize("name", ["messy-directed", "hub"])
+@pytest.mark.parametrize("order", ["agg", "upd"])
+@pytest.mark.parametrize("give_count", [True, False])
+def test_layer_bwd_row_sparse_matches_dense_definition(mg, ctx, name, order, give_count):
+    """G_out with a few non-zero rows: the row-sparse path (compacted products when the count is
+    given, masked aggregation otherwise) must give the dense definition's gradients."""
+    go, gg = build_both(mg, ctx, name)
+    n, d_in, d_out = go.n, 40, 24
+    o = mg.ORDER_AGG_FIRST if order == "agg" else mg.ORDER_UPD_FIRST
+    X = synth.uniform_tensor((n, d_in), 301, -1, 1)
+    W = synth.glorot_uniform(d_in, d_out, 302)
+    b = synth.uniform_tensor((d_out,), 303, -0.2, 0.2)
+    rows = synth.bernoulli_mask(n, 0.05, 304)
+    rows[0] = 1                                                       # the hub's own row is among them
+    Gout = synth.uniform_tensor((n, d_out), 305, -1, 1) * rows[:, None].float()
+    desc = mg.layer_desc(d_in, d_out, round4(d_in), round4(d_out), round4(max(d_in, d_out)), o, mg.PREC_FP32,
+                         mg.LAYER_RELU | mg.LAYER_GATE_GIN)
+    Xd, Wd, bd = padded(X), W.cuda(), b.cuda()
+    saved = torch.zeros(n, round4(max(d_in, d_out)), device="cuda")
+    Xout = torch.zeros(n, round4(d_out), device="cuda")
+    mg.layer_fwd(ctx, gg, desc, Xd, Wd, bd, None, saved, Xout)
+    rows_d = rows.cuda()
+    gin_mask = torch.full((n,), 7, dtype=torch.uint8, device="cuda")
+    desc.gout_row_mask = rows_d.data_ptr()
+    desc.gout_row_count = int(rows.sum()) if give_count else 0
+    desc.gin_row_mask = gin_mask.data_ptr()
+    Gd = padded(Gout)
+    Gin = torch.full((n, round4(d_in)), 5.0, device="cuda")
+    dW = torch.zeros(d_in, d_out, device="cuda"); db = torch.zeros(d_out, device="cuda")
+    mg.layer_bwd(ctx, gg, desc, Xd, saved, Xout, None, Wd, Gd, Gin, dW, db)
+    Z = orc.aggregate(go, X.numpy())
+    Pp = orc.update(Z, W.numpy(), b.numpy())
+    _, dWo, dbo, dZo = orc.update_bwd(Z, Pp, W.numpy(), Gout.numpy(), True)
+    want_gin = orc.aggregate(go, dZo, transposed=True) * (X.numpy() > 0)
+    assert rel_fro(host(dW), dWo) <= TOL_FP32 and rel_fro(db.cpu().numpy(), dbo) <= TOL_FP32
+    assert rel_fro(host(Gin, d_in), want_gin) <= TOL_FP32
+    m = gin_mask.cpu().numpy()
+    assert set(np.unique(m)) <= {0, 1}
+    nonzero_rows = np.abs(orc.aggregate(go, dZo, transposed=True)).sum(axis=1) > 0
+    assert np.all(m[nonzero_rows] == 1)                              # the reported mask covers every non-zero row
+    assert np.all(host(Gin, d_in)[m == 0] == 0)
+    assert mg.ctx_poll_status(ctx, raise_on_error=False) == 0
+
+
+def test_row_sparse_wrong_count_is_reported_not_a_fault(mg, ctx):
+    go, gg = build_both(mg, ctx, "messy-sym")
+    n, d = go.n, 8
+    desc = mg.layer_desc(d, d, 8, 8, 8, mg.ORDER_AGG_FIRST, mg.PREC_FP32, mg.LAYER_FIRST)
+    rows = torch.zeros(n, dtype=torch.uint8, device="cuda"); rows[:10] = 1
+    desc.gout_row_mask = rows.data_ptr(); desc.gout_row_count = 3      # wrong on purpose (host-side mistake)
+    X = torch.zeros(n, 8, device="cuda"); sv = torch.zeros(n, 8, device="cuda"); W = torch.zeros(d, d, device="cuda")
+    G = torch.zeros(n, 8, device="cuda"); dW = torch.zeros(d, d, device="cuda")
+    mg.layer_bwd(ctx, gg, desc, X, sv, X, None, W, G, None, dW, None)
+    assert mg.ctx_poll_status(ctx, raise_on_error=False) == 4
+
+
+@pytest.mark.parametrize("levels", [1, 2])
+def test_training_epoch_row_sparse_matches_oracle(mg, ctx, levels):
+    from paper_2501_01951_b200.train import GcnTrainer
+    wl, s, d, X, y, m, Ws, bs = _tiny_problem()
+    m = synth.bernoulli_mask(wl.n, 0.03, 77)                           # few train nodes
+    go = orc.graph_build(wl.n, s.numpy(), d.numpy())
+    gg = mg.graph_create(ctx, wl.n, s, d)
+    dims = (64, 32, 16, 8)                                             # three layers so that two levels exist
+    Ws = [synth.glorot_uniform(dims[i], dims[i + 1], 400 + i) for i in range(3)]
+    bs = [synth.uniform_tensor((dims[i + 1],), 410 + i, -0.1, 0.1) for i in range(3)]
+    tr = GcnTrainer(ctx, gg, dims, mg.PREC_FP32, order=mg.ORDER_AGG_FIRST, row_sparse=levels)
+    tr.set_params(Ws, bs)
+    tr.set_inputs(padded(X), y.cuda(), m.cuda())
+    assert tr.row_sparse_levels == levels
+    tr.forward(); tr.compute_loss(); tr.backward()
+    ref = orc.train_epoch(go, X.numpy(), [w.numpy() for w in Ws], [b.numpy() for b in bs], y.numpy(), m.numpy(), None, 1, **ADAM)
+    assert abs(tr.loss.item() - ref["loss"]) <= 1e-5 * abs(ref["loss"])
+    for l in range(3):
+        assert rel_fro(tr.dW[l].cpu().numpy(), ref["dW"][l]) <= TOL_FP32
+        assert rel_fro(tr.db[l].cpu().numpy(), ref["db"][l]) <= TOL_FP32
+    assert mg.ctx_poll_status(ctx, raise_on_error=False) == 0
