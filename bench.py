@@ -125,12 +125,18 @@ def spmm_alg_bytes(n, nnz, w):
     return 8 * (n + 1) + 4 * nnz + 4 * nnz + 4 * n * w + 4 * n * w
 
 
-def gemm_flops(n, dims, orders):
-    """2*M*N*K over the dense products of one epoch (forward, dW, and dX where it exists)."""
+def gemm_flops(n, dims, orders, compact_last_rows=None):
+    """2*M*N*K over the dense products of one epoch (forward, dW, and dX where it exists).  When the
+    last layer's backward runs on `compact_last_rows` compacted rows, its two products count those rows."""
     f = 0
-    for l in range(len(dims) - 1):
+    L = len(dims) - 1
+    for l in range(L):
         per = 2 * n * dims[l] * dims[l + 1]
-        f += per * (2 if l == 0 else 3)
+        nb = 1 if l == 0 else 2
+        if l == L - 1 and compact_last_rows is not None:
+            f += per + nb * 2 * compact_last_rows * dims[l] * dims[l + 1]
+        else:
+            f += per * (1 + nb)
     return f
 
 
@@ -222,7 +228,13 @@ def run_ours(args, rank, world, local_rank):
                     traffic=NCU_SPMM_CALL_DRAM_BYTES.get(args.workload), calls=spmm_calls, avg_call_ms=round(spmm_ms / max(spmm_calls, 1), 4),
                     alg_bytes_per_call=int(alg_bytes / max(spmm_calls, 1)),
                     gather_gbs=round(sum(4 * nnz * w * k for w, k in plan) * args.steps / (spmm_ms / 1e3) / 1e9, 1) if spmm_ms > 0 else 0.0)
-    flops = gemm_flops(n, wl.dims, tr.orders) * args.steps
+    if roofline["traffic"] and spmm_ms > 0:
+        # real DRAM throughput of the call: captured bytes over the call's measured duration
+        dram_gbs = roofline["traffic"] / (spmm_ms / max(spmm_calls, 1) / 1e3) / 1e9
+        roofline.update(dram_gbs=round(dram_gbs, 1), dram_frac=round(dram_gbs / peaks["hbm_gbs"], 4))
+    from paper_2501_01951_b200 import binding as _mg
+    compact = n_train if (tr.row_sparse_levels >= 1 and tr.orders[-1] == _mg.ORDER_AGG_FIRST and 4 * n_train < n) else None
+    flops = gemm_flops(n, wl.dims, tr.orders, compact) * args.steps
     gemm_ms = phase_ms["gemm"]
     gemm = dict(tflops=round(flops / (gemm_ms / 1e3) / 1e12, 2) if gemm_ms > 0 else 0.0,
                 frac_of_bf16_sustained=round(flops / (gemm_ms / 1e3) / 1e12 / peaks["bf16_tflops_sustained"], 4) if gemm_ms > 0 else 0.0,
