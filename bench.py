@@ -140,6 +140,20 @@ def gemm_flops(n, dims, orders, compact_last_rows=None):
     return f
 
 
+def gemm_min_bytes(n, dims, compact_last_rows=None):
+    """Minimum HBM bytes of the dense products of one epoch: forward reads n x d_in, writes n x d_out;
+    dW reads both; dX reads n x d_out, writes n x d_in (weights are negligible)."""
+    bts = 0
+    L = len(dims) - 1
+    for l in range(L):
+        rows_b = compact_last_rows if (l == L - 1 and compact_last_rows is not None) else n
+        bts += 4 * n * (dims[l] + dims[l + 1])
+        bts += 4 * rows_b * (dims[l] + dims[l + 1])
+        if l > 0:
+            bts += 4 * rows_b * (dims[l] + dims[l + 1])
+    return bts
+
+
 def build_problem(wl, device):
     src, dst = synth.rmat_graph(wl.n, wl.undirected_edges, wl.seed("graph"), device=device)
     torch.cuda.synchronize()
@@ -236,8 +250,14 @@ def run_ours(args, rank, world, local_rank):
     compact = n_train if (tr.row_sparse_levels >= 1 and tr.orders[-1] == _mg.ORDER_AGG_FIRST and 4 * n_train < n) else None
     flops = gemm_flops(n, wl.dims, tr.orders, compact) * args.steps
     gemm_ms = phase_ms["gemm"]
-    gemm = dict(tflops=round(flops / (gemm_ms / 1e3) / 1e12, 2) if gemm_ms > 0 else 0.0,
-                frac_of_bf16_sustained=round(flops / (gemm_ms / 1e3) / 1e12 / peaks["bf16_tflops_sustained"], 4) if gemm_ms > 0 else 0.0,
+    # The dense products run TF32 on the tensor cores: their peak is the measured bf16 peak times the
+    # nominal tf32/bf16 ratio (1.1 / 2.25).  Their minimum HBM bytes: every n x d operand and result once.
+    tf32_peak = peaks["bf16_tflops"] * 1.1 / 2.25
+    gbytes = gemm_min_bytes(n, wl.dims, compact) * args.steps
+    tfl = flops / (gemm_ms / 1e3) / 1e12 if gemm_ms > 0 else 0.0
+    gemm = dict(tflops=round(tfl, 2), tf32_peak_tflops=round(tf32_peak, 1), frac_of_tf32_peak=round(tfl / tf32_peak, 4),
+                min_hbm_gbs=round(gbytes / (gemm_ms / 1e3) / 1e9, 1) if gemm_ms > 0 else 0.0,
+                frac_of_hbm_peak=round(gbytes / (gemm_ms / 1e3) / 1e9 / peaks["hbm_gbs"], 4) if gemm_ms > 0 else 0.0,
                 ms_per_epoch=round(gemm_ms / args.steps, 3))
     breakdown = {k: round(v / args.steps, 3) for k, v in phase_ms.items()}
 
