@@ -64,6 +64,14 @@ mixgcn_status mixgcn_ctx_reserve(mixgcn_ctx* ctx, int64_t bytes);
  * 4 gout_row_count does not match gout_row_mask. */
 mixgcn_status mixgcn_ctx_poll_status(mixgcn_ctx* ctx, int32_t* code);
 
+/* Tuning options.  MIXGCN_OPT_SPMM_SLICE_COLS: width of the feature-column slices an aggregation is
+ * processed in (Algorithm 2's p:q-1 column ranges on one GPU): 0 = one slice up to 1024 columns
+ * (default); otherwise a multiple of 4 in [4, 1024].  Narrow slices shrink the part of the input
+ * that must stay in the L2 at the price of re-reading the index once per slice; results do not
+ * depend on the slicing. */
+#define MIXGCN_OPT_SPMM_SLICE_COLS 1
+mixgcn_status mixgcn_ctx_set_option(mixgcn_ctx* ctx, int32_t option, int64_t value);
+
 /* Per-phase profiling.  While enabled the library brackets every kernel it launches with
  * CUDA events on the launching stream.  mixgcn_ctx_profile_read synchronises and returns, for
  * each phase, accumulated milliseconds and launch counts since the last read, then resets.

@@ -38,7 +38,7 @@ SYMBOLS = (
     "mixgcn_graph_create", "mixgcn_graph_create_from_csr", "mixgcn_graph_info", "mixgcn_graph_export",
     "mixgcn_graph_export_schedule", "mixgcn_graph_destroy", "mixgcn_spmm", "mixgcn_gemm",
     "mixgcn_layer_plan", "mixgcn_layer_fwd", "mixgcn_layer_bwd", "mixgcn_loss_softmax_xent",
-    "mixgcn_adam_step", "mixgcn_train_step_host", "mixgcn_loss_softmax_xent_noalloc",
+    "mixgcn_adam_step", "mixgcn_train_step_host", "mixgcn_loss_softmax_xent_noalloc", "mixgcn_ctx_set_option",
 )
 
 
@@ -131,6 +131,13 @@ def ctx_poll_status(ctx: Ctx, raise_on_error: bool = True) -> int:
     if raise_on_error:
         _check(st)
     return code.value
+
+
+OPT_SPMM_SLICE_COLS = 1
+
+
+def ctx_set_option(ctx: Ctx, option: int, value: int):
+    _check(lib.mixgcn_ctx_set_option(ctx.h, C.c_int32(option), C.c_int64(value)))
 
 
 def ctx_profile_enable(ctx: Ctx, enable: bool = True):

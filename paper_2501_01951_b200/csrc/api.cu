@@ -184,6 +184,17 @@ extern "C" mixgcn_status mixgcn_ctx_poll_status(mixgcn_ctx* ctx, int32_t* code) 
     MIXGCN_FAIL(MIXGCN_EDEVICE, h == DEV_EMPTY_MASK ? "loss: the train mask is empty" : h == DEV_BAD_LABEL ? "loss: a label lies outside [0, C)" : "layer_bwd: gout_row_count does not match gout_row_mask");
 }
 
+extern "C" mixgcn_status mixgcn_ctx_set_option(mixgcn_ctx* ctx, int32_t option, int64_t value) {
+    if (!ctx) MIXGCN_FAIL(MIXGCN_EINVAL, "ctx_set_option: null ctx");
+    if (option == MIXGCN_OPT_SPMM_SLICE_COLS) {
+        if (value != 0 && (value < 4 || value > 1024 || (value & 3)))
+            MIXGCN_FAIL(MIXGCN_EINVAL, "ctx_set_option: slice width must be 0 or a multiple of 4 in [4, 1024] (got %lld)", (long long)value);
+        ctx->spmm_slice_cols = (int)value;
+        return MIXGCN_OK;
+    }
+    MIXGCN_FAIL(MIXGCN_EINVAL, "ctx_set_option: unknown option %d", option);
+}
+
 extern "C" mixgcn_status mixgcn_ctx_profile_enable(mixgcn_ctx* ctx, int enable) {
     if (!ctx) MIXGCN_FAIL(MIXGCN_EINVAL, "ctx_profile_enable: null ctx");
     ctx->profile = enable ? 1 : 0;

@@ -57,6 +57,7 @@ struct mixgcn_ctx {
     cudaStream_t side_stream[2];
     cudaEvent_t fork_ev, join_ev[2];
     cudaEvent_t chunk_ev[64];
+    int spmm_slice_cols;      // 0 = default (one slice up to 1024 columns)
     // profiling
     int profile;
     mixgcn::ProfSpan* spans;
@@ -127,7 +128,12 @@ namespace mixgcn {
 constexpr int SPMM_SEG = MIXGCN_SPMM_SEG;                 // rows longer than this are cut into segments of at most this many entries
 constexpr int SPMM_BLK_MIN_ENTRIES = MIXGCN_SPMM_BLK_MIN; // a long row uses 2^k column blocks while it keeps >= this many entries per block
 constexpr int SPMM_MAX_LOG_BLOCKS = MIXGCN_SPMM_LOG_BLOCKS; // at most 2^this column blocks per row
-constexpr int SPMM_PACK_DEG[3] = {12, 5, 2};       // rows up to these lengths share a warp 2-, 4-, 8-fold
+#ifndef MIXGCN_SPMM_PACK0
+#define MIXGCN_SPMM_PACK0 12
+#define MIXGCN_SPMM_PACK1 5
+#define MIXGCN_SPMM_PACK2 2
+#endif
+constexpr int SPMM_PACK_DEG[3] = {MIXGCN_SPMM_PACK0, MIXGCN_SPMM_PACK1, MIXGCN_SPMM_PACK2};   // rows up to these lengths share a warp 2-, 4-, 8-fold
 
 // Launch bookkeeping: counts the launch and, when profiling, brackets it with events.
 struct LaunchScope {

@@ -343,9 +343,10 @@ mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView&
     }
     p.rec = S.rec;
     if (sparse) { p.in_mask = sparse->in_mask; p.in_pos = sparse->in_pos; p.out_mask = sparse->out_mask; }
-    for (int j0 = 0; j0 < w; j0 += MAX_SLICE) {
+    const int slice = ctx->spmm_slice_cols > 0 ? ctx->spmm_slice_cols : MAX_SLICE;
+    for (int j0 = 0; j0 < w; j0 += slice) {
         p.j0 = j0;
-        p.w = (w - j0) < MAX_SLICE ? (w - j0) : MAX_SLICE;
+        p.w = (w - j0) < slice ? (w - j0) : slice;
         if (sparse) {
             // same units, sparse-input kernel: long-row segments to scratch + combine, then every other row
             if (S.total_segs > 0) {

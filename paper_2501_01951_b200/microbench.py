@@ -48,10 +48,13 @@ def main():
     ap.add_argument("--iters", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=2)
     ap.add_argument("--seed", type=int, default=1005)
+    ap.add_argument("--slice", type=int, default=0, help="feature-column slice width of the aggregation (0 = default)")
     args = ap.parse_args()
 
     dev = torch.device("cuda", 0)
     ctx = mg.ctx_create(0)
+    if args.slice:
+        mg.ctx_set_option(ctx, mg.OPT_SPMM_SLICE_COLS, args.slice)
     out = dict(op=args.op)
     if args.op == "spmm":
         s, d = synth.rmat_graph(args.n, args.edges, args.seed, device=dev)

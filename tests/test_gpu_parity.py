@@ -659,3 +659,23 @@ def test_training_epoch_row_sparse_matches_oracle(mg, ctx, levels):
         assert rel_fro(tr.dW[l].cpu().numpy(), ref["dW"][l]) <= TOL_FP32
         assert rel_fro(tr.db[l].cpu().numpy(), ref["db"][l]) <= TOL_FP32
     assert mg.ctx_poll_status(ctx, raise_on_error=False) == 0
+
+
+def test_spmm_column_slices_do_not_change_the_result(mg):
+    """Feature-column slicing (the p:q-1 ranges of Algorithm 2) is a schedule, not arithmetic."""
+    c2 = mg.ctx_create(0)
+    n, s, d, sym = GRAPHS["hub"]()
+    gg = mg.graph_create(c2, n, i32(s), i32(d))
+    X = padded(synth.uniform_tensor((n, 172), 501, -1, 1))
+    Z0 = torch.zeros_like(X); Z1 = torch.zeros_like(X); Z2 = torch.zeros_like(X)
+    mg.spmm(c2, gg, X, Z0, 172)
+    mg.ctx_set_option(c2, mg.OPT_SPMM_SLICE_COLS, 32)
+    mg.spmm(c2, gg, X, Z1, 172)
+    mg.ctx_set_option(c2, mg.OPT_SPMM_SLICE_COLS, 100)
+    mg.spmm(c2, gg, X, Z2, 172)
+    assert torch.equal(Z0, Z1) and torch.equal(Z0, Z2)
+    with pytest.raises(mg.MixgcnError):
+        mg.ctx_set_option(c2, mg.OPT_SPMM_SLICE_COLS, 6)
+    with pytest.raises(mg.MixgcnError):
+        mg.ctx_set_option(c2, 99, 1)
+    gg.close(); c2.close()
