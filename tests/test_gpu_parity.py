@@ -679,3 +679,86 @@ def test_spmm_column_slices_do_not_change_the_result(mg):
     with pytest.raises(mg.MixgcnError):
         mg.ctx_set_option(c2, 99, 1)
     gg.close(); c2.close()
+
+
+# --------------------------------------------------------------------------- more tensor-core paths
+
+def test_gemm_tf32_generic_epilogue_and_wide_bias(mg, ctx):
+    """The tensor-core kernel's per-element epilogue (dropout mask, gate) and the bias path for N > 1024."""
+    from helpers import TOL_LOWP
+    M, N, K = 333, 70, 96
+    A, B = synth.uniform_tensor((M, K), 601, -1, 1), synth.uniform_tensor((K, N), 602, -1, 1)
+    bias = synth.uniform_tensor((N,), 603, -1, 1)
+    drop = (synth.uniform_tensor((M, N), 604, 0, 1) < 0.5).to(torch.uint8)
+    gate = synth.uniform_tensor((M, N), 605, -1, 1)
+    Cd = torch.zeros(M, round4(N), device="cuda")
+    epi = mg.make_epilogue(bias=bias.cuda(), relu=True, drop_mask=drop.cuda(), keep_scale=2.0, gate=padded(gate), gate_scale=0.5)
+    mg.gemm(ctx, mg.PREC_TF32, False, False, M, N, K, padded(A), padded(B), Cd, epi=epi)
+    want = orc.activation(orc.update(A.numpy(), B.numpy(), bias.numpy()), True, drop.numpy(), 2.0) * np.where(gate.numpy() > 0, 0.5, 0.0)
+    assert rel_fro(host(Cd, N), want) <= TOL_LOWP
+    M, N, K = 200, 1100, 64
+    A, B = synth.uniform_tensor((M, K), 611, -1, 1), synth.uniform_tensor((K, N), 612, -1, 1)
+    bias = synth.uniform_tensor((N,), 613, -1, 1)
+    Cd = torch.zeros(M, round4(N), device="cuda")
+    mg.gemm(ctx, mg.PREC_TF32, False, False, M, N, K, padded(A), padded(B), Cd, epi=mg.make_epilogue(bias=bias.cuda(), relu=True))
+    assert rel_fro(host(Cd, N), orc.activation(orc.update(A.numpy(), B.numpy(), bias.numpy()), True)) <= TOL_LOWP
+    assert mg.ctx_poll_status(ctx, raise_on_error=False) == 0
+
+
+@pytest.mark.parametrize("order", ["agg", "upd"])
+def test_layer_tf32_with_dropout_both_orders(mg, ctx, order):
+    from helpers import TOL_LOWP
+    go, gg = build_both(mg, ctx, "messy-directed")
+    n, d_in, d_out = go.n, 48, 40
+    o = mg.ORDER_AGG_FIRST if order == "agg" else mg.ORDER_UPD_FIRST
+    X = synth.uniform_tensor((n, d_in), 621, -1, 1)
+    W = synth.glorot_uniform(d_in, d_out, 622)
+    b = synth.uniform_tensor((d_out,), 623, -0.2, 0.2)
+    Gout = synth.uniform_tensor((n, d_out), 624, -1, 1)
+    drop = (synth.uniform_tensor((n, d_out), 625, 0, 1) < 0.6).to(torch.uint8)
+    ks = 1 / 0.6
+    desc = mg.layer_desc(d_in, d_out, round4(d_in), round4(d_out), round4(max(d_in, d_out)), o, mg.PREC_TF32,
+                         mg.LAYER_RELU | mg.LAYER_GATE_GIN, ks, 1.0, 0)
+    Xd, Wd, bd, dd = padded(X), W.cuda(), b.cuda(), drop.cuda()
+    saved = torch.zeros(n, round4(max(d_in, d_out)), device="cuda"); Xout = torch.zeros(n, round4(d_out), device="cuda")
+    mg.layer_fwd(ctx, gg, desc, Xd, Wd, bd, dd, saved, Xout)
+    Z = orc.aggregate(go, X.numpy()); Pp = orc.update(Z, W.numpy(), b.numpy())
+    assert rel_fro(host(Xout, d_out), orc.activation(Pp, True, drop.numpy(), ks)) <= TOL_LOWP
+    Gd = padded(Gout); Gin = torch.zeros(n, round4(d_in), device="cuda")
+    dW = torch.zeros(d_in, d_out, device="cuda"); db = torch.zeros(d_out, device="cuda")
+    mg.layer_bwd(ctx, gg, desc, Xd, saved, Xout, dd, Wd, Gd, Gin, dW, db)
+    dP, dWo, dbo, dZo = orc.update_bwd(Z, Pp, W.numpy(), Gout.numpy(), True, drop.numpy(), ks)
+    assert np.linalg.norm(host(dW) - dWo) <= TOL_LOWP * np.linalg.norm(np.abs(Z).T @ np.abs(dP))
+    assert rel_fro(db.cpu().numpy(), dbo) <= TOL_LOWP
+    want_gin = orc.aggregate(go, dZo, transposed=True) * (X.numpy() > 0)
+    assert rel_fro(host(Gin, d_in), want_gin) <= TOL_LOWP
+    assert mg.ctx_poll_status(ctx, raise_on_error=False) == 0
+
+
+def test_train_step_host_row_sparse_matches_oracle(mg, ctx):
+    """Few train nodes: the host-buffer step takes the row-sparse backward."""
+    wl, s, d, X, y, m, Ws, bs = _tiny_problem()
+    m = synth.bernoulli_mask(wl.n, 0.02, 88)
+    gg = mg.graph_create(ctx, wl.n, s, d)
+    go = orc.graph_build(wl.n, s.numpy(), d.numpy())
+    W = [w.clone() for w in Ws]; b = [x.clone() for x in bs]
+    z = lambda lst: [torch.zeros_like(x) for x in lst]
+    mW, vW, mb, vb = z(W), z(W), z(b), z(b)
+    loss = mg.train_step_host(ctx, gg, wl.dims, mg.PREC_FP32, X, y, m, W, b, mW, vW, mb, vb, 1, **ADAM)
+    ref = orc.train_epoch(go, X.numpy(), [w.numpy() for w in Ws], [x.numpy() for x in bs], y.numpy(), m.numpy(), None, 1, **ADAM)
+    assert abs(loss - ref["loss"]) <= 1e-5 * abs(ref["loss"])
+    for l in range(len(W)):
+        # first moments are (1 - beta1) * gradient after one step: an exact view of dW, db
+        assert rel_fro(mW[l].numpy() / (1 - ADAM["beta1"]), ref["dW"][l]) <= 2e-5
+        assert rel_fro(mb[l].numpy() / (1 - ADAM["beta1"]), ref["db"][l]) <= 2e-5
+    assert mg.ctx_poll_status(ctx, raise_on_error=False) == 0
+
+
+def test_graph_size_limits_are_checked_on_the_host(mg, ctx):
+    e = i32([])
+    with pytest.raises(mg.MixgcnError) as ex:
+        mg.graph_create(ctx, 2**31 - 1, e, e)
+    assert ex.value.status == mg.EBADGRAPH
+    with pytest.raises(mg.MixgcnError) as ex:
+        mg.graph_create(ctx, -5, e, e)
+    assert ex.value.status == mg.EINVAL
