@@ -267,3 +267,65 @@ void oracle_adam(int64_t numel, double* theta, const double* g, double* m, doubl
         theta[i] -= lr * (m[i] / c1) / (sqrt(v[i] / c2) + eps);
     }
 }
+
+/* ------------------------------------------------------------------------------------------------
+ * Node reordering for the fine-grain pipeline (Section 3.2.2).
+ * ------------------------------------------------------------------------------------------------ */
+
+/* Graph bandwidth b = max over stored entries (u,v) of p_v - p_u, p = position in the processing
+ * sequence (pos == NULL: identity). */
+int64_t oracle_bandwidth(int64_t n, const int64_t* rowptr, const int32_t* col, const int64_t* pos) {
+    int64_t b = 0;
+    for (int64_t u = 0; u < n; ++u)
+        for (int64_t i = rowptr[u]; i < rowptr[u + 1]; ++i) {
+            int64_t pu = pos ? pos[u] : u, pv = pos ? pos[col[i]] : col[i];
+            if (pv - pu > b) b = pv - pu;
+        }
+    return b;
+}
+
+/* Reverse Cuthill-McKee on a symmetric structure: components are started from the unvisited node of
+ * fewest entries (lowest id on ties); a dequeued node appends its unvisited neighbours by increasing
+ * entry count (lowest id on ties); the resulting sequence is reversed.  order[k] = node at position k. */
+void oracle_rcm(int64_t n, const int64_t* rowptr, const int32_t* col, int64_t* order) {
+    char* seen = (char*)calloc((size_t)n, 1);
+    int64_t* byd = (int64_t*)malloc((size_t)n * sizeof(int64_t));
+    int64_t* tmp = (int64_t*)malloc((size_t)n * sizeof(int64_t));
+    int64_t head = 0, tail = 0, next_start = 0;
+    /* nodes by (entry count, id): counting sort on the entry count */
+    int64_t maxd = 0;
+    for (int64_t u = 0; u < n; ++u) { int64_t d = rowptr[u + 1] - rowptr[u]; if (d > maxd) maxd = d; }
+    int64_t* cnt = (int64_t*)calloc((size_t)maxd + 2, sizeof(int64_t));
+    for (int64_t u = 0; u < n; ++u) cnt[rowptr[u + 1] - rowptr[u] + 1]++;
+    for (int64_t d = 0; d <= maxd; ++d) cnt[d + 1] += cnt[d];
+    for (int64_t u = 0; u < n; ++u) byd[cnt[rowptr[u + 1] - rowptr[u]]++] = u;
+    while (tail < n) {
+        while (seen[byd[next_start]]) ++next_start;
+        int64_t s = byd[next_start];
+        seen[s] = 1; order[tail++] = s;
+        while (head < tail) {
+            int64_t x = order[head++];
+            int64_t m = 0;
+            for (int64_t i = rowptr[x]; i < rowptr[x + 1]; ++i) {
+                int64_t y = col[i];
+                if (!seen[y]) { seen[y] = 1; tmp[m++] = y; }
+            }
+            /* insertion sort by entry count; the list is in ascending id, so ties keep the lower id first */
+            for (int64_t a = 1; a < m; ++a) {
+                int64_t y = tmp[a], dy = rowptr[y + 1] - rowptr[y], b = a;
+                while (b > 0 && rowptr[tmp[b - 1] + 1] - rowptr[tmp[b - 1]] > dy) { tmp[b] = tmp[b - 1]; --b; }
+                tmp[b] = y;
+            }
+            for (int64_t a = 0; a < m; ++a) order[tail++] = tmp[a];
+        }
+    }
+    for (int64_t a = 0, b = n - 1; a < b; ++a, --b) { int64_t t = order[a]; order[a] = order[b]; order[b] = t; }
+    free(seen); free(byd); free(tmp); free(cnt);
+}
+
+/* Proposition 3.5: with s batches idleness disappears when (n - b) / (2n) >= 1 / s; the stage count
+ * the evaluation uses is the smallest such s, ceil(2n / (n - b)).  Returns -1 when b >= n. */
+int64_t oracle_pipeline_stages(int64_t n, int64_t b) {
+    if (b >= n) return -1;
+    return (2 * n + (n - b) - 1) / (n - b);
+}

@@ -257,3 +257,30 @@ def train_epoch(g: Graph, X0, Ws, bs, labels, train_mask, state=None, t=1, lr=0.
         newW.append(W2); newb.append(b2)
     return dict(loss=lo, logits=Xs[-1], pred=pred, n_correct=ncorrect, n_train=T, G=G,
                 Zs=Zs, Ps=Ps, Xs=Xs, dW=dWs, db=dbs, W=newW, b=newb, state=state)
+
+
+# ------------------------------------------------------------------------------ node reordering
+
+def bandwidth(g: Graph, order=None) -> int:
+    """b = max over stored entries (u,v) of p_v - p_u (Section 3.2.2); order[k] = node at position k."""
+    pos = None
+    if order is not None:
+        pos = np.empty(g.n, dtype=np.int64)
+        pos[np.asarray(order, dtype=np.int64)] = np.arange(g.n, dtype=np.int64)
+    L = lib()
+    L.oracle_bandwidth.restype = C.c_int64
+    return int(L.oracle_bandwidth(C.c_int64(g.n), _p(g.rowptr, C.c_int64), _p(g.col, C.c_int32), _p(pos, C.c_int64)))
+
+
+def rcm(g: Graph):
+    """Reverse Cuthill-McKee order of a symmetric graph: order[k] = node at position k."""
+    order = np.zeros(g.n, dtype=np.int64)
+    lib().oracle_rcm(C.c_int64(g.n), _p(g.rowptr, C.c_int64), _p(g.col, C.c_int32), _p(order, C.c_int64))
+    return order
+
+
+def pipeline_stages(n: int, b: int) -> int:
+    """ceil(2n / (n - b)) (Proposition 3.5 and the stage count of the evaluation)."""
+    L = lib()
+    L.oracle_pipeline_stages.restype = C.c_int64
+    return int(L.oracle_pipeline_stages(C.c_int64(n), C.c_int64(b)))

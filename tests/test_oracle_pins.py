@@ -401,3 +401,66 @@ def test_workloads_take_the_papers_table_shapes():
     assert c2.dims[0] == feats and c2.classes == classes
     _, _, feats, classes = rows["ogbn-papers100M"]
     assert c5.dims[0] == feats and c5.classes == classes
+
+
+# ----------------------------------------------------------------------- node reordering (Section 3.2.2)
+
+def _brute_bandwidth(n, g, order):
+    pos = np.empty(n, dtype=np.int64); pos[order] = np.arange(n)
+    return max(abs(pos[u] - pos[v]) for u in range(n) for v in g.col[g.rowptr[u]:g.rowptr[u + 1]])
+
+
+def test_bandwidth_closed_forms_and_bruteforce():
+    n = 40
+    s = np.arange(n - 1)
+    path = orc.graph_build(n, s, s + 1)
+    assert orc.bandwidth(path) == 1                                   # a path in its natural order
+    assert orc.bandwidth(orc.graph_build(n, *ring(n))) == n - 1       # the closing edge of a ring
+    assert orc.bandwidth(orc.graph_build(n, np.zeros(n - 1, np.int64), np.arange(1, n))) == n - 1    # star, centre first
+    assert orc.bandwidth(orc.graph_build(n, [], [])) == 0
+    rng = np.random.default_rng(5)
+    g = orc.graph_build(n, rng.integers(0, n, 90), rng.integers(0, n, 90))
+    order = rng.permutation(n)
+    assert orc.bandwidth(g, order) == _brute_bandwidth(n, g, order)
+
+
+def test_rcm_is_a_valid_order_and_matches_scipy_quality():
+    from scipy.sparse.csgraph import reverse_cuthill_mckee
+    rng = np.random.default_rng(6)
+    for n, m in ((30, 40), (200, 400), (500, 700)):
+        g = orc.graph_build(n, rng.integers(0, n, m), rng.integers(0, n, m))
+        order = orc.rcm(g)
+        assert np.array_equal(np.sort(order), np.arange(n))
+        M = sp.csr_matrix((np.ones(g.nnz), g.col, g.rowptr), shape=(n, n))
+        ref = reverse_cuthill_mckee(M, symmetric_mode=True)
+        b_ours, b_ref, b_nat = orc.bandwidth(g, order), orc.bandwidth(g, ref.astype(np.int64)), orc.bandwidth(g)
+        # tie-breaking rules differ between implementations, so compare the quality of the result
+        assert b_ours <= 1.25 * b_ref + 2 and b_ours < b_nat
+
+
+def test_rcm_on_structured_graphs():
+    # a path given in scrambled labels is recovered as a path: bandwidth 1
+    n = 64
+    rng = np.random.default_rng(7)
+    lab = rng.permutation(n)
+    g = orc.graph_build(n, lab[:-1], lab[1:])
+    assert orc.bandwidth(g) > 1 and orc.bandwidth(g, orc.rcm(g)) == 1
+    # a 2-D grid r x c has bandwidth min(r, c) under the level order RCM produces
+    r, c = 6, 9
+    idx = np.arange(r * c).reshape(r, c)
+    s = np.concatenate([idx[:, :-1].ravel(), idx[:-1, :].ravel()]); d = np.concatenate([idx[:, 1:].ravel(), idx[1:, :].ravel()])
+    g = orc.graph_build(r * c, s, d)
+    assert orc.bandwidth(g, orc.rcm(g)) <= min(r, c) + 1
+    # components: every node appears once; isolated nodes are placed too
+    g = orc.graph_build(10, [0, 1, 5], [1, 2, 6])
+    assert np.array_equal(np.sort(orc.rcm(g)), np.arange(10))
+
+
+def test_pipeline_stage_count():
+    # the paper's remark: b = 0.8 n still allows a pipeline, with 2 / 0.2 = 10 stages
+    assert orc.pipeline_stages(1000, 800) == 10
+    assert orc.pipeline_stages(1000, 0) == 2 and orc.pipeline_stages(1000, 1) == 3
+    assert orc.pipeline_stages(1000, 999) == 2000 and orc.pipeline_stages(1000, 1000) == -1
+    for n, b in ((37, 5), (100, 33), (12345, 6789)):
+        s = orc.pipeline_stages(n, b)
+        assert (n - b) / (2 * n) >= 1 / s and (s == 1 or (n - b) / (2 * n) < 1 / (s - 1))
