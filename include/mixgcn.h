@@ -125,6 +125,25 @@ mixgcn_status mixgcn_graph_export_schedule(const mixgcn_graph* g, int transposed
 
 mixgcn_status mixgcn_graph_destroy(mixgcn_graph* g);
 
+/* Node reordering for the fine-grain pipeline (Section 3.2.2).
+ * mixgcn_graph_bandwidth: b = max over stored entries (u,v) of p_v - p_u, where p is the position
+ *   of a node in the processing sequence `order` (host int32[n], order[k] = node at position k;
+ *   NULL = the identity).  Runs on the device; synchronises.
+ * mixgcn_graph_rcm: the reverse Cuthill-McKee order of a symmetric graph into `order` (host
+ *   int32[n]): components start from the unvisited node with the fewest entries (lowest id on ties), a
+ *   visited node appends its unvisited neighbours by increasing entry count (lowest id on ties), and
+ *   the sequence is reversed.  A host (C++) breadth-first search, as the paper's preprocessing is;
+ *   synchronises and copies the structure to the host.  MIXGCN_EUNSUPPORTED if not symmetric.
+ * mixgcn_pipeline_stages: the stage count ceil(2n / (n - b)) of Proposition 3.5 (idleness is
+ *   eliminated when (n - b) / (2n) >= 1 / s); MIXGCN_EINVAL when b >= n.
+ * mixgcn_graph_create_permuted: a new graph in which node order[k] has become node k (same
+ *   entries, relabelled); the caller permutes features, labels and masks the same way. */
+mixgcn_status mixgcn_graph_bandwidth(const mixgcn_graph* g, const int32_t* order, int64_t* bandwidth);
+mixgcn_status mixgcn_graph_rcm(const mixgcn_graph* g, int32_t* order);
+mixgcn_status mixgcn_pipeline_stages(int64_t n, int64_t b, int64_t* stages);
+mixgcn_status mixgcn_graph_create_permuted(mixgcn_ctx* ctx, const mixgcn_graph* g, const int32_t* order,
+                                           mixgcn_graph** out);
+
 /* ------------------------------------------------------------------------------------------
  * Building blocks (device pointers).  The layer calls below are compositions of these.
  * ------------------------------------------------------------------------------------------ */

@@ -39,6 +39,7 @@ SYMBOLS = (
     "mixgcn_graph_export_schedule", "mixgcn_graph_destroy", "mixgcn_spmm", "mixgcn_gemm",
     "mixgcn_layer_plan", "mixgcn_layer_fwd", "mixgcn_layer_bwd", "mixgcn_loss_softmax_xent",
     "mixgcn_adam_step", "mixgcn_train_step_host", "mixgcn_loss_softmax_xent_noalloc", "mixgcn_ctx_set_option",
+    "mixgcn_graph_bandwidth", "mixgcn_graph_rcm", "mixgcn_pipeline_stages", "mixgcn_graph_create_permuted",
 )
 
 
@@ -217,6 +218,36 @@ def graph_export_schedule(g: Graph, transposed: bool = False) -> torch.Tensor:
     perm = torch.empty(g.n, dtype=torch.int32)
     _check(lib.mixgcn_graph_export_schedule(g.h, C.c_int(int(transposed)), _ptr(perm)))
     return perm
+
+
+def graph_bandwidth(g: Graph, order: torch.Tensor | None = None) -> int:
+    """b = max over stored entries of p_v - p_u for the processing sequence `order` (host int32; None = identity)."""
+    if order is not None and (order.is_cuda or order.dtype != torch.int32 or order.numel() != g.n):
+        raise TypeError("order: host int32 tensor of length n")
+    b = C.c_int64(0)
+    _check(lib.mixgcn_graph_bandwidth(g.h, _ptr(None if order is None else order.contiguous()), C.byref(b)))
+    return b.value
+
+
+def graph_rcm(g: Graph) -> torch.Tensor:
+    """Reverse Cuthill-McKee order (host int32 tensor, order[k] = node at position k)."""
+    order = torch.empty(g.n, dtype=torch.int32)
+    _check(lib.mixgcn_graph_rcm(g.h, _ptr(order)))
+    return order
+
+
+def pipeline_stages(n: int, b: int) -> int:
+    s = C.c_int64(0)
+    _check(lib.mixgcn_pipeline_stages(C.c_int64(n), C.c_int64(b), C.byref(s)))
+    return s.value
+
+
+def graph_create_permuted(ctx: Ctx, g: Graph, order: torch.Tensor) -> Graph:
+    if order.is_cuda or order.dtype != torch.int32 or order.numel() != g.n:
+        raise TypeError("order: host int32 tensor of length n")
+    h = C.c_void_p()
+    _check(lib.mixgcn_graph_create_permuted(ctx.h, g.h, _ptr(order.contiguous()), C.byref(h)))
+    return Graph(ctx, h)
 
 
 # ------------------------------------------------------------------------------ building blocks

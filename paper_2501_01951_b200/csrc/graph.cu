@@ -92,6 +92,24 @@ __global__ void symmetry_kernel(int64_t n, const int64_t* __restrict__ rowptr, c
     }
 }
 
+// Rows that store their own diagonal entry (binary search of u in row u).
+__global__ void diagonal_count_kernel(int64_t n, const int64_t* __restrict__ rowptr, const int32_t* __restrict__ col,
+                                      unsigned long long* count) {
+    const int64_t u = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    bool has = false;
+    if (u < n) {
+        int64_t lo = rowptr[u], hi = rowptr[u + 1];
+        while (lo < hi) {
+            const int64_t mid = (lo + hi) >> 1;
+            const int32_t c = col[mid];
+            if (c == (int32_t)u) { has = true; break; }
+            if (c < (int32_t)u) lo = mid + 1; else hi = mid;
+        }
+    }
+    const unsigned b = __ballot_sync(0xFFFFFFFFu, has);
+    if ((threadIdx.x & 31) == 0 && b) atomicAdd(count, (unsigned long long)__popc(b));
+}
+
 __global__ void transpose_keys_kernel(int64_t n, const int64_t* __restrict__ rowptr,
                                       const int32_t* __restrict__ col, uint64_t* __restrict__ keys) {
     int64_t u = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -361,6 +379,16 @@ mixgcn_status finish_graph(mixgcn_graph* g, cudaStream_t s) {
     MIXGCN_CUDA(cudaMemcpyAsync(&hf, flags.p, sizeof(hf), cudaMemcpyDeviceToHost, s));
     MIXGCN_CUDA(cudaStreamSynchronize(s));
     g->symmetric = (hf & F_NOT_SYMMETRIC) ? 0 : 1;
+    {
+        DevBuf dc;
+        MIXGCN_CUDA(cudaMalloc(&dc.p, sizeof(unsigned long long)));
+        MIXGCN_CUDA(cudaMemsetAsync(dc.p, 0, sizeof(unsigned long long), s));
+        diagonal_count_kernel<<<blocks_for(n), TPB, 0, s>>>(n, A.rowptr, A.col, dc.as<unsigned long long>());
+        unsigned long long hd = 0;
+        MIXGCN_CUDA(cudaMemcpyAsync(&hd, dc.p, sizeof(hd), cudaMemcpyDeviceToHost, s));
+        MIXGCN_CUDA(cudaStreamSynchronize(s));
+        g->has_diagonal = hd == (unsigned long long)n ? 1 : (hd == 0 ? 0 : 2);
+    }
     MIXGCN_TRY(build_schedule(n, A.rowptr, A.col, 0, n, A.full, s));
     if (g->symmetric) {
         g->bwd = A;  // alias: the same index serves the backward aggregation

@@ -109,6 +109,7 @@ struct mixgcn_graph {
     mixgcn_ctx* ctx;
     int64_t n, nnz;
     int symmetric;
+    int has_diagonal;  // 1: every row stores its diagonal entry, 0: none does, 2: some do
     int32_t* deg;      // [n] entries per row of the stored matrix
     float* dinv;       // [n]
     CsrView fwd, bwd;  // bwd aliases fwd when symmetric
