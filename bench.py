@@ -103,9 +103,10 @@ class ClockSampler:
 
 # ------------------------------------------------------------------------------------ workload
 
-def spmm_plan(wl, orders, sparse_levels=0):
+def spmm_plan(wl, orders, sparse_levels=0, rows_only=False):
     """Widths of the DENSE-input aggregation calls of one epoch: (width, count) per layer, from the
-    ordering; the backward aggregations of the top `sparse_levels` layers run row-sparse and are not counted."""
+    ordering; the backward aggregations of the top `sparse_levels` layers run row-sparse and are not counted,
+    nor is the last layer's forward aggregation when it is restricted to train rows (`rows_only`)."""
     from paper_2501_01951_b200 import binding as mg
     calls = []
     L = len(wl.dims) - 1
@@ -115,6 +116,8 @@ def spmm_plan(wl, orders, sparse_levels=0):
         k = 1 + (0 if (l == 0 and agg) else 1)          # forward, plus backward unless first layer agg-first
         if l >= L - sparse_levels and k == 2:
             k = 1                                        # this layer's backward aggregation takes the row-sparse path
+        if rows_only and l == L - 1:
+            k -= 1                                       # forward aggregation on train rows only
         calls.append((w, k))
     return calls
 
@@ -125,29 +128,30 @@ def spmm_alg_bytes(n, nnz, w):
     return 8 * (n + 1) + 4 * nnz + 4 * nnz + 4 * n * w + 4 * n * w
 
 
-def gemm_flops(n, dims, orders, compact_last_rows=None):
+def gemm_flops(n, dims, orders, compact_last_rows=None, compact_last_fwd=False):
     """2*M*N*K over the dense products of one epoch (forward, dW, and dX where it exists).  When the
-    last layer's backward runs on `compact_last_rows` compacted rows, its two products count those rows."""
+    last layer's backward runs on `compact_last_rows` compacted rows, its two products count those rows
+    (and so does its forward product with `compact_last_fwd`)."""
     f = 0
     L = len(dims) - 1
     for l in range(L):
         per = 2 * n * dims[l] * dims[l + 1]
         nb = 1 if l == 0 else 2
         if l == L - 1 and compact_last_rows is not None:
-            f += per + nb * 2 * compact_last_rows * dims[l] * dims[l + 1]
+            f += (2 * compact_last_rows * dims[l] * dims[l + 1] if compact_last_fwd else per) + nb * 2 * compact_last_rows * dims[l] * dims[l + 1]
         else:
             f += per * (1 + nb)
     return f
 
 
-def gemm_min_bytes(n, dims, compact_last_rows=None):
+def gemm_min_bytes(n, dims, compact_last_rows=None, compact_last_fwd=False):
     """Minimum HBM bytes of the dense products of one epoch: forward reads n x d_in, writes n x d_out;
     dW reads both; dX reads n x d_out, writes n x d_in (weights are negligible)."""
     bts = 0
     L = len(dims) - 1
     for l in range(L):
         rows_b = compact_last_rows if (l == L - 1 and compact_last_rows is not None) else n
-        bts += 4 * n * (dims[l] + dims[l + 1])
+        bts += 4 * (rows_b if compact_last_fwd else n) * (dims[l] + dims[l + 1])
         bts += 4 * rows_b * (dims[l] + dims[l + 1])
         if l > 0:
             bts += 4 * rows_b * (dims[l] + dims[l + 1])
@@ -188,7 +192,8 @@ def run_ours(args, rank, world, local_rank):
     torch.cuda.empty_cache()
     n, nnz = g.n, g.nnz
     tr = GcnTrainer(ctx, g, wl.dims, prec, n_chunks=args.chunks,
-                    row_sparse=args.row_sparse if args.row_sparse == "auto" else int(args.row_sparse))
+                    row_sparse=args.row_sparse if args.row_sparse == "auto" else int(args.row_sparse),
+                    train_rows_only=args.train_rows_only)
     X0 = synth.normal_features(n, wl.dims[0], wl.seed("features"), device=dev, ld=round4(wl.dims[0]))
     y = synth.uniform_labels(n, wl.classes, wl.seed("labels"), device=dev)
     m = synth.bernoulli_mask(n, wl.mask_p, wl.seed("mask"), device=dev)
@@ -231,8 +236,31 @@ def run_ours(args, rank, world, local_rank):
     ms_total, value = replicas_throughput(ms_total, args.steps, world, dev)
     ms_per_step = ms_total / args.steps
 
+    # Opt-in shortcut, reported beside the headline (never instead of it): the last layer's output, the
+    # loss and its gradient on train rows only -- same loss and gradients, no logits for the other nodes.
+    shortcut = None
+    if not args.train_rows_only and tr.row_sparse_levels >= 1 and n_train > 0:
+        tr.train_rows_only = True
+        tr._plan_row_sparsity()
+        for _ in range(2):
+            t += 1
+            tr.epoch(t)
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.steps):
+            t += 1
+            tr.epoch(t)
+        e1.record()
+        barrier()
+        ms_s, value_s = replicas_throughput(e0.elapsed_time(e1), args.steps, world, dev)
+        shortcut = dict(value=round(value_s, 4), unit=UNIT, ms_per_step=round(ms_s / args.steps, 3), loss=round(tr.loss.item(), 6),
+                        note="last layer forward, loss and gradient on train rows only (opt-in; not the headline)")
+        tr.train_rows_only = False
+        tr._plan_row_sparsity()
+
     # roofline of the aggregation kernels over the timed steps
-    plan = spmm_plan(wl, tr.orders, tr.row_sparse_levels)
+    plan = spmm_plan(wl, tr.orders, tr.row_sparse_levels, args.train_rows_only)
     spmm_calls = sum(k for _, k in plan) * args.steps
     alg_bytes = sum(spmm_alg_bytes(n, nnz, w) * k for w, k in plan) * args.steps
     spmm_ms = phase_ms["spmm"]
@@ -248,12 +276,15 @@ def run_ours(args, rank, world, local_rank):
         roofline.update(dram_gbs=round(dram_gbs, 1), dram_frac=round(dram_gbs / peaks["hbm_gbs"], 4))
     from paper_2501_01951_b200 import binding as _mg
     compact = n_train if (tr.row_sparse_levels >= 1 and tr.orders[-1] == _mg.ORDER_AGG_FIRST and 4 * n_train < n) else None
-    flops = gemm_flops(n, wl.dims, tr.orders, compact) * args.steps
+    rows_fwd = bool(args.train_rows_only and tr.orders[-1] == _mg.ORDER_AGG_FIRST)
+    if rows_fwd:
+        compact = n_train
+    flops = gemm_flops(n, wl.dims, tr.orders, compact, rows_fwd) * args.steps
     gemm_ms = phase_ms["gemm"]
     # The dense products run TF32 on the tensor cores: their peak is the measured bf16 peak times the
     # nominal tf32/bf16 ratio (1.1 / 2.25).  Their minimum HBM bytes: every n x d operand and result once.
     tf32_peak = peaks["bf16_tflops"] * 1.1 / 2.25
-    gbytes = gemm_min_bytes(n, wl.dims, compact) * args.steps
+    gbytes = gemm_min_bytes(n, wl.dims, compact, rows_fwd) * args.steps
     tfl = flops / (gemm_ms / 1e3) / 1e12 if gemm_ms > 0 else 0.0
     gemm = dict(tflops=round(tfl, 2), tf32_peak_tflops=round(tf32_peak, 1), frac_of_tf32_peak=round(tfl / tf32_peak, 4),
                 min_hbm_gbs=round(gbytes / (gemm_ms / 1e3) / 1e9, 1) if gemm_ms > 0 else 0.0,
@@ -266,10 +297,12 @@ def run_ours(args, rank, world, local_rank):
                dtype={mg.PREC_FP32: "f32", mg.PREC_TF32: "tf32", mg.PREC_BF16: "bf16"}[prec], data="synthetic",
                config=dict(workload=wl.name, n=n, nnz=nnz, dims=list(wl.dims), train_nodes=n_train,
                            orders=["agg-first" if o == mg.ORDER_AGG_FIRST else "upd-first" for o in tr.orders],
-                           chunks=args.chunks, row_sparse_levels=tr.row_sparse_levels, l2="inputs larger than L2" if 4 * n * wl.dims[0] > 126e6 else "inputs fit L2 (no flush)",
+                           chunks=args.chunks, row_sparse_levels=tr.row_sparse_levels, train_rows_only=bool(args.train_rows_only), l2="inputs larger than L2" if 4 * n * wl.dims[0] > 126e6 else "inputs fit L2 (no flush)",
                            parallelism=f"replicas x{world}" if world > 1 else "single GPU", setup_s=round(setup_s, 1)),
                clocks=clk, gpu_launches=int(launches_after - launches_before),
                roofline=roofline, gemm=gemm, phase_ms_per_epoch=breakdown, loss=round(loss_val, 6), device_status=status)
+    if shortcut:
+        out["train_rows_only"] = shortcut
 
     if rank == 0:
         # free the trainer and the device copy of the features before the host-buffer run allocates its arena
@@ -393,6 +426,9 @@ def main():
     ap.add_argument("--workload", default=os.environ.get("MIXGCN_WORKLOAD", "C5"), choices=list(synth.CONFIGS))
     ap.add_argument("--precision", default=None, choices=["fp32", "tf32", "bf16"])
     ap.add_argument("--chunks", type=int, default=0)
+    ap.add_argument("--train-rows-only", action="store_true",
+                    help="opt-in shortcut: the last layer's output, the loss and its gradient on train rows only "
+                         "(same loss and gradients; no predictions for the other nodes)")
     ap.add_argument("--row-sparse", default="auto", help="layers (from the top) whose backward gets a row mask: auto, 0, 1, 2, ...")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-seconds", type=float, default=20.0)

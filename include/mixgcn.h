@@ -70,6 +70,12 @@ mixgcn_status mixgcn_ctx_poll_status(mixgcn_ctx* ctx, int32_t* code);
  * that must stay in the L2 at the price of re-reading the index once per slice; results do not
  * depend on the slicing. */
 #define MIXGCN_OPT_SPMM_SLICE_COLS 1
+/* MIXGCN_OPT_LOSS_TRAIN_ROWS_ONLY: 0 (default) = mixgcn_loss_softmax_xent as documented; 1 = rows
+ * outside the train mask are not looked at: their logits are not read, their dlogits rows are
+ * left UNCHANGED (not zeroed) and pred, if given, receives -1 there.  Loss, n_correct and the
+ * train rows of dlogits are unchanged.  For use with MIXGCN_LAYER_OUT_ROWS_ONLY and a row-sparse
+ * backward pass, which read train rows only. */
+#define MIXGCN_OPT_LOSS_TRAIN_ROWS_ONLY 2
 mixgcn_status mixgcn_ctx_set_option(mixgcn_ctx* ctx, int32_t option, int64_t value);
 
 /* Per-phase profiling.  While enabled the library brackets every kernel it launches with
@@ -202,6 +208,15 @@ mixgcn_status mixgcn_gemm(mixgcn_ctx* ctx, int32_t precision, int32_t trans_a, i
                                        layer's aggregation epilogue (Eq. 4, backward form) */
 #define MIXGCN_LAYER_GOUT_GATED 8u  /* backward: G_out already carries this layer's ReLU/dropout
                                        mask (the layer above used GATE_GIN) */
+
+#define MIXGCN_LAYER_OUT_ROWS_ONLY 16u /* forward: only the rows of X_out whose gout_row_mask byte is
+                                       non-zero are wanted (the last layer of a training step: the
+                                       loss reads train rows only; the paper computes every row of
+                                       H^(L) in Algorithm 2, the gradients are the same).  The other
+                                       rows of X_out and of `saved` are left UNCHANGED.  Needs
+                                       gout_row_mask and gout_row_count (> 0, exact); no dropout
+                                       mask; n_chunks is ignored.  The backward call must then be
+                                       given the same gout_row_mask. */
 
 typedef struct {
     int32_t d_in, d_out;

@@ -26,7 +26,7 @@ OK, EINVAL, ENOMEM, ECUDA, EUNSUPPORTED, EBADGRAPH, ETIMEOUT, EDEVICE = range(8)
 GRAPH_SYMMETRISE, GRAPH_ADD_SELF_LOOPS, GRAPH_EDGES_ON_DEVICE = 1, 2, 4
 PREC_FP32, PREC_TF32, PREC_BF16 = 0, 1, 2
 ORDER_AUTO, ORDER_AGG_FIRST, ORDER_UPD_FIRST = 0, 1, 2
-LAYER_RELU, LAYER_FIRST, LAYER_GATE_GIN, LAYER_GOUT_GATED = 1, 2, 4, 8
+LAYER_RELU, LAYER_FIRST, LAYER_GATE_GIN, LAYER_GOUT_GATED, LAYER_OUT_ROWS_ONLY = 1, 2, 4, 8, 16
 N_PHASES = 7
 PHASES = ("spmm", "gemm", "elementwise", "loss", "adam", "graph", "spmm_sparse")
 PRECISIONS = {"fp32": PREC_FP32, "tf32": PREC_TF32, "bf16": PREC_BF16}
@@ -135,6 +135,7 @@ def ctx_poll_status(ctx: Ctx, raise_on_error: bool = True) -> int:
 
 
 OPT_SPMM_SLICE_COLS = 1
+OPT_LOSS_TRAIN_ROWS_ONLY = 2
 
 
 def ctx_set_option(ctx: Ctx, option: int, value: int):

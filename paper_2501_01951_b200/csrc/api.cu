@@ -192,6 +192,11 @@ extern "C" mixgcn_status mixgcn_ctx_set_option(mixgcn_ctx* ctx, int32_t option, 
         ctx->spmm_slice_cols = (int)value;
         return MIXGCN_OK;
     }
+    if (option == MIXGCN_OPT_LOSS_TRAIN_ROWS_ONLY) {
+        if (value != 0 && value != 1) MIXGCN_FAIL(MIXGCN_EINVAL, "ctx_set_option: loss rows option takes 0 or 1 (got %lld)", (long long)value);
+        ctx->loss_train_rows_only = (int)value;
+        return MIXGCN_OK;
+    }
     MIXGCN_FAIL(MIXGCN_EINVAL, "ctx_set_option: unknown option %d", option);
 }
 
@@ -296,6 +301,29 @@ extern "C" mixgcn_status mixgcn_layer_fwd(mixgcn_ctx* ctx, const mixgcn_graph* g
     const int64_t ldw = d->d_out;  // W is dense; the GEMM uses scalar loads for it when d_out % 4 != 0
     const int chunks = d->n_chunks > 1 ? d->n_chunks : 1;
 
+    if (d->flags & MIXGCN_LAYER_OUT_ROWS_ONLY) {
+        // Only the rows in gout_row_mask are wanted: aggregate those rows alone; in agg-first order the
+        // update then runs on the compacted rows and its result is scattered back.
+        const uint8_t* rows = d->gout_row_mask;
+        const int64_t cnt = d->gout_row_count;
+        if (!rows || cnt <= 0 || cnt > n) MIXGCN_FAIL(MIXGCN_EINVAL, "layer_fwd: OUT_ROWS_ONLY needs gout_row_mask and its exact count");
+        if (drop_mask) MIXGCN_FAIL(MIXGCN_EUNSUPPORTED, "layer_fwd: OUT_ROWS_ONLY does not take a dropout mask");
+        if (order == MIXGCN_ORDER_AGG_FIRST) {
+            MIXGCN_TRY(launch_spmm(ctx, g, g->fwd, 1, 0, d->d_in, X_in, d->ld_in, saved, d->ld_saved, nullptr, s, nullptr, rows));
+            RowSet rs;
+            const int64_t lda = (d->d_in + 3) / 4 * 4, ldb = (d->d_out + 3) / 4 * 4;
+            MIXGCN_TRY(build_row_set(ctx, n, rows, cnt, lda, ldb, &rs, s));
+            MIXGCN_TRY(launch_gather_rows(ctx, cnt, d->d_in, rs.idx, saved, d->ld_saved, rs.a, lda, s));
+            MIXGCN_TRY(launch_gemm(ctx, d->precision, 0, 0, cnt, d->d_out, d->d_in, rs.a, lda, W, ldw, rs.b, ldb, &epi, 0, s));
+            MIXGCN_TRY(launch_scatter_rows(ctx, cnt, d->d_out, rs.idx, rs.b, ldb, X_out, d->ld_out, s));
+            return MIXGCN_OK;
+        }
+        MIXGCN_TRY(launch_gemm(ctx, d->precision, 0, 0, n, d->d_out, d->d_in, X_in, d->ld_in, W, ldw, saved, d->ld_saved,
+                               nullptr, 0, s));
+        MIXGCN_TRY(launch_spmm(ctx, g, g->fwd, 1, 0, d->d_out, saved, d->ld_saved, X_out, d->ld_out, &epi, s, nullptr, rows));
+        return MIXGCN_OK;
+    }
+
     if (order == MIXGCN_ORDER_AGG_FIRST) {
         if (chunks == 1) {
             MIXGCN_TRY(launch_spmm(ctx, g, g->fwd, 1, 0, d->d_in, X_in, d->ld_in, saved, d->ld_saved, nullptr, s));
@@ -366,7 +394,9 @@ extern "C" mixgcn_status mixgcn_layer_bwd(mixgcn_ctx* ctx, const mixgcn_graph* g
 
     if (order == MIXGCN_ORDER_AGG_FIRST) {
         const int64_t cnt = d->gout_row_count;
-        if (rmask && cnt > 0 && cnt * 4 < n) {
+        const bool rows_only = (d->flags & MIXGCN_LAYER_OUT_ROWS_ONLY) != 0;   // other rows of G_out / saved are not data
+        if (rows_only && !(rmask && cnt > 0)) MIXGCN_FAIL(MIXGCN_EINVAL, "layer_bwd: OUT_ROWS_ONLY needs gout_row_mask and its exact count");
+        if (rmask && cnt > 0 && (cnt * 4 < n || rows_only)) {
             // Few non-zero rows: dW, db and dZ from the compacted rows, then a row-sparse aggregation.
             RowSet rs;
             const int64_t lda = (d->d_in + 3) / 4 * 4, ldb = (d->d_out + 3) / 4 * 4;
@@ -396,7 +426,20 @@ extern "C" mixgcn_status mixgcn_layer_bwd(mixgcn_ctx* ctx, const mixgcn_graph* g
     // update first: dQ = A_hat^T dZ (into `saved`) ; dW = X_in^T dQ ; G_in = dQ W^T
     // (rows of dQ that received no contribution are zero, and so are those rows of G_in: the mask the
     // aggregation reports is G_in's row mask as well)
-    if (dbias) MIXGCN_TRY(launch_colsum(ctx, n, d->d_out, G_out, d->ld_out, dbias, s));
+    if (d->flags & MIXGCN_LAYER_OUT_ROWS_ONLY) {
+        // only the masked rows of G_out are data: the bias gradient sums those rows alone
+        const int64_t cnt = d->gout_row_count;
+        if (!(rmask && cnt > 0)) MIXGCN_FAIL(MIXGCN_EINVAL, "layer_bwd: OUT_ROWS_ONLY needs gout_row_mask and its exact count");
+        if (dbias) {
+            RowSet rs;
+            const int64_t ldb = (d->d_out + 3) / 4 * 4;
+            MIXGCN_TRY(build_row_set(ctx, n, rmask, cnt, 4, ldb, &rs, s));
+            MIXGCN_TRY(launch_gather_rows(ctx, cnt, d->d_out, rs.idx, G_out, d->ld_out, rs.b, ldb, s));
+            MIXGCN_TRY(launch_colsum(ctx, cnt, d->d_out, rs.b, ldb, dbias, s));
+        }
+    } else if (dbias) {
+        MIXGCN_TRY(launch_colsum(ctx, n, d->d_out, G_out, d->ld_out, dbias, s));
+    }
     MIXGCN_TRY(launch_spmm(ctx, g, g->bwd, 1, 0, d->d_out, G_out, d->ld_out, saved, d->ld_saved, nullptr, s, spp));
     MIXGCN_TRY(launch_gemm(ctx, d->precision, 1, 0, d->d_in, d->d_out, n, X_in, d->ld_in, saved, d->ld_saved, dW, ldw,
                            nullptr, 0, s));

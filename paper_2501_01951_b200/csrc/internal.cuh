@@ -58,6 +58,7 @@ struct mixgcn_ctx {
     cudaEvent_t fork_ev, join_ev[2];
     cudaEvent_t chunk_ev[64];
     int spmm_slice_cols;      // 0 = default (one slice up to 1024 columns)
+    int loss_train_rows_only; // 1 = the loss skips rows outside the train mask entirely
     // profiling
     int profile;
     mixgcn::ProfSpan* spans;
@@ -163,7 +164,8 @@ struct SpmmRowSparse {
 // Aggregation over all rows (chunks <= 1) or over chunk k of `chunks` row chunks.
 mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView& A, int chunks, int k,
                           int32_t w, const float* Y, int64_t ldy, float* Z, int64_t ldz,
-                          const mixgcn_epilogue* epi, cudaStream_t s, const SpmmRowSparse* sparse = nullptr);
+                          const mixgcn_epilogue* epi, cudaStream_t s, const SpmmRowSparse* sparse = nullptr,
+                          const uint8_t* row_filter = nullptr);
 mixgcn_status launch_gemm(mixgcn_ctx* ctx, int precision, int ta, int tb, int64_t M, int64_t N, int64_t K,
                           const float* A, int64_t lda, const float* B, int64_t ldb, float* C, int64_t ldc,
                           const mixgcn_epilogue* epi, int64_t epi_row0, cudaStream_t s);
@@ -184,6 +186,10 @@ mixgcn_status build_row_set(mixgcn_ctx* ctx, int64_t n, const uint8_t* mask, int
                             RowSet* rs, cudaStream_t s);
 mixgcn_status launch_gather_rows(mixgcn_ctx* ctx, int64_t count, int32_t d, const int32_t* idx, const float* src,
                                  int64_t ld_src, float* dst, int64_t ld_dst, cudaStream_t s);
+
+// dst[idx[i], :] = src[i, :] for i < count (the inverse of launch_gather_rows)
+mixgcn_status launch_scatter_rows(mixgcn_ctx* ctx, int64_t count, int32_t d, const int32_t* idx, const float* src,
+                                  int64_t ld_src, float* dst, int64_t ld_dst, cudaStream_t s);
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 

@@ -205,6 +205,71 @@ __global__ void __launch_bounds__(LOSS_WARPS * 32) loss_rows_vec_kernel(
     }
 }
 
+// Train rows only: a warp scans 32 mask bytes, then handles the train rows among them one by one.
+// Rows outside the mask are neither read nor written (pred receives -1 there).
+__global__ void __launch_bounds__(LOSS_WARPS * 32) loss_rows_subset_kernel(
+    int64_t n, int C, const float* logits, int64_t ld, const int32_t* __restrict__ labels,
+    const uint8_t* __restrict__ mask, const unsigned long long* __restrict__ count, float* dlogits,
+    int32_t* __restrict__ pred, unsigned long long* n_correct, double* __restrict__ part, int32_t* status) {
+    __shared__ double sm[LOSS_WARPS];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const unsigned long long T = *count;
+    const float invT = T ? (float)(1.0 / (double)T) : 0.0f;
+    double local = 0.0;
+    unsigned int correct = 0;
+    const int64_t stride = (int64_t)gridDim.x * LOSS_WARPS * 32;
+    for (int64_t v0 = ((int64_t)blockIdx.x * LOSS_WARPS + warp) * 32; v0 < n; v0 += stride) {
+        const int64_t vl = v0 + lane;
+        const bool mine = vl < n && mask[vl] != 0 && T != 0;
+        if (pred && vl < n && !mine) pred[vl] = -1;
+        unsigned live = __ballot_sync(0xFFFFFFFFu, mine);
+        while (live) {
+            const int64_t v = v0 + __ffs(live) - 1;
+            live &= live - 1;
+            const float* row = logits + v * ld;
+            float mx = -INFINITY; int arg = 0x7FFFFFFF;
+            for (int c = lane; c < C; c += 32) {
+                const float x = row[c];
+                if (x > mx || (x == mx && c < arg)) { mx = x; arg = c; }
+            }
+            if (arg == 0x7FFFFFFF) arg = lane < C ? lane : 0;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                const float omx = __shfl_xor_sync(0xFFFFFFFFu, mx, o);
+                const int oarg = __shfl_xor_sync(0xFFFFFFFFu, arg, o);
+                if (omx > mx || (omx == mx && oarg < arg)) { mx = omx; arg = oarg; }
+            }
+            if (pred && lane == 0) pred[v] = arg;
+            const int y = labels[v];
+            if (y < 0 || y >= C) {
+                if (lane == 0) atomicMax(status, DEV_BAD_LABEL);
+                __syncwarp();
+                if (dlogits) for (int c = lane; c < C; c += 32) dlogits[v * ld + c] = 0.0f;
+                continue;
+            }
+            float s = 0.0f;
+            for (int c = lane; c < C; c += 32) s += expf(row[c] - mx);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
+            const float lse = mx + logf(s);
+            const float py = row[y];
+            if (lane == 0) { local += (double)(lse - py); if (arg == y) ++correct; }
+            __syncwarp();  // dlogits may alias logits: every read of the row precedes the writes
+            if (dlogits)
+                for (int c = lane; c < C; c += 32) dlogits[v * ld + c] = (expf(row[c] - lse) - (c == y ? 1.0f : 0.0f)) * invT;
+            __syncwarp();
+        }
+    }
+    if (lane == 0) sm[warp] = local;
+    if (n_correct && lane == 0 && correct) atomicAdd(n_correct, (unsigned long long)correct);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double t = 0.0;
+        for (int w = 0; w < LOSS_WARPS; ++w) t += sm[w];
+        part[blockIdx.x] = t;
+    }
+}
+
 // Picks the register-resident kernel when the row fits (C <= 256) and the layout allows float4 access.
 void launch_loss_rows(unsigned blocks, cudaStream_t s, int64_t n, int C, const float* logits, int64_t ld,
                       const int32_t* labels, const uint8_t* mask, const unsigned long long* count, float* dlogits,
@@ -282,8 +347,12 @@ extern "C" mixgcn_status mixgcn_loss_softmax_xent(mixgcn_ctx* ctx, int64_t n, in
     }
     {
         LaunchScope scope(ctx, PH_LOSS, s);
-        launch_loss_rows((unsigned)blocks, s, n, C, logits, ld, labels, train_mask, count, dlogits, pred,
-                         reinterpret_cast<unsigned long long*>(n_correct), part, ctx->d_status);
+        if (ctx->loss_train_rows_only)
+            loss_rows_subset_kernel<<<(unsigned)blocks, LOSS_WARPS * 32, 0, s>>>(n, C, logits, ld, labels, train_mask, count, dlogits, pred,
+                                                                              reinterpret_cast<unsigned long long*>(n_correct), part, ctx->d_status);
+        else
+            launch_loss_rows((unsigned)blocks, s, n, C, logits, ld, labels, train_mask, count, dlogits, pred,
+                             reinterpret_cast<unsigned long long*>(n_correct), part, ctx->d_status);
     }
     {
         LaunchScope scope(ctx, PH_LOSS, s);

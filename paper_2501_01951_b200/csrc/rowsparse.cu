@@ -27,6 +27,15 @@ __global__ void gather_rows_kernel(int64_t count, int d4, const int32_t* __restr
     reinterpret_cast<float4*>(dst + i * ld_dst)[c] = __ldg(reinterpret_cast<const float4*>(src + (int64_t)idx[i] * ld_src) + c);
 }
 
+// dst[idx[i], :] = src[i, :]
+__global__ void scatter_rows_kernel(int64_t count, int d4, const int32_t* __restrict__ idx, const float* __restrict__ src,
+                                    int64_t ld_src, float* __restrict__ dst, int64_t ld_dst) {
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= count * d4) return;
+    const int64_t i = t / d4; const int c = (int)(t % d4);
+    reinterpret_cast<float4*>(dst + (int64_t)idx[i] * ld_dst)[c] = __ldg(reinterpret_cast<const float4*>(src + i * ld_src) + c);
+}
+
 }  // namespace
 
 namespace mixgcn {
@@ -81,6 +90,16 @@ mixgcn_status launch_gather_rows(mixgcn_ctx* ctx, int64_t count, int32_t d, cons
     const int d4 = (d + 3) / 4;
     LaunchScope scope(ctx, PH_ELEM, s);
     gather_rows_kernel<<<(unsigned)((count * d4 + 255) / 256), 256, 0, s>>>(count, d4, idx, src, ld_src, dst, ld_dst);
+    MIXGCN_CUDA(cudaGetLastError());
+    return MIXGCN_OK;
+}
+
+mixgcn_status launch_scatter_rows(mixgcn_ctx* ctx, int64_t count, int32_t d, const int32_t* idx, const float* src,
+                                  int64_t ld_src, float* dst, int64_t ld_dst, cudaStream_t s) {
+    if (count <= 0) return MIXGCN_OK;
+    const int d4 = (d + 3) / 4;
+    LaunchScope scope(ctx, PH_ELEM, s);
+    scatter_rows_kernel<<<(unsigned)((count * d4 + 255) / 256), 256, 0, s>>>(count, d4, idx, src, ld_src, dst, ld_dst);
     MIXGCN_CUDA(cudaGetLastError());
     return MIXGCN_OK;
 }

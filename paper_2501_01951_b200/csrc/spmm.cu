@@ -49,6 +49,9 @@ struct SpmmParams {
     const uint8_t* in_mask;
     const int32_t* in_pos;
     uint8_t* out_mask;     // nullable: receives 1 for output rows that received a contribution, else 0
+    // row filter (spmm_filtered_kernel): only output rows u with row_filter[u] != 0 are computed and written
+    const uint8_t* row_filter;
+    const int32_t* seg_perm;   // segment records carry the long row's index i; its row is seg_perm[i] (null: the record's row)
     // epilogue
     const float* bias; int relu;
     const uint8_t* drop; float keep_scale;
@@ -237,6 +240,51 @@ __global__ void __launch_bounds__(256) spmm_sparse_kernel(const SpmmParams p) {
     }
 }
 
+// Row-filtered output: only the rows u with row_filter[u] != 0 are wanted (the last layer of a
+// training step needs its output on train nodes only).  A warp scans 32 schedule records, tests the
+// filter byte of each record's row and computes the kept ones one after the other with all 32 lanes,
+// entries in the same order as spmm_group_kernel (bitwise the same rows).
+template <int VPL>
+__global__ void __launch_bounds__(256) spmm_filtered_kernel(const SpmmParams p) {
+    const int lane = threadIdx.x & 31;
+    const int64_t idx0 = p.idx_begin + ((((int64_t)blockIdx.x * 256 + threadIdx.x) >> 5) << 5);
+    if (idx0 >= p.idx_end) return;
+    int4 rc = make_int4(0, 0, 0, 0);
+    bool live = false;
+    if (idx0 + lane < p.idx_end) {
+        rc = __ldg(reinterpret_cast<const int4*>(p.rec + idx0 + lane));
+        live = __ldg(p.row_filter + (p.seg_perm ? __ldg(p.seg_perm + rc.w) : rc.w)) != 0;
+    }
+    unsigned bits = __ballot_sync(0xFFFFFFFFu, live);
+    const int w4 = (p.w + 3) >> 2;
+    while (bits) {
+        const int src = __ffs(bits) - 1;
+        bits &= bits - 1;
+        const uint32_t lo = (uint32_t)__shfl_sync(0xFFFFFFFFu, rc.x, src), hi = (uint32_t)__shfl_sync(0xFFFFFFFFu, rc.y, src);
+        const int len = __shfl_sync(0xFFFFFFFFu, rc.z, src);
+        const int64_t u = __shfl_sync(0xFFFFFFFFu, rc.w, src);
+        const int64_t b = ((int64_t)hi << 32) | lo, e = b + len;
+        float4 acc[VPL];
+#pragma unroll
+        for (int v = 0; v < VPL; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+        row_segment<32, VPL>(p, b, e, lane, 0xFFFFFFFFu, w4, acc);
+        if (p.partial) {
+            float4* dst = reinterpret_cast<float4*>(p.partial + (idx0 + src) * p.ldp);
+#pragma unroll
+            for (int v = 0; v < VPL; ++v) {
+                const int c4 = lane + v * 32;
+                if (c4 < w4) dst[c4] = acc[v];
+            }
+        } else {
+#pragma unroll
+            for (int v = 0; v < VPL; ++v) {
+                const int c4 = lane + v * 32;
+                if (c4 < w4) store_row(p, u, c4, acc[v]);
+            }
+        }
+    }
+}
+
 // Long rows: add the segments' partial rows in entry order, apply the epilogue, write Z.
 // One group of 32 lanes per long row.
 __global__ void __launch_bounds__(256) spmm_combine_kernel(const SpmmParams p, int64_t n_long,
@@ -248,6 +296,7 @@ __global__ void __launch_bounds__(256) spmm_combine_kernel(const SpmmParams p, i
     if (i >= n_long) return;
     const int64_t s0 = seg_off[i], s1 = seg_off[i + 1];
     const int64_t u = perm[i];
+    if (p.row_filter && !__ldg(p.row_filter + u)) return;
     const int w4 = (p.w + 3) >> 2;
     if (p.out_mask && lane == 0) p.out_mask[u] = 1;    // long rows are kept without looking (conservative)
     for (int c4 = lane; c4 < w4; c4 += 32) {
@@ -316,6 +365,20 @@ void dispatch_sparse(const SpmmParams& p, int fold, cudaStream_t s) {
 #undef MIXGCN_SPMM_CASE
 }
 
+void dispatch_filtered(const SpmmParams& p, cudaStream_t s) {
+    const int64_t units = p.idx_end - p.idx_begin;
+    if (units <= 0) return;
+    const unsigned blocks = (unsigned)((units + 255) / 256);   // 8 warps x 32 records
+    const int vpl = (((p.w + 3) >> 2) + 31) / 32;
+    switch (vpl) {
+#define MIXGCN_SPMM_CASE(V) case V: spmm_filtered_kernel<V><<<blocks, 256, 0, s>>>(p); break;
+        MIXGCN_SPMM_CASE(1) MIXGCN_SPMM_CASE(2) MIXGCN_SPMM_CASE(3) MIXGCN_SPMM_CASE(4)
+        MIXGCN_SPMM_CASE(5) MIXGCN_SPMM_CASE(6) MIXGCN_SPMM_CASE(7) MIXGCN_SPMM_CASE(8)
+#undef MIXGCN_SPMM_CASE
+        default: break;
+    }
+}
+
 constexpr int MAX_SLICE = 1024;  // columns per launch: 8 float4 per lane
 
 }  // namespace
@@ -326,8 +389,10 @@ namespace mixgcn {
 // with its own schedule: long rows as column-ordered segments, then rows longest first, short rows packed.
 mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView& A, int chunks, int k,
                           int32_t w, const float* Y, int64_t ldy, float* Z, int64_t ldz,
-                          const mixgcn_epilogue* epi, cudaStream_t s, const SpmmRowSparse* sparse) {
+                          const mixgcn_epilogue* epi, cudaStream_t s, const SpmmRowSparse* sparse,
+                          const uint8_t* row_filter) {
     if (w <= 0) return MIXGCN_OK;
+    if (sparse && row_filter) MIXGCN_FAIL(MIXGCN_EUNSUPPORTED, "spmm: a row filter cannot be combined with a row-sparse input");
     if (chunks > 1) {
         MIXGCN_TRY(ensure_chunk_schedules(g, A, chunks));
         if (k < 0 || k >= A.n_chunk) MIXGCN_FAIL(MIXGCN_EINVAL, "spmm: chunk %d of %d does not exist", k, chunks);
@@ -343,6 +408,7 @@ mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView&
     }
     p.rec = S.rec;
     if (sparse) { p.in_mask = sparse->in_mask; p.in_pos = sparse->in_pos; p.out_mask = sparse->out_mask; }
+    p.row_filter = row_filter;
     const int slice = ctx->spmm_slice_cols > 0 ? ctx->spmm_slice_cols : MAX_SLICE;
     for (int j0 = 0; j0 < w; j0 += slice) {
         p.j0 = j0;
@@ -382,6 +448,33 @@ mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView&
                     dispatch_sparse(p, fold, s);
                     begin = end;
                 }
+            }
+            continue;
+        }
+        if (row_filter) {
+            // kept rows only: segments of kept long rows, their combination, then every other kept row
+            if (S.total_segs > 0) {
+                const int64_t ldp = ((int64_t)p.w + 3) / 4 * 4;
+                MIXGCN_TRY(ensure_workspace_spmm(ctx, S.total_segs * ldp * (int64_t)sizeof(float)));
+                p.partial = reinterpret_cast<float*>(ctx->workspace_spmm); p.ldp = ldp;
+                {
+                    LaunchScope scope(ctx, PH_SPMM_SPARSE, s);
+                    p.idx_begin = 0; p.idx_end = S.total_segs;
+                    p.seg_perm = S.perm;
+                    dispatch_filtered(p, s);
+                    p.seg_perm = nullptr;
+                }
+                {
+                    LaunchScope scope(ctx, PH_SPMM_SPARSE, s);
+                    const int64_t blocks = (S.n_long * 32 + 255) / 256;
+                    spmm_combine_kernel<<<(unsigned)blocks, 256, 0, s>>>(p, S.n_long, S.seg_off, S.seg_pos, S.perm);
+                }
+                p.partial = nullptr;
+            }
+            if (S.n_rows > S.n_long) {
+                LaunchScope scope(ctx, PH_SPMM_SPARSE, s);
+                p.idx_begin = S.total_segs; p.idx_end = S.total_segs + (S.n_rows - S.n_long);
+                dispatch_filtered(p, s);
             }
             continue;
         }

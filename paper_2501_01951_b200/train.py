@@ -18,7 +18,8 @@ def round4(x: int) -> int:
 
 class GcnTrainer:
     def __init__(self, ctx: mg.Ctx, graph: mg.Graph, dims, precision=mg.PREC_FP32, order=mg.ORDER_AUTO,
-                 n_chunks=0, fuse_gate=True, keep_scale=1.0, device=None, row_sparse="auto"):
+                 n_chunks=0, fuse_gate=True, keep_scale=1.0, device=None, row_sparse="auto",
+                 train_rows_only=False):
         self.ctx, self.g = ctx, graph
         self.dims = tuple(int(d) for d in dims)
         self.L = len(self.dims) - 1
@@ -28,6 +29,9 @@ class GcnTrainer:
         self.fuse_gate = fuse_gate
         self.row_sparse = row_sparse          # "auto" | number of layers (from the top) whose backward gets a row mask
         self.row_masks = None
+        # opt-in: the last layer's output, the loss and its gradient on train rows only (needs a
+        # row-sparse backward for the last layer; predictions exist for train rows only)
+        self.train_rows_only = bool(train_rows_only)
         n, L = self.n, self.L
         orders = order if isinstance(order, (list, tuple)) else [order] * L
         self.descs, self.orders = [], []
@@ -101,11 +105,19 @@ class GcnTrainer:
         if levels == "auto":
             mean_entries = self.g.nnz / max(n, 1)
             levels = 0 if frac >= 0.25 else (2 if frac * mean_entries < 0.5 else 1)
+        if self.train_rows_only and self.row_sparse == "auto" and levels == 0:
+            levels = 1
         levels = max(0, min(int(levels), L))
         self.row_sparse_levels = levels
         self.row_masks = [None] * (L + 1)
         for d in self.descs:
             d.gout_row_mask, d.gout_row_count, d.gin_row_mask = None, 0, None
+            d.flags &= ~mg.LAYER_OUT_ROWS_ONLY
+        if self.train_rows_only:
+            if levels == 0 or n_train == 0 or self.masks[L - 1] is not None:
+                raise ValueError("train_rows_only needs a row-sparse backward (row_sparse >= 1), a non-empty "
+                                 "train mask and no dropout mask on the last layer")
+            self.descs[L - 1].flags |= mg.LAYER_OUT_ROWS_ONLY
         if levels == 0:
             return
         self.row_masks[L] = self.train_mask
@@ -125,6 +137,14 @@ class GcnTrainer:
                          self.saved[l], self.X[l + 1])
 
     def compute_loss(self):
+        if self.train_rows_only:
+            mg.ctx_set_option(self.ctx, mg.OPT_LOSS_TRAIN_ROWS_ONLY, 1)
+            try:
+                mg.loss_softmax_xent(self.ctx, self.X[self.L], self.labels, self.train_mask, self.loss,
+                                     dlogits=self.X[self.L], pred=self.pred, n_correct=self.n_correct, C_=self.dims[-1])
+            finally:
+                mg.ctx_set_option(self.ctx, mg.OPT_LOSS_TRAIN_ROWS_ONLY, 0)
+            return
         mg.loss_softmax_xent(self.ctx, self.X[self.L], self.labels, self.train_mask, self.loss,
                              dlogits=self.X[self.L], pred=self.pred, n_correct=self.n_correct, C_=self.dims[-1])
 

@@ -205,5 +205,22 @@ def test_full_size_workload(mg, key):
     assert abs(float(tr.db[l].double() @ bv) - want_db) <= tol * scale + 1e-12
     for t in tr.dW + tr.db:
         assert bool(torch.isfinite(t).all())
+
+    # ---- the train-rows-only shortcut at full size: same loss and gradients as the full computation
+    # above; rows outside the train mask hold NaN beforehand, so reading one of them would show
+    ref_loss, ref_dW, ref_db = tr.loss.item(), [t.clone() for t in tr.dW], [t.clone() for t in tr.db]
+    tr.train_rows_only = True
+    tr._plan_row_sparsity()
+    assert tr.row_sparse_levels >= 1
+    tr.X[L].fill_(float("nan"))
+    if agg_first:
+        tr.saved[l].fill_(float("nan"))
+    tr.forward(); tr.compute_loss(); tr.backward()
+    torch.cuda.synchronize()
+    assert mg.ctx_poll_status(ctx, raise_on_error=False) == 0
+    assert abs(tr.loss.item() - ref_loss) <= 1e-5 * abs(ref_loss)
+    for k in range(L):
+        assert _rel(tr.dW[k].double().cpu().numpy(), ref_dW[k].double().cpu().numpy()) <= 4 * tol, f"dW[{k}] with the shortcut"
+        assert _rel(tr.db[k].double().cpu().numpy(), ref_db[k].double().cpu().numpy()) <= 4 * tol, f"db[{k}] with the shortcut"
     g.close()
     ctx.close()
