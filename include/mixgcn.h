@@ -317,6 +317,8 @@ mixgcn_status mixgcn_adam_step(mixgcn_ctx* ctx, int32_t n_tensors, float* const*
  * dims is int32[L+1] (d_0 .. d_L); W, b, mW, vW, mb, vb are host arrays of L host pointers
  * (dense fp32, updated in place); X is n x d_0 dense fp32; loss host fp32 scalar; pred
  * (nullable) host int32[n].  Uses AUTO ordering, ReLU on all layers but the last, no dropout.
+ * When pred is NULL and the backward pass runs row-sparse, the last layer, the loss and its
+ * gradient are computed on the train rows alone (nothing returned depends on the other rows).
  * Device buffers are taken from the context workspace (grown on demand).  Synchronises. */
 mixgcn_status mixgcn_train_step_host(mixgcn_ctx* ctx, const mixgcn_graph* g, int32_t L,
                                      const int32_t* dims, int32_t precision, const float* X,

@@ -106,6 +106,7 @@ extern "C" mixgcn_status mixgcn_train_step_host(mixgcn_ctx* ctx, const mixgcn_gr
     // aggregation later on their neighbours only (same rule as the device-buffer trainer).
     int64_t n_train = 0;
     for (int64_t i = 0; i < n; ++i) n_train += train_mask[i] ? 1 : 0;
+    bool rows_only = false;
     {
         const double frac = (double)n_train / (double)n, mean_entries = (double)g->nnz / (double)n;
         int levels = frac >= 0.25 ? 0 : (frac * mean_entries < 0.5 ? 2 : 1);
@@ -117,6 +118,10 @@ extern "C" mixgcn_status mixgcn_train_step_host(mixgcn_ctx* ctx, const mixgcn_gr
             lo.desc[l].gout_row_count = i == 0 ? n_train : 0;
             if (l > 0 && i + 1 < levels) { lo.desc[l].gin_row_mask = lo.rowmask[l]; in_mask = lo.rowmask[l]; }
         }
+        // Without `pred` nothing this call returns depends on the last layer's output outside the train
+        // rows: compute that layer, the loss and its gradient on the train rows alone.
+        rows_only = !pred && levels >= 1 && n_train > 0;
+        if (rows_only) lo.desc[L - 1].flags |= MIXGCN_LAYER_OUT_ROWS_ONLY;
     }
     cudaStream_t s = ctx->side_stream[0];
     const cudaMemcpyKind H2D = cudaMemcpyHostToDevice, D2H = cudaMemcpyDeviceToHost;
@@ -139,8 +144,14 @@ extern "C" mixgcn_status mixgcn_train_step_host(mixgcn_ctx* ctx, const mixgcn_gr
     // forward, loss, backward, update
     for (int l = 0; l < L; ++l)
         MIXGCN_TRY(mixgcn_layer_fwd(ctx, g, &lo.desc[l], lo.X[l], lo.W[l], lo.b[l], nullptr, lo.saved[l], lo.X[l + 1], s));
-    MIXGCN_TRY(mixgcn_loss_softmax_xent(ctx, n, dims[L], lo.X[L], round4(dims[L]), lo.labels, lo.mask, lo.loss, lo.X[L],
-                                        lo.pred, nullptr, s));
+    {
+        const int keep = ctx->loss_train_rows_only;
+        ctx->loss_train_rows_only = rows_only ? 1 : keep;
+        const mixgcn_status st = mixgcn_loss_softmax_xent(ctx, n, dims[L], lo.X[L], round4(dims[L]), lo.labels, lo.mask, lo.loss,
+                                                          lo.X[L], pred ? lo.pred : nullptr, nullptr, s);
+        ctx->loss_train_rows_only = keep;
+        MIXGCN_TRY(st);
+    }
     for (int l = L - 1; l >= 0; --l)
         MIXGCN_TRY(mixgcn_layer_bwd(ctx, g, &lo.desc[l], lo.X[l], lo.saved[l], lo.X[l + 1], nullptr, lo.W[l], lo.G[l + 1],
                                     l > 0 ? lo.G[l] : nullptr, lo.dW[l], lo.db[l], s));

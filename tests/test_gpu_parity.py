@@ -735,8 +735,10 @@ def test_layer_tf32_with_dropout_both_orders(mg, ctx, order):
     assert mg.ctx_poll_status(ctx, raise_on_error=False) == 0
 
 
-def test_train_step_host_row_sparse_matches_oracle(mg, ctx):
-    """Few train nodes: the host-buffer step takes the row-sparse backward."""
+@pytest.mark.parametrize("with_pred", [False, True])
+def test_train_step_host_row_sparse_matches_oracle(mg, ctx, with_pred):
+    """Few train nodes: the host-buffer step takes the row-sparse backward; without `pred` it also
+    restricts the last layer and the loss to the train rows."""
     wl, s, d, X, y, m, Ws, bs = _tiny_problem()
     m = synth.bernoulli_mask(wl.n, 0.02, 88)
     gg = mg.graph_create(ctx, wl.n, s, d)
@@ -744,7 +746,11 @@ def test_train_step_host_row_sparse_matches_oracle(mg, ctx):
     W = [w.clone() for w in Ws]; b = [x.clone() for x in bs]
     z = lambda lst: [torch.zeros_like(x) for x in lst]
     mW, vW, mb, vb = z(W), z(W), z(b), z(b)
-    loss = mg.train_step_host(ctx, gg, wl.dims, mg.PREC_FP32, X, y, m, W, b, mW, vW, mb, vb, 1, **ADAM)
+    pred = torch.full((wl.n,), -7, dtype=torch.int32) if with_pred else None
+    loss = mg.train_step_host(ctx, gg, wl.dims, mg.PREC_FP32, X, y, m, W, b, mW, vW, mb, vb, 1, **ADAM, pred=pred)
+    if with_pred:
+        p = pred.numpy()
+        assert p.min() >= 0 and p.max() < wl.classes                 # every node has a prediction
     ref = orc.train_epoch(go, X.numpy(), [w.numpy() for w in Ws], [x.numpy() for x in bs], y.numpy(), m.numpy(), None, 1, **ADAM)
     assert abs(loss - ref["loss"]) <= 1e-5 * abs(ref["loss"])
     for l in range(len(W)):
