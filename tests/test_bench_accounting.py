@@ -1,0 +1,65 @@
+"""The byte and FLOP accounting behind bench.py's roofline figures, checked by hand on small cases
+(host logic only; no GPU)."""
+import importlib.util
+import os
+import types
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def bench():
+    from paper_2501_01951_b200 import build
+    build.build()
+    spec = importlib.util.spec_from_file_location("bench_module", os.path.join(ROOT, "bench.py"))
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    return mod
+
+
+def _wl(dims):
+    return types.SimpleNamespace(dims=tuple(dims))
+
+
+def test_spmm_plan_counts_dense_input_calls(bench):
+    from paper_2501_01951_b200 import binding as mg
+    A, U = mg.ORDER_AGG_FIRST, mg.ORDER_UPD_FIRST
+    wl = _wl((128, 128, 128, 172))
+    # agg-first everywhere: forward aggregates at d_in; the first layer's backward needs no aggregation
+    assert bench.spmm_plan(wl, [A, A, A], 0) == [(128, 1), (128, 2), (128, 2)]
+    # the top two layers' backward aggregations take the row-sparse path
+    assert bench.spmm_plan(wl, [A, A, A], 2) == [(128, 1), (128, 1), (128, 1)]
+    # and the last layer's forward aggregation runs on train rows only
+    assert bench.spmm_plan(wl, [A, A, A], 2, True) == [(128, 1), (128, 1), (128, 0)]
+    # update-first aggregates at d_out, forward and backward, first layer included
+    assert bench.spmm_plan(_wl((602, 256, 41)), [U, U], 0) == [(256, 2), (41, 2)]
+
+
+def test_spmm_algorithmic_bytes(bench):
+    # 3 rows, 5 stored entries, width 4: row pointers 4 x 8, column ids and values 5 x 4 each,
+    # one read of the 3 x 4 input and one write of the 3 x 4 output
+    assert bench.spmm_alg_bytes(3, 5, 4) == 32 + 20 + 20 + 48 + 48
+
+
+def test_gemm_flops_and_bytes(bench):
+    from paper_2501_01951_b200 import binding as mg
+    A = mg.ORDER_AGG_FIRST
+    n, dims = 10, (4, 3, 2)
+    # layer 0: forward + dW; layer 1: forward + dW + dX; each product 2 * n * d_in * d_out
+    assert bench.gemm_flops(n, dims, [A, A]) == 2 * 10 * 4 * 3 * 2 + 2 * 10 * 3 * 2 * 3
+    # last layer's backward on 5 compacted rows
+    assert bench.gemm_flops(n, dims, [A, A], 5) == 2 * 10 * 4 * 3 * 2 + 2 * 10 * 3 * 2 + 2 * (2 * 5 * 3 * 2)
+    # ... and its forward too
+    assert bench.gemm_flops(n, dims, [A, A], 5, True) == 2 * 10 * 4 * 3 * 2 + 3 * (2 * 5 * 3 * 2)
+    # bytes: every n x d operand and result once per product
+    full = 4 * 10 * (4 + 3) * 2 + 4 * 10 * (3 + 2) * 3
+    assert bench.gemm_min_bytes(n, dims) == full
+    assert bench.gemm_min_bytes(n, dims, 5) == 4 * 10 * (4 + 3) * 2 + 4 * 10 * (3 + 2) + 2 * 4 * 5 * (3 + 2)
+    assert bench.gemm_min_bytes(n, dims, 5, True) == 4 * 10 * (4 + 3) * 2 + 3 * 4 * 5 * (3 + 2)
+
+
+def test_peaks_are_read_from_the_measured_file_or_fall_back(bench):
+    p = bench.load_peaks()
+    assert p["source"] in ("measured", "fallback") and p["hbm_gbs"] > 1000 and p["bf16_tflops"] > 100
