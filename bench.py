@@ -128,33 +128,30 @@ def spmm_alg_bytes(n, nnz, w):
     return 8 * (n + 1) + 4 * nnz + 4 * nnz + 4 * n * w + 4 * n * w
 
 
-def gemm_flops(n, dims, orders, compact_last_rows=None, compact_last_fwd=False):
-    """2*M*N*K over the dense products of one epoch (forward, dW, and dX where it exists).  When the
-    last layer's backward runs on `compact_last_rows` compacted rows, its two products count those rows
-    (and so does its forward product with `compact_last_fwd`)."""
+def gemm_flops(n, dims, orders, bwd_rows=None, fwd_rows_last=None):
+    """2*M*N*K over the dense products of one epoch (forward, dW, and dX where it exists).
+    bwd_rows[l] (default n) is the number of rows layer l's backward products run on (the compacted
+    rows of a row-sparse backward); fwd_rows_last likewise for the last layer's forward product."""
     f = 0
     L = len(dims) - 1
     for l in range(L):
-        per = 2 * n * dims[l] * dims[l + 1]
+        rb = n if bwd_rows is None or bwd_rows[l] is None else bwd_rows[l]
+        rf = fwd_rows_last if (l == L - 1 and fwd_rows_last is not None) else n
         nb = 1 if l == 0 else 2
-        if l == L - 1 and compact_last_rows is not None:
-            f += (2 * compact_last_rows * dims[l] * dims[l + 1] if compact_last_fwd else per) + nb * 2 * compact_last_rows * dims[l] * dims[l + 1]
-        else:
-            f += per * (1 + nb)
+        f += 2 * dims[l] * dims[l + 1] * (rf + nb * rb)
     return f
 
 
-def gemm_min_bytes(n, dims, compact_last_rows=None, compact_last_fwd=False):
-    """Minimum HBM bytes of the dense products of one epoch: forward reads n x d_in, writes n x d_out;
-    dW reads both; dX reads n x d_out, writes n x d_in (weights are negligible)."""
+def gemm_min_bytes(n, dims, bwd_rows=None, fwd_rows_last=None):
+    """Minimum HBM bytes of the dense products of one epoch: forward reads rows x d_in, writes rows x d_out;
+    dW reads both; dX reads rows x d_out, writes rows x d_in (weights are negligible)."""
     bts = 0
     L = len(dims) - 1
     for l in range(L):
-        rows_b = compact_last_rows if (l == L - 1 and compact_last_rows is not None) else n
-        bts += 4 * (rows_b if compact_last_fwd else n) * (dims[l] + dims[l + 1])
-        bts += 4 * rows_b * (dims[l] + dims[l + 1])
-        if l > 0:
-            bts += 4 * rows_b * (dims[l] + dims[l + 1])
+        rb = n if bwd_rows is None or bwd_rows[l] is None else bwd_rows[l]
+        rf = fwd_rows_last if (l == L - 1 and fwd_rows_last is not None) else n
+        nb = 1 if l == 0 else 2
+        bts += 4 * (dims[l] + dims[l + 1]) * (rf + nb * rb)
     return bts
 
 
@@ -236,6 +233,14 @@ def run_ours(args, rank, world, local_rank):
     ms_total, value = replicas_throughput(ms_total, args.steps, world, dev)
     ms_per_step = ms_total / args.steps
 
+    # rows the dense products of each layer's backward ran on (compacted rows where layer_bwd took that path)
+    bwd_rows = []
+    for l, d in enumerate(tr.descs):
+        cnt = int(d.gout_row_count)
+        rows_flag = bool(d.flags & mg.LAYER_OUT_ROWS_ONLY)
+        compacted = bool(d.gout_row_mask) and cnt > 0 and tr.orders[l] == mg.ORDER_AGG_FIRST and (4 * cnt < n or rows_flag)
+        bwd_rows.append(cnt if compacted else None)
+
     # Opt-in shortcut, reported beside the headline (never instead of it): the last layer's output, the
     # loss and its gradient on train rows only -- same loss and gradients, no logits for the other nodes.
     shortcut = None
@@ -274,17 +279,13 @@ def run_ours(args, rank, world, local_rank):
         # real DRAM throughput of the call: captured bytes over the call's measured duration
         dram_gbs = roofline["traffic"] / (spmm_ms / max(spmm_calls, 1) / 1e3) / 1e9
         roofline.update(dram_gbs=round(dram_gbs, 1), dram_frac=round(dram_gbs / peaks["hbm_gbs"], 4))
-    from paper_2501_01951_b200 import binding as _mg
-    compact = n_train if (tr.row_sparse_levels >= 1 and tr.orders[-1] == _mg.ORDER_AGG_FIRST and 4 * n_train < n) else None
-    rows_fwd = bool(args.train_rows_only and tr.orders[-1] == _mg.ORDER_AGG_FIRST)
-    if rows_fwd:
-        compact = n_train
-    flops = gemm_flops(n, wl.dims, tr.orders, compact, rows_fwd) * args.steps
+    fwd_rows_last = n_train if (args.train_rows_only and tr.orders[-1] == mg.ORDER_AGG_FIRST) else None
+    flops = gemm_flops(n, wl.dims, tr.orders, bwd_rows, fwd_rows_last) * args.steps
     gemm_ms = phase_ms["gemm"]
     # The dense products run TF32 on the tensor cores: their peak is the measured bf16 peak times the
     # nominal tf32/bf16 ratio (1.1 / 2.25).  Their minimum HBM bytes: every n x d operand and result once.
     tf32_peak = peaks["bf16_tflops"] * 1.1 / 2.25
-    gbytes = gemm_min_bytes(n, wl.dims, compact, rows_fwd) * args.steps
+    gbytes = gemm_min_bytes(n, wl.dims, bwd_rows, fwd_rows_last) * args.steps
     tfl = flops / (gemm_ms / 1e3) / 1e12 if gemm_ms > 0 else 0.0
     gemm = dict(tflops=round(tfl, 2), tf32_peak_tflops=round(tf32_peak, 1), frac_of_tf32_peak=round(tfl / tf32_peak, 4),
                 min_hbm_gbs=round(gbytes / (gemm_ms / 1e3) / 1e9, 1) if gemm_ms > 0 else 0.0,
@@ -297,7 +298,7 @@ def run_ours(args, rank, world, local_rank):
                dtype={mg.PREC_FP32: "f32", mg.PREC_TF32: "tf32", mg.PREC_BF16: "bf16"}[prec], data="synthetic",
                config=dict(workload=wl.name, n=n, nnz=nnz, dims=list(wl.dims), train_nodes=n_train,
                            orders=["agg-first" if o == mg.ORDER_AGG_FIRST else "upd-first" for o in tr.orders],
-                           chunks=args.chunks, row_sparse_levels=tr.row_sparse_levels, train_rows_only=bool(args.train_rows_only), l2="inputs larger than L2" if 4 * n * wl.dims[0] > 126e6 else "inputs fit L2 (no flush)",
+                           chunks=args.chunks, row_sparse_levels=tr.row_sparse_levels, backward_rows=[r if r is not None else n for r in bwd_rows], train_rows_only=bool(args.train_rows_only), l2="inputs larger than L2" if 4 * n * wl.dims[0] > 126e6 else "inputs fit L2 (no flush)",
                            parallelism=f"replicas x{world}" if world > 1 else "single GPU", setup_s=round(setup_s, 1)),
                clocks=clk, gpu_launches=int(launches_after - launches_before),
                roofline=roofline, gemm=gemm, phase_ms_per_epoch=breakdown, loss=round(loss_val, 6), device_status=status)

@@ -267,6 +267,12 @@ mixgcn_status mixgcn_layer_bwd(mixgcn_ctx* ctx, const mixgcn_graph* g, const mix
                                const uint8_t* drop_mask, const float* W, float* G_out,
                                float* G_in, float* dW, float* dbias, void* stream);
 
+/* Number of non-zero bytes of a device row mask (uint8[n]); *count is a HOST int64.  For callers
+ * that want to hand layer_bwd the exact gout_row_count of a mask the library produced
+ * (gin_row_mask).  Synchronises `stream`.  Not in the paper: bookkeeping of the row-sparse backward. */
+mixgcn_status mixgcn_count_rows(mixgcn_ctx* ctx, int64_t n, const uint8_t* row_mask, int64_t* count,
+                                void* stream);
+
 /* Masked softmax cross-entropy (the loss line of Algorithm 2; mean over train nodes, natural
  * log): loss = -(1/#T) sum_{v in T} log softmax(logits_v)[label_v]; dlogits_v =
  * (softmax(logits_v) - e_label) / #T on T and 0 elsewhere; pred_v = lowest index of the row

@@ -40,6 +40,7 @@ SYMBOLS = (
     "mixgcn_layer_plan", "mixgcn_layer_fwd", "mixgcn_layer_bwd", "mixgcn_loss_softmax_xent",
     "mixgcn_adam_step", "mixgcn_train_step_host", "mixgcn_loss_softmax_xent_noalloc", "mixgcn_ctx_set_option",
     "mixgcn_graph_bandwidth", "mixgcn_graph_rcm", "mixgcn_pipeline_stages", "mixgcn_graph_create_permuted",
+    "mixgcn_count_rows",
 )
 
 
@@ -357,6 +358,14 @@ def adam_step(ctx: Ctx, params, grads, ms, vs, t, lr=0.01, beta1=0.9, beta2=0.99
     numel = (C.c_int64 * k)(*[x.numel() for x in params])
     _check(lib.mixgcn_adam_step(ctx.h, C.c_int32(k), arr(params), arr(grads), arr(ms), arr(vs), numel, C.c_int64(t),
                                 C.c_float(lr), C.c_float(beta1), C.c_float(beta2), C.c_float(eps), _stream()))
+
+
+def count_rows(ctx: Ctx, row_mask) -> int:
+    """Non-zero bytes of a device uint8 row mask (synchronises the current stream)."""
+    _dev(row_mask, torch.uint8, "row_mask")
+    out = C.c_int64(0)
+    _check(lib.mixgcn_count_rows(ctx.h, C.c_int64(row_mask.numel()), _ptr(row_mask), C.byref(out), _stream()))
+    return out.value
 
 
 def train_step_host(ctx: Ctx, g: Graph, dims, precision, X, labels, train_mask, W, b, mW, vW, mb, vb, t,

@@ -152,9 +152,16 @@ extern "C" mixgcn_status mixgcn_train_step_host(mixgcn_ctx* ctx, const mixgcn_gr
         ctx->loss_train_rows_only = keep;
         MIXGCN_TRY(st);
     }
-    for (int l = L - 1; l >= 0; --l)
+    for (int l = L - 1; l >= 0; --l) {
+        if (lo.desc[l].gout_row_mask && lo.desc[l].gout_row_count == 0 && l < L - 1) {
+            // the mask the layer above reported: with its count the dense products run on compacted rows
+            int64_t cnt = 0;
+            MIXGCN_TRY(mixgcn_count_rows(ctx, n, lo.desc[l].gout_row_mask, &cnt, s));
+            lo.desc[l].gout_row_count = cnt;
+        }
         MIXGCN_TRY(mixgcn_layer_bwd(ctx, g, &lo.desc[l], lo.X[l], lo.saved[l], lo.X[l + 1], nullptr, lo.W[l], lo.G[l + 1],
                                     l > 0 ? lo.G[l] : nullptr, lo.dW[l], lo.db[l], s));
+    }
     std::vector<float*> P, M1, M2; std::vector<const float*> Gr; std::vector<int64_t> numel;
     for (int l = 0; l < L; ++l) { P.push_back(lo.W[l]); Gr.push_back(lo.dW[l]); M1.push_back(lo.mW[l]); M2.push_back(lo.vW[l]); numel.push_back((int64_t)dims[l] * dims[l + 1]); }
     for (int l = 0; l < L; ++l) { P.push_back(lo.b[l]); Gr.push_back(lo.db[l]); M1.push_back(lo.mb[l]); M2.push_back(lo.vb[l]); numel.push_back(dims[l + 1]); }

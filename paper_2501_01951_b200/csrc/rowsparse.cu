@@ -27,6 +27,15 @@ __global__ void gather_rows_kernel(int64_t count, int d4, const int32_t* __restr
     reinterpret_cast<float4*>(dst + i * ld_dst)[c] = __ldg(reinterpret_cast<const float4*>(src + (int64_t)idx[i] * ld_src) + c);
 }
 
+// number of non-zero bytes (integer sum: order-free)
+__global__ void count_rows_kernel(int64_t n, const uint8_t* __restrict__ mask, unsigned long long* count) {
+    unsigned int c = 0;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
+        c += mask[i] ? 1u : 0u;
+    for (int o = 16; o > 0; o >>= 1) c += __shfl_down_sync(0xFFFFFFFFu, c, o);
+    if ((threadIdx.x & 31) == 0 && c) atomicAdd(count, (unsigned long long)c);
+}
+
 // dst[idx[i], :] = src[i, :]
 __global__ void scatter_rows_kernel(int64_t count, int d4, const int32_t* __restrict__ idx, const float* __restrict__ src,
                                     int64_t ld_src, float* __restrict__ dst, int64_t ld_dst) {
@@ -105,3 +114,25 @@ mixgcn_status launch_scatter_rows(mixgcn_ctx* ctx, int64_t count, int32_t d, con
 }
 
 }  // namespace mixgcn
+
+extern "C" mixgcn_status mixgcn_count_rows(mixgcn_ctx* ctx, int64_t n, const uint8_t* row_mask, int64_t* count,
+                                           void* stream) {
+    if (!ctx || !row_mask || !count || n < 0) MIXGCN_FAIL(MIXGCN_EINVAL, "count_rows: bad argument");
+    MIXGCN_CUDA(cudaSetDevice(ctx->device));
+    cudaStream_t s = (cudaStream_t)stream;
+    MIXGCN_TRY(ensure_workspace_rows(ctx, 256));
+    unsigned long long* d = reinterpret_cast<unsigned long long*>(ctx->workspace_rows);
+    MIXGCN_CUDA(cudaMemsetAsync(d, 0, sizeof(unsigned long long), s));
+    if (n > 0) {
+        LaunchScope scope(ctx, PH_ELEM, s);
+        int64_t blocks = (n + 255) / 256;
+        const int64_t cap = (int64_t)ctx->sm_count * 16;
+        if (blocks > cap) blocks = cap;
+        count_rows_kernel<<<(unsigned)blocks, 256, 0, s>>>(n, row_mask, d);
+    }
+    unsigned long long h = 0;
+    MIXGCN_CUDA(cudaMemcpyAsync(&h, d, sizeof(h), cudaMemcpyDeviceToHost, s));
+    MIXGCN_CUDA(cudaStreamSynchronize(s));
+    *count = (int64_t)h;
+    return MIXGCN_OK;
+}

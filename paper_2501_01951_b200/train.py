@@ -150,7 +150,13 @@ class GcnTrainer:
 
     def backward(self):
         for l in range(self.L - 1, -1, -1):
-            mg.layer_bwd(self.ctx, self.g, self.descs[l], self.X[l], self.saved[l], self.X[l + 1], self.masks[l],
+            d = self.descs[l]
+            if d.gout_row_mask and d.gout_row_count == 0 and self.row_masks[l + 1] is not self.train_mask:
+                # A row mask the library reported one layer up.  It depends on the graph and the train
+                # mask only, so its count is taken once (a stream synchronisation) and kept; with the
+                # count layer_bwd can run its dense products on the compacted rows.
+                d.gout_row_count = mg.count_rows(self.ctx, self.row_masks[l + 1])
+            mg.layer_bwd(self.ctx, self.g, d, self.X[l], self.saved[l], self.X[l + 1], self.masks[l],
                          self.W[l], self.G[l + 1], self.G[l] if l > 0 else None, self.dW[l], self.db[l])
 
     def step(self, t, lr=0.01, beta1=0.9, beta2=0.999, eps=1e-8):

@@ -47,17 +47,18 @@ def test_gemm_flops_and_bytes(bench):
     from paper_2501_01951_b200 import binding as mg
     A = mg.ORDER_AGG_FIRST
     n, dims = 10, (4, 3, 2)
-    # layer 0: forward + dW; layer 1: forward + dW + dX; each product 2 * n * d_in * d_out
+    # layer 0: forward + dW; layer 1: forward + dW + dX; each product 2 * rows * d_in * d_out
     assert bench.gemm_flops(n, dims, [A, A]) == 2 * 10 * 4 * 3 * 2 + 2 * 10 * 3 * 2 * 3
     # last layer's backward on 5 compacted rows
-    assert bench.gemm_flops(n, dims, [A, A], 5) == 2 * 10 * 4 * 3 * 2 + 2 * 10 * 3 * 2 + 2 * (2 * 5 * 3 * 2)
+    assert bench.gemm_flops(n, dims, [A, A], [None, 5]) == 2 * 10 * 4 * 3 * 2 + 2 * 10 * 3 * 2 + 2 * (2 * 5 * 3 * 2)
     # ... and its forward too
-    assert bench.gemm_flops(n, dims, [A, A], 5, True) == 2 * 10 * 4 * 3 * 2 + 3 * (2 * 5 * 3 * 2)
-    # bytes: every n x d operand and result once per product
-    full = 4 * 10 * (4 + 3) * 2 + 4 * 10 * (3 + 2) * 3
-    assert bench.gemm_min_bytes(n, dims) == full
-    assert bench.gemm_min_bytes(n, dims, 5) == 4 * 10 * (4 + 3) * 2 + 4 * 10 * (3 + 2) + 2 * 4 * 5 * (3 + 2)
-    assert bench.gemm_min_bytes(n, dims, 5, True) == 4 * 10 * (4 + 3) * 2 + 3 * 4 * 5 * (3 + 2)
+    assert bench.gemm_flops(n, dims, [A, A], [None, 5], 5) == 2 * 10 * 4 * 3 * 2 + 3 * (2 * 5 * 3 * 2)
+    # first layer's backward (dW only) on 2 rows
+    assert bench.gemm_flops(n, dims, [A, A], [2, None]) == 2 * 4 * 3 * (10 + 2) + 2 * 10 * 3 * 2 * 3
+    # bytes: every rows x d operand and result once per product
+    assert bench.gemm_min_bytes(n, dims) == 4 * 10 * (4 + 3) * 2 + 4 * 10 * (3 + 2) * 3
+    assert bench.gemm_min_bytes(n, dims, [None, 5]) == 4 * 10 * (4 + 3) * 2 + 4 * 10 * (3 + 2) + 2 * 4 * 5 * (3 + 2)
+    assert bench.gemm_min_bytes(n, dims, [None, 5], 5) == 4 * 10 * (4 + 3) * 2 + 3 * 4 * 5 * (3 + 2)
 
 
 def test_peaks_are_read_from_the_measured_file_or_fall_back(bench):

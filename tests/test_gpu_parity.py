@@ -661,6 +661,37 @@ def test_training_epoch_row_sparse_matches_oracle(mg, ctx, levels):
     assert mg.ctx_poll_status(ctx, raise_on_error=False) == 0
 
 
+def test_second_level_row_set_is_counted_and_compacted(mg, ctx):
+    """Very few train nodes: the row mask reported by the top layer's backward is small enough for the
+    layer below to run its dense products on the compacted rows (count taken by mixgcn_count_rows)."""
+    from paper_2501_01951_b200.train import GcnTrainer
+    wl, s, d, X, y, m, Ws, bs = _tiny_problem()
+    m = torch.zeros(wl.n, dtype=torch.uint8)
+    deg = np.bincount(np.concatenate([s.numpy(), d.numpy()]), minlength=wl.n)
+    m[torch.as_tensor(np.nonzero((deg > 0) & (deg <= 3))[0][:6])] = 1        # six low-degree train nodes
+    go = orc.graph_build(wl.n, s.numpy(), d.numpy())
+    gg = mg.graph_create(ctx, wl.n, s, d)
+    dims = (64, 32, 16, 8)
+    Ws = [synth.glorot_uniform(dims[i], dims[i + 1], 400 + i) for i in range(3)]
+    bs = [synth.uniform_tensor((dims[i + 1],), 410 + i, -0.1, 0.1) for i in range(3)]
+    tr = GcnTrainer(ctx, gg, dims, mg.PREC_FP32, order=mg.ORDER_AGG_FIRST, row_sparse=2)
+    tr.set_params(Ws, bs)
+    tr.set_inputs(padded(X), y.cuda(), m.cuda())
+    ref = orc.train_epoch(go, X.numpy(), [w.numpy() for w in Ws], [b.numpy() for b in bs], y.numpy(), m.numpy(), None, 1, **ADAM)
+    for _ in range(2):                                                   # second pass reuses the stored count
+        tr.forward(); tr.compute_loss(); tr.backward()
+        cnt = tr.descs[1].gout_row_count
+        assert cnt == int(tr.row_masks[2].sum().item()) == mg.count_rows(ctx, tr.row_masks[2])
+        assert 0 < cnt * 4 < wl.n                                        # the compacted path was taken
+        nonzero = np.abs(orc.aggregate(go, orc.update_bwd(ref["Zs"][2], ref["Ps"][2], Ws[2].numpy(), ref["G"], relu=False)[3],
+                                       transposed=True)).sum(axis=1) > 0
+        assert np.all(tr.row_masks[2].cpu().numpy()[nonzero] == 1)
+        for l in range(3):
+            assert rel_fro(tr.dW[l].cpu().numpy(), ref["dW"][l]) <= TOL_FP32
+            assert rel_fro(tr.db[l].cpu().numpy(), ref["db"][l]) <= TOL_FP32
+    assert mg.ctx_poll_status(ctx, raise_on_error=False) == 0
+
+
 def test_spmm_column_slices_do_not_change_the_result(mg):
     """Feature-column slicing (the p:q-1 ranges of Algorithm 2) is a schedule, not arithmetic."""
     c2 = mg.ctx_create(0)
