@@ -190,7 +190,7 @@ def run_ours(args, rank, world, local_rank):
     n, nnz = g.n, g.nnz
     tr = GcnTrainer(ctx, g, wl.dims, prec, n_chunks=args.chunks,
                     row_sparse=args.row_sparse if args.row_sparse == "auto" else int(args.row_sparse),
-                    train_rows_only=args.train_rows_only)
+                    train_rows_only=args.train_rows_only, row_plans=not args.no_row_plans)
     X0 = synth.normal_features(n, wl.dims[0], wl.seed("features"), device=dev, ld=round4(wl.dims[0]))
     y = synth.uniform_labels(n, wl.classes, wl.seed("labels"), device=dev)
     m = synth.bernoulli_mask(n, wl.mask_p, wl.seed("mask"), device=dev)
@@ -238,7 +238,7 @@ def run_ours(args, rank, world, local_rank):
     for l, d in enumerate(tr.descs):
         cnt = int(d.gout_row_count)
         rows_flag = bool(d.flags & mg.LAYER_OUT_ROWS_ONLY)
-        compacted = bool(d.gout_row_mask) and cnt > 0 and tr.orders[l] == mg.ORDER_AGG_FIRST and (4 * cnt < n or rows_flag)
+        compacted = bool(d.gout_row_mask) and cnt > 0 and tr.orders[l] == mg.ORDER_AGG_FIRST and (4 * cnt < n or rows_flag or bool(d.gout_plan))
         bwd_rows.append(cnt if compacted else None)
 
     # Opt-in shortcut, reported beside the headline (never instead of it): the last layer's output, the
@@ -298,7 +298,7 @@ def run_ours(args, rank, world, local_rank):
                dtype={mg.PREC_FP32: "f32", mg.PREC_TF32: "tf32", mg.PREC_BF16: "bf16"}[prec], data="synthetic",
                config=dict(workload=wl.name, n=n, nnz=nnz, dims=list(wl.dims), train_nodes=n_train,
                            orders=["agg-first" if o == mg.ORDER_AGG_FIRST else "upd-first" for o in tr.orders],
-                           chunks=args.chunks, row_sparse_levels=tr.row_sparse_levels, backward_rows=[r if r is not None else n for r in bwd_rows], train_rows_only=bool(args.train_rows_only), l2="inputs larger than L2" if 4 * n * wl.dims[0] > 126e6 else "inputs fit L2 (no flush)",
+                           chunks=args.chunks, row_sparse_levels=tr.row_sparse_levels, backward_rows=[r if r is not None else n for r in bwd_rows], train_rows_only=bool(args.train_rows_only), row_plans=not args.no_row_plans, l2="inputs larger than L2" if 4 * n * wl.dims[0] > 126e6 else "inputs fit L2 (no flush)",
                            parallelism=f"replicas x{world}" if world > 1 else "single GPU", setup_s=round(setup_s, 1)),
                clocks=clk, gpu_launches=int(launches_after - launches_before),
                roofline=roofline, gemm=gemm, phase_ms_per_epoch=breakdown, loss=round(loss_val, 6), device_status=status)
@@ -430,6 +430,9 @@ def main():
     ap.add_argument("--train-rows-only", action="store_true",
                     help="opt-in shortcut: the last layer's output, the loss and its gradient on train rows only "
                          "(same loss and gradients; no predictions for the other nodes)")
+    ap.add_argument("--no-row-plans", action="store_true",
+                    help="row-sparse backward by testing the row masks inside the aggregation kernel every iteration "
+                         "instead of on restricted matrices built once")
     ap.add_argument("--row-sparse", default="auto", help="layers (from the top) whose backward gets a row mask: auto, 0, 1, 2, ...")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-seconds", type=float, default=20.0)

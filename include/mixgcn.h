@@ -44,6 +44,7 @@ typedef enum {
 
 typedef struct mixgcn_ctx mixgcn_ctx;
 typedef struct mixgcn_graph mixgcn_graph;
+typedef struct mixgcn_rowplan mixgcn_rowplan;   /* see mixgcn_rowplan_create */
 
 const char* mixgcn_status_string(mixgcn_status s);
 const char* mixgcn_last_error(void); /* thread-local, never NULL */
@@ -218,6 +219,10 @@ mixgcn_status mixgcn_gemm(mixgcn_ctx* ctx, int32_t precision, int32_t trans_a, i
                                        mask; n_chunks is ignored.  The backward call must then be
                                        given the same gout_row_mask. */
 
+#define MIXGCN_LAYER_GIN_ROWS_ONLY 32u /* backward with gout_plan: write only the rows of G_in in the
+                                       plan's out_row_mask (the other rows are exactly zero and
+                                       are left unchanged) */
+
 typedef struct {
     int32_t d_in, d_out;
     int64_t ld_in, ld_out, ld_saved;
@@ -241,7 +246,40 @@ typedef struct {
     const uint8_t* gout_row_mask;
     int64_t gout_row_count;
     uint8_t* gin_row_mask;
+    /* Backward with a row plan (optional; replaces gout_row_mask / gout_row_count / gin_row_mask in
+     * mixgcn_layer_bwd): a plan of A_hat^T created from the row mask of G_out.  The dense products run
+     * on the plan's compacted rows and the aggregation on its restricted matrix.  The rows of G_in that
+     * can be non-zero are the plan's out_row_mask; with MIXGCN_LAYER_GIN_ROWS_ONLY only those rows of
+     * G_in are written (for a layer below that itself runs with a plan made from that mask). */
+    const mixgcn_rowplan* gout_plan;
 } mixgcn_layer_desc;
+
+/* Row plan of a row-sparse aggregation.  Which rows of a gradient are non-zero depends on the graph
+ * and the train mask only, so what follows from it is computed once and reused every iteration: the
+ * kept rows (ascending) and the CSR of A_hat (transposed != 0: A_hat^T) restricted to the kept columns,
+ * renumbered to positions in the compacted input, with its own aggregation schedule.  in_row_mask is a
+ * device uint8[n] (non-zero = kept); it is read during the call only.  Synchronises the device.
+ * A plan may be used only while its context and graph exist; it may be destroyed after them.
+ * (The paper's sampled SpMM, Eq. 4, masks outputs; this is its counterpart on the operand's rows.) */
+mixgcn_status mixgcn_rowplan_create(mixgcn_ctx* ctx, const mixgcn_graph* g, int transposed,
+                                    const uint8_t* in_row_mask, mixgcn_rowplan** out);
+mixgcn_status mixgcn_rowplan_destroy(mixgcn_rowplan* plan);
+/* in_count kept input rows; out_count output rows with at least one kept entry; nnz kept entries.
+ * All nullable. */
+mixgcn_status mixgcn_rowplan_info(const mixgcn_rowplan* plan, int64_t* in_count, int64_t* out_count,
+                                  int64_t* nnz);
+/* Copies to DEVICE buffers (nullable): in_rows int32[in_count], the kept rows ascending;
+ * out_row_mask uint8[n], 1 for output rows with at least one kept entry (exactly the rows of the
+ * result that can be non-zero). */
+mixgcn_status mixgcn_rowplan_export(const mixgcn_rowplan* plan, int32_t* in_rows, uint8_t* out_row_mask,
+                                    void* stream);
+/* Z = epilogue(A_restricted Yc): Yc is the COMPACTED input, in_count x ldy, row i = row in_rows[i] of
+ * the full input; Z is n x ldz.  The same sum as mixgcn_spmm on the full input whose other rows are
+ * zero.  rows_only != 0: only the rows of Z in the plan's out_row_mask are written (the others are
+ * exactly zero in the full result and are left unchanged here).  Other arguments as mixgcn_spmm. */
+mixgcn_status mixgcn_spmm_rowplan(mixgcn_ctx* ctx, const mixgcn_rowplan* plan, int32_t w, const float* Yc,
+                                  int64_t ldy, float* Z, int64_t ldz, const mixgcn_epilogue* epi,
+                                  int32_t rows_only, void* stream);
 
 /* Resolves MIXGCN_ORDER_AUTO: cost(agg-first) = c * d_in with c = 1 for a FIRST layer (its
  * backward needs no aggregation) else 2; cost(upd-first) = 2 * d_out; the smaller wins, ties

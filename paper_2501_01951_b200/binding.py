@@ -26,7 +26,7 @@ OK, EINVAL, ENOMEM, ECUDA, EUNSUPPORTED, EBADGRAPH, ETIMEOUT, EDEVICE = range(8)
 GRAPH_SYMMETRISE, GRAPH_ADD_SELF_LOOPS, GRAPH_EDGES_ON_DEVICE = 1, 2, 4
 PREC_FP32, PREC_TF32, PREC_BF16 = 0, 1, 2
 ORDER_AUTO, ORDER_AGG_FIRST, ORDER_UPD_FIRST = 0, 1, 2
-LAYER_RELU, LAYER_FIRST, LAYER_GATE_GIN, LAYER_GOUT_GATED, LAYER_OUT_ROWS_ONLY = 1, 2, 4, 8, 16
+LAYER_RELU, LAYER_FIRST, LAYER_GATE_GIN, LAYER_GOUT_GATED, LAYER_OUT_ROWS_ONLY, LAYER_GIN_ROWS_ONLY = 1, 2, 4, 8, 16, 32
 N_PHASES = 7
 PHASES = ("spmm", "gemm", "elementwise", "loss", "adam", "graph", "spmm_sparse")
 PRECISIONS = {"fp32": PREC_FP32, "tf32": PREC_TF32, "bf16": PREC_BF16}
@@ -40,7 +40,8 @@ SYMBOLS = (
     "mixgcn_layer_plan", "mixgcn_layer_fwd", "mixgcn_layer_bwd", "mixgcn_loss_softmax_xent",
     "mixgcn_adam_step", "mixgcn_train_step_host", "mixgcn_loss_softmax_xent_noalloc", "mixgcn_ctx_set_option",
     "mixgcn_graph_bandwidth", "mixgcn_graph_rcm", "mixgcn_pipeline_stages", "mixgcn_graph_create_permuted",
-    "mixgcn_count_rows",
+    "mixgcn_count_rows", "mixgcn_rowplan_create", "mixgcn_rowplan_destroy", "mixgcn_rowplan_info",
+    "mixgcn_rowplan_export", "mixgcn_spmm_rowplan",
 )
 
 
@@ -55,7 +56,7 @@ class LayerDesc(C.Structure):
                 ("ld_saved", C.c_int64), ("order", C.c_int32), ("precision", C.c_int32),
                 ("flags", C.c_uint32), ("keep_scale", C.c_float), ("in_scale", C.c_float),
                 ("n_chunks", C.c_int32), ("gout_row_mask", C.c_void_p), ("gout_row_count", C.c_int64),
-                ("gin_row_mask", C.c_void_p)]
+                ("gin_row_mask", C.c_void_p), ("gout_plan", C.c_void_p)]
 
 
 lib.mixgcn_status_string.restype = C.c_char_p
@@ -358,6 +359,57 @@ def adam_step(ctx: Ctx, params, grads, ms, vs, t, lr=0.01, beta1=0.9, beta2=0.99
     numel = (C.c_int64 * k)(*[x.numel() for x in params])
     _check(lib.mixgcn_adam_step(ctx.h, C.c_int32(k), arr(params), arr(grads), arr(ms), arr(vs), numel, C.c_int64(t),
                                 C.c_float(lr), C.c_float(beta1), C.c_float(beta2), C.c_float(eps), _stream()))
+
+
+class RowPlan:
+    """Row plan of a row-sparse aggregation (see mixgcn_rowplan_create)."""
+
+    def __init__(self, ctx: Ctx, g: Graph, handle):
+        self.ctx, self.g, self.h = ctx, g, handle
+        a, b, c = C.c_int64(), C.c_int64(), C.c_int64()
+        _check(lib.mixgcn_rowplan_info(self.h, C.byref(a), C.byref(b), C.byref(c)))
+        self.in_count, self.out_count, self.nnz = a.value, b.value, c.value
+
+    def in_rows(self) -> torch.Tensor:
+        out = torch.empty(self.in_count, dtype=torch.int32, device=torch.device("cuda", self.ctx.device))
+        _check(lib.mixgcn_rowplan_export(self.h, _ptr(out), None, _stream()))
+        return out
+
+    def out_row_mask(self) -> torch.Tensor:
+        out = torch.empty(self.g.n, dtype=torch.uint8, device=torch.device("cuda", self.ctx.device))
+        _check(lib.mixgcn_rowplan_export(self.h, None, _ptr(out), _stream()))
+        return out
+
+    def close(self):
+        if self.h:
+            lib.mixgcn_rowplan_destroy(self.h)
+            self.h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def rowplan_create(ctx: Ctx, g: Graph, in_row_mask: torch.Tensor, transposed: bool = True) -> RowPlan:
+    _dev(in_row_mask, torch.uint8, "in_row_mask")
+    if in_row_mask.numel() != g.n:
+        raise ValueError("rowplan_create: the mask needs one byte per node")
+    torch.cuda.current_stream().synchronize()
+    h = C.c_void_p()
+    _check(lib.mixgcn_rowplan_create(ctx.h, g.h, C.c_int(1 if transposed else 0), _ptr(in_row_mask), C.byref(h)))
+    return RowPlan(ctx, g, h)
+
+
+def spmm_rowplan(ctx: Ctx, plan: RowPlan, Yc: torch.Tensor, Z: torch.Tensor, w: int, epi=None, rows_only=False):
+    """Z = epilogue(A_restricted Yc) with Yc the compacted input (plan.in_count rows)."""
+    _dev(Yc, torch.float32, "Yc"); _dev(Z, torch.float32, "Z")
+    if Yc.shape[0] != plan.in_count or Z.shape[0] != plan.g.n:
+        raise ValueError("spmm_rowplan: Yc needs plan.in_count rows and Z one row per node")
+    _check(lib.mixgcn_spmm_rowplan(ctx.h, plan.h, C.c_int32(w), _ptr(Yc), C.c_int64(Yc.stride(0)), _ptr(Z),
+                                   C.c_int64(Z.stride(0)), C.byref(epi) if epi is not None else None,
+                                   C.c_int32(1 if rows_only else 0), _stream()))
 
 
 def count_rows(ctx: Ctx, row_mask) -> int:

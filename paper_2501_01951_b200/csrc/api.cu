@@ -388,6 +388,35 @@ extern "C" mixgcn_status mixgcn_layer_bwd(mixgcn_ctx* ctx, const mixgcn_graph* g
         gin_epi.gate = X_in; gin_epi.ld_gate = d->ld_in; gin_epi.gate_scale = d->in_scale; gin_epi.keep_scale = 1.0f;
         gin = &gin_epi;
     }
+    if (const mixgcn_rowplan* plan = d->gout_plan) {
+        // Row plan: dense products on the plan's compacted rows, aggregation on its restricted matrix.
+        if (plan->ctx != ctx || plan->g != g || !plan->transposed) MIXGCN_FAIL(MIXGCN_EINVAL, "layer_bwd: gout_plan must be a plan of this graph's transposed orientation");
+        const int64_t cnt = plan->in_count;
+        const int64_t lda = (d->d_in + 3) / 4 * 4, ldb = (d->d_out + 3) / 4 * 4;
+        auto up = [](int64_t x) { return (x + 255) & ~(int64_t)255; };
+        const int64_t rows_alloc = cnt > 0 ? cnt : 1;
+        MIXGCN_TRY(ensure_workspace_rows(ctx, up(rows_alloc * lda * 4) + up(rows_alloc * ldb * 4)));
+        float* ca = reinterpret_cast<float*>(ctx->workspace_rows);
+        float* cb = reinterpret_cast<float*>(reinterpret_cast<char*>(ctx->workspace_rows) + up(rows_alloc * lda * 4));
+        const uint8_t* gin_rows = (d->flags & MIXGCN_LAYER_GIN_ROWS_ONLY) ? plan->out_mask : nullptr;
+        MIXGCN_TRY(launch_gather_rows(ctx, cnt, d->d_out, plan->idx, G_out, d->ld_out, cb, ldb, s));         // dP_T
+        if (dbias) MIXGCN_TRY(launch_colsum(ctx, cnt, d->d_out, cb, ldb, dbias, s));
+        if (order == MIXGCN_ORDER_AGG_FIRST) {
+            MIXGCN_TRY(launch_gather_rows(ctx, cnt, d->d_in, plan->idx, saved, d->ld_saved, ca, lda, s));     // Z_T
+            MIXGCN_TRY(launch_gemm(ctx, d->precision, 1, 0, d->d_in, d->d_out, cnt, ca, lda, cb, ldb, dW, ldw, nullptr, 0, s));
+            if (!first) {
+                MIXGCN_TRY(launch_gemm(ctx, d->precision, 0, 1, cnt, d->d_in, d->d_out, cb, ldb, W, ldw, ca, lda, nullptr, 0, s));
+                MIXGCN_TRY(launch_spmm(ctx, g, plan->view, 1, 0, d->d_in, ca, lda, G_in, d->ld_in, gin, s, nullptr, gin_rows, PH_SPMM_SPARSE));
+            }
+            return MIXGCN_OK;
+        }
+        // update first: dQ = A_hat^T dZ from the compacted rows (into `saved`, every row), then the dense products
+        MIXGCN_TRY(launch_spmm(ctx, g, plan->view, 1, 0, d->d_out, cb, ldb, saved, d->ld_saved, nullptr, s, nullptr, nullptr, PH_SPMM_SPARSE));
+        MIXGCN_TRY(launch_gemm(ctx, d->precision, 1, 0, d->d_in, d->d_out, n, X_in, d->ld_in, saved, d->ld_saved, dW, ldw, nullptr, 0, s));
+        if (!first)
+            MIXGCN_TRY(launch_gemm(ctx, d->precision, 0, 1, n, d->d_in, d->d_out, saved, d->ld_saved, W, ldw, G_in, d->ld_in, gin, 0, s));
+        return MIXGCN_OK;
+    }
     const uint8_t* rmask = d->gout_row_mask;
     SpmmRowSparse sp{rmask, nullptr, d->gin_row_mask};
     const SpmmRowSparse* spp = rmask ? &sp : nullptr;

@@ -428,6 +428,12 @@ mixgcn_status check_common(mixgcn_ctx* ctx, int64_t n, mixgcn_graph** out) {
 
 namespace mixgcn {
 
+mixgcn_status build_view_schedule(int64_t n_cols, int64_t n, CsrView& v, cudaStream_t s) {
+    return build_schedule(n_cols, v.rowptr, v.col, 0, n, v.full, s);
+}
+
+void release_view(CsrView& v) { free_view(v); }
+
 mixgcn_status ensure_chunk_schedules(const mixgcn_graph* g, const CsrView& A_const, int chunks) {
     // a cache inside the graph object; a symmetric graph keeps one set (in fwd) and mirrors it into the alias
     CsrView& A = const_cast<CsrView&>(g->symmetric ? g->fwd : A_const);

@@ -116,6 +116,20 @@ struct mixgcn_graph {
     CsrView fwd, bwd;  // bwd aliases fwd when symmetric
 };
 
+// Everything about a row-sparse aggregation that depends only on the graph and on WHICH rows of the
+// input are non-zero: the kept rows, their positions, and the orientation's CSR restricted to the kept
+// columns (column ids renumbered to positions in the compacted input) with its own schedule.
+struct mixgcn_rowplan {
+    mixgcn_ctx* ctx;
+    int device;          // kept apart from ctx: a plan may be destroyed after its context
+    const mixgcn_graph* g;
+    int transposed;
+    int64_t n, in_count, out_count, nnz;
+    int32_t* idx;        // [in_count] kept input rows, ascending
+    CsrView view;        // n rows; columns in [0, in_count)
+    uint8_t* out_mask;   // [n] 1 for output rows that have at least one kept entry
+};
+
 namespace mixgcn {
 
 #ifndef MIXGCN_SPMM_SEG
@@ -165,7 +179,10 @@ struct SpmmRowSparse {
 mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView& A, int chunks, int k,
                           int32_t w, const float* Y, int64_t ldy, float* Z, int64_t ldz,
                           const mixgcn_epilogue* epi, cudaStream_t s, const SpmmRowSparse* sparse = nullptr,
-                          const uint8_t* row_filter = nullptr);
+                          const uint8_t* row_filter = nullptr, int phase = PH_SPMM);
+// schedule of all n rows of a view whose column ids lie in [0, n_cols); release of a view's memory
+mixgcn_status build_view_schedule(int64_t n_cols, int64_t n, CsrView& v, cudaStream_t s);
+void release_view(CsrView& v);
 mixgcn_status launch_gemm(mixgcn_ctx* ctx, int precision, int ta, int tb, int64_t M, int64_t N, int64_t K,
                           const float* A, int64_t lda, const float* B, int64_t ldb, float* C, int64_t ldc,
                           const mixgcn_epilogue* epi, int64_t epi_row0, cudaStream_t s);
@@ -187,6 +204,7 @@ mixgcn_status build_row_set(mixgcn_ctx* ctx, int64_t n, const uint8_t* mask, int
 mixgcn_status launch_gather_rows(mixgcn_ctx* ctx, int64_t count, int32_t d, const int32_t* idx, const float* src,
                                  int64_t ld_src, float* dst, int64_t ld_dst, cudaStream_t s);
 
+mixgcn_status ensure_workspace_rows(mixgcn_ctx* ctx, int64_t bytes);
 // dst[idx[i], :] = src[i, :] for i < count (the inverse of launch_gather_rows)
 mixgcn_status launch_scatter_rows(mixgcn_ctx* ctx, int64_t count, int32_t d, const int32_t* idx, const float* src,
                                   int64_t ld_src, float* dst, int64_t ld_dst, cudaStream_t s);

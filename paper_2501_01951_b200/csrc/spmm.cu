@@ -390,7 +390,7 @@ namespace mixgcn {
 mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView& A, int chunks, int k,
                           int32_t w, const float* Y, int64_t ldy, float* Z, int64_t ldz,
                           const mixgcn_epilogue* epi, cudaStream_t s, const SpmmRowSparse* sparse,
-                          const uint8_t* row_filter) {
+                          const uint8_t* row_filter, int phase) {
     if (w <= 0) return MIXGCN_OK;
     if (sparse && row_filter) MIXGCN_FAIL(MIXGCN_EUNSUPPORTED, "spmm: a row filter cannot be combined with a row-sparse input");
     if (chunks > 1) {
@@ -483,12 +483,12 @@ mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView&
             MIXGCN_TRY(ensure_workspace_spmm(ctx, S.total_segs * ldp * (int64_t)sizeof(float)));
             p.partial = reinterpret_cast<float*>(ctx->workspace_spmm); p.ldp = ldp;
             {
-                LaunchScope scope(ctx, PH_SPMM, s);
+                LaunchScope scope(ctx, phase, s);
                 p.idx_begin = 0; p.idx_end = S.total_segs;
                 dispatch(p, 1, s);
             }
             {
-                LaunchScope scope(ctx, PH_SPMM, s);
+                LaunchScope scope(ctx, phase, s);
                 const int64_t blocks = (S.n_long * 32 + 255) / 256;
                 spmm_combine_kernel<<<(unsigned)blocks, 256, 0, s>>>(p, S.n_long, S.seg_off, S.seg_pos, S.perm);
             }
@@ -506,7 +506,7 @@ mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView&
             if (end <= begin) continue;
             p.idx_begin = S.total_segs + (begin - S.n_long);
             p.idx_end = S.total_segs + (end - S.n_long);
-            LaunchScope scope(ctx, PH_SPMM, s);
+            LaunchScope scope(ctx, phase, s);
             dispatch(p, fold, s);
             begin = end;
         }

@@ -19,7 +19,7 @@ def round4(x: int) -> int:
 class GcnTrainer:
     def __init__(self, ctx: mg.Ctx, graph: mg.Graph, dims, precision=mg.PREC_FP32, order=mg.ORDER_AUTO,
                  n_chunks=0, fuse_gate=True, keep_scale=1.0, device=None, row_sparse="auto",
-                 train_rows_only=False):
+                 train_rows_only=False, row_plans=True):
         self.ctx, self.g = ctx, graph
         self.dims = tuple(int(d) for d in dims)
         self.L = len(self.dims) - 1
@@ -32,6 +32,9 @@ class GcnTrainer:
         # opt-in: the last layer's output, the loss and its gradient on train rows only (needs a
         # row-sparse backward for the last layer; predictions exist for train rows only)
         self.train_rows_only = bool(train_rows_only)
+        # row plans: the row-sparse backward on restricted matrices built once per (graph, train mask);
+        # False = the masks are tested inside the aggregation kernel every iteration
+        self.use_row_plans = bool(row_plans)
         n, L = self.n, self.L
         orders = order if isinstance(order, (list, tuple)) else [order] * L
         self.descs, self.orders = [], []
@@ -110,9 +113,10 @@ class GcnTrainer:
         levels = max(0, min(int(levels), L))
         self.row_sparse_levels = levels
         self.row_masks = [None] * (L + 1)
+        self.row_plans = [None] * L
         for d in self.descs:
-            d.gout_row_mask, d.gout_row_count, d.gin_row_mask = None, 0, None
-            d.flags &= ~mg.LAYER_OUT_ROWS_ONLY
+            d.gout_row_mask, d.gout_row_count, d.gin_row_mask, d.gout_plan = None, 0, None, None
+            d.flags &= ~(mg.LAYER_OUT_ROWS_ONLY | mg.LAYER_GIN_ROWS_ONLY)
         if self.train_rows_only:
             if levels == 0 or n_train == 0 or self.masks[L - 1] is not None:
                 raise ValueError("train_rows_only needs a row-sparse backward (row_sparse >= 1), a non-empty "
@@ -125,10 +129,20 @@ class GcnTrainer:
             l = L - 1 - i                                 # layer whose backward receives row_masks[l + 1]
             d = self.descs[l]
             d.gout_row_mask = self.row_masks[l + 1].data_ptr()
-            d.gout_row_count = n_train if i == 0 else 0
-            if l > 0 and i + 1 < levels:
-                self.row_masks[l] = torch.zeros(n, dtype=torch.uint8, device=self.device)
-                d.gin_row_mask = self.row_masks[l].data_ptr()
+            if self.use_row_plans and n_train > 0:
+                # everything that depends on the graph and the mask only, computed once
+                plan = mg.rowplan_create(self.ctx, self.g, self.row_masks[l + 1])
+                self.row_plans[l] = plan
+                d.gout_plan = plan.h
+                d.gout_row_count = plan.in_count
+                if l > 0 and i + 1 < levels:
+                    self.row_masks[l] = plan.out_row_mask()
+                    d.flags |= mg.LAYER_GIN_ROWS_ONLY     # the layer below gathers exactly these rows of G_in
+            else:
+                d.gout_row_count = n_train if i == 0 else 0
+                if l > 0 and i + 1 < levels:
+                    self.row_masks[l] = torch.zeros(n, dtype=torch.uint8, device=self.device)
+                    d.gin_row_mask = self.row_masks[l].data_ptr()
 
     # -- the iteration --------------------------------------------------------------------------
     def forward(self):

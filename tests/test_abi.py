@@ -36,8 +36,9 @@ def test_status_strings(mg):
 def test_struct_layouts_match_the_header(mg):
     # the header's structs, field by field, on an LP64 ABI
     assert C.sizeof(mg.Epilogue) == 56
-    assert C.sizeof(mg.LayerDesc) == 80
+    assert C.sizeof(mg.LayerDesc) == 88
     assert mg.LayerDesc.gout_row_mask.offset == 56 and mg.LayerDesc.gin_row_mask.offset == 72
+    assert mg.LayerDesc.gout_plan.offset == 80
     assert mg.LayerDesc.ld_in.offset == 8 and mg.LayerDesc.order.offset == 32 and mg.LayerDesc.n_chunks.offset == 52
     assert mg.Epilogue.keep_scale.offset == 24 and mg.Epilogue.ld_gate.offset == 40
 

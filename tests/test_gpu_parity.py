@@ -639,7 +639,8 @@ def test_row_sparse_wrong_count_is_reported_not_a_fault(mg, ctx):
 
 
 @pytest.mark.parametrize("levels", [1, 2])
-def test_training_epoch_row_sparse_matches_oracle(mg, ctx, levels):
+@pytest.mark.parametrize("row_plans", [True, False])
+def test_training_epoch_row_sparse_matches_oracle(mg, ctx, levels, row_plans):
     from paper_2501_01951_b200.train import GcnTrainer
     wl, s, d, X, y, m, Ws, bs = _tiny_problem()
     m = synth.bernoulli_mask(wl.n, 0.03, 77)                           # few train nodes
@@ -648,10 +649,11 @@ def test_training_epoch_row_sparse_matches_oracle(mg, ctx, levels):
     dims = (64, 32, 16, 8)                                             # three layers so that two levels exist
     Ws = [synth.glorot_uniform(dims[i], dims[i + 1], 400 + i) for i in range(3)]
     bs = [synth.uniform_tensor((dims[i + 1],), 410 + i, -0.1, 0.1) for i in range(3)]
-    tr = GcnTrainer(ctx, gg, dims, mg.PREC_FP32, order=mg.ORDER_AGG_FIRST, row_sparse=levels)
+    tr = GcnTrainer(ctx, gg, dims, mg.PREC_FP32, order=mg.ORDER_AGG_FIRST, row_sparse=levels, row_plans=row_plans)
     tr.set_params(Ws, bs)
     tr.set_inputs(padded(X), y.cuda(), m.cuda())
     assert tr.row_sparse_levels == levels
+    assert all((p is not None) == (row_plans and l >= 3 - levels) for l, p in enumerate(tr.row_plans))
     tr.forward(); tr.compute_loss(); tr.backward()
     ref = orc.train_epoch(go, X.numpy(), [w.numpy() for w in Ws], [b.numpy() for b in bs], y.numpy(), m.numpy(), None, 1, **ADAM)
     assert abs(tr.loss.item() - ref["loss"]) <= 1e-5 * abs(ref["loss"])
@@ -674,7 +676,7 @@ def test_second_level_row_set_is_counted_and_compacted(mg, ctx):
     dims = (64, 32, 16, 8)
     Ws = [synth.glorot_uniform(dims[i], dims[i + 1], 400 + i) for i in range(3)]
     bs = [synth.uniform_tensor((dims[i + 1],), 410 + i, -0.1, 0.1) for i in range(3)]
-    tr = GcnTrainer(ctx, gg, dims, mg.PREC_FP32, order=mg.ORDER_AGG_FIRST, row_sparse=2)
+    tr = GcnTrainer(ctx, gg, dims, mg.PREC_FP32, order=mg.ORDER_AGG_FIRST, row_sparse=2, row_plans=False)
     tr.set_params(Ws, bs)
     tr.set_inputs(padded(X), y.cuda(), m.cuda())
     ref = orc.train_epoch(go, X.numpy(), [w.numpy() for w in Ws], [b.numpy() for b in bs], y.numpy(), m.numpy(), None, 1, **ADAM)
