@@ -398,7 +398,8 @@ extern "C" mixgcn_status mixgcn_layer_bwd(mixgcn_ctx* ctx, const mixgcn_graph* g
         MIXGCN_TRY(ensure_workspace_rows(ctx, up(rows_alloc * lda * 4) + up(rows_alloc * ldb * 4)));
         float* ca = reinterpret_cast<float*>(ctx->workspace_rows);
         float* cb = reinterpret_cast<float*>(reinterpret_cast<char*>(ctx->workspace_rows) + up(rows_alloc * lda * 4));
-        const uint8_t* gin_rows = (d->flags & MIXGCN_LAYER_GIN_ROWS_ONLY) ? plan->out_mask : nullptr;
+        // rows of the restricted matrix are scheduled longest first: its non-empty rows are the first out_count
+        const int64_t gin_rows = (d->flags & MIXGCN_LAYER_GIN_ROWS_ONLY) ? plan->out_count : -1;
         MIXGCN_TRY(launch_gather_rows(ctx, cnt, d->d_out, plan->idx, G_out, d->ld_out, cb, ldb, s));         // dP_T
         if (dbias) MIXGCN_TRY(launch_colsum(ctx, cnt, d->d_out, cb, ldb, dbias, s));
         if (order == MIXGCN_ORDER_AGG_FIRST) {
@@ -406,7 +407,7 @@ extern "C" mixgcn_status mixgcn_layer_bwd(mixgcn_ctx* ctx, const mixgcn_graph* g
             MIXGCN_TRY(launch_gemm(ctx, d->precision, 1, 0, d->d_in, d->d_out, cnt, ca, lda, cb, ldb, dW, ldw, nullptr, 0, s));
             if (!first) {
                 MIXGCN_TRY(launch_gemm(ctx, d->precision, 0, 1, cnt, d->d_in, d->d_out, cb, ldb, W, ldw, ca, lda, nullptr, 0, s));
-                MIXGCN_TRY(launch_spmm(ctx, g, plan->view, 1, 0, d->d_in, ca, lda, G_in, d->ld_in, gin, s, nullptr, gin_rows, PH_SPMM_SPARSE));
+                MIXGCN_TRY(launch_spmm(ctx, g, plan->view, 1, 0, d->d_in, ca, lda, G_in, d->ld_in, gin, s, nullptr, nullptr, PH_SPMM_SPARSE, gin_rows));
             }
             return MIXGCN_OK;
         }

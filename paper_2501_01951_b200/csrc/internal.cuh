@@ -179,7 +179,7 @@ struct SpmmRowSparse {
 mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView& A, int chunks, int k,
                           int32_t w, const float* Y, int64_t ldy, float* Z, int64_t ldz,
                           const mixgcn_epilogue* epi, cudaStream_t s, const SpmmRowSparse* sparse = nullptr,
-                          const uint8_t* row_filter = nullptr, int phase = PH_SPMM);
+                          const uint8_t* row_filter = nullptr, int phase = PH_SPMM, int64_t row_limit = -1);
 // schedule of all n rows of a view whose column ids lie in [0, n_cols); release of a view's memory
 mixgcn_status build_view_schedule(int64_t n_cols, int64_t n, CsrView& v, cudaStream_t s);
 void release_view(CsrView& v);

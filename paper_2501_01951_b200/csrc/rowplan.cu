@@ -196,6 +196,7 @@ extern "C" mixgcn_status mixgcn_spmm_rowplan(mixgcn_ctx* ctx, const mixgcn_rowpl
     if (Yc == Z) MIXGCN_FAIL(MIXGCN_EINVAL, "spmm_rowplan: Yc and Z must not overlap");
     if (epi && epi->gate && epi->ld_gate < w) MIXGCN_FAIL(MIXGCN_EINVAL, "spmm_rowplan: gate leading dimension < w");
     MIXGCN_CUDA(cudaSetDevice(ctx->device));
-    return launch_spmm(ctx, p->g, p->view, 1, 0, w, Yc, ldy, Z, ldz, epi, (cudaStream_t)stream, nullptr,
-                       rows_only ? p->out_mask : nullptr, PH_SPMM_SPARSE);
+    // rows of the restricted matrix are scheduled longest first, so its non-empty rows are the first out_count
+    return launch_spmm(ctx, p->g, p->view, 1, 0, w, Yc, ldy, Z, ldz, epi, (cudaStream_t)stream, nullptr, nullptr,
+                       PH_SPMM_SPARSE, rows_only ? p->out_count : -1);
 }

@@ -70,6 +70,12 @@ __device__ __forceinline__ void store_row(const SpmmParams& p, int64_t u, int c4
     const int j = p.j0 + c4 * 4;           // global column of a.x
     const int jend = p.j0 + p.w;           // one past the last valid column of the slice
     float r[4] = {a.x, a.y, a.z, a.w};
+    if (!p.bias && a.x == 0.0f && a.y == 0.0f && a.z == 0.0f && a.w == 0.0f) {
+        // ReLU, dropout and the gate all map 0 to 0: no mask or gate byte needs to be read (the empty
+        // rows of a row-sparse aggregation take this path)
+        *reinterpret_cast<float4*>(p.Z + u * p.ldz + j) = make_float4(0.f, 0.f, 0.f, 0.f);
+        return;
+    }
 #pragma unroll
     for (int t = 0; t < 4; ++t) r[t] = (j + t < jend) ? epilogue1(p, r[t], u, j + t) : 0.0f;
     *reinterpret_cast<float4*>(p.Z + u * p.ldz + j) = make_float4(r[0], r[1], r[2], r[3]);
@@ -390,7 +396,7 @@ namespace mixgcn {
 mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView& A, int chunks, int k,
                           int32_t w, const float* Y, int64_t ldy, float* Z, int64_t ldz,
                           const mixgcn_epilogue* epi, cudaStream_t s, const SpmmRowSparse* sparse,
-                          const uint8_t* row_filter, int phase) {
+                          const uint8_t* row_filter, int phase, int64_t row_limit) {
     if (w <= 0) return MIXGCN_OK;
     if (sparse && row_filter) MIXGCN_FAIL(MIXGCN_EUNSUPPORTED, "spmm: a row filter cannot be combined with a row-sparse input");
     if (chunks > 1) {
@@ -499,6 +505,11 @@ mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView&
         bound[0] = S.n_long;
         for (int q = 0; q < 3; ++q) bound[q + 1] = S.rows_above[q] > S.n_long ? S.rows_above[q] : S.n_long;
         bound[4] = S.n_rows;
+        if (row_limit >= 0 && row_limit < S.n_rows) {
+            // rows come longest first: only the first row_limit of them are wanted (the rest are empty)
+            const int64_t lim = row_limit > S.n_long ? row_limit : S.n_long;
+            for (int q = 1; q < 5; ++q) if (bound[q] > lim) bound[q] = lim;
+        }
         int64_t begin = bound[0];
         int fold = 1;
         for (int q = 0; q < 4; ++q, fold <<= 1) {
