@@ -219,6 +219,12 @@ mixgcn_status mixgcn_gemm(mixgcn_ctx* ctx, int32_t precision, int32_t trans_a, i
                                        mask; n_chunks is ignored.  The backward call must then be
                                        given the same gout_row_mask. */
 
+#define MIXGCN_LAYER_SAVED_IS_VALID 64u /* forward of a FIRST layer in agg-first order: `saved` already
+                                       holds A_hat X_in from an earlier call and neither the graph
+                                       nor X_in has changed since (full-graph training feeds the
+                                       same features every epoch, and the first layer's backward
+                                       leaves `saved` intact): the aggregation is skipped.  Not in
+                                       the paper, which recomputes it every iteration. */
 #define MIXGCN_LAYER_GIN_ROWS_ONLY 32u /* backward with gout_plan: write only the rows of G_in in the
                                        plan's out_row_mask (the other rows are exactly zero and
                                        are left unchanged) */

@@ -299,7 +299,13 @@ extern "C" mixgcn_status mixgcn_layer_fwd(mixgcn_ctx* ctx, const mixgcn_graph* g
     epi.drop_mask = drop_mask;
     epi.keep_scale = d->keep_scale;
     const int64_t ldw = d->d_out;  // W is dense; the GEMM uses scalar loads for it when d_out % 4 != 0
-    const int chunks = d->n_chunks > 1 ? d->n_chunks : 1;
+    int chunks = d->n_chunks > 1 ? d->n_chunks : 1;
+    const bool saved_valid = (d->flags & MIXGCN_LAYER_SAVED_IS_VALID) != 0;
+    if (saved_valid) {
+        if (!(d->flags & MIXGCN_LAYER_FIRST) || order != MIXGCN_ORDER_AGG_FIRST)
+            MIXGCN_FAIL(MIXGCN_EINVAL, "layer_fwd: SAVED_IS_VALID is for a FIRST layer in agg-first order");
+        chunks = 1;
+    }
 
     if (d->flags & MIXGCN_LAYER_OUT_ROWS_ONLY) {
         // Only the rows in gout_row_mask are wanted: aggregate those rows alone; in agg-first order the
@@ -309,7 +315,8 @@ extern "C" mixgcn_status mixgcn_layer_fwd(mixgcn_ctx* ctx, const mixgcn_graph* g
         if (!rows || cnt <= 0 || cnt > n) MIXGCN_FAIL(MIXGCN_EINVAL, "layer_fwd: OUT_ROWS_ONLY needs gout_row_mask and its exact count");
         if (drop_mask) MIXGCN_FAIL(MIXGCN_EUNSUPPORTED, "layer_fwd: OUT_ROWS_ONLY does not take a dropout mask");
         if (order == MIXGCN_ORDER_AGG_FIRST) {
-            MIXGCN_TRY(launch_spmm(ctx, g, g->fwd, 1, 0, d->d_in, X_in, d->ld_in, saved, d->ld_saved, nullptr, s, nullptr, rows));
+            if (!saved_valid)
+                MIXGCN_TRY(launch_spmm(ctx, g, g->fwd, 1, 0, d->d_in, X_in, d->ld_in, saved, d->ld_saved, nullptr, s, nullptr, rows));
             RowSet rs;
             const int64_t lda = (d->d_in + 3) / 4 * 4, ldb = (d->d_out + 3) / 4 * 4;
             MIXGCN_TRY(build_row_set(ctx, n, rows, cnt, lda, ldb, &rs, s));
@@ -326,7 +333,8 @@ extern "C" mixgcn_status mixgcn_layer_fwd(mixgcn_ctx* ctx, const mixgcn_graph* g
 
     if (order == MIXGCN_ORDER_AGG_FIRST) {
         if (chunks == 1) {
-            MIXGCN_TRY(launch_spmm(ctx, g, g->fwd, 1, 0, d->d_in, X_in, d->ld_in, saved, d->ld_saved, nullptr, s));
+            if (!saved_valid)
+                MIXGCN_TRY(launch_spmm(ctx, g, g->fwd, 1, 0, d->d_in, X_in, d->ld_in, saved, d->ld_saved, nullptr, s));
             MIXGCN_TRY(launch_gemm(ctx, d->precision, 0, 0, n, d->d_out, d->d_in, saved, d->ld_saved, W, ldw, X_out,
                                    d->ld_out, &epi, 0, s));
             return MIXGCN_OK;

@@ -19,7 +19,7 @@ def round4(x: int) -> int:
 class GcnTrainer:
     def __init__(self, ctx: mg.Ctx, graph: mg.Graph, dims, precision=mg.PREC_FP32, order=mg.ORDER_AUTO,
                  n_chunks=0, fuse_gate=True, keep_scale=1.0, device=None, row_sparse="auto",
-                 train_rows_only=False, row_plans=True):
+                 train_rows_only=False, row_plans=True, cache_first_aggregation=False):
         self.ctx, self.g = ctx, graph
         self.dims = tuple(int(d) for d in dims)
         self.L = len(self.dims) - 1
@@ -35,6 +35,10 @@ class GcnTrainer:
         # row plans: the row-sparse backward on restricted matrices built once per (graph, train mask);
         # False = the masks are tested inside the aggregation kernel every iteration
         self.use_row_plans = bool(row_plans)
+        # opt-in: keep A_hat X^(0) of an agg-first first layer across iterations (features and graph are
+        # the same every epoch); the paper recomputes it
+        self.cache_first_aggregation = bool(cache_first_aggregation)
+        self._first_aggregation_valid = False
         n, L = self.n, self.L
         orders = order if isinstance(order, (list, tuple)) else [order] * L
         self.descs, self.orders = [], []
@@ -95,6 +99,8 @@ class GcnTrainer:
         self.X[0], self.labels, self.train_mask = X0, labels, train_mask
         if drop_masks is not None:
             self.masks = list(drop_masks) + [None] * (self.L - len(drop_masks))
+        self._first_aggregation_valid = False
+        self.descs[0].flags &= ~mg.LAYER_SAVED_IS_VALID
         self._plan_row_sparsity()
 
     def _plan_row_sparsity(self):
@@ -146,9 +152,14 @@ class GcnTrainer:
 
     # -- the iteration --------------------------------------------------------------------------
     def forward(self):
+        d0 = self.descs[0]
+        reuse = self.cache_first_aggregation and self._first_aggregation_valid and self.orders[0] == mg.ORDER_AGG_FIRST
+        d0.flags = (d0.flags | mg.LAYER_SAVED_IS_VALID) if reuse else (d0.flags & ~mg.LAYER_SAVED_IS_VALID)
         for l in range(self.L):
             mg.layer_fwd(self.ctx, self.g, self.descs[l], self.X[l], self.W[l], self.b[l], self.masks[l],
                          self.saved[l], self.X[l + 1])
+        # saved[0] now holds A_hat X^(0) unless the single layer of a one-layer model also restricted it to train rows
+        self._first_aggregation_valid = self.orders[0] == mg.ORDER_AGG_FIRST and not (d0.flags & mg.LAYER_OUT_ROWS_ONLY)
 
     def compute_loss(self):
         if self.train_rows_only:

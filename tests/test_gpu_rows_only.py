@@ -196,3 +196,51 @@ def test_train_rows_only_needs_row_sparse_backward(mg, ctx):
     tr.set_params(Ws, bs)
     with pytest.raises(ValueError):
         tr.set_inputs(padded(X), y.cuda(), m.cuda())
+
+
+def test_cached_first_aggregation_matches_oracle_and_skips_the_call(mg):
+    """Opt-in: A_hat X^(0) of the first layer is kept across iterations (features and graph do not
+    change); every epoch still matches the oracle, which recomputes it."""
+    from paper_2501_01951_b200.train import GcnTrainer
+    c2 = mg.ctx_create(0)
+    wl, s, d, X, y, m, Ws, bs = _tiny_problem()
+    go = orc.graph_build(wl.n, s.numpy(), d.numpy())
+    gg = mg.graph_create(c2, wl.n, s, d)
+    tr = GcnTrainer(c2, gg, wl.dims, mg.PREC_FP32, order=mg.ORDER_AGG_FIRST, cache_first_aggregation=True)
+    tr.set_params(Ws, bs)
+    tr.set_inputs(padded(X), y.cuda(), m.cuda())
+    Wo, bo, state = [w.numpy() for w in Ws], [b.numpy() for b in bs], None
+    mg.ctx_profile_enable(c2, True)
+    spmm_launches = []
+    for t in (1, 2, 3):
+        mg.ctx_profile_read(c2)
+        tr.forward()
+        _, launches, _ = mg.ctx_profile_read(c2)
+        spmm_launches.append(launches["spmm"])
+        tr.compute_loss(); tr.backward(); tr.step(t, **ADAM)
+        ref = orc.train_epoch(go, X.numpy(), Wo, bo, y.numpy(), m.numpy(), state, t, **ADAM)
+        assert abs(tr.loss.item() - ref["loss"]) <= 1e-5 * abs(ref["loss"])
+        for l in range(tr.L):
+            assert rel_fro(tr.dW[l].cpu().numpy(), ref["dW"][l]) <= TOL_FP32
+            assert rel_fro(tr.db[l].cpu().numpy(), ref["db"][l]) <= TOL_FP32
+        Wo, bo, state = ref["W"], ref["b"], ref["state"]
+        tr.W = [torch.tensor(w, dtype=torch.float32, device="cuda") for w in Wo]
+        tr.b = [torch.tensor(b, dtype=torch.float32, device="cuda") for b in bo]
+        for l in range(tr.L):
+            tr.mW[l].copy_(torch.tensor(state["mW"][l])); tr.vW[l].copy_(torch.tensor(state["vW"][l]))
+            tr.mb[l].copy_(torch.tensor(state["mb"][l])); tr.vb[l].copy_(torch.tensor(state["vb"][l]))
+    mg.ctx_profile_enable(c2, False)
+    assert spmm_launches[1] == spmm_launches[2] < spmm_launches[0]   # one aggregation fewer from the second epoch on
+    # new inputs invalidate the cached product
+    X2 = synth.normal_features(wl.n, wl.dims[0], 4242)
+    tr.set_inputs(padded(X2), y.cuda(), m.cuda())
+    tr.forward()
+    want = orc.aggregate(go, X2.numpy())
+    assert rel_fro(host(tr.saved[0], wl.dims[0]), want) <= TOL_FP32
+    # the flag is refused where `saved` would not survive the backward pass
+    desc = mg.layer_desc(8, 8, 8, 8, 8, mg.ORDER_AGG_FIRST, mg.PREC_FP32, mg.LAYER_SAVED_IS_VALID)
+    Z = torch.zeros(wl.n, 8, device="cuda"); W = torch.zeros(8, 8, device="cuda")
+    with pytest.raises(mg.MixgcnError):
+        mg.layer_fwd(c2, gg, desc, Z, W, None, None, Z.clone(), Z.clone())
+    assert mg.ctx_poll_status(c2, raise_on_error=False) == 0
+    gg.close(); c2.close()
