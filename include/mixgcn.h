@@ -369,6 +369,8 @@ mixgcn_status mixgcn_adam_step(mixgcn_ctx* ctx, int32_t n_tensors, float* const*
  * (nullable) host int32[n].  Uses AUTO ordering, ReLU on all layers but the last, no dropout.
  * When pred is NULL and the backward pass runs row-sparse, the last layer, the loss and its
  * gradient are computed on the train rows alone (nothing returned depends on the other rows).
+ * The row plans of the backward pass are kept in the context and reused by the next call while the
+ * graph and the train mask are unchanged (the mask is compared on the device every call).
  * Device buffers are taken from the context workspace (grown on demand).  Synchronises. */
 mixgcn_status mixgcn_train_step_host(mixgcn_ctx* ctx, const mixgcn_graph* g, int32_t L,
                                      const int32_t* dims, int32_t precision, const float* X,

@@ -156,6 +156,7 @@ extern "C" mixgcn_status mixgcn_ctx_destroy(mixgcn_ctx* ctx) {
     for (int i = 0; i < 64; ++i) if (ctx->chunk_ev[i]) cudaEventDestroy(ctx->chunk_ev[i]);
     for (int i = 0; i < 2; ++i) { if (ctx->join_ev[i]) cudaEventDestroy(ctx->join_ev[i]); if (ctx->side_stream[i]) cudaStreamDestroy(ctx->side_stream[i]); }
     if (ctx->fork_ev) cudaEventDestroy(ctx->fork_ev);
+    free_step_cache(ctx);
     cudaFree(ctx->workspace);
     cudaFree(ctx->workspace_spmm);
     cudaFree(ctx->workspace_rows);
@@ -312,7 +313,9 @@ extern "C" mixgcn_status mixgcn_layer_fwd(mixgcn_ctx* ctx, const mixgcn_graph* g
         // update then runs on the compacted rows and its result is scattered back.
         const uint8_t* rows = d->gout_row_mask;
         const int64_t cnt = d->gout_row_count;
-        if (!rows || cnt <= 0 || cnt > n) MIXGCN_FAIL(MIXGCN_EINVAL, "layer_fwd: OUT_ROWS_ONLY needs gout_row_mask and its exact count");
+        if (!rows || cnt <= 0 || cnt > n)
+            MIXGCN_FAIL(MIXGCN_EINVAL, "layer_fwd: OUT_ROWS_ONLY needs gout_row_mask and its exact count (mask %s, count %lld, n %lld)",
+                        rows ? "given" : "null", (long long)cnt, (long long)n);
         if (drop_mask) MIXGCN_FAIL(MIXGCN_EUNSUPPORTED, "layer_fwd: OUT_ROWS_ONLY does not take a dropout mask");
         if (order == MIXGCN_ORDER_AGG_FIRST) {
             if (!saved_valid)

@@ -10,7 +10,14 @@
 
 using namespace mixgcn;
 
+#include <atomic>
+
 namespace {
+
+uint64_t next_graph_uid() {
+    static std::atomic<uint64_t> counter{0};
+    return ++counter;
+}
 
 constexpr int TPB = 256;
 inline unsigned blocks_for(int64_t n) { return (unsigned)((n + TPB - 1) / TPB); }
@@ -482,6 +489,7 @@ extern "C" mixgcn_status mixgcn_graph_create(mixgcn_ctx* ctx, int64_t n, int64_t
     const int64_t total = m * (sym ? 2 : 1) + (self ? n : 0);
 
     mixgcn_graph* g = new (std::nothrow) mixgcn_graph();
+    if (g) g->uid = next_graph_uid();
     if (!g) MIXGCN_FAIL(MIXGCN_ENOMEM, "graph_create: host allocation failed");
     g->ctx = ctx; g->n = n; g->nnz = 0; g->symmetric = 1;
     struct Guard { mixgcn_graph* g; bool keep = false; ~Guard() { if (!keep) { g->symmetric = g->bwd.rowptr == g->fwd.rowptr; mixgcn_graph_destroy(g); } } } guard{g};
@@ -558,6 +566,7 @@ extern "C" mixgcn_status mixgcn_graph_create_from_csr(mixgcn_ctx* ctx, int64_t n
     if (nnz > 0 && !col) MIXGCN_FAIL(MIXGCN_EINVAL, "graph_create_from_csr: null col");
 
     mixgcn_graph* g = new (std::nothrow) mixgcn_graph();
+    if (g) g->uid = next_graph_uid();
     if (!g) MIXGCN_FAIL(MIXGCN_ENOMEM, "graph_create_from_csr: host allocation failed");
     g->ctx = ctx; g->n = n; g->nnz = nnz; g->symmetric = 1;
     struct Guard { mixgcn_graph* g; bool keep = false; ~Guard() { if (!keep) { g->symmetric = g->bwd.rowptr == g->fwd.rowptr; mixgcn_graph_destroy(g); } } } guard{g};

@@ -1,13 +1,37 @@
 // One whole training iteration (the loop body of Algorithm 2) with host inputs and outputs:
 // host -> device copies, all layers forward, loss, backward, Adam, device -> host copies.
 // Device buffers come from an arena the context keeps between calls.
+#include <new>
 #include <vector>
 
 #include "internal.cuh"
 
 using namespace mixgcn;
 
+// Row plans depend on the graph and the train mask only; a training loop calls with the same ones
+// every iteration, so the plans of the last call are kept and reused while both are unchanged (the
+// mask is compared byte by byte on the device).
+struct HostStepCache {
+    uint64_t graph_uid = 0;
+    int64_t n = 0;
+    int levels = 0;
+    uint8_t* mask = nullptr;            // device copy of the train mask the plans were made from
+    mixgcn_rowplan* plan[2] = {nullptr, nullptr};
+};
+
 namespace {
+
+__global__ void mask_differs_kernel(int64_t n, const uint8_t* __restrict__ a, const uint8_t* __restrict__ b, int32_t* differs) {
+    bool d = false;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
+        d |= (a[i] != 0) != (b[i] != 0);
+    if (__any_sync(0xFFFFFFFFu, d) && (threadIdx.x & 31) == 0) *differs = 1;
+}
+
+void drop_plans(HostStepCache* c) {
+    for (int i = 0; i < 2; ++i) { if (c->plan[i]) mixgcn_rowplan_destroy(c->plan[i]); c->plan[i] = nullptr; }
+    c->graph_uid = 0; c->levels = 0;
+}
 
 inline int64_t round4(int64_t x) { return (x + 3) / 4 * 4; }
 
@@ -70,6 +94,17 @@ mixgcn_status lay_out(char* base, int64_t n, int L, const int32_t* dims, int pre
 
 }  // namespace
 
+namespace mixgcn {
+void free_step_cache(mixgcn_ctx* ctx) {
+    HostStepCache* c = ctx->step_cache;
+    if (!c) return;
+    drop_plans(c);
+    cudaFree(c->mask);
+    delete c;
+    ctx->step_cache = nullptr;
+}
+}  // namespace mixgcn
+
 extern "C" mixgcn_status mixgcn_train_step_host(mixgcn_ctx* ctx, const mixgcn_graph* g, int32_t L,
                                                 const int32_t* dims, int32_t precision, const float* X,
                                                 const int32_t* labels, const uint8_t* train_mask,
@@ -100,38 +135,74 @@ extern "C" mixgcn_status mixgcn_train_step_host(mixgcn_ctx* ctx, const mixgcn_gr
         }
         ctx->arena = p; ctx->arena_bytes = lo.bytes;
         MIXGCN_CUDA(cudaMemset(p, 0, (size_t)lo.bytes));
+        MIXGCN_CUDA(cudaDeviceSynchronize());   // the copies below run on a non-blocking stream: the clear must have finished
     }
     MIXGCN_TRY(lay_out(reinterpret_cast<char*>(ctx->arena), n, L, dims, precision, lo));
+    cudaStream_t s = ctx->side_stream[0];
+    const cudaMemcpyKind H2D = cudaMemcpyHostToDevice, D2H = cudaMemcpyDeviceToHost;
+
     // Row sparsity of the backward pass: the loss gradient is non-zero on train rows only, and one
-    // aggregation later on their neighbours only (same rule as the device-buffer trainer).
+    // aggregation later on their neighbours only (same rule as the device-buffer trainer).  The row
+    // plans are kept between calls and reused while the graph and the mask are the same.
     int64_t n_train = 0;
     for (int64_t i = 0; i < n; ++i) n_train += train_mask[i] ? 1 : 0;
     bool rows_only = false;
+    MIXGCN_CUDA(cudaMemcpyAsync(lo.mask, train_mask, n * sizeof(uint8_t), H2D, s));
     {
         const double frac = (double)n_train / (double)n, mean_entries = (double)g->nnz / (double)n;
         int levels = frac >= 0.25 ? 0 : (frac * mean_entries < 0.5 ? 2 : 1);
         if (levels > L) levels = L;
-        const uint8_t* in_mask = lo.mask;
-        for (int i = 0; i < levels; ++i) {
-            const int l = L - 1 - i;
-            lo.desc[l].gout_row_mask = in_mask;
-            lo.desc[l].gout_row_count = i == 0 ? n_train : 0;
-            if (l > 0 && i + 1 < levels) { lo.desc[l].gin_row_mask = lo.rowmask[l]; in_mask = lo.rowmask[l]; }
+        if (n_train == 0) levels = 0;
+        if (levels > 0) {
+            if (!ctx->step_cache) ctx->step_cache = new (std::nothrow) HostStepCache();
+            HostStepCache* c = ctx->step_cache;
+            if (!c) MIXGCN_FAIL(MIXGCN_ENOMEM, "train_step_host: host allocation failed");
+            bool reuse = c->graph_uid == g->uid && c->n == n && c->levels == levels && c->mask;
+            if (reuse) {
+                int32_t* flag = reinterpret_cast<int32_t*>(lo.loss) + 1;      // spare words beside the loss scalar
+                int32_t differs = 0;
+                MIXGCN_CUDA(cudaMemsetAsync(flag, 0, sizeof(int32_t), s));
+                mask_differs_kernel<<<(unsigned)(ctx->sm_count * 8), 256, 0, s>>>(n, lo.mask, c->mask, flag);
+                MIXGCN_CUDA(cudaMemcpyAsync(&differs, flag, sizeof(int32_t), D2H, s));
+                MIXGCN_CUDA(cudaStreamSynchronize(s));
+                reuse = differs == 0;
+            }
+            if (!reuse) {
+                drop_plans(c);
+                if (c->n != n) { cudaFree(c->mask); c->mask = nullptr; c->n = 0; }
+                if (!c->mask) { MIXGCN_CUDA(cudaMalloc((void**)&c->mask, (size_t)n)); c->n = n; }
+                MIXGCN_CUDA(cudaStreamSynchronize(s));
+                const uint8_t* in_mask = lo.mask;
+                for (int i = 0; i < levels; ++i) {
+                    MIXGCN_TRY(mixgcn_rowplan_create(ctx, g, 1, in_mask, &c->plan[i]));
+                    if (i + 1 < levels) {
+                        MIXGCN_TRY(mixgcn_rowplan_export(c->plan[i], nullptr, lo.rowmask[L - 1 - i], s));
+                        MIXGCN_CUDA(cudaStreamSynchronize(s));
+                        in_mask = lo.rowmask[L - 1 - i];
+                    }
+                }
+                MIXGCN_CUDA(cudaMemcpyAsync(c->mask, lo.mask, (size_t)n, cudaMemcpyDeviceToDevice, s));
+                c->graph_uid = g->uid; c->levels = levels;
+            }
+            for (int i = 0; i < levels; ++i) {
+                const int l = L - 1 - i;
+                lo.desc[l].gout_plan = c->plan[i];
+                lo.desc[l].gout_row_mask = i == 0 ? lo.mask : nullptr;      // the forward's OUT_ROWS_ONLY reads it
+                lo.desc[l].gout_row_count = c->plan[i]->in_count;
+                if (l > 0 && i + 1 < levels) lo.desc[l].flags |= MIXGCN_LAYER_GIN_ROWS_ONLY;
+            }
         }
         // Without `pred` nothing this call returns depends on the last layer's output outside the train
         // rows: compute that layer, the loss and its gradient on the train rows alone.
         rows_only = !pred && levels >= 1 && n_train > 0;
         if (rows_only) lo.desc[L - 1].flags |= MIXGCN_LAYER_OUT_ROWS_ONLY;
     }
-    cudaStream_t s = ctx->side_stream[0];
-    const cudaMemcpyKind H2D = cudaMemcpyHostToDevice, D2H = cudaMemcpyDeviceToHost;
 
     // inputs
     const int64_t d0 = dims[0], ld0 = round4(d0);
     if (ld0 == d0) MIXGCN_CUDA(cudaMemcpyAsync(lo.X[0], X, (size_t)(n * d0) * sizeof(float), H2D, s));
     else MIXGCN_CUDA(cudaMemcpy2DAsync(lo.X[0], ld0 * sizeof(float), X, d0 * sizeof(float), d0 * sizeof(float), (size_t)n, H2D, s));
     MIXGCN_CUDA(cudaMemcpyAsync(lo.labels, labels, n * sizeof(int32_t), H2D, s));
-    MIXGCN_CUDA(cudaMemcpyAsync(lo.mask, train_mask, n * sizeof(uint8_t), H2D, s));
     for (int l = 0; l < L; ++l) {
         const size_t wb = (size_t)dims[l] * dims[l + 1] * sizeof(float), bb = (size_t)dims[l + 1] * sizeof(float);
         MIXGCN_CUDA(cudaMemcpyAsync(lo.W[l], W[l], wb, H2D, s));
@@ -153,12 +224,6 @@ extern "C" mixgcn_status mixgcn_train_step_host(mixgcn_ctx* ctx, const mixgcn_gr
         MIXGCN_TRY(st);
     }
     for (int l = L - 1; l >= 0; --l) {
-        if (lo.desc[l].gout_row_mask && lo.desc[l].gout_row_count == 0 && l < L - 1) {
-            // the mask the layer above reported: with its count the dense products run on compacted rows
-            int64_t cnt = 0;
-            MIXGCN_TRY(mixgcn_count_rows(ctx, n, lo.desc[l].gout_row_mask, &cnt, s));
-            lo.desc[l].gout_row_count = cnt;
-        }
         MIXGCN_TRY(mixgcn_layer_bwd(ctx, g, &lo.desc[l], lo.X[l], lo.saved[l], lo.X[l + 1], nullptr, lo.W[l], lo.G[l + 1],
                                     l > 0 ? lo.G[l] : nullptr, lo.dW[l], lo.db[l], s));
     }

@@ -68,6 +68,8 @@ struct mixgcn_ctx {
     // device arena of mixgcn_train_step_host (activations, parameters, gradients), grown on demand
     void* arena;
     int64_t arena_bytes;
+    // row plans of the last mixgcn_train_step_host call, reused while graph and train mask stay the same
+    struct HostStepCache* step_cache;
 };
 
 // One unit of aggregation work: `len` stored entries starting at `begin`.  For an ordinary row `row`
@@ -108,6 +110,7 @@ struct CsrView {
 
 struct mixgcn_graph {
     mixgcn_ctx* ctx;
+    uint64_t uid;      // unique per created graph (a freed graph's address may be reused)
     int64_t n, nnz;
     int symmetric;
     int has_diagonal;  // 1: every row stores its diagonal entry, 0: none does, 2: some do
@@ -205,6 +208,7 @@ mixgcn_status launch_gather_rows(mixgcn_ctx* ctx, int64_t count, int32_t d, cons
                                  int64_t ld_src, float* dst, int64_t ld_dst, cudaStream_t s);
 
 mixgcn_status ensure_workspace_rows(mixgcn_ctx* ctx, int64_t bytes);
+void free_step_cache(mixgcn_ctx* ctx);
 // dst[idx[i], :] = src[i, :] for i < count (the inverse of launch_gather_rows)
 mixgcn_status launch_scatter_rows(mixgcn_ctx* ctx, int64_t count, int32_t d, const int32_t* idx, const float* src,
                                   int64_t ld_src, float* dst, int64_t ld_dst, cudaStream_t s);

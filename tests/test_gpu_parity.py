@@ -793,6 +793,31 @@ def test_train_step_host_row_sparse_matches_oracle(mg, ctx, with_pred):
     assert mg.ctx_poll_status(ctx, raise_on_error=False) == 0
 
 
+def test_train_step_host_reuses_and_rebuilds_its_row_plans(mg):
+    """Same graph and mask: the second call reuses the plans of the first.  A changed mask, or another
+    graph, must rebuild them -- every call matches the oracle for its own inputs."""
+    c2 = mg.ctx_create(0)
+    wl, s, d, X, y, m, Ws, bs = _tiny_problem()
+    masks = [synth.bernoulli_mask(wl.n, 0.02, 88), synth.bernoulli_mask(wl.n, 0.02, 88), synth.bernoulli_mask(wl.n, 0.03, 89)]
+    gg = mg.graph_create(c2, wl.n, s, d)
+    go = orc.graph_build(wl.n, s.numpy(), d.numpy())
+    s2, d2 = synth.rmat_graph(wl.n, wl.undirected_edges, 999)
+    graphs = [(gg, go)] * 3 + [(mg.graph_create(c2, wl.n, s2, d2), orc.graph_build(wl.n, s2.numpy(), d2.numpy()))]
+    masks.append(masks[2])
+    for (g_gpu, g_orc), mask in zip(graphs, masks):
+        W = [w.clone() for w in Ws]; b = [x.clone() for x in bs]
+        z = lambda lst: [torch.zeros_like(x) for x in lst]
+        mW, vW, mb, vb = z(W), z(W), z(b), z(b)
+        loss = mg.train_step_host(c2, g_gpu, wl.dims, mg.PREC_FP32, X, y, mask, W, b, mW, vW, mb, vb, 1, **ADAM)
+        ref = orc.train_epoch(g_orc, X.numpy(), [w.numpy() for w in Ws], [x.numpy() for x in bs], y.numpy(), mask.numpy(), None, 1, **ADAM)
+        assert abs(loss - ref["loss"]) <= 1e-5 * abs(ref["loss"])
+        for l in range(len(W)):
+            assert rel_fro(mW[l].numpy() / (1 - ADAM["beta1"]), ref["dW"][l]) <= 2e-5
+            assert rel_fro(mb[l].numpy() / (1 - ADAM["beta1"]), ref["db"][l]) <= 2e-5
+    assert mg.ctx_poll_status(c2, raise_on_error=False) == 0
+    c2.close()
+
+
 def test_graph_size_limits_are_checked_on_the_host(mg, ctx):
     e = i32([])
     with pytest.raises(mg.MixgcnError) as ex:
