@@ -75,7 +75,9 @@ mixgcn_status mixgcn_ctx_poll_status(mixgcn_ctx* ctx, int32_t* code);
  * outside the train mask are not looked at: their logits are not read, their dlogits rows are
  * left UNCHANGED (not zeroed) and pred, if given, receives -1 there.  Loss, n_correct and the
  * train rows of dlogits are unchanged.  For use with MIXGCN_LAYER_OUT_ROWS_ONLY and a row-sparse
- * backward pass, which read train rows only. */
+ * backward pass, which read train rows only.  2 = every row's logits are read (pred for all nodes) but
+ * the dlogits rows of non-train nodes are left UNCHANGED instead of zeroed: for a backward pass that
+ * reads train rows only (gout_plan, or gout_row_mask with a count below n/4 in agg-first order). */
 #define MIXGCN_OPT_LOSS_TRAIN_ROWS_ONLY 2
 mixgcn_status mixgcn_ctx_set_option(mixgcn_ctx* ctx, int32_t option, int64_t value);
 
@@ -130,6 +132,7 @@ mixgcn_status mixgcn_graph_export(const mixgcn_graph* g, int transposed, int64_t
  * entry count (ties by ascending id). */
 mixgcn_status mixgcn_graph_export_schedule(const mixgcn_graph* g, int transposed, int32_t* perm);
 
+/* A graph may be used only while its context exists; it may be destroyed after it. */
 mixgcn_status mixgcn_graph_destroy(mixgcn_graph* g);
 
 /* Node reordering for the fine-grain pipeline (Section 3.2.2).

@@ -194,7 +194,7 @@ extern "C" mixgcn_status mixgcn_ctx_set_option(mixgcn_ctx* ctx, int32_t option, 
         return MIXGCN_OK;
     }
     if (option == MIXGCN_OPT_LOSS_TRAIN_ROWS_ONLY) {
-        if (value != 0 && value != 1) MIXGCN_FAIL(MIXGCN_EINVAL, "ctx_set_option: loss rows option takes 0 or 1 (got %lld)", (long long)value);
+        if (value < 0 || value > 2) MIXGCN_FAIL(MIXGCN_EINVAL, "ctx_set_option: loss rows option takes 0, 1 or 2 (got %lld)", (long long)value);
         ctx->loss_train_rows_only = (int)value;
         return MIXGCN_OK;
     }

@@ -470,7 +470,7 @@ mixgcn_status ensure_chunk_schedules(const mixgcn_graph* g, const CsrView& A_con
 
 extern "C" mixgcn_status mixgcn_graph_destroy(mixgcn_graph* g) {
     if (!g) return MIXGCN_OK;
-    cudaSetDevice(g->ctx->device);
+    cudaSetDevice(g->device);
     if (!g->symmetric) free_view(g->bwd);
     free_view(g->fwd);
     cudaFree(g->deg);
@@ -491,7 +491,7 @@ extern "C" mixgcn_status mixgcn_graph_create(mixgcn_ctx* ctx, int64_t n, int64_t
     mixgcn_graph* g = new (std::nothrow) mixgcn_graph();
     if (g) g->uid = next_graph_uid();
     if (!g) MIXGCN_FAIL(MIXGCN_ENOMEM, "graph_create: host allocation failed");
-    g->ctx = ctx; g->n = n; g->nnz = 0; g->symmetric = 1;
+    g->ctx = ctx; g->device = ctx->device; g->n = n; g->nnz = 0; g->symmetric = 1;
     struct Guard { mixgcn_graph* g; bool keep = false; ~Guard() { if (!keep) { g->symmetric = g->bwd.rowptr == g->fwd.rowptr; mixgcn_graph_destroy(g); } } } guard{g};
     LaunchScope scope(ctx, PH_GRAPH, s, 12);
 
@@ -568,7 +568,7 @@ extern "C" mixgcn_status mixgcn_graph_create_from_csr(mixgcn_ctx* ctx, int64_t n
     mixgcn_graph* g = new (std::nothrow) mixgcn_graph();
     if (g) g->uid = next_graph_uid();
     if (!g) MIXGCN_FAIL(MIXGCN_ENOMEM, "graph_create_from_csr: host allocation failed");
-    g->ctx = ctx; g->n = n; g->nnz = nnz; g->symmetric = 1;
+    g->ctx = ctx; g->device = ctx->device; g->n = n; g->nnz = nnz; g->symmetric = 1;
     struct Guard { mixgcn_graph* g; bool keep = false; ~Guard() { if (!keep) { g->symmetric = g->bwd.rowptr == g->fwd.rowptr; mixgcn_graph_destroy(g); } } } guard{g};
     LaunchScope scope(ctx, PH_GRAPH, s, 8);
     DevBuf fl;

@@ -111,6 +111,7 @@ struct CsrView {
 struct mixgcn_graph {
     mixgcn_ctx* ctx;
     uint64_t uid;      // unique per created graph (a freed graph's address may be reused)
+    int device;        // kept apart from ctx: a graph may be destroyed after its context
     int64_t n, nnz;
     int symmetric;
     int has_diagonal;  // 1: every row stores its diagonal entry, 0: none does, 2: some do

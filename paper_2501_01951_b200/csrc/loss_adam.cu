@@ -30,7 +30,7 @@ __global__ void count_mask_kernel(int64_t n, const uint8_t* __restrict__ mask, u
 __global__ void __launch_bounds__(LOSS_WARPS * 32) loss_rows_kernel(
     int64_t n, int C, const float* logits, int64_t ld, const int32_t* __restrict__ labels,
     const uint8_t* __restrict__ mask, const unsigned long long* __restrict__ count, float* dlogits,
-    int32_t* __restrict__ pred, unsigned long long* n_correct, double* __restrict__ part, int32_t* status) {
+    int32_t* __restrict__ pred, unsigned long long* n_correct, double* __restrict__ part, int32_t* status, bool zero_rows) {
     __shared__ double sm[LOSS_WARPS];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const unsigned long long T = *count;
@@ -63,7 +63,7 @@ __global__ void __launch_bounds__(LOSS_WARPS * 32) loss_rows_kernel(
             if (!ok && lane == 0) atomicMax(status, DEV_BAD_LABEL);
         }
         if (!train || !ok) {
-            if (dlogits) for (int c = lane; c < C; c += 32) dlogits[v * ld + c] = 0.0f;
+            if (dlogits && (zero_rows || train)) for (int c = lane; c < C; c += 32) dlogits[v * ld + c] = 0.0f;
             continue;
         }
         float s = 0.0f;
@@ -96,7 +96,7 @@ template <int VPL>
 __global__ void __launch_bounds__(LOSS_WARPS * 32) loss_rows_vec_kernel(
     int64_t n, int C, const float* logits, int64_t ld, const int32_t* __restrict__ labels,
     const uint8_t* __restrict__ mask, const unsigned long long* __restrict__ count, float* dlogits,
-    int32_t* __restrict__ pred, unsigned long long* n_correct, double* __restrict__ part, int32_t* status) {
+    int32_t* __restrict__ pred, unsigned long long* n_correct, double* __restrict__ part, int32_t* status, bool zero_rows) {
     __shared__ double sm[LOSS_WARPS];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const unsigned long long T = *count;
@@ -152,7 +152,7 @@ __global__ void __launch_bounds__(LOSS_WARPS * 32) loss_rows_vec_kernel(
         }
         float4* out4 = dlogits ? reinterpret_cast<float4*>(dlogits + v * ld) : nullptr;
         if (!train || !ok) {
-            if (out4) {
+            if (out4 && (zero_rows || train)) {
 #pragma unroll
                 for (int q = 0; q < VPL; ++q) {
                     const int g = lane + 32 * q;
@@ -273,14 +273,14 @@ __global__ void __launch_bounds__(LOSS_WARPS * 32) loss_rows_subset_kernel(
 // Picks the register-resident kernel when the row fits (C <= 256) and the layout allows float4 access.
 void launch_loss_rows(unsigned blocks, cudaStream_t s, int64_t n, int C, const float* logits, int64_t ld,
                       const int32_t* labels, const uint8_t* mask, const unsigned long long* count, float* dlogits,
-                      int32_t* pred, unsigned long long* n_correct, double* part, int32_t* status) {
+                      int32_t* pred, unsigned long long* n_correct, double* part, int32_t* status, bool zero_rows = true) {
     const bool vec = (ld & 3) == 0 && aligned16(logits) && (!dlogits || aligned16(dlogits));
     if (vec && C <= 128)
-        loss_rows_vec_kernel<1><<<blocks, LOSS_WARPS * 32, 0, s>>>(n, C, logits, ld, labels, mask, count, dlogits, pred, n_correct, part, status);
+        loss_rows_vec_kernel<1><<<blocks, LOSS_WARPS * 32, 0, s>>>(n, C, logits, ld, labels, mask, count, dlogits, pred, n_correct, part, status, zero_rows);
     else if (vec && C <= 256)
-        loss_rows_vec_kernel<2><<<blocks, LOSS_WARPS * 32, 0, s>>>(n, C, logits, ld, labels, mask, count, dlogits, pred, n_correct, part, status);
+        loss_rows_vec_kernel<2><<<blocks, LOSS_WARPS * 32, 0, s>>>(n, C, logits, ld, labels, mask, count, dlogits, pred, n_correct, part, status, zero_rows);
     else
-        loss_rows_kernel<<<blocks, LOSS_WARPS * 32, 0, s>>>(n, C, logits, ld, labels, mask, count, dlogits, pred, n_correct, part, status);
+        loss_rows_kernel<<<blocks, LOSS_WARPS * 32, 0, s>>>(n, C, logits, ld, labels, mask, count, dlogits, pred, n_correct, part, status, zero_rows);
 }
 
 __global__ void loss_final_kernel(int blocks, const double* __restrict__ part,
@@ -347,12 +347,12 @@ extern "C" mixgcn_status mixgcn_loss_softmax_xent(mixgcn_ctx* ctx, int64_t n, in
     }
     {
         LaunchScope scope(ctx, PH_LOSS, s);
-        if (ctx->loss_train_rows_only)
+        if (ctx->loss_train_rows_only == 1)
             loss_rows_subset_kernel<<<(unsigned)blocks, LOSS_WARPS * 32, 0, s>>>(n, C, logits, ld, labels, train_mask, count, dlogits, pred,
                                                                               reinterpret_cast<unsigned long long*>(n_correct), part, ctx->d_status);
         else
             launch_loss_rows((unsigned)blocks, s, n, C, logits, ld, labels, train_mask, count, dlogits, pred,
-                             reinterpret_cast<unsigned long long*>(n_correct), part, ctx->d_status);
+                             reinterpret_cast<unsigned long long*>(n_correct), part, ctx->d_status, ctx->loss_train_rows_only != 2);
     }
     {
         LaunchScope scope(ctx, PH_LOSS, s);

@@ -170,6 +170,16 @@ class GcnTrainer:
             finally:
                 mg.ctx_set_option(self.ctx, mg.OPT_LOSS_TRAIN_ROWS_ONLY, 0)
             return
+        if self.row_plans[self.L - 1] is not None:
+            # the last layer's backward reads the plan's (train) rows of the gradient only: no need to
+            # write zeros into the other rows; the logits of every node are still read for `pred`
+            mg.ctx_set_option(self.ctx, mg.OPT_LOSS_TRAIN_ROWS_ONLY, 2)
+            try:
+                mg.loss_softmax_xent(self.ctx, self.X[self.L], self.labels, self.train_mask, self.loss,
+                                     dlogits=self.X[self.L], pred=self.pred, n_correct=self.n_correct, C_=self.dims[-1])
+            finally:
+                mg.ctx_set_option(self.ctx, mg.OPT_LOSS_TRAIN_ROWS_ONLY, 0)
+            return
         mg.loss_softmax_xent(self.ctx, self.X[self.L], self.labels, self.train_mask, self.loss,
                              dlogits=self.X[self.L], pred=self.pred, n_correct=self.n_correct, C_=self.dims[-1])
 

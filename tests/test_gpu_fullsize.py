@@ -152,6 +152,8 @@ def test_full_size_workload(mg, key):
     labels_train = tr.labels[train_idx].cpu().numpy()
     lo, Gt, pred_t, nc, T = orc.loss(logits_train, labels_train, np.ones(len(labels_train), np.uint8))
     logits_rows = rows_of(tr.X[L], rows, C)
+    untrained = torch.nonzero(tr.train_mask == 0).flatten()[:1000]
+    logits_untrained = tr.X[L][untrained].clone()
     tr.compute_loss()
     torch.cuda.synchronize()
     assert abs(tr.loss.item() - lo) <= 2e-6 * abs(lo)
@@ -161,8 +163,10 @@ def test_full_size_workload(mg, key):
     pick = np.random.default_rng(2).integers(0, len(train_idx), 64)
     got = tr.X[L][train_idx[torch.as_tensor(pick, device="cuda")]][:, :C].cpu().numpy()
     assert _rel(got, Gt[pick]) <= TOL_FP32
-    untrained = torch.nonzero(tr.train_mask == 0).flatten()[:1000]
-    assert float(tr.X[L][untrained][:, :C].abs().max()) == 0.0
+    if tr.row_plans[L - 1] is None:
+        assert float(tr.X[L][untrained][:, :C].abs().max()) == 0.0      # zero gradient outside the train mask
+    else:
+        assert torch.equal(tr.X[L][untrained], logits_untrained)          # rows the row-plan backward never reads are left alone
 
     # ---- backward of the last layer: dW, db probed with random vectors; input gradient on sampled rows
     l = L - 1
@@ -172,19 +176,26 @@ def test_full_size_workload(mg, key):
     a = torch.as_tensor(rng.standard_normal(d_in), device="cuda", dtype=torch.float64)
     bv = torch.as_tensor(rng.standard_normal(d_out), device="cuda", dtype=torch.float64)
 
-    def probe(lhs, rhs):
+    # The gradient w.r.t. the logits is defined as zero outside the train mask; with a row plan the
+    # library leaves those rows of the buffer alone (they are never read), so the checks apply the mask.
+    train_f = tr.train_mask.double()
+
+    def probe(lhs, rhs, rhs_is_dlogits=False):
         """a^T (lhs^T rhs) b = sum_k (lhs a)_k (rhs b)_k and 1^T rhs b, in fp64 by chunks (torch, not this library)."""
         val, colsum, scale = 0.0, 0.0, 0.0
         step = 1 << 20
         for r0 in range(0, n, step):
             za = lhs[r0:r0 + step, :d_in].double() @ a
             gb = rhs[r0:r0 + step, :d_out].double() @ bv
+            if rhs_is_dlogits:
+                gb = gb * train_f[r0:r0 + step]
             val += float(za @ gb); scale += float(za.abs() @ gb.abs()); colsum += float(gb.sum())
         return val, colsum, scale
 
     dP_nodes = rows_of(tr.G[L], nodes, d_out)                      # gradient w.r.t. the logits, rows the sample needs
+    dP_nodes = dP_nodes * tr.train_mask[torch.as_tensor(nodes, device="cuda")].cpu().numpy()[:, None]
     if agg_first:
-        want_probe, want_db, scale = probe(tr.saved[l], tr.G[L])    # before the call: it consumes `saved`
+        want_probe, want_db, scale = probe(tr.saved[l], tr.G[L], True)    # before the call: it consumes `saved`
     tr.backward()
     torch.cuda.synchronize()
     assert mg.ctx_poll_status(ctx, raise_on_error=False) == 0
@@ -199,7 +210,7 @@ def test_full_size_workload(mg, key):
         want_dq = orc.aggregate_rows(sub, dP_nodes, crow)
         assert _rel(rows_of(tr.saved[l], rows, d_out), want_dq) <= TOL_FP32
         want_probe, _, scale = probe(tr.X[l], tr.saved[l])
-        _, want_db, _ = probe(tr.X[l], tr.G[L])
+        _, want_db, _ = probe(tr.X[l], tr.G[L], True)
         assert _rel(rows_of(tr.G[l], rows, d_in), orc.update(rows_of(tr.saved[l], rows, d_out), Wt) * gate) <= tol
     assert abs(float(a @ tr.dW[l].double() @ bv) - want_probe) <= tol * scale
     assert abs(float(tr.db[l].double() @ bv) - want_db) <= tol * scale + 1e-12

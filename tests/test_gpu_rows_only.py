@@ -142,8 +142,16 @@ def test_loss_train_rows_only_option(mg, C):
     mg.ctx_set_option(c2, mg.OPT_LOSS_TRAIN_ROWS_ONLY, 0)
     assert torch.equal(Pa[m.cuda().bool(), :C], d1[m.cuda().bool(), :C])
     assert torch.equal(Pa[~m.cuda().bool()], P[~m.cuda().bool()])
+    # value 2: logits of every row are read (pred everywhere), gradient rows outside the mask left alone
+    mg.ctx_set_option(c2, mg.OPT_LOSS_TRAIN_ROWS_ONLY, 2)
+    loss2 = torch.zeros(1, device="cuda"); d2 = torch.full((n, ld), 3.0, device="cuda")
+    pred2 = torch.zeros(n, dtype=torch.int32, device="cuda"); nc2 = torch.zeros(1, dtype=torch.int64, device="cuda")
+    mg.loss_softmax_xent(c2, P, y.cuda(), m.cuda(), loss2, dlogits=d2, pred=pred2, n_correct=nc2, C_=C)
+    mg.ctx_set_option(c2, mg.OPT_LOSS_TRAIN_ROWS_ONLY, 0)
+    assert loss2.item() == loss0.item() and nc2.item() == nc0.item() and torch.equal(pred2, pred0)
+    assert torch.equal(d2[m.cuda().bool()], d0[m.cuda().bool()]) and np.all(d2.cpu().numpy()[~keep] == 3.0)
     with pytest.raises(mg.MixgcnError):
-        mg.ctx_set_option(c2, mg.OPT_LOSS_TRAIN_ROWS_ONLY, 2)
+        mg.ctx_set_option(c2, mg.OPT_LOSS_TRAIN_ROWS_ONLY, 3)
     assert mg.ctx_poll_status(c2, raise_on_error=False) == 0
     c2.close()
 
