@@ -270,17 +270,220 @@ __global__ void __launch_bounds__(LOSS_WARPS * 32) loss_rows_subset_kernel(
     }
 }
 
-// Picks the register-resident kernel when the row fits (C <= 256) and the layout allows float4 access.
-void launch_loss_rows(unsigned blocks, cudaStream_t s, int64_t n, int C, const float* logits, int64_t ld,
-                      const int32_t* labels, const uint8_t* mask, const unsigned long long* count, float* dlogits,
-                      int32_t* pred, unsigned long long* n_correct, double* part, int32_t* status, bool zero_rows = true) {
+// ---- rows staged through shared memory, four lanes per row ------------------------------------
+// For C up to a few hundred the warp-per-row kernels spend more issue slots on shuffles than on data.
+// Here a CTA takes tiles of ROWS consecutive rows: a tile is one contiguous piece of memory
+// (ROWS x ld floats), fetched by a single bulk-async copy into shared memory while the previous tile
+// is being worked on (two buffers).  Four adjacent lanes own a row, a quarter of its columns each,
+// walked from a lane-dependent starting point so that a warp's 32 lanes spread over the banks; the
+// arg-max keeps the lowest index among equal maxima explicitly, so the order does not matter.  The few
+// train rows are then finished by whole warps (exponentials and gradient stores over 32 lanes).
+constexpr uint32_t LOSS_WAIT_LIMIT = 1u << 22;
+#ifndef MIXGCN_LOSS_TILE_KB
+#define MIXGCN_LOSS_TILE_KB 72
+#endif
+constexpr int LOSS_LANES_PER_ROW = 4;
+
+__device__ __forceinline__ uint32_t loss_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ bool loss_mbar_wait(uint64_t* bar, uint32_t parity) {
+    for (uint32_t it = 0; it < LOSS_WAIT_LIMIT; ++it) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok) : "r"(loss_smem_u32(bar)), "r"(parity) : "memory");
+        if (ok) return true;
+    }
+    return false;
+}
+
+template <int ROWS>
+__global__ void __launch_bounds__(ROWS * LOSS_LANES_PER_ROW) loss_rows_tile_kernel(
+    int64_t n, int C, const float* logits, int64_t ld, const int32_t* __restrict__ labels,
+    const uint8_t* __restrict__ mask, const unsigned long long* __restrict__ count, float* dlogits,
+    int32_t* __restrict__ pred, unsigned long long* n_correct, double* __restrict__ part, int32_t* status,
+    bool zero_rows, int64_t n_tiles) {
+    constexpr int THREADS = ROWS * LOSS_LANES_PER_ROW;
+    extern __shared__ __align__(128) unsigned char loss_smem[];
+    float* const tile0 = reinterpret_cast<float*>(loss_smem);
+    float* const tile1 = tile0 + (int64_t)ROWS * ld;
+    __shared__ __align__(8) uint64_t bar[2];
+    __shared__ double red[THREADS / 32];
+    __shared__ uint8_t keep_row[2][ROWS];      // rows of the tile whose gradient row was written as a train row
+    __shared__ int expired;
+    const int tid = threadIdx.x, lane = tid & 31;
+    const int r_own = tid / LOSS_LANES_PER_ROW, q = tid % LOSS_LANES_PER_ROW;
+    const unsigned long long T = *count;
+    const float invT = T ? (float)(1.0 / (double)T) : 0.0f;
+    const int ld4 = (int)(ld >> 2);
+    const int seg = (C + LOSS_LANES_PER_ROW - 1) / LOSS_LANES_PER_ROW;
+    const int c_lo = q * seg < C ? q * seg : C, c_hi = (q + 1) * seg < C ? (q + 1) * seg : C;
+    if (tid == 0) {
+        expired = 0;
+        for (int b = 0; b < 2; ++b)
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(loss_smem_u32(&bar[b])), "r"(1u) : "memory");
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+    auto issue = [&](int64_t t, int b) {
+        const int64_t row0 = t * ROWS;
+        const int64_t rows = (n - row0) < ROWS ? (n - row0) : ROWS;
+        const uint32_t bytes = (uint32_t)(rows * ld * (int64_t)sizeof(float));    // a multiple of 16: ld % 4 == 0
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(loss_smem_u32(&bar[b])), "r"(bytes) : "memory");
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                     ::"r"(loss_smem_u32(b ? tile1 : tile0)), "l"(reinterpret_cast<uint64_t>(logits + row0 * ld)), "r"(bytes),
+                       "r"(loss_smem_u32(&bar[b])) : "memory");
+    };
+    double local = 0.0;
+    unsigned int correct = 0;
+    uint32_t phase0 = 0u, phase1 = 0u;       // parity to wait for on each buffer's barrier
+    int buf = 0;
+    int64_t t = blockIdx.x;
+    if (tid == 0 && t < n_tiles) issue(t, 0);                       // the first tile; later ones are requested one iteration ahead
+    for (; t < n_tiles; t += gridDim.x, buf ^= 1) {
+        const int64_t row0 = t * ROWS, v = row0 + r_own;
+        // mask byte and label of this thread's row, requested before the wait so that their latency is hidden
+        uint8_t my_mask = 0; int my_y = 0;
+        if (v < n && q == 0) { my_mask = mask[v]; my_y = labels[v]; }
+        if (!loss_mbar_wait(&bar[buf], buf ? phase1 : phase0)) expired = 1;       // bounded: give up instead of hanging
+        if (buf) phase1 ^= 1u; else phase0 ^= 1u;
+        __syncthreads();               // this tile has landed; every thread is done with the previous tile
+        if (expired) {
+            if (tid == 0) atomicMax(status, DEV_WAIT_EXPIRED);         // no other copy is in flight at this point
+            break;
+        }
+        // refill the other buffer (the previous tile's) while this one is worked on
+        if (tid == 0 && t + gridDim.x < n_tiles) issue(t + gridDim.x, buf ^ 1);
+        const int rows = (int)((n - row0) < ROWS ? (n - row0) : ROWS);
+        const float* tile = buf ? tile1 : tile0;
+        const float* row = tile + (int64_t)r_own * ld;
+        float mx = -INFINITY; int arg = 0x7FFFFFFF;
+        if (v < n && c_hi > c_lo) {
+            // two independent (max, index) chains over [start, c_hi) then [c_lo, start): plain counted
+            // loops so that the shared-memory loads are issued ahead of the compares
+            const int start = c_lo + lane % (c_hi - c_lo);
+            float mx2 = -INFINITY; int arg2 = 0x7FFFFFFF;
+            auto scan = [&](int c0, int c1) {
+                int c = c0;
+#pragma unroll 4
+                for (; c + 1 < c1; c += 2) {
+                    const float x = row[c], x2 = row[c + 1];
+                    if (x > mx || (x == mx && c < arg)) { mx = x; arg = c; }
+                    if (x2 > mx2 || (x2 == mx2 && c + 1 < arg2)) { mx2 = x2; arg2 = c + 1; }
+                }
+                if (c < c1) { const float x = row[c]; if (x > mx || (x == mx && c < arg)) { mx = x; arg = c; } }
+            };
+            scan(start, c_hi);
+            scan(c_lo, start);
+            if (mx2 > mx || (mx2 == mx && arg2 < arg)) { mx = mx2; arg = arg2; }
+        }
+        // the four lanes of a row agree on its maximum and the lowest index that attains it
+#pragma unroll
+        for (int o = 1; o < LOSS_LANES_PER_ROW; o <<= 1) {
+            const float omx = __shfl_xor_sync(0xFFFFFFFFu, mx, o);
+            const int oarg = __shfl_xor_sync(0xFFFFFFFFu, arg, o);
+            if (omx > mx || (omx == mx && oarg < arg)) { mx = omx; arg = oarg; }
+        }
+        if (arg == 0x7FFFFFFF) arg = 0;                                // every entry NaN
+        const bool wrote = v < n && q == 0 && my_mask != 0 && T != 0;
+        if (v < n && q == 0 && pred) pred[v] = arg;
+        if (dlogits && zero_rows) {
+            if (q == 0) keep_row[buf][r_own] = wrote ? 1 : 0;
+            __syncthreads();           // keep_row is complete
+            // zero gradient rows of the other nodes, written by the whole CTA in memory order
+            float4* out4 = reinterpret_cast<float4*>(dlogits + row0 * ld);
+            const int total4 = rows * ld4;
+            for (int i = tid; i < total4; i += THREADS) {
+                const int r = i / ld4;
+                if (!keep_row[buf][r]) out4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+        }
+        // train rows (few): the whole warp works on each of them in turn -- lanes stride over the columns
+        unsigned live = __ballot_sync(0xFFFFFFFFu, wrote);
+        while (live) {
+            const int src = __ffs(live) - 1;
+            live &= live - 1;
+            const float r_mx = __shfl_sync(0xFFFFFFFFu, mx, src);
+            const int r_arg = __shfl_sync(0xFFFFFFFFu, arg, src);
+            const int y = __shfl_sync(0xFFFFFFFFu, my_y, src);
+            const int r = ((tid & ~31) + src) / LOSS_LANES_PER_ROW;
+            const float* rr = tile + (int64_t)r * ld;
+            float* out = dlogits ? dlogits + (row0 + r) * ld : nullptr;
+            if (y < 0 || y >= C) {
+                if (lane == 0) atomicMax(status, DEV_BAD_LABEL);
+                if (out) for (int j = lane; j < C; j += 32) out[j] = 0.0f;
+                continue;
+            }
+            float sum = 0.0f;
+            for (int j = lane; j < C; j += 32) sum += expf(rr[j] - r_mx);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xFFFFFFFFu, sum, o);
+            const float lse = r_mx + logf(sum);
+            if (lane == 0) { local += (double)(lse - rr[y]); if (r_arg == y) ++correct; }
+            if (out) for (int j = lane; j < C; j += 32) out[j] = (expf(rr[j] - lse) - (j == y ? 1.0f : 0.0f)) * invT;
+        }
+    }
+    // fixed-order block sum of the per-warp losses
+    for (int o = 16; o > 0; o >>= 1) local += __shfl_down_sync(0xFFFFFFFFu, local, o);
+    for (int o = 16; o > 0; o >>= 1) correct += __shfl_down_sync(0xFFFFFFFFu, correct, o);
+    if (lane == 0) red[tid >> 5] = local;
+    if (n_correct && lane == 0 && correct) atomicAdd(n_correct, (unsigned long long)correct);
+    __syncthreads();
+    if (tid == 0) {
+        double s = 0.0;
+        for (int w = 0; w < THREADS / 32; ++w) s += red[w];
+        part[blockIdx.x] = s;
+    }
+}
+
+template <int ROWS>
+cudaError_t launch_loss_tile(int grid, size_t smem, cudaStream_t s, int64_t n, int C, const float* logits, int64_t ld,
+                             const int32_t* labels, const uint8_t* mask, const unsigned long long* count, float* dlogits,
+                             int32_t* pred, unsigned long long* n_correct, double* part, int32_t* status, bool zero_rows,
+                             int64_t n_tiles) {
+    cudaError_t e = cudaFuncSetAttribute(loss_rows_tile_kernel<ROWS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    loss_rows_tile_kernel<ROWS><<<grid, ROWS * LOSS_LANES_PER_ROW, smem, s>>>(n, C, logits, ld, labels, mask, count, dlogits, pred, n_correct, part,
+                                                         status, zero_rows, n_tiles);
+    return cudaGetLastError();
+}
+
+// Launches the row pass and returns how many block partials it writes to `part` (<= warp_blocks, the
+// capacity the caller sized `part` for), or -1 on a launch error.  With sm_count > 0 and a row that
+// fits, the shared-memory tile kernel (one lane per row) is used; otherwise one warp per row, with
+// the row in registers when C <= 256 and the layout allows float4 access.
+int launch_loss_rows(unsigned warp_blocks, cudaStream_t s, int64_t n, int C, const float* logits, int64_t ld,
+                     const int32_t* labels, const uint8_t* mask, const unsigned long long* count, float* dlogits,
+                     int32_t* pred, unsigned long long* n_correct, double* part, int32_t* status, bool zero_rows = true,
+                     int sm_count = 0) {
     const bool vec = (ld & 3) == 0 && aligned16(logits) && (!dlogits || aligned16(dlogits));
+    // Several CTAs per SM (each with two tile buffers) keep some computing while others wait for their
+    // copies: a CTA takes at most MIXGCN_LOSS_TILE_KB of shared memory; rows per tile follow from that.
+    constexpr int64_t TILE_SMEM = MIXGCN_LOSS_TILE_KB * 1024;
+    if (vec && sm_count > 0 && C >= 8 && 2 * 32 * ld * 4 <= TILE_SMEM) {
+        const int rows = 2 * 128 * ld * 4 <= TILE_SMEM ? 128 : (2 * 64 * ld * 4 <= TILE_SMEM ? 64 : 32);
+        const int64_t n_tiles = (n + rows - 1) / rows;
+        int64_t per_sm = (220 * 1024) / (2 * rows * ld * 4 + 1024);
+        if (per_sm > 2048 / (rows * LOSS_LANES_PER_ROW)) per_sm = 2048 / (rows * LOSS_LANES_PER_ROW);
+        if (per_sm < 1) per_sm = 1;
+        int64_t grid = n_tiles < per_sm * sm_count ? n_tiles : per_sm * sm_count;
+        if (grid > (int64_t)warp_blocks) grid = warp_blocks;
+        const size_t smem = (size_t)(2 * rows * ld * 4);
+        cudaError_t e = rows == 128 ? launch_loss_tile<128>((int)grid, smem, s, n, C, logits, ld, labels, mask, count, dlogits, pred, n_correct, part, status, zero_rows, n_tiles)
+                      : rows == 64  ? launch_loss_tile<64>((int)grid, smem, s, n, C, logits, ld, labels, mask, count, dlogits, pred, n_correct, part, status, zero_rows, n_tiles)
+                                    : launch_loss_tile<32>((int)grid, smem, s, n, C, logits, ld, labels, mask, count, dlogits, pred, n_correct, part, status, zero_rows, n_tiles);
+        return e == cudaSuccess ? (int)grid : -1;
+    }
     if (vec && C <= 128)
-        loss_rows_vec_kernel<1><<<blocks, LOSS_WARPS * 32, 0, s>>>(n, C, logits, ld, labels, mask, count, dlogits, pred, n_correct, part, status, zero_rows);
+        loss_rows_vec_kernel<1><<<warp_blocks, LOSS_WARPS * 32, 0, s>>>(n, C, logits, ld, labels, mask, count, dlogits, pred, n_correct, part, status, zero_rows);
     else if (vec && C <= 256)
-        loss_rows_vec_kernel<2><<<blocks, LOSS_WARPS * 32, 0, s>>>(n, C, logits, ld, labels, mask, count, dlogits, pred, n_correct, part, status, zero_rows);
+        loss_rows_vec_kernel<2><<<warp_blocks, LOSS_WARPS * 32, 0, s>>>(n, C, logits, ld, labels, mask, count, dlogits, pred, n_correct, part, status, zero_rows);
     else
-        loss_rows_kernel<<<blocks, LOSS_WARPS * 32, 0, s>>>(n, C, logits, ld, labels, mask, count, dlogits, pred, n_correct, part, status, zero_rows);
+        loss_rows_kernel<<<warp_blocks, LOSS_WARPS * 32, 0, s>>>(n, C, logits, ld, labels, mask, count, dlogits, pred, n_correct, part, status, zero_rows);
+    return cudaGetLastError() == cudaSuccess ? (int)warp_blocks : -1;
 }
 
 __global__ void loss_final_kernel(int blocks, const double* __restrict__ part,
@@ -345,18 +548,21 @@ extern "C" mixgcn_status mixgcn_loss_softmax_xent(mixgcn_ctx* ctx, int64_t n, in
         int64_t cb = (n + 255) / 256; if (cb > cap) cb = cap;
         count_mask_kernel<<<(unsigned)cb, 256, 0, s>>>(n, train_mask, count);
     }
+    int n_part = (int)blocks;
     {
         LaunchScope scope(ctx, PH_LOSS, s);
         if (ctx->loss_train_rows_only == 1)
             loss_rows_subset_kernel<<<(unsigned)blocks, LOSS_WARPS * 32, 0, s>>>(n, C, logits, ld, labels, train_mask, count, dlogits, pred,
                                                                               reinterpret_cast<unsigned long long*>(n_correct), part, ctx->d_status);
         else
-            launch_loss_rows((unsigned)blocks, s, n, C, logits, ld, labels, train_mask, count, dlogits, pred,
-                             reinterpret_cast<unsigned long long*>(n_correct), part, ctx->d_status, ctx->loss_train_rows_only != 2);
+            n_part = launch_loss_rows((unsigned)blocks, s, n, C, logits, ld, labels, train_mask, count, dlogits, pred,
+                                      reinterpret_cast<unsigned long long*>(n_correct), part, ctx->d_status,
+                                      ctx->loss_train_rows_only != 2, ctx->sm_count);
     }
+    if (n_part < 0) MIXGCN_FAIL(MIXGCN_ECUDA, "loss: kernel launch failed: %s", cudaGetErrorString(cudaGetLastError()));
     {
         LaunchScope scope(ctx, PH_LOSS, s);
-        loss_final_kernel<<<1, 32, 0, s>>>((int)blocks, part, count, loss, ctx->d_status);
+        loss_final_kernel<<<1, 32, 0, s>>>(n_part, part, count, loss, ctx->d_status);
     }
     MIXGCN_CUDA(cudaGetLastError());
     return MIXGCN_OK;
@@ -459,9 +665,12 @@ extern "C" mixgcn_status mixgcn_loss_softmax_xent_noalloc(int64_t n, int32_t C, 
     int64_t cb = (n + 255) / 256;
     if (cb > 4096) cb = 4096;
     count_mask_kernel<<<(unsigned)cb, 256, 0, s>>>(n, train_mask, &sc->count);
-    launch_loss_rows((unsigned)blocks, s, n, C, logits, ld, labels, train_mask, &sc->count, dlogits, pred,
-                     reinterpret_cast<unsigned long long*>(n_correct), sc->part, &sc->status);
-    loss_final_kernel<<<1, 32, 0, s>>>((int)blocks, sc->part, &sc->count, loss, &sc->status);
+    int sm_count = 0;
+    MIXGCN_CUDA(cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, device));
+    const int n_part = launch_loss_rows((unsigned)blocks, s, n, C, logits, ld, labels, train_mask, &sc->count, dlogits, pred,
+                                        reinterpret_cast<unsigned long long*>(n_correct), sc->part, &sc->status, true, sm_count);
+    if (n_part < 0) MIXGCN_FAIL(MIXGCN_ECUDA, "loss_noalloc: kernel launch failed: %s", cudaGetErrorString(cudaGetLastError()));
+    loss_final_kernel<<<1, 32, 0, s>>>(n_part, sc->part, &sc->count, loss, &sc->status);
     if (status) MIXGCN_CUDA(cudaMemcpyAsync(status, &sc->status, sizeof(int32_t), cudaMemcpyDeviceToDevice, s));
     MIXGCN_CUDA(cudaGetLastError());
     return MIXGCN_OK;
