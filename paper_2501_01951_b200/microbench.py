@@ -3,6 +3,7 @@ and as a small, self-ending target for profiler captures.
 
     python -m paper_2501_01951_b200.microbench --op spmm --n 4000000 --edges 32000000 --w 128
     python -m paper_2501_01951_b200.microbench --op gemm --M 1000000 --N 1024 --K 1024 --precision tf32
+    python -m paper_2501_01951_b200.microbench --op loss --n 4000000 --w 172 --mask-p 0.01 --loss-rows 0
 
 Prints one JSON line with the median time and the derived algorithmic GB/s or TFLOP/s.
 """
@@ -35,7 +36,7 @@ def _time(fn, iters, warmup):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--op", required=True, choices=["spmm", "gemm"])
+    ap.add_argument("--op", required=True, choices=["spmm", "gemm", "loss"])
     ap.add_argument("--n", type=int, default=1 << 20)
     ap.add_argument("--edges", type=int, default=8 << 20, help="distinct undirected edges of the R-MAT graph")
     ap.add_argument("--w", type=int, default=128)
@@ -48,6 +49,8 @@ def main():
     ap.add_argument("--iters", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=2)
     ap.add_argument("--seed", type=int, default=1005)
+    ap.add_argument("--mask-p", type=float, default=0.01, help="loss: fraction of train rows")
+    ap.add_argument("--loss-rows", type=int, default=0, choices=[0, 1, 2], help="loss: MIXGCN_OPT_LOSS_TRAIN_ROWS_ONLY value")
     ap.add_argument("--slice", type=int, default=0, help="feature-column slice width of the aggregation (0 = default)")
     args = ap.parse_args()
 
@@ -67,6 +70,25 @@ def main():
         alg = 8 * (g.n + 1) + 8 * g.nnz + 8 * g.n * args.w
         out.update(n=g.n, nnz=g.nnz, w=args.w, max_deg=g.max_deg, ms_median=round(med, 4), ms_best=round(best, 4),
                    alg_bytes=alg, alg_gbs=round(alg / med / 1e6, 1), gather_gbs=round(4 * g.nnz * args.w / med / 1e6, 1))
+    elif args.op == "loss":
+        n, C = args.n, args.w
+        ld = (C + 3) // 4 * 4
+        P = synth.normal_features(n, C, 7, device=dev, ld=ld)
+        G = torch.empty_like(P)
+        y = synth.uniform_labels(n, C, 8, device=dev)
+        m = synth.bernoulli_mask(n, args.mask_p, 9, device=dev)
+        loss = torch.zeros(1, device=dev)
+        pred = torch.zeros(n, dtype=torch.int32, device=dev)
+        nc = torch.zeros(1, dtype=torch.int64, device=dev)
+        mg.ctx_set_option(ctx, mg.OPT_LOSS_TRAIN_ROWS_ONLY, args.loss_rows)
+        med, best = _time(lambda: mg.loss_softmax_xent(ctx, P, y, m, loss, dlogits=G, pred=pred, n_correct=nc, C_=C),
+                          args.iters, args.warmup)
+        n_train = int(m.sum().item())
+        rows_read = n_train if args.loss_rows == 1 else n
+        rows_written = n if args.loss_rows == 0 else n_train
+        alg = 4 * C * (rows_read + rows_written) + 9 * n
+        out.update(n=n, C=C, train_rows=n_train, loss_rows_option=args.loss_rows, loss=round(loss.item(), 6),
+                   ms_median=round(med, 4), ms_best=round(best, 4), alg_bytes=alg, alg_gbs=round(alg / med / 1e6, 1))
     else:
         M, N, K = args.M, args.N, args.K
         r4 = lambda x: (x + 3) // 4 * 4
