@@ -25,6 +25,9 @@ using namespace mixgcn;
 #ifndef MIXGCN_SPMM_MINB
 #define MIXGCN_SPMM_MINB 1
 #endif
+#ifndef MIXGCN_SPMM_SHORT_MAXE
+#define MIXGCN_SPMM_SHORT_MAXE 2     // 0 = rows of 1..2 entries go through the packed group kernel
+#endif
 #ifndef MIXGCN_SPMM_U
 #define MIXGCN_SPMM_U 8
 #endif
@@ -164,6 +167,57 @@ __global__ void __launch_bounds__(256, MIXGCN_SPMM_MINB) spmm_group_kernel(const
     for (int v = 0; v < VPL; ++v) {
         const int c4 = lig + v * LPR;
         if (c4 < w4) store_row(p, u, c4, acc[v]);
+    }
+}
+
+// Rows of at most MAXE entries, width <= 128: a warp takes RB schedule records at once.  Lanes read the
+// records, column ids and values in one coalesced load each; every gathered row of Y is then a single
+// 512-byte request of the whole warp (lane = float4 column), RB of them in flight; entries of a row are
+// added in entry order, as everywhere else.
+template <int RB, int MAXE>
+__global__ void __launch_bounds__(256, 3) spmm_short_kernel(const SpmmParams p) {
+    static_assert(RB * MAXE <= 32, "one lane per (row, entry)");
+    const int lane = threadIdx.x & 31;
+    const int64_t idx0 = p.idx_begin + (((int64_t)blockIdx.x * 256 + threadIdx.x) >> 5) * RB;
+    if (idx0 >= p.idx_end) return;
+    int4 rc = make_int4(0, 0, 0, 0);
+    if (lane < RB && idx0 + lane < p.idx_end) rc = __ldg(reinterpret_cast<const int4*>(p.rec + idx0 + lane));
+    // lane (k, e) = (lane % RB, lane / RB) fetches entry e of row k
+    const int k_of = lane % RB, e_of = lane / RB;
+    const uint32_t lo = (uint32_t)__shfl_sync(0xFFFFFFFFu, rc.x, k_of), hi = (uint32_t)__shfl_sync(0xFFFFFFFFu, rc.y, k_of);
+    const int len_of = __shfl_sync(0xFFFFFFFFu, rc.z, k_of);
+    int c = 0; float a = 0.0f;
+    if (e_of < MAXE && e_of < len_of) {
+        const int64_t at = (((int64_t)hi << 32) | lo) + e_of;
+        c = __ldg(p.col + at); a = __ldg(p.val + at);
+    }
+    const int w4 = (p.w + 3) >> 2;
+    const float* Yb = p.Y + p.j0;
+    const bool col_ok = lane < w4;
+    float4 acc[RB];
+#pragma unroll
+    for (int k = 0; k < RB; ++k) acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int e = 0; e < MAXE; ++e) {
+        float4 y[RB]; float ak[RB];
+#pragma unroll
+        for (int k = 0; k < RB; ++k) {
+            const int ck = __shfl_sync(0xFFFFFFFFu, c, k + e * RB);
+            ak[k] = __shfl_sync(0xFFFFFFFFu, a, k + e * RB);
+            const int len_k = __shfl_sync(0xFFFFFFFFu, rc.z, k);
+            const bool live = e < len_k && col_ok;
+            y[k] = live ? __ldg(reinterpret_cast<const float4*>(Yb + (int64_t)ck * p.ldy) + lane) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int k = 0; k < RB; ++k) {
+            const int len_k = __shfl_sync(0xFFFFFFFFu, rc.z, k);
+            if (e < len_k) fma4(acc[k], ak[k], y[k]);
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < RB; ++k) {
+        const int64_t u = __shfl_sync(0xFFFFFFFFu, rc.w, k);
+        if (idx0 + k < p.idx_end && col_ok) store_row(p, u, lane, acc[k]);
     }
 }
 
@@ -518,7 +572,15 @@ mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView&
             p.idx_begin = S.total_segs + (begin - S.n_long);
             p.idx_end = S.total_segs + (end - S.n_long);
             LaunchScope scope(ctx, phase, s);
-            dispatch(p, fold, s);
+            if (q == 3 && p.w <= 128 && SPMM_PACK_DEG[2] <= MIXGCN_SPMM_SHORT_MAXE && MIXGCN_SPMM_SHORT_MAXE > 0) {
+                // rows of at most SPMM_PACK_DEG[2] entries: several rows per warp, whole-warp gathers
+                constexpr int RB = 8, MAXE = MIXGCN_SPMM_SHORT_MAXE > 0 ? MIXGCN_SPMM_SHORT_MAXE : 1;
+                const int64_t units = p.idx_end - p.idx_begin;
+                const int64_t warps = (units + RB - 1) / RB;
+                spmm_short_kernel<RB, MAXE><<<(unsigned)((warps + 7) / 8), 256, 0, s>>>(p);
+            } else {
+                dispatch(p, fold, s);
+            }
             begin = end;
         }
     }
