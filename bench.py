@@ -256,9 +256,7 @@ def run_ours(args, rank, world, local_rank):
     if can_rows and can_cache:
         variants.append(("both", True, True))
     for name, rows_only, cache in variants:
-        tr.train_rows_only = rows_only or args.train_rows_only
-        tr.cache_first_aggregation = cache or args.cache_first_aggregation
-        tr._plan_row_sparsity()
+        tr.configure(train_rows_only=rows_only or args.train_rows_only, cache_first_aggregation=cache or args.cache_first_aggregation)
         for _ in range(2):
             t += 1
             tr.epoch(t)
@@ -273,8 +271,7 @@ def run_ours(args, rank, world, local_rank):
         ms_s, value_s = replicas_throughput(e0.elapsed_time(e1), args.steps, world, dev)
         opt_in[name] = dict(value=round(value_s, 4), unit=UNIT, ms_per_step=round(ms_s / args.steps, 3), loss=round(tr.loss.item(), 6))
     if variants:
-        tr.train_rows_only, tr.cache_first_aggregation = args.train_rows_only, args.cache_first_aggregation
-        tr._plan_row_sparsity()
+        tr.configure(train_rows_only=args.train_rows_only, cache_first_aggregation=args.cache_first_aggregation)
 
     # roofline of the aggregation kernels over the timed steps
     plan = spmm_plan(wl, tr.orders, tr.row_sparse_levels, args.train_rows_only)

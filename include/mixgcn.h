@@ -21,6 +21,9 @@
  *    produces zeros, and mixgcn_ctx_poll_status() reports them.
  *  - Deterministic: no atomics on floating-point data; the same inputs give bitwise the same
  *    outputs on every call.
+ *  - Threads: a context and the objects created from it (graphs, row plans) keep scratch buffers
+ *    and options in the context; use them from one host thread at a time.  Different contexts are
+ *    independent.
  */
 #ifndef MIXGCN_H_
 #define MIXGCN_H_

@@ -313,13 +313,14 @@ extern "C" mixgcn_status mixgcn_layer_fwd(mixgcn_ctx* ctx, const mixgcn_graph* g
         // update then runs on the compacted rows and its result is scattered back.
         const uint8_t* rows = d->gout_row_mask;
         const int64_t cnt = d->gout_row_count;
+        SpmmOpts filter_rows; filter_rows.row_filter = rows;
         if (!rows || cnt <= 0 || cnt > n)
             MIXGCN_FAIL(MIXGCN_EINVAL, "layer_fwd: OUT_ROWS_ONLY needs gout_row_mask and its exact count (mask %s, count %lld, n %lld)",
                         rows ? "given" : "null", (long long)cnt, (long long)n);
         if (drop_mask) MIXGCN_FAIL(MIXGCN_EUNSUPPORTED, "layer_fwd: OUT_ROWS_ONLY does not take a dropout mask");
         if (order == MIXGCN_ORDER_AGG_FIRST) {
             if (!saved_valid)
-                MIXGCN_TRY(launch_spmm(ctx, g, g->fwd, 1, 0, d->d_in, X_in, d->ld_in, saved, d->ld_saved, nullptr, s, nullptr, rows));
+                MIXGCN_TRY(launch_spmm(ctx, g, g->fwd, 1, 0, d->d_in, X_in, d->ld_in, saved, d->ld_saved, nullptr, s, filter_rows));
             RowSet rs;
             const int64_t lda = (d->d_in + 3) / 4 * 4, ldb = (d->d_out + 3) / 4 * 4;
             MIXGCN_TRY(build_row_set(ctx, n, rows, cnt, lda, ldb, &rs, s));
@@ -330,7 +331,7 @@ extern "C" mixgcn_status mixgcn_layer_fwd(mixgcn_ctx* ctx, const mixgcn_graph* g
         }
         MIXGCN_TRY(launch_gemm(ctx, d->precision, 0, 0, n, d->d_out, d->d_in, X_in, d->ld_in, W, ldw, saved, d->ld_saved,
                                nullptr, 0, s));
-        MIXGCN_TRY(launch_spmm(ctx, g, g->fwd, 1, 0, d->d_out, saved, d->ld_saved, X_out, d->ld_out, &epi, s, nullptr, rows));
+        MIXGCN_TRY(launch_spmm(ctx, g, g->fwd, 1, 0, d->d_out, saved, d->ld_saved, X_out, d->ld_out, &epi, s, filter_rows));
         return MIXGCN_OK;
     }
 
@@ -410,7 +411,8 @@ extern "C" mixgcn_status mixgcn_layer_bwd(mixgcn_ctx* ctx, const mixgcn_graph* g
         float* ca = reinterpret_cast<float*>(ctx->workspace_rows);
         float* cb = reinterpret_cast<float*>(reinterpret_cast<char*>(ctx->workspace_rows) + up(rows_alloc * lda * 4));
         // rows of the restricted matrix are scheduled longest first: its non-empty rows are the first out_count
-        const int64_t gin_rows = (d->flags & MIXGCN_LAYER_GIN_ROWS_ONLY) ? plan->out_count : -1;
+        SpmmOpts plan_all; plan_all.phase = PH_SPMM_SPARSE;
+        SpmmOpts plan_opts = plan_all; plan_opts.row_limit = (d->flags & MIXGCN_LAYER_GIN_ROWS_ONLY) ? plan->out_count : -1;
         MIXGCN_TRY(launch_gather_rows(ctx, cnt, d->d_out, plan->idx, G_out, d->ld_out, cb, ldb, s));         // dP_T
         if (dbias) MIXGCN_TRY(launch_colsum(ctx, cnt, d->d_out, cb, ldb, dbias, s));
         if (order == MIXGCN_ORDER_AGG_FIRST) {
@@ -418,12 +420,12 @@ extern "C" mixgcn_status mixgcn_layer_bwd(mixgcn_ctx* ctx, const mixgcn_graph* g
             MIXGCN_TRY(launch_gemm(ctx, d->precision, 1, 0, d->d_in, d->d_out, cnt, ca, lda, cb, ldb, dW, ldw, nullptr, 0, s));
             if (!first) {
                 MIXGCN_TRY(launch_gemm(ctx, d->precision, 0, 1, cnt, d->d_in, d->d_out, cb, ldb, W, ldw, ca, lda, nullptr, 0, s));
-                MIXGCN_TRY(launch_spmm(ctx, g, plan->view, 1, 0, d->d_in, ca, lda, G_in, d->ld_in, gin, s, nullptr, nullptr, PH_SPMM_SPARSE, gin_rows));
+                MIXGCN_TRY(launch_spmm(ctx, g, plan->view, 1, 0, d->d_in, ca, lda, G_in, d->ld_in, gin, s, plan_opts));
             }
             return MIXGCN_OK;
         }
         // update first: dQ = A_hat^T dZ from the compacted rows (into `saved`, every row), then the dense products
-        MIXGCN_TRY(launch_spmm(ctx, g, plan->view, 1, 0, d->d_out, cb, ldb, saved, d->ld_saved, nullptr, s, nullptr, nullptr, PH_SPMM_SPARSE));
+        MIXGCN_TRY(launch_spmm(ctx, g, plan->view, 1, 0, d->d_out, cb, ldb, saved, d->ld_saved, nullptr, s, plan_all));
         MIXGCN_TRY(launch_gemm(ctx, d->precision, 1, 0, d->d_in, d->d_out, n, X_in, d->ld_in, saved, d->ld_saved, dW, ldw, nullptr, 0, s));
         if (!first)
             MIXGCN_TRY(launch_gemm(ctx, d->precision, 0, 1, n, d->d_in, d->d_out, saved, d->ld_saved, W, ldw, G_in, d->ld_in, gin, 0, s));
@@ -431,7 +433,7 @@ extern "C" mixgcn_status mixgcn_layer_bwd(mixgcn_ctx* ctx, const mixgcn_graph* g
     }
     const uint8_t* rmask = d->gout_row_mask;
     SpmmRowSparse sp{rmask, nullptr, d->gin_row_mask};
-    const SpmmRowSparse* spp = rmask ? &sp : nullptr;
+    SpmmOpts sparse_opts; sparse_opts.sparse = rmask ? &sp : nullptr;
 
     if (order == MIXGCN_ORDER_AGG_FIRST) {
         const int64_t cnt = d->gout_row_count;
@@ -449,7 +451,7 @@ extern "C" mixgcn_status mixgcn_layer_bwd(mixgcn_ctx* ctx, const mixgcn_graph* g
             if (!first) {
                 MIXGCN_TRY(launch_gemm(ctx, d->precision, 0, 1, cnt, d->d_in, d->d_out, rs.b, ldb, W, ldw, rs.a, lda, nullptr, 0, s));
                 sp.in_pos = rs.pos;                                                                             // dZ_T is compact
-                MIXGCN_TRY(launch_spmm(ctx, g, g->bwd, 1, 0, d->d_in, rs.a, lda, G_in, d->ld_in, gin, s, &sp));
+                MIXGCN_TRY(launch_spmm(ctx, g, g->bwd, 1, 0, d->d_in, rs.a, lda, G_in, d->ld_in, gin, s, sparse_opts));
             }
             return MIXGCN_OK;
         }
@@ -460,7 +462,7 @@ extern "C" mixgcn_status mixgcn_layer_bwd(mixgcn_ctx* ctx, const mixgcn_graph* g
         if (!first) {
             MIXGCN_TRY(launch_gemm(ctx, d->precision, 0, 1, n, d->d_in, d->d_out, G_out, d->ld_out, W, ldw, saved,
                                    d->ld_saved, nullptr, 0, s));
-            MIXGCN_TRY(launch_spmm(ctx, g, g->bwd, 1, 0, d->d_in, saved, d->ld_saved, G_in, d->ld_in, gin, s, spp));
+            MIXGCN_TRY(launch_spmm(ctx, g, g->bwd, 1, 0, d->d_in, saved, d->ld_saved, G_in, d->ld_in, gin, s, sparse_opts));
         }
         return MIXGCN_OK;
     }
@@ -481,7 +483,7 @@ extern "C" mixgcn_status mixgcn_layer_bwd(mixgcn_ctx* ctx, const mixgcn_graph* g
     } else if (dbias) {
         MIXGCN_TRY(launch_colsum(ctx, n, d->d_out, G_out, d->ld_out, dbias, s));
     }
-    MIXGCN_TRY(launch_spmm(ctx, g, g->bwd, 1, 0, d->d_out, G_out, d->ld_out, saved, d->ld_saved, nullptr, s, spp));
+    MIXGCN_TRY(launch_spmm(ctx, g, g->bwd, 1, 0, d->d_out, G_out, d->ld_out, saved, d->ld_saved, nullptr, s, sparse_opts));
     MIXGCN_TRY(launch_gemm(ctx, d->precision, 1, 0, d->d_in, d->d_out, n, X_in, d->ld_in, saved, d->ld_saved, dW, ldw,
                            nullptr, 0, s));
     if (!first)

@@ -180,10 +180,16 @@ struct SpmmRowSparse {
 
 // kernels' host launchers (all asynchronous on `s`)
 // Aggregation over all rows (chunks <= 1) or over chunk k of `chunks` row chunks.
+// Optional behaviour of one aggregation call.
+struct SpmmOpts {
+    const SpmmRowSparse* sparse = nullptr;   // row-sparse input: test the input's row mask inside the kernel
+    const uint8_t* row_filter = nullptr;     // compute only the output rows whose byte is non-zero (not with `sparse`)
+    int phase = PH_SPMM;                     // profiling phase the launches are booked under
+    int64_t row_limit = -1;                  // >= 0: only the first row_limit rows of the schedule (longest first)
+};
 mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView& A, int chunks, int k,
                           int32_t w, const float* Y, int64_t ldy, float* Z, int64_t ldz,
-                          const mixgcn_epilogue* epi, cudaStream_t s, const SpmmRowSparse* sparse = nullptr,
-                          const uint8_t* row_filter = nullptr, int phase = PH_SPMM, int64_t row_limit = -1);
+                          const mixgcn_epilogue* epi, cudaStream_t s, const SpmmOpts& opts = SpmmOpts());
 // schedule of all n rows of a view whose column ids lie in [0, n_cols); release of a view's memory
 mixgcn_status build_view_schedule(int64_t n_cols, int64_t n, CsrView& v, cudaStream_t s);
 void release_view(CsrView& v);

@@ -197,6 +197,8 @@ extern "C" mixgcn_status mixgcn_spmm_rowplan(mixgcn_ctx* ctx, const mixgcn_rowpl
     if (epi && epi->gate && epi->ld_gate < w) MIXGCN_FAIL(MIXGCN_EINVAL, "spmm_rowplan: gate leading dimension < w");
     MIXGCN_CUDA(cudaSetDevice(ctx->device));
     // rows of the restricted matrix are scheduled longest first, so its non-empty rows are the first out_count
-    return launch_spmm(ctx, p->g, p->view, 1, 0, w, Yc, ldy, Z, ldz, epi, (cudaStream_t)stream, nullptr, nullptr,
-                       PH_SPMM_SPARSE, rows_only ? p->out_count : -1);
+    SpmmOpts opts;
+    opts.phase = PH_SPMM_SPARSE;
+    opts.row_limit = rows_only ? p->out_count : -1;
+    return launch_spmm(ctx, p->g, p->view, 1, 0, w, Yc, ldy, Z, ldz, epi, (cudaStream_t)stream, opts);
 }

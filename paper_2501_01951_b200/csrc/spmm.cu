@@ -449,8 +449,11 @@ namespace mixgcn {
 // with its own schedule: long rows as column-ordered segments, then rows longest first, short rows packed.
 mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView& A, int chunks, int k,
                           int32_t w, const float* Y, int64_t ldy, float* Z, int64_t ldz,
-                          const mixgcn_epilogue* epi, cudaStream_t s, const SpmmRowSparse* sparse,
-                          const uint8_t* row_filter, int phase, int64_t row_limit) {
+                          const mixgcn_epilogue* epi, cudaStream_t s, const SpmmOpts& opts) {
+    const SpmmRowSparse* sparse = opts.sparse;
+    const uint8_t* row_filter = opts.row_filter;
+    const int phase = opts.phase;
+    const int64_t row_limit = opts.row_limit;
     if (w <= 0) return MIXGCN_OK;
     if (sparse && row_filter) MIXGCN_FAIL(MIXGCN_EUNSUPPORTED, "spmm: a row filter cannot be combined with a row-sparse input");
     if (chunks > 1) {

@@ -103,6 +103,17 @@ class GcnTrainer:
         self.descs[0].flags &= ~mg.LAYER_SAVED_IS_VALID
         self._plan_row_sparsity()
 
+    def configure(self, train_rows_only=None, cache_first_aggregation=None, row_sparse=None):
+        """Switch the opt-in variants of an existing trainer (buffers and inputs stay); rebuilds the row plans."""
+        if train_rows_only is not None:
+            self.train_rows_only = bool(train_rows_only)
+        if cache_first_aggregation is not None:
+            self.cache_first_aggregation = bool(cache_first_aggregation)
+            self._first_aggregation_valid = False
+        if row_sparse is not None:
+            self.row_sparse = row_sparse
+        self._plan_row_sparsity()
+
     def _plan_row_sparsity(self):
         """The loss gradient is non-zero on train rows only; one aggregation later on their neighbours
         only.  Hand those row masks to layer_bwd for the top `levels` layers (plumbing: the masks are

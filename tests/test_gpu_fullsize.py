@@ -220,8 +220,7 @@ def test_full_size_workload(mg, key):
     # ---- the train-rows-only shortcut at full size: same loss and gradients as the full computation
     # above; rows outside the train mask hold NaN beforehand, so reading one of them would show
     ref_loss, ref_dW, ref_db = tr.loss.item(), [t.clone() for t in tr.dW], [t.clone() for t in tr.db]
-    tr.train_rows_only = True
-    tr._plan_row_sparsity()
+    tr.configure(train_rows_only=True)
     assert tr.row_sparse_levels >= 1
     tr.X[L].fill_(float("nan"))
     if agg_first:
