@@ -23,7 +23,13 @@
 using namespace mixgcn;
 
 #ifndef MIXGCN_SPMM_MINB
-#define MIXGCN_SPMM_MINB 1
+#define MIXGCN_SPMM_MINB 4      // CTAs per SM asked of the compiler for the narrow (VPL <= 2) group kernels
+#endif
+#ifndef MIXGCN_SPMM_FOLD_SEG
+#define MIXGCN_SPMM_FOLD_SEG 2      // lanes-per-unit fold for long-row segments at widths <= 128 (1: 32 lanes, 2: 16 lanes x 2 float4, ...)
+#endif
+#ifndef MIXGCN_SPMM_FOLD_MED
+#define MIXGCN_SPMM_FOLD_MED 2      // the same for rows of 13..512 entries
 #endif
 #ifndef MIXGCN_SPMM_SHORT_MAXE
 #define MIXGCN_SPMM_SHORT_MAXE 2     // 0 = rows of 1..2 entries go through the packed group kernel
@@ -133,7 +139,7 @@ __device__ __forceinline__ void row_segment(const SpmmParams& p, int64_t b, int6
 }
 
 template <int LPR, int VPL>
-__global__ void __launch_bounds__(256, MIXGCN_SPMM_MINB) spmm_group_kernel(const SpmmParams p) {
+__global__ void __launch_bounds__(256, VPL <= 2 ? MIXGCN_SPMM_MINB : 1) spmm_group_kernel(const SpmmParams p) {
     const int lig = threadIdx.x % LPR;
     const int64_t idx = p.idx_begin + ((int64_t)blockIdx.x * 256 + threadIdx.x) / LPR;
     if (idx >= p.idx_end) return;  // the whole group leaves together
@@ -548,7 +554,7 @@ mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView&
             {
                 LaunchScope scope(ctx, phase, s);
                 p.idx_begin = 0; p.idx_end = S.total_segs;
-                dispatch(p, 1, s);
+                dispatch(p, p.w <= 128 ? MIXGCN_SPMM_FOLD_SEG : 1, s);
             }
             {
                 LaunchScope scope(ctx, phase, s);
@@ -582,7 +588,7 @@ mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView&
                 const int64_t warps = (units + RB - 1) / RB;
                 spmm_short_kernel<RB, MAXE><<<(unsigned)((warps + 7) / 8), 256, 0, s>>>(p);
             } else {
-                dispatch(p, fold, s);
+                dispatch(p, q == 0 ? (p.w <= 128 ? MIXGCN_SPMM_FOLD_MED : 1) : fold, s);
             }
             begin = end;
         }
