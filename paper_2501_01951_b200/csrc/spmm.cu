@@ -25,6 +25,9 @@ using namespace mixgcn;
 #ifndef MIXGCN_SPMM_MINB
 #define MIXGCN_SPMM_MINB 4      // CTAs per SM asked of the compiler for the narrow (VPL <= 2) group kernels
 #endif
+#ifndef MIXGCN_SPMM_FOLD_WMAX
+#define MIXGCN_SPMM_FOLD_WMAX 128   // widest aggregation the two folds below apply to
+#endif
 #ifndef MIXGCN_SPMM_FOLD_SEG
 #define MIXGCN_SPMM_FOLD_SEG 2      // lanes-per-unit fold for long-row segments at widths <= 128 (1: 32 lanes, 2: 16 lanes x 2 float4, ...)
 #endif
@@ -554,7 +557,7 @@ mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView&
             {
                 LaunchScope scope(ctx, phase, s);
                 p.idx_begin = 0; p.idx_end = S.total_segs;
-                dispatch(p, p.w <= 128 ? MIXGCN_SPMM_FOLD_SEG : 1, s);
+                dispatch(p, p.w <= MIXGCN_SPMM_FOLD_WMAX ? MIXGCN_SPMM_FOLD_SEG : 1, s);
             }
             {
                 LaunchScope scope(ctx, phase, s);
@@ -588,7 +591,7 @@ mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView&
                 const int64_t warps = (units + RB - 1) / RB;
                 spmm_short_kernel<RB, MAXE><<<(unsigned)((warps + 7) / 8), 256, 0, s>>>(p);
             } else {
-                dispatch(p, q == 0 ? (p.w <= 128 ? MIXGCN_SPMM_FOLD_MED : 1) : fold, s);
+                dispatch(p, q == 0 ? (p.w <= MIXGCN_SPMM_FOLD_WMAX ? MIXGCN_SPMM_FOLD_MED : 1) : fold, s);
             }
             begin = end;
         }
