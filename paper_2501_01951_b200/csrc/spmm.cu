@@ -34,6 +34,12 @@ using namespace mixgcn;
 #ifndef MIXGCN_SPMM_FOLD_MED
 #define MIXGCN_SPMM_FOLD_MED 2      // the same for rows of 13..512 entries
 #endif
+#ifndef MIXGCN_SPMM_SHORT_RB
+#define MIXGCN_SPMM_SHORT_RB 4       // rows a warp of the short-row kernel takes at once
+#endif
+#ifndef MIXGCN_SPMM_SHORT_MINB
+#define MIXGCN_SPMM_SHORT_MINB 6     // CTAs per SM asked of the compiler for it
+#endif
 #ifndef MIXGCN_SPMM_SHORT_MAXE
 #define MIXGCN_SPMM_SHORT_MAXE 2     // 0 = rows of 1..2 entries go through the packed group kernel
 #endif
@@ -184,7 +190,7 @@ __global__ void __launch_bounds__(256, VPL <= 2 ? MIXGCN_SPMM_MINB : 1) spmm_gro
 // 512-byte request of the whole warp (lane = float4 column), RB of them in flight; entries of a row are
 // added in entry order, as everywhere else.
 template <int RB, int MAXE>
-__global__ void __launch_bounds__(256, 3) spmm_short_kernel(const SpmmParams p) {
+__global__ void __launch_bounds__(256, MIXGCN_SPMM_SHORT_MINB) spmm_short_kernel(const SpmmParams p) {
     static_assert(RB * MAXE <= 32, "one lane per (row, entry)");
     const int lane = threadIdx.x & 31;
     const int64_t idx0 = p.idx_begin + (((int64_t)blockIdx.x * 256 + threadIdx.x) >> 5) * RB;
@@ -586,7 +592,7 @@ mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView&
             LaunchScope scope(ctx, phase, s);
             if (q == 3 && p.w <= 128 && SPMM_PACK_DEG[2] <= MIXGCN_SPMM_SHORT_MAXE && MIXGCN_SPMM_SHORT_MAXE > 0) {
                 // rows of at most SPMM_PACK_DEG[2] entries: several rows per warp, whole-warp gathers
-                constexpr int RB = 8, MAXE = MIXGCN_SPMM_SHORT_MAXE > 0 ? MIXGCN_SPMM_SHORT_MAXE : 1;
+                constexpr int RB = MIXGCN_SPMM_SHORT_RB, MAXE = MIXGCN_SPMM_SHORT_MAXE > 0 ? MIXGCN_SPMM_SHORT_MAXE : 1;
                 const int64_t units = p.idx_end - p.idx_begin;
                 const int64_t warps = (units + RB - 1) / RB;
                 spmm_short_kernel<RB, MAXE><<<(unsigned)((warps + 7) / 8), 256, 0, s>>>(p);
