@@ -7,6 +7,7 @@
 // in the same order.  (The paper's sampled SpMM, Eq. 4, skips work by a mask on the output; here the
 // mask is on the operand's rows and the skipping is done ahead of time.)
 #include <cub/cub.cuh>
+#include <thrust/iterator/counting_iterator.h>
 
 #include <new>
 
@@ -106,7 +107,7 @@ extern "C" mixgcn_status mixgcn_rowplan_create(mixgcn_ctx* ctx, const mixgcn_gra
     // kept rows, ascending, and their positions
     DevMem sel, tmp, pos, cnt;
     size_t tb = 0;
-    cub::CountingInputIterator<int32_t> ids(0);
+    thrust::counting_iterator<int32_t> ids(0);
     MIXGCN_CUDA(cudaMalloc((void**)&p->idx, (size_t)(n > 0 ? n : 1) * sizeof(int32_t)));
     MIXGCN_CUDA(cudaMalloc(&sel.p, sizeof(int64_t)));
     MIXGCN_CUDA(cub::DeviceSelect::Flagged(nullptr, tb, ids, in_row_mask, p->idx, sel.as<int64_t>(), n, s));

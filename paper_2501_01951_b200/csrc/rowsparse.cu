@@ -2,6 +2,7 @@
 // non-zero rows (the masked loss gives non-zero rows on train nodes only), the dense products
 // run on the compacted rows and the aggregation skips the zero rows.
 #include <cub/cub.cuh>
+#include <thrust/iterator/counting_iterator.h>
 
 #include "internal.cuh"
 
@@ -71,7 +72,7 @@ mixgcn_status ensure_workspace_rows(mixgcn_ctx* ctx, int64_t bytes) {
 mixgcn_status build_row_set(mixgcn_ctx* ctx, int64_t n, const uint8_t* mask, int64_t count, int64_t ld_a, int64_t ld_b,
                             RowSet* rs, cudaStream_t s) {
     size_t tb = 0;
-    cub::CountingInputIterator<int32_t> ids(0);
+    thrust::counting_iterator<int32_t> ids(0);
     MIXGCN_CUDA(cub::DeviceSelect::Flagged(nullptr, tb, ids, mask, (int32_t*)nullptr, (int64_t*)nullptr, n, s));
     auto up = [](int64_t x) { return (x + 255) & ~(int64_t)255; };
     const int64_t o_pos = 0, o_idx = o_pos + up(n * 4), o_sel = o_idx + up(n * 4), o_tmp = o_sel + 256,
