@@ -175,6 +175,15 @@ typedef struct {
     const float* gate;
     int64_t ld_gate;
     float gate_scale;
+    /* y = y + residual_scale * residual[i*ld_residual + j], applied FIRST (before the bias), when
+     * residual != NULL (fp32, n x d; may be the aggregation's own input, must not overlap its output).
+     * Aggregation only (mixgcn_spmm, mixgcn_spmm_rowplan): it turns A_hat Y into (s I + A_hat) Y, the
+     * form sum-aggregator layers with a weighted self term use (GIN's (1 + eps) h + sum of
+     * neighbours; the paper names that architecture in its evaluation without defining it).
+     * mixgcn_gemm rejects it. */
+    const float* residual;
+    int64_t ld_residual;
+    float residual_scale;
 } mixgcn_epilogue;
 
 /* Neighbour aggregation Z = A_hat Y (transposed != 0: A_hat^T Y), n x w (Algorithm 2,

@@ -49,7 +49,8 @@ SYMBOLS = (
 class Epilogue(C.Structure):
     _fields_ = [("bias", C.c_void_p), ("relu", C.c_int32), ("drop_mask", C.c_void_p),
                 ("keep_scale", C.c_float), ("gate", C.c_void_p), ("ld_gate", C.c_int64),
-                ("gate_scale", C.c_float)]
+                ("gate_scale", C.c_float), ("residual", C.c_void_p), ("ld_residual", C.c_int64),
+                ("residual_scale", C.c_float)]
 
 
 class LayerDesc(C.Structure):
@@ -256,7 +257,8 @@ def graph_create_permuted(ctx: Ctx, g: Graph, order: torch.Tensor) -> Graph:
 
 # ------------------------------------------------------------------------------ building blocks
 
-def make_epilogue(bias=None, relu=False, drop_mask=None, keep_scale=1.0, gate=None, gate_scale=1.0):
+def make_epilogue(bias=None, relu=False, drop_mask=None, keep_scale=1.0, gate=None, gate_scale=1.0,
+                  residual=None, residual_scale=1.0):
     e = Epilogue()
     e.bias = None if bias is None else _dev(bias, torch.float32, "bias").data_ptr()
     e.relu = int(relu)
@@ -266,7 +268,11 @@ def make_epilogue(bias=None, relu=False, drop_mask=None, keep_scale=1.0, gate=No
         gate, ldg = _mat(gate, "gate")
         e.gate, e.ld_gate = gate.data_ptr(), ldg
     e.gate_scale = gate_scale
-    e._keep = (bias, drop_mask, gate)
+    if residual is not None:
+        residual, ldr = _mat(residual, "residual")
+        e.residual, e.ld_residual = residual.data_ptr(), ldr
+    e.residual_scale = residual_scale
+    e._keep = (bias, drop_mask, gate, residual)
     return e
 
 

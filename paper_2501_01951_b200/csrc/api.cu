@@ -236,6 +236,7 @@ extern "C" mixgcn_status mixgcn_gemm(mixgcn_ctx* ctx, int32_t precision, int32_t
         MIXGCN_FAIL(MIXGCN_EINVAL, "gemm: leading dimensions must cover the matrix (lda=%lld ldb=%lld ldc=%lld)",
                     (long long)lda, (long long)ldb, (long long)ldc);
     if (C == A || C == B) MIXGCN_FAIL(MIXGCN_EINVAL, "gemm: C must not overlap A or B");
+    if (epi && epi->residual) MIXGCN_FAIL(MIXGCN_EUNSUPPORTED, "gemm: the residual term is an aggregation epilogue");
     MIXGCN_CUDA(cudaSetDevice(ctx->device));
     return launch_gemm(ctx, precision, trans_a, trans_b, M, N, K, A, lda, B, ldb, C, ldc, epi, 0, (cudaStream_t)stream);
 }

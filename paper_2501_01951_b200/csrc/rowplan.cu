@@ -196,6 +196,8 @@ extern "C" mixgcn_status mixgcn_spmm_rowplan(mixgcn_ctx* ctx, const mixgcn_rowpl
     if (!aligned16(Yc) || !aligned16(Z)) MIXGCN_FAIL(MIXGCN_EINVAL, "spmm_rowplan: Yc and Z must be 16-byte aligned");
     if (Yc == Z) MIXGCN_FAIL(MIXGCN_EINVAL, "spmm_rowplan: Yc and Z must not overlap");
     if (epi && epi->gate && epi->ld_gate < w) MIXGCN_FAIL(MIXGCN_EINVAL, "spmm_rowplan: gate leading dimension < w");
+    if (epi && epi->residual && (epi->ld_residual < w || epi->residual == Z)) MIXGCN_FAIL(MIXGCN_EINVAL, "spmm_rowplan: residual needs ld_residual >= w and must not be the output");
+    if (epi && epi->residual && rows_only) MIXGCN_FAIL(MIXGCN_EUNSUPPORTED, "spmm_rowplan: rows_only cannot be combined with a residual (rows without a kept entry are not zero then)");
     MIXGCN_CUDA(cudaSetDevice(ctx->device));
     // rows of the restricted matrix are scheduled longest first, so its non-empty rows are the first out_count
     SpmmOpts opts;

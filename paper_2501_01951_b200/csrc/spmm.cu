@@ -74,9 +74,11 @@ struct SpmmParams {
     const float* bias; int relu;
     const uint8_t* drop; float keep_scale;
     const float* gate; int64_t ld_gate; float gate_scale;
+    const float* residual; int64_t ld_residual; float residual_scale;
 };
 
 __device__ __forceinline__ float epilogue1(const SpmmParams& p, float y, int64_t u, int j) {
+    if (p.residual) y = fmaf(p.residual_scale, p.residual[u * p.ld_residual + j], y);
     if (p.bias) y += p.bias[j];
     if (p.relu) y = fmaxf(y, 0.0f);
     if (p.drop) y = p.drop[u * p.w_total + j] ? y * p.keep_scale : 0.0f;
@@ -88,7 +90,7 @@ __device__ __forceinline__ void store_row(const SpmmParams& p, int64_t u, int c4
     const int j = p.j0 + c4 * 4;           // global column of a.x
     const int jend = p.j0 + p.w;           // one past the last valid column of the slice
     float r[4] = {a.x, a.y, a.z, a.w};
-    if (!p.bias && a.x == 0.0f && a.y == 0.0f && a.z == 0.0f && a.w == 0.0f) {
+    if (!p.bias && !p.residual && a.x == 0.0f && a.y == 0.0f && a.z == 0.0f && a.w == 0.0f) {
         // ReLU, dropout and the gate all map 0 to 0: no mask or gate byte needs to be read (the empty
         // rows of a row-sparse aggregation take this path)
         *reinterpret_cast<float4*>(p.Z + u * p.ldz + j) = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -483,6 +485,7 @@ mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView&
     if (epi) {
         p.bias = epi->bias; p.relu = epi->relu; p.drop = epi->drop_mask; p.keep_scale = epi->keep_scale;
         p.gate = epi->gate; p.ld_gate = epi->ld_gate; p.gate_scale = epi->gate_scale;
+        p.residual = epi->residual; p.ld_residual = epi->ld_residual; p.residual_scale = epi->residual_scale;
     }
     p.rec = S.rec;
     if (sparse) { p.in_mask = sparse->in_mask; p.in_pos = sparse->in_pos; p.out_mask = sparse->out_mask; }
@@ -619,6 +622,7 @@ extern "C" mixgcn_status mixgcn_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, int
     if (!aligned16(Y) || !aligned16(Z)) MIXGCN_FAIL(MIXGCN_EINVAL, "spmm: Y and Z must be 16-byte aligned");
     if (Y == Z) MIXGCN_FAIL(MIXGCN_EINVAL, "spmm: Y and Z must not overlap");
     if (epi && epi->gate && epi->ld_gate < w) MIXGCN_FAIL(MIXGCN_EINVAL, "spmm: gate leading dimension < w");
+    if (epi && epi->residual && (epi->ld_residual < w || epi->residual == Z)) MIXGCN_FAIL(MIXGCN_EINVAL, "spmm: residual needs ld_residual >= w and must not be the output");
     MIXGCN_CUDA(cudaSetDevice(ctx->device));
     return launch_spmm(ctx, g, transposed ? g->bwd : g->fwd, 1, 0, w, Y, ldy, Z, ldz, epi, (cudaStream_t)stream);
 }

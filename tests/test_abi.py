@@ -35,7 +35,8 @@ def test_status_strings(mg):
 
 def test_struct_layouts_match_the_header(mg):
     # the header's structs, field by field, on an LP64 ABI
-    assert C.sizeof(mg.Epilogue) == 56
+    assert C.sizeof(mg.Epilogue) == 80
+    assert mg.Epilogue.residual.offset == 56 and mg.Epilogue.ld_residual.offset == 64 and mg.Epilogue.residual_scale.offset == 72
     assert C.sizeof(mg.LayerDesc) == 88
     assert mg.LayerDesc.gout_row_mask.offset == 56 and mg.LayerDesc.gin_row_mask.offset == 72
     assert mg.LayerDesc.gout_plan.offset == 80

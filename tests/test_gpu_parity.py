@@ -694,6 +694,33 @@ def test_second_level_row_set_is_counted_and_compacted(mg, ctx):
     assert mg.ctx_poll_status(ctx, raise_on_error=False) == 0
 
 
+@pytest.mark.parametrize("name", ["messy-directed", "hub"])
+@pytest.mark.parametrize("transposed", [False, True])
+def test_spmm_residual_epilogue(mg, ctx, name, transposed):
+    """Z = gate(relu?(s * R + A_hat Y + bias)): the residual term comes first, then bias and gate."""
+    go, gg = build_both(mg, ctx, name)
+    n, w = go.n, 44
+    Y = synth.uniform_tensor((n, w), 701, -1, 1)
+    R = synth.uniform_tensor((n, w), 702, -1, 1)
+    b = synth.uniform_tensor((w,), 703, -0.5, 0.5)
+    gate = synth.uniform_tensor((n, w), 704, -1, 1)
+    Yd, Rd, gd = padded(Y), padded(R), padded(gate)
+    Z = torch.zeros(n, round4(w), device="cuda")
+    mg.spmm(ctx, gg, Yd, Z, w, transposed=transposed, epi=mg.make_epilogue(bias=b.cuda(), residual=Rd, residual_scale=1.25,
+                                                                              gate=gd, gate_scale=2.0))
+    want = (1.25 * R.numpy() + orc.aggregate(go, Y.numpy(), transposed=transposed) + b.numpy()) * (gate.numpy() > 0) * 2.0
+    assert rel_fro(host(Z, w), want) <= TOL_FP32
+    # the self term with the input itself as residual: (s I + A_hat) Y
+    mg.spmm(ctx, gg, Yd, Z, w, transposed=transposed, epi=mg.make_epilogue(residual=Yd, residual_scale=0.5))
+    assert rel_fro(host(Z, w), 0.5 * Y.numpy() + orc.aggregate(go, Y.numpy(), transposed=transposed)) <= TOL_FP32
+    with pytest.raises(mg.MixgcnError):
+        mg.spmm(ctx, gg, Yd, Z, w, epi=mg.make_epilogue(residual=Z))                     # residual must not be the output
+    with pytest.raises(mg.MixgcnError):
+        mg.gemm(ctx, mg.PREC_FP32, False, False, 8, 8, 8, torch.zeros(8, 8, device="cuda"), torch.zeros(8, 8, device="cuda"),
+                torch.zeros(8, 8, device="cuda"), epi=mg.make_epilogue(residual=torch.zeros(8, 8, device="cuda")))
+    assert mg.ctx_poll_status(ctx, raise_on_error=False) == 0
+
+
 def test_spmm_column_slices_do_not_change_the_result(mg):
     """Feature-column slicing (the p:q-1 ranges of Algorithm 2) is a schedule, not arithmetic."""
     c2 = mg.ctx_create(0)
