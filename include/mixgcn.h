@@ -105,6 +105,15 @@ mixgcn_status mixgcn_ctx_profile_read(mixgcn_ctx* ctx, double ms[MIXGCN_N_PHASES
 #define MIXGCN_GRAPH_SYMMETRISE     1u /* store (v,u) for every (u,v) */
 #define MIXGCN_GRAPH_ADD_SELF_LOOPS 2u /* the "+ I" of Section 2.1 */
 #define MIXGCN_GRAPH_EDGES_ON_DEVICE 4u /* src/dst (or rowptr/col) are device pointers */
+/* Values of the stored matrix.  Default: the symmetric normalisation of Section 2.1,
+ * val_uv = 1/sqrt(deg_u deg_v).  The paper's evaluation also names GraphSAGE and GIN without defining
+ * them; their textbook aggregation matrices are offered on the same structure and kernels:
+ * NORM_ROW  val_uv = 1 / (entries in row u): the row mean (GraphSAGE's mean aggregator); A_hat^T then
+ *           differs from A_hat even on a symmetric structure, and the library keeps its own copy;
+ * NORM_NONE val_uv = 1: the plain sum (GIN's sum aggregator; its (1 + eps) self term is the
+ *           aggregation epilogue's residual).  At most one of the two. */
+#define MIXGCN_GRAPH_NORM_ROW  8u
+#define MIXGCN_GRAPH_NORM_NONE 16u
 
 /* Build from an edge list of m pairs (src[e], dst[e]) meaning entry (src, dst) of A.
  * Input self-loops are dropped, duplicates collapse (A is binary), then one diagonal entry

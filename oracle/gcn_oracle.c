@@ -129,6 +129,26 @@ void oracle_normalise(int64_t n, const int64_t* rowptr, const int32_t* col,
     }
 }
 
+/* Other aggregators on the same stored structure.  The paper evaluates GraphSAGE and GIN besides
+ * GCN (Section 5, "The Model and Datasets") without defining them; these are their textbook
+ * aggregation matrices: mode 1 = row mean, val_uv = 1 / (entries in row u) (GraphSAGE's mean
+ * aggregator), mode 2 = plain sum, val_uv = 1 (GIN's sum aggregator).  val32 follows the fp32
+ * storage recipe: one IEEE division of 1 by the entry count. */
+void oracle_normalise_mode(int64_t n, const int64_t* rowptr, int32_t mode, double* val64, float* val32) {
+    for (int64_t u = 0; u < n; ++u) {
+        int64_t d = rowptr[u + 1] - rowptr[u];
+        for (int64_t i = rowptr[u]; i < rowptr[u + 1]; ++i) {
+            if (mode == 1) {
+                if (val64) val64[i] = 1.0 / (double)d;
+                if (val32) { volatile float r = 1.0f / (float)d; val32[i] = r; }
+            } else {
+                if (val64) val64[i] = 1.0;
+                if (val32) val32[i] = 1.0f;
+            }
+        }
+    }
+}
+
 /* Neighbour aggregation Z = A_hat X (Algorithm 2, aggregation line): row u of Z is the
  * weighted sum of the rows of X listed in row u of the matrix, in ascending column order. */
 void oracle_aggregate(int64_t n, const int64_t* rowptr, const int32_t* col, const double* val,

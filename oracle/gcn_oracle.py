@@ -75,8 +75,12 @@ class Graph:
         return int(self.rowptr[-1])
 
 
-def graph_build(n, src, dst, flags=SYMMETRISE | ADD_SELF_LOOPS) -> Graph:
-    """A_tilde = A + I and A_hat = D^-1/2 A_tilde D^-1/2 (Section 2.1) from an edge list."""
+NORMS = {"sym": 0, "row": 1, "none": 2}
+
+
+def graph_build(n, src, dst, flags=SYMMETRISE | ADD_SELF_LOOPS, norm="sym") -> Graph:
+    """A_tilde = A + I and A_hat = D^-1/2 A_tilde D^-1/2 (Section 2.1) from an edge list.
+    norm = "row": row-mean values (GraphSAGE mean aggregator); "none": ones (GIN sum aggregator)."""
     src = np.ascontiguousarray(src, dtype=np.int32)
     dst = np.ascontiguousarray(dst, dtype=np.int32)
     m = len(src)
@@ -90,10 +94,10 @@ def graph_build(n, src, dst, flags=SYMMETRISE | ADD_SELF_LOOPS) -> Graph:
     L.oracle_graph_build(C.c_int64(n), C.c_int64(m), _p(src, C.c_int32), _p(dst, C.c_int32),
                          C.c_uint32(flags), _p(rowptr, C.c_int64), _p(col, C.c_int32))
     col = col[:nnz]
-    return graph_from_csr(n, rowptr, col)
+    return graph_from_csr(n, rowptr, col, norm)
 
 
-def graph_from_csr(n, rowptr, col) -> Graph:
+def graph_from_csr(n, rowptr, col, norm="sym") -> Graph:
     L = lib()
     rowptr = np.ascontiguousarray(rowptr, dtype=np.int64)
     col = np.ascontiguousarray(col, dtype=np.int32)
@@ -104,6 +108,8 @@ def graph_from_csr(n, rowptr, col) -> Graph:
     deg = np.zeros(n, dtype=np.int32)
     L.oracle_normalise(C.c_int64(n), _p(rowptr, C.c_int64), _p(col, C.c_int32), _p(val, C.c_double),
                        _p(dinv32, C.c_float), _p(val32, C.c_float), _p(deg, C.c_int32))
+    if NORMS[norm] != 0:
+        L.oracle_normalise_mode(C.c_int64(n), _p(rowptr, C.c_int64), C.c_int32(NORMS[norm]), _p(val, C.c_double), _p(val32, C.c_float))
     rowptr_t = np.zeros(n + 1, dtype=np.int64)
     col_t = np.zeros(max(nnz, 1), dtype=np.int32)
     sidx = np.zeros(max(nnz, 1), dtype=np.int64)

@@ -24,6 +24,7 @@ lib = C.CDLL(LIB_PATH)
 
 OK, EINVAL, ENOMEM, ECUDA, EUNSUPPORTED, EBADGRAPH, ETIMEOUT, EDEVICE = range(8)
 GRAPH_SYMMETRISE, GRAPH_ADD_SELF_LOOPS, GRAPH_EDGES_ON_DEVICE = 1, 2, 4
+GRAPH_NORM_ROW, GRAPH_NORM_NONE = 8, 16
 PREC_FP32, PREC_TF32, PREC_BF16 = 0, 1, 2
 ORDER_AUTO, ORDER_AGG_FIRST, ORDER_UPD_FIRST = 0, 1, 2
 LAYER_RELU, LAYER_FIRST, LAYER_GATE_GIN, LAYER_GOUT_GATED, LAYER_OUT_ROWS_ONLY, LAYER_GIN_ROWS_ONLY = 1, 2, 4, 8, 16, 32
@@ -197,11 +198,11 @@ def graph_create(ctx: Ctx, n: int, src: torch.Tensor, dst: torch.Tensor,
     return Graph(ctx, h)
 
 
-def graph_create_from_csr(ctx: Ctx, n: int, rowptr: torch.Tensor, col: torch.Tensor) -> Graph:
+def graph_create_from_csr(ctx: Ctx, n: int, rowptr: torch.Tensor, col: torch.Tensor, flags: int = 0) -> Graph:
     if rowptr.dtype != torch.int64 or col.dtype != torch.int32 or rowptr.numel() != n + 1:
         raise TypeError("graph_create_from_csr: rowptr int64[n+1], col int32[nnz]")
     rowptr, col = rowptr.contiguous(), col.contiguous()
-    flags = GRAPH_EDGES_ON_DEVICE if rowptr.is_cuda else 0
+    flags = (flags & (GRAPH_NORM_ROW | GRAPH_NORM_NONE)) | (GRAPH_EDGES_ON_DEVICE if rowptr.is_cuda else 0)
     if rowptr.is_cuda:
         torch.cuda.current_stream().synchronize()
     h = C.c_void_p()

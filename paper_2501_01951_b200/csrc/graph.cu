@@ -68,14 +68,21 @@ __global__ void degree_kernel(int64_t n, const int64_t* __restrict__ rowptr, int
     dinv[u] = d > 0 ? __frcp_rn(__fsqrt_rn((float)d)) : 0.0f;
 }
 
-// One warp per row: val_uv = dinv_u * dinv_v.
+// One warp per row.  norm 0: val_uv = dinv_u * dinv_v (Section 2.1); 1: 1 / (entries in row u), the row
+// mean (GraphSAGE's mean aggregator); 2: 1, the plain sum (GIN's sum aggregator).
 __global__ void values_kernel(int64_t n, const int64_t* __restrict__ rowptr, const int32_t* __restrict__ col,
-                              const float* __restrict__ dinv, float* __restrict__ val) {
+                              const float* __restrict__ dinv, int norm, float* __restrict__ val) {
     int64_t u = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     int lane = threadIdx.x & 31;
     if (u >= n) return;
-    float du = dinv[u];
-    for (int64_t i = rowptr[u] + lane; i < rowptr[u + 1]; i += 32) val[i] = __fmul_rn(du, dinv[col[i]]);
+    const int64_t b = rowptr[u], e = rowptr[u + 1];
+    if (norm == 0) {
+        float du = dinv[u];
+        for (int64_t i = b + lane; i < e; i += 32) val[i] = __fmul_rn(du, dinv[col[i]]);
+    } else {
+        const float v = norm == 1 ? __frcp_rn((float)(e - b)) : 1.0f;   // IEEE reciprocal of the entry count
+        for (int64_t i = b + lane; i < e; i += 32) val[i] = v;
+    }
 }
 
 // For every stored (u,v), u != v, look v's row up for u.
@@ -380,7 +387,7 @@ mixgcn_status finish_graph(mixgcn_graph* g, cudaStream_t s) {
     MIXGCN_CUDA(cudaMalloc((void**)&g->dinv, n * sizeof(float)));
     MIXGCN_CUDA(cudaMalloc((void**)&A.val, (nnz > 0 ? nnz : 1) * sizeof(float)));
     degree_kernel<<<blocks_for(n), TPB, 0, s>>>(n, A.rowptr, g->deg, g->dinv);
-    values_kernel<<<blocks_for(n * 32), TPB, 0, s>>>(n, A.rowptr, A.col, g->dinv, A.val);
+    values_kernel<<<blocks_for(n * 32), TPB, 0, s>>>(n, A.rowptr, A.col, g->dinv, g->norm, A.val);
     symmetry_kernel<<<blocks_for(n * 32), TPB, 0, s>>>(n, A.rowptr, A.col, flags.as<int32_t>());
     int32_t hf = 0;
     MIXGCN_CUDA(cudaMemcpyAsync(&hf, flags.p, sizeof(hf), cudaMemcpyDeviceToHost, s));
@@ -397,7 +404,8 @@ mixgcn_status finish_graph(mixgcn_graph* g, cudaStream_t s) {
         g->has_diagonal = hd == (unsigned long long)n ? 1 : (hd == 0 ? 0 : 2);
     }
     MIXGCN_TRY(build_schedule(n, A.rowptr, A.col, 0, n, A.full, s));
-    if (g->symmetric) {
+    g->bwd_is_fwd = (g->symmetric && g->norm != 1) ? 1 : 0;   // row-mean values are not symmetric: A_hat^T needs its own copy
+    if (g->bwd_is_fwd) {
         g->bwd = A;  // alias: the same index serves the backward aggregation
         return MIXGCN_OK;
     }
@@ -443,7 +451,7 @@ void release_view(CsrView& v) { free_view(v); }
 
 mixgcn_status ensure_chunk_schedules(const mixgcn_graph* g, const CsrView& A_const, int chunks) {
     // a cache inside the graph object; a symmetric graph keeps one set (in fwd) and mirrors it into the alias
-    CsrView& A = const_cast<CsrView&>(g->symmetric ? g->fwd : A_const);
+    CsrView& A = const_cast<CsrView&>(g->bwd_is_fwd ? g->fwd : A_const);
     if (chunks <= 1 || A.n_chunk == chunks) return MIXGCN_OK;
     MIXGCN_CUDA(cudaDeviceSynchronize());         // earlier launches may still read the schedules being replaced
     for (int k = 0; k < A.n_chunk; ++k) free_schedule(A.chunk[k]);
@@ -462,7 +470,7 @@ mixgcn_status ensure_chunk_schedules(const mixgcn_graph* g, const CsrView& A_con
         }
     }
     A.chunk = sc; A.n_chunk = chunks;
-    if (g->symmetric) const_cast<mixgcn_graph*>(g)->bwd = g->fwd;   // keep the alias in step
+    if (g->bwd_is_fwd) const_cast<mixgcn_graph*>(g)->bwd = g->fwd;   // keep the alias in step
     return MIXGCN_OK;
 }
 
@@ -471,7 +479,7 @@ mixgcn_status ensure_chunk_schedules(const mixgcn_graph* g, const CsrView& A_con
 extern "C" mixgcn_status mixgcn_graph_destroy(mixgcn_graph* g) {
     if (!g) return MIXGCN_OK;
     cudaSetDevice(g->device);
-    if (!g->symmetric) free_view(g->bwd);
+    if (!g->bwd_is_fwd) free_view(g->bwd);
     free_view(g->fwd);
     cudaFree(g->deg);
     cudaFree(g->dinv);
@@ -485,14 +493,16 @@ extern "C" mixgcn_status mixgcn_graph_create(mixgcn_ctx* ctx, int64_t n, int64_t
     if (m < 0 || (m > 0 && (!src || !dst))) MIXGCN_FAIL(MIXGCN_EINVAL, "graph_create: bad edge list (m=%lld)", (long long)m);
     MIXGCN_CUDA(cudaSetDevice(ctx->device));
     cudaStream_t s = ctx->side_stream[0];
+    if ((flags & MIXGCN_GRAPH_NORM_ROW) && (flags & MIXGCN_GRAPH_NORM_NONE)) MIXGCN_FAIL(MIXGCN_EINVAL, "graph_create: NORM_ROW and NORM_NONE exclude each other");
     const int sym = (flags & MIXGCN_GRAPH_SYMMETRISE) != 0, self = (flags & MIXGCN_GRAPH_ADD_SELF_LOOPS) != 0;
     const int64_t total = m * (sym ? 2 : 1) + (self ? n : 0);
 
     mixgcn_graph* g = new (std::nothrow) mixgcn_graph();
     if (g) g->uid = next_graph_uid();
     if (!g) MIXGCN_FAIL(MIXGCN_ENOMEM, "graph_create: host allocation failed");
-    g->ctx = ctx; g->device = ctx->device; g->n = n; g->nnz = 0; g->symmetric = 1;
-    struct Guard { mixgcn_graph* g; bool keep = false; ~Guard() { if (!keep) { g->symmetric = g->bwd.rowptr == g->fwd.rowptr; mixgcn_graph_destroy(g); } } } guard{g};
+    g->ctx = ctx; g->device = ctx->device; g->n = n; g->nnz = 0; g->symmetric = 1; g->bwd_is_fwd = 1;
+    g->norm = (flags & MIXGCN_GRAPH_NORM_ROW) ? 1 : ((flags & MIXGCN_GRAPH_NORM_NONE) ? 2 : 0);
+    struct Guard { mixgcn_graph* g; bool keep = false; ~Guard() { if (!keep) { g->bwd_is_fwd = g->bwd.rowptr == g->fwd.rowptr; mixgcn_graph_destroy(g); } } } guard{g};
     LaunchScope scope(ctx, PH_GRAPH, s, 12);
 
     DevBuf dsrc, ddst, k0, k1, tmp, fl, cnt;
@@ -568,8 +578,9 @@ extern "C" mixgcn_status mixgcn_graph_create_from_csr(mixgcn_ctx* ctx, int64_t n
     mixgcn_graph* g = new (std::nothrow) mixgcn_graph();
     if (g) g->uid = next_graph_uid();
     if (!g) MIXGCN_FAIL(MIXGCN_ENOMEM, "graph_create_from_csr: host allocation failed");
-    g->ctx = ctx; g->device = ctx->device; g->n = n; g->nnz = nnz; g->symmetric = 1;
-    struct Guard { mixgcn_graph* g; bool keep = false; ~Guard() { if (!keep) { g->symmetric = g->bwd.rowptr == g->fwd.rowptr; mixgcn_graph_destroy(g); } } } guard{g};
+    g->ctx = ctx; g->device = ctx->device; g->n = n; g->nnz = nnz; g->symmetric = 1; g->bwd_is_fwd = 1;
+    g->norm = (flags & MIXGCN_GRAPH_NORM_ROW) ? 1 : ((flags & MIXGCN_GRAPH_NORM_NONE) ? 2 : 0);
+    struct Guard { mixgcn_graph* g; bool keep = false; ~Guard() { if (!keep) { g->bwd_is_fwd = g->bwd.rowptr == g->fwd.rowptr; mixgcn_graph_destroy(g); } } } guard{g};
     LaunchScope scope(ctx, PH_GRAPH, s, 8);
     DevBuf fl;
     MIXGCN_CUDA(cudaMalloc(&fl.p, sizeof(int32_t)));

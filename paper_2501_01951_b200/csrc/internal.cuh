@@ -113,7 +113,9 @@ struct mixgcn_graph {
     uint64_t uid;      // unique per created graph (a freed graph's address may be reused)
     int device;        // kept apart from ctx: a graph may be destroyed after its context
     int64_t n, nnz;
-    int symmetric;
+    int symmetric;     // the stored STRUCTURE is symmetric
+    int bwd_is_fwd;    // bwd aliases fwd (symmetric structure and symmetric values)
+    int norm;          // 0 symmetric normalisation, 1 row mean, 2 ones
     int has_diagonal;  // 1: every row stores its diagonal entry, 0: none does, 2: some do
     int32_t* deg;      // [n] entries per row of the stored matrix
     float* dinv;       // [n]

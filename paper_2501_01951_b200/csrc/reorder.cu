@@ -156,5 +156,6 @@ extern "C" mixgcn_status mixgcn_graph_create_permuted(mixgcn_ctx* ctx, const mix
     MIXGCN_CUDA(cudaDeviceSynchronize());
     // Every stored entry is carried over; the diagonal (if the source has one) comes back through ADD_SELF_LOOPS.
     return mixgcn_graph_create(ctx, n, nnz, reinterpret_cast<const int32_t*>(dsrc.p), reinterpret_cast<const int32_t*>(ddst.p),
-                               MIXGCN_GRAPH_EDGES_ON_DEVICE | (g->has_diagonal == 1 ? MIXGCN_GRAPH_ADD_SELF_LOOPS : 0u), out);
+                               MIXGCN_GRAPH_EDGES_ON_DEVICE | (g->has_diagonal == 1 ? MIXGCN_GRAPH_ADD_SELF_LOOPS : 0u) |
+                                   (g->norm == 1 ? MIXGCN_GRAPH_NORM_ROW : (g->norm == 2 ? MIXGCN_GRAPH_NORM_NONE : 0u)), out);
 }

@@ -694,6 +694,32 @@ def test_second_level_row_set_is_counted_and_compacted(mg, ctx):
     assert mg.ctx_poll_status(ctx, raise_on_error=False) == 0
 
 
+@pytest.mark.parametrize("name", ["messy-sym", "messy-directed", "hub"])
+@pytest.mark.parametrize("norm", ["row", "none"])
+def test_graph_aggregator_modes(mg, ctx, name, norm):
+    """Row-mean and plain-sum values: stored values bit-exact against the oracle's fp32 recipe in both
+    orientations, aggregation in both orientations within the fp32 tolerance."""
+    n, s, d, sym = GRAPHS[name]()
+    flags_o = orc.ADD_SELF_LOOPS | (orc.SYMMETRISE if sym else 0)
+    flags_g = mg.GRAPH_ADD_SELF_LOOPS | (mg.GRAPH_SYMMETRISE if sym else 0) | (mg.GRAPH_NORM_ROW if norm == "row" else mg.GRAPH_NORM_NONE)
+    go = orc.graph_build(n, s, d, flags_o, norm=norm)
+    gg = mg.graph_create(ctx, n, i32(s), i32(d), flags_g)
+    ex, ext = mg.graph_export(gg), mg.graph_export(gg, transposed=True)
+    assert np.array_equal(ex["rowptr"].numpy(), go.rowptr) and np.array_equal(ex["col"].numpy(), go.col)
+    assert ex["val"].numpy().tobytes() == go.val32.tobytes()
+    assert np.array_equal(ext["rowptr"].numpy(), go.rowptr_t) and np.array_equal(ext["col"].numpy(), go.col_t)
+    assert ext["val"].numpy().tobytes() == go.val32[go.src_index_t].tobytes()
+    w = 36
+    Y = synth.uniform_tensor((n, w), 801, -1, 1)
+    Z = torch.zeros(n, round4(w), device="cuda")
+    for tr_ in (False, True):
+        mg.spmm(ctx, gg, padded(Y), Z, w, transposed=tr_)
+        assert rel_fro(host(Z, w), orc.aggregate(go, Y.numpy(), transposed=tr_)) <= TOL_FP32
+    with pytest.raises(mg.MixgcnError):
+        mg.graph_create(ctx, n, i32(s), i32(d), mg.GRAPH_NORM_ROW | mg.GRAPH_NORM_NONE)
+    assert mg.ctx_poll_status(ctx, raise_on_error=False) == 0
+
+
 @pytest.mark.parametrize("name", ["messy-directed", "hub"])
 @pytest.mark.parametrize("transposed", [False, True])
 def test_spmm_residual_epilogue(mg, ctx, name, transposed):

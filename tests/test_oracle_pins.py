@@ -216,6 +216,37 @@ def test_adjoint_identity_on_directed_graph():
 
 # ----------------------------------------------------------------------- O3: update / epilogue
 
+@pytest.mark.parametrize("norm", ["row", "none"])
+@pytest.mark.parametrize("sym", [True, False])
+def test_other_aggregators_match_their_definitions(norm, sym):
+    """Row-mean (GraphSAGE mean aggregator) and plain-sum (GIN) values on the stored structure, against
+    the dense matrices written out: A_tilde with rows divided by their entry count, and A_tilde itself."""
+    n = 37
+    rng = np.random.default_rng(5)
+    src, dst = rng.integers(0, 30, 160).astype(np.int32), rng.integers(0, 30, 160).astype(np.int32)   # ids >= 30 stay isolated
+    flags = orc.ADD_SELF_LOOPS | (orc.SYMMETRISE if sym else 0)
+    g = orc.graph_build(n, src, dst, flags, norm=norm)
+    At = np.zeros((n, n))
+    At[src, dst] = 1.0
+    if sym:
+        At[dst, src] = 1.0
+    At[np.arange(n), np.arange(n)] = 1.0
+    dense = At / At.sum(axis=1, keepdims=True) if norm == "row" else At
+    got = np.zeros((n, n)); gotT = np.zeros((n, n))
+    for u in range(n):
+        got[u, g.col[g.rowptr[u]:g.rowptr[u + 1]]] = g.val[g.rowptr[u]:g.rowptr[u + 1]]
+        gotT[u, g.col_t[g.rowptr_t[u]:g.rowptr_t[u + 1]]] = g.val_t[g.rowptr_t[u]:g.rowptr_t[u + 1]]
+    assert np.allclose(got, dense, rtol=0, atol=1e-15) and np.allclose(gotT, dense.T, rtol=0, atol=1e-15)
+    X = rng.standard_normal((n, 5))
+    assert np.allclose(orc.aggregate(g, X), dense @ X, atol=1e-12)
+    assert np.allclose(orc.aggregate(g, X, transposed=True), dense.T @ X, atol=1e-12)
+    if norm == "row":
+        assert np.allclose(orc.aggregate(g, np.ones((n, 1))), 1.0)              # a mean of ones is one
+        assert np.array_equal(g.val32, (np.float32(1.0) / np.diff(g.rowptr).astype(np.float32))[np.repeat(np.arange(n), np.diff(g.rowptr))])
+    else:
+        assert np.array_equal(orc.aggregate(g, np.ones((n, 1)))[:, 0], np.diff(g.rowptr).astype(np.float64))   # row sums = entry counts
+
+
 def test_update_and_activation_vs_numpy():
     rng = np.random.default_rng(4)
     Z, W, b = rng.standard_normal((37, 11)), rng.standard_normal((11, 6)), rng.standard_normal(6)
