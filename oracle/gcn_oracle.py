@@ -267,6 +267,78 @@ def train_epoch(g: Graph, X0, Ws, bs, labels, train_mask, state=None, t=1, lr=0.
 
 # ------------------------------------------------------------------------------ node reordering
 
+# ------------------------------------------------------------------------------ GraphSAGE (mean) and GIN
+# The paper evaluates these two architectures besides GCN (Section 5, "The Model and Datasets") and
+# does not define them; the layers below are their textbook full-graph forms, built from the same
+# aggregation and update steps as the GCN layer, on graphs made with norm="row" (mean of the
+# neighbours, no self loops) and norm="none" (sum of the neighbours, no self loops).
+
+def _adam_all(params, grads, state, t, lr, beta1, beta2, eps):
+    if state is None:
+        state = dict(m=[np.zeros_like(p) for p in params], v=[np.zeros_like(p) for p in params])
+    new = []
+    for i, (p, g) in enumerate(zip(params, grads)):
+        p2, state["m"][i], state["v"][i] = adam(p, g, state["m"][i], state["v"][i], t, lr, beta1, beta2, eps)
+        new.append(p2)
+    return new, state
+
+
+def sage_epoch(g_mean: Graph, X0, Ws_self, Ws_neigh, bs, labels, train_mask, state=None, t=1, lr=0.01,
+               beta1=0.9, beta2=0.999, eps=1e-8):
+    """One training iteration of a mean-aggregator GraphSAGE: H' = sigma(H W_self + (M H) W_neigh + b),
+    M = D^-1 A the row mean over the neighbours, ReLU on every layer but the last; masked softmax
+    cross-entropy; Adam.  Parameter order of the returned lists: W_self[0..L), W_neigh[0..L), b[0..L)."""
+    L = len(Ws_self)
+    Ws_self, Ws_neigh, bs = [_f64(w) for w in Ws_self], [_f64(w) for w in Ws_neigh], [_f64(b) for b in bs]
+    Hs, MHs, Ps = [_f64(X0)], [], []
+    for l in range(L):
+        MH = aggregate(g_mean, Hs[-1])
+        P = Hs[-1] @ Ws_self[l] + MH @ Ws_neigh[l] + bs[l]
+        MHs.append(MH); Ps.append(P)
+        Hs.append(P if l == L - 1 else np.maximum(P, 0.0))
+    lo, G, pred, ncorrect, T = loss(Hs[-1], labels, train_mask)
+    dS, dN, db = [None] * L, [None] * L, [None] * L
+    Gout = G
+    for l in range(L - 1, -1, -1):
+        dP = Gout if l == L - 1 else Gout * (Ps[l] > 0)
+        dS[l], dN[l], db[l] = Hs[l].T @ dP, MHs[l].T @ dP, dP.sum(axis=0)
+        if l > 0:
+            Gout = dP @ Ws_self[l].T + aggregate(g_mean, dP @ Ws_neigh[l].T, transposed=True)
+    params, grads = Ws_self + Ws_neigh + bs, dS + dN + db
+    new, state = _adam_all(params, grads, state, t, lr, beta1, beta2, eps)
+    return dict(loss=lo, logits=Hs[-1], pred=pred, n_correct=ncorrect, G=G, grads=grads, params=new, state=state)
+
+
+def gin_epoch(g_sum: Graph, X0, W1s, b1s, W2s, b2s, labels, train_mask, gin_eps=0.0, state=None, t=1, lr=0.01,
+              beta1=0.9, beta2=0.999, eps=1e-8):
+    """One training iteration of GIN: Z = (1 + gin_eps) H + A H (sum over the neighbours), then a
+    two-layer perceptron H' = sigma(relu(Z W1 + b1) W2 + b2), sigma = ReLU on every layer but the last
+    (gin_eps is a constant here).  Parameter order: W1[0..L), b1[0..L), W2[0..L), b2[0..L)."""
+    L = len(W1s)
+    W1s, b1s, W2s, b2s = ([_f64(x) for x in lst] for lst in (W1s, b1s, W2s, b2s))
+    Hs, Zs, Ts, Ps = [_f64(X0)], [], [], []
+    for l in range(L):
+        Z = (1.0 + gin_eps) * Hs[-1] + aggregate(g_sum, Hs[-1])
+        Tl = np.maximum(Z @ W1s[l] + b1s[l], 0.0)
+        P = Tl @ W2s[l] + b2s[l]
+        Zs.append(Z); Ts.append(Tl); Ps.append(P)
+        Hs.append(P if l == L - 1 else np.maximum(P, 0.0))
+    lo, G, pred, ncorrect, T = loss(Hs[-1], labels, train_mask)
+    dW1, db1, dW2, db2 = [None] * L, [None] * L, [None] * L, [None] * L
+    Gout = G
+    for l in range(L - 1, -1, -1):
+        dP = Gout if l == L - 1 else Gout * (Ps[l] > 0)
+        dW2[l], db2[l] = Ts[l].T @ dP, dP.sum(axis=0)
+        dT = (dP @ W2s[l].T) * (Ts[l] > 0)
+        dW1[l], db1[l] = Zs[l].T @ dT, dT.sum(axis=0)
+        if l > 0:
+            dZ = dT @ W1s[l].T
+            Gout = (1.0 + gin_eps) * dZ + aggregate(g_sum, dZ, transposed=True)
+    params, grads = W1s + b1s + W2s + b2s, dW1 + db1 + dW2 + db2
+    new, state = _adam_all(params, grads, state, t, lr, beta1, beta2, eps)
+    return dict(loss=lo, logits=Hs[-1], pred=pred, n_correct=ncorrect, G=G, grads=grads, params=new, state=state)
+
+
 def bandwidth(g: Graph, order=None) -> int:
     """b = max over stored entries (u,v) of p_v - p_u (Section 3.2.2); order[k] = node at position k."""
     pos = None

@@ -387,6 +387,79 @@ def test_gradients_vs_torch_autograd_on_dense_ahat(directed):
 
 # ----------------------------------------------------------------------- O6: Adam
 
+def _dense_aggregator(n, src, dst, norm):
+    A = np.zeros((n, n))
+    A[src, dst] = 1.0; A[dst, src] = 1.0
+    np.fill_diagonal(A, 0.0)
+    if norm == "row":
+        rs = A.sum(axis=1, keepdims=True)
+        A = np.divide(A, rs, out=np.zeros_like(A), where=rs > 0)
+    return A
+
+
+def _small_model_problem(seed):
+    rng = np.random.default_rng(seed)
+    n, dims = 40, (6, 5, 4, 3)
+    src, dst = rng.integers(0, 34, 120).astype(np.int32), rng.integers(0, 34, 120).astype(np.int32)
+    keep = src != dst
+    src, dst = src[keep], dst[keep]
+    X = rng.standard_normal((n, dims[0]))
+    y = rng.integers(0, dims[-1], n).astype(np.int32)
+    m = (rng.random(n) < 0.5).astype(np.uint8); m[0] = 1
+    return rng, n, dims, src, dst, X, y, m
+
+
+def test_sage_gradients_vs_torch_autograd_on_dense_mean_matrix():
+    """The oracle's GraphSAGE-mean iteration against autograd on the dense row-mean matrix."""
+    rng, n, dims, src, dst, X, y, m = _small_model_problem(11)
+    g = orc.graph_build(n, src, dst, orc.SYMMETRISE, norm="row")
+    Ws = [rng.standard_normal((dims[i], dims[i + 1])) * 0.4 for i in range(3)]
+    Wn = [rng.standard_normal((dims[i], dims[i + 1])) * 0.4 for i in range(3)]
+    bs = [rng.standard_normal(dims[i + 1]) * 0.1 for i in range(3)]
+    ref = orc.sage_epoch(g, X, Ws, Wn, bs, y, m)
+    M = torch.tensor(_dense_aggregator(n, src, dst, "row"))
+    tw = [torch.tensor(w, requires_grad=True) for w in Ws + Wn + bs]
+    H = torch.tensor(X)
+    for l in range(3):
+        P = H @ tw[l] + (M @ H) @ tw[3 + l] + tw[6 + l]
+        H = P if l == 2 else torch.relu(P)
+    idx = torch.tensor(np.nonzero(m)[0])
+    lt = torch.nn.functional.cross_entropy(H[idx], torch.tensor(y, dtype=torch.int64)[idx])
+    lt.backward()
+    assert abs(ref["loss"] - lt.item()) <= 1e-12 * abs(lt.item())
+    for got, t_ in zip(ref["grads"], tw):
+        assert np.allclose(got, t_.grad.numpy(), rtol=1e-10, atol=1e-13)
+    # isolated nodes average nothing: their neighbour term is zero
+    iso = np.setdiff1d(np.arange(n), np.union1d(src, dst))
+    assert len(iso) > 0 and np.all(orc.aggregate(g, X)[iso] == 0.0)
+
+
+@pytest.mark.parametrize("gin_eps", [0.0, 0.3])
+def test_gin_gradients_vs_torch_autograd_on_dense_adjacency(gin_eps):
+    """The oracle's GIN iteration against autograd on the dense adjacency matrix."""
+    rng, n, dims, src, dst, X, y, m = _small_model_problem(12)
+    g = orc.graph_build(n, src, dst, orc.SYMMETRISE, norm="none")
+    hid = 7
+    W1 = [rng.standard_normal((dims[i], hid)) * 0.3 for i in range(3)]
+    b1 = [rng.standard_normal(hid) * 0.1 for i in range(3)]
+    W2 = [rng.standard_normal((hid, dims[i + 1])) * 0.3 for i in range(3)]
+    b2 = [rng.standard_normal(dims[i + 1]) * 0.1 for i in range(3)]
+    ref = orc.gin_epoch(g, X, W1, b1, W2, b2, y, m, gin_eps=gin_eps)
+    A = torch.tensor(_dense_aggregator(n, src, dst, "none"))
+    tw = [torch.tensor(w, requires_grad=True) for w in W1 + b1 + W2 + b2]
+    H = torch.tensor(X)
+    for l in range(3):
+        Z = (1.0 + gin_eps) * H + A @ H
+        P = torch.relu(Z @ tw[l] + tw[3 + l]) @ tw[6 + l] + tw[9 + l]
+        H = P if l == 2 else torch.relu(P)
+    idx = torch.tensor(np.nonzero(m)[0])
+    lt = torch.nn.functional.cross_entropy(H[idx], torch.tensor(y, dtype=torch.int64)[idx])
+    lt.backward()
+    assert abs(ref["loss"] - lt.item()) <= 1e-12 * abs(lt.item())
+    for got, t_ in zip(ref["grads"], tw):
+        assert np.allclose(got, t_.grad.numpy(), rtol=1e-10, atol=1e-13)
+
+
 def test_adam_closed_forms():
     rng = np.random.default_rng(8)
     th0, g = rng.standard_normal(50), rng.standard_normal(50)
