@@ -311,6 +311,12 @@ mixgcn_status mixgcn_spmm_rowplan(mixgcn_ctx* ctx, const mixgcn_rowplan* plan, i
                                   int64_t ldy, float* Z, int64_t ldz, const mixgcn_epilogue* epi,
                                   int32_t rows_only, void* stream);
 
+/* out[j] = sum_i X[i*ld + j] for j < d (the bias gradient of an update, db = 1^T dP): per-block
+ * partial sums in a fixed order, then one pass over the partials in fp64.  X is n x ld on the device,
+ * out has d floats. */
+mixgcn_status mixgcn_colsum(mixgcn_ctx* ctx, int64_t n, int32_t d, const float* X, int64_t ld, float* out,
+                            void* stream);
+
 /* Resolves MIXGCN_ORDER_AUTO: cost(agg-first) = c * d_in with c = 1 for a FIRST layer (its
  * backward needs no aggregation) else 2; cost(upd-first) = 2 * d_out; the smaller wins, ties
  * go to agg-first.  *saved_cols receives the number of columns the `saved` buffer needs

@@ -43,7 +43,7 @@ SYMBOLS = (
     "mixgcn_adam_step", "mixgcn_train_step_host", "mixgcn_loss_softmax_xent_noalloc", "mixgcn_ctx_set_option",
     "mixgcn_graph_bandwidth", "mixgcn_graph_rcm", "mixgcn_pipeline_stages", "mixgcn_graph_create_permuted",
     "mixgcn_count_rows", "mixgcn_rowplan_create", "mixgcn_rowplan_destroy", "mixgcn_rowplan_info",
-    "mixgcn_rowplan_export", "mixgcn_spmm_rowplan",
+    "mixgcn_rowplan_export", "mixgcn_spmm_rowplan", "mixgcn_colsum",
 )
 
 
@@ -295,6 +295,13 @@ def gemm(ctx: Ctx, precision: int, trans_a: bool, trans_b: bool, M: int, N: int,
 
 
 # ------------------------------------------------------------------------------ layers
+
+def colsum(ctx: Ctx, X: torch.Tensor, out: torch.Tensor, d: int):
+    """out[j] = sum over rows of X[:, j], j < d."""
+    X, ld = _mat(X, "X")
+    _dev(out, torch.float32, "out")
+    _check(lib.mixgcn_colsum(ctx.h, C.c_int64(X.shape[0]), C.c_int32(d), _ptr(X), C.c_int64(ld), _ptr(out), _stream()))
+
 
 def layer_desc(d_in, d_out, ld_in, ld_out, ld_saved, order=ORDER_AUTO, precision=PREC_FP32, flags=0,
                keep_scale=1.0, in_scale=1.0, n_chunks=0) -> LayerDesc:

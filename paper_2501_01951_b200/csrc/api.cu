@@ -274,6 +274,14 @@ inline int64_t chunk_bound(int64_t k, int i, int m) { return (k * (int64_t)i) / 
 
 }  // namespace
 
+extern "C" mixgcn_status mixgcn_colsum(mixgcn_ctx* ctx, int64_t n, int32_t d, const float* X, int64_t ld, float* out,
+                                       void* stream) {
+    if (!ctx || !X || !out) MIXGCN_FAIL(MIXGCN_EINVAL, "colsum: null argument");
+    if (n <= 0 || d <= 0 || ld < d) MIXGCN_FAIL(MIXGCN_EINVAL, "colsum: need n > 0, d > 0 and ld >= d");
+    MIXGCN_CUDA(cudaSetDevice(ctx->device));
+    return launch_colsum(ctx, n, d, X, ld, out, (cudaStream_t)stream);
+}
+
 extern "C" mixgcn_status mixgcn_layer_plan(const mixgcn_layer_desc* desc, int32_t* order, int32_t* saved_cols) {
     if (!desc) MIXGCN_FAIL(MIXGCN_EINVAL, "layer_plan: null descriptor");
     if (desc->d_in <= 0 || desc->d_out <= 0 || desc->order < 0 || desc->order > 2)
