@@ -4,6 +4,7 @@ and as a small, self-ending target for profiler captures.
     python -m paper_2501_01951_b200.microbench --op spmm --n 4000000 --edges 32000000 --w 128
     python -m paper_2501_01951_b200.microbench --op gemm --M 1000000 --N 1024 --K 1024 --precision tf32
     python -m paper_2501_01951_b200.microbench --op loss --n 4000000 --w 172 --mask-p 0.01 --loss-rows 0
+    python -m paper_2501_01951_b200.microbench --op model --model sage --n 2449029 --edges 61859140 --dims 100,128,128,47 --precision tf32
 
 Prints one JSON line with the median time and the derived algorithmic GB/s or TFLOP/s.
 """
@@ -36,7 +37,7 @@ def _time(fn, iters, warmup):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--op", required=True, choices=["spmm", "gemm", "loss"])
+    ap.add_argument("--op", required=True, choices=["spmm", "gemm", "loss", "model"])
     ap.add_argument("--n", type=int, default=1 << 20)
     ap.add_argument("--edges", type=int, default=8 << 20, help="distinct undirected edges of the R-MAT graph")
     ap.add_argument("--w", type=int, default=128)
@@ -49,7 +50,10 @@ def main():
     ap.add_argument("--iters", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=2)
     ap.add_argument("--seed", type=int, default=1005)
-    ap.add_argument("--mask-p", type=float, default=0.01, help="loss: fraction of train rows")
+    ap.add_argument("--model", default="sage", choices=["gcn", "sage", "gin"], help="model: architecture of the timed training epochs")
+    ap.add_argument("--dims", default="128,128,128,64", help="model: layer widths d_0,...,d_L")
+    ap.add_argument("--hidden", type=int, default=128, help="model: width of GIN's inner perceptron layer")
+    ap.add_argument("--mask-p", type=float, default=0.01, help="loss / model: fraction of train rows")
     ap.add_argument("--loss-rows", type=int, default=0, choices=[0, 1, 2], help="loss: MIXGCN_OPT_LOSS_TRAIN_ROWS_ONLY value")
     ap.add_argument("--slice", type=int, default=0, help="feature-column slice width of the aggregation (0 = default)")
     args = ap.parse_args()
@@ -70,6 +74,45 @@ def main():
         alg = 8 * (g.n + 1) + 8 * g.nnz + 8 * g.n * args.w
         out.update(n=g.n, nnz=g.nnz, w=args.w, max_deg=g.max_deg, ms_median=round(med, 4), ms_best=round(best, 4),
                    alg_bytes=alg, alg_gbs=round(alg / med / 1e6, 1), gather_gbs=round(4 * g.nnz * args.w / med / 1e6, 1))
+    elif args.op == "model":
+        from .sage_gin import GinTrainer, SageTrainer
+        from .train import GcnTrainer
+        dims = tuple(int(x) for x in args.dims.split(","))
+        L = len(dims) - 1
+        s, d = synth.rmat_graph(args.n, args.edges, args.seed, device=dev)
+        norm = {"gcn": mg.GRAPH_ADD_SELF_LOOPS, "sage": mg.GRAPH_NORM_ROW, "gin": mg.GRAPH_NORM_NONE}[args.model]
+        g = mg.graph_create(ctx, args.n, s, d, mg.GRAPH_SYMMETRISE | norm)
+        del s, d
+        torch.cuda.empty_cache()
+        prec = mg.PRECISIONS[args.precision]
+        X0 = synth.normal_features(args.n, dims[0], 7, device=dev, ld=(dims[0] + 3) // 4 * 4)
+        y = synth.uniform_labels(args.n, dims[-1], 8, device=dev)
+        m = synth.bernoulli_mask(args.n, args.mask_p, 9, device=dev)
+        W = lambda a, b, k, scale=1.0: synth.glorot_uniform(a, b, k, device=dev) * scale
+        zb = lambda k: torch.zeros(k, device=dev)
+        if args.model == "gcn":
+            tr = GcnTrainer(ctx, g, dims, prec)
+            tr.set_params([W(dims[i], dims[i + 1], 20 + i) for i in range(L)], [zb(dims[i + 1]) for i in range(L)])
+            tr.set_inputs(X0, y, m)
+        elif args.model == "sage":
+            tr = SageTrainer(ctx, g, dims, prec)
+            tr.set_params([W(dims[i], dims[i + 1], 20 + i) for i in range(L)], [W(dims[i], dims[i + 1], 40 + i) for i in range(L)],
+                          [zb(dims[i + 1]) for i in range(L)])
+            tr.set_inputs(X0, y, m)
+        else:
+            tr = GinTrainer(ctx, g, dims, args.hidden, prec)
+            tr.set_params([W(dims[i], args.hidden, 20 + i, 0.05) for i in range(L)], [zb(args.hidden) for i in range(L)],
+                          [W(args.hidden, dims[i + 1], 40 + i) for i in range(L)], [zb(dims[i + 1]) for i in range(L)])
+            tr.set_inputs(X0, y, m)
+        step = [0]
+
+        def one():
+            step[0] += 1
+            tr.epoch(step[0])
+        med, best = _time(one, args.iters, args.warmup)
+        out.update(model=args.model, n=g.n, nnz=g.nnz, dims=list(dims), precision=args.precision, loss=round(tr.loss.item(), 6),
+                   ms_median=round(med, 4), ms_best=round(best, 4), epochs_per_s=round(1e3 / med, 3),
+                   device_status=mg.ctx_poll_status(ctx, raise_on_error=False))
     elif args.op == "loss":
         n, C = args.n, args.w
         ld = (C + 3) // 4 * 4
