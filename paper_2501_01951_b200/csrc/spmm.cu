@@ -38,7 +38,7 @@ using namespace mixgcn;
 #define MIXGCN_SPMM_SHORT_RB 4       // rows a warp of the short-row kernel takes at once
 #endif
 #ifndef MIXGCN_SPMM_SHORT_MINB
-#define MIXGCN_SPMM_SHORT_MINB 6     // CTAs per SM asked of the compiler for it
+#define MIXGCN_SPMM_SHORT_MINB 5     // CTAs per SM asked of the compiler for it
 #endif
 #ifndef MIXGCN_SPMM_SHORT_MAXE
 #define MIXGCN_SPMM_SHORT_MAXE 2     // 0 = rows of 1..2 entries go through the packed group kernel
