@@ -69,8 +69,9 @@ mixgcn_status mixgcn_ctx_reserve(mixgcn_ctx* ctx, int64_t bytes);
 mixgcn_status mixgcn_ctx_poll_status(mixgcn_ctx* ctx, int32_t* code);
 
 /* Tuning options.  MIXGCN_OPT_SPMM_SLICE_COLS: width of the feature-column slices an aggregation is
- * processed in (Algorithm 2's p:q-1 column ranges on one GPU): 0 = one slice up to 1024 columns
- * (default); otherwise a multiple of 4 in [4, 1024].  Narrow slices shrink the part of the input
+ * processed in (Algorithm 2's p:q-1 column ranges on one GPU): 0 = slices of 256 columns (default:
+ * the two-float4-per-lane kernels keep four CTAs per SM; measured fastest at width 1024); otherwise
+ * a multiple of 4 in [4, 1024].  Narrow slices shrink the part of the input
  * that must stay in the L2 at the price of re-reading the index once per slice; results do not
  * depend on the slicing. */
 #define MIXGCN_OPT_SPMM_SLICE_COLS 1

@@ -456,7 +456,8 @@ void dispatch_filtered(const SpmmParams& p, cudaStream_t s) {
     }
 }
 
-constexpr int MAX_SLICE = 1024;  // columns per launch: 8 float4 per lane
+constexpr int MAX_SLICE = 1024;      // columns per launch at most: 8 float4 per lane
+constexpr int DEFAULT_SLICE = 256;   // widths above this run as slices of this many columns (2 float4 per lane, four CTAs per SM)
 
 }  // namespace
 
@@ -490,7 +491,7 @@ mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView&
     p.rec = S.rec;
     if (sparse) { p.in_mask = sparse->in_mask; p.in_pos = sparse->in_pos; p.out_mask = sparse->out_mask; }
     p.row_filter = row_filter;
-    const int slice = ctx->spmm_slice_cols > 0 ? ctx->spmm_slice_cols : MAX_SLICE;
+    const int slice = ctx->spmm_slice_cols > 0 ? (ctx->spmm_slice_cols < MAX_SLICE ? ctx->spmm_slice_cols : MAX_SLICE) : DEFAULT_SLICE;
     for (int j0 = 0; j0 < w; j0 += slice) {
         p.j0 = j0;
         p.w = (w - j0) < slice ? (w - j0) : slice;
