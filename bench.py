@@ -35,8 +35,8 @@ import torch
 from paper_2501_01951_b200 import synth
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of ONE aggregation call at the workload's
-# size and width, from the ncu capture summarised in profiles/spmm_C5_dram_traffic.md (every
-# aggregation of C5 has width 128 and the same graph, so the figure holds for each of its calls).
+# size and width, from a single-pass ncu capture of one call at full size, summarised under profiles/
+# (every aggregation of C5 has width 128 and the same graph, so the figure holds for each of its calls).
 NCU_SPMM_CALL_DRAM_BYTES = {"C5": 131232026368}
 
 METRIC = "full-graph GCN train epochs/s"
