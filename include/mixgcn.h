@@ -83,7 +83,21 @@ mixgcn_status mixgcn_ctx_poll_status(mixgcn_ctx* ctx, int32_t* code);
  * the dlogits rows of non-train nodes are left UNCHANGED instead of zeroed: for a backward pass that
  * reads train rows only (gout_plan, or gout_row_mask with a count below n/4 in agg-first order). */
 #define MIXGCN_OPT_LOSS_TRAIN_ROWS_ONLY 2
+/* Test hooks of the bounded device-side waits (the failure-detection path), both 0 by default.
+ * MIXGCN_OPT_DEBUG_WAIT_LIMIT: > 0 = number of polls after which a wait inside the tensor-core kernels
+ * gives up (default about four million).  MIXGCN_OPT_DEBUG_DROP_LOAD: 1 = the next tensor-core products
+ * in the K-major form leave the first stage of every CTA unfilled, so that the wait on it runs out: the
+ * kernel records code 3 in the status word, frees its tensor memory and returns with C undefined;
+ * mixgcn_ctx_poll_status then gives MIXGCN_ETIMEOUT.  Nothing traps, spins without limit or faults. */
+#define MIXGCN_OPT_DEBUG_WAIT_LIMIT 3
+#define MIXGCN_OPT_DEBUG_DROP_LOAD 4
 mixgcn_status mixgcn_ctx_set_option(mixgcn_ctx* ctx, int32_t option, int64_t value);
+
+/* Which kernel served the dense products of this context since it was created: counts[0] fp32 FMA
+ * kernel, counts[1] tcgen05 with TF32 operands, counts[2] tcgen05 with BF16 operands.  A TF32 or BF16
+ * request whose shape or alignment the tensor-core kernels do not take is served by the next kernel
+ * down that list (never a lower precision than asked for); these counters make that visible. */
+mixgcn_status mixgcn_ctx_gemm_paths(const mixgcn_ctx* ctx, int64_t counts[3]);
 
 /* Per-phase profiling.  While enabled the library brackets every kernel it launches with
  * CUDA events on the launching stream.  mixgcn_ctx_profile_read synchronises and returns, for
@@ -206,7 +220,8 @@ mixgcn_status mixgcn_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, int transposed
 
 #define MIXGCN_PREC_FP32 0 /* fp32 FMA on the CUDA cores */
 #define MIXGCN_PREC_TF32 1 /* tensor cores, TF32 operands, fp32 accumulate */
-#define MIXGCN_PREC_BF16 2 /* tensor cores, BF16 operands, fp32 accumulate */
+#define MIXGCN_PREC_BF16 2 /* tensor cores, BF16 operands (the fp32 operands rounded to nearest even),
+                              fp32 accumulate, fp32 results */
 
 /* Dense update GEMM  C = op(A) op(B)  with fp32 storage (Algorithm 2, update line, and its
  * two backward products).  op(A) is M x K, op(B) is K x N, C is M x N row-major with ldc.
@@ -283,6 +298,29 @@ typedef struct {
      * can be non-zero are the plan's out_row_mask; with MIXGCN_LAYER_GIN_ROWS_ONLY only those rows of
      * G_in are written (for a layer below that itself runs with a plan made from that mask). */
     const mixgcn_rowplan* gout_plan;
+    /* bf16 companions of the activations, used with MIXGCN_PREC_BF16 only (all optional).  The dense
+     * products then read bf16 operands; the kernel that PRODUCES an activation (the aggregation's or the
+     * update's epilogue) writes its bf16 copy beside the fp32 one, so no product has to convert its
+     * operand first.  A NULL companion is replaced by a conversion pass inside the call (same result,
+     * one more read of the fp32 operand).  Device uint16 (bf16 bits), 16-byte aligned, n rows; leading
+     * dimensions in bf16 elements, multiples of 8, at least the tensor's width.
+     *   saved_lp   n x ld_saved_lp   copy of `saved`: written by layer_fwd (agg-first: bf16(A_hat X_in)) and
+     *                                read by layer_bwd; upd-first backward uses it as scratch.  With
+     *                                MIXGCN_LAYER_SAVED_IS_VALID it must be valid as well.
+     *   x_in_lp    n x ld_in_lp      copy of X_in, read (upd-first order: forward product and dW)
+     *   x_out_lp   n x ld_out_lp     layer_fwd writes the copy of X_out (the next layer's x_in_lp)
+     *   g_out_lp   n x ld_out_lp     layer_bwd reads the copy of G_out; used only when G_out arrives
+     *                                already gated (MIXGCN_LAYER_GOUT_GATED, or a layer without ReLU and
+     *                                dropout), i.e. when this call does not change G_out first
+     *   g_in_lp    n x ld_in_lp      layer_bwd writes the copy of G_in (the layer below's g_out_lp) */
+    uint16_t* saved_lp;
+    int64_t ld_saved_lp;
+    const uint16_t* x_in_lp;
+    int64_t ld_in_lp;
+    uint16_t* x_out_lp;
+    int64_t ld_out_lp;
+    uint16_t* g_out_lp;
+    uint16_t* g_in_lp;
 } mixgcn_layer_desc;
 
 /* Row plan of a row-sparse aggregation.  Which rows of a gradient are non-zero depends on the graph
@@ -314,6 +352,7 @@ mixgcn_status mixgcn_spmm_rowplan(mixgcn_ctx* ctx, const mixgcn_rowplan* plan, i
 
 /* out[j] = sum_i X[i*ld + j] for j < d (the bias gradient of an update, db = 1^T dP): per-block
  * partial sums in a fixed order, then one pass over the partials in fp64.  X is n x ld on the device,
+ * 16-byte aligned with ld a multiple of 4 (the activations' layout; MIXGCN_EINVAL otherwise);
  * out has d floats. */
 mixgcn_status mixgcn_colsum(mixgcn_ctx* ctx, int64_t n, int32_t d, const float* X, int64_t ld, float* out,
                             void* stream);
@@ -371,11 +410,13 @@ mixgcn_status mixgcn_loss_softmax_xent(mixgcn_ctx* ctx, int64_t n, int32_t C, co
  * process exits.
  *  - Runs on the calling thread's CURRENT device; all pointers are device pointers of it.
  *  - Arguments and results as mixgcn_loss_softmax_xent; `status` (device int32, nullable)
- *    receives 0, 1 (empty train mask) or 2 (label outside [0,C)) when the stream reaches it.
+ *    receives 0, 1 (empty train mask), 2 (label outside [0,C)) or 3 (a bounded wait inside the
+ *    kernel gave up; loss, dlogits and pred are then undefined) when the stream reaches it.
  *  - Limit: n <= 33,554,432 rows (32768 partials x 1024 rows) and 1 <= C <= 4096; larger sizes
  *    return MIXGCN_EUNSUPPORTED and launch nothing.
  *  - The first call on each device looks up the scratch array's device address (one
- *    cudaGetSymbolAddress, cached per device); make that first call before any stream capture.
+ *    cudaGetSymbolAddress, cached per device in an atomic pointer, so host threads may race to be
+ *    first); make that first call before any stream capture.
  *  - All calls on a device share the one array, which keeps the previous call's contents; each
  *    call clears the counter and status word first.  Two calls that overlap on the GPU (different
  *    streams, no ordering between them) race on it: order them. */

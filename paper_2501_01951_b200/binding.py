@@ -43,7 +43,7 @@ SYMBOLS = (
     "mixgcn_adam_step", "mixgcn_train_step_host", "mixgcn_loss_softmax_xent_noalloc", "mixgcn_ctx_set_option",
     "mixgcn_graph_bandwidth", "mixgcn_graph_rcm", "mixgcn_pipeline_stages", "mixgcn_graph_create_permuted",
     "mixgcn_count_rows", "mixgcn_rowplan_create", "mixgcn_rowplan_destroy", "mixgcn_rowplan_info",
-    "mixgcn_rowplan_export", "mixgcn_spmm_rowplan", "mixgcn_colsum",
+    "mixgcn_rowplan_export", "mixgcn_spmm_rowplan", "mixgcn_colsum", "mixgcn_ctx_gemm_paths",
 )
 
 
@@ -59,7 +59,9 @@ class LayerDesc(C.Structure):
                 ("ld_saved", C.c_int64), ("order", C.c_int32), ("precision", C.c_int32),
                 ("flags", C.c_uint32), ("keep_scale", C.c_float), ("in_scale", C.c_float),
                 ("n_chunks", C.c_int32), ("gout_row_mask", C.c_void_p), ("gout_row_count", C.c_int64),
-                ("gin_row_mask", C.c_void_p), ("gout_plan", C.c_void_p)]
+                ("gin_row_mask", C.c_void_p), ("gout_plan", C.c_void_p),
+                ("saved_lp", C.c_void_p), ("ld_saved_lp", C.c_int64), ("x_in_lp", C.c_void_p), ("ld_in_lp", C.c_int64),
+                ("x_out_lp", C.c_void_p), ("ld_out_lp", C.c_int64), ("g_out_lp", C.c_void_p), ("g_in_lp", C.c_void_p)]
 
 
 lib.mixgcn_status_string.restype = C.c_char_p
@@ -141,10 +143,19 @@ def ctx_poll_status(ctx: Ctx, raise_on_error: bool = True) -> int:
 
 OPT_SPMM_SLICE_COLS = 1
 OPT_LOSS_TRAIN_ROWS_ONLY = 2
+OPT_DEBUG_WAIT_LIMIT = 3
+OPT_DEBUG_DROP_LOAD = 4
 
 
 def ctx_set_option(ctx: Ctx, option: int, value: int):
     _check(lib.mixgcn_ctx_set_option(ctx.h, C.c_int32(option), C.c_int64(value)))
+
+
+def ctx_gemm_paths(ctx: Ctx) -> dict:
+    """Dense products served so far by the fp32 FMA kernel, the tcgen05 TF32 kernels, the tcgen05 BF16 kernels."""
+    counts = (C.c_int64 * 3)()
+    _check(lib.mixgcn_ctx_gemm_paths(ctx.h, counts))
+    return dict(simt=int(counts[0]), tc_tf32=int(counts[1]), tc_bf16=int(counts[2]))
 
 
 def ctx_profile_enable(ctx: Ctx, enable: bool = True):

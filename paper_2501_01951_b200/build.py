@@ -21,7 +21,7 @@ LIB = os.path.join(HERE, "libmixgcn.so")
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
 CFLAGS = ["-O3", "-std=c++17", "-lineinfo", "-Xcompiler", "-fPIC",
-          "-I", INCLUDE, "-I", CSRC, "--expt-relaxed-constexpr"] + os.environ.get("MIXGCN_NVCC_FLAGS", "").split()
+          "-I", os.path.relpath(INCLUDE, CSRC), "-I", ".", "--expt-relaxed-constexpr"]   # relative: nvcc runs inside csrc/
 
 
 def sources():
@@ -38,11 +38,13 @@ def _compile(src, force, verbose):
     obj = os.path.join(OBJDIR, os.path.basename(src)[:-3] + ".o")
     stale = force or not os.path.exists(obj) or os.path.getmtime(obj) < max(os.path.getmtime(src), _deps_mtime())
     if stale:
-        cmd = [NVCC, *ARCH, *CFLAGS, "-c", src, "-o", obj]
+        # compiled from inside csrc/ under its bare file name, so that __FILE__ in error strings is
+        # "graph.cu", not a path of the build machine
+        cmd = [NVCC, *ARCH, *CFLAGS, "-c", os.path.basename(src), "-o", obj]
         if verbose:
             cmd.insert(1, "-Xptxas")
             cmd.insert(2, "-v")
-        r = subprocess.run(cmd, capture_output=True, text=True)
+        r = subprocess.run(cmd, capture_output=True, text=True, cwd=CSRC)
         if verbose or r.returncode != 0:
             sys.stderr.write(r.stdout + r.stderr)
         if r.returncode != 0:

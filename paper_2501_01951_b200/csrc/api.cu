@@ -81,25 +81,73 @@ mixgcn_status ensure_workspace_spmm(mixgcn_ctx* ctx, int64_t bytes) {
     return MIXGCN_OK;
 }
 
-mixgcn_status launch_gemm_simt(mixgcn_ctx* ctx, int ta, int tb, int64_t M, int64_t N, int64_t K,
-                               const float* A, int64_t lda, const float* B, int64_t ldb, float* C, int64_t ldc,
-                               const mixgcn_epilogue* epi, int64_t epi_row0, cudaStream_t s);
-
-mixgcn_status launch_gemm_tc(mixgcn_ctx* ctx, int ta, int tb, int64_t M, int64_t N, int64_t K, const float* A,
-                             int64_t lda, const float* B, int64_t ldb, float* C, int64_t ldc,
-                             const mixgcn_epilogue* epi, int64_t epi_row0, cudaStream_t s);
+mixgcn_status ensure_workspace_lp(mixgcn_ctx* ctx, int64_t bytes) {
+    if (bytes <= ctx->workspace_lp_bytes) return MIXGCN_OK;
+    int64_t want = bytes + (bytes >> 3);
+    want = (want + 255) & ~(int64_t)255;
+    void* p = nullptr;
+    MIXGCN_CUDA(cudaDeviceSynchronize());
+    if (ctx->workspace_lp) cudaFree(ctx->workspace_lp);
+    ctx->workspace_lp = nullptr; ctx->workspace_lp_bytes = 0;
+    if (cudaMalloc(&p, (size_t)want) != cudaSuccess) {
+        cudaGetLastError();
+        MIXGCN_FAIL(MIXGCN_ENOMEM, "bf16 operand workspace of %lld bytes could not be allocated", (long long)want);
+    }
+    ctx->workspace_lp = p; ctx->workspace_lp_bytes = want;
+    return MIXGCN_OK;
+}
 
 mixgcn_status launch_gemm(mixgcn_ctx* ctx, int precision, int ta, int tb, int64_t M, int64_t N, int64_t K,
                           const float* A, int64_t lda, const float* B, int64_t ldb, float* C, int64_t ldc,
-                          const mixgcn_epilogue* epi, int64_t epi_row0, cudaStream_t s) {
-    // TF32 / BF16 requests go to the tcgen05 kernels (TF32 operands serve both: at least the requested
-    // precision); shapes or alignments they do not take, and fp32 requests, use the FMA kernel.
-    static const bool disable_tc = getenv("MIXGCN_DISABLE_TC") != nullptr;
-    if (precision != MIXGCN_PREC_FP32 && !disable_tc) {
-        mixgcn_status st = launch_gemm_tc(ctx, ta, tb, M, N, K, A, lda, B, ldb, C, ldc, epi, epi_row0, s);
-        if (st != MIXGCN_EUNSUPPORTED) return st;
+                          const mixgcn_epilogue* epi, int64_t epi_row0, cudaStream_t s, const GemmLP* lp) {
+    // BF16 requests go to the tcgen05 kind::f16 kernels on bf16 copies of the activation operands: the
+    // copies a producer already wrote (lp), else copies made here by a conversion kernel.  TF32
+    // requests, and BF16 requests whose shape the bf16 kernels do not take, go to the kind::tf32
+    // kernels (at least the requested precision); whatever those do not take, and fp32 requests, use the
+    // FMA kernel.  ctx->gemm_path counts which kernel served each product.
+    uint16_t* c_lp = lp ? lp->C : nullptr;
+    const int64_t ldc_lp = lp ? lp->ldc : 0;
+    bool c_lp_done = false;
+    mixgcn_status st = MIXGCN_EUNSUPPORTED;
+    const bool fp32_layout = aligned16(A) && (lda & 3) == 0 && (!ta || (aligned16(B) && (ldb & 3) == 0));
+    if (precision == MIXGCN_PREC_BF16 && !(ta && tb) && fp32_layout && M > 0 && N > 0 && K > 0) {
+        auto round8 = [](int64_t x) { return (x + 7) & ~(int64_t)7; };
+        auto up = [](int64_t x) { return (x + 255) & ~(int64_t)255; };
+        const int64_t a_rows = ta ? K : M, a_cols = ta ? M : K;
+        const uint16_t* a_lp = lp ? lp->A : nullptr;
+        int64_t lda_lp = lp ? lp->lda : 0;
+        const uint16_t* b_lp = (ta && lp) ? lp->B : nullptr;
+        int64_t ldb_lp = (ta && lp) ? lp->ldb : 0;
+        const int64_t need_a = a_lp ? 0 : up(a_rows * round8(a_cols) * 2);
+        const int64_t need_b = (ta && !b_lp) ? up(K * round8(N) * 2) : 0;
+        if (need_a + need_b > 0) MIXGCN_TRY(ensure_workspace_lp(ctx, need_a + need_b));
+        if (!a_lp) {
+            uint16_t* dst = reinterpret_cast<uint16_t*>(ctx->workspace_lp);
+            lda_lp = round8(a_cols);
+            MIXGCN_TRY(launch_to_bf16(ctx, a_rows, (int32_t)a_cols, A, lda, dst, lda_lp, s));
+            a_lp = dst;
+        }
+        if (ta && !b_lp) {
+            uint16_t* dst = reinterpret_cast<uint16_t*>(reinterpret_cast<char*>(ctx->workspace_lp) + need_a);
+            ldb_lp = round8(N);
+            MIXGCN_TRY(launch_to_bf16(ctx, K, (int32_t)N, B, ldb, dst, ldb_lp, s));
+            b_lp = dst;
+        }
+        st = launch_gemm_tc(ctx, 1, ta, tb, M, N, K, a_lp, lda_lp, ta ? (const void*)b_lp : (const void*)B, ta ? ldb_lp : ldb,
+                            C, ldc, epi, epi_row0, s, ta ? nullptr : c_lp, ldc_lp);
+        if (st == MIXGCN_OK) { ctx->gemm_path[2]++; c_lp_done = !ta && c_lp; }
     }
-    return launch_gemm_simt(ctx, ta, tb, M, N, K, A, lda, B, ldb, C, ldc, epi, epi_row0, s);
+    if (st == MIXGCN_EUNSUPPORTED && precision != MIXGCN_PREC_FP32) {
+        st = launch_gemm_tc(ctx, 0, ta, tb, M, N, K, A, lda, B, ldb, C, ldc, epi, epi_row0, s, ta ? nullptr : c_lp, ldc_lp);
+        if (st == MIXGCN_OK) { ctx->gemm_path[1]++; c_lp_done = !ta && c_lp; }
+    }
+    if (st == MIXGCN_EUNSUPPORTED) {
+        st = launch_gemm_simt(ctx, ta, tb, M, N, K, A, lda, B, ldb, C, ldc, epi, epi_row0, s);
+        if (st == MIXGCN_OK) ctx->gemm_path[0]++;
+    }
+    if (st != MIXGCN_OK) return st;
+    if (c_lp && !c_lp_done) MIXGCN_TRY(launch_to_bf16(ctx, M, (int32_t)N, C, ldc, c_lp, ldc_lp, s));
+    return MIXGCN_OK;
 }
 
 }  // namespace mixgcn
@@ -160,6 +208,7 @@ extern "C" mixgcn_status mixgcn_ctx_destroy(mixgcn_ctx* ctx) {
     cudaFree(ctx->workspace);
     cudaFree(ctx->workspace_spmm);
     cudaFree(ctx->workspace_rows);
+    cudaFree(ctx->workspace_lp);
     cudaFree(ctx->arena);
     cudaFree(ctx->d_status);
     delete ctx;
@@ -198,7 +247,23 @@ extern "C" mixgcn_status mixgcn_ctx_set_option(mixgcn_ctx* ctx, int32_t option, 
         ctx->loss_train_rows_only = (int)value;
         return MIXGCN_OK;
     }
+    if (option == MIXGCN_OPT_DEBUG_WAIT_LIMIT) {
+        if (value < 0 || value > (1ll << 30)) MIXGCN_FAIL(MIXGCN_EINVAL, "ctx_set_option: wait limit must lie in [0, 2^30] (got %lld)", (long long)value);
+        ctx->debug_wait_limit = (int)value;
+        return MIXGCN_OK;
+    }
+    if (option == MIXGCN_OPT_DEBUG_DROP_LOAD) {
+        if (value != 0 && value != 1) MIXGCN_FAIL(MIXGCN_EINVAL, "ctx_set_option: drop-load takes 0 or 1 (got %lld)", (long long)value);
+        ctx->debug_drop_load = (int)value;
+        return MIXGCN_OK;
+    }
     MIXGCN_FAIL(MIXGCN_EINVAL, "ctx_set_option: unknown option %d", option);
+}
+
+extern "C" mixgcn_status mixgcn_ctx_gemm_paths(const mixgcn_ctx* ctx, int64_t counts[3]) {
+    if (!ctx || !counts) MIXGCN_FAIL(MIXGCN_EINVAL, "ctx_gemm_paths: null argument");
+    for (int i = 0; i < 3; ++i) counts[i] = ctx->gemm_path[i];
+    return MIXGCN_OK;
 }
 
 extern "C" mixgcn_status mixgcn_ctx_profile_enable(mixgcn_ctx* ctx, int enable) {
@@ -266,8 +331,28 @@ mixgcn_status check_desc(const mixgcn_layer_desc* d, const char* who) {
     if (d->ld_in < d->d_in || d->ld_out < d->d_out || d->ld_saved < saved_cols || (d->ld_in & 3) || (d->ld_out & 3) || (d->ld_saved & 3))
         MIXGCN_FAIL(MIXGCN_EINVAL, "%s: leading dimensions must be multiples of 4 with ld_in >= d_in, ld_out >= d_out, ld_saved >= %d", who, saved_cols);
     if (d->n_chunks < 0 || d->n_chunks > 64) MIXGCN_FAIL(MIXGCN_EINVAL, "%s: n_chunks must lie in [0, 64]", who);
+    // bf16 companions: 16-byte aligned, leading dimensions multiples of 8 that cover the width
+    auto lp_ok = [](const void* ptr, int64_t ld, int64_t cols) { return !ptr || (aligned16(ptr) && (ld & 7) == 0 && ld >= cols); };
+    if (!lp_ok(d->saved_lp, d->ld_saved_lp, saved_cols) || !lp_ok(d->x_in_lp, d->ld_in_lp, d->d_in) || !lp_ok(d->g_in_lp, d->ld_in_lp, d->d_in) ||
+        !lp_ok(d->x_out_lp, d->ld_out_lp, d->d_out) || !lp_ok(d->g_out_lp, d->ld_out_lp, d->d_out))
+        MIXGCN_FAIL(MIXGCN_EINVAL, "%s: bf16 companions must be 16-byte aligned with leading dimensions that are multiples of 8 and cover the width", who);
     return MIXGCN_OK;
 }
+
+// The bf16 companions of a layer are used only when its dense products run in BF16.
+struct LayerLP {
+    uint16_t* saved; int64_t ld_saved;
+    const uint16_t* x_in; int64_t ld_in;
+    uint16_t* x_out; uint16_t* g_out; int64_t ld_out;
+    uint16_t* g_in;
+    explicit LayerLP(const mixgcn_layer_desc* d) {
+        const bool on = d->precision == MIXGCN_PREC_BF16;
+        saved = on ? d->saved_lp : nullptr; ld_saved = d->ld_saved_lp;
+        x_in = on ? d->x_in_lp : nullptr; ld_in = d->ld_in_lp;
+        x_out = on ? d->x_out_lp : nullptr; g_out = on ? d->g_out_lp : nullptr; ld_out = d->ld_out_lp;
+        g_in = on ? d->g_in_lp : nullptr;
+    }
+};
 
 // Row range of chunk i of m over k rows: the floor(k*i/m) boundaries of Algorithm 2's update loop.
 inline int64_t chunk_bound(int64_t k, int i, int m) { return (k * (int64_t)i) / m; }
@@ -278,6 +363,7 @@ extern "C" mixgcn_status mixgcn_colsum(mixgcn_ctx* ctx, int64_t n, int32_t d, co
                                        void* stream) {
     if (!ctx || !X || !out) MIXGCN_FAIL(MIXGCN_EINVAL, "colsum: null argument");
     if (n <= 0 || d <= 0 || ld < d) MIXGCN_FAIL(MIXGCN_EINVAL, "colsum: need n > 0, d > 0 and ld >= d");
+    if (!aligned16(X) || (ld & 3)) MIXGCN_FAIL(MIXGCN_EINVAL, "colsum: X must be 16-byte aligned with ld a multiple of 4 (ld=%lld)", (long long)ld);
     MIXGCN_CUDA(cudaSetDevice(ctx->device));
     return launch_colsum(ctx, n, d, X, ld, out, (cudaStream_t)stream);
 }
@@ -344,12 +430,15 @@ extern "C" mixgcn_status mixgcn_layer_fwd(mixgcn_ctx* ctx, const mixgcn_graph* g
         return MIXGCN_OK;
     }
 
+    const LayerLP lp(d);
     if (order == MIXGCN_ORDER_AGG_FIRST) {
+        SpmmOpts agg_opts; agg_opts.Z_lp = lp.saved; agg_opts.ldz_lp = lp.ld_saved;     // the aggregation also writes bf16(A_hat X)
         if (chunks == 1) {
             if (!saved_valid)
-                MIXGCN_TRY(launch_spmm(ctx, g, g->fwd, 1, 0, d->d_in, X_in, d->ld_in, saved, d->ld_saved, nullptr, s));
+                MIXGCN_TRY(launch_spmm(ctx, g, g->fwd, 1, 0, d->d_in, X_in, d->ld_in, saved, d->ld_saved, nullptr, s, agg_opts));
+            GemmLP glp; glp.A = lp.saved; glp.lda = lp.ld_saved; glp.C = lp.x_out; glp.ldc = lp.ld_out;
             MIXGCN_TRY(launch_gemm(ctx, d->precision, 0, 0, n, d->d_out, d->d_in, saved, d->ld_saved, W, ldw, X_out,
-                                   d->ld_out, &epi, 0, s));
+                                   d->ld_out, &epi, 0, s, &glp));
             return MIXGCN_OK;
         }
         // aggregation of chunk k+1 on stream A overlaps the update of chunk k on stream B
@@ -361,11 +450,17 @@ extern "C" mixgcn_status mixgcn_layer_fwd(mixgcn_ctx* ctx, const mixgcn_graph* g
         for (int k = 0; k < chunks; ++k) {
             const int64_t r0 = chunk_bound(n, k, chunks), r1 = chunk_bound(n, k + 1, chunks);
             if (r1 <= r0) continue;
-            MIXGCN_TRY(launch_spmm(ctx, g, g->fwd, chunks, k, d->d_in, X_in, d->ld_in, saved, d->ld_saved, nullptr, sa));
+            MIXGCN_TRY(launch_spmm(ctx, g, g->fwd, chunks, k, d->d_in, X_in, d->ld_in, saved, d->ld_saved, nullptr, sa, agg_opts));
             MIXGCN_CUDA(cudaEventRecord(ctx->chunk_ev[k], sa));
             MIXGCN_CUDA(cudaStreamWaitEvent(sb, ctx->chunk_ev[k], 0));
-            MIXGCN_TRY(launch_gemm(ctx, d->precision, 0, 0, r1 - r0, d->d_out, d->d_in, saved + r0 * d->ld_saved,
-                                   d->ld_saved, W, ldw, X_out + r0 * d->ld_out, d->ld_out, &epi, r0, sb));
+            // without the caller's bf16 copy of `saved` a BF16 product would convert into the one shared
+            // workspace from two streams: the chunks then run TF32 (at least the requested precision)
+            GemmLP glp;
+            glp.A = lp.saved ? lp.saved + r0 * lp.ld_saved : nullptr; glp.lda = lp.ld_saved;
+            glp.C = lp.x_out ? lp.x_out + r0 * lp.ld_out : nullptr; glp.ldc = lp.ld_out;
+            const int prec_k = (d->precision == MIXGCN_PREC_BF16 && !lp.saved) ? MIXGCN_PREC_TF32 : d->precision;
+            MIXGCN_TRY(launch_gemm(ctx, prec_k, 0, 0, r1 - r0, d->d_out, d->d_in, saved + r0 * d->ld_saved,
+                                   d->ld_saved, W, ldw, X_out + r0 * d->ld_out, d->ld_out, &epi, r0, sb, &glp));
         }
         MIXGCN_CUDA(cudaEventRecord(ctx->join_ev[0], sa));
         MIXGCN_CUDA(cudaEventRecord(ctx->join_ev[1], sb));
@@ -375,9 +470,13 @@ extern "C" mixgcn_status mixgcn_layer_fwd(mixgcn_ctx* ctx, const mixgcn_graph* g
     }
     // update first: Q = X_in W (into `saved`), then X_out = epilogue(A_hat Q).  Every row of Q is
     // needed before any aggregated row can be produced, so there is nothing to chunk here.
-    MIXGCN_TRY(launch_gemm(ctx, d->precision, 0, 0, n, d->d_out, d->d_in, X_in, d->ld_in, W, ldw, saved, d->ld_saved,
-                           nullptr, 0, s));
-    MIXGCN_TRY(launch_spmm(ctx, g, g->fwd, 1, 0, d->d_out, saved, d->ld_saved, X_out, d->ld_out, &epi, s));
+    {
+        GemmLP glp; glp.A = lp.x_in; glp.lda = lp.ld_in;
+        MIXGCN_TRY(launch_gemm(ctx, d->precision, 0, 0, n, d->d_out, d->d_in, X_in, d->ld_in, W, ldw, saved, d->ld_saved,
+                               nullptr, 0, s, &glp));
+    }
+    SpmmOpts out_opts; out_opts.Z_lp = lp.x_out; out_opts.ldz_lp = lp.ld_out;
+    MIXGCN_TRY(launch_spmm(ctx, g, g->fwd, 1, 0, d->d_out, saved, d->ld_saved, X_out, d->ld_out, &epi, s, out_opts));
     return MIXGCN_OK;
 }
 
@@ -400,8 +499,11 @@ extern "C" mixgcn_status mixgcn_layer_bwd(mixgcn_ctx* ctx, const mixgcn_graph* g
     const int64_t ldw = d->d_out;
 
     // gradient w.r.t. the pre-activation, in place in G_out
-    if (!(d->flags & MIXGCN_LAYER_GOUT_GATED) && (relu || drop_mask))
+    LayerLP lp(d);
+    if (!(d->flags & MIXGCN_LAYER_GOUT_GATED) && (relu || drop_mask)) {
         MIXGCN_TRY(launch_gate(ctx, n, d->d_out, G_out, d->ld_out, X_out, d->ld_out, relu, drop_mask, d->keep_scale, s));
+        lp.g_out = nullptr;      // the caller's bf16 copy predates the gate
+    }
 
     mixgcn_epilogue gin_epi{};
     const mixgcn_epilogue* gin = nullptr;
@@ -422,6 +524,8 @@ extern "C" mixgcn_status mixgcn_layer_bwd(mixgcn_ctx* ctx, const mixgcn_graph* g
         // rows of the restricted matrix are scheduled longest first: its non-empty rows are the first out_count
         SpmmOpts plan_all; plan_all.phase = PH_SPMM_SPARSE;
         SpmmOpts plan_opts = plan_all; plan_opts.row_limit = (d->flags & MIXGCN_LAYER_GIN_ROWS_ONLY) ? plan->out_count : -1;
+        plan_opts.Z_lp = lp.g_in; plan_opts.ldz_lp = lp.ld_in;
+        plan_all.Z_lp = lp.saved; plan_all.ldz_lp = lp.ld_saved;
         MIXGCN_TRY(launch_gather_rows(ctx, cnt, d->d_out, plan->idx, G_out, d->ld_out, cb, ldb, s));         // dP_T
         if (dbias) MIXGCN_TRY(launch_colsum(ctx, cnt, d->d_out, cb, ldb, dbias, s));
         if (order == MIXGCN_ORDER_AGG_FIRST) {
@@ -435,14 +539,19 @@ extern "C" mixgcn_status mixgcn_layer_bwd(mixgcn_ctx* ctx, const mixgcn_graph* g
         }
         // update first: dQ = A_hat^T dZ from the compacted rows (into `saved`, every row), then the dense products
         MIXGCN_TRY(launch_spmm(ctx, g, plan->view, 1, 0, d->d_out, cb, ldb, saved, d->ld_saved, nullptr, s, plan_all));
-        MIXGCN_TRY(launch_gemm(ctx, d->precision, 1, 0, d->d_in, d->d_out, n, X_in, d->ld_in, saved, d->ld_saved, dW, ldw, nullptr, 0, s));
-        if (!first)
-            MIXGCN_TRY(launch_gemm(ctx, d->precision, 0, 1, n, d->d_in, d->d_out, saved, d->ld_saved, W, ldw, G_in, d->ld_in, gin, 0, s));
+        GemmLP wlp; wlp.A = lp.x_in; wlp.lda = lp.ld_in; wlp.B = lp.saved; wlp.ldb = lp.ld_saved;
+        MIXGCN_TRY(launch_gemm(ctx, d->precision, 1, 0, d->d_in, d->d_out, n, X_in, d->ld_in, saved, d->ld_saved, dW, ldw, nullptr, 0, s, &wlp));
+        if (!first) {
+            GemmLP xlp; xlp.A = lp.saved; xlp.lda = lp.ld_saved; xlp.C = lp.g_in; xlp.ldc = lp.ld_in;
+            MIXGCN_TRY(launch_gemm(ctx, d->precision, 0, 1, n, d->d_in, d->d_out, saved, d->ld_saved, W, ldw, G_in, d->ld_in, gin, 0, s, &xlp));
+        }
         return MIXGCN_OK;
     }
     const uint8_t* rmask = d->gout_row_mask;
     SpmmRowSparse sp{rmask, nullptr, d->gin_row_mask};
     SpmmOpts sparse_opts; sparse_opts.sparse = rmask ? &sp : nullptr;
+    SpmmOpts gin_opts = sparse_opts; gin_opts.Z_lp = lp.g_in; gin_opts.ldz_lp = lp.ld_in;         // aggregations that produce G_in
+    SpmmOpts dq_opts = sparse_opts; dq_opts.Z_lp = lp.saved; dq_opts.ldz_lp = lp.ld_saved;        // upd-first: dQ into `saved`
 
     if (order == MIXGCN_ORDER_AGG_FIRST) {
         const int64_t cnt = d->gout_row_count;
@@ -460,18 +569,20 @@ extern "C" mixgcn_status mixgcn_layer_bwd(mixgcn_ctx* ctx, const mixgcn_graph* g
             if (!first) {
                 MIXGCN_TRY(launch_gemm(ctx, d->precision, 0, 1, cnt, d->d_in, d->d_out, rs.b, ldb, W, ldw, rs.a, lda, nullptr, 0, s));
                 sp.in_pos = rs.pos;                                                                             // dZ_T is compact
-                MIXGCN_TRY(launch_spmm(ctx, g, g->bwd, 1, 0, d->d_in, rs.a, lda, G_in, d->ld_in, gin, s, sparse_opts));
+                MIXGCN_TRY(launch_spmm(ctx, g, g->bwd, 1, 0, d->d_in, rs.a, lda, G_in, d->ld_in, gin, s, gin_opts));
             }
             return MIXGCN_OK;
         }
         // dW = (A_hat X_in)^T dP ; dZ = dP W^T (over `saved`) ; G_in = A_hat^T dZ
         if (dbias) MIXGCN_TRY(launch_colsum(ctx, n, d->d_out, G_out, d->ld_out, dbias, s));
+        GemmLP wlp; wlp.A = lp.saved; wlp.lda = lp.ld_saved; wlp.B = lp.g_out; wlp.ldb = lp.ld_out;
         MIXGCN_TRY(launch_gemm(ctx, d->precision, 1, 0, d->d_in, d->d_out, n, saved, d->ld_saved, G_out, d->ld_out, dW,
-                               ldw, nullptr, 0, s));
+                               ldw, nullptr, 0, s, &wlp));
         if (!first) {
+            GemmLP zlp; zlp.A = lp.g_out; zlp.lda = lp.ld_out;
             MIXGCN_TRY(launch_gemm(ctx, d->precision, 0, 1, n, d->d_in, d->d_out, G_out, d->ld_out, W, ldw, saved,
-                                   d->ld_saved, nullptr, 0, s));
-            MIXGCN_TRY(launch_spmm(ctx, g, g->bwd, 1, 0, d->d_in, saved, d->ld_saved, G_in, d->ld_in, gin, s, sparse_opts));
+                                   d->ld_saved, nullptr, 0, s, &zlp));
+            MIXGCN_TRY(launch_spmm(ctx, g, g->bwd, 1, 0, d->d_in, saved, d->ld_saved, G_in, d->ld_in, gin, s, gin_opts));
         }
         return MIXGCN_OK;
     }
@@ -492,11 +603,14 @@ extern "C" mixgcn_status mixgcn_layer_bwd(mixgcn_ctx* ctx, const mixgcn_graph* g
     } else if (dbias) {
         MIXGCN_TRY(launch_colsum(ctx, n, d->d_out, G_out, d->ld_out, dbias, s));
     }
-    MIXGCN_TRY(launch_spmm(ctx, g, g->bwd, 1, 0, d->d_out, G_out, d->ld_out, saved, d->ld_saved, nullptr, s, sparse_opts));
+    MIXGCN_TRY(launch_spmm(ctx, g, g->bwd, 1, 0, d->d_out, G_out, d->ld_out, saved, d->ld_saved, nullptr, s, dq_opts));
+    GemmLP wlp; wlp.A = lp.x_in; wlp.lda = lp.ld_in; wlp.B = lp.saved; wlp.ldb = lp.ld_saved;
     MIXGCN_TRY(launch_gemm(ctx, d->precision, 1, 0, d->d_in, d->d_out, n, X_in, d->ld_in, saved, d->ld_saved, dW, ldw,
-                           nullptr, 0, s));
-    if (!first)
+                           nullptr, 0, s, &wlp));
+    if (!first) {
+        GemmLP xlp; xlp.A = lp.saved; xlp.lda = lp.ld_saved; xlp.C = lp.g_in; xlp.ldc = lp.ld_in;
         MIXGCN_TRY(launch_gemm(ctx, d->precision, 0, 1, n, d->d_in, d->d_out, saved, d->ld_saved, W, ldw, G_in, d->ld_in,
-                               gin, 0, s));
+                               gin, 0, s, &xlp));
+    }
     return MIXGCN_OK;
 }

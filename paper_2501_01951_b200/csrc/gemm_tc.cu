@@ -1,34 +1,50 @@
 // Dense update products on the 5th-generation tensor cores (tcgen05) for sm_100a:
 // the update line of Algorithm 2 (P = Z W) and its two backward products (dZ = dP W^T,
-// dW = Z^T dP) with TF32 operands read straight from the fp32 activations and fp32 accumulation
-// in tensor memory.
+// dW = Z^T dP) with fp32 accumulation in tensor memory, in two operand kinds:
+//   TF32 -- operands read straight from the fp32 activations (tcgen05.mma.kind::tf32);
+//   BF16 -- operands are bf16 copies of the activations (tcgen05.mma.kind::f16), half the bytes per
+//           operand element on the way from the L2 to shared memory and into the tensor core.
+// The two kinds share every line of the kernels except the element size: a stage row is 128 bytes of
+// K (32 fp32 or 64 bf16) and one instruction consumes 32 bytes of it (K = 8 or 16).
 //
 //  * Operands reach shared memory by TMA (cp.async.bulk.tensor, 128-byte swizzle, out-of-bounds
 //    elements filled with zeros, so ragged M / N / K tails need no special code).
-//  * One elected thread issues tcgen05.mma (M = 128, N <= 256, K = 8 per instruction); the
-//    128 x N fp32 accumulator lives in TMEM and is read back by four warps with tcgen05.ld for the
-//    fused epilogue (bias, ReLU, dropout mask, gate) and the single store of C.
-//  * Warp roles: warps 0-3 epilogue (TMEM lane quarter = warp id), warp 4 TMA producer,
-//    warp 5 TMEM allocation + MMA issue.  Stages are handed over with mbarriers; every wait is
-//    bounded: on expiry the CTA records DEV_WAIT_EXPIRED in the status word, stops issuing work,
-//    frees its TMEM and returns.
+//  * One elected thread issues tcgen05.mma (M = 128, N <= 256); the 128 x N fp32 accumulator lives in
+//    TMEM and is read back with tcgen05.ld for the fused epilogue (bias, ReLU, dropout mask, gate), the
+//    single store of C and, on request, a bf16 copy of C for the next product.
+//  * Stages are handed over with mbarriers; every wait is bounded: on expiry the CTA records
+//    DEV_WAIT_EXPIRED in the status word, stops issuing work, frees its TMEM and returns.
 //  * Two operand forms.  "KK": A is M x K row-major (K contiguous) and B is N x K row-major -- the
 //    forward product and dZ, with the small weight matrix first packed (transposed if needed, zero
-//    padded) into the workspace.  "MM": A is K x M and B is K x N row-major (M / N contiguous,
-//    K = node count) -- the weight gradient, split over CTAs along K into partial tiles that the
-//    fixed-order fp64 reduction combines.
+//    padded, converted to the kind's type) into the workspace.  "MM": A is K x M and B is K x N
+//    row-major (M / N contiguous, K = node count) -- the weight gradient, split over CTAs along K into
+//    partial tiles that the fixed-order fp64 reduction combines.
 #include <cuda.h>
 
 #include "internal.cuh"
+#include "tc_ptx.cuh"
 
 using namespace mixgcn;
+using namespace mixgcn::tc;
 
 namespace {
 
 constexpr int TC_BM = 128;          // rows of D per CTA = UMMA M
-constexpr int TC_BK = 32;           // fp32 elements per stage along K (one 128-byte swizzle row / 32 k-rows)
 constexpr int TC_THREADS = 192;
-constexpr uint32_t WAIT_LIMIT = 1u << 22;
+
+// What differs between the operand kinds.
+template <int KIND>
+struct KindCfg {
+    static constexpr int EB = KIND == KIND_TF32 ? 4 : 2;        // bytes per operand element
+    static constexpr int BK = 128 / EB;                         // elements of K per stage (one 128-byte swizzle row; BK k-rows in the MN-major form)
+    static constexpr int MMA_K = 32 / EB;                       // K of one tcgen05.mma
+    // MN-major form: a chunk is 128 bytes of M / N (BK elements wide) by BK k-rows
+    static constexpr int CHUNK = 128 / EB;                      // elements of M / N per chunk
+    static constexpr uint32_t MN_LAYOUT = KIND == KIND_TF32 ? 1u : 2u;
+    static constexpr uint32_t MN_SBO = KIND == KIND_TF32 ? 512u : 1024u;   // one K atom (4 / 8 k-rows of 128 bytes)
+    static constexpr uint32_t MN_CHUNK_BYTES = BK * 128;        // = leading byte offset
+    static constexpr uint32_t MN_STEP = MMA_K * 128;            // k-rows of one instruction
+};
 
 struct TcEpi {
     const float* bias; int relu;
@@ -42,98 +58,16 @@ struct TcParams {
     int bn;                 // UMMA N: multiple of 16, 16..256
     int stages;
     int64_t m_tiles, n_tiles;
-    int64_t k_per_split;    // MM form: multiple of TC_BK
+    int64_t k_per_split;    // MM form: multiple of the kind's BK
     int splits;
     float* C; int64_t ldc; int vec_c;
+    uint16_t* C_lp; int64_t ldc_lp;   // nullable: bf16 copy of C (after the epilogue); ldc_lp a multiple of 8
     int raw;                // 1: store the accumulator unchanged (split-K partial)
     TcEpi epi;
     int32_t* status;
+    uint32_t wait_limit;    // polls after which a wait gives up
+    int debug_drop_load;    // test hook: the producer leaves out the loads of its first stage (the wait on it then expires)
 };
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-    return ok != 0;
-}
-// Bounded wait: false when the limit is reached (the caller then abandons the tile).
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-    for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 1023u) == 1023u && *abort_flag) return false;
-    }
-    return false;
-}
-__device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* map, int32_t c0, int32_t c1, uint64_t* bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-__device__ __forceinline__ void tc_commit(uint64_t* bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void tc_mma_tf32(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr) : "memory");
-}
-__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-// Shared-memory matrix descriptor, 128-byte swizzle, version 1 (sm_100).
-//   K-major operand (rows of 128 bytes = 32 fp32 along K, 8-row groups of 1024 bytes):
-//     leading byte offset unused (1), stride byte offset = 1024.
-//   MN-major TF32 operand (k-rows of 128 bytes = 32 fp32 along M/N; one 32-wide chunk holds TC_BK
-//     k-rows): only the 128-byte swizzle with 32-byte atoms is defined for it (layout type 1; the
-//     TMA counterpart is SWIZZLE_128B_ATOM_32B); its K atom is 4 k-rows, so the stride byte offset
-//     is 512 and the leading byte offset is the distance between 32-wide chunks.
-__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint32_t layout_type) {
-    uint64_t d = 0;
-    d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
-    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
-    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
-    d |= (uint64_t)1 << 46;   // descriptor version
-    d |= (uint64_t)layout_type << 61;   // 2 = SWIZZLE_128B, 1 = SWIZZLE_128B with 32-byte atoms
-    return d;
-}
-
-// Instruction descriptor: fp32 accumulate, TF32 x TF32, dense, M = 128.
-__host__ __device__ inline uint32_t make_idesc_tf32(int n, bool mn_major) {
-    uint32_t d = 0;
-    d |= 1u << 4;                       // D format F32
-    d |= 2u << 7;                       // A format TF32
-    d |= 2u << 10;                      // B format TF32
-    if (mn_major) d |= (1u << 15) | (1u << 16);
-    d |= (uint32_t)(n >> 3) << 17;
-    d |= (uint32_t)(TC_BM >> 4) << 24;
-    return d;
-}
 
 __device__ __forceinline__ float tc_apply_epi(const TcEpi& e, float y, int64_t m, int64_t n, int64_t N) {
     if (e.bias) y += e.bias[n];
@@ -143,18 +77,37 @@ __device__ __forceinline__ float tc_apply_epi(const TcEpi& e, float y, int64_t m
     return y;
 }
 
-template <bool MN_MAJOR>
+// 32 consecutive columns of one row as bf16 (round to nearest even); dst is 16-byte aligned when full.
+__device__ __forceinline__ void store_lp_row(uint16_t* dst, const float (&v)[32], int valid) {
+    if (valid >= 32) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+            reinterpret_cast<uint4*>(dst)[q] = make_uint4(pack_bf16(v[8 * q], v[8 * q + 1]), pack_bf16(v[8 * q + 2], v[8 * q + 3]),
+                                                           pack_bf16(v[8 * q + 4], v[8 * q + 5]), pack_bf16(v[8 * q + 6], v[8 * q + 7]));
+    } else {
+#pragma unroll
+        for (int q = 0; q < 32; ++q)
+            if (q < valid) dst[q] = (uint16_t)(pack_bf16(v[q], 0.0f) & 0xFFFFu);
+    }
+}
+
+// One output tile per CTA; MN_MAJOR = true is the split-K weight-gradient form (grid.z = split).
+// Warp roles: warps 0-3 epilogue (TMEM lane quarter = warp id), warp 4 TMA producer, warp 5 TMEM
+// allocation + MMA issue.
+template <int KIND, bool MN_MAJOR>
 __global__ void __launch_bounds__(TC_THREADS) gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a,
                                                              const __grid_constant__ CUtensorMap map_b,
                                                              const TcParams p) {
+    using Cfg = KindCfg<KIND>;
+    constexpr int BK = Cfg::BK;
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t full_bar[8], empty_bar[8], acc_bar;
     __shared__ uint32_t tmem_holder;
     __shared__ int abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int bn32 = (p.bn + 31) & ~31;
-    const uint32_t a_bytes = TC_BM * TC_BK * 4, b_bytes = (uint32_t)bn32 * TC_BK * 4;
+    const int bn_pad = MN_MAJOR ? (p.bn + Cfg::CHUNK - 1) / Cfg::CHUNK * Cfg::CHUNK : (p.bn + 31) & ~31;
+    const uint32_t a_bytes = TC_BM * 128, b_bytes = (uint32_t)bn_pad * 128;
     const uint32_t stage_bytes = a_bytes + b_bytes;
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
 
@@ -165,7 +118,7 @@ __global__ void __launch_bounds__(TC_THREADS) gemm_tc_kernel(const __grid_consta
         kb = (int64_t)blockIdx.z * p.k_per_split;
         ke = kb + p.k_per_split < p.K ? kb + p.k_per_split : p.K;
     }
-    const int nk = (int)((ke - kb + TC_BK - 1) / TC_BK);
+    const int nk = (int)((ke - kb + BK - 1) / BK);
     uint32_t tmem_cols = 32;
     while ((int)tmem_cols < p.bn) tmem_cols <<= 1;
 
@@ -191,44 +144,44 @@ __global__ void __launch_bounds__(TC_THREADS) gemm_tc_kernel(const __grid_consta
             for (int ks = 0; ks < nk; ++ks) {
                 const int s = ks % p.stages;
                 const uint32_t ph = ((ks / p.stages) & 1) ^ 1;
-                if (!mbar_wait(&empty_bar[s], ph, &abort_flag)) { abort_flag = 1; atomicMax(p.status, DEV_WAIT_EXPIRED); break; }
+                if (!mbar_wait(&empty_bar[s], ph, &abort_flag, p.wait_limit)) { abort_flag = 1; atomicMax(p.status, DEV_WAIT_EXPIRED); break; }
                 uint8_t* sa = smem + (size_t)s * stage_bytes;
                 uint8_t* sb = sa + a_bytes;
                 mbar_expect_tx(&full_bar[s], stage_bytes);
-                const int32_t k0 = (int32_t)(kb + (int64_t)ks * TC_BK);
+                const int32_t k0 = (int32_t)(kb + (int64_t)ks * BK);
                 if (!MN_MAJOR) {
-                    tma_load_2d(sa, &map_a, k0, (int32_t)m0, &full_bar[s]);                  // 128 rows x 32 k
-                    tma_load_2d(sb, &map_b, k0, (int32_t)n0, &full_bar[s]);                  // bn32 rows x 32 k
+                    tma_load_2d(sa, &map_a, k0, (int32_t)m0, &full_bar[s]);                  // 128 rows x 128 bytes of k
+                    tma_load_2d(sb, &map_b, k0, (int32_t)n0, &full_bar[s]);                  // bn_pad rows x 128 bytes of k
                 } else {
-                    for (int c = 0; c < TC_BM / 32; ++c)                                      // 32 k-rows x 32 m each
-                        tma_load_2d(sa + c * (TC_BK * 128), &map_a, (int32_t)(m0 + 32 * c), k0, &full_bar[s]);
-                    for (int c = 0; c < bn32 / 32; ++c)
-                        tma_load_2d(sb + c * (TC_BK * 128), &map_b, (int32_t)(n0 + 32 * c), k0, &full_bar[s]);
+                    for (int c = 0; c < TC_BM / Cfg::CHUNK; ++c)                              // BK k-rows x 128 bytes of m each
+                        tma_load_2d(sa + c * Cfg::MN_CHUNK_BYTES, &map_a, (int32_t)(m0 + Cfg::CHUNK * c), k0, &full_bar[s]);
+                    for (int c = 0; c < bn_pad / Cfg::CHUNK; ++c)
+                        tma_load_2d(sb + c * Cfg::MN_CHUNK_BYTES, &map_b, (int32_t)(n0 + Cfg::CHUNK * c), k0, &full_bar[s]);
                 }
             }
         }
     } else if (warp == 5) {
         if (lane == 0) {
             // ---------------- MMA issuer ----------------
-            const uint32_t idesc = make_idesc_tf32(p.bn, MN_MAJOR);
+            const uint32_t idesc = make_idesc<KIND>(TC_BM, p.bn, MN_MAJOR);
             bool ok = true;
             for (int ks = 0; ks < nk && ok; ++ks) {
                 const int s = ks % p.stages;
                 const uint32_t ph = (ks / p.stages) & 1;
-                if (!mbar_wait(&full_bar[s], ph, &abort_flag)) { abort_flag = 1; atomicMax(p.status, DEV_WAIT_EXPIRED); ok = false; break; }
+                if (!mbar_wait(&full_bar[s], ph, &abort_flag, p.wait_limit)) { abort_flag = 1; atomicMax(p.status, DEV_WAIT_EXPIRED); ok = false; break; }
                 tc_fence_after();
                 const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes), sb = sa + a_bytes;
 #pragma unroll
-                for (int k8 = 0; k8 < TC_BK / 8; ++k8) {
+                for (int kq = 0; kq < BK / Cfg::MMA_K; ++kq) {
                     uint64_t ad, bd;
                     if (!MN_MAJOR) {
-                        ad = make_desc(sa + k8 * 32, 16, 1024, 2);
-                        bd = make_desc(sb + k8 * 32, 16, 1024, 2);
+                        ad = make_desc(sa + kq * 32, 16, 1024, 2);
+                        bd = make_desc(sb + kq * 32, 16, 1024, 2);
                     } else {
-                        ad = make_desc(sa + k8 * 1024, TC_BK * 128, 512, 1);
-                        bd = make_desc(sb + k8 * 1024, TC_BK * 128, 512, 1);
+                        ad = make_desc(sa + kq * Cfg::MN_STEP, Cfg::MN_CHUNK_BYTES, Cfg::MN_SBO, Cfg::MN_LAYOUT);
+                        bd = make_desc(sb + kq * Cfg::MN_STEP, Cfg::MN_CHUNK_BYTES, Cfg::MN_SBO, Cfg::MN_LAYOUT);
                     }
-                    tc_mma_tf32(tmem_base, ad, bd, idesc, (ks | k8) != 0 ? 1u : 0u);
+                    tc_mma<KIND>(tmem_base, ad, bd, idesc, (ks | kq) != 0 ? 1u : 0u);
                 }
                 tc_commit(&empty_bar[s]);     // the stage is free once these MMAs have read it
             }
@@ -238,7 +191,7 @@ __global__ void __launch_bounds__(TC_THREADS) gemm_tc_kernel(const __grid_consta
         // ---------------- epilogue: warps 0..3 own TMEM lanes 32*warp .. 32*warp+31 ----------------
         bool ok = true;
         if (nk > 0) {
-            if (lane == 0) ok = mbar_wait(&acc_bar, 0, &abort_flag);
+            if (lane == 0) ok = mbar_wait(&acc_bar, 0, &abort_flag, p.wait_limit);
             ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
             if (!ok && lane == 0) { abort_flag = 1; atomicMax(p.status, DEV_WAIT_EXPIRED); }
         }
@@ -290,18 +243,6 @@ __global__ void __launch_bounds__(TC_THREADS) gemm_tc_kernel(const __grid_consta
     }
 }
 
-__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, const void* smem_src, int32_t c0, int32_t c1) {
-    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
-                 ::"l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(smem_u32(smem_src)) : "memory");
-}
-__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-template <int N> __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
-__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-
 constexpr int KK_EPI_WARPS = 8;                       // two per TMEM lane quarter, each takes every other 32-column chunk
 constexpr int KK_THREADS = (KK_EPI_WARPS + 2) * 32;    // + TMA producer warp + MMA warp
 constexpr int KK_BIAS_MAX = 1024;
@@ -312,11 +253,15 @@ constexpr int KK_BIAS_MAX = 1024;
 // epilogue of tile j overlaps the loads and MMAs of tile j+1, and when the packed weight matrix is
 // small enough it is loaded into shared memory once per CTA and stays there.  The epilogue (eight
 // warps) applies bias / ReLU from registers and shared memory, writes 32-row x 128-byte boxes in the
-// 128-byte swizzle and hands them to TMA stores, which also clip ragged M / N edges.
+// 128-byte swizzle and hands them to TMA stores, which also clip ragged M / N edges; the optional bf16
+// copy of C goes out with 16-byte stores straight from the registers.
+template <int KIND>
 __global__ void __launch_bounds__(KK_THREADS) gemm_tc_kk_kernel(const __grid_constant__ CUtensorMap map_a,
                                                                 const __grid_constant__ CUtensorMap map_b,
                                                                 const __grid_constant__ CUtensorMap map_c,
                                                                 const TcParams p, const int b_resident, const int tma_store) {
+    using Cfg = KindCfg<KIND>;
+    constexpr int BK = Cfg::BK;
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t full_bar[8], empty_bar[8], acc_full[2], acc_empty[2], b_bar;
     __shared__ __align__(16) float s_bias[KK_BIAS_MAX + 32];
@@ -325,8 +270,8 @@ __global__ void __launch_bounds__(KK_THREADS) gemm_tc_kk_kernel(const __grid_con
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int bn32 = (p.bn + 31) & ~31;
-    const uint32_t a_bytes = TC_BM * TC_BK * 4, b_bytes = (uint32_t)bn32 * TC_BK * 4;
-    const int nk = (int)((p.K + TC_BK - 1) / TC_BK);
+    const uint32_t a_bytes = TC_BM * 128, b_bytes = (uint32_t)bn32 * 128;
+    const int nk = (int)((p.K + BK - 1) / BK);
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     // layout: [resident B: nk * b_bytes] [ring of stages: A (+ B when not resident)] [one output box per epilogue warp]
     uint8_t* smem_b_res = smem;
@@ -365,7 +310,7 @@ __global__ void __launch_bounds__(KK_THREADS) gemm_tc_kk_kernel(const __grid_con
             bool ok = true;
             if (b_resident) {
                 mbar_expect_tx(&b_bar, (uint32_t)nk * b_bytes);
-                for (int ks = 0; ks < nk; ++ks) tma_load_2d(smem_b_res + (size_t)ks * b_bytes, &map_b, ks * TC_BK, 0, &b_bar);
+                for (int ks = 0; ks < nk; ++ks) tma_load_2d(smem_b_res + (size_t)ks * b_bytes, &map_b, ks * BK, 0, &b_bar);
             }
             uint32_t it = 0;
             for (int64_t tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x) {
@@ -373,39 +318,40 @@ __global__ void __launch_bounds__(KK_THREADS) gemm_tc_kk_kernel(const __grid_con
                 for (int ks = 0; ks < nk; ++ks, ++it) {
                     const int s = it % p.stages;
                     const uint32_t ph = ((it / p.stages) & 1) ^ 1;
-                    if (!mbar_wait(&empty_bar[s], ph, &abort_flag)) { abort_flag = 1; atomicMax(p.status, DEV_WAIT_EXPIRED); ok = false; break; }
+                    if (!mbar_wait(&empty_bar[s], ph, &abort_flag, p.wait_limit)) { abort_flag = 1; atomicMax(p.status, DEV_WAIT_EXPIRED); ok = false; break; }
                     uint8_t* sa = smem_ring + (size_t)s * stage_bytes;
                     mbar_expect_tx(&full_bar[s], stage_bytes);
-                    tma_load_2d(sa, &map_a, ks * TC_BK, m0, &full_bar[s]);
-                    if (!b_resident) tma_load_2d(sa + a_bytes, &map_b, ks * TC_BK, n0, &full_bar[s]);
+                    if (p.debug_drop_load && it == 0) continue;      // test hook: this stage never fills
+                    tma_load_2d(sa, &map_a, ks * BK, m0, &full_bar[s]);
+                    if (!b_resident) tma_load_2d(sa + a_bytes, &map_b, ks * BK, n0, &full_bar[s]);
                 }
             }
         }
     } else if (warp == KK_EPI_WARPS + 1) {
         if (lane == 0) {
             // ---------------- MMA issuer ----------------
-            const uint32_t idesc = make_idesc_tf32(p.bn, false);
+            const uint32_t idesc = make_idesc<KIND>(TC_BM, p.bn, false);
             bool ok = true;
             if (b_resident) {
-                if (!mbar_wait(&b_bar, 0, &abort_flag)) { abort_flag = 1; atomicMax(p.status, DEV_WAIT_EXPIRED); ok = false; }
+                if (!mbar_wait(&b_bar, 0, &abort_flag, p.wait_limit)) { abort_flag = 1; atomicMax(p.status, DEV_WAIT_EXPIRED); ok = false; }
             }
             uint32_t it = 0, j = 0;
             for (int64_t tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x, ++j) {
                 const uint32_t buf = j & 1;
-                if (!mbar_wait(&acc_empty[buf], ((j >> 1) & 1) ^ 1, &abort_flag)) { abort_flag = 1; atomicMax(p.status, DEV_WAIT_EXPIRED); ok = false; break; }
+                if (!mbar_wait(&acc_empty[buf], ((j >> 1) & 1) ^ 1, &abort_flag, p.wait_limit)) { abort_flag = 1; atomicMax(p.status, DEV_WAIT_EXPIRED); ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + buf * acc_stride;
                 for (int ks = 0; ks < nk; ++ks, ++it) {
                     const int s = it % p.stages;
                     const uint32_t ph = (it / p.stages) & 1;
-                    if (!mbar_wait(&full_bar[s], ph, &abort_flag)) { abort_flag = 1; atomicMax(p.status, DEV_WAIT_EXPIRED); ok = false; break; }
+                    if (!mbar_wait(&full_bar[s], ph, &abort_flag, p.wait_limit)) { abort_flag = 1; atomicMax(p.status, DEV_WAIT_EXPIRED); ok = false; break; }
                     tc_fence_after();
                     const uint32_t sa = smem_u32(smem_ring + (size_t)s * stage_bytes);
                     const uint32_t sb = b_resident ? smem_u32(smem_b_res + (size_t)ks * b_bytes) : sa + a_bytes;
 #pragma unroll
-                    for (int k8 = 0; k8 < TC_BK / 8; ++k8)
-                        tc_mma_tf32(d_tmem, make_desc(sa + k8 * 32, 16, 1024, 2), make_desc(sb + k8 * 32, 16, 1024, 2), idesc,
-                                    (ks | k8) != 0 ? 1u : 0u);
+                    for (int kq = 0; kq < BK / Cfg::MMA_K; ++kq)
+                        tc_mma<KIND>(d_tmem, make_desc(sa + kq * 32, 16, 1024, 2), make_desc(sb + kq * 32, 16, 1024, 2), idesc,
+                                     (ks | kq) != 0 ? 1u : 0u);
                     tc_commit(&empty_bar[s]);
                 }
                 if (ok) tc_commit(&acc_full[buf]);
@@ -423,7 +369,7 @@ __global__ void __launch_bounds__(KK_THREADS) gemm_tc_kk_kernel(const __grid_con
             const uint32_t buf = j & 1;
             const int64_t m0 = (tile / p.n_tiles) * TC_BM;
             const int n0 = (int)((tile % p.n_tiles) * p.bn);
-            if (lane == 0) ok = mbar_wait(&acc_full[buf], (j >> 1) & 1, &abort_flag);
+            if (lane == 0) ok = mbar_wait(&acc_full[buf], (j >> 1) & 1, &abort_flag, p.wait_limit);
             ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
             if (!ok) { if (lane == 0) { abort_flag = 1; atomicMax(p.status, DEV_WAIT_EXPIRED); } break; }
             tc_fence_after();
@@ -454,6 +400,11 @@ __global__ void __launch_bounds__(KK_THREADS) gemm_tc_kk_kernel(const __grid_con
 #pragma unroll
                     for (int q = 0; q < 32; ++q)
                         if (nb + q < p.N) v[q] = tc_apply_epi(p.epi, v[q], m, nb + q, p.N);
+                }
+                if (p.C_lp && row_ok) {
+                    const int64_t left = p.N - nb, here = p.bn - c0;
+                    const int valid = (int)(left < here ? left : here);
+                    store_lp_row(p.C_lp + m * p.ldc_lp + nb, v, valid);
                 }
                 if (tma_store) {
                     // rows of 128 bytes in the 128-byte swizzle the tensor map expects: 16-byte chunk q of row r
@@ -501,15 +452,34 @@ __global__ void __launch_bounds__(KK_THREADS) gemm_tc_kk_kernel(const __grid_con
     }
 }
 
-// dst[n][k] = trans ? src[k][n] : src[n][k] for n < N, k < K, zero elsewhere; dst is rows x kpad.
+// dst[n][k] = trans ? src[k][n] : src[n][k] for n < N, k < K, zero elsewhere; dst is rows x kpad of
+// fp32 (TF32 kind) or bf16 (round to nearest even).
+template <int KIND>
 __global__ void pack_b_kernel(const float* __restrict__ src, int64_t ld, int trans, int N, int K, int rows, int kpad,
-                              float* __restrict__ dst) {
+                              void* __restrict__ dst) {
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= (int64_t)rows * kpad) return;
     const int n = (int)(i / kpad), k = (int)(i % kpad);
     float v = 0.0f;
     if (n < N && k < K) v = trans ? src[(int64_t)k * ld + n] : src[(int64_t)n * ld + k];
-    dst[i] = v;
+    if (KIND == KIND_TF32) reinterpret_cast<float*>(dst)[i] = v;
+    else reinterpret_cast<uint16_t*>(dst)[i] = (uint16_t)(pack_bf16(v, 0.0f) & 0xFFFFu);
+}
+
+// dst[r][c] = bf16(src[r][c]) for c < d (round to nearest even); four columns per thread.
+__global__ void to_bf16_kernel(int64_t rows, int d4, const float* __restrict__ src, int64_t ld_src, int d,
+                               uint16_t* __restrict__ dst, int64_t ld_dst) {
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= rows * d4) return;
+    const int64_t r = t / d4; const int c = (int)(t % d4) * 4;
+    const float4 v = __ldg(reinterpret_cast<const float4*>(src + r * ld_src + c));
+    uint16_t* o = dst + r * ld_dst + c;
+    if (c + 3 < d) {
+        *reinterpret_cast<uint2*>(o) = make_uint2(pack_bf16(v.x, v.y), pack_bf16(v.z, v.w));
+    } else {
+        const float f[4] = {v.x, v.y, v.z, v.w};
+        for (int q = 0; q < 4; ++q) if (c + q < d) o[q] = (uint16_t)(pack_bf16(f[q], 0.0f) & 0xFFFFu);
+    }
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -532,17 +502,18 @@ EncodeTiledFn get_encode() {
     return fn;
 }
 
-// 2-D fp32 tensor, `inner` contiguous elements per row, `outer` rows of `ld` elements; 128-byte swizzle.
-bool encode_2d(CUtensorMap* map, const float* base, int64_t inner, int64_t outer, int64_t ld, int box_inner, int box_outer,
-               CUtensorMapSwizzle swizzle = CU_TENSOR_MAP_SWIZZLE_128B) {
+// 2-D tensor of fp32 (eb = 4) or bf16 (eb = 2): `inner` contiguous elements per row, `outer` rows of `ld`
+// elements; 128-byte swizzle unless stated.
+bool encode_2d(CUtensorMap* map, const void* base, int eb, int64_t inner, int64_t outer, int64_t ld, int box_inner,
+               int box_outer, CUtensorMapSwizzle swizzle = CU_TENSOR_MAP_SWIZZLE_128B) {
     EncodeTiledFn fn = get_encode();
     if (!fn) return false;
     cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)outer};
-    cuuint64_t strides[1] = {(cuuint64_t)ld * sizeof(float)};
+    cuuint64_t strides[1] = {(cuuint64_t)ld * (cuuint64_t)eb};
     cuuint32_t box[2] = {(cuuint32_t)box_inner, (cuuint32_t)box_outer};
     cuuint32_t estr[2] = {1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+    return fn(map, eb == 4 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base),
+              dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -556,42 +527,30 @@ int pick_bn(int64_t N) {
     return (int)bn;
 }
 
-int pick_stages(int bn) {
-    const int bn32 = (bn + 31) & ~31;
-    const int stage = TC_BM * TC_BK * 4 + bn32 * TC_BK * 4;
-    int s = (96 * 1024) / stage;      // aim at two CTAs per SM
-    if (s < 2) s = 2;
-    if (s > 6) s = 6;
-    return s;
-}
-
-}  // namespace
-
-namespace mixgcn {
-
-mixgcn_status launch_splitk_reduce(mixgcn_ctx* ctx, int64_t M, int64_t N, int splits, const float* part, float* C,
-                                   int64_t ldc, const mixgcn_epilogue* epi, cudaStream_t s);
-
-// Returns MIXGCN_EUNSUPPORTED (without touching anything) when this shape / alignment is not
-// served by the tensor-core kernels; the caller then uses the fp32 kernel.
-mixgcn_status launch_gemm_tc(mixgcn_ctx* ctx, int ta, int tb, int64_t M, int64_t N, int64_t K, const float* A,
-                             int64_t lda, const float* B, int64_t ldb, float* C, int64_t ldc,
-                             const mixgcn_epilogue* epi, int64_t epi_row0, cudaStream_t s) {
+template <int KIND>
+mixgcn_status launch_kind(mixgcn_ctx* ctx, int ta, int tb, int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,
+                          const void* B, int64_t ldb, float* C, int64_t ldc, const mixgcn_epilogue* epi, int64_t epi_row0,
+                          cudaStream_t s, uint16_t* C_lp, int64_t ldc_lp) {
+    using Cfg = KindCfg<KIND>;
+    constexpr int EB = Cfg::EB, BK = Cfg::BK;
+    constexpr int64_t LD_ALIGN = 16 / EB;           // TMA strides are multiples of 16 bytes
     if (M <= 0 || N <= 0 || K <= 0) return MIXGCN_EUNSUPPORTED;
     if (ta && tb) return MIXGCN_EUNSUPPORTED;
-    if (!aligned16(A) || (lda & 3)) return MIXGCN_EUNSUPPORTED;
-    if (ta && (!aligned16(B) || (ldb & 3))) return MIXGCN_EUNSUPPORTED;
+    if (!aligned16(A) || (lda % LD_ALIGN)) return MIXGCN_EUNSUPPORTED;
+    if (ta && (!aligned16(B) || (ldb % LD_ALIGN))) return MIXGCN_EUNSUPPORTED;
     if (M >= (1ll << 31) || N >= (1ll << 31) || K >= (1ll << 31)) return MIXGCN_EUNSUPPORTED;
+    if (C_lp && (ta || !aligned16(C_lp) || (ldc_lp & 7) || ldc_lp < N)) return MIXGCN_EUNSUPPORTED;
     if (!get_encode()) return MIXGCN_EUNSUPPORTED;
 
     TcParams p{};
     p.M = M; p.N = N; p.K = K;
     p.bn = pick_bn(N);
-    p.stages = pick_stages(p.bn);
     p.m_tiles = (M + TC_BM - 1) / TC_BM;
     p.n_tiles = (N + p.bn - 1) / p.bn;
     p.C = C; p.ldc = ldc; p.vec_c = aligned16(C) && (ldc & 3) == 0;
+    p.C_lp = C_lp; p.ldc_lp = ldc_lp;
     p.status = ctx->d_status;
+    p.wait_limit = ctx->debug_wait_limit > 0 ? (uint32_t)ctx->debug_wait_limit : WAIT_LIMIT_DEFAULT;
     if (epi) {
         p.epi.bias = epi->bias; p.epi.relu = epi->relu; p.epi.drop = epi->drop_mask; p.epi.keep_scale = epi->keep_scale;
         p.epi.gate = epi->gate; p.epi.ld_gate = epi->ld_gate; p.epi.gate_scale = epi->gate_scale;
@@ -600,28 +559,29 @@ mixgcn_status launch_gemm_tc(mixgcn_ctx* ctx, int ta, int tb, int64_t M, int64_t
     const int64_t tiles = p.m_tiles * p.n_tiles;
     if (tiles > 0x7FFFFFFFll) return MIXGCN_EUNSUPPORTED;
     const int bn32 = (p.bn + 31) & ~31;
-    const size_t smem = (size_t)p.stages * (TC_BM * TC_BK * 4 + bn32 * TC_BK * 4) + 1024;
     CUtensorMap map_a, map_b;
 
     if (!ta) {
         // KK form: pack B as rows x kpad (K contiguous), rows = n_tiles * bn32
-        const int kpad = (int)((K + TC_BK - 1) / TC_BK * TC_BK);
+        const int kpad = (int)((K + BK - 1) / BK * BK);
         const int rows = (int)(p.n_tiles * p.bn > bn32 ? p.n_tiles * p.bn : bn32);
-        MIXGCN_TRY(ensure_workspace(ctx, (int64_t)rows * kpad * (int64_t)sizeof(float)));
-        float* packed = reinterpret_cast<float*>(ctx->workspace);
-        if (!encode_2d(&map_a, A, K, M, lda, TC_BK, TC_BM)) return MIXGCN_EUNSUPPORTED;
-        if (!encode_2d(&map_b, packed, kpad, rows, kpad, TC_BK, bn32)) return MIXGCN_EUNSUPPORTED;
+        MIXGCN_TRY(ensure_workspace(ctx, (int64_t)rows * kpad * EB));
+        void* packed = ctx->workspace;
+        if (!encode_2d(&map_a, A, EB, K, M, lda, BK, TC_BM)) return MIXGCN_EUNSUPPORTED;
+        if (!encode_2d(&map_b, packed, EB, kpad, rows, kpad, BK, bn32)) return MIXGCN_EUNSUPPORTED;
         {
             LaunchScope scope(ctx, PH_GEMM, s);
             const int64_t total = (int64_t)rows * kpad;
-            pack_b_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(B, ldb, tb ? 0 : 1, (int)N, (int)K, rows, kpad, packed);
+            pack_b_kernel<KIND><<<(unsigned)((total + 255) / 256), 256, 0, s>>>(reinterpret_cast<const float*>(B), ldb, tb ? 0 : 1,
+                                                                                 (int)N, (int)K, rows, kpad, packed);
         }
         p.splits = 1; p.k_per_split = K; p.raw = 0;
+        p.debug_drop_load = ctx->debug_drop_load;
         // keep the packed weights resident in shared memory when they are small and there is one n-tile
-        const int nk = kpad / TC_BK;
-        const size_t b_all = (size_t)nk * bn32 * TC_BK * 4;
+        const int nk = kpad / BK;
+        const size_t b_all = (size_t)nk * bn32 * 128;
         const int b_resident = (p.n_tiles == 1 && b_all <= 96 * 1024) ? 1 : 0;
-        const size_t stage = TC_BM * TC_BK * 4 + (b_resident ? 0 : (size_t)bn32 * TC_BK * 4);
+        const size_t stage = TC_BM * 128 + (b_resident ? 0 : (size_t)bn32 * 128);
         const size_t budget = (b_resident ? 168 * 1024 - b_all : 160 * 1024);
         int stages = (int)(budget / stage);
         if (stages > 8) stages = 8;
@@ -630,11 +590,11 @@ mixgcn_status launch_gemm_tc(mixgcn_ctx* ctx, int ta, int tb, int64_t M, int64_t
         const size_t smem_kk = (b_resident ? b_all : 0) + (size_t)stages * stage + 8 * 4096 + 1024;
         const int tma_store = p.vec_c ? 1 : 0;
         CUtensorMap map_c = map_a;
-        if (tma_store && !encode_2d(&map_c, C, N, M, ldc, 32, 32)) return MIXGCN_EUNSUPPORTED;
+        if (tma_store && !encode_2d(&map_c, C, 4, N, M, ldc, 32, 32)) return MIXGCN_EUNSUPPORTED;
         int64_t grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
-        MIXGCN_CUDA(cudaFuncSetAttribute(gemm_tc_kk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_kk));
+        MIXGCN_CUDA(cudaFuncSetAttribute(gemm_tc_kk_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_kk));
         LaunchScope scope(ctx, PH_GEMM, s);
-        gemm_tc_kk_kernel<<<dim3((unsigned)grid, 1, 1), KK_THREADS, smem_kk, s>>>(map_a, map_b, map_c, p, b_resident, tma_store);
+        gemm_tc_kk_kernel<KIND><<<dim3((unsigned)grid, 1, 1), KK_THREADS, smem_kk, s>>>(map_a, map_b, map_c, p, b_resident, tma_store);
         MIXGCN_CUDA(cudaGetLastError());
         return MIXGCN_OK;
     }
@@ -649,24 +609,61 @@ mixgcn_status launch_gemm_tc(mixgcn_ctx* ctx, int ta, int tb, int64_t M, int64_t
         if (splits > 2048) splits = 2048;
     }
     int64_t kps = (K + splits - 1) / splits;
-    kps = (kps + TC_BK - 1) / TC_BK * TC_BK;
+    kps = (kps + BK - 1) / BK * BK;
     splits = (int)((K + kps - 1) / kps);
     p.k_per_split = kps; p.splits = splits;
-    if (!encode_2d(&map_a, A, M, K, lda, 32, TC_BK, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B)) return MIXGCN_EUNSUPPORTED;
-    if (!encode_2d(&map_b, B, N, K, ldb, 32, TC_BK, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B)) return MIXGCN_EUNSUPPORTED;
+    const CUtensorMapSwizzle sw = KIND == KIND_TF32 ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B : CU_TENSOR_MAP_SWIZZLE_128B;
+    if (!encode_2d(&map_a, A, EB, M, K, lda, Cfg::CHUNK, BK, sw)) return MIXGCN_EUNSUPPORTED;
+    if (!encode_2d(&map_b, B, EB, N, K, ldb, Cfg::CHUNK, BK, sw)) return MIXGCN_EUNSUPPORTED;
+    const int bn_pad = (p.bn + Cfg::CHUNK - 1) / Cfg::CHUNK * Cfg::CHUNK;
+    const size_t stage_mm = (size_t)TC_BM * 128 + (size_t)bn_pad * 128;
+    int stages_mm = (int)((96 * 1024) / stage_mm);      // aim at two CTAs per SM
+    if (stages_mm < 2) stages_mm = 2;
+    if (stages_mm > 6) stages_mm = 6;
+    p.stages = stages_mm;
+    const size_t smem = (size_t)stages_mm * stage_mm + 1024;
     if (splits > 1) {
         MIXGCN_TRY(ensure_workspace(ctx, (int64_t)splits * M * N * (int64_t)sizeof(float)));
         p.C = reinterpret_cast<float*>(ctx->workspace); p.ldc = N; p.vec_c = (N & 3) == 0; p.raw = 1;
     } else {
         p.raw = 0;
     }
-    MIXGCN_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    MIXGCN_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<KIND, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     {
         LaunchScope scope(ctx, PH_GEMM, s);
-        gemm_tc_kernel<true><<<dim3((unsigned)tiles, 1, (unsigned)splits), TC_THREADS, smem, s>>>(map_a, map_b, p);
+        gemm_tc_kernel<KIND, true><<<dim3((unsigned)tiles, 1, (unsigned)splits), TC_THREADS, smem, s>>>(map_a, map_b, p);
     }
     MIXGCN_CUDA(cudaGetLastError());
     if (splits > 1) MIXGCN_TRY(launch_splitk_reduce(ctx, M, N, splits, p.C, C, ldc, epi, s));
+    return MIXGCN_OK;
+}
+
+}  // namespace
+
+namespace mixgcn {
+
+// Returns MIXGCN_EUNSUPPORTED (without touching anything) when this shape / alignment is not
+// served by the tensor-core kernels; the caller then uses another kernel.
+//   kind 0 (TF32): A, and B in the MM form, are fp32 (lda, ldb in fp32 elements, multiples of 4);
+//   kind 1 (BF16): they are bf16 (lda, ldb in bf16 elements, multiples of 8).
+// In the KK form B is always the fp32 weight matrix (packed and converted here).  C_lp (KK form only,
+// nullable) receives a bf16 copy of C.
+mixgcn_status launch_gemm_tc(mixgcn_ctx* ctx, int kind, int ta, int tb, int64_t M, int64_t N, int64_t K, const void* A,
+                             int64_t lda, const void* B, int64_t ldb, float* C, int64_t ldc,
+                             const mixgcn_epilogue* epi, int64_t epi_row0, cudaStream_t s, uint16_t* C_lp, int64_t ldc_lp) {
+    if (kind == KIND_BF16)
+        return launch_kind<KIND_BF16>(ctx, ta, tb, M, N, K, A, lda, B, ldb, C, ldc, epi, epi_row0, s, C_lp, ldc_lp);
+    return launch_kind<KIND_TF32>(ctx, ta, tb, M, N, K, A, lda, B, ldb, C, ldc, epi, epi_row0, s, C_lp, ldc_lp);
+}
+
+// dst (rows x ld_dst bf16, ld_dst a multiple of 4) = bf16(src (rows x ld_src fp32, 16-byte aligned, ld_src % 4 == 0)), columns < d
+mixgcn_status launch_to_bf16(mixgcn_ctx* ctx, int64_t rows, int32_t d, const float* src, int64_t ld_src, uint16_t* dst,
+                             int64_t ld_dst, cudaStream_t s) {
+    if (rows <= 0 || d <= 0) return MIXGCN_OK;
+    const int d4 = (d + 3) / 4;
+    LaunchScope scope(ctx, PH_ELEM, s);
+    to_bf16_kernel<<<(unsigned)((rows * d4 + 255) / 256), 256, 0, s>>>(rows, d4, src, ld_src, d, dst, ld_dst);
+    MIXGCN_CUDA(cudaGetLastError());
     return MIXGCN_OK;
 }
 

@@ -57,6 +57,11 @@ struct mixgcn_ctx {
     cudaStream_t side_stream[2];
     cudaEvent_t fork_ev, join_ev[2];
     cudaEvent_t chunk_ev[64];
+    void* workspace_lp;       // bf16 copies of fp32 operands converted on the fly (BF16 products whose caller gave no copy)
+    int64_t workspace_lp_bytes;
+    int64_t gemm_path[3];     // dense products served by: 0 fp32 FMA kernel, 1 tcgen05 TF32, 2 tcgen05 BF16
+    int debug_wait_limit;     // > 0: polls after which the tensor-core kernels' waits give up (test of that path)
+    int debug_drop_load;      // 1: the next K-major tensor-core product leaves one stage unfilled (test of that path)
     int spmm_slice_cols;      // 0 = default (one slice up to 1024 columns)
     int loss_train_rows_only; // 1 = the loss skips rows outside the train mask entirely
     // profiling
@@ -188,6 +193,8 @@ struct SpmmOpts {
     const uint8_t* row_filter = nullptr;     // compute only the output rows whose byte is non-zero (not with `sparse`)
     int phase = PH_SPMM;                     // profiling phase the launches are booked under
     int64_t row_limit = -1;                  // >= 0: only the first row_limit rows of the schedule (longest first)
+    uint16_t* Z_lp = nullptr;                // nullable: also write a bf16 copy of Z (after the epilogue), ldz_lp a multiple of 4
+    int64_t ldz_lp = 0;
 };
 mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView& A, int chunks, int k,
                           int32_t w, const float* Y, int64_t ldy, float* Z, int64_t ldz,
@@ -195,9 +202,28 @@ mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView&
 // schedule of all n rows of a view whose column ids lie in [0, n_cols); release of a view's memory
 mixgcn_status build_view_schedule(int64_t n_cols, int64_t n, CsrView& v, cudaStream_t s);
 void release_view(CsrView& v);
+// bf16 companions of one dense product (all nullable): copies of A and of B (the MM form's second
+// activation operand) that a producer already wrote, and a bf16 copy of C to write for the next product.
+// Leading dimensions in bf16 elements, multiples of 8; pointers 16-byte aligned.
+struct GemmLP {
+    const uint16_t* A = nullptr; int64_t lda = 0;
+    const uint16_t* B = nullptr; int64_t ldb = 0;
+    uint16_t* C = nullptr; int64_t ldc = 0;
+};
 mixgcn_status launch_gemm(mixgcn_ctx* ctx, int precision, int ta, int tb, int64_t M, int64_t N, int64_t K,
                           const float* A, int64_t lda, const float* B, int64_t ldb, float* C, int64_t ldc,
-                          const mixgcn_epilogue* epi, int64_t epi_row0, cudaStream_t s);
+                          const mixgcn_epilogue* epi, int64_t epi_row0, cudaStream_t s, const GemmLP* lp = nullptr);
+mixgcn_status launch_gemm_simt(mixgcn_ctx* ctx, int ta, int tb, int64_t M, int64_t N, int64_t K,
+                               const float* A, int64_t lda, const float* B, int64_t ldb, float* C, int64_t ldc,
+                               const mixgcn_epilogue* epi, int64_t epi_row0, cudaStream_t s);
+mixgcn_status launch_gemm_tc(mixgcn_ctx* ctx, int kind, int ta, int tb, int64_t M, int64_t N, int64_t K, const void* A,
+                             int64_t lda, const void* B, int64_t ldb, float* C, int64_t ldc,
+                             const mixgcn_epilogue* epi, int64_t epi_row0, cudaStream_t s, uint16_t* C_lp, int64_t ldc_lp);
+mixgcn_status launch_splitk_reduce(mixgcn_ctx* ctx, int64_t M, int64_t N, int splits, const float* part, float* C,
+                                   int64_t ldc, const mixgcn_epilogue* epi, cudaStream_t s);
+mixgcn_status launch_to_bf16(mixgcn_ctx* ctx, int64_t rows, int32_t d, const float* src, int64_t ld_src, uint16_t* dst,
+                             int64_t ld_dst, cudaStream_t s);
+mixgcn_status ensure_workspace_lp(mixgcn_ctx* ctx, int64_t bytes);
 mixgcn_status launch_colsum(mixgcn_ctx* ctx, int64_t n, int32_t d, const float* X, int64_t ld, float* out,
                             cudaStream_t s);
 mixgcn_status launch_gate(mixgcn_ctx* ctx, int64_t n, int32_t d, float* G, int64_t ldg, const float* X_out,

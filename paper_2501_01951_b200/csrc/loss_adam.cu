@@ -3,6 +3,8 @@
 // reductions run in a fixed order (per-warp shuffles, per-CTA partials, one final pass).
 #include <stddef.h>
 
+#include <atomic>
+
 #include "internal.cuh"
 
 using namespace mixgcn;
@@ -463,7 +465,11 @@ int launch_loss_rows(unsigned warp_blocks, cudaStream_t s, int64_t n, int C, con
     // Several CTAs per SM (each with two tile buffers) keep some computing while others wait for their
     // copies: a CTA takes at most MIXGCN_LOSS_TILE_KB of shared memory; rows per tile follow from that.
     constexpr int64_t TILE_SMEM = MIXGCN_LOSS_TILE_KB * 1024;
-    if (vec && sm_count > 0 && C >= 8 && 2 * 32 * ld * 4 <= TILE_SMEM) {
+    // The tile kernel treats a tile as one dense piece of rows x ld floats (it copies and zeroes whole
+    // rows), so it is taken only when the row holds nothing but its C columns and their pad to a multiple
+    // of 4; a wider ld (a column slice of a larger buffer) goes to the per-row kernels, which touch columns
+    // below round4(C) only.
+    if (vec && sm_count > 0 && C >= 8 && ld == ((int64_t)C + 3) / 4 * 4 && 2 * 32 * ld * 4 <= TILE_SMEM) {
         const int rows = 2 * 128 * ld * 4 <= TILE_SMEM ? 128 : (2 * 64 * ld * 4 <= TILE_SMEM ? 64 : 32);
         const int64_t n_tiles = (n + rows - 1) / rows;
         int64_t per_sm = (220 * 1024) / (2 * rows * ld * 4 + 1024);
@@ -619,7 +625,7 @@ constexpr int NOALLOC_MAX_DEVICES = 64;
 
 struct NoAllocScratch {
     unsigned long long count;      // train nodes, cleared at the start of every call
-    int32_t status;                // 0 ok, 1 empty train mask, 2 label out of range; cleared likewise
+    int32_t status;                // 0 ok, 1 empty train mask, 2 label out of range, 3 bounded wait expired; cleared likewise
     int32_t pad;
     double part[NOALLOC_MAX_PARTIALS];
 };
@@ -628,8 +634,10 @@ struct NoAllocScratch {
 static __device__ __align__(256) unsigned char g_noalloc_scratch[sizeof(NoAllocScratch)];
 
 // In host code the array's name is only a handle for the runtime, not a device address; the real
-// address is looked up once per device (with that device current) and cached here.
-NoAllocScratch* g_noalloc_ptr[NOALLOC_MAX_DEVICES] = {};
+// address is looked up once per device (with that device current) and cached here.  Host threads that
+// make their first call on a device at the same time both store the same address: the entries are
+// atomic so that this is well defined.
+std::atomic<NoAllocScratch*> g_noalloc_ptr[NOALLOC_MAX_DEVICES] = {};
 
 }  // namespace
 
@@ -649,14 +657,14 @@ extern "C" mixgcn_status mixgcn_loss_softmax_xent_noalloc(int64_t n, int32_t C, 
     int device = -1;
     MIXGCN_CUDA(cudaGetDevice(&device));
     if (device < 0 || device >= NOALLOC_MAX_DEVICES) MIXGCN_FAIL(MIXGCN_EUNSUPPORTED, "loss_noalloc: device index %d not supported", device);
-    if (!g_noalloc_ptr[device]) {
+    if (!g_noalloc_ptr[device].load(std::memory_order_acquire)) {
         // first call on this device: resolve the device address of the scratch array
         void* p = nullptr;
         MIXGCN_CUDA(cudaGetSymbolAddress(&p, g_noalloc_scratch));
         if (!p) MIXGCN_FAIL(MIXGCN_ECUDA, "loss_noalloc: the scratch symbol has no device address");
-        g_noalloc_ptr[device] = reinterpret_cast<NoAllocScratch*>(p);
+        g_noalloc_ptr[device].store(reinterpret_cast<NoAllocScratch*>(p), std::memory_order_release);
     }
-    NoAllocScratch* sc = g_noalloc_ptr[device];
+    NoAllocScratch* sc = g_noalloc_ptr[device].load(std::memory_order_acquire);
     cudaStream_t s = (cudaStream_t)stream;
     const int64_t blocks = (n + NOALLOC_ROWS_PER_BLOCK - 1) / NOALLOC_ROWS_PER_BLOCK;
     // the array keeps the previous call's contents: clear the counter and the status word

@@ -15,8 +15,14 @@ __global__ void pos_scatter_kernel(int64_t count, const int32_t* __restrict__ id
     if (i < count) pos[idx[i]] = (int32_t)i;
 }
 
-__global__ void check_count_kernel(const int64_t* selected, int64_t expected, int32_t* status) {
-    if (threadIdx.x == 0 && blockIdx.x == 0 && *selected != expected) atomicMax(status, DEV_BAD_ROW_COUNT);
+// The selection filled idx[0, *selected).  If the caller's count differs, report it; slots
+// [*selected, expected) were not written by the selection and still hold old workspace contents, so
+// they are pointed at row 0 (a valid row) before the gather / scatter / position kernels read them.
+__global__ void check_count_kernel(const int64_t* selected, int64_t expected, int32_t* idx, int32_t* status) {
+    const int64_t sel = *selected;
+    if (threadIdx.x == 0 && blockIdx.x == 0 && sel != expected) atomicMax(status, DEV_BAD_ROW_COUNT);
+    for (int64_t i = sel + (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < expected; i += (int64_t)gridDim.x * blockDim.x)
+        idx[i] = 0;
 }
 
 // dst[i, :] = src[idx[i], :], float4 wide (ld multiples of 4, 16-byte aligned), d4 = ceil(d/4) groups per row
@@ -67,10 +73,11 @@ mixgcn_status ensure_workspace_rows(mixgcn_ctx* ctx, int64_t bytes) {
 }
 
 // Carves the row-sparse workspace and fills the row list and the position map of `mask`.
-// idx has capacity n (memory-safe whatever the mask holds); if the number of set rows differs from
-// `count` the device status word receives DEV_BAD_ROW_COUNT.
+// idx has capacity n >= count (memory-safe whatever the mask holds); if the number of set rows differs
+// from `count` the device status word receives DEV_BAD_ROW_COUNT and the unfilled slots name row 0.
 mixgcn_status build_row_set(mixgcn_ctx* ctx, int64_t n, const uint8_t* mask, int64_t count, int64_t ld_a, int64_t ld_b,
                             RowSet* rs, cudaStream_t s) {
+    if (count < 0 || count > n) MIXGCN_FAIL(MIXGCN_EINVAL, "row set: the row count must lie in [0, n] (count %lld, n %lld)", (long long)count, (long long)n);
     size_t tb = 0;
     thrust::counting_iterator<int32_t> ids(0);
     MIXGCN_CUDA(cub::DeviceSelect::Flagged(nullptr, tb, ids, mask, (int32_t*)nullptr, (int64_t*)nullptr, n, s));
@@ -87,7 +94,7 @@ mixgcn_status build_row_set(mixgcn_ctx* ctx, int64_t n, const uint8_t* mask, int
     rs->count = count;
     LaunchScope scope(ctx, PH_ELEM, s, 4);
     MIXGCN_CUDA(cub::DeviceSelect::Flagged(base + o_tmp, tb, ids, mask, rs->idx, selected, n, s));
-    check_count_kernel<<<1, 32, 0, s>>>(selected, count, ctx->d_status);
+    check_count_kernel<<<64, 256, 0, s>>>(selected, count, rs->idx, ctx->d_status);
     MIXGCN_CUDA(cudaMemsetAsync(rs->pos, 0xFF, (size_t)n * 4, s));       // -1 everywhere
     if (count > 0) pos_scatter_kernel<<<(unsigned)((count + 255) / 256), 256, 0, s>>>(count, rs->idx, rs->pos);
     MIXGCN_CUDA(cudaGetLastError());

@@ -60,6 +60,7 @@ struct SpmmParams {
     int32_t w_total;       // full width (for the dense drop-mask index)
     const float* Y; int64_t ldy;
     float* Z; int64_t ldz;
+    uint16_t* Z_lp; int64_t ldz_lp;   // nullable: bf16 copy of Z (after the epilogue) for a bf16 dense product that follows
     float* partial;        // non-null: unit idx writes its raw sums to partial[idx * ldp + ...]
     int64_t ldp;
     // row-sparse input (spmm_sparse_kernel): rows v of the input with in_mask[v] == 0 are exactly zero
@@ -86,6 +87,14 @@ __device__ __forceinline__ float epilogue1(const SpmmParams& p, float y, int64_t
     return y;
 }
 
+// four fp32 -> four bf16 (round to nearest even), 8 bytes
+__device__ __forceinline__ void store_lp4(uint16_t* dst, float x, float y, float z, float w) {
+    uint32_t lo, hi;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(lo) : "f"(y), "f"(x));
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(hi) : "f"(w), "f"(z));
+    *reinterpret_cast<uint2*>(dst) = make_uint2(lo, hi);
+}
+
 __device__ __forceinline__ void store_row(const SpmmParams& p, int64_t u, int c4, float4 a) {
     const int j = p.j0 + c4 * 4;           // global column of a.x
     const int jend = p.j0 + p.w;           // one past the last valid column of the slice
@@ -94,11 +103,13 @@ __device__ __forceinline__ void store_row(const SpmmParams& p, int64_t u, int c4
         // ReLU, dropout and the gate all map 0 to 0: no mask or gate byte needs to be read (the empty
         // rows of a row-sparse aggregation take this path)
         *reinterpret_cast<float4*>(p.Z + u * p.ldz + j) = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (p.Z_lp) *reinterpret_cast<uint2*>(p.Z_lp + u * p.ldz_lp + j) = make_uint2(0u, 0u);
         return;
     }
 #pragma unroll
     for (int t = 0; t < 4; ++t) r[t] = (j + t < jend) ? epilogue1(p, r[t], u, j + t) : 0.0f;
     *reinterpret_cast<float4*>(p.Z + u * p.ldz + j) = make_float4(r[0], r[1], r[2], r[3]);
+    if (p.Z_lp) store_lp4(p.Z_lp + u * p.ldz_lp + j, r[0], r[1], r[2], r[3]);
 }
 
 __device__ __forceinline__ void fma4(float4& acc, float a, const float4& y) {
@@ -483,6 +494,7 @@ mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView&
     SpmmParams p{};
     p.rowptr = A.rowptr; p.col = A.col; p.val = A.val;
     p.Y = Y; p.ldy = ldy; p.Z = Z; p.ldz = ldz; p.w_total = w;
+    p.Z_lp = opts.Z_lp; p.ldz_lp = opts.ldz_lp;
     if (epi) {
         p.bias = epi->bias; p.relu = epi->relu; p.drop = epi->drop_mask; p.keep_scale = epi->keep_scale;
         p.gate = epi->gate; p.ld_gate = epi->ld_gate; p.gate_scale = epi->gate_scale;

@@ -16,10 +16,14 @@ def round4(x: int) -> int:
     return (x + 3) // 4 * 4
 
 
+def round8(x: int) -> int:
+    return (x + 7) // 8 * 8
+
+
 class GcnTrainer:
     def __init__(self, ctx: mg.Ctx, graph: mg.Graph, dims, precision=mg.PREC_FP32, order=mg.ORDER_AUTO,
                  n_chunks=0, fuse_gate=True, keep_scale=1.0, device=None, row_sparse="auto",
-                 train_rows_only=False, row_plans=True, cache_first_aggregation=False):
+                 train_rows_only=False, row_plans=True, cache_first_aggregation=False, lp_copies=True):
         self.ctx, self.g = ctx, graph
         self.dims = tuple(int(d) for d in dims)
         self.L = len(self.dims) - 1
@@ -75,6 +79,32 @@ class GcnTrainer:
         for i, l in enumerate(range(L - 1, 0, -1)):
             buf = pool[i % 2]
             self.G[l] = buf.view(-1)[: n * self.ld[l]].view(n, self.ld[l])
+        # BF16 products: bf16 companions of the activations, written by the kernels that produce them
+        # (buffers only; lp_copies=False leaves them out and the library converts operands on the fly)
+        self.lp = []
+        if precision == mg.PREC_BF16 and lp_copies:
+            zb = lambda c: torch.zeros((n, round8(c)), dtype=torch.bfloat16, device=self.device)
+            keep = lambda t: (self.lp.append(t), t)[1]
+            x_lp = [None] * (L + 1)      # copy of X[l], wanted where layer l multiplies X[l] itself (upd-first)
+            g_lp = [None] * (L + 1)      # copy of G[l], wanted where layer l-1 multiplies G[l] itself (agg-first, gated on arrival)
+            for l in range(1, L):
+                if self.orders[l] == mg.ORDER_UPD_FIRST:
+                    x_lp[l] = keep(zb(self.dims[l]))
+                if self.orders[l - 1] == mg.ORDER_AGG_FIRST and fuse_gate:
+                    g_lp[l] = keep(zb(self.dims[l]))
+            for l, d in enumerate(self.descs):
+                cols = self.dims[l] if self.orders[l] == mg.ORDER_AGG_FIRST else self.dims[l + 1]
+                t = keep(zb(cols))
+                d.saved_lp, d.ld_saved_lp = t.data_ptr(), t.stride(0)
+                d.ld_in_lp, d.ld_out_lp = round8(self.dims[l]), round8(self.dims[l + 1])
+                if x_lp[l] is not None:
+                    d.x_in_lp = x_lp[l].data_ptr()
+                if x_lp[l + 1] is not None:
+                    d.x_out_lp = x_lp[l + 1].data_ptr()
+                if g_lp[l + 1] is not None:
+                    d.g_out_lp = g_lp[l + 1].data_ptr()
+                if g_lp[l] is not None:
+                    d.g_in_lp = g_lp[l].data_ptr()
         self.loss = torch.zeros(1, dtype=torch.float32, device=self.device)
         self.pred = torch.zeros(n, dtype=torch.int32, device=self.device)
         self.n_correct = torch.zeros(1, dtype=torch.int64, device=self.device)

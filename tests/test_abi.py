@@ -37,7 +37,9 @@ def test_struct_layouts_match_the_header(mg):
     # the header's structs, field by field, on an LP64 ABI
     assert C.sizeof(mg.Epilogue) == 80
     assert mg.Epilogue.residual.offset == 56 and mg.Epilogue.ld_residual.offset == 64 and mg.Epilogue.residual_scale.offset == 72
-    assert C.sizeof(mg.LayerDesc) == 88
+    assert C.sizeof(mg.LayerDesc) == 152
+    assert mg.LayerDesc.saved_lp.offset == 88 and mg.LayerDesc.x_in_lp.offset == 104 and mg.LayerDesc.ld_out_lp.offset == 128
+    assert mg.LayerDesc.g_in_lp.offset == 144
     assert mg.LayerDesc.gout_row_mask.offset == 56 and mg.LayerDesc.gin_row_mask.offset == 72
     assert mg.LayerDesc.gout_plan.offset == 80
     assert mg.LayerDesc.ld_in.offset == 8 and mg.LayerDesc.order.offset == 32 and mg.LayerDesc.n_chunks.offset == 52

@@ -295,6 +295,30 @@ def test_loss_matches_oracle(mg, ctx, Cc):
     assert torch.equal(P2[:, :Cc], Gd[:, :Cc])
 
 
+@pytest.mark.parametrize("Cc,ld", [(41, 256), (172, 176), (47, 64)])
+def test_loss_on_a_column_slice_leaves_the_other_columns_alone(mg, ctx, Cc, ld):
+    """logits / dlogits are n x C views of a wider buffer (ld > round4(C)): columns beyond the pad to a
+    multiple of 4 belong to the caller and must survive, and the result must be the dense layout's."""
+    n = 1500
+    P = synth.uniform_tensor((n, Cc), 160 + Cc, -6, 6)
+    labels = synth.uniform_labels(n, Cc, 161)
+    mask = synth.bernoulli_mask(n, 0.3, 162)
+    lo, G, pred, nc, T = orc.loss(P.numpy(), labels.numpy(), mask.numpy())
+    wide = torch.full((n, ld), 123.0, device="cuda")
+    wide[:, :Cc] = P.cuda()
+    Gw = torch.full((n, ld), -77.0, device="cuda")
+    loss = torch.zeros(1, device="cuda")
+    predd = torch.zeros(n, dtype=torch.int32, device="cuda"); ncd = torch.zeros(1, dtype=torch.int64, device="cuda")
+    mg.loss_softmax_xent(ctx, wide, labels.cuda(), mask.cuda(), loss, Gw, predd, ncd, C_=Cc)
+    assert abs(loss.item() - lo) <= 1e-6 * max(1.0, abs(lo))
+    assert rel_fro(host(Gw, Cc), G) <= TOL_FP32
+    assert np.array_equal(predd.cpu().numpy(), pred) and ncd.item() == nc
+    assert torch.all(Gw[:, round4(Cc):] == -77.0) and torch.all(wide[:, Cc:] == 123.0)
+    # in place over the slice
+    mg.loss_softmax_xent(ctx, wide, labels.cuda(), mask.cuda(), loss, wide, None, None, C_=Cc)
+    assert rel_fro(host(wide, Cc), G) <= TOL_FP32 and torch.all(wide[:, round4(Cc):] == 123.0)
+
+
 def test_loss_closed_form_and_ties(mg, ctx):
     n, Cc = 50, 41
     labels = synth.uniform_labels(n, Cc, 1).cuda()
@@ -551,6 +575,94 @@ def test_gemm_tf32_weight_gradient_form(mg, ctx, M, N, K):
     assert mg.ctx_poll_status(ctx, raise_on_error=False) == 0
 
 
+def _bf16_round(a):
+    """fp32 values rounded to bf16 (nearest, ties to even), as fp64."""
+    u = np.ascontiguousarray(a, dtype=np.float32).view(np.uint32).astype(np.uint64)
+    u = (u + 0x7FFF + ((u >> 16) & 1)) & 0xFFFF0000
+    return u.astype(np.uint32).view(np.float32).astype(np.float64)
+
+
+@pytest.mark.parametrize("M,N,K", TC_SHAPES + [(1000, 256, 1024), (333, 1024, 200)])
+@pytest.mark.parametrize("tb", [False, True])
+def test_gemm_bf16_forward_forms(mg, ctx, M, N, K, tb):
+    """bf16 x bf16 -> fp32 on the tensor cores: within the low-precision bound of the fp64 product, and
+    fp32-accurate against the product of the bf16-rounded operands (which an fp32 or TF32 kernel would miss)."""
+    from helpers import TOL_LOWP
+    A = synth.uniform_tensor((M, K), 231 + M, -1, 1)
+    B = synth.uniform_tensor((N, K) if tb else (K, N), 232 + N, -1, 1)
+    bias = synth.uniform_tensor((N,), 233, -1, 1)
+    Cd = torch.full((M, round4(N) + 4), 3.0, device="cuda")
+    epi = mg.make_epilogue(bias=bias.cuda(), relu=True)
+    before = mg.ctx_gemm_paths(ctx)["tc_bf16"]
+    mg.gemm(ctx, mg.PREC_BF16, False, tb, M, N, K, padded(A, fill=float("nan")), B.cuda().contiguous(), Cd, epi=epi)
+    assert mg.ctx_gemm_paths(ctx)["tc_bf16"] == before + 1          # the bf16 kernel served it, not a fallback
+    Bo = B.numpy().T if tb else B.numpy()
+    want = orc.activation(orc.update(A.numpy(), Bo, bias.numpy()), True)
+    assert rel_fro(host(Cd, N), want) <= TOL_LOWP
+    assert torch.all(Cd[:, round4(N):] == 3.0)
+    want_r = orc.activation(orc.update(_bf16_round(A.numpy()), _bf16_round(Bo), bias.numpy()), True)
+    assert rel_fro(host(Cd, N), want_r) <= 2e-5
+    assert rel_fro(host(Cd, N), want) > 1e-4                         # and it really is a bf16 product
+    assert mg.ctx_poll_status(ctx, raise_on_error=False) == 0
+
+
+@pytest.mark.parametrize("M,N,K", [(128, 128, 64), (64, 32, 4096), (100, 47, 70001), (602, 256, 9000), (1024, 64, 5000),
+                                   (128, 172, 33333), (1024, 1024, 20000)])
+def test_gemm_bf16_weight_gradient_form(mg, ctx, M, N, K):
+    from helpers import TOL_LOWP
+    A, B = synth.normal_features(K, M, 241), synth.normal_features(K, N, 242)
+    Cd = torch.full((M, N), 3.0, device="cuda")
+    before = mg.ctx_gemm_paths(ctx)["tc_bf16"]
+    mg.gemm(ctx, mg.PREC_BF16, True, False, M, N, K, padded(A, fill=float("nan")), padded(B, fill=float("nan")), Cd)
+    assert mg.ctx_gemm_paths(ctx)["tc_bf16"] == before + 1
+    want = A.numpy().astype(np.float64).T @ B.numpy().astype(np.float64)
+    assert rel_fro(host(Cd), want) <= TOL_LOWP
+    want_r = _bf16_round(A.numpy()).T @ _bf16_round(B.numpy())
+    assert rel_fro(host(Cd), want_r) <= 2e-5
+    Cd2 = torch.zeros_like(Cd)
+    mg.gemm(ctx, mg.PREC_BF16, True, False, M, N, K, padded(A, fill=float("nan")), padded(B, fill=float("nan")), Cd2)
+    assert torch.equal(Cd, Cd2)
+    assert mg.ctx_poll_status(ctx, raise_on_error=False) == 0
+
+
+@pytest.mark.parametrize("orders", ["auto", "agg", "upd"])
+@pytest.mark.parametrize("lp_copies", [True, False])
+def test_training_epoch_bf16_within_low_precision_bound(mg, ctx, orders, lp_copies):
+    """A whole iteration with bf16 operands in every dense product: with the bf16 companions written by
+    the producing kernels and with on-the-fly conversion the results are the same bits, and both are
+    within the low-precision bound of the oracle."""
+    from helpers import TOL_LOWP
+    from paper_2501_01951_b200.train import GcnTrainer
+    wl, s, d, X, y, m, Ws, bs = _tiny_problem()
+    go = orc.graph_build(wl.n, s.numpy(), d.numpy())
+    gg = mg.graph_create(ctx, wl.n, s, d)
+    order = {"auto": mg.ORDER_AUTO, "agg": mg.ORDER_AGG_FIRST, "upd": mg.ORDER_UPD_FIRST}[orders]
+    outs = []
+    for copies in ([True, False] if lp_copies else [False]):
+        tr = GcnTrainer(ctx, gg, wl.dims, mg.PREC_BF16, order=order, lp_copies=copies, row_sparse=0)
+        tr.set_params(Ws, bs)
+        tr.set_inputs(padded(X), y.cuda(), m.cuda())
+        before = mg.ctx_gemm_paths(ctx)
+        tr.forward()
+        logits = host(tr.X[-1], wl.classes).astype(np.float64)
+        tr.compute_loss(); tr.backward()
+        after = mg.ctx_gemm_paths(ctx)
+        assert after["tc_bf16"] - before["tc_bf16"] == 3 * tr.L - 1 and after["simt"] == before["simt"] and after["tc_tf32"] == before["tc_tf32"]
+        outs.append((logits, [w.cpu().numpy().astype(np.float64) for w in tr.dW], [b.cpu().numpy().astype(np.float64) for b in tr.db]))
+    if len(outs) == 2:
+        assert np.array_equal(outs[0][0], outs[1][0])
+        for a, b in zip(outs[0][1] + outs[0][2], outs[1][1] + outs[1][2]):
+            assert np.array_equal(a, b)
+    logits, dWs, dbs = outs[0]
+    ref = orc.train_epoch(go, X.numpy(), [w.numpy() for w in Ws], [b.numpy() for b in bs], y.numpy(), m.numpy(), None, 1, **ADAM)
+    assert rel_fro(logits, ref["logits"]) <= TOL_LOWP
+    for l in range(len(dWs)):
+        print(f"bf16 epoch ({orders}): layer {l} rel. Frobenius error dW {rel_fro(dWs[l], ref['dW'][l]):.2e} db {rel_fro(dbs[l], ref['db'][l]):.2e}")
+        assert rel_fro(dWs[l], ref["dW"][l]) <= 2 * TOL_LOWP      # measured values are printed; see the tolerance notes
+    assert mg.ctx_poll_status(ctx, raise_on_error=False) == 0
+    gg.close()
+
+
 def test_training_epoch_tf32_within_low_precision_bound(mg, ctx):
     from helpers import TOL_LOWP
     from paper_2501_01951_b200.train import GcnTrainer
@@ -576,6 +688,8 @@ def test_training_epoch_tf32_within_low_precision_bound(mg, ctx):
         scale_b = np.linalg.norm(np.abs(dP).sum(axis=0))
         assert np.linalg.norm(tr.dW[l].cpu().numpy() - ref["dW"][l]) <= TOL_LOWP * scale_w
         assert np.linalg.norm(tr.db[l].cpu().numpy() - ref["db"][l]) <= TOL_LOWP * scale_b
+        print(f"tf32 epoch: layer {l} rel. Frobenius error dW {rel_fro(tr.dW[l].cpu().numpy(), ref['dW'][l]):.2e} "
+              f"db {rel_fro(tr.db[l].cpu().numpy(), ref['db'][l]):.2e}")
         if l > 0:
             Gout = orc.aggregate(go, dZ, transposed=True)
 

@@ -2,9 +2,11 @@
 
 Collected last on purpose (file name): if it fails, a run that stops at the first failure has
 already run every other test.  It must pass alone in a fresh process and after the other tests."""
+import numpy as np
 import pytest
 import torch
 
+from oracle import gcn_oracle as orc
 from paper_2501_01951_b200 import synth
 
 pytestmark = pytest.mark.gpu
@@ -27,7 +29,8 @@ def _outputs(n, ld, dev):
 def test_noalloc_loss_matches_the_regular_entry_point_twice(mg):
     """Two calls in a row (different inputs, so stale scratch contents would show) against
     mixgcn_loss_softmax_xent: same kernels, so the loss agrees to 1e-6 relative (the partial sums are
-    grouped differently), the gradient and the integer outputs exactly."""
+    grouped differently), the gradient and the integer outputs exactly.  Each call is also held to the
+    CPU oracle within the fp32 tolerance."""
     dev = torch.device("cuda", 0)
     torch.cuda.set_device(dev)
     ctx = mg.ctx_create(0)
@@ -45,6 +48,12 @@ def test_noalloc_loss_matches_the_regular_entry_point_twice(mg):
         assert abs(a["loss"].item() - b["loss"].item()) <= 1e-6 * abs(a["loss"].item())
         assert torch.equal(a["G"], b["G"]) and torch.equal(a["pred"], b["pred"]) and torch.equal(a["nc"], b["nc"])
         assert st.item() == 0
+        # and against the CPU oracle, like the regular entry point's own parity test
+        lo, G, pred, nc, _ = orc.loss(P[:, :Cc].cpu().numpy(), y.cpu().numpy(), m.cpu().numpy())
+        assert abs(b["loss"].item() - lo) <= 1e-6 * max(1.0, abs(lo))
+        Gb = b["G"][:, :Cc].cpu().numpy().astype(np.float64)
+        assert np.linalg.norm(Gb - G) <= 1e-5 * np.linalg.norm(G)
+        assert np.array_equal(b["pred"].cpu().numpy(), pred) and b["nc"].item() == nc
     # device-visible errors come back through the caller's status word, and the next call starts clean
     n, Cc = 64, 5
     P = torch.zeros(n, 8, device=dev); y = torch.zeros(n, dtype=torch.int32, device=dev)
