@@ -77,6 +77,8 @@ __device__ __forceinline__ float tc_apply_epi(const TcEpi& e, float y, int64_t m
     return y;
 }
 
+__device__ __forceinline__ bool aligned16_dev(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
 // 32 consecutive columns of one row as bf16 (round to nearest even); dst is 16-byte aligned when full.
 __device__ __forceinline__ void store_lp_row(uint16_t* dst, const float (&v)[32], int valid) {
     if (valid >= 32) {
@@ -256,7 +258,7 @@ constexpr int KK_BIAS_MAX = 1024;
 // 128-byte swizzle and hands them to TMA stores, which also clip ragged M / N edges; the optional bf16
 // copy of C goes out with 16-byte stores straight from the registers.
 template <int KIND>
-__global__ void __launch_bounds__(KK_THREADS) gemm_tc_kk_kernel(const __grid_constant__ CUtensorMap map_a,
+__global__ void __launch_bounds__(KK_THREADS, 1) gemm_tc_kk_kernel(const __grid_constant__ CUtensorMap map_a,
                                                                 const __grid_constant__ CUtensorMap map_b,
                                                                 const __grid_constant__ CUtensorMap map_c,
                                                                 const TcParams p, const int b_resident, const int tma_store) {
@@ -360,8 +362,15 @@ __global__ void __launch_bounds__(KK_THREADS) gemm_tc_kk_kernel(const __grid_con
     } else {
         // ---------------- epilogue: warp w reads TMEM lanes 32*(w&3).., 32-column chunks (w>>2), (w>>2)+2, ... ----------------
         const int quarter = warp & 3, half = warp >> 2;
-        const bool generic = p.epi.drop != nullptr || p.epi.gate != nullptr || (p.epi.bias != nullptr && !bias_in_smem);
-        const bool add_bias = p.epi.bias != nullptr, relu = p.epi.relu != 0;
+        // The dropout mask and the gate are per-element tensors of C's shape.  With TMA stores they are
+        // applied on the staged box, where a row's 128 bytes belong to eight adjacent lanes (coalesced
+        // reads of the gate); otherwise element by element from the registers, like a bias wider than the
+        // shared-memory copy.
+        const bool post = (p.epi.drop != nullptr || p.epi.gate != nullptr) && tma_store;
+        const bool generic = !post && (p.epi.drop != nullptr || p.epi.gate != nullptr || (p.epi.bias != nullptr && !bias_in_smem));
+        const bool wide_bias = post && p.epi.bias != nullptr && !bias_in_smem;
+        const bool add_bias = p.epi.bias != nullptr && bias_in_smem, relu = p.epi.relu != 0;
+        const bool gate_vec = p.epi.gate != nullptr && aligned16_dev(p.epi.gate) && (p.epi.ld_gate & 3) == 0;
         uint8_t* box = smem_out + (size_t)warp * 4096;
         uint32_t j = 0;
         bool ok = true;
@@ -376,10 +385,22 @@ __global__ void __launch_bounds__(KK_THREADS) gemm_tc_kk_kernel(const __grid_con
             const int64_t m = m0 + quarter * 32 + lane;
             const bool row_ok = m < p.M;
             for (int c0 = half * 32; c0 < p.bn; c0 += 64) {
+                const int nb = n0 + c0;
+                // the gate's 32 x 32 block in the staged-box orientation (lane = row it * 4 + lane / 8,
+                // 16-byte chunk lane % 8), requested before the accumulator is read so that the loads overlap it
+                float4 g4[8];
+                if (post && gate_vec) {
+#pragma unroll
+                    for (int it = 0; it < 8; ++it) {
+                        const int64_t mr = m0 + quarter * 32 + it * 4 + (lane >> 3);
+                        const int nc = nb + (lane & 7) * 4;
+                        g4[it] = (mr < p.M && nc < p.N) ? __ldg(reinterpret_cast<const float4*>(p.epi.gate + (p.epi.row0 + mr) * p.epi.ld_gate + nc))
+                                                         : make_float4(0.f, 0.f, 0.f, 0.f);
+                    }
+                }
                 uint32_t r[32];
                 tc_ld32(tmem_base + buf * acc_stride + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0, r);
                 tc_wait_ld();
-                const int nb = n0 + c0;
                 float v[32];
 #pragma unroll
                 for (int q = 0; q < 32; ++q) v[q] = __uint_as_float(r[q]);
@@ -391,6 +412,10 @@ __global__ void __launch_bounds__(KK_THREADS) gemm_tc_kk_kernel(const __grid_con
                             const float4 b4 = sb4[q];
                             v[4 * q] += b4.x; v[4 * q + 1] += b4.y; v[4 * q + 2] += b4.z; v[4 * q + 3] += b4.w;
                         }
+                    } else if (wide_bias) {
+#pragma unroll
+                        for (int q = 0; q < 32; ++q)
+                            if (nb + q < p.N) v[q] += p.epi.bias[nb + q];
                     }
                     if (relu) {
 #pragma unroll
@@ -401,7 +426,7 @@ __global__ void __launch_bounds__(KK_THREADS) gemm_tc_kk_kernel(const __grid_con
                     for (int q = 0; q < 32; ++q)
                         if (nb + q < p.N) v[q] = tc_apply_epi(p.epi, v[q], m, nb + q, p.N);
                 }
-                if (p.C_lp && row_ok) {
+                if (p.C_lp && row_ok && !post) {
                     const int64_t left = p.N - nb, here = p.bn - c0;
                     const int valid = (int)(left < here ? left : here);
                     store_lp_row(p.C_lp + m * p.ldc_lp + nb, v, valid);
@@ -415,6 +440,46 @@ __global__ void __launch_bounds__(KK_THREADS) gemm_tc_kk_kernel(const __grid_con
                     for (int q = 0; q < 8; ++q)
                         *reinterpret_cast<float4*>(box + lane * 128 + ((q ^ (lane & 7)) << 4)) =
                             make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+                    if (post) {
+                        __syncwarp();
+#pragma unroll
+                        for (int it = 0; it < 8; ++it) {
+                            const int rr = it * 4 + (lane >> 3), ch = lane & 7;
+                            const int64_t mr = m0 + quarter * 32 + rr;
+                            const int nc = nb + ch * 4;
+                            if (mr >= p.M || nc >= p.N || c0 + ch * 4 >= p.bn) continue;
+                            float4* cell = reinterpret_cast<float4*>(box + rr * 128 + ((ch ^ (rr & 7)) << 4));
+                            const float4 y4 = *cell;
+                            float y[4] = {y4.x, y4.y, y4.z, y4.w};
+                            const int nv = p.N - nc < 4 ? (int)(p.N - nc) : 4;
+                            if (p.epi.drop) {
+                                const uint8_t* dm = p.epi.drop + (p.epi.row0 + mr) * p.N + nc;
+#pragma unroll
+                                for (int t = 0; t < 4; ++t) if (t < nv) y[t] = dm[t] ? y[t] * p.epi.keep_scale : 0.0f;
+                            }
+                            if (p.epi.gate) {
+                                const float* gp = p.epi.gate + (p.epi.row0 + mr) * p.epi.ld_gate + nc;
+                                float gq[4] = {0.f, 0.f, 0.f, 0.f};
+                                if (gate_vec) {       // the whole group lies inside the row's allocation (ld_gate % 4 == 0)
+                                    gq[0] = g4[it].x; gq[1] = g4[it].y; gq[2] = g4[it].z; gq[3] = g4[it].w;
+                                } else {
+#pragma unroll
+                                    for (int t = 0; t < 4; ++t) if (t < nv) gq[t] = __ldg(gp + t);
+                                }
+#pragma unroll
+                                for (int t = 0; t < 4; ++t) y[t] = gq[t] > 0.0f ? y[t] * p.epi.gate_scale : 0.0f;
+                            }
+                            *cell = make_float4(y[0], y[1], y[2], y[3]);
+                            if (p.C_lp) {
+                                uint16_t* dl = p.C_lp + mr * p.ldc_lp + nc;
+                                if (nv == 4) *reinterpret_cast<uint2*>(dl) = make_uint2(pack_bf16(y[0], y[1]), pack_bf16(y[2], y[3]));
+                                else {
+#pragma unroll
+                                    for (int t = 0; t < 4; ++t) if (t < nv) dl[t] = (uint16_t)(pack_bf16(y[t], 0.0f) & 0xFFFFu);
+                                }
+                            }
+                        }
+                    }
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                     __syncwarp();
                     if (lane == 0) {

@@ -110,6 +110,13 @@ def main():
             step[0] += 1
             tr.epoch(step[0])
         med, best = _time(one, args.iters, args.warmup)
+        mg.ctx_profile_read(ctx)
+        mg.ctx_profile_enable(ctx, True)
+        for _ in range(args.iters):
+            one()
+        phase_ms, _, _ = mg.ctx_profile_read(ctx)
+        mg.ctx_profile_enable(ctx, False)
+        out.update(phase_ms_per_epoch={k: round(v / args.iters, 3) for k, v in phase_ms.items()}, paths=mg.ctx_gemm_paths(ctx))
         out.update(model=args.model, n=g.n, nnz=g.nnz, dims=list(dims), precision=args.precision, loss=round(tr.loss.item(), 6),
                    ms_median=round(med, 4), ms_best=round(best, 4), epochs_per_s=round(1e3 / med, 3),
                    device_status=mg.ctx_poll_status(ctx, raise_on_error=False))
@@ -140,9 +147,21 @@ def main():
         Cm = torch.zeros((M, r4(N)), device=dev)
         prec = mg.PRECISIONS[args.precision]
         med, best = _time(lambda: mg.gemm(ctx, prec, bool(args.ta), bool(args.tb), M, N, K, A, B, Cm), args.iters, args.warmup)
+        # the product's own kernels (phase "gemm"), apart from the on-the-fly bf16 conversion of fp32
+        # operands (phase "elementwise") that a layer avoids by having its producers write bf16 copies
+        mg.ctx_profile_read(ctx)
+        mg.ctx_profile_enable(ctx, True)
+        for _ in range(args.iters):
+            mg.gemm(ctx, prec, bool(args.ta), bool(args.tb), M, N, K, A, B, Cm)
+        phase_ms, _, _ = mg.ctx_profile_read(ctx)
+        mg.ctx_profile_enable(ctx, False)
+        kern = phase_ms["gemm"] / args.iters
         out.update(M=M, N=N, K=K, ta=args.ta, tb=args.tb, precision=args.precision, ms_median=round(med, 4),
                    ms_best=round(best, 4), tflops=round(2 * M * N * K / med / 1e9, 2),
-                   min_gbs=round(4 * (M * K + K * N + M * N) / med / 1e6, 1))
+                   min_gbs=round(4 * (M * K + K * N + M * N) / med / 1e6, 1),
+                   kernel_ms=round(kern, 4), kernel_tflops=round(2 * M * N * K / kern / 1e9, 2) if kern > 0 else None,
+                   convert_ms=round(phase_ms["elementwise"] / args.iters, 4), paths=mg.ctx_gemm_paths(ctx),
+                   device_status=mg.ctx_poll_status(ctx, raise_on_error=False))
     print(json.dumps(out), flush=True)
 
 
