@@ -224,7 +224,9 @@ class GcnTrainer:
         mg.loss_softmax_xent(self.ctx, self.X[self.L], self.labels, self.train_mask, self.loss,
                              dlogits=self.X[self.L], pred=self.pred, n_correct=self.n_correct, C_=self.dims[-1])
 
-    def backward(self):
+    def backward(self, on_layer=None):
+        """on_layer(l, "before" | "after"), if given, is called around each layer's backward call (tests
+        use it to look at a layer's operands before the call consumes them)."""
         for l in range(self.L - 1, -1, -1):
             d = self.descs[l]
             if d.gout_row_mask and d.gout_row_count == 0 and self.row_masks[l + 1] is not self.train_mask:
@@ -232,8 +234,12 @@ class GcnTrainer:
                 # mask only, so its count is taken once (a stream synchronisation) and kept; with the
                 # count layer_bwd can run its dense products on the compacted rows.
                 d.gout_row_count = mg.count_rows(self.ctx, self.row_masks[l + 1])
+            if on_layer is not None:
+                on_layer(l, "before")
             mg.layer_bwd(self.ctx, self.g, d, self.X[l], self.saved[l], self.X[l + 1], self.masks[l],
                          self.W[l], self.G[l + 1], self.G[l] if l > 0 else None, self.dW[l], self.db[l])
+            if on_layer is not None:
+                on_layer(l, "after")
 
     def step(self, t, lr=0.01, beta1=0.9, beta2=0.999, eps=1e-8):
         mg.adam_step(self.ctx, self.W + self.b, self.dW + self.db, self.mW + self.mb, self.vW + self.vb, t,
