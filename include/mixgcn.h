@@ -169,8 +169,10 @@ mixgcn_status mixgcn_graph_destroy(mixgcn_graph* g);
  * mixgcn_graph_rcm: the reverse Cuthill-McKee order of a symmetric graph into `order` (host
  *   int32[n]): components start from the unvisited node with the fewest entries (lowest id on ties), a
  *   visited node appends its unvisited neighbours by increasing entry count (lowest id on ties), and
- *   the sequence is reversed.  A host (C++) breadth-first search, as the paper's preprocessing is;
- *   synchronises and copies the structure to the host.  MIXGCN_EUNSUPPORTED if not symmetric.
+ *   the sequence is reversed.  Runs on the device as a level-synchronous breadth-first search (a
+ *   level's nodes sorted by the position of their earliest-placed neighbour, then entry count, then id:
+ *   the order a one-node-at-a-time queue gives); the paper's preprocessing is a CPU program.
+ *   Synchronises (once per level).  MIXGCN_EUNSUPPORTED if not symmetric.
  * mixgcn_pipeline_stages: the stage count ceil(2n / (n - b)) of Proposition 3.5 (idleness is
  *   eliminated when (n - b) / (2n) >= 1 / s); MIXGCN_EINVAL when b >= n.
  * mixgcn_graph_create_permuted: a new graph in which node order[k] has become node k (same

@@ -46,7 +46,9 @@ def test_rcm_and_bandwidth_match_the_oracle(mg, case):
     assert mg.graph_bandwidth(gg) == orc.bandwidth(go)
     order = mg.graph_rcm(gg)
     want = orc.rcm(go)
-    assert np.array_equal(order.numpy().astype(np.int64), want)              # same rule, same ties: identical order
+    # a level-synchronous device search against the oracle's one-node-at-a-time queue: same rule and
+    # ties, so the same order although the two share no structure
+    assert np.array_equal(order.numpy().astype(np.int64), want)
     b = mg.graph_bandwidth(gg, order)
     assert b == orc.bandwidth(go, want)
     if name == "scrambled-path":
@@ -81,3 +83,64 @@ def test_rcm_needs_a_symmetric_graph(mg):
         mg.graph_rcm(gg)
     assert e.value.status == mg.EUNSUPPORTED
     gg.close(); ctx.close()
+
+
+def _grid_edges(rows, cols):
+    """A rows x cols grid graph under scrambled labels: a graph that HAS locality for the ordering to find."""
+    ids = np.arange(rows * cols).reshape(rows, cols)
+    s = np.concatenate([ids[:, :-1].ravel(), ids[:-1, :].ravel()])
+    d = np.concatenate([ids[:, 1:].ravel(), ids[1:, :].ravel()])
+    lab = np.random.default_rng(21).permutation(rows * cols)
+    return rows * cols, lab[s], lab[d]
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("kind", ["grid", "rmat"])
+def test_pipeline_with_the_stage_count_of_the_reordered_graph(mg, kind):
+    """The fine-grain pipeline as Section 3.2.2 composes it: reorder the nodes (RCM), take the stage count
+    s = ceil(2n / (n - b)) of Proposition 3.5 from the bandwidth b of the new order, and run the layer in s
+    row chunks (aggregation of chunk k+1 overlapping the update of chunk k).  Forward output and every
+    gradient must be the oracle's on the permuted inputs."""
+    from helpers import round4
+    if kind == "grid":
+        n, s, d = _grid_edges(40, 50)
+    else:
+        n = 4096
+        ss, dd = synth.rmat_graph(n, 32768, 1001)
+        s, d = ss.numpy(), dd.numpy()
+    ctx = mg.ctx_create(0)
+    g0 = mg.graph_create(ctx, n, torch.tensor(s, dtype=torch.int32), torch.tensor(d, dtype=torch.int32))
+    order = mg.graph_rcm(g0)
+    b = mg.graph_bandwidth(g0, order)
+    stages = mg.pipeline_stages(n, b)
+    assert stages == orc.pipeline_stages(n, b) and stages >= 3
+    if kind == "grid":
+        assert b <= 2 * 50 and stages == 3          # the ordering recovered the grid's band: the smallest stage count
+    n_chunks = min(stages, 64)
+    gp = mg.graph_create_permuted(ctx, g0, order)
+    assert mg.graph_bandwidth(gp) == b
+    # the oracle sees the relabelled edge list and the permuted inputs
+    o = order.numpy().astype(np.int64)
+    pos = np.empty(n, dtype=np.int64); pos[o] = np.arange(n)
+    go = orc.graph_build(n, pos[np.asarray(s)], pos[np.asarray(d)])
+    d_in, d_out = 48, 40
+    X = synth.uniform_tensor((n, d_in), 31, -1, 1)[torch.tensor(o)]
+    W = synth.glorot_uniform(d_in, d_out, 32)
+    bias = synth.uniform_tensor((d_out,), 33, -0.2, 0.2)
+    Gout = synth.uniform_tensor((n, d_out), 34, -1, 1)[torch.tensor(o)]
+    desc = mg.layer_desc(d_in, d_out, round4(d_in), round4(d_out), round4(d_in), mg.ORDER_AGG_FIRST, mg.PREC_FP32,
+                         mg.LAYER_RELU, 1.0, 1.0, n_chunks)
+    Xd, Wd, bd = padded(X), W.cuda(), bias.cuda()
+    saved = torch.zeros(n, round4(d_in), device="cuda"); Xout = torch.zeros(n, round4(d_out), device="cuda")
+    mg.layer_fwd(ctx, gp, desc, Xd, Wd, bd, None, saved, Xout)
+    Z = orc.aggregate(go, X.numpy())
+    P = orc.update(Z, W.numpy(), bias.numpy())
+    assert rel_fro(host(Xout, d_out), orc.activation(P, True)) <= TOL_FP32
+    Gd = padded(Gout); Gin = torch.zeros(n, round4(d_in), device="cuda")
+    dW = torch.zeros(d_in, d_out, device="cuda"); db = torch.zeros(d_out, device="cuda")
+    mg.layer_bwd(ctx, gp, desc, Xd, saved, Xout, None, Wd, Gd, Gin, dW, db)
+    _, dWo, dbo, dZo = orc.update_bwd(Z, P, W.numpy(), Gout.numpy(), True, None, 1.0, need_dZ=True)
+    assert rel_fro(host(dW), dWo) <= TOL_FP32 and rel_fro(db.cpu().numpy(), dbo) <= TOL_FP32
+    assert rel_fro(host(Gin, d_in), orc.aggregate(go, dZo, transposed=True)) <= TOL_FP32
+    assert mg.ctx_poll_status(ctx, raise_on_error=False) == 0
+    gp.close(); g0.close(); ctx.close()
