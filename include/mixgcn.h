@@ -445,7 +445,8 @@ mixgcn_status mixgcn_adam_step(mixgcn_ctx* ctx, int32_t n_tensors, float* const*
  * gradient are computed on the train rows alone (nothing returned depends on the other rows).
  * The row plans of the backward pass are kept in the context and reused by the next call while the
  * graph and the train mask are unchanged (the mask is compared on the device every call).
- * Device buffers are taken from the context workspace (grown on demand).  Synchronises. */
+ * Device buffers are taken from the context workspace (grown on demand).  Synchronises the streams it
+ * used, except for a feature copy started for the next call (mixgcn_train_step_host_prefetch). */
 mixgcn_status mixgcn_train_step_host(mixgcn_ctx* ctx, const mixgcn_graph* g, int32_t L,
                                      const int32_t* dims, int32_t precision, const float* X,
                                      const int32_t* labels, const uint8_t* train_mask,
@@ -453,6 +454,27 @@ mixgcn_status mixgcn_train_step_host(mixgcn_ctx* ctx, const mixgcn_graph* g, int
                                      float* const* vW, float* const* mb, float* const* vb,
                                      int64_t t, float lr, float beta1, float beta2, float eps,
                                      float* loss, int32_t* pred);
+
+/* Announces the features the NEXT mixgcn_train_step_host call on this context will be given (host
+ * pointer, same n x d_0 shape; pinned memory if the copy is to overlap anything).  The call that runs
+ * before it then starts that host-to-device copy itself, on a second stream, as soon as its own
+ * features are no longer needed (after the first layer's forward in agg-first order, whose backward
+ * reads A_hat X from `saved` and not X), so the copy overlaps the rest of that iteration; the next
+ * call, given the same pointer, waits for it instead of copying again.  The buffer must stay valid and
+ * unchanged until that next call returns.  One announcement serves one call; with a first layer in
+ * upd-first order, or when the next call passes another pointer, nothing is lost but the overlap.
+ * Not in the paper: Algorithm 2 keeps its inputs resident. */
+mixgcn_status mixgcn_train_step_host_prefetch(mixgcn_ctx* ctx, const float* X_next);
+
+/* Measurement helper (the paper has no counterpart): `table` is rows x 128 fp32 on the device; every
+ * warp of a grid that fills the GPU reads gathers_per_warp (a multiple of 8) pseudo-random rows of 512
+ * bytes, eight in flight, and discards them.  *total_gathers (host, nullable) receives the number of rows
+ * read; time the call with events on `stream`: rows * 512 bytes / time is the row-gather rate of the
+ * memory level the table lives in (L2 when it fits, HBM otherwise) -- the denominator the benchmark
+ * quotes aggregations with an L2-resident input against.  `sink` is one device float, never written
+ * in practice. */
+mixgcn_status mixgcn_probe_gather(mixgcn_ctx* ctx, const float* table, int64_t rows, int64_t gathers_per_warp,
+                                  uint64_t seed, float* sink, int64_t* total_gathers, void* stream);
 
 #ifdef __cplusplus
 }

@@ -44,6 +44,7 @@ SYMBOLS = (
     "mixgcn_graph_bandwidth", "mixgcn_graph_rcm", "mixgcn_pipeline_stages", "mixgcn_graph_create_permuted",
     "mixgcn_count_rows", "mixgcn_rowplan_create", "mixgcn_rowplan_destroy", "mixgcn_rowplan_info",
     "mixgcn_rowplan_export", "mixgcn_spmm_rowplan", "mixgcn_colsum", "mixgcn_ctx_gemm_paths",
+    "mixgcn_train_step_host_prefetch", "mixgcn_probe_gather",
 )
 
 
@@ -229,6 +230,13 @@ def graph_export(g: Graph, transposed: bool = False):
     _check(lib.mixgcn_graph_export(g.h, C.c_int(int(transposed)), _ptr(out["rowptr"]), _ptr(out["col"]),
                                    _ptr(out["val"]), _ptr(out["deg"]), _ptr(out["dinv"])))
     return out
+
+
+def graph_degrees(g: Graph) -> torch.Tensor:
+    """Entries per row of the stored matrix (host int32); on a symmetric graph also the number of rows that gather node v."""
+    deg = torch.empty(g.n, dtype=torch.int32)
+    _check(lib.mixgcn_graph_export(g.h, C.c_int(0), None, None, None, _ptr(deg), None))
+    return deg
 
 
 def graph_export_schedule(g: Graph, transposed: bool = False) -> torch.Tensor:
@@ -462,3 +470,21 @@ def train_step_host(ctx: Ctx, g: Graph, dims, precision, X, labels, train_mask, 
                                       C.c_int64(t), C.c_float(lr), C.c_float(beta1), C.c_float(beta2), C.c_float(eps),
                                       C.byref(loss), _ptr(pred)))
     return loss.value
+
+
+def train_step_host_prefetch(ctx: Ctx, X_next):
+    """Announce the (pinned) host features of the next train_step_host call so that the call before it overlaps their copy."""
+    if X_next is not None and (X_next.is_cuda or not X_next.is_contiguous()):
+        raise TypeError("train_step_host_prefetch takes a contiguous host tensor")
+    _check(lib.mixgcn_train_step_host_prefetch(ctx.h, _ptr(X_next)))
+
+
+def probe_gather(ctx: Ctx, table: torch.Tensor, gathers_per_warp: int, sink: torch.Tensor, seed: int = 1) -> int:
+    """Enqueue the row-gather probe on a rows x 128 fp32 table; returns the number of rows it reads."""
+    table, ld = _mat(table, "table")
+    if ld != 128 or table.shape[1] != 128:
+        raise TypeError("table: expected a dense rows x 128 fp32 tensor")
+    total = C.c_int64(0)
+    _check(lib.mixgcn_probe_gather(ctx.h, _ptr(table), C.c_int64(table.shape[0]), C.c_int64(gathers_per_warp),
+                                   C.c_uint64(seed), _ptr(sink), C.byref(total), _stream()))
+    return total.value

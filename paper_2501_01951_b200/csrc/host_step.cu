@@ -19,6 +19,15 @@ struct HostStepCache {
     mixgcn_rowplan* plan[2] = {nullptr, nullptr};
 };
 
+// Feature prefetch between calls of mixgcn_train_step_host (see mixgcn_train_step_host_prefetch).
+struct HostStepPrefetch {
+    const float* announced = nullptr;   // host pointer the caller announced for the next call
+    const float* in_flight = nullptr;   // host pointer whose copy into X[0] was started by the last call
+    float* dst = nullptr;               // where it was copied to
+    int64_t n = 0, d0 = 0;
+    cudaEvent_t done = nullptr;         // recorded after that copy
+};
+
 namespace {
 
 __global__ void mask_differs_kernel(int64_t n, const uint8_t* __restrict__ a, const uint8_t* __restrict__ b, int32_t* differs) {
@@ -96,6 +105,11 @@ mixgcn_status lay_out(char* base, int64_t n, int L, const int32_t* dims, int pre
 
 namespace mixgcn {
 void free_step_cache(mixgcn_ctx* ctx) {
+    if (HostStepPrefetch* pf = ctx->step_prefetch) {
+        if (pf->done) cudaEventDestroy(pf->done);
+        delete pf;
+        ctx->step_prefetch = nullptr;
+    }
     HostStepCache* c = ctx->step_cache;
     if (!c) return;
     drop_plans(c);
@@ -125,8 +139,10 @@ extern "C" mixgcn_status mixgcn_train_step_host(mixgcn_ctx* ctx, const mixgcn_gr
     const int64_t n = g->n;
     StepLayout lo;
     MIXGCN_TRY(lay_out(nullptr, n, L, dims, precision, lo));
+    HostStepPrefetch* pf = ctx->step_prefetch;
     if (lo.bytes > ctx->arena_bytes) {
         MIXGCN_CUDA(cudaDeviceSynchronize());
+        if (pf) pf->in_flight = nullptr;        // the buffer a prefetch went to is gone
         cudaFree(ctx->arena); ctx->arena = nullptr; ctx->arena_bytes = 0;
         void* p = nullptr;
         if (cudaMalloc(&p, (size_t)lo.bytes) != cudaSuccess) {
@@ -200,8 +216,18 @@ extern "C" mixgcn_status mixgcn_train_step_host(mixgcn_ctx* ctx, const mixgcn_gr
 
     // inputs
     const int64_t d0 = dims[0], ld0 = round4(d0);
-    if (ld0 == d0) MIXGCN_CUDA(cudaMemcpyAsync(lo.X[0], X, (size_t)(n * d0) * sizeof(float), H2D, s));
-    else MIXGCN_CUDA(cudaMemcpy2DAsync(lo.X[0], ld0 * sizeof(float), X, d0 * sizeof(float), d0 * sizeof(float), (size_t)n, H2D, s));
+    auto copy_features = [&](const float* src, cudaStream_t st) -> cudaError_t {
+        if (ld0 == d0) return cudaMemcpyAsync(lo.X[0], src, (size_t)(n * d0) * sizeof(float), H2D, st);
+        return cudaMemcpy2DAsync(lo.X[0], ld0 * sizeof(float), src, d0 * sizeof(float), d0 * sizeof(float), (size_t)n, H2D, st);
+    };
+    if (pf && pf->in_flight == X && pf->dst == lo.X[0] && pf->n == n && pf->d0 == d0) {
+        // the previous call already started this copy: wait for it instead of copying again
+        MIXGCN_CUDA(cudaStreamWaitEvent(s, pf->done, 0));
+    } else {
+        if (pf && pf->in_flight) MIXGCN_CUDA(cudaStreamWaitEvent(s, pf->done, 0));   // a stale prefetch still writes X[0]: let it finish first
+        MIXGCN_CUDA(copy_features(X, s));
+    }
+    if (pf) pf->in_flight = nullptr;
     MIXGCN_CUDA(cudaMemcpyAsync(lo.labels, labels, n * sizeof(int32_t), H2D, s));
     for (int l = 0; l < L; ++l) {
         const size_t wb = (size_t)dims[l] * dims[l + 1] * sizeof(float), bb = (size_t)dims[l + 1] * sizeof(float);
@@ -213,8 +239,21 @@ extern "C" mixgcn_status mixgcn_train_step_host(mixgcn_ctx* ctx, const mixgcn_gr
         MIXGCN_CUDA(cudaMemcpyAsync(lo.vb[l], vb[l], bb, H2D, s));
     }
     // forward, loss, backward, update
-    for (int l = 0; l < L; ++l)
+    for (int l = 0; l < L; ++l) {
         MIXGCN_TRY(mixgcn_layer_fwd(ctx, g, &lo.desc[l], lo.X[l], lo.W[l], lo.b[l], nullptr, lo.saved[l], lo.X[l + 1], s));
+        if (l == 0 && pf && pf->announced && lo.desc[0].order == MIXGCN_ORDER_AGG_FIRST) {
+            // In agg-first order nothing after the first layer's forward reads the features again (its
+            // backward uses A_hat X from `saved`): the announced features of the NEXT call are copied
+            // into X[0] on the second stream while the rest of this iteration runs.
+            cudaStream_t s2 = ctx->side_stream[1];
+            MIXGCN_CUDA(cudaEventRecord(ctx->fork_ev, s));
+            MIXGCN_CUDA(cudaStreamWaitEvent(s2, ctx->fork_ev, 0));
+            MIXGCN_CUDA(copy_features(pf->announced, s2));
+            MIXGCN_CUDA(cudaEventRecord(pf->done, s2));
+            pf->in_flight = pf->announced; pf->dst = lo.X[0]; pf->n = n; pf->d0 = d0;
+        }
+    }
+    if (pf) pf->announced = nullptr;
     {
         const int keep = ctx->loss_train_rows_only;
         ctx->loss_train_rows_only = rows_only ? 1 : keep;
@@ -244,5 +283,21 @@ extern "C" mixgcn_status mixgcn_train_step_host(mixgcn_ctx* ctx, const mixgcn_gr
         MIXGCN_CUDA(cudaMemcpyAsync(vb[l], lo.vb[l], bb, D2H, s));
     }
     MIXGCN_CUDA(cudaStreamSynchronize(s));
+    return MIXGCN_OK;
+}
+
+extern "C" mixgcn_status mixgcn_train_step_host_prefetch(mixgcn_ctx* ctx, const float* X_next) {
+    if (!ctx) MIXGCN_FAIL(MIXGCN_EINVAL, "train_step_host_prefetch: null ctx");
+    MIXGCN_CUDA(cudaSetDevice(ctx->device));
+    if (!ctx->step_prefetch) {
+        HostStepPrefetch* pf = new (std::nothrow) HostStepPrefetch();
+        if (!pf) MIXGCN_FAIL(MIXGCN_ENOMEM, "train_step_host_prefetch: host allocation failed");
+        if (cudaEventCreateWithFlags(&pf->done, cudaEventDisableTiming) != cudaSuccess) {
+            delete pf;
+            MIXGCN_FAIL(MIXGCN_ECUDA, "train_step_host_prefetch: event creation failed");
+        }
+        ctx->step_prefetch = pf;
+    }
+    ctx->step_prefetch->announced = X_next;
     return MIXGCN_OK;
 }

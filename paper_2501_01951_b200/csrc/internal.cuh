@@ -75,6 +75,7 @@ struct mixgcn_ctx {
     int64_t arena_bytes;
     // row plans of the last mixgcn_train_step_host call, reused while graph and train mask stay the same
     struct HostStepCache* step_cache;
+    struct HostStepPrefetch* step_prefetch;
 };
 
 // One unit of aggregation work: `len` stored entries starting at `begin`.  For an ordinary row `row`

@@ -526,6 +526,38 @@ def test_train_step_host_matches_oracle_and_device_path(mg, ctx):
     assert abs(loss - ref["loss"]) <= 1e-5 * abs(ref["loss"])
 
 
+def test_train_step_host_prefetch_gives_the_same_iterations(mg):
+    """Announcing the next call's features lets a call start their copy early; the iterations must be the
+    ones without the announcement, bit for bit, also when the features change between calls, when the
+    announcement is not honoured by the next call, and with the oracle's loss on the first step."""
+    wl, s, d, X, y, m, Ws, bs = _tiny_problem()
+    Xa = X.clone().pin_memory()
+    Xb = (X * 0.5 + 0.25).contiguous().pin_memory()
+    feats = [Xa, Xb, Xb, Xa, Xa]
+    results = []
+    for announce in (False, True):
+        c = mg.ctx_create(0)
+        gg = mg.graph_create(c, wl.n, s, d)
+        W = [w.clone() for w in Ws]; b = [x.clone() for x in bs]
+        z = lambda lst: [torch.zeros_like(x) for x in lst]
+        mW, vW, mb, vb = z(W), z(W), z(b), z(b)
+        losses = []
+        for t, Xt in enumerate(feats, start=1):
+            if announce and t < len(feats):
+                # step 3 announces a buffer the next call does not use: the announcement must simply lapse
+                mg.train_step_host_prefetch(c, Xb if t == 3 else feats[t])
+            losses.append(mg.train_step_host(c, gg, wl.dims, mg.PREC_FP32, Xt, y, m, W, b, mW, vW, mb, vb, t, **ADAM))
+        assert mg.ctx_poll_status(c, raise_on_error=False) == 0
+        results.append((losses, [w.clone() for w in W], [x.clone() for x in b]))
+        gg.close(); c.close()
+    assert results[0][0] == results[1][0]
+    for a, b_ in zip(results[0][1] + results[0][2], results[1][1] + results[1][2]):
+        assert torch.equal(a, b_)
+    go = orc.graph_build(wl.n, s.numpy(), d.numpy())
+    ref = orc.train_epoch(go, X.numpy(), [w.numpy() for w in Ws], [x.numpy() for x in bs], y.numpy(), m.numpy(), None, 1, **ADAM)
+    assert abs(results[1][0][0] - ref["loss"]) <= 1e-5 * abs(ref["loss"])
+
+
 # --------------------------------------------------------------------------- tensor-core products
 
 def _tf32_trunc(a):
