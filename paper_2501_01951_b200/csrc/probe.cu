@@ -23,15 +23,19 @@ __global__ void __launch_bounds__(256) probe_gather_kernel(const float* __restri
     const int lane = threadIdx.x & 31;
     const uint64_t warp = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int64_t i = 0; i < per_warp; i += 8) {
-        float4 y[8];
+    for (int64_t i = 0; i < per_warp; i += 32) {
+        // lane l draws the row of gather i + l (uniform in [0, rows) by a multiply-high: no division in the loop)
+        const uint64_t mine = __umul64hi(probe_mix(seed ^ (warp * 0x100000001B3ull + (uint64_t)(i + lane))), (uint64_t)rows);
+        for (int t0 = 0; t0 < 32 && i + t0 < per_warp; t0 += 8) {
+            float4 y[8];
 #pragma unroll
-        for (int t = 0; t < 8; ++t) {
-            const uint64_t r = probe_mix(seed ^ (warp * 0x100000001B3ull + (uint64_t)(i + t))) % (uint64_t)rows;
-            y[t] = __ldg(reinterpret_cast<const float4*>(table + r * 128) + lane);
+            for (int t = 0; t < 8; ++t) {
+                const uint64_t r = __shfl_sync(0xFFFFFFFFu, mine, t0 + t);
+                y[t] = __ldg(reinterpret_cast<const float4*>(table + r * 128) + lane);
+            }
+#pragma unroll
+            for (int t = 0; t < 8; ++t) { acc.x += y[t].x; acc.y += y[t].y; acc.z += y[t].z; acc.w += y[t].w; }
         }
-#pragma unroll
-        for (int t = 0; t < 8; ++t) { acc.x += y[t].x; acc.y += y[t].y; acc.z += y[t].z; acc.w += y[t].w; }
     }
     if (acc.x + acc.y + acc.z + acc.w == 1.2345678e38f) sink[0] = acc.x;
 }
