@@ -91,13 +91,18 @@ mixgcn_status mixgcn_ctx_poll_status(mixgcn_ctx* ctx, int32_t* code);
  * mixgcn_ctx_poll_status then gives MIXGCN_ETIMEOUT.  Nothing traps, spins without limit or faults. */
 #define MIXGCN_OPT_DEBUG_WAIT_LIMIT 3
 #define MIXGCN_OPT_DEBUG_DROP_LOAD 4
+/* MIXGCN_OPT_GEMM_CTA_PAIRS: 1 (default) = wide and deep K-major products (N >= 512, K >= 512, M >= 4096)
+ * run on pairs of CTAs that share one 256 x 256 tile (tcgen05 .cta_group::2); 0 = every product on single
+ * CTAs with 128 x 256 tiles.  Same results up to the order of fp32 accumulation inside the tensor core. */
+#define MIXGCN_OPT_GEMM_CTA_PAIRS 5
 mixgcn_status mixgcn_ctx_set_option(mixgcn_ctx* ctx, int32_t option, int64_t value);
 
 /* Which kernel served the dense products of this context since it was created: counts[0] fp32 FMA
- * kernel, counts[1] tcgen05 with TF32 operands, counts[2] tcgen05 with BF16 operands.  A TF32 or BF16
- * request whose shape or alignment the tensor-core kernels do not take is served by the next kernel
- * down that list (never a lower precision than asked for); these counters make that visible. */
-mixgcn_status mixgcn_ctx_gemm_paths(const mixgcn_ctx* ctx, int64_t counts[3]);
+ * kernel, counts[1] tcgen05 with TF32 operands, counts[2] tcgen05 with BF16 operands; counts[3] = how
+ * many of the tcgen05 products ran on CTA pairs.  A TF32 or BF16 request whose shape or alignment the
+ * tensor-core kernels do not take is served by the next kernel down that list (never a lower precision
+ * than asked for); these counters make that visible. */
+mixgcn_status mixgcn_ctx_gemm_paths(const mixgcn_ctx* ctx, int64_t counts[4]);
 
 /* Per-phase profiling.  While enabled the library brackets every kernel it launches with
  * CUDA events on the launching stream.  mixgcn_ctx_profile_read synchronises and returns, for

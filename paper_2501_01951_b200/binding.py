@@ -146,6 +146,7 @@ OPT_SPMM_SLICE_COLS = 1
 OPT_LOSS_TRAIN_ROWS_ONLY = 2
 OPT_DEBUG_WAIT_LIMIT = 3
 OPT_DEBUG_DROP_LOAD = 4
+OPT_GEMM_CTA_PAIRS = 5
 
 
 def ctx_set_option(ctx: Ctx, option: int, value: int):
@@ -154,9 +155,9 @@ def ctx_set_option(ctx: Ctx, option: int, value: int):
 
 def ctx_gemm_paths(ctx: Ctx) -> dict:
     """Dense products served so far by the fp32 FMA kernel, the tcgen05 TF32 kernels, the tcgen05 BF16 kernels."""
-    counts = (C.c_int64 * 3)()
+    counts = (C.c_int64 * 4)()
     _check(lib.mixgcn_ctx_gemm_paths(ctx.h, counts))
-    return dict(simt=int(counts[0]), tc_tf32=int(counts[1]), tc_bf16=int(counts[2]))
+    return dict(simt=int(counts[0]), tc_tf32=int(counts[1]), tc_bf16=int(counts[2]), cta_pairs=int(counts[3]))
 
 
 def ctx_profile_enable(ctx: Ctx, enable: bool = True):

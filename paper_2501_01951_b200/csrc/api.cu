@@ -247,6 +247,11 @@ extern "C" mixgcn_status mixgcn_ctx_set_option(mixgcn_ctx* ctx, int32_t option, 
         ctx->loss_train_rows_only = (int)value;
         return MIXGCN_OK;
     }
+    if (option == MIXGCN_OPT_GEMM_CTA_PAIRS) {
+        if (value != 0 && value != 1) MIXGCN_FAIL(MIXGCN_EINVAL, "ctx_set_option: cta-pairs takes 0 or 1 (got %lld)", (long long)value);
+        ctx->no_cta_pairs = value ? 0 : 1;
+        return MIXGCN_OK;
+    }
     if (option == MIXGCN_OPT_DEBUG_WAIT_LIMIT) {
         if (value < 0 || value > (1ll << 30)) MIXGCN_FAIL(MIXGCN_EINVAL, "ctx_set_option: wait limit must lie in [0, 2^30] (got %lld)", (long long)value);
         ctx->debug_wait_limit = (int)value;
@@ -260,9 +265,10 @@ extern "C" mixgcn_status mixgcn_ctx_set_option(mixgcn_ctx* ctx, int32_t option, 
     MIXGCN_FAIL(MIXGCN_EINVAL, "ctx_set_option: unknown option %d", option);
 }
 
-extern "C" mixgcn_status mixgcn_ctx_gemm_paths(const mixgcn_ctx* ctx, int64_t counts[3]) {
+extern "C" mixgcn_status mixgcn_ctx_gemm_paths(const mixgcn_ctx* ctx, int64_t counts[4]) {
     if (!ctx || !counts) MIXGCN_FAIL(MIXGCN_EINVAL, "ctx_gemm_paths: null argument");
     for (int i = 0; i < 3; ++i) counts[i] = ctx->gemm_path[i];
+    counts[3] = ctx->gemm_pair_launches;
     return MIXGCN_OK;
 }
 

@@ -517,6 +517,267 @@ __global__ void __launch_bounds__(KK_THREADS, 1) gemm_tc_kk_kernel(const __grid_
     }
 }
 
+// The same persistent K-major product on PAIRS of CTAs (a thread-block cluster of two, tcgen05
+// .cta_group::2): a pair owns a 256 x 256 output tile.  Each CTA loads its own 128 rows of A and its own
+// half (128 rows) of the packed B tile per stage -- 32 KB per CTA instead of the 48 KB a lone CTA needs
+// for a 128 x 256 tile, which is what the L2-to-shared-memory path and the operand reads from shared
+// memory were short of -- and the pair's leader (even cluster rank) issues one M = 256 instruction that
+// both SMs' tensor cores execute, each accumulating its 128 rows in its own tensor memory.
+//  * full[s] lives in the leader: its producer arms it with the bytes of BOTH CTAs' loads, and the
+//    peer's TMA loads report their bytes to it as well.
+//  * empty[s] and acc_full[b] exist in both CTAs and are signalled together by a commit that arrives on
+//    the barrier at the same offset in each CTA.
+//  * acc_empty[b] lives in the leader and counts the epilogue warps of both CTAs (the peer's arrive
+//    remotely).
+// The CTAs of a pair meet at a cluster barrier after the barriers are initialised and before tensor memory
+// is freed, so neither can exit while the other's loads, MMAs or arrivals still refer to it.
+constexpr int PAIR_BM = 256, PAIR_BN = 256;
+
+template <int KIND>
+__global__ void __launch_bounds__(KK_THREADS, 1) gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a,
+                                                                     const __grid_constant__ CUtensorMap map_b,
+                                                                     const __grid_constant__ CUtensorMap map_c,
+                                                                     const TcParams p, const int tma_store) {
+    using Cfg = KindCfg<KIND>;
+    constexpr int BK = Cfg::BK;
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t full_bar[8], empty_bar[8], acc_full[2], acc_empty[2];
+    __shared__ __align__(16) float s_bias[KK_BIAS_MAX + 32];
+    __shared__ uint32_t tmem_holder;
+    __shared__ int abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();              // 0 = leader of the pair
+    const bool leader = rank == 0;
+    constexpr uint32_t a_bytes = TC_BM * 128, b_bytes = (PAIR_BN / 2) * 128;
+    constexpr uint32_t stage_bytes = a_bytes + b_bytes;   // per CTA
+    const int nk = (int)((p.K + BK - 1) / BK);
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t* smem_ring = smem;
+    uint8_t* smem_out = smem_ring + (size_t)p.stages * stage_bytes;
+
+    const int64_t tiles = p.m_tiles * p.n_tiles;          // 256 x 256 tiles
+    constexpr uint32_t acc_stride = PAIR_BN, tmem_cols = 2 * PAIR_BN;
+    const bool bias_in_smem = p.epi.bias != nullptr && p.N <= KK_BIAS_MAX;
+
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        for (int s = 0; s < p.stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 2 * KK_EPI_WARPS); }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (bias_in_smem)
+        for (int i = threadIdx.x; i < KK_BIAS_MAX + 32; i += KK_THREADS) s_bias[i] = i < p.N ? p.epi.bias[i] : 0.0f;
+    if (warp == KK_EPI_WARPS + 1) {
+        // the same warp of each CTA of the pair allocates, to the same shared-memory word
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_holder)), "r"(tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();                                   // both CTAs' barriers exist before anything signals them
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_holder;
+    const uint32_t n_clusters = num_clusters_x(), cluster = cluster_id_x();
+
+    if (warp == KK_EPI_WARPS) {
+        if (lane == 0) {
+            // ---------------- TMA producer (both CTAs) ----------------
+            bool ok = true;
+            uint32_t it = 0;
+            for (int64_t tile = cluster; tile < tiles && ok; tile += n_clusters) {
+                const int32_t m0 = (int32_t)((tile / p.n_tiles) * PAIR_BM + rank * TC_BM);
+                const int32_t n0 = (int32_t)((tile % p.n_tiles) * PAIR_BN + rank * (PAIR_BN / 2));
+                for (int ks = 0; ks < nk; ++ks, ++it) {
+                    const int s = it % p.stages;
+                    const uint32_t ph = ((it / p.stages) & 1) ^ 1;
+                    if (!mbar_wait(&empty_bar[s], ph, &abort_flag, p.wait_limit)) { abort_flag = 1; atomicMax(p.status, DEV_WAIT_EXPIRED); ok = false; break; }
+                    uint8_t* sa = smem_ring + (size_t)s * stage_bytes;
+                    const uint32_t lead_full = mapa_shared(smem_u32(&full_bar[s]), 0);
+                    if (leader) mbar_expect_tx(&full_bar[s], 2 * stage_bytes);
+                    tma_load_2d_pair(sa, &map_a, ks * BK, m0, lead_full);
+                    tma_load_2d_pair(sa + a_bytes, &map_b, ks * BK, n0, lead_full);
+                }
+            }
+        }
+    } else if (warp == KK_EPI_WARPS + 1) {
+        if (lane == 0 && leader) {
+            // ---------------- MMA issuer (leader only) ----------------
+            const uint32_t idesc = make_idesc<KIND>(PAIR_BM, PAIR_BN, false);
+            bool ok = true;
+            uint32_t it = 0, j = 0;
+            for (int64_t tile = cluster; tile < tiles && ok; tile += n_clusters, ++j) {
+                const uint32_t buf = j & 1;
+                if (!mbar_wait(&acc_empty[buf], ((j >> 1) & 1) ^ 1, &abort_flag, p.wait_limit)) { abort_flag = 1; atomicMax(p.status, DEV_WAIT_EXPIRED); ok = false; break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + buf * acc_stride;
+                for (int ks = 0; ks < nk; ++ks, ++it) {
+                    const int s = it % p.stages;
+                    const uint32_t ph = (it / p.stages) & 1;
+                    if (!mbar_wait(&full_bar[s], ph, &abort_flag, p.wait_limit)) { abort_flag = 1; atomicMax(p.status, DEV_WAIT_EXPIRED); ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t sa = smem_u32(smem_ring + (size_t)s * stage_bytes), sb = sa + a_bytes;
+#pragma unroll
+                    for (int kq = 0; kq < BK / Cfg::MMA_K; ++kq)
+                        tc_mma_pair<KIND>(d_tmem, make_desc(sa + kq * 32, 16, 1024, 2), make_desc(sb + kq * 32, 16, 1024, 2), idesc,
+                                          (ks | kq) != 0 ? 1u : 0u);
+                    tc_commit_pair(&empty_bar[s], 3);
+                }
+                if (ok) tc_commit_pair(&acc_full[buf], 3);
+            }
+        }
+    } else {
+        // ---------------- epilogue (both CTAs): this CTA's 128 rows of the tile ----------------
+        const int quarter = warp & 3, half = warp >> 2;
+        const bool post = (p.epi.drop != nullptr || p.epi.gate != nullptr) && tma_store;
+        const bool generic = !post && (p.epi.drop != nullptr || p.epi.gate != nullptr || (p.epi.bias != nullptr && !bias_in_smem));
+        const bool wide_bias = post && p.epi.bias != nullptr && !bias_in_smem;
+        const bool add_bias = p.epi.bias != nullptr && bias_in_smem, relu = p.epi.relu != 0;
+        const bool gate_vec = p.epi.gate != nullptr && aligned16_dev(p.epi.gate) && (p.epi.ld_gate & 3) == 0;
+        uint8_t* box = smem_out + (size_t)warp * 4096;
+        uint32_t j = 0;
+        bool ok = true;
+        for (int64_t tile = cluster; tile < tiles && ok; tile += n_clusters, ++j) {
+            const uint32_t buf = j & 1;
+            const int64_t m0 = (tile / p.n_tiles) * PAIR_BM + rank * TC_BM;
+            const int n0 = (int)((tile % p.n_tiles) * PAIR_BN);
+            if (lane == 0) ok = mbar_wait(&acc_full[buf], (j >> 1) & 1, &abort_flag, p.wait_limit);
+            ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
+            if (!ok) { if (lane == 0) { abort_flag = 1; atomicMax(p.status, DEV_WAIT_EXPIRED); } break; }
+            tc_fence_after();
+            const int64_t m = m0 + quarter * 32 + lane;
+            const bool row_ok = m < p.M;
+            for (int c0 = half * 32; c0 < PAIR_BN; c0 += 64) {
+                const int nb = n0 + c0;
+                if (nb >= p.N) break;                     // columns beyond N: nothing to store (warp-uniform)
+                float4 g4[8];
+                if (post && gate_vec) {
+#pragma unroll
+                    for (int it = 0; it < 8; ++it) {
+                        const int64_t mr = m0 + quarter * 32 + it * 4 + (lane >> 3);
+                        const int nc = nb + (lane & 7) * 4;
+                        g4[it] = (mr < p.M && nc < p.N) ? __ldg(reinterpret_cast<const float4*>(p.epi.gate + (p.epi.row0 + mr) * p.epi.ld_gate + nc))
+                                                         : make_float4(0.f, 0.f, 0.f, 0.f);
+                    }
+                }
+                uint32_t r[32];
+                tc_ld32(tmem_base + buf * acc_stride + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0, r);
+                tc_wait_ld();
+                float v[32];
+#pragma unroll
+                for (int q = 0; q < 32; ++q) v[q] = __uint_as_float(r[q]);
+                if (!generic) {
+                    if (add_bias) {
+                        const float4* sb4 = reinterpret_cast<const float4*>(s_bias + nb);
+#pragma unroll
+                        for (int q = 0; q < 8; ++q) {
+                            const float4 b4 = sb4[q];
+                            v[4 * q] += b4.x; v[4 * q + 1] += b4.y; v[4 * q + 2] += b4.z; v[4 * q + 3] += b4.w;
+                        }
+                    } else if (wide_bias) {
+#pragma unroll
+                        for (int q = 0; q < 32; ++q)
+                            if (nb + q < p.N) v[q] += p.epi.bias[nb + q];
+                    }
+                    if (relu) {
+#pragma unroll
+                        for (int q = 0; q < 32; ++q) v[q] = fmaxf(v[q], 0.0f);
+                    }
+                } else if (row_ok) {
+#pragma unroll
+                    for (int q = 0; q < 32; ++q)
+                        if (nb + q < p.N) v[q] = tc_apply_epi(p.epi, v[q], m, nb + q, p.N);
+                }
+                if (p.C_lp && row_ok && !post) {
+                    const int64_t left = p.N - nb;
+                    store_lp_row(p.C_lp + m * p.ldc_lp + nb, v, (int)(left < 32 ? left : 32));
+                }
+                if (tma_store) {
+                    if (lane == 0) bulk_wait_read<0>();
+                    __syncwarp();
+#pragma unroll
+                    for (int q = 0; q < 8; ++q)
+                        *reinterpret_cast<float4*>(box + lane * 128 + ((q ^ (lane & 7)) << 4)) =
+                            make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+                    if (post) {
+                        __syncwarp();
+#pragma unroll
+                        for (int it = 0; it < 8; ++it) {
+                            const int rr = it * 4 + (lane >> 3), ch = lane & 7;
+                            const int64_t mr = m0 + quarter * 32 + rr;
+                            const int nc = nb + ch * 4;
+                            if (mr >= p.M || nc >= p.N) continue;
+                            float4* cell = reinterpret_cast<float4*>(box + rr * 128 + ((ch ^ (rr & 7)) << 4));
+                            const float4 y4 = *cell;
+                            float y[4] = {y4.x, y4.y, y4.z, y4.w};
+                            const int nv = p.N - nc < 4 ? (int)(p.N - nc) : 4;
+                            if (p.epi.drop) {
+                                const uint8_t* dm = p.epi.drop + (p.epi.row0 + mr) * p.N + nc;
+#pragma unroll
+                                for (int t = 0; t < 4; ++t) if (t < nv) y[t] = dm[t] ? y[t] * p.epi.keep_scale : 0.0f;
+                            }
+                            if (p.epi.gate) {
+                                const float* gp = p.epi.gate + (p.epi.row0 + mr) * p.epi.ld_gate + nc;
+                                float gq[4] = {0.f, 0.f, 0.f, 0.f};
+                                if (gate_vec) {
+                                    gq[0] = g4[it].x; gq[1] = g4[it].y; gq[2] = g4[it].z; gq[3] = g4[it].w;
+                                } else {
+#pragma unroll
+                                    for (int t = 0; t < 4; ++t) if (t < nv) gq[t] = __ldg(gp + t);
+                                }
+#pragma unroll
+                                for (int t = 0; t < 4; ++t) y[t] = gq[t] > 0.0f ? y[t] * p.epi.gate_scale : 0.0f;
+                            }
+                            *cell = make_float4(y[0], y[1], y[2], y[3]);
+                            if (p.C_lp) {
+                                uint16_t* dl = p.C_lp + mr * p.ldc_lp + nc;
+                                if (nv == 4) *reinterpret_cast<uint2*>(dl) = make_uint2(pack_bf16(y[0], y[1]), pack_bf16(y[2], y[3]));
+                                else {
+#pragma unroll
+                                    for (int t = 0; t < 4; ++t) if (t < nv) dl[t] = (uint16_t)(pack_bf16(y[t], 0.0f) & 0xFFFFu);
+                                }
+                            }
+                        }
+                    }
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0) {
+                        tma_store_2d(&map_c, box, nb, (int32_t)(m0 + quarter * 32));
+                        bulk_commit();
+                    }
+                } else if (row_ok) {
+                    float* dst = p.C + m * p.ldc + nb;
+                    if (p.vec_c && nb + 31 < p.N) {
+#pragma unroll
+                        for (int q = 0; q < 32; q += 4)
+                            *reinterpret_cast<float4*>(dst + q) = make_float4(v[q], v[q + 1], v[q + 2], v[q + 3]);
+                    } else {
+#pragma unroll
+                        for (int q = 0; q < 32; ++q)
+                            if (nb + q < p.N) dst[q] = v[q];
+                    }
+                }
+            }
+            // this warp is done reading the buffer: tell the leader's MMA issuer
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(mapa_shared(smem_u32(&acc_empty[buf]), 0));
+        }
+        if (tma_store && lane == 0) bulk_wait_all();
+    }
+    if (threadIdx.x == 0 && abort_flag) {
+        for (int i = 0; i < 200; ++i) __nanosleep(1000);
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();                                   // the peer is done with this CTA's shared and tensor memory
+    if (warp == KK_EPI_WARPS + 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
+    }
+}
+
 // dst[n][k] = trans ? src[k][n] : src[n][k] for n < N, k < K, zero elsewhere; dst is rows x kpad of
 // fp32 (TF32 kind) or bf16 (round to nearest even).
 template <int KIND>
@@ -629,7 +890,13 @@ mixgcn_status launch_kind(mixgcn_ctx* ctx, int ta, int tb, int64_t M, int64_t N,
     if (!ta) {
         // KK form: pack B as rows x kpad (K contiguous), rows = n_tiles * bn32
         const int kpad = (int)((K + BK - 1) / BK * BK);
-        const int rows = (int)(p.n_tiles * p.bn > bn32 ? p.n_tiles * p.bn : bn32);
+        // Wide, deep products (the compute-bound ones) run on CTA pairs with 256 x 256 tiles.
+        const bool want_pairs = N >= 512 && K >= 512 && M >= 4096 && !ctx->debug_drop_load && !ctx->no_cta_pairs;
+        int rows = (int)(p.n_tiles * p.bn > bn32 ? p.n_tiles * p.bn : bn32);
+        if (want_pairs) {
+            const int rows_pairs = (int)((N + PAIR_BN - 1) / PAIR_BN * PAIR_BN);
+            if (rows_pairs > rows) rows = rows_pairs;
+        }
         MIXGCN_TRY(ensure_workspace(ctx, (int64_t)rows * kpad * EB));
         void* packed = ctx->workspace;
         if (!encode_2d(&map_a, A, EB, K, M, lda, BK, TC_BM)) return MIXGCN_EUNSUPPORTED;
@@ -642,6 +909,43 @@ mixgcn_status launch_kind(mixgcn_ctx* ctx, int ta, int tb, int64_t M, int64_t N,
         }
         p.splits = 1; p.k_per_split = K; p.raw = 0;
         p.debug_drop_load = ctx->debug_drop_load;
+        if (want_pairs) {
+            TcParams q = p;
+            q.bn = PAIR_BN;
+            q.m_tiles = (M + PAIR_BM - 1) / PAIR_BM;
+            q.n_tiles = (N + PAIR_BN - 1) / PAIR_BN;
+            const int rows2 = (int)(q.n_tiles * PAIR_BN);
+            const size_t stage2 = TC_BM * 128 + (PAIR_BN / 2) * 128;
+            q.stages = 5;
+            const size_t smem2 = (size_t)q.stages * stage2 + 8 * 4096 + 1024;
+            const int tma_store2 = q.vec_c ? 1 : 0;
+            CUtensorMap map_b2, map_c2 = map_a;
+            bool ok2 = rows2 <= rows && encode_2d(&map_b2, packed, EB, kpad, rows2, kpad, BK, PAIR_BN / 2);
+            if (ok2 && tma_store2) ok2 = encode_2d(&map_c2, C, 4, N, M, ldc, 32, 32);
+            if (ok2) {
+                MIXGCN_CUDA(cudaFuncSetAttribute(gemm_tc_pair_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2));
+                cudaLaunchConfig_t cfg = {};
+                cudaLaunchAttribute attr[1];
+                attr[0].id = cudaLaunchAttributeClusterDimension;
+                attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+                cfg.blockDim = dim3(KK_THREADS, 1, 1);
+                cfg.dynamicSmemBytes = smem2;
+                cfg.stream = s;
+                cfg.attrs = attr; cfg.numAttrs = 1;
+                cfg.gridDim = dim3((unsigned)(ctx->sm_count & ~1), 1, 1);
+                int max_clusters = 0;
+                if (cudaOccupancyMaxActiveClusters(&max_clusters, gemm_tc_pair_kernel<KIND>, &cfg) != cudaSuccess) { cudaGetLastError(); max_clusters = 0; }
+                const int64_t tiles2 = q.m_tiles * q.n_tiles;
+                int64_t clusters = max_clusters < tiles2 ? max_clusters : tiles2;
+                if (clusters >= 1) {
+                    cfg.gridDim = dim3((unsigned)(2 * clusters), 1, 1);
+                    LaunchScope scope(ctx, PH_GEMM, s);
+                    MIXGCN_CUDA(cudaLaunchKernelEx(&cfg, gemm_tc_pair_kernel<KIND>, map_a, map_b2, map_c2, q, tma_store2));
+                    ctx->gemm_pair_launches++;
+                    return MIXGCN_OK;
+                }
+            }
+        }
         // keep the packed weights resident in shared memory when they are small and there is one n-tile
         const int nk = kpad / BK;
         const size_t b_all = (size_t)nk * bn32 * 128;

@@ -60,6 +60,8 @@ struct mixgcn_ctx {
     void* workspace_lp;       // bf16 copies of fp32 operands converted on the fly (BF16 products whose caller gave no copy)
     int64_t workspace_lp_bytes;
     int64_t gemm_path[3];     // dense products served by: 0 fp32 FMA kernel, 1 tcgen05 TF32, 2 tcgen05 BF16
+    int64_t gemm_pair_launches;   // of those, products that ran on CTA pairs (tcgen05 .cta_group::2)
+    int no_cta_pairs;         // 1: keep every product on single CTAs (option, for comparison)
     int debug_wait_limit;     // > 0: polls after which the tensor-core kernels' waits give up (test of that path)
     int debug_drop_load;      // 1: the next K-major tensor-core product leaves one stage unfilled (test of that path)
     int spmm_slice_cols;      // 0 = default (one slice up to 1024 columns)

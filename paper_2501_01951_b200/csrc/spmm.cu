@@ -124,14 +124,18 @@ struct Cfg {
 };
 
 // Accumulate entries [b, e) into acc[] for the lane's column groups, ascending entry order.
+// The (col, val) pair of the NEXT batch of LPR entries is requested before the current batch's gathers,
+// so that the index load's latency is hidden behind them instead of preceding every batch.
 template <int LPR, int VPL>
 __device__ __forceinline__ void row_segment(const SpmmParams& p, int64_t b, int64_t e, int lig, unsigned mask,
                                             int w4, float4 (&acc)[VPL]) {
     constexpr int U = Cfg<LPR, VPL>::U;
     const float* Yb = p.Y + p.j0;
+    int c = 0; float a = 0.0f;
+    if (b + lig < e) { c = __ldg(p.col + b + lig); a = __ldg(p.val + b + lig); }
     for (int64_t i0 = b; i0 < e; i0 += LPR) {
-        int c = 0; float a = 0.0f;
-        if (i0 + lig < e) { c = __ldg(p.col + i0 + lig); a = __ldg(p.val + i0 + lig); }
+        int c_next = 0; float a_next = 0.0f;
+        if (i0 + LPR + lig < e) { c_next = __ldg(p.col + i0 + LPR + lig); a_next = __ldg(p.val + i0 + LPR + lig); }
         const int cnt = (int)((e - i0) < LPR ? (e - i0) : LPR);
         for (int k = 0; k < cnt; k += U) {
             int ck[U]; float ak[U]; float4 y[U][VPL];
@@ -157,6 +161,7 @@ __device__ __forceinline__ void row_segment(const SpmmParams& p, int64_t b, int6
                     for (int v = 0; v < VPL; ++v) fma4(acc[v], ak[t], y[t][v]);
                 }
         }
+        c = c_next; a = a_next;
     }
 }
 

@@ -715,6 +715,59 @@ def test_training_epoch_bf16_within_low_precision_bound(mg, ctx, orders, lp_copi
     gg.close()
 
 
+PAIR_SHAPES = [(4096, 512, 512), (5000, 1024, 520), (4100, 600, 1000), (8191, 777, 513)]   # M, N, K: ragged in every dimension
+
+
+@pytest.mark.parametrize("M,N,K", PAIR_SHAPES)
+@pytest.mark.parametrize("prec", ["tf32", "bf16"])
+@pytest.mark.parametrize("tb", [False, True])
+def test_gemm_on_cta_pairs(mg, ctx, M, N, K, prec, tb):
+    """Wide, deep K-major products run on pairs of CTAs (one 256 x 256 tile per pair): same checks as the
+    single-CTA kernels, and the single-CTA kernel must agree with the pair kernel to fp32 accuracy."""
+    from helpers import TOL_LOWP
+    P = mg.PRECISIONS[prec]
+    rnd = _tf32_trunc if prec == "tf32" else _bf16_round
+    A = synth.uniform_tensor((M, K), 331 + M, -1, 1)
+    B = synth.uniform_tensor((N, K) if tb else (K, N), 332 + N, -1, 1)
+    bias = synth.uniform_tensor((N,), 333, -1, 1)
+    Cd = torch.full((M, round4(N) + 4), 3.0, device="cuda")
+    epi = mg.make_epilogue(bias=bias.cuda(), relu=True)
+    before = mg.ctx_gemm_paths(ctx)["cta_pairs"]
+    mg.gemm(ctx, P, False, tb, M, N, K, padded(A, fill=float("nan")), B.cuda().contiguous(), Cd, epi=epi)
+    assert mg.ctx_gemm_paths(ctx)["cta_pairs"] == before + 1
+    Bo = B.numpy().T if tb else B.numpy()
+    assert rel_fro(host(Cd, N), orc.activation(orc.update(A.numpy(), Bo, bias.numpy()), True)) <= TOL_LOWP
+    assert rel_fro(host(Cd, N), orc.activation(orc.update(rnd(A.numpy()), rnd(Bo), bias.numpy()), True)) <= 2e-5
+    assert torch.all(Cd[:, round4(N):] == 3.0)
+    mg.ctx_set_option(ctx, mg.OPT_GEMM_CTA_PAIRS, 0)
+    try:
+        C1 = torch.full_like(Cd, 3.0)
+        mg.gemm(ctx, P, False, tb, M, N, K, padded(A, fill=float("nan")), B.cuda().contiguous(), C1, epi=epi)
+        assert mg.ctx_gemm_paths(ctx)["cta_pairs"] == before + 1
+    finally:
+        mg.ctx_set_option(ctx, mg.OPT_GEMM_CTA_PAIRS, 1)
+    assert rel_fro(host(Cd, N), host(C1, N)) <= 2e-6
+    assert mg.ctx_poll_status(ctx, raise_on_error=False) == 0
+
+
+def test_gemm_on_cta_pairs_with_gate_and_dropout(mg, ctx):
+    """The per-element epilogue terms (gate by another tensor's sign, dropout mask) on the pair kernel."""
+    M, N, K = 4200, 520, 512
+    A = synth.uniform_tensor((M, K), 341, -1, 1); B = synth.uniform_tensor((K, N), 342, -1, 1)
+    gate = synth.uniform_tensor((M, N), 343, -1, 1)
+    drop = (synth.uniform_tensor((M, N), 344, 0, 1) < 0.7).to(torch.uint8)
+    Cd = torch.zeros(M, round4(N), device="cuda")
+    epi = mg.make_epilogue(drop_mask=drop.cuda(), keep_scale=1.25, gate=padded(gate), gate_scale=0.5)
+    before = mg.ctx_gemm_paths(ctx)["cta_pairs"]
+    mg.gemm(ctx, mg.PREC_BF16, False, False, M, N, K, padded(A), B.cuda(), Cd, epi=epi)
+    assert mg.ctx_gemm_paths(ctx)["cta_pairs"] == before + 1
+    want = _bf16_round(A.numpy()) @ _bf16_round(B.numpy())
+    want = np.where(drop.numpy() != 0, want * 1.25, 0.0)
+    want = np.where(gate.numpy() > 0, want * 0.5, 0.0)
+    assert rel_fro(host(Cd, N), want) <= 2e-5
+    assert mg.ctx_poll_status(ctx, raise_on_error=False) == 0
+
+
 @pytest.mark.parametrize("prec", ["tf32", "bf16"])
 def test_bounded_wait_runs_out_and_the_context_stays_usable(mg, ctx, prec):
     """Failure detection without a fault: a test hook makes the TMA producer of the tensor-core kernel
