@@ -778,6 +778,148 @@ __global__ void __launch_bounds__(KK_THREADS, 1) gemm_tc_pair_kernel(const __gri
     }
 }
 
+// The weight-gradient form (both operands MN-major, K = node count split over the grid's z dimension) on
+// CTA pairs: a pair owns a 256 x 256 tile of one K split; each CTA loads its 128 columns of A and of B per
+// stage and writes its 128 rows of the (partial) tile.  Barriers as in gemm_tc_pair_kernel.
+template <int KIND>
+__global__ void __launch_bounds__(TC_THREADS, 1) gemm_tc_mm_pair_kernel(const __grid_constant__ CUtensorMap map_a,
+                                                                        const __grid_constant__ CUtensorMap map_b,
+                                                                        const TcParams p) {
+    using Cfg = KindCfg<KIND>;
+    constexpr int BK = Cfg::BK;
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t full_bar[8], empty_bar[8], acc_bar;
+    __shared__ uint32_t tmem_holder;
+    __shared__ int abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();
+    const bool leader = rank == 0;
+    constexpr uint32_t a_bytes = TC_BM * 128, b_bytes = (PAIR_BN / 2) * 128;
+    constexpr uint32_t stage_bytes = a_bytes + b_bytes;
+    constexpr int CHUNKS = TC_BM / Cfg::CHUNK;            // 128-byte-wide chunks per 128 columns of A or B
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+
+    const int64_t tile = cluster_id_x();
+    const int64_t m0 = (tile / p.n_tiles) * PAIR_BM + rank * TC_BM;
+    const int64_t n0 = (tile % p.n_tiles) * PAIR_BN;
+    const int64_t kb = (int64_t)blockIdx.z * p.k_per_split;
+    const int64_t ke = kb + p.k_per_split < p.K ? kb + p.k_per_split : p.K;
+    const int nk = (int)((ke - kb + BK - 1) / BK);
+    constexpr uint32_t tmem_cols = PAIR_BN;
+
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        for (int s = 0; s < p.stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        mbar_init(&acc_bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 5) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_holder)), "r"(tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_holder;
+
+    if (warp == 4) {
+        if (lane == 0) {
+            // ---------------- TMA producer (both CTAs) ----------------
+            for (int ks = 0; ks < nk; ++ks) {
+                const int s = ks % p.stages;
+                const uint32_t ph = ((ks / p.stages) & 1) ^ 1;
+                if (!mbar_wait(&empty_bar[s], ph, &abort_flag, p.wait_limit)) { abort_flag = 1; atomicMax(p.status, DEV_WAIT_EXPIRED); break; }
+                uint8_t* sa = smem + (size_t)s * stage_bytes;
+                uint8_t* sb = sa + a_bytes;
+                const uint32_t lead_full = mapa_shared(smem_u32(&full_bar[s]), 0);
+                if (leader) mbar_expect_tx(&full_bar[s], 2 * stage_bytes);
+                const int32_t k0 = (int32_t)(kb + (int64_t)ks * BK);
+                for (int c = 0; c < CHUNKS; ++c)
+                    tma_load_2d_pair(sa + c * Cfg::MN_CHUNK_BYTES, &map_a, (int32_t)(m0 + Cfg::CHUNK * c), k0, lead_full);
+                for (int c = 0; c < CHUNKS; ++c)
+                    tma_load_2d_pair(sb + c * Cfg::MN_CHUNK_BYTES, &map_b, (int32_t)(n0 + rank * (PAIR_BN / 2) + Cfg::CHUNK * c), k0, lead_full);
+            }
+        }
+    } else if (warp == 5) {
+        if (lane == 0 && leader) {
+            // ---------------- MMA issuer (leader only) ----------------
+            const uint32_t idesc = make_idesc<KIND>(PAIR_BM, PAIR_BN, true);
+            bool ok = true;
+            for (int ks = 0; ks < nk && ok; ++ks) {
+                const int s = ks % p.stages;
+                const uint32_t ph = (ks / p.stages) & 1;
+                if (!mbar_wait(&full_bar[s], ph, &abort_flag, p.wait_limit)) { abort_flag = 1; atomicMax(p.status, DEV_WAIT_EXPIRED); ok = false; break; }
+                tc_fence_after();
+                const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes), sb = sa + a_bytes;
+#pragma unroll
+                for (int kq = 0; kq < BK / Cfg::MMA_K; ++kq)
+                    tc_mma_pair<KIND>(tmem_base, make_desc(sa + kq * Cfg::MN_STEP, Cfg::MN_CHUNK_BYTES, Cfg::MN_SBO, Cfg::MN_LAYOUT),
+                                      make_desc(sb + kq * Cfg::MN_STEP, Cfg::MN_CHUNK_BYTES, Cfg::MN_SBO, Cfg::MN_LAYOUT), idesc,
+                                      (ks | kq) != 0 ? 1u : 0u);
+                tc_commit_pair(&empty_bar[s], 3);
+            }
+            if (ok) tc_commit_pair(&acc_bar, 3);
+        }
+    } else {
+        // ---------------- epilogue: this CTA's 128 rows ----------------
+        bool ok = true;
+        if (nk > 0) {
+            if (lane == 0) ok = mbar_wait(&acc_bar, 0, &abort_flag, p.wait_limit);
+            ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
+            if (!ok && lane == 0) { abort_flag = 1; atomicMax(p.status, DEV_WAIT_EXPIRED); }
+        }
+        __syncwarp();
+        tc_fence_after();
+        if (ok) {
+            const int64_t m = m0 + warp * 32 + lane;
+            float* Cb = p.C + (p.raw ? (int64_t)blockIdx.z * p.M * p.N : 0);
+            for (int c0 = 0; c0 < PAIR_BN; c0 += 32) {
+                const int64_t nb = n0 + c0;
+                if (nb >= p.N) break;
+                uint32_t r[32];
+                if (nk > 0) {
+                    tc_ld32(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, r);
+                    tc_wait_ld();
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) r[j] = 0u;
+                }
+                if (m < p.M) {
+                    float* dst = Cb + m * p.ldc + nb;
+                    float v[32];
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        v[j] = __uint_as_float(r[j]);
+                        if (!p.raw && nb + j < p.N) v[j] = tc_apply_epi(p.epi, v[j], m, nb + j, p.N);
+                    }
+                    if (p.vec_c && nb + 31 < p.N) {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4)
+                            *reinterpret_cast<float4*>(dst + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (nb + j < p.N) dst[j] = v[j];
+                    }
+                }
+            }
+        }
+    }
+    if (threadIdx.x == 0 && abort_flag) {
+        for (int i = 0; i < 200; ++i) __nanosleep(1000);
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();
+    if (warp == 5) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
+    }
+}
+
 // dst[n][k] = trans ? src[k][n] : src[n][k] for n < N, k < K, zero elsewhere; dst is rows x kpad of
 // fp32 (TF32 kind) or bf16 (round to nearest even).
 template <int KIND>
@@ -851,6 +993,24 @@ int pick_bn(int64_t N) {
         bn = ((N + tiles - 1) / tiles + 31) / 32 * 32;
     }
     return (int)bn;
+}
+
+// Number of K splits for `tiles` output tiles on a machine that runs `slots` CTAs (or CTA pairs) at a
+// time: the split count, up to max_splits, whose tiles * splits units fill whole waves of `slots` best
+// (a last wave that is one sixth full costs a third of the time of a two-wave launch).
+int pick_splits(int64_t tiles, int64_t slots, int64_t max_splits) {
+    int64_t hi = 4 * slots / tiles + 1;
+    if (hi > max_splits) hi = max_splits;
+    if (hi < 1) hi = 1;
+    int best = (int)hi;
+    double best_eff = 0.0;
+    for (int64_t sp = 1; sp <= hi; ++sp) {
+        const int64_t units = tiles * sp, waves = (units + slots - 1) / slots;
+        if (units < slots && sp < hi) continue;                 // does not fill the machine once
+        const double eff = (double)units / (double)(waves * slots);
+        if (eff > best_eff + 1e-9) { best_eff = eff; best = (int)sp; }
+    }
+    return best;
 }
 
 template <int KIND>
@@ -968,15 +1128,53 @@ mixgcn_status launch_kind(mixgcn_ctx* ctx, int ta, int tb, int64_t M, int64_t N,
         return MIXGCN_OK;
     }
 
-    // MM form (weight gradient): split K over CTAs
-    int splits = 1;
-    {
-        const int64_t want = (4 * (int64_t)ctx->sm_count + tiles - 1) / tiles;
-        const int64_t maxs = (K + 2047) / 2048;
-        splits = (int)(want < maxs ? want : maxs);
-        if (splits < 1) splits = 1;
-        if (splits > 2048) splits = 2048;
+    // MM form (weight gradient): wide results (both widths >= 512) on CTA pairs with 256 x 256 tiles
+    if (M >= 512 && N >= 512 && K >= 4096 && !ctx->no_cta_pairs) {
+        TcParams q = p;
+        q.bn = PAIR_BN;
+        q.m_tiles = (M + PAIR_BM - 1) / PAIR_BM;
+        q.n_tiles = (N + PAIR_BN - 1) / PAIR_BN;
+        const int64_t tiles2 = q.m_tiles * q.n_tiles;
+        const int pairs = ctx->sm_count / 2;
+        int64_t sp = pick_splits(tiles2, pairs, (K + 4095) / 4096);
+        int64_t kps2 = (K + sp - 1) / sp;
+        kps2 = (kps2 + BK - 1) / BK * BK;
+        sp = (K + kps2 - 1) / kps2;
+        q.k_per_split = kps2; q.splits = (int)sp;
+        q.stages = 6;
+        const CUtensorMapSwizzle sw2 = KIND == KIND_TF32 ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B : CU_TENSOR_MAP_SWIZZLE_128B;
+        bool ok2 = tiles2 <= 0x3FFFFFFF && encode_2d(&map_a, A, EB, M, K, lda, Cfg::CHUNK, BK, sw2) &&
+                   encode_2d(&map_b, B, EB, N, K, ldb, Cfg::CHUNK, BK, sw2);
+        if (ok2) {
+            if (sp > 1) {
+                MIXGCN_TRY(ensure_workspace(ctx, sp * M * N * (int64_t)sizeof(float)));
+                q.C = reinterpret_cast<float*>(ctx->workspace); q.ldc = N; q.vec_c = (N & 3) == 0; q.raw = 1;
+            } else {
+                q.raw = 0;
+            }
+            const size_t smem2 = (size_t)q.stages * (TC_BM * 128 + (PAIR_BN / 2) * 128) + 1024;
+            MIXGCN_CUDA(cudaFuncSetAttribute(gemm_tc_mm_pair_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2));
+            cudaLaunchConfig_t cfg = {};
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeClusterDimension;
+            attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+            cfg.gridDim = dim3((unsigned)(2 * tiles2), 1, (unsigned)sp);
+            cfg.blockDim = dim3(TC_THREADS, 1, 1);
+            cfg.dynamicSmemBytes = smem2;
+            cfg.stream = s;
+            cfg.attrs = attr; cfg.numAttrs = 1;
+            {
+                LaunchScope scope(ctx, PH_GEMM, s);
+                MIXGCN_CUDA(cudaLaunchKernelEx(&cfg, gemm_tc_mm_pair_kernel<KIND>, map_a, map_b, q));
+            }
+            ctx->gemm_pair_launches++;
+            if (sp > 1) MIXGCN_TRY(launch_splitk_reduce(ctx, M, N, (int)sp, q.C, C, ldc, epi, s));
+            return MIXGCN_OK;
+        }
     }
+    // split K over CTAs
+    int splits = pick_splits(tiles, 2 * (int64_t)ctx->sm_count, (K + 2047) / 2048);      // two CTAs per SM
+    if (splits > 2048) splits = 2048;
     int64_t kps = (K + splits - 1) / splits;
     kps = (kps + BK - 1) / BK * BK;
     splits = (int)((K + kps - 1) / kps);

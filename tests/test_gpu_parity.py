@@ -750,6 +750,25 @@ def test_gemm_on_cta_pairs(mg, ctx, M, N, K, prec, tb):
     assert mg.ctx_poll_status(ctx, raise_on_error=False) == 0
 
 
+@pytest.mark.parametrize("M,N,K", [(512, 512, 4096), (1024, 1024, 20000), (600, 777, 9001), (520, 1000, 33333)])
+@pytest.mark.parametrize("prec", ["tf32", "bf16"])
+def test_weight_gradient_on_cta_pairs(mg, ctx, M, N, K, prec):
+    from helpers import TOL_LOWP
+    P = mg.PRECISIONS[prec]
+    rnd = _tf32_trunc if prec == "tf32" else _bf16_round
+    A, B = synth.normal_features(K, M, 351), synth.normal_features(K, N, 352)
+    Cd = torch.full((M, round4(N)), 3.0, device="cuda")
+    before = mg.ctx_gemm_paths(ctx)["cta_pairs"]
+    mg.gemm(ctx, P, True, False, M, N, K, padded(A, fill=float("nan")), padded(B, fill=float("nan")), Cd)
+    assert mg.ctx_gemm_paths(ctx)["cta_pairs"] == before + 1
+    assert rel_fro(host(Cd, N), A.numpy().astype(np.float64).T @ B.numpy().astype(np.float64)) <= TOL_LOWP
+    assert rel_fro(host(Cd, N), rnd(A.numpy()).T @ rnd(B.numpy())) <= 2e-5
+    C2 = torch.zeros_like(Cd)
+    mg.gemm(ctx, P, True, False, M, N, K, padded(A, fill=float("nan")), padded(B, fill=float("nan")), C2)
+    assert torch.equal(Cd[:, :N], C2[:, :N])                               # fixed-order reduction: reproducible bits
+    assert mg.ctx_poll_status(ctx, raise_on_error=False) == 0
+
+
 def test_gemm_on_cta_pairs_with_gate_and_dropout(mg, ctx):
     """The per-element epilogue terms (gate by another tensor's sign, dropout mask) on the pair kernel."""
     M, N, K = 4200, 520, 512
