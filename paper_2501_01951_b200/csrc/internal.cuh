@@ -146,24 +146,10 @@ struct mixgcn_rowplan {
 
 namespace mixgcn {
 
-#ifndef MIXGCN_SPMM_SEG
-#define MIXGCN_SPMM_SEG 512
-#endif
-#ifndef MIXGCN_SPMM_BLK_MIN
-#define MIXGCN_SPMM_BLK_MIN 64
-#endif
-#ifndef MIXGCN_SPMM_LOG_BLOCKS
-#define MIXGCN_SPMM_LOG_BLOCKS 8
-#endif
-constexpr int SPMM_SEG = MIXGCN_SPMM_SEG;                 // rows longer than this are cut into segments of at most this many entries
-constexpr int SPMM_BLK_MIN_ENTRIES = MIXGCN_SPMM_BLK_MIN; // a long row uses 2^k column blocks while it keeps >= this many entries per block
-constexpr int SPMM_MAX_LOG_BLOCKS = MIXGCN_SPMM_LOG_BLOCKS; // at most 2^this column blocks per row
-#ifndef MIXGCN_SPMM_PACK0
-#define MIXGCN_SPMM_PACK0 12
-#define MIXGCN_SPMM_PACK1 5
-#define MIXGCN_SPMM_PACK2 2
-#endif
-constexpr int SPMM_PACK_DEG[3] = {MIXGCN_SPMM_PACK0, MIXGCN_SPMM_PACK1, MIXGCN_SPMM_PACK2};   // rows up to these lengths share a warp 2-, 4-, 8-fold
+constexpr int SPMM_SEG = 512;               // rows longer than this are cut into segments of at most this many entries
+constexpr int SPMM_BLK_MIN_ENTRIES = 64;    // a long row uses 2^k column blocks while it keeps >= this many entries per block
+constexpr int SPMM_MAX_LOG_BLOCKS = 8;      // at most 2^this column blocks per row
+constexpr int SPMM_PACK_DEG[3] = {12, 5, 2};   // rows up to these lengths share a warp 2-, 4-, 8-fold
 
 // Launch bookkeeping: counts the launch and, when profiling, brackets it with events.
 struct LaunchScope {

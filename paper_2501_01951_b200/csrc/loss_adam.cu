@@ -281,9 +281,7 @@ __global__ void __launch_bounds__(LOSS_WARPS * 32) loss_rows_subset_kernel(
 // arg-max keeps the lowest index among equal maxima explicitly, so the order does not matter.  The few
 // train rows are then finished by whole warps (exponentials and gradient stores over 32 lanes).
 constexpr uint32_t LOSS_WAIT_LIMIT = 1u << 22;
-#ifndef MIXGCN_LOSS_TILE_KB
-#define MIXGCN_LOSS_TILE_KB 72
-#endif
+constexpr int LOSS_TILE_KB = 72;     // shared memory a CTA of the tile kernel takes at most (two tile buffers)
 constexpr int LOSS_LANES_PER_ROW = 4;
 
 __device__ __forceinline__ uint32_t loss_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -463,8 +461,8 @@ int launch_loss_rows(unsigned warp_blocks, cudaStream_t s, int64_t n, int C, con
                      int sm_count = 0) {
     const bool vec = (ld & 3) == 0 && aligned16(logits) && (!dlogits || aligned16(dlogits));
     // Several CTAs per SM (each with two tile buffers) keep some computing while others wait for their
-    // copies: a CTA takes at most MIXGCN_LOSS_TILE_KB of shared memory; rows per tile follow from that.
-    constexpr int64_t TILE_SMEM = MIXGCN_LOSS_TILE_KB * 1024;
+    // copies: a CTA takes at most LOSS_TILE_KB of shared memory; rows per tile follow from that.
+    constexpr int64_t TILE_SMEM = LOSS_TILE_KB * 1024;
     // The tile kernel treats a tile as one dense piece of rows x ld floats (it copies and zeroes whole
     // rows), so it is taken only when the row holds nothing but its C columns and their pad to a multiple
     // of 4; a wider ld (a column slice of a larger buffer) goes to the per-row kernels, which touch columns

@@ -22,30 +22,15 @@
 
 using namespace mixgcn;
 
-#ifndef MIXGCN_SPMM_MINB
-#define MIXGCN_SPMM_MINB 4      // CTAs per SM asked of the compiler for the narrow (VPL <= 2) group kernels
-#endif
-#ifndef MIXGCN_SPMM_FOLD_WMAX
-#define MIXGCN_SPMM_FOLD_WMAX 128   // widest aggregation the two folds below apply to
-#endif
-#ifndef MIXGCN_SPMM_FOLD_SEG
-#define MIXGCN_SPMM_FOLD_SEG 2      // lanes-per-unit fold for long-row segments at widths <= 128 (1: 32 lanes, 2: 16 lanes x 2 float4, ...)
-#endif
-#ifndef MIXGCN_SPMM_FOLD_MED
-#define MIXGCN_SPMM_FOLD_MED 2      // the same for rows of 13..512 entries
-#endif
-#ifndef MIXGCN_SPMM_SHORT_RB
-#define MIXGCN_SPMM_SHORT_RB 4       // rows a warp of the short-row kernel takes at once
-#endif
-#ifndef MIXGCN_SPMM_SHORT_MINB
-#define MIXGCN_SPMM_SHORT_MINB 5     // CTAs per SM asked of the compiler for it
-#endif
-#ifndef MIXGCN_SPMM_SHORT_MAXE
-#define MIXGCN_SPMM_SHORT_MAXE 2     // 0 = rows of 1..2 entries go through the packed group kernel
-#endif
-#ifndef MIXGCN_SPMM_U
-#define MIXGCN_SPMM_U 8
-#endif
+// Launch shapes the measurements settled on (workload with 30M nodes, width 128, and the wide / dense ones).
+constexpr int SPMM_MINB = 4;          // CTAs per SM asked of the compiler for the narrow (VPL <= 2) group kernels
+constexpr int SPMM_FOLD_WMAX = 128;   // widest aggregation the two folds below apply to
+constexpr int SPMM_FOLD_SEG = 2;      // long-row segments at widths <= 128: 16 lanes x 2 float4 per unit (1 would be 32 lanes x 1)
+constexpr int SPMM_FOLD_MED = 2;      // the same for rows of 13..512 entries
+constexpr int SPMM_SHORT_RB = 4;      // rows a warp of the short-row kernel takes at once
+constexpr int SPMM_SHORT_MINB = 5;    // CTAs per SM asked of the compiler for it
+constexpr int SPMM_SHORT_MAXE = 2;    // rows of at most this many entries go to the short-row kernel
+constexpr int SPMM_U = 8;             // float4 loads a lane keeps in flight
 
 namespace {
 
@@ -119,7 +104,7 @@ __device__ __forceinline__ void fma4(float4& acc, float a, const float4& y) {
 
 template <int LPR, int VPL>
 struct Cfg {
-    static constexpr int U0 = MIXGCN_SPMM_U / VPL < 1 ? 1 : MIXGCN_SPMM_U / VPL;
+    static constexpr int U0 = SPMM_U / VPL < 1 ? 1 : SPMM_U / VPL;
     static constexpr int U = U0 > LPR ? LPR : U0;   // gathered rows in flight per lane group
 };
 
@@ -166,7 +151,7 @@ __device__ __forceinline__ void row_segment(const SpmmParams& p, int64_t b, int6
 }
 
 template <int LPR, int VPL>
-__global__ void __launch_bounds__(256, VPL <= 2 ? MIXGCN_SPMM_MINB : 1) spmm_group_kernel(const SpmmParams p) {
+__global__ void __launch_bounds__(256, VPL <= 2 ? SPMM_MINB : 1) spmm_group_kernel(const SpmmParams p) {
     const int lig = threadIdx.x % LPR;
     const int64_t idx = p.idx_begin + ((int64_t)blockIdx.x * 256 + threadIdx.x) / LPR;
     if (idx >= p.idx_end) return;  // the whole group leaves together
@@ -208,7 +193,7 @@ __global__ void __launch_bounds__(256, VPL <= 2 ? MIXGCN_SPMM_MINB : 1) spmm_gro
 // 512-byte request of the whole warp (lane = float4 column), RB of them in flight; entries of a row are
 // added in entry order, as everywhere else.
 template <int RB, int MAXE>
-__global__ void __launch_bounds__(256, MIXGCN_SPMM_SHORT_MINB) spmm_short_kernel(const SpmmParams p) {
+__global__ void __launch_bounds__(256, SPMM_SHORT_MINB) spmm_short_kernel(const SpmmParams p) {
     static_assert(RB * MAXE <= 32, "one lane per (row, entry)");
     const int lane = threadIdx.x & 31;
     const int64_t idx0 = p.idx_begin + (((int64_t)blockIdx.x * 256 + threadIdx.x) >> 5) * RB;
@@ -584,7 +569,7 @@ mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView&
             {
                 LaunchScope scope(ctx, phase, s);
                 p.idx_begin = 0; p.idx_end = S.total_segs;
-                dispatch(p, p.w <= MIXGCN_SPMM_FOLD_WMAX ? MIXGCN_SPMM_FOLD_SEG : 1, s);
+                dispatch(p, p.w <= SPMM_FOLD_WMAX ? SPMM_FOLD_SEG : 1, s);
             }
             {
                 LaunchScope scope(ctx, phase, s);
@@ -611,14 +596,14 @@ mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView&
             p.idx_begin = S.total_segs + (begin - S.n_long);
             p.idx_end = S.total_segs + (end - S.n_long);
             LaunchScope scope(ctx, phase, s);
-            if (q == 3 && p.w <= 128 && SPMM_PACK_DEG[2] <= MIXGCN_SPMM_SHORT_MAXE && MIXGCN_SPMM_SHORT_MAXE > 0) {
+            if (q == 3 && p.w <= 128 && SPMM_PACK_DEG[2] <= SPMM_SHORT_MAXE) {
                 // rows of at most SPMM_PACK_DEG[2] entries: several rows per warp, whole-warp gathers
-                constexpr int RB = MIXGCN_SPMM_SHORT_RB, MAXE = MIXGCN_SPMM_SHORT_MAXE > 0 ? MIXGCN_SPMM_SHORT_MAXE : 1;
+                constexpr int RB = SPMM_SHORT_RB, MAXE = SPMM_SHORT_MAXE;
                 const int64_t units = p.idx_end - p.idx_begin;
                 const int64_t warps = (units + RB - 1) / RB;
                 spmm_short_kernel<RB, MAXE><<<(unsigned)((warps + 7) / 8), 256, 0, s>>>(p);
             } else {
-                dispatch(p, q == 0 ? (p.w <= MIXGCN_SPMM_FOLD_WMAX ? MIXGCN_SPMM_FOLD_MED : 1) : fold, s);
+                dispatch(p, q == 0 ? (p.w <= SPMM_FOLD_WMAX ? SPMM_FOLD_MED : 1) : fold, s);
             }
             begin = end;
         }
