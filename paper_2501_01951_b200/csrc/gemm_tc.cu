@@ -542,7 +542,6 @@ __global__ void __launch_bounds__(KK_THREADS, 1) gemm_tc_pair_kernel(const __gri
     constexpr int BK = Cfg::BK;
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t full_bar[8], empty_bar[8], acc_full[2], acc_empty[2];
-    __shared__ __align__(16) float s_bias[KK_BIAS_MAX + 32];
     __shared__ uint32_t tmem_holder;
     __shared__ int abort_flag;
 
@@ -558,7 +557,9 @@ __global__ void __launch_bounds__(KK_THREADS, 1) gemm_tc_pair_kernel(const __gri
 
     const int64_t tiles = p.m_tiles * p.n_tiles;          // 256 x 256 tiles
     constexpr uint32_t acc_stride = PAIR_BN, tmem_cols = 2 * PAIR_BN;
-    const bool bias_in_smem = p.epi.bias != nullptr && p.N <= KK_BIAS_MAX;
+    // the bias is read from global memory (every lane the same 128 bytes: a broadcast the L1 serves), which
+    // leaves the shared memory a copy of it would take to a sixth stage of the ring
+    const bool bias_vec = p.epi.bias != nullptr && aligned16_dev(p.epi.bias);
 
     if (threadIdx.x == 0) {
         abort_flag = 0;
@@ -567,8 +568,6 @@ __global__ void __launch_bounds__(KK_THREADS, 1) gemm_tc_pair_kernel(const __gri
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    if (bias_in_smem)
-        for (int i = threadIdx.x; i < KK_BIAS_MAX + 32; i += KK_THREADS) s_bias[i] = i < p.N ? p.epi.bias[i] : 0.0f;
     if (warp == KK_EPI_WARPS + 1) {
         // the same warp of each CTA of the pair allocates, to the same shared-memory word
         asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_holder)), "r"(tmem_cols) : "memory");
@@ -631,9 +630,8 @@ __global__ void __launch_bounds__(KK_THREADS, 1) gemm_tc_pair_kernel(const __gri
         // ---------------- epilogue (both CTAs): this CTA's 128 rows of the tile ----------------
         const int quarter = warp & 3, half = warp >> 2;
         const bool post = (p.epi.drop != nullptr || p.epi.gate != nullptr) && tma_store;
-        const bool generic = !post && (p.epi.drop != nullptr || p.epi.gate != nullptr || (p.epi.bias != nullptr && !bias_in_smem));
-        const bool wide_bias = post && p.epi.bias != nullptr && !bias_in_smem;
-        const bool add_bias = p.epi.bias != nullptr && bias_in_smem, relu = p.epi.relu != 0;
+        const bool generic = !post && (p.epi.drop != nullptr || p.epi.gate != nullptr);
+        const bool add_bias = p.epi.bias != nullptr, relu = p.epi.relu != 0;
         const bool gate_vec = p.epi.gate != nullptr && aligned16_dev(p.epi.gate) && (p.epi.ld_gate & 3) == 0;
         uint8_t* box = smem_out + (size_t)warp * 4096;
         uint32_t j = 0;
@@ -669,16 +667,18 @@ __global__ void __launch_bounds__(KK_THREADS, 1) gemm_tc_pair_kernel(const __gri
                 for (int q = 0; q < 32; ++q) v[q] = __uint_as_float(r[q]);
                 if (!generic) {
                     if (add_bias) {
-                        const float4* sb4 = reinterpret_cast<const float4*>(s_bias + nb);
+                        if (bias_vec && nb + 31 < p.N) {
+                            const float4* gb4 = reinterpret_cast<const float4*>(p.epi.bias + nb);
 #pragma unroll
-                        for (int q = 0; q < 8; ++q) {
-                            const float4 b4 = sb4[q];
-                            v[4 * q] += b4.x; v[4 * q + 1] += b4.y; v[4 * q + 2] += b4.z; v[4 * q + 3] += b4.w;
+                            for (int q = 0; q < 8; ++q) {
+                                const float4 b4 = __ldg(gb4 + q);
+                                v[4 * q] += b4.x; v[4 * q + 1] += b4.y; v[4 * q + 2] += b4.z; v[4 * q + 3] += b4.w;
+                            }
+                        } else {
+#pragma unroll
+                            for (int q = 0; q < 32; ++q)
+                                if (nb + q < p.N) v[q] += __ldg(p.epi.bias + nb + q);
                         }
-                    } else if (wide_bias) {
-#pragma unroll
-                        for (int q = 0; q < 32; ++q)
-                            if (nb + q < p.N) v[q] += p.epi.bias[nb + q];
                     }
                     if (relu) {
 #pragma unroll
@@ -1076,7 +1076,7 @@ mixgcn_status launch_kind(mixgcn_ctx* ctx, int ta, int tb, int64_t M, int64_t N,
             q.n_tiles = (N + PAIR_BN - 1) / PAIR_BN;
             const int rows2 = (int)(q.n_tiles * PAIR_BN);
             const size_t stage2 = TC_BM * 128 + (PAIR_BN / 2) * 128;
-            q.stages = 5;
+            q.stages = 6;
             const size_t smem2 = (size_t)q.stages * stage2 + 8 * 4096 + 1024;
             const int tma_store2 = q.vec_c ? 1 : 0;
             CUtensorMap map_b2, map_c2 = map_a;
