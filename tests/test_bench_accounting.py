@@ -64,3 +64,27 @@ def test_gemm_flops_and_bytes(bench):
 def test_peaks_are_read_from_the_measured_file_or_fall_back(bench):
     p = bench.load_peaks()
     assert p["source"] in ("measured", "fallback") and p["hbm_gbs"] > 1000 and p["bf16_tflops"] > 100
+
+
+def test_ideal_static_cache_floor_by_hand(bench):
+    import torch
+    # 6 rows of width 4 (16-byte rows): pretend the cache holds 2 rows.  Rows are gathered 5, 3, 1, 1, 0, 0
+    # times (10 stored entries).  Cached: the rows gathered 5 and 3 times -> 2 reads; the two rows gathered
+    # once -> 2 reads; nothing else.  Bytes: row pointers 8*7, ids + values 8*10, output 4*6*4, gathers 16*4.
+    old = bench.L2_BYTES
+    bench.L2_BYTES = 2 * 16
+    try:
+        deg = torch.tensor([1, 5, 0, 3, 1, 0], dtype=torch.int32)
+        floor, k, hit = bench.ideal_cache_floor(deg, 6, 10, 4)
+    finally:
+        bench.L2_BYTES = old
+    assert k == 2 and abs(hit - 0.8) < 1e-12
+    assert floor == 8 * 7 + 8 * 10 + 4 * 6 * 4 + 16 * (2 + 2)
+
+
+def test_tensor_peak_labels(bench):
+    peaks = dict(bf16_tflops=1600.0, bf16_tflops_sustained=1300.0, source="measured")
+    assert bench.gemm_peak_for("bf16", peaks, None)[0] == 1600.0
+    assert bench.gemm_peak_for("tf32", peaks, dict(tf32_tflops_measured=700.0))[0] == 700.0
+    assert abs(bench.gemm_peak_for("tf32", peaks, None)[0] - 1600.0 * 1.1 / 2.25) < 1e-9
+    assert bench.gemm_peak_for("fp32", peaks, None)[0] is None
