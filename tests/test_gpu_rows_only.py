@@ -252,3 +252,47 @@ def test_cached_first_aggregation_matches_oracle_and_skips_the_call(mg):
         mg.layer_fwd(c2, gg, desc, Z, W, None, None, Z.clone(), Z.clone())
     assert mg.ctx_poll_status(c2, raise_on_error=False) == 0
     gg.close(); c2.close()
+
+
+@pytest.mark.parametrize("prec", ["tf32", "bf16"])
+@pytest.mark.parametrize("row_plans", [True, False])
+@pytest.mark.parametrize("rows_only", [False, True])
+def test_low_precision_products_on_the_row_sparse_paths(mg, ctx, prec, row_plans, rows_only):
+    """TF32 / BF16 products through the compacted-row backward (row plans or in-kernel row masks) and the
+    train-rows-only last layer: the compact operands have no bf16 copy from a producer, so the library
+    converts them on the fly.  Loss and the last layer's gradient (no ReLU mask below the loss) within the
+    low-precision bound of the oracle; every other gradient within the inner-product bound."""
+    from helpers import TOL_LOWP
+    from paper_2501_01951_b200.train import GcnTrainer
+    wl, s, d, _, _, _, _, _ = _tiny_problem()
+    go = orc.graph_build(wl.n, s.numpy(), d.numpy())
+    gg = mg.graph_create(ctx, wl.n, s, d)
+    dims = (40, 32, 24, 10)
+    n = go.n
+    X = synth.normal_features(n, dims[0], 71)
+    y = synth.uniform_labels(n, dims[-1], 72)
+    m = synth.bernoulli_mask(n, 0.02, 73); m[5] = 1
+    Ws = [synth.glorot_uniform(dims[l], dims[l + 1], 74 + l) for l in range(3)]
+    bs = [synth.uniform_tensor((dims[l + 1],), 84 + l, -0.1, 0.1) for l in range(3)]
+    ref = orc.train_epoch(go, X.numpy(), [w.numpy() for w in Ws], [b.numpy() for b in bs], y.numpy(), m.numpy(), None, 1, **ADAM)
+    tr = GcnTrainer(ctx, gg, dims, mg.PRECISIONS[prec], order=mg.ORDER_AGG_FIRST, row_sparse=2, row_plans=row_plans,
+                    train_rows_only=rows_only)
+    tr.set_params(Ws, bs)
+    tr.set_inputs(padded(X), y.cuda(), m.cuda())
+    before = mg.ctx_gemm_paths(ctx)
+    tr.forward(); tr.compute_loss(); tr.backward()
+    torch.cuda.synchronize()
+    after = mg.ctx_gemm_paths(ctx)
+    key = "tc_tf32" if prec == "tf32" else "tc_bf16"
+    assert after[key] - before[key] == 8 and after["simt"] == before["simt"]          # every product on the requested kernels
+    assert mg.ctx_poll_status(ctx, raise_on_error=False) == 0
+    assert abs(tr.loss.item() - ref["loss"]) <= TOL_LOWP * abs(ref["loss"])
+    assert rel_fro(tr.dW[2].cpu().numpy(), ref["dW"][2]) <= TOL_LOWP
+    Gout = ref["G"]
+    for l in range(2, -1, -1):
+        dP, dW, db, dZ = orc.update_bwd(ref["Zs"][l], ref["Ps"][l], Ws[l].numpy(), Gout, relu=l < 2, need_dZ=l > 0)
+        scale_w = np.linalg.norm(np.abs(ref["Zs"][l]).T @ np.abs(dP))
+        assert np.linalg.norm(tr.dW[l].cpu().numpy() - ref["dW"][l]) <= TOL_LOWP * scale_w
+        if l > 0:
+            Gout = orc.aggregate(go, dZ, transposed=True)
+    gg.close()
