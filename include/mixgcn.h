@@ -225,6 +225,22 @@ mixgcn_status mixgcn_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, int transposed
                           const float* Y, int64_t ldy, float* Z, int64_t ldz,
                           const mixgcn_epilogue* epi, void* stream);
 
+/* Sampled aggregation (the paper's S-SpMM, Eq. 4): Z = (A_hat Y) (.) M for a binary output mask M held as
+ * a BITMAP (the output mask buffer of Section 3.2.1): bit (j % 32) of word mask_bits[u * ld_bits + j / 32]
+ * says whether output (u, j) is kept.  Masked outputs are written as zero and are not computed: a lane all
+ * of whose output columns of a row are masked skips its gathers of that row's neighbours (on a GPU a
+ * gather moves 16 bytes per lane, so whole 16-byte groups must be masked for a load to disappear; a 50 %
+ * element mask removes few of them -- the call exists for parity with the paper's operation and for
+ * masks with structure).  The mask is applied after the epilogue's other terms.  Other arguments as
+ * mixgcn_spmm.  mixgcn_mask_pack builds a bitmap: bit (u, j) = (X == NULL or X[u*ldx + j] > 0) and
+ * (bytes == NULL or bytes[u*w + j] != 0) -- the ReLU mask of an activation (backward form) and / or a
+ * dropout byte mask (forward form); ld_bits >= ceil(w / 32) words per row. */
+mixgcn_status mixgcn_spmm_sampled(mixgcn_ctx* ctx, const mixgcn_graph* g, int transposed, int32_t w,
+                                  const float* Y, int64_t ldy, float* Z, int64_t ldz, const uint32_t* mask_bits,
+                                  int64_t ld_bits, const mixgcn_epilogue* epi, void* stream);
+mixgcn_status mixgcn_mask_pack(mixgcn_ctx* ctx, int64_t n, int32_t w, const float* X, int64_t ldx,
+                               const uint8_t* bytes, uint32_t* bits, int64_t ld_bits, void* stream);
+
 #define MIXGCN_PREC_FP32 0 /* fp32 FMA on the CUDA cores */
 #define MIXGCN_PREC_TF32 1 /* tensor cores, TF32 operands, fp32 accumulate */
 #define MIXGCN_PREC_BF16 2 /* tensor cores, BF16 operands (the fp32 operands rounded to nearest even),

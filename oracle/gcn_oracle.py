@@ -132,6 +132,11 @@ def aggregate(g: Graph, X, transposed=False):
     return Z
 
 
+def sampled_aggregate(g: Graph, X, M, transposed=False):
+    """Z = (A_hat X) (.) M, the sampled aggregation of Eq. 4: M is a 0/1 array of Z's shape (1 = kept)."""
+    return aggregate(g, X, transposed) * (np.asarray(M) != 0)
+
+
 def aggregate_rows(g: Graph, X, rows, transposed=False):
     """Rows ``rows`` of A_hat X (or A_hat^T X) only; X may be any array indexable by node id
     whose needed rows are present (here: a full n x d array)."""

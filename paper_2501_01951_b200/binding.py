@@ -44,7 +44,7 @@ SYMBOLS = (
     "mixgcn_graph_bandwidth", "mixgcn_graph_rcm", "mixgcn_pipeline_stages", "mixgcn_graph_create_permuted",
     "mixgcn_count_rows", "mixgcn_rowplan_create", "mixgcn_rowplan_destroy", "mixgcn_rowplan_info",
     "mixgcn_rowplan_export", "mixgcn_spmm_rowplan", "mixgcn_colsum", "mixgcn_ctx_gemm_paths",
-    "mixgcn_train_step_host_prefetch", "mixgcn_probe_gather",
+    "mixgcn_train_step_host_prefetch", "mixgcn_probe_gather", "mixgcn_spmm_sampled", "mixgcn_mask_pack",
 )
 
 
@@ -489,3 +489,27 @@ def probe_gather(ctx: Ctx, table: torch.Tensor, gathers_per_warp: int, sink: tor
     _check(lib.mixgcn_probe_gather(ctx.h, _ptr(table), C.c_int64(table.shape[0]), C.c_int64(gathers_per_warp),
                                    C.c_uint64(seed), _ptr(sink), C.byref(total), _stream()))
     return total.value
+
+
+def mask_pack(ctx: Ctx, w: int, bits: torch.Tensor, X: torch.Tensor | None = None, bytes_mask: torch.Tensor | None = None):
+    """bits (n x ld_bits int32 device tensor) <- bitmap of (X > 0) and / or (bytes_mask != 0)."""
+    _dev(bits, torch.int32, "bits")
+    n, ld_bits = bits.shape[0], bits.stride(0)
+    ldx = 0
+    if X is not None:
+        X, ldx = _mat(X, "X")
+    if bytes_mask is not None:
+        _dev(bytes_mask, torch.uint8, "bytes_mask")
+    _check(lib.mixgcn_mask_pack(ctx.h, C.c_int64(n), C.c_int32(w), _ptr(X), C.c_int64(ldx), _ptr(bytes_mask), _ptr(bits),
+                                C.c_int64(ld_bits), _stream()))
+
+
+def spmm_sampled(ctx: Ctx, g: Graph, Y: torch.Tensor, Z: torch.Tensor, w: int, bits: torch.Tensor, transposed: bool = False,
+                 epi: Epilogue | None = None):
+    """Z = (A_hat Y) (.) M with M given as a bitmap (n x ld_bits int32 words)."""
+    Y, ldy = _mat(Y, "Y")
+    Z, ldz = _mat(Z, "Z")
+    _dev(bits, torch.int32, "bits")
+    _check(lib.mixgcn_spmm_sampled(ctx.h, g.h, C.c_int(int(transposed)), C.c_int32(w), _ptr(Y), C.c_int64(ldy), _ptr(Z),
+                                   C.c_int64(ldz), _ptr(bits), C.c_int64(bits.stride(0)), None if epi is None else C.byref(epi),
+                                   _stream()))

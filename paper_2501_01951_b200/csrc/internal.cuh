@@ -184,6 +184,8 @@ struct SpmmOpts {
     int64_t row_limit = -1;                  // >= 0: only the first row_limit rows of the schedule (longest first)
     uint16_t* Z_lp = nullptr;                // nullable: also write a bf16 copy of Z (after the epilogue), ldz_lp a multiple of 4
     int64_t ldz_lp = 0;
+    const uint32_t* out_bits = nullptr;      // nullable: bit-packed output mask of a sampled aggregation (Eq. 4), n x ld_bits words
+    int64_t ld_bits = 0;
 };
 mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView& A, int chunks, int k,
                           int32_t w, const float* Y, int64_t ldy, float* Z, int64_t ldz,

@@ -56,6 +56,9 @@ struct SpmmParams {
     // row filter (spmm_filtered_kernel): only output rows u with row_filter[u] != 0 are computed and written
     const uint8_t* row_filter;
     const int32_t* seg_perm;   // segment records carry the long row's index i; its row is seg_perm[i] (null: the record's row)
+    // sampled aggregation Z = (A_hat Y) (.) M, Eq. 4: bit j of row u of the bitmap says whether output (u, j) is kept
+    const uint32_t* out_bits;  // [n x ld_bits] words, null: every output is kept
+    int64_t ld_bits;
     // epilogue
     const float* bias; int relu;
     const uint8_t* drop; float keep_scale;
@@ -93,6 +96,11 @@ __device__ __forceinline__ void store_row(const SpmmParams& p, int64_t u, int c4
     }
 #pragma unroll
     for (int t = 0; t < 4; ++t) r[t] = (j + t < jend) ? epilogue1(p, r[t], u, j + t) : 0.0f;
+    if (p.out_bits) {
+        const uint32_t nib = (__ldg(p.out_bits + u * p.ld_bits + (j >> 5)) >> (j & 31)) & 0xFu;   // j % 4 == 0: one word
+#pragma unroll
+        for (int t = 0; t < 4; ++t) r[t] = ((nib >> t) & 1u) ? r[t] : 0.0f;
+    }
     *reinterpret_cast<float4*>(p.Z + u * p.ldz + j) = make_float4(r[0], r[1], r[2], r[3]);
     if (p.Z_lp) store_lp4(p.Z_lp + u * p.ldz_lp + j, r[0], r[1], r[2], r[3]);
 }
@@ -113,7 +121,7 @@ struct Cfg {
 // so that the index load's latency is hidden behind them instead of preceding every batch.
 template <int LPR, int VPL>
 __device__ __forceinline__ void row_segment(const SpmmParams& p, int64_t b, int64_t e, int lig, unsigned mask,
-                                            int w4, float4 (&acc)[VPL]) {
+                                            int w4, float4 (&acc)[VPL], unsigned keep = 0xFFFFFFFFu) {
     constexpr int U = Cfg<LPR, VPL>::U;
     const float* Yb = p.Y + p.j0;
     int c = 0; float a = 0.0f;
@@ -136,7 +144,7 @@ __device__ __forceinline__ void row_segment(const SpmmParams& p, int64_t b, int6
 #pragma unroll
                 for (int v = 0; v < VPL; ++v) {
                     const int c4 = lig + v * LPR;
-                    y[t][v] = (live && c4 < w4) ? __ldg(yr + c4) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    y[t][v] = (live && c4 < w4 && ((keep >> v) & 1u)) ? __ldg(yr + c4) : make_float4(0.f, 0.f, 0.f, 0.f);
                 }
             }
 #pragma unroll
@@ -171,7 +179,22 @@ __global__ void __launch_bounds__(256, VPL <= 2 ? SPMM_MINB : 1) spmm_group_kern
     float4 acc[VPL];
 #pragma unroll
     for (int v = 0; v < VPL; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
-    row_segment<LPR, VPL>(p, b, e, lig, mask, w4, acc);
+    unsigned keep = 0xFFFFFFFFu;
+    if (p.out_bits) {
+        // Eq. 4: outputs the mask drops are never computed -- a lane whose four columns of this row are all
+        // masked skips its gathers of every neighbour (the mask is known before the aggregation)
+        const int64_t row = p.seg_perm ? __ldg(p.seg_perm + u) : u;
+        keep = 0u;
+#pragma unroll
+        for (int v = 0; v < VPL; ++v) {
+            const int c4 = lig + v * LPR;
+            if (c4 < w4) {
+                const int j = p.j0 + c4 * 4;
+                if ((__ldg(p.out_bits + row * p.ld_bits + (j >> 5)) >> (j & 31)) & 0xFu) keep |= 1u << v;
+            }
+        }
+    }
+    row_segment<LPR, VPL>(p, b, e, lig, mask, w4, acc, keep);
     if (p.partial) {
         float4* dst = reinterpret_cast<float4*>(p.partial + idx * p.ldp);
 #pragma unroll
@@ -485,6 +508,7 @@ mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView&
     p.rowptr = A.rowptr; p.col = A.col; p.val = A.val;
     p.Y = Y; p.ldy = ldy; p.Z = Z; p.ldz = ldz; p.w_total = w;
     p.Z_lp = opts.Z_lp; p.ldz_lp = opts.ldz_lp;
+    p.out_bits = opts.out_bits; p.ld_bits = opts.ld_bits;
     if (epi) {
         p.bias = epi->bias; p.relu = epi->relu; p.drop = epi->drop_mask; p.keep_scale = epi->keep_scale;
         p.gate = epi->gate; p.ld_gate = epi->ld_gate; p.gate_scale = epi->gate_scale;
@@ -569,7 +593,9 @@ mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView&
             {
                 LaunchScope scope(ctx, phase, s);
                 p.idx_begin = 0; p.idx_end = S.total_segs;
+                if (p.out_bits) p.seg_perm = S.perm;       // a segment's record names its long row by ordinal
                 dispatch(p, p.w <= SPMM_FOLD_WMAX ? SPMM_FOLD_SEG : 1, s);
+                p.seg_perm = nullptr;
             }
             {
                 LaunchScope scope(ctx, phase, s);
@@ -628,4 +654,55 @@ extern "C" mixgcn_status mixgcn_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, int
     if (epi && epi->residual && (epi->ld_residual < w || epi->residual == Z)) MIXGCN_FAIL(MIXGCN_EINVAL, "spmm: residual needs ld_residual >= w and must not be the output");
     MIXGCN_CUDA(cudaSetDevice(ctx->device));
     return launch_spmm(ctx, g, transposed ? g->bwd : g->fwd, 1, 0, w, Y, ldy, Z, ldz, epi, (cudaStream_t)stream);
+}
+
+namespace {
+
+// bits[u][j] = (X == null || X[u][j] > 0) && (bytes == null || bytes[u*w + j] != 0): one thread per 32-bit word
+__global__ void mask_pack_kernel(int64_t n, int w, const float* __restrict__ X, int64_t ldx, const uint8_t* __restrict__ bytes,
+                                 uint32_t* __restrict__ bits, int64_t ld_bits) {
+    const int words = (w + 31) >> 5;
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= n * words) return;
+    const int64_t u = t / words; const int wd = (int)(t % words);
+    uint32_t out = 0;
+    for (int b = 0; b < 32; ++b) {
+        const int j = wd * 32 + b;
+        if (j >= w) break;
+        bool on = true;
+        if (X) on = X[u * ldx + j] > 0.0f;
+        if (bytes) on = on && bytes[u * (int64_t)w + j] != 0;
+        out |= (on ? 1u : 0u) << b;
+    }
+    bits[u * ld_bits + wd] = out;
+}
+
+}  // namespace
+
+extern "C" mixgcn_status mixgcn_mask_pack(mixgcn_ctx* ctx, int64_t n, int32_t w, const float* X, int64_t ldx,
+                                          const uint8_t* bytes, uint32_t* bits, int64_t ld_bits, void* stream) {
+    if (!ctx || !bits || (!X && !bytes)) MIXGCN_FAIL(MIXGCN_EINVAL, "mask_pack: null argument");
+    if (n <= 0 || w <= 0 || ld_bits < (w + 31) / 32 || (X && ldx < w)) MIXGCN_FAIL(MIXGCN_EINVAL, "mask_pack: need n, w > 0, ld_bits >= ceil(w/32), ldx >= w");
+    MIXGCN_CUDA(cudaSetDevice(ctx->device));
+    const int64_t total = n * ((w + 31) / 32);
+    LaunchScope scope(ctx, PH_ELEM, (cudaStream_t)stream);
+    mask_pack_kernel<<<(unsigned)((total + 255) / 256), 256, 0, (cudaStream_t)stream>>>(n, w, X, ldx, bytes, bits, ld_bits);
+    MIXGCN_CUDA(cudaGetLastError());
+    return MIXGCN_OK;
+}
+
+extern "C" mixgcn_status mixgcn_spmm_sampled(mixgcn_ctx* ctx, const mixgcn_graph* g, int transposed, int32_t w,
+                                             const float* Y, int64_t ldy, float* Z, int64_t ldz, const uint32_t* mask_bits,
+                                             int64_t ld_bits, const mixgcn_epilogue* epi, void* stream) {
+    if (!ctx || !g || !Y || !Z || !mask_bits) MIXGCN_FAIL(MIXGCN_EINVAL, "spmm_sampled: null argument");
+    if (w <= 0) MIXGCN_FAIL(MIXGCN_EINVAL, "spmm_sampled: w must be positive (got %d)", w);
+    if (ldy < w || ldz < w || (ldy & 3) || (ldz & 3) || ld_bits < (w + 31) / 32)
+        MIXGCN_FAIL(MIXGCN_EINVAL, "spmm_sampled: leading dimensions must be multiples of 4 and >= w, ld_bits >= ceil(w/32)");
+    if (!aligned16(Y) || !aligned16(Z)) MIXGCN_FAIL(MIXGCN_EINVAL, "spmm_sampled: Y and Z must be 16-byte aligned");
+    if (Y == Z) MIXGCN_FAIL(MIXGCN_EINVAL, "spmm_sampled: Y and Z must not overlap");
+    if (epi && epi->gate && epi->ld_gate < w) MIXGCN_FAIL(MIXGCN_EINVAL, "spmm_sampled: gate leading dimension < w");
+    if (epi && epi->residual && (epi->ld_residual < w || epi->residual == Z)) MIXGCN_FAIL(MIXGCN_EINVAL, "spmm_sampled: residual needs ld_residual >= w and must not be the output");
+    MIXGCN_CUDA(cudaSetDevice(ctx->device));
+    SpmmOpts opts; opts.out_bits = mask_bits; opts.ld_bits = ld_bits;
+    return launch_spmm(ctx, g, transposed ? g->bwd : g->fwd, 1, 0, w, Y, ldy, Z, ldz, epi, (cudaStream_t)stream, opts);
 }

@@ -56,6 +56,7 @@ def main():
     ap.add_argument("--mask-p", type=float, default=0.01, help="loss / model: fraction of train rows")
     ap.add_argument("--loss-rows", type=int, default=0, choices=[0, 1, 2], help="loss: MIXGCN_OPT_LOSS_TRAIN_ROWS_ONLY value")
     ap.add_argument("--slice", type=int, default=0, help="feature-column slice width of the aggregation (0 = default)")
+    ap.add_argument("--sampled", type=float, default=0.0, help="spmm: also time the sampled aggregation (Eq. 4) with this fraction of outputs kept")
     args = ap.parse_args()
 
     dev = torch.device("cuda", 0)
@@ -74,6 +75,22 @@ def main():
         alg = 8 * (g.n + 1) + 8 * g.nnz + 8 * g.n * args.w
         out.update(n=g.n, nnz=g.nnz, w=args.w, max_deg=g.max_deg, ms_median=round(med, 4), ms_best=round(best, 4),
                    alg_bytes=alg, alg_gbs=round(alg / med / 1e6, 1), gather_gbs=round(4 * g.nnz * args.w / med / 1e6, 1))
+        if args.sampled:
+            # the sampled aggregation of Eq. 4 on the same graph: a random element mask, and a mask that
+            # drops the same fraction as whole 16-byte groups
+            bits = torch.zeros((g.n, (args.w + 31) // 32), dtype=torch.int32, device=dev)
+            for name, group in (("element_mask", 1), ("group_mask", 4)):
+                cols = (args.w + group - 1) // group
+                m8 = torch.empty((g.n, args.w), dtype=torch.uint8, device=dev)
+                gen = torch.Generator(device=dev).manual_seed(11)
+                for r0 in range(0, g.n, 1 << 21):                       # a seeded mask, drawn in row blocks
+                    r1 = min(g.n, r0 + (1 << 21))
+                    keep = (torch.rand((r1 - r0, cols), generator=gen, device=dev) < args.sampled).to(torch.uint8)
+                    m8[r0:r1] = keep.repeat_interleave(group, dim=1)[:, : args.w]
+                mg.mask_pack(ctx, args.w, bits, bytes_mask=m8)
+                del keep, m8
+                med_s, best_s = _time(lambda: mg.spmm_sampled(ctx, g, Y, Z, args.w, bits), args.iters, args.warmup)
+                out["sampled_" + name] = dict(keep_fraction=args.sampled, ms_median=round(med_s, 4), ms_best=round(best_s, 4))
     elif args.op == "model":
         from .sage_gin import GinTrainer, SageTrainer
         from .train import GcnTrainer

@@ -411,6 +411,44 @@ def test_layer_chunked_pipeline_matches_unchunked(mg, ctx, n_chunks):
                n_chunks=n_chunks, seed=95)
 
 
+@pytest.mark.parametrize("name", ["messy-sym", "messy-directed", "hub"])
+@pytest.mark.parametrize("w", [8, 41, 128, 300])
+@pytest.mark.parametrize("transposed", [False, True])
+def test_sampled_spmm_matches_eq4(mg, ctx, name, w, transposed):
+    """Z = (A_hat Y) (.) M (Eq. 4) with M as a bitmap: against the oracle, bitwise equal to the unmasked
+    aggregation where the mask keeps an output, exactly zero where it does not -- for a random half mask, a
+    mask with whole 16-byte groups and whole rows dropped (the loads that can be skipped), and the ReLU form."""
+    go, gg = build_both(mg, ctx, name)
+    n = go.n
+    Y = synth.uniform_tensor((n, w), 511 + w, -1, 1)
+    ld_bits = (w + 31) // 32 + 1                                     # one spare word per row: must stay untouched
+    Yd = padded(Y, fill=float("nan"))
+    plain = torch.zeros(n, round4(w), device="cuda")
+    mg.spmm(ctx, gg, Yd, plain, w, transposed=transposed)
+    rng = np.random.default_rng(w)
+    M1 = rng.integers(0, 2, (n, w)).astype(np.uint8)
+    M2 = np.repeat(rng.integers(0, 2, (n, (w + 3) // 4)), 4, axis=1)[:, :w].astype(np.uint8)
+    M2[rng.integers(0, 2, n) == 0] = 0
+    for M in (M1, M2):
+        bits = torch.full((n, ld_bits), -1, dtype=torch.int32, device="cuda")
+        mg.mask_pack(ctx, w, bits, bytes_mask=torch.tensor(M).cuda().contiguous())
+        assert torch.all(bits[:, -1] == -1)
+        Z = torch.full((n, round4(w)), 7.0, device="cuda")
+        mg.spmm_sampled(ctx, gg, Yd, Z, w, bits, transposed=transposed)
+        want = orc.sampled_aggregate(go, Y.numpy(), M, transposed=transposed)
+        assert rel_fro(host(Z, w), want) <= TOL_FP32
+        Mt = torch.tensor(M).cuda().bool()
+        assert torch.equal(Z[:, :w][Mt], plain[:, :w][Mt]) and torch.all(Z[:, :w][~Mt] == 0)
+    # backward form: the mask is the ReLU mask of another activation
+    A = synth.uniform_tensor((n, w), 512 + w, -1, 1)
+    bits = torch.zeros((n, ld_bits), dtype=torch.int32, device="cuda")
+    mg.mask_pack(ctx, w, bits, X=padded(A))
+    Z = torch.zeros(n, round4(w), device="cuda")
+    mg.spmm_sampled(ctx, gg, Yd, Z, w, bits, transposed=transposed)
+    assert rel_fro(host(Z, w), orc.sampled_aggregate(go, Y.numpy(), A.numpy() > 0, transposed=transposed)) <= TOL_FP32
+    assert mg.ctx_poll_status(ctx, raise_on_error=False) == 0
+
+
 def _tiny_problem():
     wl = synth.CONFIGS["C1"]
     s, d = synth.rmat_graph(wl.n, wl.undirected_edges, wl.seed("graph"))

@@ -180,6 +180,20 @@ def test_aggregate_matches_dense(ne, sym, d):
     np.testing.assert_allclose(orc.aggregate_rows(g, X, rows, transposed=True), (Ah.T @ X)[rows], rtol=1e-12, atol=1e-13)
 
 
+def test_sampled_aggregate_is_the_masked_dense_product():
+    # Eq. 4 on a dense matrix: (A_hat X) (.) M, with a mask that keeps nothing, everything, and a random half
+    n, d = 12, 7
+    rng = np.random.default_rng(4)
+    src, dst = rng.integers(0, n, 30), rng.integers(0, n, 30)
+    g = orc.graph_build(n, src, dst)
+    Ah = dense_ahat(n, list(src), list(dst), True)
+    X = rng.standard_normal((n, d))
+    for M in (np.zeros((n, d)), np.ones((n, d)), rng.integers(0, 2, (n, d))):
+        np.testing.assert_allclose(orc.sampled_aggregate(g, X, M), (Ah @ X) * M, rtol=1e-12, atol=1e-13)
+    M = rng.integers(0, 2, (n, d))
+    assert np.all(orc.sampled_aggregate(g, X, M)[M == 0] == 0.0)
+
+
 def test_aggregate_vs_scipy_at_tiny_size():
     from paper_2501_01951_b200 import synth
     wl = synth.CONFIGS["C1"]
