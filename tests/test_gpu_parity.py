@@ -807,6 +807,56 @@ def test_weight_gradient_on_cta_pairs(mg, ctx, M, N, K, prec):
     assert mg.ctx_poll_status(ctx, raise_on_error=False) == 0
 
 
+def test_weight_gradient_on_cta_pairs_without_a_split(mg, ctx):
+    """K too short to split: the pair kernel writes the final tile itself and applies the epilogue."""
+    M, N, K = 2048, 2048, 4096
+    A, B = synth.normal_features(K, M, 361), synth.normal_features(K, N, 362)
+    bias = synth.uniform_tensor((N,), 363, -1, 1)
+    Cd = torch.zeros(M, N, device="cuda")
+    before = mg.ctx_gemm_paths(ctx)["cta_pairs"]
+    mg.gemm(ctx, mg.PREC_BF16, True, False, M, N, K, A.cuda(), B.cuda(), Cd, epi=mg.make_epilogue(bias=bias.cuda(), relu=True))
+    assert mg.ctx_gemm_paths(ctx)["cta_pairs"] == before + 1
+    want = np.maximum(_bf16_round(A.numpy()).T @ _bf16_round(B.numpy()) + bias.numpy().astype(np.float64), 0.0)
+    assert rel_fro(host(Cd), want) <= 2e-5
+    assert mg.ctx_poll_status(ctx, raise_on_error=False) == 0
+
+
+@pytest.mark.parametrize("with_copies", [True, False])
+def test_chunked_pipeline_with_bf16_products(mg, ctx, with_copies):
+    """Row chunks on two streams with BF16 products: with the caller's bf16 copy of `saved` each chunk's
+    update reads its rows of it; without, the chunks fall back to TF32 (two streams cannot share the
+    conversion workspace).  Output within the low-precision bound either way."""
+    from helpers import TOL_LOWP
+    go, gg = build_both(mg, ctx, "hub")
+    n, d_in, d_out = go.n, 64, 48
+    X = synth.uniform_tensor((n, d_in), 371, -1, 1); W = synth.glorot_uniform(d_in, d_out, 372)
+    b = synth.uniform_tensor((d_out,), 373, -0.2, 0.2)
+    desc = mg.layer_desc(d_in, d_out, round4(d_in), round4(d_out), round4(d_in), mg.ORDER_AGG_FIRST, mg.PREC_BF16, mg.LAYER_RELU,
+                         1.0, 1.0, 3)
+    saved = torch.zeros(n, round4(d_in), device="cuda"); Xout = torch.zeros(n, round4(d_out), device="cuda")
+    keep = []
+    if with_copies:
+        s_lp = torch.zeros(n, 64, dtype=torch.bfloat16, device="cuda"); o_lp = torch.zeros(n, 48, dtype=torch.bfloat16, device="cuda")
+        keep = [s_lp, o_lp]
+        desc.saved_lp, desc.ld_saved_lp = s_lp.data_ptr(), 64
+        desc.x_out_lp, desc.ld_out_lp = o_lp.data_ptr(), 48
+        desc.ld_in_lp = 64
+    before = mg.ctx_gemm_paths(ctx)
+    mg.layer_fwd(ctx, gg, desc, padded(X), W.cuda(), b.cuda(), None, saved, Xout)
+    torch.cuda.synchronize()
+    after = mg.ctx_gemm_paths(ctx)
+    key = "tc_bf16" if with_copies else "tc_tf32"
+    assert after[key] - before[key] == 3
+    Z = orc.aggregate(go, X.numpy())
+    want = orc.activation(orc.update(Z, W.numpy(), b.numpy()), True)
+    assert rel_fro(host(Xout, d_out), want) <= TOL_LOWP
+    assert rel_fro(host(saved, d_in), Z) <= TOL_FP32
+    if with_copies:
+        assert rel_fro(keep[0].float().cpu().numpy(), _bf16_round(host(saved, d_in))) == 0.0          # the copy is bf16(saved), bit for bit
+        assert rel_fro(keep[1].float().cpu().numpy(), _bf16_round(host(Xout, d_out))) == 0.0
+    assert mg.ctx_poll_status(ctx, raise_on_error=False) == 0
+
+
 def test_gemm_on_cta_pairs_with_gate_and_dropout(mg, ctx):
     """The per-element epilogue terms (gate by another tensor's sign, dropout mask) on the pair kernel."""
     M, N, K = 4200, 520, 512
