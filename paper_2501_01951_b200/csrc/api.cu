@@ -99,7 +99,7 @@ mixgcn_status ensure_workspace_lp(mixgcn_ctx* ctx, int64_t bytes) {
 
 mixgcn_status launch_gemm(mixgcn_ctx* ctx, int precision, int ta, int tb, int64_t M, int64_t N, int64_t K,
                           const float* A, int64_t lda, const float* B, int64_t ldb, float* C, int64_t ldc,
-                          const mixgcn_epilogue* epi, int64_t epi_row0, cudaStream_t s, const GemmLP* lp) {
+                          const mixgcn_epilogue* epi, int64_t epi_row0, cudaStream_t s, const GemmLP* lp, float* colsum_b) {
     // BF16 requests go to the tcgen05 kind::f16 kernels on bf16 copies of the activation operands: the
     // copies a producer already wrote (lp), else copies made here by a conversion kernel.  TF32
     // requests, and BF16 requests whose shape the bf16 kernels do not take, go to the kind::tf32
@@ -137,8 +137,11 @@ mixgcn_status launch_gemm(mixgcn_ctx* ctx, int precision, int ta, int tb, int64_
                             C, ldc, epi, epi_row0, s, ta ? nullptr : c_lp, ldc_lp);
         if (st == MIXGCN_OK) { ctx->gemm_path[2]++; c_lp_done = !ta && c_lp; }
     }
+    bool colsum_done = false;
+    if (colsum_b && !ta) MIXGCN_FAIL(MIXGCN_EINVAL, "gemm: column sums of B are a by-product of the weight-gradient form only");
     if (st == MIXGCN_EUNSUPPORTED && precision != MIXGCN_PREC_FP32) {
-        st = launch_gemm_tc(ctx, 0, ta, tb, M, N, K, A, lda, B, ldb, C, ldc, epi, epi_row0, s, ta ? nullptr : c_lp, ldc_lp);
+        st = launch_gemm_tc(ctx, 0, ta, tb, M, N, K, A, lda, B, ldb, C, ldc, epi, epi_row0, s, ta ? nullptr : c_lp, ldc_lp,
+                            colsum_b, &colsum_done);
         if (st == MIXGCN_OK) { ctx->gemm_path[1]++; c_lp_done = !ta && c_lp; }
     }
     if (st == MIXGCN_EUNSUPPORTED) {
@@ -147,6 +150,7 @@ mixgcn_status launch_gemm(mixgcn_ctx* ctx, int precision, int ta, int tb, int64_
     }
     if (st != MIXGCN_OK) return st;
     if (c_lp && !c_lp_done) MIXGCN_TRY(launch_to_bf16(ctx, M, (int32_t)N, C, ldc, c_lp, ldc_lp, s));
+    if (colsum_b && !colsum_done) MIXGCN_TRY(launch_colsum(ctx, K, (int32_t)N, B, ldb, colsum_b, s));
     return MIXGCN_OK;
 }
 
@@ -533,10 +537,10 @@ extern "C" mixgcn_status mixgcn_layer_bwd(mixgcn_ctx* ctx, const mixgcn_graph* g
         plan_opts.Z_lp = lp.g_in; plan_opts.ldz_lp = lp.ld_in;
         plan_all.Z_lp = lp.saved; plan_all.ldz_lp = lp.ld_saved;
         MIXGCN_TRY(launch_gather_rows(ctx, cnt, d->d_out, plan->idx, G_out, d->ld_out, cb, ldb, s));         // dP_T
-        if (dbias) MIXGCN_TRY(launch_colsum(ctx, cnt, d->d_out, cb, ldb, dbias, s));
         if (order == MIXGCN_ORDER_AGG_FIRST) {
             MIXGCN_TRY(launch_gather_rows(ctx, cnt, d->d_in, plan->idx, saved, d->ld_saved, ca, lda, s));     // Z_T
-            MIXGCN_TRY(launch_gemm(ctx, d->precision, 1, 0, d->d_in, d->d_out, cnt, ca, lda, cb, ldb, dW, ldw, nullptr, 0, s));
+            // dW = Z_T^T dP_T, and db = 1^T dP_T as its by-product
+            MIXGCN_TRY(launch_gemm(ctx, d->precision, 1, 0, d->d_in, d->d_out, cnt, ca, lda, cb, ldb, dW, ldw, nullptr, 0, s, nullptr, dbias));
             if (!first) {
                 MIXGCN_TRY(launch_gemm(ctx, d->precision, 0, 1, cnt, d->d_in, d->d_out, cb, ldb, W, ldw, ca, lda, nullptr, 0, s));
                 MIXGCN_TRY(launch_spmm(ctx, g, plan->view, 1, 0, d->d_in, ca, lda, G_in, d->ld_in, gin, s, plan_opts));
@@ -544,6 +548,7 @@ extern "C" mixgcn_status mixgcn_layer_bwd(mixgcn_ctx* ctx, const mixgcn_graph* g
             return MIXGCN_OK;
         }
         // update first: dQ = A_hat^T dZ from the compacted rows (into `saved`, every row), then the dense products
+        if (dbias) MIXGCN_TRY(launch_colsum(ctx, cnt, d->d_out, cb, ldb, dbias, s));
         MIXGCN_TRY(launch_spmm(ctx, g, plan->view, 1, 0, d->d_out, cb, ldb, saved, d->ld_saved, nullptr, s, plan_all));
         GemmLP wlp; wlp.A = lp.x_in; wlp.lda = lp.ld_in; wlp.B = lp.saved; wlp.ldb = lp.ld_saved;
         MIXGCN_TRY(launch_gemm(ctx, d->precision, 1, 0, d->d_in, d->d_out, n, X_in, d->ld_in, saved, d->ld_saved, dW, ldw, nullptr, 0, s, &wlp));
@@ -570,8 +575,7 @@ extern "C" mixgcn_status mixgcn_layer_bwd(mixgcn_ctx* ctx, const mixgcn_graph* g
             MIXGCN_TRY(build_row_set(ctx, n, rmask, cnt, lda, ldb, &rs, s));
             MIXGCN_TRY(launch_gather_rows(ctx, cnt, d->d_in, rs.idx, saved, d->ld_saved, rs.a, lda, s));     // Z_T
             MIXGCN_TRY(launch_gather_rows(ctx, cnt, d->d_out, rs.idx, G_out, d->ld_out, rs.b, ldb, s));      // dP_T
-            if (dbias) MIXGCN_TRY(launch_colsum(ctx, cnt, d->d_out, rs.b, ldb, dbias, s));
-            MIXGCN_TRY(launch_gemm(ctx, d->precision, 1, 0, d->d_in, d->d_out, cnt, rs.a, lda, rs.b, ldb, dW, ldw, nullptr, 0, s));
+            MIXGCN_TRY(launch_gemm(ctx, d->precision, 1, 0, d->d_in, d->d_out, cnt, rs.a, lda, rs.b, ldb, dW, ldw, nullptr, 0, s, nullptr, dbias));
             if (!first) {
                 MIXGCN_TRY(launch_gemm(ctx, d->precision, 0, 1, cnt, d->d_in, d->d_out, rs.b, ldb, W, ldw, rs.a, lda, nullptr, 0, s));
                 sp.in_pos = rs.pos;                                                                             // dZ_T is compact
@@ -580,10 +584,10 @@ extern "C" mixgcn_status mixgcn_layer_bwd(mixgcn_ctx* ctx, const mixgcn_graph* g
             return MIXGCN_OK;
         }
         // dW = (A_hat X_in)^T dP ; dZ = dP W^T (over `saved`) ; G_in = A_hat^T dZ
-        if (dbias) MIXGCN_TRY(launch_colsum(ctx, n, d->d_out, G_out, d->ld_out, dbias, s));
+        // dW = (A_hat X_in)^T dP, and db = 1^T dP as its by-product
         GemmLP wlp; wlp.A = lp.saved; wlp.lda = lp.ld_saved; wlp.B = lp.g_out; wlp.ldb = lp.ld_out;
         MIXGCN_TRY(launch_gemm(ctx, d->precision, 1, 0, d->d_in, d->d_out, n, saved, d->ld_saved, G_out, d->ld_out, dW,
-                               ldw, nullptr, 0, s, &wlp));
+                               ldw, nullptr, 0, s, &wlp, dbias));
         if (!first) {
             GemmLP zlp; zlp.A = lp.g_out; zlp.lda = lp.ld_out;
             MIXGCN_TRY(launch_gemm(ctx, d->precision, 0, 1, n, d->d_in, d->d_out, G_out, d->ld_out, W, ldw, saved,

@@ -63,6 +63,7 @@ struct TcParams {
     float* C; int64_t ldc; int vec_c;
     uint16_t* C_lp; int64_t ldc_lp;   // nullable: bf16 copy of C (after the epilogue); ldc_lp a multiple of 8
     int raw;                // 1: store the accumulator unchanged (split-K partial)
+    double* colsum_part;    // weight-gradient form, TF32: nullable [splits][N] column sums of B over this split's k-rows
     TcEpi epi;
     int32_t* status;
     uint32_t wait_limit;    // polls after which a wait gives up
@@ -124,9 +125,14 @@ __global__ void __launch_bounds__(TC_THREADS) gemm_tc_kernel(const __grid_consta
     uint32_t tmem_cols = 32;
     while ((int)tmem_cols < p.bn) tmem_cols <<= 1;
 
+    // Column sums of B (the bias gradient 1^T dP when B = dP) as a by-product: the four epilogue warps are
+    // idle while the tiles stream through shared memory, so in the CTAs of the first row of tiles they add up
+    // each stage's B tile (fp32 words, TF32 kind only) before the stage is released.
+    const bool do_colsum = MN_MAJOR && KIND == KIND_TF32 && p.colsum_part != nullptr && tile / p.n_tiles == 0;
+
     if (threadIdx.x == 0) {
         abort_flag = 0;
-        for (int s = 0; s < p.stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        for (int s = 0; s < p.stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], do_colsum ? 5 : 1); }
         mbar_init(&acc_bar, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -192,7 +198,43 @@ __global__ void __launch_bounds__(TC_THREADS) gemm_tc_kernel(const __grid_consta
     } else {
         // ---------------- epilogue: warps 0..3 own TMEM lanes 32*warp .. 32*warp+31 ----------------
         bool ok = true;
-        if (nk > 0) {
+        if (do_colsum) {
+            // warp w takes the 32-column chunks w and w + 4 of the B tile, lane l their column l.  A chunk is BK
+            // k-rows of 128 bytes in the 128-byte swizzle with 32-byte atoms: the 32-byte group g of k-row r sits
+            // at group position g ^ (r & 3).
+            double sum[2] = {0.0, 0.0};
+            const int chunks = bn_pad / Cfg::CHUNK;
+            for (int ks = 0; ks < nk && ok; ++ks) {
+                const int s = ks % p.stages;
+                const uint32_t ph = (ks / p.stages) & 1;
+                if (lane == 0) ok = mbar_wait(&full_bar[s], ph, &abort_flag, p.wait_limit);
+                ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
+                if (!ok) { if (lane == 0) { abort_flag = 1; atomicMax(p.status, DEV_WAIT_EXPIRED); } break; }
+                const uint8_t* sb = smem + (size_t)s * stage_bytes + a_bytes;
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const int cc = warp + 4 * h;
+                    if (cc < chunks) {
+                        const float* chunk = reinterpret_cast<const float*>(sb + (size_t)cc * Cfg::MN_CHUNK_BYTES);
+                        float part = 0.0f;
+#pragma unroll 8
+                        for (int r = 0; r < BK; ++r) part += chunk[r * 32 + (lane ^ ((r & 3) << 3))];
+                        sum[h] += (double)part;
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&empty_bar[s]);      // this warp has read the stage
+            }
+            if (ok) {
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const int cc = warp + 4 * h;
+                    const int64_t n = n0 + cc * 32 + lane;
+                    if (cc < chunks && cc * 32 + lane < p.bn && n < p.N) p.colsum_part[(int64_t)blockIdx.z * p.N + n] = sum[h];
+                }
+            }
+        }
+        if (ok && nk > 0) {
             if (lane == 0) ok = mbar_wait(&acc_bar, 0, &abort_flag, p.wait_limit);
             ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
             if (!ok && lane == 0) { abort_flag = 1; atomicMax(p.status, DEV_WAIT_EXPIRED); }
@@ -934,6 +976,15 @@ __global__ void pack_b_kernel(const float* __restrict__ src, int64_t ld, int tra
     else reinterpret_cast<uint16_t*>(dst)[i] = (uint16_t)(pack_bf16(v, 0.0f) & 0xFFFFu);
 }
 
+// out[n] = sum over splits (ascending) of part[z][n]
+__global__ void colsum_splits_kernel(int64_t N, int splits, const double* __restrict__ part, float* __restrict__ out) {
+    const int64_t n = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (n >= N) return;
+    double sacc = 0.0;
+    for (int z = 0; z < splits; ++z) sacc += part[(int64_t)z * N + n];
+    out[n] = (float)sacc;
+}
+
 // dst[r][c] = bf16(src[r][c]) for c < d (round to nearest even); four columns per thread.
 __global__ void to_bf16_kernel(int64_t rows, int d4, const float* __restrict__ src, int64_t ld_src, int d,
                                uint16_t* __restrict__ dst, int64_t ld_dst) {
@@ -1016,7 +1067,7 @@ int pick_splits(int64_t tiles, int64_t slots, int64_t max_splits) {
 template <int KIND>
 mixgcn_status launch_kind(mixgcn_ctx* ctx, int ta, int tb, int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,
                           const void* B, int64_t ldb, float* C, int64_t ldc, const mixgcn_epilogue* epi, int64_t epi_row0,
-                          cudaStream_t s, uint16_t* C_lp, int64_t ldc_lp) {
+                          cudaStream_t s, uint16_t* C_lp, int64_t ldc_lp, float* colsum_b, bool* colsum_done) {
     using Cfg = KindCfg<KIND>;
     constexpr int EB = Cfg::EB, BK = Cfg::BK;
     constexpr int64_t LD_ALIGN = 16 / EB;           // TMA strides are multiples of 16 bytes
@@ -1189,12 +1240,17 @@ mixgcn_status launch_kind(mixgcn_ctx* ctx, int ta, int tb, int64_t M, int64_t N,
     if (stages_mm > 6) stages_mm = 6;
     p.stages = stages_mm;
     const size_t smem = (size_t)stages_mm * stage_mm + 1024;
+    // with fp32 words in shared memory (TF32 kind) the kernel also sums B's columns on request
+    const bool fuse_colsum = KIND == KIND_TF32 && colsum_b != nullptr;
+    const int64_t part_bytes = splits > 1 ? (((int64_t)splits * M * N * (int64_t)sizeof(float) + 255) & ~(int64_t)255) : 0;
+    const int64_t cs_bytes = fuse_colsum ? (int64_t)splits * N * (int64_t)sizeof(double) : 0;
+    if (part_bytes + cs_bytes > 0) MIXGCN_TRY(ensure_workspace(ctx, part_bytes + cs_bytes));
     if (splits > 1) {
-        MIXGCN_TRY(ensure_workspace(ctx, (int64_t)splits * M * N * (int64_t)sizeof(float)));
         p.C = reinterpret_cast<float*>(ctx->workspace); p.ldc = N; p.vec_c = (N & 3) == 0; p.raw = 1;
     } else {
         p.raw = 0;
     }
+    p.colsum_part = fuse_colsum ? reinterpret_cast<double*>(reinterpret_cast<char*>(ctx->workspace) + part_bytes) : nullptr;
     MIXGCN_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<KIND, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     {
         LaunchScope scope(ctx, PH_GEMM, s);
@@ -1202,6 +1258,12 @@ mixgcn_status launch_kind(mixgcn_ctx* ctx, int ta, int tb, int64_t M, int64_t N,
     }
     MIXGCN_CUDA(cudaGetLastError());
     if (splits > 1) MIXGCN_TRY(launch_splitk_reduce(ctx, M, N, splits, p.C, C, ldc, epi, s));
+    if (fuse_colsum) {
+        LaunchScope scope(ctx, PH_GEMM, s);
+        colsum_splits_kernel<<<(unsigned)((N + 127) / 128), 128, 0, s>>>(N, splits, p.colsum_part, colsum_b);
+        MIXGCN_CUDA(cudaGetLastError());
+        if (colsum_done) *colsum_done = true;
+    }
     return MIXGCN_OK;
 }
 
@@ -1214,13 +1276,17 @@ namespace mixgcn {
 //   kind 0 (TF32): A, and B in the MM form, are fp32 (lda, ldb in fp32 elements, multiples of 4);
 //   kind 1 (BF16): they are bf16 (lda, ldb in bf16 elements, multiples of 8).
 // In the KK form B is always the fp32 weight matrix (packed and converted here).  C_lp (KK form only,
-// nullable) receives a bf16 copy of C.
+// nullable) receives a bf16 copy of C.  colsum_b (nullable; weight-gradient form): where the kernel taken
+// can also produce the column sums of B (out[n] = sum_k B[k][n]) it does and sets *colsum_done; otherwise
+// the caller computes them.
 mixgcn_status launch_gemm_tc(mixgcn_ctx* ctx, int kind, int ta, int tb, int64_t M, int64_t N, int64_t K, const void* A,
                              int64_t lda, const void* B, int64_t ldb, float* C, int64_t ldc,
-                             const mixgcn_epilogue* epi, int64_t epi_row0, cudaStream_t s, uint16_t* C_lp, int64_t ldc_lp) {
+                             const mixgcn_epilogue* epi, int64_t epi_row0, cudaStream_t s, uint16_t* C_lp, int64_t ldc_lp,
+                             float* colsum_b, bool* colsum_done) {
+    if (colsum_done) *colsum_done = false;
     if (kind == KIND_BF16)
-        return launch_kind<KIND_BF16>(ctx, ta, tb, M, N, K, A, lda, B, ldb, C, ldc, epi, epi_row0, s, C_lp, ldc_lp);
-    return launch_kind<KIND_TF32>(ctx, ta, tb, M, N, K, A, lda, B, ldb, C, ldc, epi, epi_row0, s, C_lp, ldc_lp);
+        return launch_kind<KIND_BF16>(ctx, ta, tb, M, N, K, A, lda, B, ldb, C, ldc, epi, epi_row0, s, C_lp, ldc_lp, colsum_b, colsum_done);
+    return launch_kind<KIND_TF32>(ctx, ta, tb, M, N, K, A, lda, B, ldb, C, ldc, epi, epi_row0, s, C_lp, ldc_lp, colsum_b, colsum_done);
 }
 
 // dst (rows x ld_dst bf16, ld_dst a multiple of 4) = bf16(src (rows x ld_src fp32, 16-byte aligned, ld_src % 4 == 0)), columns < d

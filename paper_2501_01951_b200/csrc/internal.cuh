@@ -193,6 +193,9 @@ mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView&
 // schedule of all n rows of a view whose column ids lie in [0, n_cols); release of a view's memory
 mixgcn_status build_view_schedule(int64_t n_cols, int64_t n, CsrView& v, cudaStream_t s);
 void release_view(CsrView& v);
+// colsum_b of launch_gemm (weight-gradient form, trans_a = 1, only): also out[n] = sum_k B[k][n], the bias
+// gradient when B = dP -- produced inside the product's kernel where that kernel reads B as fp32 words,
+// by the column-sum kernels otherwise.
 // bf16 companions of one dense product (all nullable): copies of A and of B (the MM form's second
 // activation operand) that a producer already wrote, and a bf16 copy of C to write for the next product.
 // Leading dimensions in bf16 elements, multiples of 8; pointers 16-byte aligned.
@@ -203,13 +206,15 @@ struct GemmLP {
 };
 mixgcn_status launch_gemm(mixgcn_ctx* ctx, int precision, int ta, int tb, int64_t M, int64_t N, int64_t K,
                           const float* A, int64_t lda, const float* B, int64_t ldb, float* C, int64_t ldc,
-                          const mixgcn_epilogue* epi, int64_t epi_row0, cudaStream_t s, const GemmLP* lp = nullptr);
+                          const mixgcn_epilogue* epi, int64_t epi_row0, cudaStream_t s, const GemmLP* lp = nullptr,
+                          float* colsum_b = nullptr);
 mixgcn_status launch_gemm_simt(mixgcn_ctx* ctx, int ta, int tb, int64_t M, int64_t N, int64_t K,
                                const float* A, int64_t lda, const float* B, int64_t ldb, float* C, int64_t ldc,
                                const mixgcn_epilogue* epi, int64_t epi_row0, cudaStream_t s);
 mixgcn_status launch_gemm_tc(mixgcn_ctx* ctx, int kind, int ta, int tb, int64_t M, int64_t N, int64_t K, const void* A,
                              int64_t lda, const void* B, int64_t ldb, float* C, int64_t ldc,
-                             const mixgcn_epilogue* epi, int64_t epi_row0, cudaStream_t s, uint16_t* C_lp, int64_t ldc_lp);
+                             const mixgcn_epilogue* epi, int64_t epi_row0, cudaStream_t s, uint16_t* C_lp, int64_t ldc_lp,
+                             float* colsum_b = nullptr, bool* colsum_done = nullptr);
 mixgcn_status launch_splitk_reduce(mixgcn_ctx* ctx, int64_t M, int64_t N, int splits, const float* part, float* C,
                                    int64_t ldc, const mixgcn_epilogue* epi, cudaStream_t s);
 mixgcn_status launch_to_bf16(mixgcn_ctx* ctx, int64_t rows, int32_t d, const float* src, int64_t ld_src, uint16_t* dst,

@@ -449,6 +449,31 @@ def test_sampled_spmm_matches_eq4(mg, ctx, name, w, transposed):
     assert mg.ctx_poll_status(ctx, raise_on_error=False) == 0
 
 
+@pytest.mark.parametrize("d_in,d_out", [(64, 41), (128, 172), (40, 300), (130, 260)])
+@pytest.mark.parametrize("prec", ["tf32", "bf16", "fp32"])
+def test_bias_gradient_beside_the_weight_gradient(mg, ctx, d_in, d_out, prec):
+    """db = 1^T dP comes out of the weight-gradient product's kernel where that kernel reads dP as fp32 words
+    (TF32), from the column-sum kernels otherwise: either way it must be the column sum of the gradient the
+    call was given, to fp32 accuracy, whatever the width (tiles of 32-column chunks, ragged last chunk)."""
+    from helpers import TOL_LOWP
+    go, gg = build_both(mg, ctx, "hub")
+    n = go.n
+    X = synth.uniform_tensor((n, d_in), 611, -1, 1); W = synth.glorot_uniform(d_in, d_out, 612)
+    G = synth.uniform_tensor((n, d_out), 613, -1, 1) + 0.25           # column sums well away from zero
+    desc = mg.layer_desc(d_in, d_out, round4(d_in), round4(d_out), round4(d_in), mg.ORDER_AGG_FIRST, mg.PRECISIONS[prec], 0)
+    Xd, Wd = padded(X), W.cuda()
+    saved = torch.zeros(n, round4(d_in), device="cuda"); Xout = torch.zeros(n, round4(d_out), device="cuda")
+    mg.layer_fwd(ctx, gg, desc, Xd, Wd, None, None, saved, Xout)
+    Gd = padded(G, fill=float("nan")); Gin = torch.zeros(n, round4(d_in), device="cuda")
+    dW = torch.zeros(d_in, d_out, device="cuda"); db = torch.full((d_out,), 9.0, device="cuda")
+    mg.layer_bwd(ctx, gg, desc, Xd, saved, Xout, None, Wd, Gd, Gin, dW, db)
+    want_db = G.numpy().astype(np.float64).sum(axis=0)
+    assert rel_fro(db.cpu().numpy(), want_db) <= 1e-6
+    Z = orc.aggregate(go, X.numpy())
+    assert rel_fro(host(dW), Z.T @ G.numpy().astype(np.float64)) <= (TOL_FP32 if prec == "fp32" else TOL_LOWP)
+    assert mg.ctx_poll_status(ctx, raise_on_error=False) == 0
+
+
 def _tiny_problem():
     wl = synth.CONFIGS["C1"]
     s, d = synth.rmat_graph(wl.n, wl.undirected_edges, wl.seed("graph"))
