@@ -68,6 +68,7 @@ struct TcParams {
     int32_t* status;
     uint32_t wait_limit;    // polls after which a wait gives up
     int debug_drop_load;    // test hook: the producer leaves out the loads of its first stage (the wait on it then expires)
+    int epi_boxes;          // single-CTA K-major kernel: staging boxes per epilogue warp (1 or 2)
 };
 
 __device__ __forceinline__ float tc_apply_epi(const TcEpi& e, float y, int64_t m, int64_t n, int64_t N) {
@@ -413,7 +414,11 @@ __global__ void __launch_bounds__(KK_THREADS, 1) gemm_tc_kk_kernel(const __grid_
         const bool wide_bias = post && p.epi.bias != nullptr && !bias_in_smem;
         const bool add_bias = p.epi.bias != nullptr && bias_in_smem, relu = p.epi.relu != 0;
         const bool gate_vec = p.epi.gate != nullptr && aligned16_dev(p.epi.gate) && (p.epi.ld_gate & 3) == 0;
-        uint8_t* box = smem_out + (size_t)warp * 4096;
+        // one staging box per warp, or two (short K: the epilogue is the critical path, and the second box is
+        // filled while the TMA store of the first is still reading it)
+        const int nboxes = p.epi_boxes;
+        uint8_t* const box_base = smem_out + (size_t)warp * nboxes * 4096;
+        uint32_t box_turn = 0;
         uint32_t j = 0;
         bool ok = true;
         for (int64_t tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x, ++j) {
@@ -476,7 +481,11 @@ __global__ void __launch_bounds__(KK_THREADS, 1) gemm_tc_kk_kernel(const __grid_
                 if (tma_store) {
                     // rows of 128 bytes in the 128-byte swizzle the tensor map expects: 16-byte chunk q of row r
                     // lives at chunk position q ^ (r & 7).  The box is clipped to the matrix by the TMA unit.
-                    if (lane == 0) bulk_wait_read<0>();          // the store that last used this box has read it
+                    uint8_t* const box = box_base + (nboxes == 2 ? (box_turn & 1u) * 4096 : 0);
+                    ++box_turn;
+                    if (lane == 0) {                             // the store that last used this box has read it
+                        if (nboxes == 2) bulk_wait_read<1>(); else bulk_wait_read<0>();
+                    }
                     __syncwarp();
 #pragma unroll
                     for (int q = 0; q < 8; ++q)
@@ -1162,12 +1171,16 @@ mixgcn_status launch_kind(mixgcn_ctx* ctx, int ta, int tb, int64_t M, int64_t N,
         const size_t b_all = (size_t)nk * bn32 * 128;
         const int b_resident = (p.n_tiles == 1 && b_all <= 96 * 1024) ? 1 : 0;
         const size_t stage = TC_BM * 128 + (b_resident ? 0 : (size_t)bn32 * 128);
-        const size_t budget = (b_resident ? 168 * 1024 - b_all : 160 * 1024);
+        // short K (one or two stages per tile): the tensor core is idle most of the time and the epilogue is
+        // the critical path -- it gets a second staging box per warp out of the ring's budget
+        p.epi_boxes = nk <= 2 ? 2 : 1;
+        const size_t box_bytes = (size_t)KK_EPI_WARPS * p.epi_boxes * 4096;
+        const size_t budget = (b_resident ? 200 * 1024 - b_all : 192 * 1024) - box_bytes;
         int stages = (int)(budget / stage);
         if (stages > 8) stages = 8;
         if (stages < 2) stages = 2;
         p.stages = stages;
-        const size_t smem_kk = (b_resident ? b_all : 0) + (size_t)stages * stage + 8 * 4096 + 1024;
+        const size_t smem_kk = (b_resident ? b_all : 0) + (size_t)stages * stage + box_bytes + 1024;
         const int tma_store = p.vec_c ? 1 : 0;
         CUtensorMap map_c = map_a;
         if (tma_store && !encode_2d(&map_c, C, 4, N, M, ldc, 32, 32)) return MIXGCN_EUNSUPPORTED;
