@@ -288,6 +288,15 @@ mixgcn_status mixgcn_gemm(mixgcn_ctx* ctx, int32_t precision, int32_t trans_a, i
                                        same features every epoch, and the first layer's backward
                                        leaves `saved` intact): the aggregation is skipped.  Not in
                                        the paper, which recomputes it every iteration. */
+#define MIXGCN_LAYER_SAVED_LP_ONLY 128u /* agg-first order with MIXGCN_PREC_BF16 and a saved_lp companion: the
+                                       forward writes A_hat X_in to saved_lp ONLY -- both products that read it
+                                       (the update and, in the backward, the weight gradient) read the bf16
+                                       copy anyway, so the fp32 copy is a write nobody reads.  `saved` (fp32) is
+                                       then left unchanged by the forward; the backward still uses it as scratch
+                                       and must be given the same flag and saved_lp.  Not with n_chunks > 1, a
+                                       row-sparse backward (gout_row_mask / gout_plan), OUT_ROWS_ONLY or
+                                       SAVED_IS_VALID; MIXGCN_EUNSUPPORTED if the BF16 kernels cannot take the
+                                       shape (there is then no fp32 operand to fall back on). */
 #define MIXGCN_LAYER_GIN_ROWS_ONLY 32u /* backward with gout_plan: write only the rows of G_in in the
                                        plan's out_row_mask (the other rows are exactly zero and
                                        are left unchanged) */

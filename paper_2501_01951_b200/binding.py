@@ -29,6 +29,7 @@ PREC_FP32, PREC_TF32, PREC_BF16 = 0, 1, 2
 ORDER_AUTO, ORDER_AGG_FIRST, ORDER_UPD_FIRST = 0, 1, 2
 LAYER_RELU, LAYER_FIRST, LAYER_GATE_GIN, LAYER_GOUT_GATED, LAYER_OUT_ROWS_ONLY, LAYER_GIN_ROWS_ONLY = 1, 2, 4, 8, 16, 32
 LAYER_SAVED_IS_VALID = 64
+LAYER_SAVED_LP_ONLY = 128
 N_PHASES = 7
 PHASES = ("spmm", "gemm", "elementwise", "loss", "adam", "graph", "spmm_sparse")
 PRECISIONS = {"fp32": PREC_FP32, "tf32": PREC_TF32, "bf16": PREC_BF16}

@@ -137,6 +137,8 @@ mixgcn_status launch_gemm(mixgcn_ctx* ctx, int precision, int ta, int tb, int64_
                             C, ldc, epi, epi_row0, s, ta ? nullptr : c_lp, ldc_lp);
         if (st == MIXGCN_OK) { ctx->gemm_path[2]++; c_lp_done = !ta && c_lp; }
     }
+    if (st == MIXGCN_EUNSUPPORTED && lp && lp->a_fp32_missing)
+        MIXGCN_FAIL(MIXGCN_EUNSUPPORTED, "gemm: the bf16 kernels cannot take this product and its fp32 operand was not kept (SAVED_LP_ONLY)");
     bool colsum_done = false;
     if (colsum_b && !ta) MIXGCN_FAIL(MIXGCN_EINVAL, "gemm: column sums of B are a by-product of the weight-gradient form only");
     if (st == MIXGCN_EUNSUPPORTED && precision != MIXGCN_PREC_FP32) {
@@ -346,6 +348,11 @@ mixgcn_status check_desc(const mixgcn_layer_desc* d, const char* who) {
     if (!lp_ok(d->saved_lp, d->ld_saved_lp, saved_cols) || !lp_ok(d->x_in_lp, d->ld_in_lp, d->d_in) || !lp_ok(d->g_in_lp, d->ld_in_lp, d->d_in) ||
         !lp_ok(d->x_out_lp, d->ld_out_lp, d->d_out) || !lp_ok(d->g_out_lp, d->ld_out_lp, d->d_out))
         MIXGCN_FAIL(MIXGCN_EINVAL, "%s: bf16 companions must be 16-byte aligned with leading dimensions that are multiples of 8 and cover the width", who);
+    if (d->flags & MIXGCN_LAYER_SAVED_LP_ONLY) {
+        if (order != MIXGCN_ORDER_AGG_FIRST || d->precision != MIXGCN_PREC_BF16 || !d->saved_lp || d->n_chunks > 1 ||
+            d->gout_row_mask || d->gout_plan || (d->flags & (MIXGCN_LAYER_OUT_ROWS_ONLY | MIXGCN_LAYER_SAVED_IS_VALID)))
+            MIXGCN_FAIL(MIXGCN_EINVAL, "%s: SAVED_LP_ONLY needs agg-first order, BF16 products, saved_lp, one chunk and a dense backward", who);
+    }
     return MIXGCN_OK;
 }
 
@@ -444,9 +451,10 @@ extern "C" mixgcn_status mixgcn_layer_fwd(mixgcn_ctx* ctx, const mixgcn_graph* g
     if (order == MIXGCN_ORDER_AGG_FIRST) {
         SpmmOpts agg_opts; agg_opts.Z_lp = lp.saved; agg_opts.ldz_lp = lp.ld_saved;     // the aggregation also writes bf16(A_hat X)
         if (chunks == 1) {
+            const bool lp_only = (d->flags & MIXGCN_LAYER_SAVED_LP_ONLY) != 0;
             if (!saved_valid)
-                MIXGCN_TRY(launch_spmm(ctx, g, g->fwd, 1, 0, d->d_in, X_in, d->ld_in, saved, d->ld_saved, nullptr, s, agg_opts));
-            GemmLP glp; glp.A = lp.saved; glp.lda = lp.ld_saved; glp.C = lp.x_out; glp.ldc = lp.ld_out;
+                MIXGCN_TRY(launch_spmm(ctx, g, g->fwd, 1, 0, d->d_in, X_in, d->ld_in, lp_only ? nullptr : saved, d->ld_saved, nullptr, s, agg_opts));
+            GemmLP glp; glp.A = lp.saved; glp.lda = lp.ld_saved; glp.C = lp.x_out; glp.ldc = lp.ld_out; glp.a_fp32_missing = lp_only;
             MIXGCN_TRY(launch_gemm(ctx, d->precision, 0, 0, n, d->d_out, d->d_in, saved, d->ld_saved, W, ldw, X_out,
                                    d->ld_out, &epi, 0, s, &glp));
             return MIXGCN_OK;
@@ -586,6 +594,7 @@ extern "C" mixgcn_status mixgcn_layer_bwd(mixgcn_ctx* ctx, const mixgcn_graph* g
         // dW = (A_hat X_in)^T dP ; dZ = dP W^T (over `saved`) ; G_in = A_hat^T dZ
         // dW = (A_hat X_in)^T dP, and db = 1^T dP as its by-product
         GemmLP wlp; wlp.A = lp.saved; wlp.lda = lp.ld_saved; wlp.B = lp.g_out; wlp.ldb = lp.ld_out;
+        wlp.a_fp32_missing = (d->flags & MIXGCN_LAYER_SAVED_LP_ONLY) != 0;
         MIXGCN_TRY(launch_gemm(ctx, d->precision, 1, 0, d->d_in, d->d_out, n, saved, d->ld_saved, G_out, d->ld_out, dW,
                                ldw, nullptr, 0, s, &wlp, dbias));
         if (!first) {

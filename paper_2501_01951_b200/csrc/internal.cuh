@@ -200,6 +200,7 @@ void release_view(CsrView& v);
 // activation operand) that a producer already wrote, and a bf16 copy of C to write for the next product.
 // Leading dimensions in bf16 elements, multiples of 8; pointers 16-byte aligned.
 struct GemmLP {
+    bool a_fp32_missing = false;      // the fp32 A holds no data (only its bf16 copy was written): no fallback below bf16
     const uint16_t* A = nullptr; int64_t lda = 0;
     const uint16_t* B = nullptr; int64_t ldb = 0;
     uint16_t* C = nullptr; int64_t ldc = 0;

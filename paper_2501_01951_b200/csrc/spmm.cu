@@ -90,7 +90,7 @@ __device__ __forceinline__ void store_row(const SpmmParams& p, int64_t u, int c4
     if (!p.bias && !p.residual && a.x == 0.0f && a.y == 0.0f && a.z == 0.0f && a.w == 0.0f) {
         // ReLU, dropout and the gate all map 0 to 0: no mask or gate byte needs to be read (the empty
         // rows of a row-sparse aggregation take this path)
-        *reinterpret_cast<float4*>(p.Z + u * p.ldz + j) = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (p.Z) *reinterpret_cast<float4*>(p.Z + u * p.ldz + j) = make_float4(0.f, 0.f, 0.f, 0.f);
         if (p.Z_lp) *reinterpret_cast<uint2*>(p.Z_lp + u * p.ldz_lp + j) = make_uint2(0u, 0u);
         return;
     }
@@ -101,7 +101,7 @@ __device__ __forceinline__ void store_row(const SpmmParams& p, int64_t u, int c4
 #pragma unroll
         for (int t = 0; t < 4; ++t) r[t] = ((nib >> t) & 1u) ? r[t] : 0.0f;
     }
-    *reinterpret_cast<float4*>(p.Z + u * p.ldz + j) = make_float4(r[0], r[1], r[2], r[3]);
+    if (p.Z) *reinterpret_cast<float4*>(p.Z + u * p.ldz + j) = make_float4(r[0], r[1], r[2], r[3]);   // null: bf16 copy only
     if (p.Z_lp) store_lp4(p.Z_lp + u * p.ldz_lp + j, r[0], r[1], r[2], r[3]);
 }
 
@@ -497,6 +497,7 @@ mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView&
     const int phase = opts.phase;
     const int64_t row_limit = opts.row_limit;
     if (w <= 0) return MIXGCN_OK;
+    if (!Z && !opts.Z_lp) MIXGCN_FAIL(MIXGCN_EINVAL, "spmm: no output");
     if (sparse && row_filter) MIXGCN_FAIL(MIXGCN_EUNSUPPORTED, "spmm: a row filter cannot be combined with a row-sparse input");
     if (chunks > 1) {
         MIXGCN_TRY(ensure_chunk_schedules(g, A, chunks));

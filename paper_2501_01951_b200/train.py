@@ -23,7 +23,7 @@ def round8(x: int) -> int:
 class GcnTrainer:
     def __init__(self, ctx: mg.Ctx, graph: mg.Graph, dims, precision=mg.PREC_FP32, order=mg.ORDER_AUTO,
                  n_chunks=0, fuse_gate=True, keep_scale=1.0, device=None, row_sparse="auto",
-                 train_rows_only=False, row_plans=True, cache_first_aggregation=False, lp_copies=True):
+                 train_rows_only=False, row_plans=True, cache_first_aggregation=False, lp_copies=True, saved_lp_only=True):
         self.ctx, self.g = ctx, graph
         self.dims = tuple(int(d) for d in dims)
         self.L = len(self.dims) - 1
@@ -82,6 +82,10 @@ class GcnTrainer:
         # BF16 products: bf16 companions of the activations, written by the kernels that produce them
         # (buffers only; lp_copies=False leaves them out and the library converts operands on the fly)
         self.lp = []
+        self.saved_lp = [None] * L       # bf16 copy of saved[l], where there is one
+        # with bf16 companions an agg-first layer's A_hat X is read only as bf16: its fp32 copy need not be written
+        # (set per iteration in forward(): only where the backward is dense and nothing else reads `saved`)
+        self.saved_lp_only = bool(saved_lp_only) and precision == mg.PREC_BF16 and lp_copies and n_chunks <= 1
         if precision == mg.PREC_BF16 and lp_copies:
             zb = lambda c: torch.zeros((n, round8(c)), dtype=torch.bfloat16, device=self.device)
             keep = lambda t: (self.lp.append(t), t)[1]
@@ -95,6 +99,7 @@ class GcnTrainer:
             for l, d in enumerate(self.descs):
                 cols = self.dims[l] if self.orders[l] == mg.ORDER_AGG_FIRST else self.dims[l + 1]
                 t = keep(zb(cols))
+                self.saved_lp[l] = t
                 d.saved_lp, d.ld_saved_lp = t.data_ptr(), t.stride(0)
                 d.ld_in_lp, d.ld_out_lp = round8(self.dims[l]), round8(self.dims[l + 1])
                 if x_lp[l] is not None:
@@ -197,10 +202,20 @@ class GcnTrainer:
         reuse = self.cache_first_aggregation and self._first_aggregation_valid and self.orders[0] == mg.ORDER_AGG_FIRST
         d0.flags = (d0.flags | mg.LAYER_SAVED_IS_VALID) if reuse else (d0.flags & ~mg.LAYER_SAVED_IS_VALID)
         for l in range(self.L):
-            mg.layer_fwd(self.ctx, self.g, self.descs[l], self.X[l], self.W[l], self.b[l], self.masks[l],
+            d = self.descs[l]
+            lp_only = (self.saved_lp_only and self.orders[l] == mg.ORDER_AGG_FIRST and not d.gout_row_mask and not d.gout_plan
+                       and not (d.flags & (mg.LAYER_OUT_ROWS_ONLY | mg.LAYER_SAVED_IS_VALID))
+                       and not (l == 0 and self.cache_first_aggregation))
+            d.flags = (d.flags | mg.LAYER_SAVED_LP_ONLY) if lp_only else (d.flags & ~mg.LAYER_SAVED_LP_ONLY)
+            mg.layer_fwd(self.ctx, self.g, d, self.X[l], self.W[l], self.b[l], self.masks[l],
                          self.saved[l], self.X[l + 1])
         # saved[0] now holds A_hat X^(0) unless the single layer of a one-layer model also restricted it to train rows
         self._first_aggregation_valid = self.orders[0] == mg.ORDER_AGG_FIRST and not (d0.flags & mg.LAYER_OUT_ROWS_ONLY)
+
+    def aggregation_of(self, l):
+        """The tensor that holds A_hat X^(l) after forward() for an agg-first layer: `saved[l]`, or its bf16
+        copy where only that was written."""
+        return self.saved_lp[l] if self.descs[l].flags & mg.LAYER_SAVED_LP_ONLY else self.saved[l]
 
     def compute_loss(self):
         if self.train_rows_only:

@@ -778,6 +778,48 @@ def test_training_epoch_bf16_within_low_precision_bound(mg, ctx, orders, lp_copi
     gg.close()
 
 
+def test_bf16_layer_keeps_only_the_bf16_copy_of_the_aggregation(mg, ctx):
+    """SAVED_LP_ONLY: the forward leaves the fp32 `saved` alone (both products read the bf16 copy), the
+    results are the bits of the run that writes both, and the flag is refused where something reads fp32."""
+    from paper_2501_01951_b200.train import GcnTrainer
+    wl, s, d, X, y, m, Ws, bs = _tiny_problem()
+    gg = mg.graph_create(ctx, wl.n, s, d)
+    outs = []
+    for only in (True, False):
+        tr = GcnTrainer(ctx, gg, wl.dims, mg.PREC_BF16, order=mg.ORDER_AGG_FIRST, row_sparse=0, saved_lp_only=only)
+        tr.set_params(Ws, bs)
+        tr.set_inputs(padded(X), y.cuda(), m.cuda())
+        for sv in tr.saved:
+            sv.fill_(7.0)
+        tr.forward()
+        for l, sv in enumerate(tr.saved):
+            assert bool(tr.descs[l].flags & mg.LAYER_SAVED_LP_ONLY) == only
+            assert bool(torch.all(sv == 7.0)) == only
+        logits = tr.X[-1].clone()
+        tr.compute_loss(); tr.backward()
+        outs.append([logits] + [w.clone() for w in tr.dW] + [b.clone() for b in tr.db])
+    for a, b in zip(*outs):
+        assert torch.equal(a, b)
+    # refused: fp32 products, and a row-sparse backward (which gathers fp32 rows of `saved`)
+    tr = GcnTrainer(ctx, gg, wl.dims, mg.PREC_BF16, order=mg.ORDER_AGG_FIRST, row_sparse=0)
+    tr.set_params(Ws, bs)
+    tr.set_inputs(padded(X), y.cuda(), m.cuda())
+    dsc = tr.descs[0]
+    for change in ("precision", "row_mask"):
+        keep = (dsc.precision, dsc.gout_row_mask)
+        dsc.flags |= mg.LAYER_SAVED_LP_ONLY
+        if change == "precision":
+            dsc.precision = mg.PREC_TF32
+        else:
+            dsc.gout_row_mask = tr.train_mask.data_ptr()
+        with pytest.raises(mg.MixgcnError) as e:
+            mg.layer_fwd(ctx, gg, dsc, tr.X[0], tr.W[0], tr.b[0], None, tr.saved[0], tr.X[1])
+        assert e.value.status == mg.EINVAL
+        dsc.precision, dsc.gout_row_mask = keep
+    assert mg.ctx_poll_status(ctx, raise_on_error=False) == 0
+    gg.close()
+
+
 PAIR_SHAPES = [(4096, 512, 512), (5000, 1024, 520), (4100, 600, 1000), (8191, 777, 513)]   # M, N, K: ragged in every dimension
 
 
