@@ -65,8 +65,21 @@ mixgcn_status mixgcn_ctx_reserve(mixgcn_ctx* ctx, int64_t bytes);
 /* Synchronises the context's device, reads and clears the device status word.
  * Returns MIXGCN_OK, MIXGCN_EDEVICE or MIXGCN_ETIMEOUT; *code (nullable) receives the raw
  * code: 0 none, 1 empty train mask, 2 label out of range, 3 bounded wait expired,
- * 4 gout_row_count does not match gout_row_mask. */
+ * 4 gout_row_count does not match gout_row_mask, 5 (bounds-checked debug build only) a kernel met an index
+ * outside its range -- mixgcn_last_error() then names the kind of index and its value. */
 mixgcn_status mixgcn_ctx_poll_status(mixgcn_ctx* ctx, int32_t* code);
+
+/* The bounds-checked debug build (libmixgcn_debug.so: the same sources compiled with -DMIXGCN_DEBUG_BOUNDS; no
+ * counterpart in the paper -- it stands in for a memory checker).  Every index a kernel takes from memory -- an
+ * aggregation's column ids, the rows and entry ranges of its schedule records, its segment tables, the row lists
+ * of the row-sparse backward -- is tested before it addresses anything; a bad one is recorded (code 5 above), the
+ * access is skipped, the kernel finishes and the context stays usable.  The release build has none of these tests.
+ * mixgcn_build_info: *debug_bounds (nullable) receives 1 in that build, 0 otherwise.
+ * mixgcn_debug_poke_col: the test hook of those checks, MIXGCN_EUNSUPPORTED in the release build: synchronises the
+ * device and overwrites column id `entry` (in [0, nnz), else MIXGCN_EINVAL) of the graph's forward CSR with
+ * `value`; *old_value (nullable, host) receives what was there. */
+mixgcn_status mixgcn_build_info(int32_t* debug_bounds);
+mixgcn_status mixgcn_debug_poke_col(mixgcn_graph* g, int64_t entry, int32_t value, int32_t* old_value);
 
 /* Tuning options.  MIXGCN_OPT_SPMM_SLICE_COLS: width of the feature-column slices an aggregation is
  * processed in (Algorithm 2's p:q-1 column ranges on one GPU): 0 = slices of 256 columns (default:

@@ -13,7 +13,11 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libmixgcn.so")
+# MIXGCN_LIBRARY=debug loads the bounds-checked build of the same sources (libmixgcn_debug.so) instead
+_VARIANT = os.environ.get("MIXGCN_LIBRARY", "")
+if _VARIANT not in ("", "debug"):
+    raise ImportError(f"MIXGCN_LIBRARY={_VARIANT!r}: the only other build is 'debug'")
+LIB_PATH = os.path.join(_HERE, "libmixgcn_debug.so" if _VARIANT == "debug" else "libmixgcn.so")
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(
@@ -46,6 +50,7 @@ SYMBOLS = (
     "mixgcn_count_rows", "mixgcn_rowplan_create", "mixgcn_rowplan_destroy", "mixgcn_rowplan_info",
     "mixgcn_rowplan_export", "mixgcn_spmm_rowplan", "mixgcn_colsum", "mixgcn_ctx_gemm_paths",
     "mixgcn_train_step_host_prefetch", "mixgcn_probe_gather", "mixgcn_spmm_sampled", "mixgcn_mask_pack",
+    "mixgcn_build_info", "mixgcn_debug_poke_col",
 )
 
 
@@ -245,6 +250,20 @@ def graph_export_schedule(g: Graph, transposed: bool = False) -> torch.Tensor:
     perm = torch.empty(g.n, dtype=torch.int32)
     _check(lib.mixgcn_graph_export_schedule(g.h, C.c_int(int(transposed)), _ptr(perm)))
     return perm
+
+
+def build_info() -> dict:
+    """Which build of the library is loaded: {"debug_bounds": bool}."""
+    flag = C.c_int32(0)
+    _check(lib.mixgcn_build_info(C.byref(flag)))
+    return {"debug_bounds": bool(flag.value)}
+
+
+def debug_poke_col(g: Graph, entry: int, value: int) -> int:
+    """Bounds-checked debug build only: overwrite one column id of the forward CSR; returns the old one."""
+    old = C.c_int32(0)
+    _check(lib.mixgcn_debug_poke_col(g.h, C.c_int64(entry), C.c_int32(value), C.byref(old)))
+    return old.value
 
 
 def graph_bandwidth(g: Graph, order: torch.Tensor | None = None) -> int:

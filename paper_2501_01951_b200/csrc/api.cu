@@ -231,13 +231,36 @@ extern "C" mixgcn_status mixgcn_ctx_poll_status(mixgcn_ctx* ctx, int32_t* code) 
     if (!ctx) MIXGCN_FAIL(MIXGCN_EINVAL, "ctx_poll_status: null ctx");
     MIXGCN_CUDA(cudaSetDevice(ctx->device));
     MIXGCN_CUDA(cudaDeviceSynchronize());
-    int32_t h = 0;
-    MIXGCN_CUDA(cudaMemcpy(&h, ctx->d_status, sizeof(h), cudaMemcpyDeviceToHost));
-    MIXGCN_CUDA(cudaMemset(ctx->d_status, 0, sizeof(int32_t)));
+    int32_t w[4] = {0, 0, 0, 0};
+    MIXGCN_CUDA(cudaMemcpy(w, ctx->d_status, sizeof(w), cudaMemcpyDeviceToHost));
+    MIXGCN_CUDA(cudaMemset(ctx->d_status, 0, sizeof(w)));
+    const int32_t h = w[0];
     if (code) *code = h;
     if (h == DEV_OK) return MIXGCN_OK;
+    if (h == DEV_BAD_INDEX) {
+        static const char* const sites[] = {"?", "aggregation: column id", "aggregation: row of a schedule record", "aggregation: entry range of a schedule record",
+                                            "aggregation: position of a kept row", "aggregation: segment table", "row list of a gather / scatter"};
+        const int site = w[1] >= 1 && w[1] <= 6 ? w[1] : 0;
+        const long long value = (long long)(((uint64_t)(uint32_t)w[3] << 32) | (uint32_t)w[2]);
+        MIXGCN_FAIL(MIXGCN_EDEVICE, "bounds-checked build: index out of range (%s, value %lld); the access was skipped", sites[site], value);
+    }
     if (h == DEV_WAIT_EXPIRED) MIXGCN_FAIL(MIXGCN_ETIMEOUT, "a bounded device-side wait expired");
     MIXGCN_FAIL(MIXGCN_EDEVICE, h == DEV_EMPTY_MASK ? "loss: the train mask is empty" : h == DEV_BAD_LABEL ? "loss: a label lies outside [0, C)" : "layer_bwd: gout_row_count does not match gout_row_mask");
+}
+
+extern "C" mixgcn_status mixgcn_build_info(int32_t* debug_bounds) {
+    if (debug_bounds) *debug_bounds = DEBUG_BOUNDS ? 1 : 0;
+    return MIXGCN_OK;
+}
+
+extern "C" mixgcn_status mixgcn_debug_poke_col(mixgcn_graph* g, int64_t entry, int32_t value, int32_t* old_value) {
+    if (!DEBUG_BOUNDS) MIXGCN_FAIL(MIXGCN_EUNSUPPORTED, "debug_poke_col: this is not the bounds-checked debug build");
+    if (!g || entry < 0 || entry >= g->nnz) MIXGCN_FAIL(MIXGCN_EINVAL, "debug_poke_col: entry outside [0, nnz)");
+    MIXGCN_CUDA(cudaSetDevice(g->device));
+    MIXGCN_CUDA(cudaDeviceSynchronize());
+    if (old_value) MIXGCN_CUDA(cudaMemcpy(old_value, g->fwd.col + entry, sizeof(int32_t), cudaMemcpyDeviceToHost));
+    MIXGCN_CUDA(cudaMemcpy(g->fwd.col + entry, &value, sizeof(int32_t), cudaMemcpyHostToDevice));
+    return MIXGCN_OK;
 }
 
 extern "C" mixgcn_status mixgcn_ctx_set_option(mixgcn_ctx* ctx, int32_t option, int64_t value) {
@@ -436,9 +459,9 @@ extern "C" mixgcn_status mixgcn_layer_fwd(mixgcn_ctx* ctx, const mixgcn_graph* g
             RowSet rs;
             const int64_t lda = (d->d_in + 3) / 4 * 4, ldb = (d->d_out + 3) / 4 * 4;
             MIXGCN_TRY(build_row_set(ctx, n, rows, cnt, lda, ldb, &rs, s));
-            MIXGCN_TRY(launch_gather_rows(ctx, cnt, d->d_in, rs.idx, saved, d->ld_saved, rs.a, lda, s));
+            MIXGCN_TRY(launch_gather_rows(ctx, n, cnt, d->d_in, rs.idx, saved, d->ld_saved, rs.a, lda, s));
             MIXGCN_TRY(launch_gemm(ctx, d->precision, 0, 0, cnt, d->d_out, d->d_in, rs.a, lda, W, ldw, rs.b, ldb, &epi, 0, s));
-            MIXGCN_TRY(launch_scatter_rows(ctx, cnt, d->d_out, rs.idx, rs.b, ldb, X_out, d->ld_out, s));
+            MIXGCN_TRY(launch_scatter_rows(ctx, n, cnt, d->d_out, rs.idx, rs.b, ldb, X_out, d->ld_out, s));
             return MIXGCN_OK;
         }
         MIXGCN_TRY(launch_gemm(ctx, d->precision, 0, 0, n, d->d_out, d->d_in, X_in, d->ld_in, W, ldw, saved, d->ld_saved,
@@ -541,12 +564,13 @@ extern "C" mixgcn_status mixgcn_layer_bwd(mixgcn_ctx* ctx, const mixgcn_graph* g
         float* cb = reinterpret_cast<float*>(reinterpret_cast<char*>(ctx->workspace_rows) + up(rows_alloc * lda * 4));
         // rows of the restricted matrix are scheduled longest first: its non-empty rows are the first out_count
         SpmmOpts plan_all; plan_all.phase = PH_SPMM_SPARSE;
+        plan_all.y_rows = cnt; plan_all.nnz = plan->nnz;          // the restricted matrix gathers from the compacted rows
         SpmmOpts plan_opts = plan_all; plan_opts.row_limit = (d->flags & MIXGCN_LAYER_GIN_ROWS_ONLY) ? plan->out_count : -1;
         plan_opts.Z_lp = lp.g_in; plan_opts.ldz_lp = lp.ld_in;
         plan_all.Z_lp = lp.saved; plan_all.ldz_lp = lp.ld_saved;
-        MIXGCN_TRY(launch_gather_rows(ctx, cnt, d->d_out, plan->idx, G_out, d->ld_out, cb, ldb, s));         // dP_T
+        MIXGCN_TRY(launch_gather_rows(ctx, n, cnt, d->d_out, plan->idx, G_out, d->ld_out, cb, ldb, s));         // dP_T
         if (order == MIXGCN_ORDER_AGG_FIRST) {
-            MIXGCN_TRY(launch_gather_rows(ctx, cnt, d->d_in, plan->idx, saved, d->ld_saved, ca, lda, s));     // Z_T
+            MIXGCN_TRY(launch_gather_rows(ctx, n, cnt, d->d_in, plan->idx, saved, d->ld_saved, ca, lda, s));     // Z_T
             // dW = Z_T^T dP_T, and db = 1^T dP_T as its by-product
             MIXGCN_TRY(launch_gemm(ctx, d->precision, 1, 0, d->d_in, d->d_out, cnt, ca, lda, cb, ldb, dW, ldw, nullptr, 0, s, nullptr, dbias));
             if (!first) {
@@ -581,12 +605,13 @@ extern "C" mixgcn_status mixgcn_layer_bwd(mixgcn_ctx* ctx, const mixgcn_graph* g
             RowSet rs;
             const int64_t lda = (d->d_in + 3) / 4 * 4, ldb = (d->d_out + 3) / 4 * 4;
             MIXGCN_TRY(build_row_set(ctx, n, rmask, cnt, lda, ldb, &rs, s));
-            MIXGCN_TRY(launch_gather_rows(ctx, cnt, d->d_in, rs.idx, saved, d->ld_saved, rs.a, lda, s));     // Z_T
-            MIXGCN_TRY(launch_gather_rows(ctx, cnt, d->d_out, rs.idx, G_out, d->ld_out, rs.b, ldb, s));      // dP_T
+            MIXGCN_TRY(launch_gather_rows(ctx, n, cnt, d->d_in, rs.idx, saved, d->ld_saved, rs.a, lda, s));     // Z_T
+            MIXGCN_TRY(launch_gather_rows(ctx, n, cnt, d->d_out, rs.idx, G_out, d->ld_out, rs.b, ldb, s));      // dP_T
             MIXGCN_TRY(launch_gemm(ctx, d->precision, 1, 0, d->d_in, d->d_out, cnt, rs.a, lda, rs.b, ldb, dW, ldw, nullptr, 0, s, nullptr, dbias));
             if (!first) {
                 MIXGCN_TRY(launch_gemm(ctx, d->precision, 0, 1, cnt, d->d_in, d->d_out, rs.b, ldb, W, ldw, rs.a, lda, nullptr, 0, s));
                 sp.in_pos = rs.pos;                                                                             // dZ_T is compact
+                gin_opts.y_rows = cnt;
                 MIXGCN_TRY(launch_spmm(ctx, g, g->bwd, 1, 0, d->d_in, rs.a, lda, G_in, d->ld_in, gin, s, gin_opts));
             }
             return MIXGCN_OK;
@@ -616,7 +641,7 @@ extern "C" mixgcn_status mixgcn_layer_bwd(mixgcn_ctx* ctx, const mixgcn_graph* g
             RowSet rs;
             const int64_t ldb = (d->d_out + 3) / 4 * 4;
             MIXGCN_TRY(build_row_set(ctx, n, rmask, cnt, 4, ldb, &rs, s));
-            MIXGCN_TRY(launch_gather_rows(ctx, cnt, d->d_out, rs.idx, G_out, d->ld_out, rs.b, ldb, s));
+            MIXGCN_TRY(launch_gather_rows(ctx, n, cnt, d->d_out, rs.idx, G_out, d->ld_out, rs.b, ldb, s));
             MIXGCN_TRY(launch_colsum(ctx, cnt, d->d_out, rs.b, ldb, dbias, s));
         }
     } else if (dbias) {

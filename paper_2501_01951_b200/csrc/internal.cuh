@@ -35,7 +35,32 @@ void set_error(const char* fmt, ...);
 enum Phase { PH_SPMM = 0, PH_GEMM = 1, PH_ELEM = 2, PH_LOSS = 3, PH_ADAM = 4, PH_GRAPH = 5, PH_SPMM_SPARSE = 6 };
 
 // device status word codes
-enum { DEV_OK = 0, DEV_EMPTY_MASK = 1, DEV_BAD_LABEL = 2, DEV_WAIT_EXPIRED = 3, DEV_BAD_ROW_COUNT = 4 };
+enum { DEV_OK = 0, DEV_EMPTY_MASK = 1, DEV_BAD_LABEL = 2, DEV_WAIT_EXPIRED = 3, DEV_BAD_ROW_COUNT = 4, DEV_BAD_INDEX = 5 };
+
+// Bounds-checked debug build (-DMIXGCN_DEBUG_BOUNDS): every index a kernel takes FROM MEMORY (a column id, a
+// schedule record's row and entry range, a segment table, a row list) is tested before it addresses anything.
+// A bad one is recorded in the status word (code DEV_BAD_INDEX, the site in word 1, the value in words 2-3;
+// the first report wins) and the access is skipped, so the kernel finishes and the context stays usable.
+// The release build compiles these tests away.
+#ifdef MIXGCN_DEBUG_BOUNDS
+constexpr bool DEBUG_BOUNDS = true;
+#else
+constexpr bool DEBUG_BOUNDS = false;
+#endif
+enum { SITE_SPMM_COL = 1, SITE_SPMM_ROW = 2, SITE_SPMM_RANGE = 3, SITE_SPMM_POS = 4, SITE_SPMM_SEG = 5, SITE_ROW_LIST = 6 };
+#ifdef __CUDACC__
+__device__ __forceinline__ bool index_ok(int64_t i, int64_t limit, int32_t* status, int site) {
+    if constexpr (DEBUG_BOUNDS) {
+        if (i < 0 || i >= limit) {
+            if (atomicCAS(status, DEV_OK, DEV_BAD_INDEX) == DEV_OK) {
+                status[1] = site; status[2] = (int32_t)(uint32_t)i; status[3] = (int32_t)(i >> 32);
+            }
+            return false;
+        }
+    }
+    return true;
+}
+#endif
 
 struct ProfSpan {
     cudaEvent_t a, b;
@@ -138,7 +163,7 @@ struct mixgcn_rowplan {
     int device;          // kept apart from ctx: a plan may be destroyed after its context
     const mixgcn_graph* g;
     int transposed;
-    int64_t n, in_count, out_count, nnz;
+    int64_t n, in_count, out_count, nnz;   // nnz: entries of the restricted matrix
     int32_t* idx;        // [in_count] kept input rows, ascending
     CsrView view;        // n rows; columns in [0, in_count)
     uint8_t* out_mask;   // [n] 1 for output rows that have at least one kept entry
@@ -186,6 +211,8 @@ struct SpmmOpts {
     int64_t ldz_lp = 0;
     const uint32_t* out_bits = nullptr;      // nullable: bit-packed output mask of a sampled aggregation (Eq. 4), n x ld_bits words
     int64_t ld_bits = 0;
+    int64_t y_rows = -1;                     // rows of Y and entries of the view, where they differ from the graph's n and
+    int64_t nnz = -1;                        // nnz (a row plan's restricted matrix, a compacted input): limits of the debug build's index tests
 };
 mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView& A, int chunks, int k,
                           int32_t w, const float* Y, int64_t ldy, float* Z, int64_t ldz,
@@ -236,13 +263,13 @@ struct RowSet {
 };
 mixgcn_status build_row_set(mixgcn_ctx* ctx, int64_t n, const uint8_t* mask, int64_t count, int64_t ld_a, int64_t ld_b,
                             RowSet* rs, cudaStream_t s);
-mixgcn_status launch_gather_rows(mixgcn_ctx* ctx, int64_t count, int32_t d, const int32_t* idx, const float* src,
+mixgcn_status launch_gather_rows(mixgcn_ctx* ctx, int64_t n_rows, int64_t count, int32_t d, const int32_t* idx, const float* src,
                                  int64_t ld_src, float* dst, int64_t ld_dst, cudaStream_t s);
 
 mixgcn_status ensure_workspace_rows(mixgcn_ctx* ctx, int64_t bytes);
 void free_step_cache(mixgcn_ctx* ctx);
 // dst[idx[i], :] = src[i, :] for i < count (the inverse of launch_gather_rows)
-mixgcn_status launch_scatter_rows(mixgcn_ctx* ctx, int64_t count, int32_t d, const int32_t* idx, const float* src,
+mixgcn_status launch_scatter_rows(mixgcn_ctx* ctx, int64_t n_rows, int64_t count, int32_t d, const int32_t* idx, const float* src,
                                   int64_t ld_src, float* dst, int64_t ld_dst, cudaStream_t s);
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }

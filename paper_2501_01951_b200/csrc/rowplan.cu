@@ -203,5 +203,6 @@ extern "C" mixgcn_status mixgcn_spmm_rowplan(mixgcn_ctx* ctx, const mixgcn_rowpl
     SpmmOpts opts;
     opts.phase = PH_SPMM_SPARSE;
     opts.row_limit = rows_only ? p->out_count : -1;
+    opts.y_rows = p->in_count; opts.nnz = p->nnz;
     return launch_spmm(ctx, p->g, p->view, 1, 0, w, Yc, ldy, Z, ldz, epi, (cudaStream_t)stream, opts);
 }

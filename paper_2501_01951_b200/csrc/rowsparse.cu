@@ -27,11 +27,13 @@ __global__ void check_count_kernel(const int64_t* selected, int64_t expected, in
 
 // dst[i, :] = src[idx[i], :], float4 wide (ld multiples of 4, 16-byte aligned), d4 = ceil(d/4) groups per row
 __global__ void gather_rows_kernel(int64_t count, int d4, const int32_t* __restrict__ idx, const float* __restrict__ src,
-                                   int64_t ld_src, float* __restrict__ dst, int64_t ld_dst) {
+                                   int64_t ld_src, float* __restrict__ dst, int64_t ld_dst, int64_t n_rows, int32_t* status) {
     const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (t >= count * d4) return;
     const int64_t i = t / d4; const int c = (int)(t % d4);
-    reinterpret_cast<float4*>(dst + i * ld_dst)[c] = __ldg(reinterpret_cast<const float4*>(src + (int64_t)idx[i] * ld_src) + c);
+    const int64_t r = idx[i];
+    if (!index_ok(r, n_rows, status, SITE_ROW_LIST)) return;
+    reinterpret_cast<float4*>(dst + i * ld_dst)[c] = __ldg(reinterpret_cast<const float4*>(src + r * ld_src) + c);
 }
 
 // number of non-zero bytes (integer sum: order-free)
@@ -45,11 +47,13 @@ __global__ void count_rows_kernel(int64_t n, const uint8_t* __restrict__ mask, u
 
 // dst[idx[i], :] = src[i, :]
 __global__ void scatter_rows_kernel(int64_t count, int d4, const int32_t* __restrict__ idx, const float* __restrict__ src,
-                                    int64_t ld_src, float* __restrict__ dst, int64_t ld_dst) {
+                                    int64_t ld_src, float* __restrict__ dst, int64_t ld_dst, int64_t n_rows, int32_t* status) {
     const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (t >= count * d4) return;
     const int64_t i = t / d4; const int c = (int)(t % d4);
-    reinterpret_cast<float4*>(dst + (int64_t)idx[i] * ld_dst)[c] = __ldg(reinterpret_cast<const float4*>(src + i * ld_src) + c);
+    const int64_t r = idx[i];
+    if (!index_ok(r, n_rows, status, SITE_ROW_LIST)) return;
+    reinterpret_cast<float4*>(dst + r * ld_dst)[c] = __ldg(reinterpret_cast<const float4*>(src + i * ld_src) + c);
 }
 
 }  // namespace
@@ -101,22 +105,22 @@ mixgcn_status build_row_set(mixgcn_ctx* ctx, int64_t n, const uint8_t* mask, int
     return MIXGCN_OK;
 }
 
-mixgcn_status launch_gather_rows(mixgcn_ctx* ctx, int64_t count, int32_t d, const int32_t* idx, const float* src,
+mixgcn_status launch_gather_rows(mixgcn_ctx* ctx, int64_t n_rows, int64_t count, int32_t d, const int32_t* idx, const float* src,
                                  int64_t ld_src, float* dst, int64_t ld_dst, cudaStream_t s) {
     if (count <= 0) return MIXGCN_OK;
     const int d4 = (d + 3) / 4;
     LaunchScope scope(ctx, PH_ELEM, s);
-    gather_rows_kernel<<<(unsigned)((count * d4 + 255) / 256), 256, 0, s>>>(count, d4, idx, src, ld_src, dst, ld_dst);
+    gather_rows_kernel<<<(unsigned)((count * d4 + 255) / 256), 256, 0, s>>>(count, d4, idx, src, ld_src, dst, ld_dst, n_rows, ctx->d_status);
     MIXGCN_CUDA(cudaGetLastError());
     return MIXGCN_OK;
 }
 
-mixgcn_status launch_scatter_rows(mixgcn_ctx* ctx, int64_t count, int32_t d, const int32_t* idx, const float* src,
+mixgcn_status launch_scatter_rows(mixgcn_ctx* ctx, int64_t n_rows, int64_t count, int32_t d, const int32_t* idx, const float* src,
                                   int64_t ld_src, float* dst, int64_t ld_dst, cudaStream_t s) {
     if (count <= 0) return MIXGCN_OK;
     const int d4 = (d + 3) / 4;
     LaunchScope scope(ctx, PH_ELEM, s);
-    scatter_rows_kernel<<<(unsigned)((count * d4 + 255) / 256), 256, 0, s>>>(count, d4, idx, src, ld_src, dst, ld_dst);
+    scatter_rows_kernel<<<(unsigned)((count * d4 + 255) / 256), 256, 0, s>>>(count, d4, idx, src, ld_src, dst, ld_dst, n_rows, ctx->d_status);
     MIXGCN_CUDA(cudaGetLastError());
     return MIXGCN_OK;
 }

@@ -64,7 +64,21 @@ struct SpmmParams {
     const uint8_t* drop; float keep_scale;
     const float* gate; int64_t ld_gate; float gate_scale;
     const float* residual; int64_t ld_residual; float residual_scale;
+    // limits for the index tests of the bounds-checked debug build (unused otherwise)
+    int32_t* status;
+    int64_t n_cols;        // column ids lie in [0, n_cols) (they index in_mask / in_pos, or Y itself)
+    int64_t y_rows;        // rows of Y
+    int64_t n_out;         // output rows
+    int64_t n_long;        // long rows of the schedule (a segment record's `row` is an ordinal among them)
+    int64_t nnz;           // stored entries
+    int64_t n_partial;     // partial-row slots
 };
+
+// entry range and row of a unit: tested in the debug build before anything is addressed with them
+__device__ __forceinline__ bool unit_ok(const SpmmParams& p, int64_t b, int64_t e, int64_t u) {
+    return index_ok(b, p.nnz + 1, p.status, SITE_SPMM_RANGE) && index_ok(e, p.nnz + 1, p.status, SITE_SPMM_RANGE) &&
+           index_ok(u, p.partial ? p.n_long : p.n_out, p.status, SITE_SPMM_ROW);   // a segment's record names its long row by ordinal
+}
 
 __device__ __forceinline__ float epilogue1(const SpmmParams& p, float y, int64_t u, int j) {
     if (p.residual) y = fmaf(p.residual_scale, p.residual[u * p.ld_residual + j], y);
@@ -140,7 +154,7 @@ __device__ __forceinline__ void row_segment(const SpmmParams& p, int64_t b, int6
 #pragma unroll
             for (int t = 0; t < U; ++t) {
                 const float4* yr = reinterpret_cast<const float4*>(Yb + (int64_t)ck[t] * p.ldy);
-                const bool live = k + t < cnt;
+                const bool live = k + t < cnt && index_ok(ck[t], p.y_rows, p.status, SITE_SPMM_COL);
 #pragma unroll
                 for (int v = 0; v < VPL; ++v) {
                     const int c4 = lig + v * LPR;
@@ -175,6 +189,7 @@ __global__ void __launch_bounds__(256, VPL <= 2 ? SPMM_MINB : 1) spmm_group_kern
         b = __ldg(p.rowptr + u);
         e = __ldg(p.rowptr + u + 1);
     }
+    if (!unit_ok(p, b, e, u)) return;
     const int w4 = (p.w + 3) >> 2;
     float4 acc[VPL];
 #pragma unroll
@@ -223,6 +238,10 @@ __global__ void __launch_bounds__(256, SPMM_SHORT_MINB) spmm_short_kernel(const 
     if (idx0 >= p.idx_end) return;
     int4 rc = make_int4(0, 0, 0, 0);
     if (lane < RB && idx0 + lane < p.idx_end) rc = __ldg(reinterpret_cast<const int4*>(p.rec + idx0 + lane));
+    if constexpr (DEBUG_BOUNDS) {
+        const int64_t b0 = ((int64_t)(uint32_t)rc.y << 32) | (uint32_t)rc.x;
+        if (!unit_ok(p, b0, b0 + rc.z, rc.w)) { rc.z = 0; rc.w = -1; }      // a bad record: no entries, no store
+    }
     // lane (k, e) = (lane % RB, lane / RB) fetches entry e of row k
     const int k_of = lane % RB, e_of = lane / RB;
     const uint32_t lo = (uint32_t)__shfl_sync(0xFFFFFFFFu, rc.x, k_of), hi = (uint32_t)__shfl_sync(0xFFFFFFFFu, rc.y, k_of);
@@ -246,7 +265,7 @@ __global__ void __launch_bounds__(256, SPMM_SHORT_MINB) spmm_short_kernel(const 
             const int ck = __shfl_sync(0xFFFFFFFFu, c, k + e * RB);
             ak[k] = __shfl_sync(0xFFFFFFFFu, a, k + e * RB);
             const int len_k = __shfl_sync(0xFFFFFFFFu, rc.z, k);
-            const bool live = e < len_k && col_ok;
+            const bool live = e < len_k && col_ok && index_ok(ck, p.y_rows, p.status, SITE_SPMM_COL);
             y[k] = live ? __ldg(reinterpret_cast<const float4*>(Yb + (int64_t)ck * p.ldy) + lane) : make_float4(0.f, 0.f, 0.f, 0.f);
         }
 #pragma unroll
@@ -258,7 +277,7 @@ __global__ void __launch_bounds__(256, SPMM_SHORT_MINB) spmm_short_kernel(const 
 #pragma unroll
     for (int k = 0; k < RB; ++k) {
         const int64_t u = __shfl_sync(0xFFFFFFFFu, rc.w, k);
-        if (idx0 + k < p.idx_end && col_ok) store_row(p, u, lane, acc[k]);
+        if (idx0 + k < p.idx_end && col_ok && (!DEBUG_BOUNDS || u >= 0)) store_row(p, u, lane, acc[k]);
     }
 }
 
@@ -276,6 +295,7 @@ __global__ void __launch_bounds__(256) spmm_sparse_kernel(const SpmmParams p) {
     const int4 rc = __ldg(reinterpret_cast<const int4*>(p.rec + idx));
     const int64_t b = ((int64_t)(uint32_t)rc.y << 32) | (uint32_t)rc.x, e = b + rc.z;
     const int64_t u = rc.w;
+    if (!unit_ok(p, b, e, u)) return;
     const int w4 = (p.w + 3) >> 2;
     const float* Yb = p.Y + p.j0;
     float4 acc[VPL];
@@ -286,7 +306,7 @@ __global__ void __launch_bounds__(256) spmm_sparse_kernel(const SpmmParams p) {
         int r = -1; float a = 0.0f;
         if (i0 + lig < e) {
             const int c = __ldg(p.col + i0 + lig);
-            if (__ldg(p.in_mask + c)) {
+            if (index_ok(c, p.n_cols, p.status, SITE_SPMM_COL) && __ldg(p.in_mask + c)) {
                 r = p.in_pos ? __ldg(p.in_pos + c) : c;
                 a = __ldg(p.val + i0 + lig);
             }
@@ -313,7 +333,7 @@ __global__ void __launch_bounds__(256) spmm_sparse_kernel(const SpmmParams p) {
 #pragma unroll
                 for (int v = 0; v < VPL; ++v) {
                     const int c4 = lig + v * LPR;
-                    y[t][v] = (t < nh && c4 < w4) ? __ldg(yr + c4) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    y[t][v] = (t < nh && c4 < w4 && index_ok(rk[t], p.y_rows, p.status, SITE_SPMM_POS)) ? __ldg(yr + c4) : make_float4(0.f, 0.f, 0.f, 0.f);
                 }
             }
 #pragma unroll
@@ -354,7 +374,11 @@ __global__ void __launch_bounds__(256) spmm_filtered_kernel(const SpmmParams p) 
     bool live = false;
     if (idx0 + lane < p.idx_end) {
         rc = __ldg(reinterpret_cast<const int4*>(p.rec + idx0 + lane));
-        live = __ldg(p.row_filter + (p.seg_perm ? __ldg(p.seg_perm + rc.w) : rc.w)) != 0;
+        const int64_t b0 = ((int64_t)(uint32_t)rc.y << 32) | (uint32_t)rc.x;
+        if (unit_ok(p, b0, b0 + rc.z, rc.w)) {
+            const int64_t row = p.seg_perm ? __ldg(p.seg_perm + rc.w) : rc.w;
+            live = index_ok(row, p.n_out, p.status, SITE_SPMM_ROW) && __ldg(p.row_filter + row) != 0;
+        }
     }
     unsigned bits = __ballot_sync(0xFFFFFFFFu, live);
     const int w4 = (p.w + 3) >> 2;
@@ -397,13 +421,17 @@ __global__ void __launch_bounds__(256) spmm_combine_kernel(const SpmmParams p, i
     if (i >= n_long) return;
     const int64_t s0 = seg_off[i], s1 = seg_off[i + 1];
     const int64_t u = perm[i];
+    if (!index_ok(s0, p.n_partial + 1, p.status, SITE_SPMM_SEG) || !index_ok(s1, p.n_partial + 1, p.status, SITE_SPMM_SEG) ||
+        !index_ok(u, p.n_out, p.status, SITE_SPMM_ROW)) return;
     if (p.row_filter && !__ldg(p.row_filter + u)) return;
     const int w4 = (p.w + 3) >> 2;
     if (p.out_mask && lane == 0) p.out_mask[u] = 1;    // long rows are kept without looking (conservative)
     for (int c4 = lane; c4 < w4; c4 += 32) {
         float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
         for (int64_t q = s0; q < s1; ++q) {
-            const float4 t = __ldg(reinterpret_cast<const float4*>(p.partial + __ldg(seg_pos + q) * p.ldp) + c4);
+            const int64_t slot = __ldg(seg_pos + q);
+            if (!index_ok(slot, p.n_partial, p.status, SITE_SPMM_SEG)) continue;
+            const float4 t = __ldg(reinterpret_cast<const float4*>(p.partial + slot * p.ldp) + c4);
             s.x += t.x; s.y += t.y; s.z += t.z; s.w += t.w;
         }
         store_row(p, u, c4, s);
@@ -515,6 +543,10 @@ mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView&
         p.gate = epi->gate; p.ld_gate = epi->ld_gate; p.gate_scale = epi->gate_scale;
         p.residual = epi->residual; p.ld_residual = epi->ld_residual; p.residual_scale = epi->residual_scale;
     }
+    p.status = ctx->d_status;
+    p.n_out = g->n; p.n_cols = g->n; p.y_rows = opts.y_rows >= 0 ? opts.y_rows : g->n;
+    p.nnz = opts.nnz >= 0 ? opts.nnz : g->nnz;
+    p.n_long = S.n_long; p.n_partial = S.total_segs;
     p.rec = S.rec;
     if (sparse) { p.in_mask = sparse->in_mask; p.in_pos = sparse->in_pos; p.out_mask = sparse->out_mask; }
     p.row_filter = row_filter;
