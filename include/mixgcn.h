@@ -416,6 +416,23 @@ mixgcn_status mixgcn_layer_fwd(mixgcn_ctx* ctx, const mixgcn_graph* g, const mix
                                const float* X_in, const float* W, const float* bias,
                                const uint8_t* drop_mask, float* saved, float* X_out, void* stream);
 
+/* The last layer's forward and the loss in one call (Algorithm 2: the last aggregation + update and the loss
+ * line).  Same results as mixgcn_layer_fwd (without a dropout mask) followed by mixgcn_loss_softmax_xent with
+ * dlogits aliasing the logits -- *loss, pred (required here) and *n_correct (nullable) as there; `dlogits`
+ * (n x ld_out) receives the gradient on train rows and zeros elsewhere, or, with
+ * MIXGCN_OPT_LOSS_TRAIN_ROWS_ONLY = 2, is left unchanged elsewhere; `saved` as in mixgcn_layer_fwd -- but where
+ * a whole row of logits is in one thread group's hands at the place that produces it, the loss is taken there
+ * and the logits are never written: in the aggregation's epilogue for an update-first layer, in the tensor-core
+ * product's epilogue for an aggregate-first layer with TF32 or BF16 products; both for d_out <= 256, no ReLU,
+ * n_chunks <= 1.  (Same formulas; the sums within a row may run in another order than in the separate calls.)
+ * Every other layer runs as the two separate steps inside this call.  MIXGCN_EUNSUPPORTED with OUT_ROWS_ONLY or
+ * MIXGCN_OPT_LOSS_TRAIN_ROWS_ONLY = 1.  Device-visible conditions (empty mask, label out of range) as in
+ * mixgcn_loss_softmax_xent. */
+mixgcn_status mixgcn_layer_fwd_loss(mixgcn_ctx* ctx, const mixgcn_graph* g, const mixgcn_layer_desc* desc,
+                                    const float* X_in, const float* W, const float* bias, float* saved,
+                                    float* dlogits, const int32_t* labels, const uint8_t* train_mask,
+                                    float* loss, int32_t* pred, int64_t* n_correct, void* stream);
+
 /* Backward.  G_out (n x ld_out) is the gradient w.r.t. X_out and is OVERWRITTEN (it becomes
  * the gradient w.r.t. the pre-activation).  `saved` is consumed: agg-first reads A_hat X_in
  * from it and then overwrites it; upd-first uses it as scratch.  dW is d_in x d_out, dbias

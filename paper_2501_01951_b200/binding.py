@@ -50,7 +50,7 @@ SYMBOLS = (
     "mixgcn_count_rows", "mixgcn_rowplan_create", "mixgcn_rowplan_destroy", "mixgcn_rowplan_info",
     "mixgcn_rowplan_export", "mixgcn_spmm_rowplan", "mixgcn_colsum", "mixgcn_ctx_gemm_paths",
     "mixgcn_train_step_host_prefetch", "mixgcn_probe_gather", "mixgcn_spmm_sampled", "mixgcn_mask_pack",
-    "mixgcn_build_info", "mixgcn_debug_poke_col",
+    "mixgcn_build_info", "mixgcn_debug_poke_col", "mixgcn_layer_fwd_loss",
 )
 
 
@@ -361,6 +361,18 @@ def layer_fwd(ctx: Ctx, g: Graph, desc: LayerDesc, X_in, W, bias, drop_mask, sav
         raise TypeError("W must be dense row-major")
     _check(lib.mixgcn_layer_fwd(ctx.h, g.h, C.byref(desc), _ptr(X_in), _ptr(W), _ptr(bias), _ptr(drop_mask),
                                 _ptr(saved), _ptr(X_out), _stream()))
+
+
+def layer_fwd_loss(ctx: Ctx, g: Graph, desc: LayerDesc, X_in, W, bias, saved, dlogits, labels, train_mask, loss, pred,
+                   n_correct=None):
+    """Last layer (update-first) with the loss taken inside its aggregation; raises EUNSUPPORTED if the layer does not qualify."""
+    _mat(X_in, "X_in"); _mat(saved, "saved"); _mat(dlogits, "dlogits"); _dev(W, torch.float32, "W")
+    if not W.is_contiguous():
+        raise TypeError("W must be dense row-major")
+    _dev(labels, torch.int32, "labels"); _dev(train_mask, torch.uint8, "train_mask"); _dev(loss, torch.float32, "loss")
+    _dev(pred, torch.int32, "pred")
+    _check(lib.mixgcn_layer_fwd_loss(ctx.h, g.h, C.byref(desc), _ptr(X_in), _ptr(W), _ptr(bias), _ptr(saved), _ptr(dlogits),
+                                     _ptr(labels), _ptr(train_mask), _ptr(loss), _ptr(pred), _ptr(n_correct), _stream()))
 
 
 def layer_bwd(ctx: Ctx, g: Graph, desc: LayerDesc, X_in, saved, X_out, drop_mask, W, G_out, G_in, dW, dbias):

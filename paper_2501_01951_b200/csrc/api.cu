@@ -107,6 +107,7 @@ mixgcn_status launch_gemm(mixgcn_ctx* ctx, int precision, int ta, int tb, int64_
     // FMA kernel.  ctx->gemm_path counts which kernel served each product.
     uint16_t* c_lp = lp ? lp->C : nullptr;
     const int64_t ldc_lp = lp ? lp->ldc : 0;
+    const LossFuse* loss = lp ? lp->loss : nullptr;
     bool c_lp_done = false;
     mixgcn_status st = MIXGCN_EUNSUPPORTED;
     const bool fp32_layout = aligned16(A) && (lda & 3) == 0 && (!ta || (aligned16(B) && (ldb & 3) == 0));
@@ -134,7 +135,7 @@ mixgcn_status launch_gemm(mixgcn_ctx* ctx, int precision, int ta, int tb, int64_
             b_lp = dst;
         }
         st = launch_gemm_tc(ctx, 1, ta, tb, M, N, K, a_lp, lda_lp, ta ? (const void*)b_lp : (const void*)B, ta ? ldb_lp : ldb,
-                            C, ldc, epi, epi_row0, s, ta ? nullptr : c_lp, ldc_lp);
+                            C, ldc, epi, epi_row0, s, ta ? nullptr : c_lp, ldc_lp, nullptr, nullptr, loss);
         if (st == MIXGCN_OK) { ctx->gemm_path[2]++; c_lp_done = !ta && c_lp; }
     }
     if (st == MIXGCN_EUNSUPPORTED && lp && lp->a_fp32_missing)
@@ -143,9 +144,10 @@ mixgcn_status launch_gemm(mixgcn_ctx* ctx, int precision, int ta, int tb, int64_
     if (colsum_b && !ta) MIXGCN_FAIL(MIXGCN_EINVAL, "gemm: column sums of B are a by-product of the weight-gradient form only");
     if (st == MIXGCN_EUNSUPPORTED && precision != MIXGCN_PREC_FP32) {
         st = launch_gemm_tc(ctx, 0, ta, tb, M, N, K, A, lda, B, ldb, C, ldc, epi, epi_row0, s, ta ? nullptr : c_lp, ldc_lp,
-                            colsum_b, &colsum_done);
+                            colsum_b, &colsum_done, loss);
         if (st == MIXGCN_OK) { ctx->gemm_path[1]++; c_lp_done = !ta && c_lp; }
     }
+    if (st == MIXGCN_EUNSUPPORTED && loss) return st;      // the caller runs the product and the loss separately
     if (st == MIXGCN_EUNSUPPORTED) {
         st = launch_gemm_simt(ctx, ta, tb, M, N, K, A, lda, B, ldb, C, ldc, epi, epi_row0, s);
         if (st == MIXGCN_OK) ctx->gemm_path[0]++;
@@ -215,6 +217,7 @@ extern "C" mixgcn_status mixgcn_ctx_destroy(mixgcn_ctx* ctx) {
     cudaFree(ctx->workspace_spmm);
     cudaFree(ctx->workspace_rows);
     cudaFree(ctx->workspace_lp);
+    cudaFree(ctx->workspace_loss);
     cudaFree(ctx->arena);
     cudaFree(ctx->d_status);
     delete ctx;
@@ -519,6 +522,69 @@ extern "C" mixgcn_status mixgcn_layer_fwd(mixgcn_ctx* ctx, const mixgcn_graph* g
     SpmmOpts out_opts; out_opts.Z_lp = lp.x_out; out_opts.ldz_lp = lp.ld_out;
     MIXGCN_TRY(launch_spmm(ctx, g, g->fwd, 1, 0, d->d_out, saved, d->ld_saved, X_out, d->ld_out, &epi, s, out_opts));
     return MIXGCN_OK;
+}
+
+extern "C" mixgcn_status mixgcn_layer_fwd_loss(mixgcn_ctx* ctx, const mixgcn_graph* g, const mixgcn_layer_desc* d,
+                                               const float* X_in, const float* W, const float* bias, float* saved,
+                                               float* dlogits, const int32_t* labels, const uint8_t* train_mask,
+                                               float* loss, int32_t* pred, int64_t* n_correct, void* stream) {
+    if (!ctx || !g || !X_in || !W || !saved || !dlogits || !labels || !train_mask || !loss || !pred)
+        MIXGCN_FAIL(MIXGCN_EINVAL, "layer_fwd_loss: null argument");
+    MIXGCN_TRY(check_desc(d, "layer_fwd_loss"));
+    if (!aligned16(X_in) || !aligned16(saved) || !aligned16(dlogits) || !aligned16(W))
+        MIXGCN_FAIL(MIXGCN_EINVAL, "layer_fwd_loss: matrices must be 16-byte aligned");
+    if ((d->flags & MIXGCN_LAYER_OUT_ROWS_ONLY) || ctx->loss_train_rows_only == 1)
+        MIXGCN_FAIL(MIXGCN_EUNSUPPORTED, "layer_fwd_loss: every row's logits are produced here (no OUT_ROWS_ONLY, no MIXGCN_OPT_LOSS_TRAIN_ROWS_ONLY = 1)");
+    if (d->d_out > 4096) MIXGCN_FAIL(MIXGCN_EINVAL, "layer_fwd_loss: at most 4096 classes");
+    MIXGCN_CUDA(cudaSetDevice(ctx->device));
+    cudaStream_t s = (cudaStream_t)stream;
+    const int64_t n = g->n;
+    const int order = resolve_order(d);
+    // The loss can be taken where the logits are produced if a whole row is in one thread group's hands there:
+    // at most 256 classes, nothing but the bias between the sums and the logits, all rows in one piece.
+    const bool plain = !(d->flags & (MIXGCN_LAYER_RELU | MIXGCN_LAYER_SAVED_IS_VALID | MIXGCN_LAYER_SAVED_LP_ONLY)) && d->n_chunks <= 1 && d->d_out <= 256;
+    mixgcn_epilogue epi{};
+    epi.bias = bias; epi.keep_scale = 1.0f;
+    if (plain && order == MIXGCN_ORDER_UPD_FIRST) {
+        // logits = A_hat (X_in W) + b: the aggregation's epilogue takes the loss
+        const LayerLP lp(d);
+        GemmLP glp; glp.A = lp.x_in; glp.lda = lp.ld_in;
+        MIXGCN_TRY(launch_gemm(ctx, d->precision, 0, 0, n, d->d_out, d->d_in, X_in, d->ld_in, W, d->d_out, saved, d->ld_saved,
+                               nullptr, 0, s, &glp));
+        LossFuse lf;
+        MIXGCN_TRY(loss_fuse_begin(ctx, n, labels, train_mask, pred, n_correct, s, &lf));
+        SpmmOpts opts; opts.loss = &lf;
+        MIXGCN_TRY(launch_spmm(ctx, g, g->fwd, 1, 0, d->d_out, saved, d->ld_saved, dlogits, d->ld_out, &epi, s, opts));
+        return loss_fuse_end(ctx, n, d->d_out, lf, loss, n_correct, s);
+    }
+    if (plain && order == MIXGCN_ORDER_AGG_FIRST && d->precision != MIXGCN_PREC_FP32) {
+        // logits = (A_hat X_in) W + b: the tensor-core product's epilogue finds every row's arg-max and writes the
+        // logits of the train rows only; the loss then runs over those rows in place
+        const LayerLP lp(d);
+        SpmmOpts agg_opts; agg_opts.Z_lp = lp.saved; agg_opts.ldz_lp = lp.ld_saved;
+        MIXGCN_TRY(launch_spmm(ctx, g, g->fwd, 1, 0, d->d_in, X_in, d->ld_in, saved, d->ld_saved, nullptr, s, agg_opts));
+        LossFuse lf;
+        lf.train_mask = train_mask; lf.pred = pred; lf.zero_rows = ctx->loss_train_rows_only == 2 ? 0 : 1;
+        GemmLP glp; glp.A = lp.saved; glp.lda = lp.ld_saved; glp.loss = &lf;
+        const mixgcn_status st = launch_gemm(ctx, d->precision, 0, 0, n, d->d_out, d->d_in, saved, d->ld_saved, W, d->d_out, dlogits,
+                                             d->ld_out, &epi, 0, s, &glp);
+        if (st == MIXGCN_OK) {
+            const int keep = ctx->loss_train_rows_only;
+            ctx->loss_train_rows_only = 1;               // train rows only, in place; pred is already complete
+            const mixgcn_status sl = mixgcn_loss_softmax_xent(ctx, n, d->d_out, dlogits, d->ld_out, labels, train_mask, loss, dlogits,
+                                                              nullptr, n_correct, stream);
+            ctx->loss_train_rows_only = keep;
+            return sl;
+        }
+        if (st != MIXGCN_EUNSUPPORTED) return st;
+        // no tensor-core kernel for this shape: the product and the loss as two steps (the aggregation is in `saved`)
+        MIXGCN_TRY(launch_gemm(ctx, d->precision, 0, 0, n, d->d_out, d->d_in, saved, d->ld_saved, W, d->d_out, dlogits, d->ld_out,
+                               &epi, 0, s, nullptr));
+        return mixgcn_loss_softmax_xent(ctx, n, d->d_out, dlogits, d->ld_out, labels, train_mask, loss, dlogits, pred, n_correct, stream);
+    }
+    // everything else: the layer, then the loss in place over its output
+    MIXGCN_TRY(mixgcn_layer_fwd(ctx, g, d, X_in, W, bias, nullptr, saved, dlogits, stream));
+    return mixgcn_loss_softmax_xent(ctx, n, d->d_out, dlogits, d->ld_out, labels, train_mask, loss, dlogits, pred, n_correct, stream);
 }
 
 extern "C" mixgcn_status mixgcn_layer_bwd(mixgcn_ctx* ctx, const mixgcn_graph* g, const mixgcn_layer_desc* d,

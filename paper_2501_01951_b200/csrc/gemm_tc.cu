@@ -69,6 +69,8 @@ struct TcParams {
     uint32_t wait_limit;    // polls after which a wait gives up
     int debug_drop_load;    // test hook: the producer leaves out the loads of its first stage (the wait on it then expires)
     int epi_boxes;          // single-CTA K-major kernel: staging boxes per epilogue warp (1 or 2)
+    // arg-max epilogue of the single-CTA K-major kernel (LOSS instances; one n-tile): C receives the train rows only
+    const uint8_t* loss_mask; int32_t* loss_pred; int loss_zero_rows;
 };
 
 __device__ __forceinline__ float tc_apply_epi(const TcEpi& e, float y, int64_t m, int64_t n, int64_t N) {
@@ -300,7 +302,11 @@ constexpr int KK_BIAS_MAX = 1024;
 // warps) applies bias / ReLU from registers and shared memory, writes 32-row x 128-byte boxes in the
 // 128-byte swizzle and hands them to TMA stores, which also clip ragged M / N edges; the optional bf16
 // copy of C goes out with 16-byte stores straight from the registers.
-template <int KIND>
+// LOSS instances (one n-tile, N <= 256: a row of C is a row of logits for a masked loss): the epilogue finds
+// every row's arg-max (-> pred) and writes the logits of the TRAIN rows only (the others are zeroed or left
+// alone) -- all the loss that follows needs.  The two epilogue warps of a lane quarter then take alternate
+// TILES (one accumulator buffer each) instead of alternate column chunks, so that one thread sees its whole row.
+template <int KIND, bool LOSS = false>
 __global__ void __launch_bounds__(KK_THREADS, 1) gemm_tc_kk_kernel(const __grid_constant__ CUtensorMap map_a,
                                                                 const __grid_constant__ CUtensorMap map_b,
                                                                 const __grid_constant__ CUtensorMap map_c,
@@ -333,7 +339,7 @@ __global__ void __launch_bounds__(KK_THREADS, 1) gemm_tc_kk_kernel(const __grid_
     if (threadIdx.x == 0) {
         abort_flag = 0;
         for (int s = 0; s < p.stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], KK_EPI_WARPS); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], LOSS ? KK_EPI_WARPS / 2 : KK_EPI_WARPS); }
         mbar_init(&b_bar, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -402,6 +408,102 @@ __global__ void __launch_bounds__(KK_THREADS, 1) gemm_tc_kk_kernel(const __grid_
                 if (ok) tc_commit(&acc_full[buf]);
             }
         }
+    } else if constexpr (LOSS) {
+        // ---------------- arg-max epilogue: warp w reads TMEM lanes 32*(w&3).. of the tiles j = (w>>2), (w>>2)+2, ... ----------------
+        // A thread sees its whole row of logits (sums + bias), 32 columns at a time: per chunk a tree of maxima
+        // and the lowest position that attains it (independent operations, no long dependent chain), then one
+        // strict comparison against the running maximum (an earlier chunk keeps a tie).  The row itself is
+        // written only if it is a train row (zeros elsewhere when every row is wanted).
+        const int quarter = warp & 3, half = warp >> 2;
+        const bool add_bias = p.epi.bias != nullptr && bias_in_smem;
+        const bool use_tma = tma_store != 0;              // every row is written: through the staged boxes
+        const int N = (int)p.N;
+        uint8_t* const box = smem_out + (size_t)warp * p.epi_boxes * 4096;
+        uint32_t j = (uint32_t)half;
+        bool ok = true;
+        for (int64_t tile = blockIdx.x + (int64_t)half * gridDim.x; tile < tiles && ok; tile += 2 * (int64_t)gridDim.x, j += 2) {
+            const uint32_t buf = j & 1;
+            const int64_t m0 = tile * TC_BM;                 // one n-tile
+            const int64_t m = m0 + quarter * 32 + lane;
+            const bool row_ok = m < p.M;
+            const bool train = row_ok && __ldg(p.loss_mask + m) != 0;     // requested before the accumulator is waited for
+            if (lane == 0) ok = mbar_wait(&acc_full[buf], (j >> 1) & 1, &abort_flag, p.wait_limit);
+            ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
+            if (!ok) { if (lane == 0) { abort_flag = 1; atomicMax(p.status, DEV_WAIT_EXPIRED); } break; }
+            tc_fence_after();
+            const uint32_t t_row = tmem_base + buf * acc_stride + ((uint32_t)(quarter * 32) << 16);
+            float mx = -INFINITY; int arg = 0;             // nothing but -inf / NaN: 0
+            for (int c0 = 0; c0 < p.bn; c0 += 32) {
+                uint32_t r[32];
+                tc_ld32(t_row + (uint32_t)c0, r);
+                tc_wait_ld();
+                float x[32];
+                if (add_bias) {
+                    const float4* sb4 = reinterpret_cast<const float4*>(s_bias + c0);
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        const float4 b4 = sb4[q];
+                        x[4 * q] = __uint_as_float(r[4 * q]) + b4.x; x[4 * q + 1] = __uint_as_float(r[4 * q + 1]) + b4.y;
+                        x[4 * q + 2] = __uint_as_float(r[4 * q + 2]) + b4.z; x[4 * q + 3] = __uint_as_float(r[4 * q + 3]) + b4.w;
+                    }
+                } else {
+#pragma unroll
+                    for (int q = 0; q < 32; ++q) x[q] = __uint_as_float(r[q]);
+                }
+                // the row's values leave first (train rows; zeros for the others when every row is written)
+                if (use_tma) {
+                    if (lane == 0) bulk_wait_read<0>();       // the store that last used this box has read it
+                    __syncwarp();
+#pragma unroll
+                    for (int q = 0; q < 8; ++q)
+                        *reinterpret_cast<float4*>(box + lane * 128 + ((q ^ (lane & 7)) << 4)) =
+                            train ? make_float4(x[4 * q], x[4 * q + 1], x[4 * q + 2], x[4 * q + 3]) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0) {
+                        tma_store_2d(&map_c, box, c0, (int32_t)(m0 + quarter * 32));
+                        bulk_commit();
+                    }
+                } else if (train || (p.loss_zero_rows && row_ok)) {
+                    float* dst = p.C + m * p.ldc + c0;
+                    if (p.vec_c && c0 + 31 < N) {
+#pragma unroll
+                        for (int q = 0; q < 32; q += 4)
+                            *reinterpret_cast<float4*>(dst + q) = train ? make_float4(x[q], x[q + 1], x[q + 2], x[q + 3]) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    } else {
+#pragma unroll
+                        for (int q = 0; q < 32; ++q)
+                            if (c0 + q < N) dst[q] = train ? x[q] : 0.0f;
+                    }
+                }
+                if (c0 + 32 > N) {                            // ragged last chunk: columns beyond N are not data
+#pragma unroll
+                    for (int q = 0; q < 32; ++q)
+                        if (c0 + q >= N) x[q] = -INFINITY;
+                }
+                float t[16];
+#pragma unroll
+                for (int q = 0; q < 16; ++q) t[q] = fmaxf(x[q], x[q + 16]);
+#pragma unroll
+                for (int w = 8; w > 0; w >>= 1)
+#pragma unroll
+                    for (int q = 0; q < w; ++q) t[q] = fmaxf(t[q], t[q + w]);
+                const float cm = t[0];
+                if (__any_sync(0xFFFFFFFFu, cm > mx)) {       // some row of the warp has a new maximum in this chunk
+                    int a4[4] = {32, 32, 32, 32};
+#pragma unroll
+                    for (int q = 31; q >= 0; --q)
+                        if (x[q] == cm) a4[q & 3] = q;
+                    const int ca = min(min(a4[0], a4[1]), min(a4[2], a4[3]));
+                    if (cm > mx) { mx = cm; arg = c0 + ca; }
+                }
+            }
+            if (row_ok && p.loss_pred) p.loss_pred[m] = arg;
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&acc_empty[buf]);
+        }
+        if (tma_store && lane == 0) bulk_wait_all();
     } else {
         // ---------------- epilogue: warp w reads TMEM lanes 32*(w&3).., 32-column chunks (w>>2), (w>>2)+2, ... ----------------
         const int quarter = warp & 3, half = warp >> 2;
@@ -1076,9 +1178,11 @@ int pick_splits(int64_t tiles, int64_t slots, int64_t max_splits) {
 template <int KIND>
 mixgcn_status launch_kind(mixgcn_ctx* ctx, int ta, int tb, int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,
                           const void* B, int64_t ldb, float* C, int64_t ldc, const mixgcn_epilogue* epi, int64_t epi_row0,
-                          cudaStream_t s, uint16_t* C_lp, int64_t ldc_lp, float* colsum_b, bool* colsum_done) {
+                          cudaStream_t s, uint16_t* C_lp, int64_t ldc_lp, float* colsum_b, bool* colsum_done, const LossFuse* loss) {
     using Cfg = KindCfg<KIND>;
     constexpr int EB = Cfg::EB, BK = Cfg::BK;
+    // the loss epilogue exists in the single-CTA K-major kernel for one n-tile and a bias-only epilogue
+    if (loss && (ta || N > 256 || C_lp || ctx->debug_drop_load || (epi && (epi->relu || epi->drop_mask || epi->gate)))) return MIXGCN_EUNSUPPORTED;
     constexpr int64_t LD_ALIGN = 16 / EB;           // TMA strides are multiples of 16 bytes
     if (M <= 0 || N <= 0 || K <= 0) return MIXGCN_EUNSUPPORTED;
     if (ta && tb) return MIXGCN_EUNSUPPORTED;
@@ -1181,10 +1285,19 @@ mixgcn_status launch_kind(mixgcn_ctx* ctx, int ta, int tb, int64_t M, int64_t N,
         if (stages < 2) stages = 2;
         p.stages = stages;
         const size_t smem_kk = (b_resident ? b_all : 0) + (size_t)stages * stage + box_bytes + 1024;
-        const int tma_store = p.vec_c ? 1 : 0;
+        const int tma_store = (p.vec_c && (!loss || loss->zero_rows)) ? 1 : 0;     // a loss that leaves the other rows alone writes train rows only
         CUtensorMap map_c = map_a;
         if (tma_store && !encode_2d(&map_c, C, 4, N, M, ldc, 32, 32)) return MIXGCN_EUNSUPPORTED;
         int64_t grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
+        if (loss) {
+            if (p.n_tiles != 1) return MIXGCN_EUNSUPPORTED;
+            p.loss_mask = loss->train_mask; p.loss_pred = loss->pred; p.loss_zero_rows = loss->zero_rows;
+            MIXGCN_CUDA(cudaFuncSetAttribute(gemm_tc_kk_kernel<KIND, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_kk));
+            LaunchScope scope(ctx, PH_GEMM, s);
+            gemm_tc_kk_kernel<KIND, true><<<dim3((unsigned)grid, 1, 1), KK_THREADS, smem_kk, s>>>(map_a, map_b, map_c, p, b_resident, tma_store);
+            MIXGCN_CUDA(cudaGetLastError());
+            return MIXGCN_OK;
+        }
         MIXGCN_CUDA(cudaFuncSetAttribute(gemm_tc_kk_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_kk));
         LaunchScope scope(ctx, PH_GEMM, s);
         gemm_tc_kk_kernel<KIND><<<dim3((unsigned)grid, 1, 1), KK_THREADS, smem_kk, s>>>(map_a, map_b, map_c, p, b_resident, tma_store);
@@ -1295,11 +1408,11 @@ namespace mixgcn {
 mixgcn_status launch_gemm_tc(mixgcn_ctx* ctx, int kind, int ta, int tb, int64_t M, int64_t N, int64_t K, const void* A,
                              int64_t lda, const void* B, int64_t ldb, float* C, int64_t ldc,
                              const mixgcn_epilogue* epi, int64_t epi_row0, cudaStream_t s, uint16_t* C_lp, int64_t ldc_lp,
-                             float* colsum_b, bool* colsum_done) {
+                             float* colsum_b, bool* colsum_done, const LossFuse* loss) {
     if (colsum_done) *colsum_done = false;
     if (kind == KIND_BF16)
-        return launch_kind<KIND_BF16>(ctx, ta, tb, M, N, K, A, lda, B, ldb, C, ldc, epi, epi_row0, s, C_lp, ldc_lp, colsum_b, colsum_done);
-    return launch_kind<KIND_TF32>(ctx, ta, tb, M, N, K, A, lda, B, ldb, C, ldc, epi, epi_row0, s, C_lp, ldc_lp, colsum_b, colsum_done);
+        return launch_kind<KIND_BF16>(ctx, ta, tb, M, N, K, A, lda, B, ldb, C, ldc, epi, epi_row0, s, C_lp, ldc_lp, colsum_b, colsum_done, loss);
+    return launch_kind<KIND_TF32>(ctx, ta, tb, M, N, K, A, lda, B, ldb, C, ldc, epi, epi_row0, s, C_lp, ldc_lp, colsum_b, colsum_done, loss);
 }
 
 // dst (rows x ld_dst bf16, ld_dst a multiple of 4) = bf16(src (rows x ld_src fp32, 16-byte aligned, ld_src % 4 == 0)), columns < d

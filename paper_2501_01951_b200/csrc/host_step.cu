@@ -239,9 +239,8 @@ extern "C" mixgcn_status mixgcn_train_step_host(mixgcn_ctx* ctx, const mixgcn_gr
         MIXGCN_CUDA(cudaMemcpyAsync(lo.vb[l], vb[l], bb, H2D, s));
     }
     // forward, loss, backward, update
-    for (int l = 0; l < L; ++l) {
-        MIXGCN_TRY(mixgcn_layer_fwd(ctx, g, &lo.desc[l], lo.X[l], lo.W[l], lo.b[l], nullptr, lo.saved[l], lo.X[l + 1], s));
-        if (l == 0 && pf && pf->announced && lo.desc[0].order == MIXGCN_ORDER_AGG_FIRST) {
+    auto after_first_layer = [&]() -> mixgcn_status {
+        if (pf && pf->announced && lo.desc[0].order == MIXGCN_ORDER_AGG_FIRST) {
             // In agg-first order nothing after the first layer's forward reads the features again (its
             // backward uses A_hat X from `saved`): the announced features of the NEXT call are copied
             // into X[0] on the second stream while the rest of this iteration runs.
@@ -252,16 +251,32 @@ extern "C" mixgcn_status mixgcn_train_step_host(mixgcn_ctx* ctx, const mixgcn_gr
             MIXGCN_CUDA(cudaEventRecord(pf->done, s2));
             pf->in_flight = pf->announced; pf->dst = lo.X[0]; pf->n = n; pf->d0 = d0;
         }
+        return MIXGCN_OK;
+    };
+    // With predictions wanted for every node the last layer and the loss are one call (the loss is taken where
+    // the logits are produced, wherever the kernels allow; rows the backward never reads are left alone).
+    const bool one_call = pred != nullptr && !rows_only;
+    for (int l = 0; l < (one_call ? L - 1 : L); ++l) {
+        MIXGCN_TRY(mixgcn_layer_fwd(ctx, g, &lo.desc[l], lo.X[l], lo.W[l], lo.b[l], nullptr, lo.saved[l], lo.X[l + 1], s));
+        if (l == 0) MIXGCN_TRY(after_first_layer());
     }
-    if (pf) pf->announced = nullptr;
     {
         const int keep = ctx->loss_train_rows_only;
-        ctx->loss_train_rows_only = rows_only ? 1 : keep;
-        const mixgcn_status st = mixgcn_loss_softmax_xent(ctx, n, dims[L], lo.X[L], round4(dims[L]), lo.labels, lo.mask, lo.loss,
-                                                          lo.X[L], pred ? lo.pred : nullptr, nullptr, s);
+        mixgcn_status st;
+        if (one_call) {
+            ctx->loss_train_rows_only = lo.desc[L - 1].gout_plan ? 2 : 0;
+            st = mixgcn_layer_fwd_loss(ctx, g, &lo.desc[L - 1], lo.X[L - 1], lo.W[L - 1], lo.b[L - 1], lo.saved[L - 1], lo.X[L],
+                                       lo.labels, lo.mask, lo.loss, lo.pred, nullptr, s);
+        } else {
+            ctx->loss_train_rows_only = rows_only ? 1 : keep;
+            st = mixgcn_loss_softmax_xent(ctx, n, dims[L], lo.X[L], round4(dims[L]), lo.labels, lo.mask, lo.loss,
+                                          lo.X[L], pred ? lo.pred : nullptr, nullptr, s);
+        }
         ctx->loss_train_rows_only = keep;
         MIXGCN_TRY(st);
+        if (one_call && L == 1) MIXGCN_TRY(after_first_layer());
     }
+    if (pf) pf->announced = nullptr;
     for (int l = L - 1; l >= 0; --l) {
         MIXGCN_TRY(mixgcn_layer_bwd(ctx, g, &lo.desc[l], lo.X[l], lo.saved[l], lo.X[l + 1], nullptr, lo.W[l], lo.G[l + 1],
                                     l > 0 ? lo.G[l] : nullptr, lo.dW[l], lo.db[l], s));

@@ -82,6 +82,8 @@ struct mixgcn_ctx {
     cudaStream_t side_stream[2];
     cudaEvent_t fork_ev, join_ev[2];
     cudaEvent_t chunk_ev[64];
+    void* workspace_loss;     // scratch of the loss taken inside a layer's last kernel (count, partial sums, per-row terms): its own
+    int64_t workspace_loss_bytes;   // block, because the product that takes the loss packs its weights into `workspace`
     void* workspace_lp;       // bf16 copies of fp32 operands converted on the fly (BF16 products whose caller gave no copy)
     int64_t workspace_lp_bytes;
     int64_t gemm_path[3];     // dense products served by: 0 fp32 FMA kernel, 1 tcgen05 TF32, 2 tcgen05 BF16
@@ -202,7 +204,25 @@ struct SpmmRowSparse {
 // kernels' host launchers (all asynchronous on `s`)
 // Aggregation over all rows (chunks <= 1) or over chunk k of `chunks` row chunks.
 // Optional behaviour of one aggregation call.
+// The loss taken inside the aggregation that produces the logits (last layer in upd-first order): each row's
+// soft-max, arg-max, loss term and gradient are computed from the registers that hold the aggregated row, so
+// the logits are never written.  Filled by loss_fuse_begin (count of train nodes, per-row loss scratch).
+struct LossFuse {
+    const int32_t* labels = nullptr;
+    const uint8_t* train_mask = nullptr;
+    const unsigned long long* count = nullptr;   // device: number of train nodes
+    float* row_loss = nullptr;                   // device [n]: lse - logit[label] of every train row
+    int32_t* pred = nullptr;                     // device [n]
+    int zero_rows = 1;                           // 1: rows outside the train mask receive a zero gradient; 0: they are left alone
+    double* part = nullptr;                      // device: partial sums of the final pass
+    int n_part = 0;
+};
+mixgcn_status loss_fuse_begin(mixgcn_ctx* ctx, int64_t n, const int32_t* labels, const uint8_t* train_mask, int32_t* pred,
+                              int64_t* n_correct, cudaStream_t s, LossFuse* out);
+mixgcn_status loss_fuse_end(mixgcn_ctx* ctx, int64_t n, int32_t C, const LossFuse& lf, float* loss, int64_t* n_correct, cudaStream_t s);
+
 struct SpmmOpts {
+    const LossFuse* loss = nullptr;          // non-null: soft-max cross-entropy epilogue (width <= 256, bias only); Z receives the gradient
     const SpmmRowSparse* sparse = nullptr;   // row-sparse input: test the input's row mask inside the kernel
     const uint8_t* row_filter = nullptr;     // compute only the output rows whose byte is non-zero (not with `sparse`)
     int phase = PH_SPMM;                     // profiling phase the launches are booked under
@@ -228,6 +248,9 @@ void release_view(CsrView& v);
 // Leading dimensions in bf16 elements, multiples of 8; pointers 16-byte aligned.
 struct GemmLP {
     bool a_fp32_missing = false;      // the fp32 A holds no data (only its bf16 copy was written): no fallback below bf16
+    const LossFuse* loss = nullptr;   // K-major form, N <= 256, C = logits of a masked loss: the epilogue writes every row's arg-max to
+                                      // loss->pred and only the rows of loss->train_mask to C (the others zeroed if loss->zero_rows, else
+                                      // left alone); MIXGCN_EUNSUPPORTED, nothing computed, if no tensor-core kernel takes the product
     const uint16_t* A = nullptr; int64_t lda = 0;
     const uint16_t* B = nullptr; int64_t ldb = 0;
     uint16_t* C = nullptr; int64_t ldc = 0;
@@ -242,7 +265,7 @@ mixgcn_status launch_gemm_simt(mixgcn_ctx* ctx, int ta, int tb, int64_t M, int64
 mixgcn_status launch_gemm_tc(mixgcn_ctx* ctx, int kind, int ta, int tb, int64_t M, int64_t N, int64_t K, const void* A,
                              int64_t lda, const void* B, int64_t ldb, float* C, int64_t ldc,
                              const mixgcn_epilogue* epi, int64_t epi_row0, cudaStream_t s, uint16_t* C_lp, int64_t ldc_lp,
-                             float* colsum_b = nullptr, bool* colsum_done = nullptr);
+                             float* colsum_b = nullptr, bool* colsum_done = nullptr, const LossFuse* loss = nullptr);
 mixgcn_status launch_splitk_reduce(mixgcn_ctx* ctx, int64_t M, int64_t N, int splits, const float* part, float* C,
                                    int64_t ldc, const mixgcn_epilogue* epi, cudaStream_t s);
 mixgcn_status launch_to_bf16(mixgcn_ctx* ctx, int64_t rows, int32_t d, const float* src, int64_t ld_src, uint16_t* dst,

@@ -500,6 +500,42 @@ __global__ void loss_final_kernel(int blocks, const double* __restrict__ part,
     *loss = (float)(t / (double)T);
 }
 
+// Final pass of the loss taken inside the aggregation: the per-row terms of the train rows are added in row
+// order (block b owns rows [b * chunk, (b + 1) * chunk), its threads stride through them, fixed-order tree
+// within the block, blocks added in order by loss_final_kernel), and the correct predictions are counted.
+constexpr int FUSE_REDUCE_THREADS = 256;
+__global__ void __launch_bounds__(FUSE_REDUCE_THREADS) loss_rows_reduce_kernel(
+    int64_t n, int C, int64_t chunk, const uint8_t* __restrict__ mask, const int32_t* __restrict__ labels,
+    const float* __restrict__ row_loss, const int32_t* __restrict__ pred, double* __restrict__ part,
+    unsigned long long* n_correct) {
+    __shared__ double sm[FUSE_REDUCE_THREADS];
+    __shared__ unsigned int sc[FUSE_REDUCE_THREADS / 32];
+    const int64_t r0 = (int64_t)blockIdx.x * chunk, r1 = r0 + chunk < n ? r0 + chunk : n;
+    double local = 0.0;
+    unsigned int correct = 0;
+    for (int64_t v = r0 + threadIdx.x; v < r1; v += FUSE_REDUCE_THREADS) {
+        if (!mask[v]) continue;
+        const int y = labels[v];
+        if (y < 0 || y >= C) continue;            // reported by the aggregation's epilogue; contributes nothing
+        local += (double)row_loss[v];
+        if (pred && pred[v] == y) ++correct;
+    }
+    sm[threadIdx.x] = local;
+    for (int o = 16; o > 0; o >>= 1) correct += __shfl_down_sync(0xFFFFFFFFu, correct, o);
+    if ((threadIdx.x & 31) == 0) sc[threadIdx.x >> 5] = correct;
+    __syncthreads();
+    for (int half = FUSE_REDUCE_THREADS / 2; half > 0; half >>= 1) {
+        if (threadIdx.x < half) sm[threadIdx.x] += sm[threadIdx.x + half];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        part[blockIdx.x] = sm[0];
+        unsigned int t = 0;
+        for (int w = 0; w < FUSE_REDUCE_THREADS / 32; ++w) t += sc[w];
+        if (n_correct && t) atomicAdd(n_correct, (unsigned long long)t);   // integer: order does not matter
+    }
+}
+
 constexpr int ADAM_MAX_TENSORS = 16;
 struct AdamBatch {
     float* p[ADAM_MAX_TENSORS];
@@ -528,6 +564,62 @@ __global__ void adam_kernel(const AdamBatch b) {
 }
 
 }  // namespace
+
+namespace mixgcn {
+
+// Scratch of the fused loss (a block of its own): [count u64][pad][partials double[blocks]][row_loss float[n]].
+// Counts the train nodes (the gradient's 1/#T is needed inside the kernel that takes the loss) and clears n_correct.
+mixgcn_status loss_fuse_begin(mixgcn_ctx* ctx, int64_t n, const int32_t* labels, const uint8_t* train_mask, int32_t* pred,
+                              int64_t* n_correct, cudaStream_t s, LossFuse* out) {
+    const int64_t cap = (int64_t)ctx->sm_count * 16;
+    int64_t blocks = (n + 4095) / 4096;
+    if (blocks > cap) blocks = cap;
+    const int64_t off_rows = (16 + blocks * (int64_t)sizeof(double) + 255) & ~(int64_t)255;
+    const int64_t need = off_rows + n * (int64_t)sizeof(float);
+    if (need > ctx->workspace_loss_bytes) {
+        MIXGCN_CUDA(cudaDeviceSynchronize());      // the old block may still be in use by enqueued kernels
+        cudaFree(ctx->workspace_loss);
+        ctx->workspace_loss = nullptr; ctx->workspace_loss_bytes = 0;
+        void* q = nullptr;
+        if (cudaMalloc(&q, (size_t)need) != cudaSuccess) {
+            cudaGetLastError();
+            MIXGCN_FAIL(MIXGCN_ENOMEM, "loss scratch of %lld bytes could not be allocated", (long long)need);
+        }
+        ctx->workspace_loss = q; ctx->workspace_loss_bytes = need;
+    }
+    char* base = reinterpret_cast<char*>(ctx->workspace_loss);
+    unsigned long long* count = reinterpret_cast<unsigned long long*>(base);
+    MIXGCN_CUDA(cudaMemsetAsync(count, 0, sizeof(unsigned long long), s));
+    if (n_correct) MIXGCN_CUDA(cudaMemsetAsync(n_correct, 0, sizeof(int64_t), s));
+    {
+        LaunchScope scope(ctx, PH_LOSS, s);
+        int64_t cb = (n + 255) / 256; if (cb > cap) cb = cap;
+        count_mask_kernel<<<(unsigned)cb, 256, 0, s>>>(n, train_mask, count);
+    }
+    MIXGCN_CUDA(cudaGetLastError());
+    out->labels = labels; out->train_mask = train_mask; out->count = count; out->pred = pred;
+    out->part = reinterpret_cast<double*>(base + 16); out->n_part = (int)blocks;
+    out->row_loss = reinterpret_cast<float*>(base + off_rows);
+    out->zero_rows = ctx->loss_train_rows_only == 2 ? 0 : 1;
+    return MIXGCN_OK;
+}
+
+mixgcn_status loss_fuse_end(mixgcn_ctx* ctx, int64_t n, int32_t C, const LossFuse& lf, float* loss, int64_t* n_correct, cudaStream_t s) {
+    const int64_t chunk = (n + lf.n_part - 1) / lf.n_part;
+    {
+        LaunchScope scope(ctx, PH_LOSS, s);
+        loss_rows_reduce_kernel<<<(unsigned)lf.n_part, FUSE_REDUCE_THREADS, 0, s>>>(n, C, chunk, lf.train_mask, lf.labels, lf.row_loss, lf.pred, lf.part,
+                                                                                  reinterpret_cast<unsigned long long*>(n_correct));
+    }
+    {
+        LaunchScope scope(ctx, PH_LOSS, s);
+        loss_final_kernel<<<1, 32, 0, s>>>(lf.n_part, lf.part, lf.count, loss, ctx->d_status);
+    }
+    MIXGCN_CUDA(cudaGetLastError());
+    return MIXGCN_OK;
+}
+
+}  // namespace mixgcn
 
 extern "C" mixgcn_status mixgcn_loss_softmax_xent(mixgcn_ctx* ctx, int64_t n, int32_t C, const float* logits,
                                                   int64_t ld, const int32_t* labels, const uint8_t* train_mask,

@@ -64,6 +64,9 @@ struct SpmmParams {
     const uint8_t* drop; float keep_scale;
     const float* gate; int64_t ld_gate; float gate_scale;
     const float* residual; int64_t ld_residual; float residual_scale;
+    // loss epilogue (kernels instantiated with LOSS): labels, train mask, number of train nodes, per-row loss, arg-max
+    const int32_t* loss_labels; const uint8_t* loss_mask; const unsigned long long* loss_count;
+    float* loss_row; int32_t* loss_pred; int loss_zero_rows;
     // limits for the index tests of the bounds-checked debug build (unused otherwise)
     int32_t* status;
     int64_t n_cols;        // column ids lie in [0, n_cols) (they index in_mask / in_pos, or Y itself)
@@ -124,6 +127,89 @@ __device__ __forceinline__ void fma4(float4& acc, float a, const float4& y) {
     acc.z = fmaf(a, y.z, acc.z); acc.w = fmaf(a, y.w, acc.w);
 }
 
+// Soft-max cross-entropy of output row u taken from the registers that hold the aggregated row (the whole
+// row belongs to one group of LPR lanes, lane `lig` holding float4 groups lig + v * LPR): logits = sums + bias;
+// arg-max with lowest-index ties -> pred; on a train row the loss term lse - logit[label] -> loss_row[u] and the
+// gradient (softmax - e_label) / #T -> Z row u.  The logits themselves are never written.
+template <int LPR, int VPL>
+__device__ __forceinline__ void loss_epilogue(const SpmmParams& p, int64_t u, int lig, unsigned mask, const float4 (&acc)[VPL]) {
+    const int C = p.w;                 // one slice: j0 == 0
+    const int w4 = (C + 3) >> 2;
+    float x[VPL][4];
+#pragma unroll
+    for (int v = 0; v < VPL; ++v) {
+        const int j = (lig + v * LPR) * 4;
+        const float a[4] = {acc[v].x, acc[v].y, acc[v].z, acc[v].w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) x[v][e] = j + e < C ? (p.bias ? a[e] + __ldg(p.bias + j + e) : a[e]) : -INFINITY;
+    }
+    float mx = -INFINITY; int arg = 0x7FFFFFFF;
+#pragma unroll
+    for (int v = 0; v < VPL; ++v)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int c = (lig + v * LPR) * 4 + e;
+            if (c < C && (x[v][e] > mx || (x[v][e] == mx && c < arg))) { mx = x[v][e]; arg = c; }
+        }
+    if (arg == 0x7FFFFFFF) arg = lig * 4 < C ? lig * 4 : 0;       // nothing but -inf / NaN in this lane's columns
+#pragma unroll
+    for (int o = LPR / 2; o > 0; o >>= 1) {
+        const float omx = __shfl_xor_sync(mask, mx, o, LPR);
+        const int oarg = __shfl_xor_sync(mask, arg, o, LPR);
+        if (omx > mx || (omx == mx && oarg < arg)) { mx = omx; arg = oarg; }
+    }
+    if (p.loss_pred && lig == 0) p.loss_pred[u] = arg;
+    const unsigned long long T = *p.loss_count;
+    const bool train = __ldg(p.loss_mask + u) != 0 && T != 0;
+    int y = 0; bool ok = false;
+    if (train) {
+        y = __ldg(p.loss_labels + u);
+        ok = y >= 0 && y < C;
+        if (!ok && lig == 0) atomicMax(p.status, DEV_BAD_LABEL);
+    }
+    if (!train || !ok) {
+        if (p.loss_zero_rows || train) {
+#pragma unroll
+            for (int v = 0; v < VPL; ++v) {
+                const int c4 = lig + v * LPR;
+                if (c4 < w4) *reinterpret_cast<float4*>(p.Z + u * p.ldz + c4 * 4) = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+        }
+        return;
+    }
+    float s = 0.0f;
+#pragma unroll
+    for (int v = 0; v < VPL; ++v)
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+            if ((lig + v * LPR) * 4 + e < C) s += expf(x[v][e] - mx);
+#pragma unroll
+    for (int o = LPR / 2; o > 0; o >>= 1) s += __shfl_xor_sync(mask, s, o, LPR);
+    const float lse = mx + logf(s);
+    float py = 0.0f;        // the label's logit lives in lane (y/4) % LPR of the group
+#pragma unroll
+    for (int v = 0; v < VPL; ++v)
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+            if ((lig + v * LPR) * 4 + e == y) py = x[v][e];
+    py = __shfl_sync(mask, py, (y >> 2) & (LPR - 1), LPR);
+    if (lig == 0) p.loss_row[u] = lse - py;
+    const float invT = (float)(1.0 / (double)T);
+#pragma unroll
+    for (int v = 0; v < VPL; ++v) {
+        const int c4 = lig + v * LPR;
+        if (c4 < w4) {
+            float r[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int c = c4 * 4 + e;
+                r[e] = c < C ? (expf(x[v][e] - lse) - (c == y ? 1.0f : 0.0f)) * invT : 0.0f;
+            }
+            *reinterpret_cast<float4*>(p.Z + u * p.ldz + c4 * 4) = make_float4(r[0], r[1], r[2], r[3]);
+        }
+    }
+}
+
 template <int LPR, int VPL>
 struct Cfg {
     static constexpr int U0 = SPMM_U / VPL < 1 ? 1 : SPMM_U / VPL;
@@ -172,7 +258,7 @@ __device__ __forceinline__ void row_segment(const SpmmParams& p, int64_t b, int6
     }
 }
 
-template <int LPR, int VPL>
+template <int LPR, int VPL, bool LOSS = false>
 __global__ void __launch_bounds__(256, VPL <= 2 ? SPMM_MINB : 1) spmm_group_kernel(const SpmmParams p) {
     const int lig = threadIdx.x % LPR;
     const int64_t idx = p.idx_begin + ((int64_t)blockIdx.x * 256 + threadIdx.x) / LPR;
@@ -217,6 +303,10 @@ __global__ void __launch_bounds__(256, VPL <= 2 ? SPMM_MINB : 1) spmm_group_kern
             const int c4 = lig + v * LPR;
             if (c4 < w4) dst[c4] = acc[v];
         }
+        return;
+    }
+    if constexpr (LOSS) {
+        loss_epilogue<LPR, VPL>(p, u, lig, mask, acc);
         return;
     }
 #pragma unroll
@@ -412,6 +502,7 @@ __global__ void __launch_bounds__(256) spmm_filtered_kernel(const SpmmParams p) 
 
 // Long rows: add the segments' partial rows in entry order, apply the epilogue, write Z.
 // One group of 32 lanes per long row.
+template <bool LOSS = false>
 __global__ void __launch_bounds__(256) spmm_combine_kernel(const SpmmParams p, int64_t n_long,
                                                            const int64_t* __restrict__ seg_off,
                                                            const int64_t* __restrict__ seg_pos,
@@ -426,6 +517,25 @@ __global__ void __launch_bounds__(256) spmm_combine_kernel(const SpmmParams p, i
     if (p.row_filter && !__ldg(p.row_filter + u)) return;
     const int w4 = (p.w + 3) >> 2;
     if (p.out_mask && lane == 0) p.out_mask[u] = 1;    // long rows are kept without looking (conservative)
+    if constexpr (LOSS) {
+        // the whole row (at most 64 float4) in registers, then the same epilogue as the other rows
+        float4 row[2];
+#pragma unroll
+        for (int v = 0; v < 2; ++v) {
+            const int c4 = lane + v * 32;
+            float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (c4 < w4)
+                for (int64_t q = s0; q < s1; ++q) {
+                    const int64_t slot = __ldg(seg_pos + q);
+                    if (!index_ok(slot, p.n_partial, p.status, SITE_SPMM_SEG)) continue;
+                    const float4 t = __ldg(reinterpret_cast<const float4*>(p.partial + slot * p.ldp) + c4);
+                    s.x += t.x; s.y += t.y; s.z += t.z; s.w += t.w;
+                }
+            row[v] = s;
+        }
+        loss_epilogue<32, 2>(p, u, lane, 0xFFFFFFFFu, row);
+        return;
+    }
     for (int c4 = lane; c4 < w4; c4 += 32) {
         float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
         for (int64_t q = s0; q < s1; ++q) {
@@ -438,13 +548,33 @@ __global__ void __launch_bounds__(256) spmm_combine_kernel(const SpmmParams p, i
     }
 }
 
-template <int LPR, int VPL>
+template <int LPR, int VPL, bool LOSS = false>
 void launch_group(const SpmmParams& p, cudaStream_t s) {
     const int64_t units = p.idx_end - p.idx_begin;
     if (units <= 0) return;
     const int per_block = 256 / LPR;
     const int64_t blocks = (units + per_block - 1) / per_block;
-    spmm_group_kernel<LPR, VPL><<<(unsigned)blocks, 256, 0, s>>>(p);
+    spmm_group_kernel<LPR, VPL, LOSS><<<(unsigned)blocks, 256, 0, s>>>(p);
+}
+
+// The same packing for an aggregation with the loss epilogue (width <= 256: at most two float4 per lane
+// before folding).  Returns 0 if the shape has no instance.
+int dispatch_loss(const SpmmParams& p, int fold, cudaStream_t s) {
+    const int w4 = (p.w + 3) >> 2;
+    int lpr = 1;
+    while (lpr < 32 && lpr < w4) lpr <<= 1;
+    int vpl = (w4 + lpr - 1) / lpr;
+    while (fold > 1 && (lpr / fold < 1 || vpl * fold > 8)) fold >>= 1;
+    lpr /= fold; vpl *= fold;
+#define MIXGCN_SPMM_CASE(L, V) if (lpr == L && vpl == V) { launch_group<L, V, true>(p, s); return fold; }
+    MIXGCN_SPMM_CASE(32, 1) MIXGCN_SPMM_CASE(32, 2)
+    MIXGCN_SPMM_CASE(16, 1) MIXGCN_SPMM_CASE(16, 2) MIXGCN_SPMM_CASE(16, 4)
+    MIXGCN_SPMM_CASE(8, 1) MIXGCN_SPMM_CASE(8, 2) MIXGCN_SPMM_CASE(8, 4) MIXGCN_SPMM_CASE(8, 8)
+    MIXGCN_SPMM_CASE(4, 1) MIXGCN_SPMM_CASE(4, 2) MIXGCN_SPMM_CASE(4, 4) MIXGCN_SPMM_CASE(4, 8)
+    MIXGCN_SPMM_CASE(2, 1) MIXGCN_SPMM_CASE(2, 2) MIXGCN_SPMM_CASE(2, 4) MIXGCN_SPMM_CASE(2, 8)
+    MIXGCN_SPMM_CASE(1, 1) MIXGCN_SPMM_CASE(1, 2) MIXGCN_SPMM_CASE(1, 4) MIXGCN_SPMM_CASE(1, 8)
+#undef MIXGCN_SPMM_CASE
+    return 0;
 }
 
 // Base configuration for a slice of w4 float4 columns, then packed `fold`-fold (fold in {1,2,4,8}):
@@ -521,12 +651,18 @@ mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView&
                           int32_t w, const float* Y, int64_t ldy, float* Z, int64_t ldz,
                           const mixgcn_epilogue* epi, cudaStream_t s, const SpmmOpts& opts) {
     const SpmmRowSparse* sparse = opts.sparse;
+    const LossFuse* lf = opts.loss;
     const uint8_t* row_filter = opts.row_filter;
     const int phase = opts.phase;
     const int64_t row_limit = opts.row_limit;
     if (w <= 0) return MIXGCN_OK;
     if (!Z && !opts.Z_lp) MIXGCN_FAIL(MIXGCN_EINVAL, "spmm: no output");
     if (sparse && row_filter) MIXGCN_FAIL(MIXGCN_EUNSUPPORTED, "spmm: a row filter cannot be combined with a row-sparse input");
+    if (lf) {
+        if (sparse || row_filter || chunks > 1 || opts.out_bits || opts.Z_lp || opts.row_limit >= 0 || !Z || w > 256 ||
+            (epi && (epi->relu || epi->drop_mask || epi->gate || epi->residual)))
+            MIXGCN_FAIL(MIXGCN_EUNSUPPORTED, "spmm: the loss epilogue takes a plain aggregation of at most 256 columns with a bias");
+    }
     if (chunks > 1) {
         MIXGCN_TRY(ensure_chunk_schedules(g, A, chunks));
         if (k < 0 || k >= A.n_chunk) MIXGCN_FAIL(MIXGCN_EINVAL, "spmm: chunk %d of %d does not exist", k, chunks);
@@ -550,7 +686,11 @@ mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView&
     p.rec = S.rec;
     if (sparse) { p.in_mask = sparse->in_mask; p.in_pos = sparse->in_pos; p.out_mask = sparse->out_mask; }
     p.row_filter = row_filter;
-    const int slice = ctx->spmm_slice_cols > 0 ? (ctx->spmm_slice_cols < MAX_SLICE ? ctx->spmm_slice_cols : MAX_SLICE) : DEFAULT_SLICE;
+    if (lf) {
+        p.loss_labels = lf->labels; p.loss_mask = lf->train_mask; p.loss_count = lf->count;
+        p.loss_row = lf->row_loss; p.loss_pred = lf->pred; p.loss_zero_rows = lf->zero_rows;
+    }
+    const int slice = lf ? MAX_SLICE : ctx->spmm_slice_cols > 0 ? (ctx->spmm_slice_cols < MAX_SLICE ? ctx->spmm_slice_cols : MAX_SLICE) : DEFAULT_SLICE;
     for (int j0 = 0; j0 < w; j0 += slice) {
         p.j0 = j0;
         p.w = (w - j0) < slice ? (w - j0) : slice;
@@ -568,7 +708,7 @@ mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView&
                 {
                     LaunchScope scope(ctx, PH_SPMM_SPARSE, s);
                     const int64_t blocks = (S.n_long * 32 + 255) / 256;
-                    spmm_combine_kernel<<<(unsigned)blocks, 256, 0, s>>>(p, S.n_long, S.seg_off, S.seg_pos, S.perm);
+                    spmm_combine_kernel<false><<<(unsigned)blocks, 256, 0, s>>>(p, S.n_long, S.seg_off, S.seg_pos, S.perm);
                 }
                 p.partial = nullptr;
             }
@@ -608,7 +748,7 @@ mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView&
                 {
                     LaunchScope scope(ctx, PH_SPMM_SPARSE, s);
                     const int64_t blocks = (S.n_long * 32 + 255) / 256;
-                    spmm_combine_kernel<<<(unsigned)blocks, 256, 0, s>>>(p, S.n_long, S.seg_off, S.seg_pos, S.perm);
+                    spmm_combine_kernel<false><<<(unsigned)blocks, 256, 0, s>>>(p, S.n_long, S.seg_off, S.seg_pos, S.perm);
                 }
                 p.partial = nullptr;
             }
@@ -633,7 +773,8 @@ mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView&
             {
                 LaunchScope scope(ctx, phase, s);
                 const int64_t blocks = (S.n_long * 32 + 255) / 256;
-                spmm_combine_kernel<<<(unsigned)blocks, 256, 0, s>>>(p, S.n_long, S.seg_off, S.seg_pos, S.perm);
+                if (lf) spmm_combine_kernel<true><<<(unsigned)blocks, 256, 0, s>>>(p, S.n_long, S.seg_off, S.seg_pos, S.perm);
+                else spmm_combine_kernel<false><<<(unsigned)blocks, 256, 0, s>>>(p, S.n_long, S.seg_off, S.seg_pos, S.perm);
             }
             p.partial = nullptr;
         }
@@ -655,7 +796,9 @@ mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView&
             p.idx_begin = S.total_segs + (begin - S.n_long);
             p.idx_end = S.total_segs + (end - S.n_long);
             LaunchScope scope(ctx, phase, s);
-            if (q == 3 && p.w <= 128 && SPMM_PACK_DEG[2] <= SPMM_SHORT_MAXE) {
+            if (lf) {
+                if (!dispatch_loss(p, q == 0 ? (p.w <= SPMM_FOLD_WMAX ? SPMM_FOLD_MED : 1) : fold, s)) MIXGCN_FAIL(MIXGCN_EUNSUPPORTED, "spmm: no loss-epilogue kernel for width %d", p.w);
+            } else if (q == 3 && p.w <= 128 && SPMM_PACK_DEG[2] <= SPMM_SHORT_MAXE) {
                 // rows of at most SPMM_PACK_DEG[2] entries: several rows per warp, whole-warp gathers
                 constexpr int RB = SPMM_SHORT_RB, MAXE = SPMM_SHORT_MAXE;
                 const int64_t units = p.idx_end - p.idx_begin;

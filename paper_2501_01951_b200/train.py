@@ -197,11 +197,39 @@ class GcnTrainer:
                     d.gin_row_mask = self.row_masks[l].data_ptr()
 
     # -- the iteration --------------------------------------------------------------------------
-    def forward(self):
+    def last_layer_takes_the_loss(self):
+        """Whether forward_and_loss() hands the last layer and the loss to ONE library call (which takes the loss
+        where the logits are produced, without writing them, wherever its kernels can)."""
+        return self.masks[self.L - 1] is None and not self.train_rows_only
+
+    def forward_and_loss(self):
+        """forward() + compute_loss() with the same results; X[L] then holds the gradient w.r.t. the logits."""
+        if not self.last_layer_takes_the_loss():
+            self.forward()
+            self.compute_loss()
+            return
+        L = self.L
+        self.forward(upto=L - 1)
+        d = self.descs[L - 1]
+        d.flags &= ~(mg.LAYER_SAVED_LP_ONLY | mg.LAYER_SAVED_IS_VALID)
+        # rows the backward never reads need no zeros (same rule as compute_loss)
+        leave = self.row_plans[L - 1] is not None
+        if leave:
+            mg.ctx_set_option(self.ctx, mg.OPT_LOSS_TRAIN_ROWS_ONLY, 2)
+        try:
+            mg.layer_fwd_loss(self.ctx, self.g, d, self.X[L - 1], self.W[L - 1], self.b[L - 1], self.saved[L - 1],
+                              self.X[L], self.labels, self.train_mask, self.loss, self.pred, self.n_correct)
+        finally:
+            if leave:
+                mg.ctx_set_option(self.ctx, mg.OPT_LOSS_TRAIN_ROWS_ONLY, 0)
+        if L == 1:
+            self._first_aggregation_valid = self.orders[0] == mg.ORDER_AGG_FIRST
+
+    def forward(self, upto=None):
         d0 = self.descs[0]
         reuse = self.cache_first_aggregation and self._first_aggregation_valid and self.orders[0] == mg.ORDER_AGG_FIRST
         d0.flags = (d0.flags | mg.LAYER_SAVED_IS_VALID) if reuse else (d0.flags & ~mg.LAYER_SAVED_IS_VALID)
-        for l in range(self.L):
+        for l in range(self.L if upto is None else upto):
             d = self.descs[l]
             lp_only = (self.saved_lp_only and self.orders[l] == mg.ORDER_AGG_FIRST and not d.gout_row_mask and not d.gout_plan
                        and not (d.flags & (mg.LAYER_OUT_ROWS_ONLY | mg.LAYER_SAVED_IS_VALID))
@@ -261,7 +289,6 @@ class GcnTrainer:
                      lr, beta1, beta2, eps)
 
     def epoch(self, t, lr=0.01):
-        self.forward()
-        self.compute_loss()
+        self.forward_and_loss()
         self.backward()
         self.step(t, lr)

@@ -232,6 +232,26 @@ def test_full_size_workload(mg, key):
     for t in tr.dW + tr.db:
         assert bool(torch.isfinite(t).all())
 
+    # ---- the iteration as the benchmark runs it: the loss taken inside the last layer's aggregation (no logits
+    # written).  Its logits are the same fp32 numbers, so the predictions must be the separate calls' bit for bit.
+    if tr.last_layer_takes_the_loss():
+        ref_pred, ref_nc = tr.pred.clone(), int(tr.n_correct.item())
+        grad_rows = train_idx[torch.as_tensor(pick, device="cuda")]
+        tr.pred.fill_(-7); tr.X[L].fill_(float("nan"))
+        tr.forward_and_loss()
+        torch.cuda.synchronize()
+        assert mg.ctx_poll_status(ctx, raise_on_error=False) == 0
+        assert abs(tr.loss.item() - lo) <= 2e-6 * abs(lo)
+        assert torch.equal(tr.pred, ref_pred) and int(tr.n_correct.item()) == ref_nc
+        assert _rel(tr.X[L][grad_rows][:, :C].cpu().numpy(), Gt[pick]) <= TOL_FP32
+        if tr.row_plans[L - 1] is None:
+            assert float(tr.X[L][untrained][:, :C].abs().max()) == 0.0
+        tr.backward()
+        torch.cuda.synchronize()
+        for k in range(L):
+            assert _rel(tr.dW[k].double().cpu().numpy(), ref_dW[k].cpu().numpy()) <= tol, f"dW[{k}] with the loss inside the aggregation"
+            assert _rel(tr.db[k].double().cpu().numpy(), ref_db[k].cpu().numpy()) <= TOL_FP32 * 10, f"db[{k}] with the loss inside the aggregation"
+
     # ---- the train-rows-only shortcut at full size: same loss and gradients as the full computation
     # above; rows outside the train mask hold NaN beforehand, so reading one of them would show
     ref_loss, ref_dW, ref_db = tr.loss.item(), [t.clone() for t in tr.dW], [t.clone() for t in tr.db]

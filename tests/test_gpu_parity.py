@@ -575,7 +575,7 @@ def test_train_step_host_matches_oracle_and_device_path(mg, ctx):
     tr.set_inputs(padded(X), y.cuda(), m.cuda())
     for t in (1, 2):
         loss = mg.train_step_host(ctx, gg, wl.dims, mg.PREC_FP32, X, y, m, W, b, mW, vW, mb, vb, t, pred=pred, **ADAM)
-        tr.forward(); tr.compute_loss(); tr.backward(); tr.step(t, **ADAM)
+        tr.forward_and_loss(); tr.backward(); tr.step(t, **ADAM)      # the iteration as epoch() runs it
         assert loss == tr.loss.item()
         for l in range(tr.L):
             assert torch.equal(W[l], tr.W[l].cpu()) and torch.equal(b[l], tr.b[l].cpu())
