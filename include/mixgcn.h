@@ -228,6 +228,18 @@ typedef struct {
     const float* residual;
     int64_t ld_residual;
     float residual_scale;
+    /* Bit-packed masks (the bitmap mask buffer of Section 3.2.1): n x ld words of 32 bits, bit (j & 31) of
+     * word [i*ld + (j >> 5)] belongs to element (i, j); ld >= ceil(d / 32).
+     *   gate_bits  (nullable) stands in for `gate` (which is then ignored): set bit = y*gate_scale, clear bit = 0.
+     *   sign_bits  (nullable) is an OUTPUT: receives bit = (final y > 0) for every element, bits of columns
+     *              >= d in a row's last word are cleared.  With relu this is the mask a later gate_bits reads
+     *              -- 1 bit per element instead of re-reading the fp32 tensor.  Written by the kernel that
+     *              produces y where it can, else by one more pass over the result.
+     * K-major / plain products and aggregations only (mixgcn_gemm with trans_a = 1 rejects both). */
+    const uint32_t* gate_bits;
+    int64_t ld_gate_bits;
+    uint32_t* sign_bits;
+    int64_t ld_sign_bits;
 } mixgcn_epilogue;
 
 /* Neighbour aggregation Z = A_hat Y (transposed != 0: A_hat^T Y), n x w (Algorithm 2,
@@ -366,6 +378,17 @@ typedef struct {
     int64_t ld_out_lp;
     uint16_t* g_out_lp;
     uint16_t* g_in_lp;
+    /* Sign bitmaps of the activations (optional; the bitmap mask buffer of Section 3.2.1 for the ReLU masks the
+     * backward pass applies -- Eq. 4's M): device uint32, n rows of ld words, bit (j & 31) of word (j >> 5) of a
+     * row = (activation > 0).
+     *   x_out_bits  n x ld_out_bits (>= ceil(d_out / 32)): with MIXGCN_LAYER_RELU, layer_fwd also writes the bitmap
+     *               of X_out (after ReLU and dropout) -- the x_in_bits of the layer above
+     *   x_in_bits   n x ld_in_bits (>= ceil(d_in / 32)): with MIXGCN_LAYER_GATE_GIN, layer_bwd reads the gate from
+     *               this bitmap instead of the sign of X_in: one bit per element instead of four bytes */
+    uint32_t* x_out_bits;
+    int64_t ld_out_bits;
+    const uint32_t* x_in_bits;
+    int64_t ld_in_bits;
 } mixgcn_layer_desc;
 
 /* Row plan of a row-sparse aggregation.  Which rows of a gradient are non-zero depends on the graph

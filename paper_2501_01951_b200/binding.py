@@ -58,7 +58,8 @@ class Epilogue(C.Structure):
     _fields_ = [("bias", C.c_void_p), ("relu", C.c_int32), ("drop_mask", C.c_void_p),
                 ("keep_scale", C.c_float), ("gate", C.c_void_p), ("ld_gate", C.c_int64),
                 ("gate_scale", C.c_float), ("residual", C.c_void_p), ("ld_residual", C.c_int64),
-                ("residual_scale", C.c_float)]
+                ("residual_scale", C.c_float), ("gate_bits", C.c_void_p), ("ld_gate_bits", C.c_int64),
+                ("sign_bits", C.c_void_p), ("ld_sign_bits", C.c_int64)]
 
 
 class LayerDesc(C.Structure):
@@ -68,7 +69,8 @@ class LayerDesc(C.Structure):
                 ("n_chunks", C.c_int32), ("gout_row_mask", C.c_void_p), ("gout_row_count", C.c_int64),
                 ("gin_row_mask", C.c_void_p), ("gout_plan", C.c_void_p),
                 ("saved_lp", C.c_void_p), ("ld_saved_lp", C.c_int64), ("x_in_lp", C.c_void_p), ("ld_in_lp", C.c_int64),
-                ("x_out_lp", C.c_void_p), ("ld_out_lp", C.c_int64), ("g_out_lp", C.c_void_p), ("g_in_lp", C.c_void_p)]
+                ("x_out_lp", C.c_void_p), ("ld_out_lp", C.c_int64), ("g_out_lp", C.c_void_p), ("g_in_lp", C.c_void_p),
+                ("x_out_bits", C.c_void_p), ("ld_out_bits", C.c_int64), ("x_in_bits", C.c_void_p), ("ld_in_bits", C.c_int64)]
 
 
 lib.mixgcn_status_string.restype = C.c_char_p
@@ -299,7 +301,7 @@ def graph_create_permuted(ctx: Ctx, g: Graph, order: torch.Tensor) -> Graph:
 # ------------------------------------------------------------------------------ building blocks
 
 def make_epilogue(bias=None, relu=False, drop_mask=None, keep_scale=1.0, gate=None, gate_scale=1.0,
-                  residual=None, residual_scale=1.0):
+                  residual=None, residual_scale=1.0, gate_bits=None, sign_bits=None):
     e = Epilogue()
     e.bias = None if bias is None else _dev(bias, torch.float32, "bias").data_ptr()
     e.relu = int(relu)
@@ -313,7 +315,13 @@ def make_epilogue(bias=None, relu=False, drop_mask=None, keep_scale=1.0, gate=No
         residual, ldr = _mat(residual, "residual")
         e.residual, e.ld_residual = residual.data_ptr(), ldr
     e.residual_scale = residual_scale
-    e._keep = (bias, drop_mask, gate, residual)
+    for name, t in (("gate_bits", gate_bits), ("sign_bits", sign_bits)):      # n x ld words of 32 bits (torch int32)
+        if t is not None:
+            _dev(t, torch.int32, name)
+            if t.dim() != 2 or t.stride(1) != 1:
+                raise TypeError(f"{name}: expected a row-major 2-D int32 tensor")
+            setattr(e, name, t.data_ptr()); setattr(e, "ld_" + name, t.stride(0))
+    e._keep = (bias, drop_mask, gate, residual, gate_bits, sign_bits)
     return e
 
 

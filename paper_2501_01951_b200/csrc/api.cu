@@ -108,7 +108,8 @@ mixgcn_status launch_gemm(mixgcn_ctx* ctx, int precision, int ta, int tb, int64_
     uint16_t* c_lp = lp ? lp->C : nullptr;
     const int64_t ldc_lp = lp ? lp->ldc : 0;
     const LossFuse* loss = lp ? lp->loss : nullptr;
-    bool c_lp_done = false;
+    bool c_lp_done = false, bits_done = false;
+    if (ta && epi && (epi->gate_bits || epi->sign_bits)) MIXGCN_FAIL(MIXGCN_EINVAL, "gemm: bit-packed masks belong to the K-major form (trans_a = 0)");
     mixgcn_status st = MIXGCN_EUNSUPPORTED;
     const bool fp32_layout = aligned16(A) && (lda & 3) == 0 && (!ta || (aligned16(B) && (ldb & 3) == 0));
     if (precision == MIXGCN_PREC_BF16 && !(ta && tb) && fp32_layout && M > 0 && N > 0 && K > 0) {
@@ -135,7 +136,7 @@ mixgcn_status launch_gemm(mixgcn_ctx* ctx, int precision, int ta, int tb, int64_
             b_lp = dst;
         }
         st = launch_gemm_tc(ctx, 1, ta, tb, M, N, K, a_lp, lda_lp, ta ? (const void*)b_lp : (const void*)B, ta ? ldb_lp : ldb,
-                            C, ldc, epi, epi_row0, s, ta ? nullptr : c_lp, ldc_lp, nullptr, nullptr, loss);
+                            C, ldc, epi, epi_row0, s, ta ? nullptr : c_lp, ldc_lp, nullptr, nullptr, loss, &bits_done);
         if (st == MIXGCN_OK) { ctx->gemm_path[2]++; c_lp_done = !ta && c_lp; }
     }
     if (st == MIXGCN_EUNSUPPORTED && lp && lp->a_fp32_missing)
@@ -144,7 +145,7 @@ mixgcn_status launch_gemm(mixgcn_ctx* ctx, int precision, int ta, int tb, int64_
     if (colsum_b && !ta) MIXGCN_FAIL(MIXGCN_EINVAL, "gemm: column sums of B are a by-product of the weight-gradient form only");
     if (st == MIXGCN_EUNSUPPORTED && precision != MIXGCN_PREC_FP32) {
         st = launch_gemm_tc(ctx, 0, ta, tb, M, N, K, A, lda, B, ldb, C, ldc, epi, epi_row0, s, ta ? nullptr : c_lp, ldc_lp,
-                            colsum_b, &colsum_done, loss);
+                            colsum_b, &colsum_done, loss, &bits_done);
         if (st == MIXGCN_OK) { ctx->gemm_path[1]++; c_lp_done = !ta && c_lp; }
     }
     if (st == MIXGCN_EUNSUPPORTED && loss) return st;      // the caller runs the product and the loss separately
@@ -154,6 +155,9 @@ mixgcn_status launch_gemm(mixgcn_ctx* ctx, int precision, int ta, int tb, int64_
     }
     if (st != MIXGCN_OK) return st;
     if (c_lp && !c_lp_done) MIXGCN_TRY(launch_to_bf16(ctx, M, (int32_t)N, C, ldc, c_lp, ldc_lp, s));
+    // sign bitmap of the result where the kernel's epilogue did not write it: one more pass over C
+    if (epi && epi->sign_bits && !bits_done)
+        MIXGCN_TRY(launch_mask_pack(ctx, M, (int32_t)N, C, ldc, nullptr, epi->sign_bits + epi_row0 * epi->ld_sign_bits, epi->ld_sign_bits, s));
     if (colsum_b && !colsum_done) MIXGCN_TRY(launch_colsum(ctx, K, (int32_t)N, B, ldb, colsum_b, s));
     return MIXGCN_OK;
 }
@@ -340,6 +344,8 @@ extern "C" mixgcn_status mixgcn_gemm(mixgcn_ctx* ctx, int32_t precision, int32_t
                     (long long)lda, (long long)ldb, (long long)ldc);
     if (C == A || C == B) MIXGCN_FAIL(MIXGCN_EINVAL, "gemm: C must not overlap A or B");
     if (epi && epi->residual) MIXGCN_FAIL(MIXGCN_EUNSUPPORTED, "gemm: the residual term is an aggregation epilogue");
+    if (epi && ((epi->gate_bits && epi->ld_gate_bits < (N + 31) / 32) || (epi->sign_bits && epi->ld_sign_bits < (N + 31) / 32)))
+        MIXGCN_FAIL(MIXGCN_EINVAL, "gemm: a bit-packed mask needs ld >= ceil(N / 32) words");
     MIXGCN_CUDA(cudaSetDevice(ctx->device));
     return launch_gemm(ctx, precision, trans_a, trans_b, M, N, K, A, lda, B, ldb, C, ldc, epi, 0, (cudaStream_t)stream);
 }
@@ -374,6 +380,8 @@ mixgcn_status check_desc(const mixgcn_layer_desc* d, const char* who) {
     if (!lp_ok(d->saved_lp, d->ld_saved_lp, saved_cols) || !lp_ok(d->x_in_lp, d->ld_in_lp, d->d_in) || !lp_ok(d->g_in_lp, d->ld_in_lp, d->d_in) ||
         !lp_ok(d->x_out_lp, d->ld_out_lp, d->d_out) || !lp_ok(d->g_out_lp, d->ld_out_lp, d->d_out))
         MIXGCN_FAIL(MIXGCN_EINVAL, "%s: bf16 companions must be 16-byte aligned with leading dimensions that are multiples of 8 and cover the width", who);
+    if ((d->x_out_bits && d->ld_out_bits < (d->d_out + 31) / 32) || (d->x_in_bits && d->ld_in_bits < (d->d_in + 31) / 32))
+        MIXGCN_FAIL(MIXGCN_EINVAL, "%s: a sign bitmap needs ld >= ceil(width / 32) words", who);
     if (d->flags & MIXGCN_LAYER_SAVED_LP_ONLY) {
         if (order != MIXGCN_ORDER_AGG_FIRST || d->precision != MIXGCN_PREC_BF16 || !d->saved_lp || d->n_chunks > 1 ||
             d->gout_row_mask || d->gout_plan || (d->flags & (MIXGCN_LAYER_OUT_ROWS_ONLY | MIXGCN_LAYER_SAVED_IS_VALID)))
@@ -474,6 +482,7 @@ extern "C" mixgcn_status mixgcn_layer_fwd(mixgcn_ctx* ctx, const mixgcn_graph* g
     }
 
     const LayerLP lp(d);
+    if (epi.relu && d->x_out_bits) { epi.sign_bits = d->x_out_bits; epi.ld_sign_bits = d->ld_out_bits; }   // the ReLU mask, one bit per element
     if (order == MIXGCN_ORDER_AGG_FIRST) {
         SpmmOpts agg_opts; agg_opts.Z_lp = lp.saved; agg_opts.ldz_lp = lp.ld_saved;     // the aggregation also writes bf16(A_hat X)
         if (chunks == 1) {
@@ -616,6 +625,7 @@ extern "C" mixgcn_status mixgcn_layer_bwd(mixgcn_ctx* ctx, const mixgcn_graph* g
     const mixgcn_epilogue* gin = nullptr;
     if (d->flags & MIXGCN_LAYER_GATE_GIN) {
         gin_epi.gate = X_in; gin_epi.ld_gate = d->ld_in; gin_epi.gate_scale = d->in_scale; gin_epi.keep_scale = 1.0f;
+        if (d->x_in_bits) { gin_epi.gate_bits = d->x_in_bits; gin_epi.ld_gate_bits = d->ld_in_bits; }     // read instead of X_in's sign
         gin = &gin_epi;
     }
     if (const mixgcn_rowplan* plan = d->gout_plan) {

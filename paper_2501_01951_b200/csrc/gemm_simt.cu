@@ -21,6 +21,7 @@ struct Epi {
     const float* bias; int relu;
     const uint8_t* drop; float keep_scale;
     const float* gate; int64_t ld_gate; float gate_scale;
+    const uint32_t* gate_bits; int64_t ld_gate_bits;   // bit-packed gate (replaces `gate`)
     int64_t row0;
 };
 
@@ -29,6 +30,7 @@ __device__ __forceinline__ float apply_epi(const Epi& e, float y, int64_t m, int
     if (e.relu) y = fmaxf(y, 0.0f);
     if (e.drop) y = e.drop[(e.row0 + m) * N + n] ? y * e.keep_scale : 0.0f;
     if (e.gate) y = e.gate[(e.row0 + m) * e.ld_gate + n] > 0.0f ? y * e.gate_scale : 0.0f;
+    if (e.gate_bits) y = ((e.gate_bits[(e.row0 + m) * e.ld_gate_bits + (n >> 5)] >> (n & 31)) & 1u) ? y * e.gate_scale : 0.0f;
     return y;
 }
 
@@ -312,8 +314,9 @@ mixgcn_status launch_gemm_simt(mixgcn_ctx* ctx, int ta, int tb, int64_t M, int64
     p.M = M; p.N = N; p.K = K; p.A = A; p.lda = lda; p.B = B; p.ldb = ldb; p.C = C; p.ldc = ldc;
     if (epi) {
         p.epi.bias = epi->bias; p.epi.relu = epi->relu; p.epi.drop = epi->drop_mask;
-        p.epi.keep_scale = epi->keep_scale; p.epi.gate = epi->gate; p.epi.ld_gate = epi->ld_gate;
+        p.epi.keep_scale = epi->keep_scale; p.epi.gate = epi->gate_bits ? nullptr : epi->gate; p.epi.ld_gate = epi->ld_gate;
         p.epi.gate_scale = epi->gate_scale;
+        p.epi.gate_bits = epi->gate_bits; p.epi.ld_gate_bits = epi->ld_gate_bits;
     }
     p.epi.row0 = epi_row0;
     p.vec_a = aligned16(A) && (lda & 3) == 0;
@@ -362,7 +365,8 @@ mixgcn_status launch_splitk_reduce(mixgcn_ctx* ctx, int64_t M, int64_t N, int sp
     Epi e{};
     if (epi) {
         e.bias = epi->bias; e.relu = epi->relu; e.drop = epi->drop_mask; e.keep_scale = epi->keep_scale;
-        e.gate = epi->gate; e.ld_gate = epi->ld_gate; e.gate_scale = epi->gate_scale;
+        e.gate = epi->gate_bits ? nullptr : epi->gate; e.ld_gate = epi->ld_gate; e.gate_scale = epi->gate_scale;
+        e.gate_bits = epi->gate_bits; e.ld_gate_bits = epi->ld_gate_bits;
     }
     LaunchScope scope(ctx, PH_GEMM, s);
     const int64_t total = M * N;

@@ -50,6 +50,8 @@ struct TcEpi {
     const float* bias; int relu;
     const uint8_t* drop; float keep_scale;
     const float* gate; int64_t ld_gate; float gate_scale;
+    const uint32_t* gate_bits; int64_t ld_gate_bits;   // bit-packed gate (replaces `gate`): bit j & 31 of word j >> 5 of row i
+    uint32_t* sign_bits; int64_t ld_sign_bits;         // output: bit = (final y > 0), written by the K-major kernels' epilogues
     int64_t row0;
 };
 
@@ -78,7 +80,17 @@ __device__ __forceinline__ float tc_apply_epi(const TcEpi& e, float y, int64_t m
     if (e.relu) y = fmaxf(y, 0.0f);
     if (e.drop) y = e.drop[(e.row0 + m) * N + n] ? y * e.keep_scale : 0.0f;
     if (e.gate) y = e.gate[(e.row0 + m) * e.ld_gate + n] > 0.0f ? y * e.gate_scale : 0.0f;
+    if (e.gate_bits) y = ((e.gate_bits[(e.row0 + m) * e.ld_gate_bits + (n >> 5)] >> (n & 31)) & 1u) ? y * e.gate_scale : 0.0f;
     return y;
+}
+
+// bit q = (v[q] > 0) for the columns nb + q < N of one row's 32-column chunk
+__device__ __forceinline__ uint32_t sign_word(const float (&v)[32], int64_t nb, int64_t N) {
+    uint32_t w = 0;
+#pragma unroll
+    for (int q = 0; q < 32; ++q) w |= (v[q] > 0.0f ? 1u : 0u) << q;
+    const int64_t left = N - nb;
+    return left >= 32 ? w : (w & ((1u << (int)left) - 1u));
 }
 
 __device__ __forceinline__ bool aligned16_dev(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -511,8 +523,9 @@ __global__ void __launch_bounds__(KK_THREADS, 1) gemm_tc_kk_kernel(const __grid_
         // applied on the staged box, where a row's 128 bytes belong to eight adjacent lanes (coalesced
         // reads of the gate); otherwise element by element from the registers, like a bias wider than the
         // shared-memory copy.
-        const bool post = (p.epi.drop != nullptr || p.epi.gate != nullptr) && tma_store;
-        const bool generic = !post && (p.epi.drop != nullptr || p.epi.gate != nullptr || (p.epi.bias != nullptr && !bias_in_smem));
+        const bool has_gate = p.epi.gate != nullptr || p.epi.gate_bits != nullptr;
+        const bool post = (p.epi.drop != nullptr || has_gate) && tma_store;
+        const bool generic = !post && (p.epi.drop != nullptr || has_gate || (p.epi.bias != nullptr && !bias_in_smem));
         const bool wide_bias = post && p.epi.bias != nullptr && !bias_in_smem;
         const bool add_bias = p.epi.bias != nullptr && bias_in_smem, relu = p.epi.relu != 0;
         const bool gate_vec = p.epi.gate != nullptr && aligned16_dev(p.epi.gate) && (p.epi.ld_gate & 3) == 0;
@@ -538,7 +551,10 @@ __global__ void __launch_bounds__(KK_THREADS, 1) gemm_tc_kk_kernel(const __grid_
                 // the gate's 32 x 32 block in the staged-box orientation (lane = row it * 4 + lane / 8,
                 // 16-byte chunk lane % 8), requested before the accumulator is read so that the loads overlap it
                 float4 g4[8];
-                if (post && gate_vec) {
+                uint32_t gw = 0;                          // bit-packed gate: this lane's row, the chunk's word
+                if (post && p.epi.gate_bits) {
+                    if (row_ok) gw = __ldg(p.epi.gate_bits + (p.epi.row0 + m) * p.epi.ld_gate_bits + (nb >> 5));
+                } else if (post && gate_vec) {
 #pragma unroll
                     for (int it = 0; it < 8; ++it) {
                         const int64_t mr = m0 + quarter * 32 + it * 4 + (lane >> 3);
@@ -575,6 +591,7 @@ __global__ void __launch_bounds__(KK_THREADS, 1) gemm_tc_kk_kernel(const __grid_
                     for (int q = 0; q < 32; ++q)
                         if (nb + q < p.N) v[q] = tc_apply_epi(p.epi, v[q], m, nb + q, p.N);
                 }
+                if (p.epi.sign_bits && row_ok && !post) p.epi.sign_bits[(p.epi.row0 + m) * p.epi.ld_sign_bits + (nb >> 5)] = sign_word(v, nb, p.N);
                 if (p.C_lp && row_ok && !post) {
                     const int64_t left = p.N - nb, here = p.bn - c0;
                     const int valid = (int)(left < here ? left : here);
@@ -598,6 +615,7 @@ __global__ void __launch_bounds__(KK_THREADS, 1) gemm_tc_kk_kernel(const __grid_
 #pragma unroll
                         for (int it = 0; it < 8; ++it) {
                             const int rr = it * 4 + (lane >> 3), ch = lane & 7;
+                            const uint32_t gw_rr = __shfl_sync(0xFFFFFFFFu, gw, rr);      // every lane takes part (before any lane skips)
                             const int64_t mr = m0 + quarter * 32 + rr;
                             const int nc = nb + ch * 4;
                             if (mr >= p.M || nc >= p.N || c0 + ch * 4 >= p.bn) continue;
@@ -610,7 +628,11 @@ __global__ void __launch_bounds__(KK_THREADS, 1) gemm_tc_kk_kernel(const __grid_
 #pragma unroll
                                 for (int t = 0; t < 4; ++t) if (t < nv) y[t] = dm[t] ? y[t] * p.epi.keep_scale : 0.0f;
                             }
-                            if (p.epi.gate) {
+                            if (p.epi.gate_bits) {
+                                const uint32_t nib = (gw_rr >> (ch * 4)) & 0xFu;
+#pragma unroll
+                                for (int t = 0; t < 4; ++t) y[t] = ((nib >> t) & 1u) ? y[t] * p.epi.gate_scale : 0.0f;
+                            } else if (p.epi.gate) {
                                 const float* gp = p.epi.gate + (p.epi.row0 + mr) * p.epi.ld_gate + nc;
                                 float gq[4] = {0.f, 0.f, 0.f, 0.f};
                                 if (gate_vec) {       // the whole group lies inside the row's allocation (ld_gate % 4 == 0)
@@ -782,8 +804,9 @@ __global__ void __launch_bounds__(KK_THREADS, 1) gemm_tc_pair_kernel(const __gri
     } else {
         // ---------------- epilogue (both CTAs): this CTA's 128 rows of the tile ----------------
         const int quarter = warp & 3, half = warp >> 2;
-        const bool post = (p.epi.drop != nullptr || p.epi.gate != nullptr) && tma_store;
-        const bool generic = !post && (p.epi.drop != nullptr || p.epi.gate != nullptr);
+        const bool has_gate = p.epi.gate != nullptr || p.epi.gate_bits != nullptr;
+        const bool post = (p.epi.drop != nullptr || has_gate) && tma_store;
+        const bool generic = !post && (p.epi.drop != nullptr || has_gate);
         const bool add_bias = p.epi.bias != nullptr, relu = p.epi.relu != 0;
         const bool gate_vec = p.epi.gate != nullptr && aligned16_dev(p.epi.gate) && (p.epi.ld_gate & 3) == 0;
         uint8_t* box = smem_out + (size_t)warp * 4096;
@@ -803,7 +826,10 @@ __global__ void __launch_bounds__(KK_THREADS, 1) gemm_tc_pair_kernel(const __gri
                 const int nb = n0 + c0;
                 if (nb >= p.N) break;                     // columns beyond N: nothing to store (warp-uniform)
                 float4 g4[8];
-                if (post && gate_vec) {
+                uint32_t gw = 0;                          // bit-packed gate: this lane's row, the chunk's word
+                if (post && p.epi.gate_bits) {
+                    if (row_ok) gw = __ldg(p.epi.gate_bits + (p.epi.row0 + m) * p.epi.ld_gate_bits + (nb >> 5));
+                } else if (post && gate_vec) {
 #pragma unroll
                     for (int it = 0; it < 8; ++it) {
                         const int64_t mr = m0 + quarter * 32 + it * 4 + (lane >> 3);
@@ -842,6 +868,7 @@ __global__ void __launch_bounds__(KK_THREADS, 1) gemm_tc_pair_kernel(const __gri
                     for (int q = 0; q < 32; ++q)
                         if (nb + q < p.N) v[q] = tc_apply_epi(p.epi, v[q], m, nb + q, p.N);
                 }
+                if (p.epi.sign_bits && row_ok && !post) p.epi.sign_bits[(p.epi.row0 + m) * p.epi.ld_sign_bits + (nb >> 5)] = sign_word(v, nb, p.N);
                 if (p.C_lp && row_ok && !post) {
                     const int64_t left = p.N - nb;
                     store_lp_row(p.C_lp + m * p.ldc_lp + nb, v, (int)(left < 32 ? left : 32));
@@ -858,6 +885,7 @@ __global__ void __launch_bounds__(KK_THREADS, 1) gemm_tc_pair_kernel(const __gri
 #pragma unroll
                         for (int it = 0; it < 8; ++it) {
                             const int rr = it * 4 + (lane >> 3), ch = lane & 7;
+                            const uint32_t gw_rr = __shfl_sync(0xFFFFFFFFu, gw, rr);      // every lane takes part (before any lane skips)
                             const int64_t mr = m0 + quarter * 32 + rr;
                             const int nc = nb + ch * 4;
                             if (mr >= p.M || nc >= p.N) continue;
@@ -870,7 +898,11 @@ __global__ void __launch_bounds__(KK_THREADS, 1) gemm_tc_pair_kernel(const __gri
 #pragma unroll
                                 for (int t = 0; t < 4; ++t) if (t < nv) y[t] = dm[t] ? y[t] * p.epi.keep_scale : 0.0f;
                             }
-                            if (p.epi.gate) {
+                            if (p.epi.gate_bits) {
+                                const uint32_t nib = (gw_rr >> (ch * 4)) & 0xFu;
+#pragma unroll
+                                for (int t = 0; t < 4; ++t) y[t] = ((nib >> t) & 1u) ? y[t] * p.epi.gate_scale : 0.0f;
+                            } else if (p.epi.gate) {
                                 const float* gp = p.epi.gate + (p.epi.row0 + mr) * p.epi.ld_gate + nc;
                                 float gq[4] = {0.f, 0.f, 0.f, 0.f};
                                 if (gate_vec) {
@@ -1178,11 +1210,13 @@ int pick_splits(int64_t tiles, int64_t slots, int64_t max_splits) {
 template <int KIND>
 mixgcn_status launch_kind(mixgcn_ctx* ctx, int ta, int tb, int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,
                           const void* B, int64_t ldb, float* C, int64_t ldc, const mixgcn_epilogue* epi, int64_t epi_row0,
-                          cudaStream_t s, uint16_t* C_lp, int64_t ldc_lp, float* colsum_b, bool* colsum_done, const LossFuse* loss) {
+                          cudaStream_t s, uint16_t* C_lp, int64_t ldc_lp, float* colsum_b, bool* colsum_done, const LossFuse* loss,
+                          bool* bits_done) {
     using Cfg = KindCfg<KIND>;
     constexpr int EB = Cfg::EB, BK = Cfg::BK;
     // the loss epilogue exists in the single-CTA K-major kernel for one n-tile and a bias-only epilogue
-    if (loss && (ta || N > 256 || C_lp || ctx->debug_drop_load || (epi && (epi->relu || epi->drop_mask || epi->gate)))) return MIXGCN_EUNSUPPORTED;
+    if (loss && (ta || N > 256 || C_lp || ctx->debug_drop_load || (epi && (epi->relu || epi->drop_mask || epi->gate || epi->gate_bits || epi->sign_bits)))) return MIXGCN_EUNSUPPORTED;
+    if (ta && epi && (epi->gate_bits || epi->sign_bits)) return MIXGCN_EUNSUPPORTED;      // bit-packed masks: K-major products only
     constexpr int64_t LD_ALIGN = 16 / EB;           // TMA strides are multiples of 16 bytes
     if (M <= 0 || N <= 0 || K <= 0) return MIXGCN_EUNSUPPORTED;
     if (ta && tb) return MIXGCN_EUNSUPPORTED;
@@ -1203,7 +1237,9 @@ mixgcn_status launch_kind(mixgcn_ctx* ctx, int ta, int tb, int64_t M, int64_t N,
     p.wait_limit = ctx->debug_wait_limit > 0 ? (uint32_t)ctx->debug_wait_limit : WAIT_LIMIT_DEFAULT;
     if (epi) {
         p.epi.bias = epi->bias; p.epi.relu = epi->relu; p.epi.drop = epi->drop_mask; p.epi.keep_scale = epi->keep_scale;
-        p.epi.gate = epi->gate; p.epi.ld_gate = epi->ld_gate; p.epi.gate_scale = epi->gate_scale;
+        p.epi.gate = epi->gate_bits ? nullptr : epi->gate; p.epi.ld_gate = epi->ld_gate; p.epi.gate_scale = epi->gate_scale;
+        p.epi.gate_bits = epi->gate_bits; p.epi.ld_gate_bits = epi->ld_gate_bits;
+        p.epi.sign_bits = epi->sign_bits; p.epi.ld_sign_bits = epi->ld_sign_bits;
     }
     p.epi.row0 = epi_row0;
     const int64_t tiles = p.m_tiles * p.n_tiles;
@@ -1266,6 +1302,8 @@ mixgcn_status launch_kind(mixgcn_ctx* ctx, int ta, int tb, int64_t M, int64_t N,
                     LaunchScope scope(ctx, PH_GEMM, s);
                     MIXGCN_CUDA(cudaLaunchKernelEx(&cfg, gemm_tc_pair_kernel<KIND>, map_a, map_b2, map_c2, q, tma_store2));
                     ctx->gemm_pair_launches++;
+                    // the epilogue wrote the sign bitmap unless the per-element terms ran on the staged boxes
+                    if (bits_done) *bits_done = q.epi.sign_bits && !(tma_store2 && (q.epi.drop || q.epi.gate || q.epi.gate_bits));
                     return MIXGCN_OK;
                 }
             }
@@ -1302,6 +1340,7 @@ mixgcn_status launch_kind(mixgcn_ctx* ctx, int ta, int tb, int64_t M, int64_t N,
         LaunchScope scope(ctx, PH_GEMM, s);
         gemm_tc_kk_kernel<KIND><<<dim3((unsigned)grid, 1, 1), KK_THREADS, smem_kk, s>>>(map_a, map_b, map_c, p, b_resident, tma_store);
         MIXGCN_CUDA(cudaGetLastError());
+        if (bits_done) *bits_done = p.epi.sign_bits && !(tma_store && (p.epi.drop || p.epi.gate || p.epi.gate_bits));
         return MIXGCN_OK;
     }
 
@@ -1408,11 +1447,12 @@ namespace mixgcn {
 mixgcn_status launch_gemm_tc(mixgcn_ctx* ctx, int kind, int ta, int tb, int64_t M, int64_t N, int64_t K, const void* A,
                              int64_t lda, const void* B, int64_t ldb, float* C, int64_t ldc,
                              const mixgcn_epilogue* epi, int64_t epi_row0, cudaStream_t s, uint16_t* C_lp, int64_t ldc_lp,
-                             float* colsum_b, bool* colsum_done, const LossFuse* loss) {
+                             float* colsum_b, bool* colsum_done, const LossFuse* loss, bool* bits_done) {
     if (colsum_done) *colsum_done = false;
+    if (bits_done) *bits_done = false;
     if (kind == KIND_BF16)
-        return launch_kind<KIND_BF16>(ctx, ta, tb, M, N, K, A, lda, B, ldb, C, ldc, epi, epi_row0, s, C_lp, ldc_lp, colsum_b, colsum_done, loss);
-    return launch_kind<KIND_TF32>(ctx, ta, tb, M, N, K, A, lda, B, ldb, C, ldc, epi, epi_row0, s, C_lp, ldc_lp, colsum_b, colsum_done, loss);
+        return launch_kind<KIND_BF16>(ctx, ta, tb, M, N, K, A, lda, B, ldb, C, ldc, epi, epi_row0, s, C_lp, ldc_lp, colsum_b, colsum_done, loss, bits_done);
+    return launch_kind<KIND_TF32>(ctx, ta, tb, M, N, K, A, lda, B, ldb, C, ldc, epi, epi_row0, s, C_lp, ldc_lp, colsum_b, colsum_done, loss, bits_done);
 }
 
 // dst (rows x ld_dst bf16, ld_dst a multiple of 4) = bf16(src (rows x ld_src fp32, 16-byte aligned, ld_src % 4 == 0)), columns < d

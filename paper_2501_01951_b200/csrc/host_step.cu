@@ -91,6 +91,15 @@ mixgcn_status lay_out(char* base, int64_t n, int L, const int32_t* dims, int pre
     lo.labels = c.take<int32_t>(n); lo.mask = c.take<uint8_t>(n); lo.loss = c.take<float>(4); lo.pred = c.take<int32_t>(n);
     lo.rowmask.resize(L);
     for (int l = 0; l < L; ++l) lo.rowmask[l] = c.take<uint8_t>(n);
+    // sign bitmaps of the hidden activations a dense product writes (agg-first layer below): the backward reads
+    // its ReLU gates from them, one bit per element
+    for (int l = 1; l < L; ++l) {
+        if (lo.desc[l - 1].order != MIXGCN_ORDER_AGG_FIRST) continue;
+        const int64_t words = (dims[l] + 31) / 32;
+        uint32_t* bits = c.take<uint32_t>(n * words);
+        lo.desc[l - 1].x_out_bits = bits; lo.desc[l - 1].ld_out_bits = words;
+        lo.desc[l].x_in_bits = bits; lo.desc[l].ld_in_bits = words;
+    }
     auto each = [&](std::vector<float*>& v, bool weight) {
         v.resize(L);
         for (int l = 0; l < L; ++l) v[l] = c.take<float>(weight ? (int64_t)dims[l] * dims[l + 1] : dims[l + 1]);

@@ -265,7 +265,11 @@ mixgcn_status launch_gemm_simt(mixgcn_ctx* ctx, int ta, int tb, int64_t M, int64
 mixgcn_status launch_gemm_tc(mixgcn_ctx* ctx, int kind, int ta, int tb, int64_t M, int64_t N, int64_t K, const void* A,
                              int64_t lda, const void* B, int64_t ldb, float* C, int64_t ldc,
                              const mixgcn_epilogue* epi, int64_t epi_row0, cudaStream_t s, uint16_t* C_lp, int64_t ldc_lp,
-                             float* colsum_b = nullptr, bool* colsum_done = nullptr, const LossFuse* loss = nullptr);
+                             float* colsum_b = nullptr, bool* colsum_done = nullptr, const LossFuse* loss = nullptr,
+                             bool* bits_done = nullptr);
+// bits[u][j] = (X == null || X[u][j] > 0) && (bytes == null || bytes[u*w + j] != 0), n x ld_bits words
+mixgcn_status launch_mask_pack(mixgcn_ctx* ctx, int64_t n, int32_t w, const float* X, int64_t ldx, const uint8_t* bytes,
+                               uint32_t* bits, int64_t ld_bits, cudaStream_t s);
 mixgcn_status launch_splitk_reduce(mixgcn_ctx* ctx, int64_t M, int64_t N, int splits, const float* part, float* C,
                                    int64_t ldc, const mixgcn_epilogue* epi, cudaStream_t s);
 mixgcn_status launch_to_bf16(mixgcn_ctx* ctx, int64_t rows, int32_t d, const float* src, int64_t ld_src, uint16_t* dst,

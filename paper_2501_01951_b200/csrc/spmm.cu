@@ -63,6 +63,7 @@ struct SpmmParams {
     const float* bias; int relu;
     const uint8_t* drop; float keep_scale;
     const float* gate; int64_t ld_gate; float gate_scale;
+    const uint32_t* gate_bits; int64_t ld_gate_bits;   // bit-packed gate (replaces `gate`): the bitmap mask buffer of Section 3.2.1
     const float* residual; int64_t ld_residual; float residual_scale;
     // loss epilogue (kernels instantiated with LOSS): labels, train mask, number of train nodes, per-row loss, arg-max
     const int32_t* loss_labels; const uint8_t* loss_mask; const unsigned long long* loss_count;
@@ -113,6 +114,11 @@ __device__ __forceinline__ void store_row(const SpmmParams& p, int64_t u, int c4
     }
 #pragma unroll
     for (int t = 0; t < 4; ++t) r[t] = (j + t < jend) ? epilogue1(p, r[t], u, j + t) : 0.0f;
+    if (p.gate_bits) {
+        const uint32_t nib = (__ldg(p.gate_bits + u * p.ld_gate_bits + (j >> 5)) >> (j & 31)) & 0xFu;   // j % 4 == 0: one word
+#pragma unroll
+        for (int t = 0; t < 4; ++t) r[t] = ((nib >> t) & 1u) ? r[t] * p.gate_scale : 0.0f;
+    }
     if (p.out_bits) {
         const uint32_t nib = (__ldg(p.out_bits + u * p.ld_bits + (j >> 5)) >> (j & 31)) & 0xFu;   // j % 4 == 0: one word
 #pragma unroll
@@ -658,6 +664,8 @@ mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView&
     if (w <= 0) return MIXGCN_OK;
     if (!Z && !opts.Z_lp) MIXGCN_FAIL(MIXGCN_EINVAL, "spmm: no output");
     if (sparse && row_filter) MIXGCN_FAIL(MIXGCN_EUNSUPPORTED, "spmm: a row filter cannot be combined with a row-sparse input");
+    if (epi && epi->sign_bits && (row_filter || opts.row_limit >= 0 || lf || !Z))
+        MIXGCN_FAIL(MIXGCN_EUNSUPPORTED, "spmm: the sign bitmap needs every row of a plain fp32 result");
     if (lf) {
         if (sparse || row_filter || chunks > 1 || opts.out_bits || opts.Z_lp || opts.row_limit >= 0 || !Z || w > 256 ||
             (epi && (epi->relu || epi->drop_mask || epi->gate || epi->residual)))
@@ -676,7 +684,8 @@ mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView&
     p.out_bits = opts.out_bits; p.ld_bits = opts.ld_bits;
     if (epi) {
         p.bias = epi->bias; p.relu = epi->relu; p.drop = epi->drop_mask; p.keep_scale = epi->keep_scale;
-        p.gate = epi->gate; p.ld_gate = epi->ld_gate; p.gate_scale = epi->gate_scale;
+        p.gate = epi->gate_bits ? nullptr : epi->gate; p.ld_gate = epi->ld_gate; p.gate_scale = epi->gate_scale;
+        p.gate_bits = epi->gate_bits; p.ld_gate_bits = epi->ld_gate_bits;
         p.residual = epi->residual; p.ld_residual = epi->ld_residual; p.residual_scale = epi->residual_scale;
     }
     p.status = ctx->d_status;
@@ -811,6 +820,10 @@ mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView&
         }
     }
     MIXGCN_CUDA(cudaGetLastError());
+    // sign bitmap of the result: one more pass over the rows this call wrote
+    if (epi && epi->sign_bits)
+        MIXGCN_TRY(launch_mask_pack(ctx, S.n_rows, w, Z + S.row0 * ldz, ldz, nullptr, epi->sign_bits + S.row0 * epi->ld_sign_bits,
+                                    epi->ld_sign_bits, s));
     return MIXGCN_OK;
 }
 
@@ -828,6 +841,8 @@ extern "C" mixgcn_status mixgcn_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, int
     if (Y == Z) MIXGCN_FAIL(MIXGCN_EINVAL, "spmm: Y and Z must not overlap");
     if (epi && epi->gate && epi->ld_gate < w) MIXGCN_FAIL(MIXGCN_EINVAL, "spmm: gate leading dimension < w");
     if (epi && epi->residual && (epi->ld_residual < w || epi->residual == Z)) MIXGCN_FAIL(MIXGCN_EINVAL, "spmm: residual needs ld_residual >= w and must not be the output");
+    if (epi && ((epi->gate_bits && epi->ld_gate_bits < (w + 31) / 32) || (epi->sign_bits && epi->ld_sign_bits < (w + 31) / 32)))
+        MIXGCN_FAIL(MIXGCN_EINVAL, "spmm: a bit-packed mask needs ld >= ceil(w / 32) words");
     MIXGCN_CUDA(cudaSetDevice(ctx->device));
     return launch_spmm(ctx, g, transposed ? g->bwd : g->fwd, 1, 0, w, Y, ldy, Z, ldz, epi, (cudaStream_t)stream);
 }
@@ -855,16 +870,24 @@ __global__ void mask_pack_kernel(int64_t n, int w, const float* __restrict__ X, 
 
 }  // namespace
 
+namespace mixgcn {
+mixgcn_status launch_mask_pack(mixgcn_ctx* ctx, int64_t n, int32_t w, const float* X, int64_t ldx, const uint8_t* bytes,
+                               uint32_t* bits, int64_t ld_bits, cudaStream_t s) {
+    if (n <= 0 || w <= 0) return MIXGCN_OK;
+    const int64_t total = n * ((w + 31) / 32);
+    LaunchScope scope(ctx, PH_ELEM, s);
+    mask_pack_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(n, w, X, ldx, bytes, bits, ld_bits);
+    MIXGCN_CUDA(cudaGetLastError());
+    return MIXGCN_OK;
+}
+}  // namespace mixgcn
+
 extern "C" mixgcn_status mixgcn_mask_pack(mixgcn_ctx* ctx, int64_t n, int32_t w, const float* X, int64_t ldx,
                                           const uint8_t* bytes, uint32_t* bits, int64_t ld_bits, void* stream) {
     if (!ctx || !bits || (!X && !bytes)) MIXGCN_FAIL(MIXGCN_EINVAL, "mask_pack: null argument");
     if (n <= 0 || w <= 0 || ld_bits < (w + 31) / 32 || (X && ldx < w)) MIXGCN_FAIL(MIXGCN_EINVAL, "mask_pack: need n, w > 0, ld_bits >= ceil(w/32), ldx >= w");
     MIXGCN_CUDA(cudaSetDevice(ctx->device));
-    const int64_t total = n * ((w + 31) / 32);
-    LaunchScope scope(ctx, PH_ELEM, (cudaStream_t)stream);
-    mask_pack_kernel<<<(unsigned)((total + 255) / 256), 256, 0, (cudaStream_t)stream>>>(n, w, X, ldx, bytes, bits, ld_bits);
-    MIXGCN_CUDA(cudaGetLastError());
-    return MIXGCN_OK;
+    return launch_mask_pack(ctx, n, w, X, ldx, bytes, bits, ld_bits, (cudaStream_t)stream);
 }
 
 extern "C" mixgcn_status mixgcn_spmm_sampled(mixgcn_ctx* ctx, const mixgcn_graph* g, int transposed, int32_t w,

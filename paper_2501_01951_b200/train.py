@@ -23,7 +23,7 @@ def round8(x: int) -> int:
 class GcnTrainer:
     def __init__(self, ctx: mg.Ctx, graph: mg.Graph, dims, precision=mg.PREC_FP32, order=mg.ORDER_AUTO,
                  n_chunks=0, fuse_gate=True, keep_scale=1.0, device=None, row_sparse="auto",
-                 train_rows_only=False, row_plans=True, cache_first_aggregation=False, lp_copies=True, saved_lp_only=True):
+                 train_rows_only=False, row_plans=True, cache_first_aggregation=False, lp_copies=True, saved_lp_only=True, sign_bitmaps=True):
         self.ctx, self.g = ctx, graph
         self.dims = tuple(int(d) for d in dims)
         self.L = len(self.dims) - 1
@@ -110,6 +110,19 @@ class GcnTrainer:
                     d.g_out_lp = g_lp[l + 1].data_ptr()
                 if g_lp[l] is not None:
                     d.g_in_lp = g_lp[l].data_ptr()
+        # Sign bitmaps of the hidden activations (one bit per element): written by the forward kernel that produces
+        # X[l], read by the backward kernel that gates the gradient w.r.t. X[l] instead of the fp32 tensor
+        self.xbits = [None] * (L + 1)
+        if fuse_gate and sign_bitmaps:
+            for l in range(1, L):
+                # where a dense product produces X[l] (agg-first layer l-1) its epilogue writes the bitmap for free;
+                # an aggregation would need one more pass over X[l], which costs what the bitmap saves
+                if self.orders[l - 1] != mg.ORDER_AGG_FIRST:
+                    continue
+                t = torch.zeros((n, (self.dims[l] + 31) // 32), dtype=torch.int32, device=self.device)
+                self.xbits[l] = t
+                self.descs[l - 1].x_out_bits, self.descs[l - 1].ld_out_bits = t.data_ptr(), t.stride(0)
+                self.descs[l].x_in_bits, self.descs[l].ld_in_bits = t.data_ptr(), t.stride(0)
         self.loss = torch.zeros(1, dtype=torch.float32, device=self.device)
         self.pred = torch.zeros(n, dtype=torch.int32, device=self.device)
         self.n_correct = torch.zeros(1, dtype=torch.int64, device=self.device)

@@ -33,17 +33,24 @@ def test_status_strings(mg):
     assert mg.lib.mixgcn_status_string(99).decode() == "unknown status"
 
 
-def test_struct_layouts_match_the_header(mg):
-    # the header's structs, field by field, on an LP64 ABI
-    assert C.sizeof(mg.Epilogue) == 80
-    assert mg.Epilogue.residual.offset == 56 and mg.Epilogue.ld_residual.offset == 64 and mg.Epilogue.residual_scale.offset == 72
-    assert C.sizeof(mg.LayerDesc) == 152
-    assert mg.LayerDesc.saved_lp.offset == 88 and mg.LayerDesc.x_in_lp.offset == 104 and mg.LayerDesc.ld_out_lp.offset == 128
-    assert mg.LayerDesc.g_in_lp.offset == 144
-    assert mg.LayerDesc.gout_row_mask.offset == 56 and mg.LayerDesc.gin_row_mask.offset == 72
-    assert mg.LayerDesc.gout_plan.offset == 80
-    assert mg.LayerDesc.ld_in.offset == 8 and mg.LayerDesc.order.offset == 32 and mg.LayerDesc.n_chunks.offset == 52
-    assert mg.Epilogue.keep_scale.offset == 24 and mg.Epilogue.ld_gate.offset == 40
+def test_struct_layouts_match_the_header(mg, tmp_path):
+    """sizeof and every field's offset as a C compiler lays the header's structs out, against the ctypes mirror."""
+    import subprocess
+    checks = []
+    for cname, cls in (("mixgcn_epilogue", mg.Epilogue), ("mixgcn_layer_desc", mg.LayerDesc)):
+        checks.append(f'printf("{cname} %zu\\n", sizeof({cname}));')
+        for field, _ in cls._fields_:
+            checks.append(f'printf("{cname}.{field} %zu\\n", offsetof({cname}, {field}));')
+    src = tmp_path / "layout.c"
+    src.write_text('#include <stddef.h>\n#include <stdio.h>\n#include "mixgcn.h"\nint main(void) {\n' + "\n".join(checks) + "\nreturn 0; }\n")
+    exe = tmp_path / "layout"
+    subprocess.run(["gcc", "-std=c99", "-I", os.path.join(ROOT, "include"), str(src), "-o", str(exe)], check=True)
+    out = dict(line.split() for line in subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.splitlines())
+    for cname, cls in (("mixgcn_epilogue", mg.Epilogue), ("mixgcn_layer_desc", mg.LayerDesc)):
+        assert int(out[cname]) == C.sizeof(cls), cname
+        for field, _ in cls._fields_:
+            assert int(out[f"{cname}.{field}"]) == getattr(cls, field).offset, f"{cname}.{field}"
+    assert C.sizeof(mg.Epilogue) == 112 and C.sizeof(mg.LayerDesc) == 184      # an ABI change is a deliberate edit here too
 
 
 @pytest.mark.parametrize("d_in,d_out,first,want", [
