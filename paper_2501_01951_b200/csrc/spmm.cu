@@ -57,13 +57,16 @@ struct SpmmParams {
     const uint8_t* row_filter;
     const int32_t* seg_perm;   // segment records carry the long row's index i; its row is seg_perm[i] (null: the record's row)
     // sampled aggregation Z = (A_hat Y) (.) M, Eq. 4: bit j of row u of the bitmap says whether output (u, j) is kept
+    // The same bitmap serves a bit-packed gate (the bitmap mask buffer of Section 3.2.1 holding a ReLU mask): kept
+    // outputs are then scaled by bits_scale and nothing is skipped (bits_skip = 0).
     const uint32_t* out_bits;  // [n x ld_bits] words, null: every output is kept
     int64_t ld_bits;
+    float bits_scale;          // factor of the kept outputs (1 for the sampled aggregation, the gate's scale for a gate)
+    int bits_skip;             // 1: lanes whose four columns of a row are all masked skip that row's gathers
     // epilogue
     const float* bias; int relu;
     const uint8_t* drop; float keep_scale;
     const float* gate; int64_t ld_gate; float gate_scale;
-    const uint32_t* gate_bits; int64_t ld_gate_bits;   // bit-packed gate (replaces `gate`): the bitmap mask buffer of Section 3.2.1
     const float* residual; int64_t ld_residual; float residual_scale;
     // loss epilogue (kernels instantiated with LOSS): labels, train mask, number of train nodes, per-row loss, arg-max
     const int32_t* loss_labels; const uint8_t* loss_mask; const unsigned long long* loss_count;
@@ -114,15 +117,10 @@ __device__ __forceinline__ void store_row(const SpmmParams& p, int64_t u, int c4
     }
 #pragma unroll
     for (int t = 0; t < 4; ++t) r[t] = (j + t < jend) ? epilogue1(p, r[t], u, j + t) : 0.0f;
-    if (p.gate_bits) {
-        const uint32_t nib = (__ldg(p.gate_bits + u * p.ld_gate_bits + (j >> 5)) >> (j & 31)) & 0xFu;   // j % 4 == 0: one word
-#pragma unroll
-        for (int t = 0; t < 4; ++t) r[t] = ((nib >> t) & 1u) ? r[t] * p.gate_scale : 0.0f;
-    }
     if (p.out_bits) {
         const uint32_t nib = (__ldg(p.out_bits + u * p.ld_bits + (j >> 5)) >> (j & 31)) & 0xFu;   // j % 4 == 0: one word
 #pragma unroll
-        for (int t = 0; t < 4; ++t) r[t] = ((nib >> t) & 1u) ? r[t] : 0.0f;
+        for (int t = 0; t < 4; ++t) r[t] = ((nib >> t) & 1u) ? r[t] * p.bits_scale : 0.0f;
     }
     if (p.Z) *reinterpret_cast<float4*>(p.Z + u * p.ldz + j) = make_float4(r[0], r[1], r[2], r[3]);   // null: bf16 copy only
     if (p.Z_lp) store_lp4(p.Z_lp + u * p.ldz_lp + j, r[0], r[1], r[2], r[3]);
@@ -287,7 +285,7 @@ __global__ void __launch_bounds__(256, VPL <= 2 ? SPMM_MINB : 1) spmm_group_kern
 #pragma unroll
     for (int v = 0; v < VPL; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
     unsigned keep = 0xFFFFFFFFu;
-    if (p.out_bits) {
+    if (p.out_bits && p.bits_skip) {
         // Eq. 4: outputs the mask drops are never computed -- a lane whose four columns of this row are all
         // masked skips its gathers of every neighbour (the mask is known before the aggregation)
         const int64_t row = p.seg_perm ? __ldg(p.seg_perm + u) : u;
@@ -681,11 +679,15 @@ mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView&
     p.rowptr = A.rowptr; p.col = A.col; p.val = A.val;
     p.Y = Y; p.ldy = ldy; p.Z = Z; p.ldz = ldz; p.w_total = w;
     p.Z_lp = opts.Z_lp; p.ldz_lp = opts.ldz_lp;
-    p.out_bits = opts.out_bits; p.ld_bits = opts.ld_bits;
+    p.out_bits = opts.out_bits; p.ld_bits = opts.ld_bits; p.bits_scale = 1.0f; p.bits_skip = 1;
+    if (epi && epi->gate_bits) {
+        // a bit-packed gate goes through the same bitmap path as the sampled aggregation's output mask
+        if (opts.out_bits) MIXGCN_FAIL(MIXGCN_EUNSUPPORTED, "spmm: a sampled aggregation takes no bit-packed gate as well");
+        p.out_bits = epi->gate_bits; p.ld_bits = epi->ld_gate_bits; p.bits_scale = epi->gate_scale; p.bits_skip = 0;
+    }
     if (epi) {
         p.bias = epi->bias; p.relu = epi->relu; p.drop = epi->drop_mask; p.keep_scale = epi->keep_scale;
         p.gate = epi->gate_bits ? nullptr : epi->gate; p.ld_gate = epi->ld_gate; p.gate_scale = epi->gate_scale;
-        p.gate_bits = epi->gate_bits; p.ld_gate_bits = epi->ld_gate_bits;
         p.residual = epi->residual; p.ld_residual = epi->ld_residual; p.residual_scale = epi->residual_scale;
     }
     p.status = ctx->d_status;
@@ -775,7 +777,7 @@ mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView&
             {
                 LaunchScope scope(ctx, phase, s);
                 p.idx_begin = 0; p.idx_end = S.total_segs;
-                if (p.out_bits) p.seg_perm = S.perm;       // a segment's record names its long row by ordinal
+                if (p.out_bits && p.bits_skip) p.seg_perm = S.perm;       // a segment's record names its long row by ordinal
                 dispatch(p, p.w <= SPMM_FOLD_WMAX ? SPMM_FOLD_SEG : 1, s);
                 p.seg_perm = nullptr;
             }

@@ -85,3 +85,21 @@ def test_null_arguments_are_rejected_without_a_device(mg):
     assert mg.lib.mixgcn_graph_info(None, None, None, None, None) == mg.EINVAL
     assert mg.lib.mixgcn_ctx_destroy(None) == mg.OK and mg.lib.mixgcn_graph_destroy(None) == mg.OK
     assert b"null" in mg.lib.mixgcn_last_error()
+
+
+def test_hot_aggregation_kernels_compile_without_register_spills(tmp_path):
+    """The aggregation kernels that carry the epochs run under a register cap (four CTAs of 256 threads per SM);
+    a spill there costs several per cent of an epoch, and nothing else would notice it: ask the assembler."""
+    import subprocess
+    from paper_2501_01951_b200 import build as b
+    cmd = [b.NVCC, *b.ARCH, *b.CFLAGS, "-Xptxas", "-v", "-c", "spmm.cu", "-o", str(tmp_path / "spmm.o")]
+    r = subprocess.run(cmd, capture_output=True, text=True, cwd=b.CSRC)
+    assert r.returncode == 0, r.stderr[-2000:]
+    log = r.stdout + r.stderr
+    entries = re.findall(r"Compiling entry function '(\S+)'.*?\n.*?\n\s+\d+ bytes stack frame, (\d+) bytes spill stores, (\d+) bytes spill loads", log)
+    assert len(entries) > 50
+    hot = [(name, int(st), int(ld)) for name, st, ld in entries
+           if ("spmm_group_kernel" in name and "Lb0E" in name) or "spmm_short_kernel" in name or "spmm_combine_kernelILb0" in name]
+    assert len(hot) >= 30
+    spilled = [(name, st, ld) for name, st, ld in hot if st or ld]
+    assert not spilled, spilled
