@@ -551,9 +551,10 @@ __global__ void __launch_bounds__(KK_THREADS, 1) gemm_tc_kk_kernel(const __grid_
                 // the gate's 32 x 32 block in the staged-box orientation (lane = row it * 4 + lane / 8,
                 // 16-byte chunk lane % 8), requested before the accumulator is read so that the loads overlap it
                 float4 g4[8];
-                uint32_t gw = 0;                          // bit-packed gate: this lane's row, the chunk's word
                 if (post && p.epi.gate_bits) {
-                    if (row_ok) gw = __ldg(p.epi.gate_bits + (p.epi.row0 + m) * p.epi.ld_gate_bits + (nb >> 5));
+                    // bit-packed gate: this lane's row, the chunk's word (kept in the first slot of the fp32 gate's registers:
+                    // the two forms exclude each other)
+                    g4[0].x = __uint_as_float(row_ok ? __ldg(p.epi.gate_bits + (p.epi.row0 + m) * p.epi.ld_gate_bits + (nb >> 5)) : 0u);
                 } else if (post && gate_vec) {
 #pragma unroll
                     for (int it = 0; it < 8; ++it) {
@@ -615,7 +616,7 @@ __global__ void __launch_bounds__(KK_THREADS, 1) gemm_tc_kk_kernel(const __grid_
 #pragma unroll
                         for (int it = 0; it < 8; ++it) {
                             const int rr = it * 4 + (lane >> 3), ch = lane & 7;
-                            const uint32_t gw_rr = __shfl_sync(0xFFFFFFFFu, gw, rr);      // every lane takes part (before any lane skips)
+                            const uint32_t gw_rr = __shfl_sync(0xFFFFFFFFu, __float_as_uint(g4[0].x), rr);   // every lane takes part (before any lane skips)
                             const int64_t mr = m0 + quarter * 32 + rr;
                             const int nc = nb + ch * 4;
                             if (mr >= p.M || nc >= p.N || c0 + ch * 4 >= p.bn) continue;
@@ -826,9 +827,10 @@ __global__ void __launch_bounds__(KK_THREADS, 1) gemm_tc_pair_kernel(const __gri
                 const int nb = n0 + c0;
                 if (nb >= p.N) break;                     // columns beyond N: nothing to store (warp-uniform)
                 float4 g4[8];
-                uint32_t gw = 0;                          // bit-packed gate: this lane's row, the chunk's word
                 if (post && p.epi.gate_bits) {
-                    if (row_ok) gw = __ldg(p.epi.gate_bits + (p.epi.row0 + m) * p.epi.ld_gate_bits + (nb >> 5));
+                    // bit-packed gate: this lane's row, the chunk's word (kept in the first slot of the fp32 gate's registers:
+                    // the two forms exclude each other)
+                    g4[0].x = __uint_as_float(row_ok ? __ldg(p.epi.gate_bits + (p.epi.row0 + m) * p.epi.ld_gate_bits + (nb >> 5)) : 0u);
                 } else if (post && gate_vec) {
 #pragma unroll
                     for (int it = 0; it < 8; ++it) {
@@ -885,7 +887,7 @@ __global__ void __launch_bounds__(KK_THREADS, 1) gemm_tc_pair_kernel(const __gri
 #pragma unroll
                         for (int it = 0; it < 8; ++it) {
                             const int rr = it * 4 + (lane >> 3), ch = lane & 7;
-                            const uint32_t gw_rr = __shfl_sync(0xFFFFFFFFu, gw, rr);      // every lane takes part (before any lane skips)
+                            const uint32_t gw_rr = __shfl_sync(0xFFFFFFFFu, __float_as_uint(g4[0].x), rr);   // every lane takes part (before any lane skips)
                             const int64_t mr = m0 + quarter * 32 + rr;
                             const int nc = nb + ch * 4;
                             if (mr >= p.M || nc >= p.N) continue;
