@@ -126,6 +126,22 @@ __device__ __forceinline__ void store_row(const SpmmParams& p, int64_t u, int c4
     if (p.Z_lp) store_lp4(p.Z_lp + u * p.ldz_lp + j, r[0], r[1], r[2], r[3]);
 }
 
+// store_row for the instances without the general epilogue (see spmm_group_kernel): nothing, or only a bit-packed
+// gate, between the sums and the stored row; pad columns of the last group are written as zeros, as store_row does.
+template <bool BITS>
+__device__ __forceinline__ void store_lean(const SpmmParams& p, int64_t u, int c4, float4 y) {
+    const int j = p.j0 + c4 * 4;
+    const int left = p.j0 + p.w - j;             // valid columns of this group (>= 1)
+    if (left < 4) { if (left < 2) y.y = 0.0f; if (left < 3) y.z = 0.0f; y.w = 0.0f; }
+    if constexpr (BITS) {
+        const uint32_t nib = (__ldg(p.out_bits + u * p.ld_bits + (j >> 5)) >> (j & 31)) & 0xFu;   // j % 4 == 0: one word
+        y.x = (nib & 1u) ? y.x * p.bits_scale : 0.0f; y.y = (nib & 2u) ? y.y * p.bits_scale : 0.0f;
+        y.z = (nib & 4u) ? y.z * p.bits_scale : 0.0f; y.w = (nib & 8u) ? y.w * p.bits_scale : 0.0f;
+    }
+    if (p.Z) *reinterpret_cast<float4*>(p.Z + u * p.ldz + j) = y;
+    if (p.Z_lp) store_lp4(p.Z_lp + u * p.ldz_lp + j, y.x, y.y, y.z, y.w);
+}
+
 __device__ __forceinline__ void fma4(float4& acc, float a, const float4& y) {
     acc.x = fmaf(a, y.x, acc.x); acc.y = fmaf(a, y.y, acc.y);
     acc.z = fmaf(a, y.z, acc.z); acc.w = fmaf(a, y.w, acc.w);
@@ -262,8 +278,16 @@ __device__ __forceinline__ void row_segment(const SpmmParams& p, int64_t b, int6
     }
 }
 
-template <int LPR, int VPL, bool LOSS = false>
+// Instances by what stands between the sums and the stored row -- the general epilogue's code costs the gather loop
+// registers under the cap, so the forms the epochs spend their time in have instances without it:
+//   EPI_PLAIN  nothing (every forward aggregation of an aggregate-first layer, every partial row of a long-row segment)
+//   EPI_BITS   a bit-packed gate only (the backward aggregation that produces a gated input gradient)
+//   EPI_LOSS   bias + soft-max cross-entropy (loss_epilogue)
+//   EPI_ANY    everything store_row knows
+enum { EPI_ANY = 0, EPI_LOSS = 1, EPI_PLAIN = 2, EPI_BITS = 3 };
+template <int LPR, int VPL, int EPI = EPI_ANY>
 __global__ void __launch_bounds__(256, VPL <= 2 ? SPMM_MINB : 1) spmm_group_kernel(const SpmmParams p) {
+    constexpr bool LOSS = EPI == EPI_LOSS, PLAIN = EPI == EPI_PLAIN || EPI == EPI_BITS;
     const int lig = threadIdx.x % LPR;
     const int64_t idx = p.idx_begin + ((int64_t)blockIdx.x * 256 + threadIdx.x) / LPR;
     if (idx >= p.idx_end) return;  // the whole group leaves together
@@ -285,7 +309,7 @@ __global__ void __launch_bounds__(256, VPL <= 2 ? SPMM_MINB : 1) spmm_group_kern
 #pragma unroll
     for (int v = 0; v < VPL; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
     unsigned keep = 0xFFFFFFFFu;
-    if (p.out_bits && p.bits_skip) {
+    if (!PLAIN && p.out_bits && p.bits_skip) {
         // Eq. 4: outputs the mask drops are never computed -- a lane whose four columns of this row are all
         // masked skips its gathers of every neighbour (the mask is known before the aggregation)
         const int64_t row = p.seg_perm ? __ldg(p.seg_perm + u) : u;
@@ -316,7 +340,13 @@ __global__ void __launch_bounds__(256, VPL <= 2 ? SPMM_MINB : 1) spmm_group_kern
 #pragma unroll
     for (int v = 0; v < VPL; ++v) {
         const int c4 = lig + v * LPR;
-        if (c4 < w4) store_row(p, u, c4, acc[v]);
+        if (c4 < w4) {
+            if constexpr (PLAIN) {
+                store_lean<EPI == EPI_BITS>(p, u, c4, acc[v]);
+            } else {
+                store_row(p, u, c4, acc[v]);
+            }
+        }
     }
 }
 
@@ -324,7 +354,7 @@ __global__ void __launch_bounds__(256, VPL <= 2 ? SPMM_MINB : 1) spmm_group_kern
 // records, column ids and values in one coalesced load each; every gathered row of Y is then a single
 // 512-byte request of the whole warp (lane = float4 column), RB of them in flight; entries of a row are
 // added in entry order, as everywhere else.
-template <int RB, int MAXE>
+template <int RB, int MAXE, int EPI = EPI_ANY>
 __global__ void __launch_bounds__(256, SPMM_SHORT_MINB) spmm_short_kernel(const SpmmParams p) {
     static_assert(RB * MAXE <= 32, "one lane per (row, entry)");
     const int lane = threadIdx.x & 31;
@@ -371,7 +401,13 @@ __global__ void __launch_bounds__(256, SPMM_SHORT_MINB) spmm_short_kernel(const 
 #pragma unroll
     for (int k = 0; k < RB; ++k) {
         const int64_t u = __shfl_sync(0xFFFFFFFFu, rc.w, k);
-        if (idx0 + k < p.idx_end && col_ok && (!DEBUG_BOUNDS || u >= 0)) store_row(p, u, lane, acc[k]);
+        if (idx0 + k < p.idx_end && col_ok && (!DEBUG_BOUNDS || u >= 0)) {
+            if constexpr (EPI == EPI_PLAIN || EPI == EPI_BITS) {      // as in spmm_group_kernel
+                store_lean<EPI == EPI_BITS>(p, u, lane, acc[k]);
+            } else {
+                store_row(p, u, lane, acc[k]);
+            }
+        }
     }
 }
 
@@ -558,7 +594,16 @@ void launch_group(const SpmmParams& p, cudaStream_t s) {
     if (units <= 0) return;
     const int per_block = 256 / LPR;
     const int64_t blocks = (units + per_block - 1) / per_block;
-    spmm_group_kernel<LPR, VPL, LOSS><<<(unsigned)blocks, 256, 0, s>>>(p);
+    // nothing between the sums and the stored row (or a partial row, which never has an epilogue): the plain instance
+    const bool no_terms = !p.bias && !p.relu && !p.drop && !p.gate && !p.residual;
+    const bool skips = p.out_bits && p.bits_skip;                  // the sampled aggregation: the general instance
+    // (one float4 per lane: the lean instances gain nothing there and the assembler spills a register in them)
+    constexpr bool lean = !LOSS && VPL >= 2;
+    if constexpr (lean) {
+        if (!skips && (p.partial || (no_terms && !p.out_bits))) { spmm_group_kernel<LPR, VPL, EPI_PLAIN><<<(unsigned)blocks, 256, 0, s>>>(p); return; }
+        if (!skips && no_terms && p.out_bits) { spmm_group_kernel<LPR, VPL, EPI_BITS><<<(unsigned)blocks, 256, 0, s>>>(p); return; }
+    }
+    spmm_group_kernel<LPR, VPL, LOSS ? EPI_LOSS : EPI_ANY><<<(unsigned)blocks, 256, 0, s>>>(p);
 }
 
 // The same packing for an aggregation with the loss epilogue (width <= 256: at most two float4 per lane
@@ -814,7 +859,11 @@ mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView&
                 constexpr int RB = SPMM_SHORT_RB, MAXE = SPMM_SHORT_MAXE;
                 const int64_t units = p.idx_end - p.idx_begin;
                 const int64_t warps = (units + RB - 1) / RB;
-                spmm_short_kernel<RB, MAXE><<<(unsigned)((warps + 7) / 8), 256, 0, s>>>(p);
+                const bool no_terms = !p.bias && !p.relu && !p.drop && !p.gate && !p.residual;
+                const unsigned grid_short = (unsigned)((warps + 7) / 8);
+                if (no_terms && !p.out_bits) spmm_short_kernel<RB, MAXE, EPI_PLAIN><<<grid_short, 256, 0, s>>>(p);
+                else if (no_terms && !p.bits_skip) spmm_short_kernel<RB, MAXE, EPI_BITS><<<grid_short, 256, 0, s>>>(p);
+                else spmm_short_kernel<RB, MAXE, EPI_ANY><<<grid_short, 256, 0, s>>>(p);
             } else {
                 dispatch(p, q == 0 ? (p.w <= SPMM_FOLD_WMAX ? SPMM_FOLD_MED : 1) : fold, s);
             }

@@ -98,8 +98,10 @@ def test_hot_aggregation_kernels_compile_without_register_spills(tmp_path):
     log = r.stdout + r.stderr
     entries = re.findall(r"Compiling entry function '(\S+)'.*?\n.*?\n\s+\d+ bytes stack frame, (\d+) bytes spill stores, (\d+) bytes spill loads", log)
     assert len(entries) > 50
+    # every instance of the group kernel but those with the loss epilogue (third template argument 1), the short-row
+    # kernel and the plain combination kernel
     hot = [(name, int(st), int(ld)) for name, st, ld in entries
-           if ("spmm_group_kernel" in name and "Lb0E" in name) or "spmm_short_kernel" in name or "spmm_combine_kernelILb0" in name]
+           if re.search(r"spmm_group_kernelILi\d+ELi\d+ELi[023]E", name) or "spmm_short_kernel" in name or "spmm_combine_kernelILb0" in name]
     assert len(hot) >= 30
     spilled = [(name, st, ld) for name, st, ld in hot if st or ld]
     assert not spilled, spilled
