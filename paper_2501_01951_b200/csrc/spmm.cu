@@ -126,20 +126,55 @@ __device__ __forceinline__ void store_row(const SpmmParams& p, int64_t u, int c4
     if (p.Z_lp) store_lp4(p.Z_lp + u * p.ldz_lp + j, r[0], r[1], r[2], r[3]);
 }
 
-// store_row for the instances without the general epilogue (see spmm_group_kernel): nothing, or only a bit-packed
-// gate, between the sums and the stored row; pad columns of the last group are written as zeros, as store_row does.
-template <bool BITS>
+// What stands between the sums and the stored row -- the general epilogue's code costs the gather loop registers
+// under the cap, so the forms the epochs spend their time in have instances without it:
+//   EPI_PLAIN  nothing (every forward aggregation of an aggregate-first layer, every partial row of a long-row segment)
+//   EPI_BITS   a bit-packed gate only (the backward aggregation that produces a gated input gradient)
+//   EPI_BIAS   bias, then ReLU if asked (the forward aggregation of an update-first layer)
+//   EPI_GATE   an fp32 gate only, 16-byte aligned with a leading dimension that is a multiple of 4
+//   EPI_LOSS   bias + soft-max cross-entropy (loss_epilogue)
+//   EPI_ANY    everything store_row knows
+enum { EPI_ANY = 0, EPI_LOSS = 1, EPI_PLAIN = 2, EPI_BITS = 3, EPI_BIAS = 4, EPI_GATE = 5 };
+constexpr bool epi_is_lean(int epi) { return epi >= EPI_PLAIN; }
+
+// store_row for the lean instances; pad columns of the last group are written as zeros, as store_row does.
+template <int EPI>
 __device__ __forceinline__ void store_lean(const SpmmParams& p, int64_t u, int c4, float4 y) {
     const int j = p.j0 + c4 * 4;
     const int left = p.j0 + p.w - j;             // valid columns of this group (>= 1)
-    if (left < 4) { if (left < 2) y.y = 0.0f; if (left < 3) y.z = 0.0f; y.w = 0.0f; }
-    if constexpr (BITS) {
+    if constexpr (EPI == EPI_BIAS) {
+        float4 b4;
+        if (left >= 4) b4 = __ldg(reinterpret_cast<const float4*>(p.bias + j));
+        else b4 = make_float4(__ldg(p.bias + j), left > 1 ? __ldg(p.bias + j + 1) : 0.0f, left > 2 ? __ldg(p.bias + j + 2) : 0.0f, 0.0f);
+        y.x += b4.x; y.y += b4.y; y.z += b4.z; y.w += b4.w;
+        if (p.relu) { y.x = fmaxf(y.x, 0.0f); y.y = fmaxf(y.y, 0.0f); y.z = fmaxf(y.z, 0.0f); y.w = fmaxf(y.w, 0.0f); }
+    }
+    if constexpr (EPI == EPI_GATE) {
+        const float4 g4 = __ldg(reinterpret_cast<const float4*>(p.gate + u * p.ld_gate + j));   // inside the row: ld_gate % 4 == 0
+        y.x = g4.x > 0.0f ? y.x * p.gate_scale : 0.0f; y.y = g4.y > 0.0f ? y.y * p.gate_scale : 0.0f;
+        y.z = g4.z > 0.0f ? y.z * p.gate_scale : 0.0f; y.w = g4.w > 0.0f ? y.w * p.gate_scale : 0.0f;
+    }
+    if constexpr (EPI == EPI_BITS) {
         const uint32_t nib = (__ldg(p.out_bits + u * p.ld_bits + (j >> 5)) >> (j & 31)) & 0xFu;   // j % 4 == 0: one word
         y.x = (nib & 1u) ? y.x * p.bits_scale : 0.0f; y.y = (nib & 2u) ? y.y * p.bits_scale : 0.0f;
         y.z = (nib & 4u) ? y.z * p.bits_scale : 0.0f; y.w = (nib & 8u) ? y.w * p.bits_scale : 0.0f;
     }
+    if (left < 4) { if (left < 2) y.y = 0.0f; if (left < 3) y.z = 0.0f; y.w = 0.0f; }
     if (p.Z) *reinterpret_cast<float4*>(p.Z + u * p.ldz + j) = y;
     if (p.Z_lp) store_lp4(p.Z_lp + u * p.ldz_lp + j, y.x, y.y, y.z, y.w);
+}
+
+// Which lean instance serves this launch (EPI_ANY: none does).
+inline int pick_epi(const SpmmParams& p) {
+    if (p.out_bits && p.bits_skip) return EPI_ANY;                 // the sampled aggregation skips gathers: general instance
+    if (p.partial) return EPI_PLAIN;                               // a partial row never has an epilogue
+    if (p.drop || p.residual) return EPI_ANY;
+    const bool bias = p.bias != nullptr || p.relu, gate = p.gate != nullptr, bits = p.out_bits != nullptr;
+    if (!bias && !gate && !bits) return EPI_PLAIN;
+    if (bits && !bias && !gate) return EPI_BITS;
+    if (bias && !gate && !bits && p.bias && (reinterpret_cast<uintptr_t>(p.bias) & 15u) == 0) return EPI_BIAS;
+    if (gate && !bias && !bits && (reinterpret_cast<uintptr_t>(p.gate) & 15u) == 0 && (p.ld_gate & 3) == 0) return EPI_GATE;
+    return EPI_ANY;
 }
 
 __device__ __forceinline__ void fma4(float4& acc, float a, const float4& y) {
@@ -278,16 +313,9 @@ __device__ __forceinline__ void row_segment(const SpmmParams& p, int64_t b, int6
     }
 }
 
-// Instances by what stands between the sums and the stored row -- the general epilogue's code costs the gather loop
-// registers under the cap, so the forms the epochs spend their time in have instances without it:
-//   EPI_PLAIN  nothing (every forward aggregation of an aggregate-first layer, every partial row of a long-row segment)
-//   EPI_BITS   a bit-packed gate only (the backward aggregation that produces a gated input gradient)
-//   EPI_LOSS   bias + soft-max cross-entropy (loss_epilogue)
-//   EPI_ANY    everything store_row knows
-enum { EPI_ANY = 0, EPI_LOSS = 1, EPI_PLAIN = 2, EPI_BITS = 3 };
 template <int LPR, int VPL, int EPI = EPI_ANY>
 __global__ void __launch_bounds__(256, VPL <= 2 ? SPMM_MINB : 1) spmm_group_kernel(const SpmmParams p) {
-    constexpr bool LOSS = EPI == EPI_LOSS, PLAIN = EPI == EPI_PLAIN || EPI == EPI_BITS;
+    constexpr bool LOSS = EPI == EPI_LOSS, PLAIN = epi_is_lean(EPI);
     const int lig = threadIdx.x % LPR;
     const int64_t idx = p.idx_begin + ((int64_t)blockIdx.x * 256 + threadIdx.x) / LPR;
     if (idx >= p.idx_end) return;  // the whole group leaves together
@@ -342,7 +370,7 @@ __global__ void __launch_bounds__(256, VPL <= 2 ? SPMM_MINB : 1) spmm_group_kern
         const int c4 = lig + v * LPR;
         if (c4 < w4) {
             if constexpr (PLAIN) {
-                store_lean<EPI == EPI_BITS>(p, u, c4, acc[v]);
+                store_lean<EPI>(p, u, c4, acc[v]);
             } else {
                 store_row(p, u, c4, acc[v]);
             }
@@ -402,8 +430,8 @@ __global__ void __launch_bounds__(256, SPMM_SHORT_MINB) spmm_short_kernel(const 
     for (int k = 0; k < RB; ++k) {
         const int64_t u = __shfl_sync(0xFFFFFFFFu, rc.w, k);
         if (idx0 + k < p.idx_end && col_ok && (!DEBUG_BOUNDS || u >= 0)) {
-            if constexpr (EPI == EPI_PLAIN || EPI == EPI_BITS) {      // as in spmm_group_kernel
-                store_lean<EPI == EPI_BITS>(p, u, lane, acc[k]);
+            if constexpr (epi_is_lean(EPI)) {      // as in spmm_group_kernel
+                store_lean<EPI>(p, u, lane, acc[k]);
             } else {
                 store_row(p, u, lane, acc[k]);
             }
@@ -595,13 +623,16 @@ void launch_group(const SpmmParams& p, cudaStream_t s) {
     const int per_block = 256 / LPR;
     const int64_t blocks = (units + per_block - 1) / per_block;
     // nothing between the sums and the stored row (or a partial row, which never has an epilogue): the plain instance
-    const bool no_terms = !p.bias && !p.relu && !p.drop && !p.gate && !p.residual;
-    const bool skips = p.out_bits && p.bits_skip;                  // the sampled aggregation: the general instance
     // (one float4 per lane: the lean instances gain nothing there and the assembler spills a register in them)
     constexpr bool lean = !LOSS && VPL >= 2;
     if constexpr (lean) {
-        if (!skips && (p.partial || (no_terms && !p.out_bits))) { spmm_group_kernel<LPR, VPL, EPI_PLAIN><<<(unsigned)blocks, 256, 0, s>>>(p); return; }
-        if (!skips && no_terms && p.out_bits) { spmm_group_kernel<LPR, VPL, EPI_BITS><<<(unsigned)blocks, 256, 0, s>>>(p); return; }
+        switch (pick_epi(p)) {
+            case EPI_PLAIN: spmm_group_kernel<LPR, VPL, EPI_PLAIN><<<(unsigned)blocks, 256, 0, s>>>(p); return;
+            case EPI_BITS: spmm_group_kernel<LPR, VPL, EPI_BITS><<<(unsigned)blocks, 256, 0, s>>>(p); return;
+            case EPI_BIAS: spmm_group_kernel<LPR, VPL, EPI_BIAS><<<(unsigned)blocks, 256, 0, s>>>(p); return;
+            case EPI_GATE: spmm_group_kernel<LPR, VPL, EPI_GATE><<<(unsigned)blocks, 256, 0, s>>>(p); return;
+            default: break;
+        }
     }
     spmm_group_kernel<LPR, VPL, LOSS ? EPI_LOSS : EPI_ANY><<<(unsigned)blocks, 256, 0, s>>>(p);
 }
@@ -859,10 +890,12 @@ mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView&
                 constexpr int RB = SPMM_SHORT_RB, MAXE = SPMM_SHORT_MAXE;
                 const int64_t units = p.idx_end - p.idx_begin;
                 const int64_t warps = (units + RB - 1) / RB;
-                const bool no_terms = !p.bias && !p.relu && !p.drop && !p.gate && !p.residual;
                 const unsigned grid_short = (unsigned)((warps + 7) / 8);
-                if (no_terms && !p.out_bits) spmm_short_kernel<RB, MAXE, EPI_PLAIN><<<grid_short, 256, 0, s>>>(p);
-                else if (no_terms && !p.bits_skip) spmm_short_kernel<RB, MAXE, EPI_BITS><<<grid_short, 256, 0, s>>>(p);
+                const int epi_short = pick_epi(p);
+                if (epi_short == EPI_PLAIN) spmm_short_kernel<RB, MAXE, EPI_PLAIN><<<grid_short, 256, 0, s>>>(p);
+                else if (epi_short == EPI_BITS) spmm_short_kernel<RB, MAXE, EPI_BITS><<<grid_short, 256, 0, s>>>(p);
+                else if (epi_short == EPI_BIAS) spmm_short_kernel<RB, MAXE, EPI_BIAS><<<grid_short, 256, 0, s>>>(p);
+                else if (epi_short == EPI_GATE) spmm_short_kernel<RB, MAXE, EPI_GATE><<<grid_short, 256, 0, s>>>(p);
                 else spmm_short_kernel<RB, MAXE, EPI_ANY><<<grid_short, 256, 0, s>>>(p);
             } else {
                 dispatch(p, q == 0 ? (p.w <= SPMM_FOLD_WMAX ? SPMM_FOLD_MED : 1) : fold, s);
