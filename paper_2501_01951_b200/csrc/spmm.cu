@@ -363,16 +363,13 @@ __global__ void __launch_bounds__(256, VPL <= 2 ? SPMM_MINB : 1) spmm_group_kern
     }
     if constexpr (LOSS) {
         loss_epilogue<LPR, VPL>(p, u, lig, mask, acc);
-        return;
-    }
+    } else {
 #pragma unroll
-    for (int v = 0; v < VPL; ++v) {
-        const int c4 = lig + v * LPR;
-        if (c4 < w4) {
-            if constexpr (PLAIN) {
-                store_lean<EPI>(p, u, c4, acc[v]);
-            } else {
-                store_row(p, u, c4, acc[v]);
+        for (int v = 0; v < VPL; ++v) {
+            const int c4 = lig + v * LPR;
+            if (c4 < w4) {
+                if constexpr (PLAIN) store_lean<EPI>(p, u, c4, acc[v]);
+                else store_row(p, u, c4, acc[v]);
             }
         }
     }
@@ -602,17 +599,17 @@ __global__ void __launch_bounds__(256) spmm_combine_kernel(const SpmmParams p, i
             row[v] = s;
         }
         loss_epilogue<32, 2>(p, u, lane, 0xFFFFFFFFu, row);
-        return;
-    }
-    for (int c4 = lane; c4 < w4; c4 += 32) {
-        float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int64_t q = s0; q < s1; ++q) {
-            const int64_t slot = __ldg(seg_pos + q);
-            if (!index_ok(slot, p.n_partial, p.status, SITE_SPMM_SEG)) continue;
-            const float4 t = __ldg(reinterpret_cast<const float4*>(p.partial + slot * p.ldp) + c4);
-            s.x += t.x; s.y += t.y; s.z += t.z; s.w += t.w;
+    } else {
+        for (int c4 = lane; c4 < w4; c4 += 32) {
+            float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int64_t q = s0; q < s1; ++q) {
+                const int64_t slot = __ldg(seg_pos + q);
+                if (!index_ok(slot, p.n_partial, p.status, SITE_SPMM_SEG)) continue;
+                const float4 t = __ldg(reinterpret_cast<const float4*>(p.partial + slot * p.ldp) + c4);
+                s.x += t.x; s.y += t.y; s.z += t.z; s.w += t.w;
+            }
+            store_row(p, u, c4, s);
         }
-        store_row(p, u, c4, s);
     }
 }
 
