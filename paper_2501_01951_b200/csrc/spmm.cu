@@ -274,7 +274,7 @@ struct Cfg {
 // Accumulate entries [b, e) into acc[] for the lane's column groups, ascending entry order.
 // The (col, val) pair of the NEXT batch of LPR entries is requested before the current batch's gathers,
 // so that the index load's latency is hidden behind them instead of preceding every batch.
-template <int LPR, int VPL>
+template <int LPR, int VPL, bool FULL = false>     // FULL: the slice has exactly LPR * VPL column groups (no lane is idle)
 __device__ __forceinline__ void row_segment(const SpmmParams& p, int64_t b, int64_t e, int lig, unsigned mask,
                                             int w4, float4 (&acc)[VPL], unsigned keep = 0xFFFFFFFFu) {
     constexpr int U = Cfg<LPR, VPL>::U;
@@ -299,7 +299,7 @@ __device__ __forceinline__ void row_segment(const SpmmParams& p, int64_t b, int6
 #pragma unroll
                 for (int v = 0; v < VPL; ++v) {
                     const int c4 = lig + v * LPR;
-                    y[t][v] = (live && c4 < w4 && ((keep >> v) & 1u)) ? __ldg(yr + c4) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    y[t][v] = (live && (FULL || c4 < w4) && ((keep >> v) & 1u)) ? __ldg(yr + c4) : make_float4(0.f, 0.f, 0.f, 0.f);
                 }
             }
 #pragma unroll
@@ -313,7 +313,8 @@ __device__ __forceinline__ void row_segment(const SpmmParams& p, int64_t b, int6
     }
 }
 
-template <int LPR, int VPL, int EPI = EPI_ANY>
+// FULL (plain and bit-gate instances): the slice has exactly LPR * VPL column groups, so no load is predicated on its column.
+template <int LPR, int VPL, int EPI = EPI_ANY, bool FULL = false>
 __global__ void __launch_bounds__(256, VPL <= 2 ? SPMM_MINB : 1) spmm_group_kernel(const SpmmParams p) {
     constexpr bool LOSS = EPI == EPI_LOSS, PLAIN = epi_is_lean(EPI);
     const int lig = threadIdx.x % LPR;
@@ -351,7 +352,7 @@ __global__ void __launch_bounds__(256, VPL <= 2 ? SPMM_MINB : 1) spmm_group_kern
             }
         }
     }
-    row_segment<LPR, VPL>(p, b, e, lig, mask, w4, acc, keep);
+    row_segment<LPR, VPL, FULL>(p, b, e, lig, mask, w4, acc, keep);
     if (p.partial) {
         float4* dst = reinterpret_cast<float4*>(p.partial + idx * p.ldp);
 #pragma unroll
@@ -623,9 +624,16 @@ void launch_group(const SpmmParams& p, cudaStream_t s) {
     // (one float4 per lane: the lean instances gain nothing there and the assembler spills a register in them)
     constexpr bool lean = !LOSS && VPL >= 2;
     if constexpr (lean) {
+        const bool full = LPR >= 8 && ((p.w + 3) >> 2) == LPR * VPL;     // (narrow groups: nothing to gain)
         switch (pick_epi(p)) {
-            case EPI_PLAIN: spmm_group_kernel<LPR, VPL, EPI_PLAIN><<<(unsigned)blocks, 256, 0, s>>>(p); return;
-            case EPI_BITS: spmm_group_kernel<LPR, VPL, EPI_BITS><<<(unsigned)blocks, 256, 0, s>>>(p); return;
+            case EPI_PLAIN:
+                if (full) spmm_group_kernel<LPR, VPL, EPI_PLAIN, (LPR >= 8)><<<(unsigned)blocks, 256, 0, s>>>(p);
+                else spmm_group_kernel<LPR, VPL, EPI_PLAIN><<<(unsigned)blocks, 256, 0, s>>>(p);
+                return;
+            case EPI_BITS:
+                if (full) spmm_group_kernel<LPR, VPL, EPI_BITS, (LPR >= 8)><<<(unsigned)blocks, 256, 0, s>>>(p);
+                else spmm_group_kernel<LPR, VPL, EPI_BITS><<<(unsigned)blocks, 256, 0, s>>>(p);
+                return;
             case EPI_BIAS: spmm_group_kernel<LPR, VPL, EPI_BIAS><<<(unsigned)blocks, 256, 0, s>>>(p); return;
             case EPI_GATE: spmm_group_kernel<LPR, VPL, EPI_GATE><<<(unsigned)blocks, 256, 0, s>>>(p); return;
             default: break;
