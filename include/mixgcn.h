@@ -450,7 +450,8 @@ mixgcn_status mixgcn_layer_fwd(mixgcn_ctx* ctx, const mixgcn_graph* g, const mix
  * n_chunks <= 1.  (Same formulas; the sums within a row may run in another order than in the separate calls.)
  * Every other layer runs as the two separate steps inside this call.  MIXGCN_EUNSUPPORTED with OUT_ROWS_ONLY or
  * MIXGCN_OPT_LOSS_TRAIN_ROWS_ONLY = 1.  Device-visible conditions (empty mask, label out of range) as in
- * mixgcn_loss_softmax_xent. */
+ * mixgcn_loss_softmax_xent.  The update-first form keeps 4 n bytes of scratch (the per-row loss terms) in the
+ * context, allocated by the first call that needs it (a cudaMalloc; not covered by mixgcn_ctx_reserve). */
 mixgcn_status mixgcn_layer_fwd_loss(mixgcn_ctx* ctx, const mixgcn_graph* g, const mixgcn_layer_desc* desc,
                                     const float* X_in, const float* W, const float* bias, float* saved,
                                     float* dlogits, const int32_t* labels, const uint8_t* train_mask,
