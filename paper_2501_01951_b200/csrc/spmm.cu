@@ -380,8 +380,8 @@ __global__ void __launch_bounds__(256, VPL <= 2 ? SPMM_MINB : 1) spmm_group_kern
 // records, column ids and values in one coalesced load each; every gathered row of Y is then a single
 // 512-byte request of the whole warp (lane = float4 column), RB of them in flight; entries of a row are
 // added in entry order, as everywhere else.
-template <int RB, int MAXE, int EPI = EPI_ANY>
-__global__ void __launch_bounds__(256, SPMM_SHORT_MINB) spmm_short_kernel(const SpmmParams p) {
+template <int RB, int MAXE, int EPI = EPI_ANY, int VPL = 1>      // VPL float4 per lane: widths up to 128 * VPL
+__global__ void __launch_bounds__(256, VPL == 1 ? SPMM_SHORT_MINB : SPMM_MINB) spmm_short_kernel(const SpmmParams p) {
     static_assert(RB * MAXE <= 32, "one lane per (row, entry)");
     const int lane = threadIdx.x & 31;
     const int64_t idx0 = p.idx_begin + (((int64_t)blockIdx.x * 256 + threadIdx.x) >> 5) * RB;
@@ -403,35 +403,45 @@ __global__ void __launch_bounds__(256, SPMM_SHORT_MINB) spmm_short_kernel(const 
     }
     const int w4 = (p.w + 3) >> 2;
     const float* Yb = p.Y + p.j0;
-    const bool col_ok = lane < w4;
-    float4 acc[RB];
+    float4 acc[RB][VPL];
 #pragma unroll
-    for (int k = 0; k < RB; ++k) acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int k = 0; k < RB; ++k)
+#pragma unroll
+        for (int v = 0; v < VPL; ++v) acc[k][v] = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
     for (int e = 0; e < MAXE; ++e) {
-        float4 y[RB]; float ak[RB];
+        float4 y[RB][VPL]; float ak[RB];
 #pragma unroll
         for (int k = 0; k < RB; ++k) {
             const int ck = __shfl_sync(0xFFFFFFFFu, c, k + e * RB);
             ak[k] = __shfl_sync(0xFFFFFFFFu, a, k + e * RB);
             const int len_k = __shfl_sync(0xFFFFFFFFu, rc.z, k);
-            const bool live = e < len_k && col_ok && index_ok(ck, p.y_rows, p.status, SITE_SPMM_COL);
-            y[k] = live ? __ldg(reinterpret_cast<const float4*>(Yb + (int64_t)ck * p.ldy) + lane) : make_float4(0.f, 0.f, 0.f, 0.f);
+            const bool live = e < len_k && index_ok(ck, p.y_rows, p.status, SITE_SPMM_COL);
+            const float4* yr = reinterpret_cast<const float4*>(Yb + (int64_t)ck * p.ldy);
+#pragma unroll
+            for (int v = 0; v < VPL; ++v)
+                y[k][v] = (live && lane + 32 * v < w4) ? __ldg(yr + lane + 32 * v) : make_float4(0.f, 0.f, 0.f, 0.f);
         }
 #pragma unroll
         for (int k = 0; k < RB; ++k) {
             const int len_k = __shfl_sync(0xFFFFFFFFu, rc.z, k);
-            if (e < len_k) fma4(acc[k], ak[k], y[k]);
+            if (e < len_k) {
+#pragma unroll
+                for (int v = 0; v < VPL; ++v) fma4(acc[k][v], ak[k], y[k][v]);
+            }
         }
     }
 #pragma unroll
     for (int k = 0; k < RB; ++k) {
         const int64_t u = __shfl_sync(0xFFFFFFFFu, rc.w, k);
-        if (idx0 + k < p.idx_end && col_ok && (!DEBUG_BOUNDS || u >= 0)) {
-            if constexpr (epi_is_lean(EPI)) {      // as in spmm_group_kernel
-                store_lean<EPI>(p, u, lane, acc[k]);
-            } else {
-                store_row(p, u, lane, acc[k]);
+        if (idx0 + k < p.idx_end && (!DEBUG_BOUNDS || u >= 0)) {
+#pragma unroll
+            for (int v = 0; v < VPL; ++v) {
+                const int c4 = lane + 32 * v;
+                if (c4 < w4) {
+                    if constexpr (epi_is_lean(EPI)) store_lean<EPI>(p, u, c4, acc[k][v]);      // as in spmm_group_kernel
+                    else store_row(p, u, c4, acc[k][v]);
+                }
             }
         }
     }
@@ -902,6 +912,18 @@ mixgcn_status launch_spmm(mixgcn_ctx* ctx, const mixgcn_graph* g, const CsrView&
                 else if (epi_short == EPI_BIAS) spmm_short_kernel<RB, MAXE, EPI_BIAS><<<grid_short, 256, 0, s>>>(p);
                 else if (epi_short == EPI_GATE) spmm_short_kernel<RB, MAXE, EPI_GATE><<<grid_short, 256, 0, s>>>(p);
                 else spmm_short_kernel<RB, MAXE, EPI_ANY><<<grid_short, 256, 0, s>>>(p);
+            } else if (q == 3 && p.w <= 256 && SPMM_PACK_DEG[2] <= SPMM_SHORT_MAXE) {
+                // the same for widths up to 256: two float4 per lane, two rows per warp
+                constexpr int RB = SPMM_SHORT_RB / 2, MAXE = SPMM_SHORT_MAXE;
+                const int64_t units = p.idx_end - p.idx_begin;
+                const int64_t warps = (units + RB - 1) / RB;
+                const unsigned grid_short = (unsigned)((warps + 7) / 8);
+                const int epi_short = pick_epi(p);
+                if (epi_short == EPI_PLAIN) spmm_short_kernel<RB, MAXE, EPI_PLAIN, 2><<<grid_short, 256, 0, s>>>(p);
+                else if (epi_short == EPI_BITS) spmm_short_kernel<RB, MAXE, EPI_BITS, 2><<<grid_short, 256, 0, s>>>(p);
+                else if (epi_short == EPI_BIAS) spmm_short_kernel<RB, MAXE, EPI_BIAS, 2><<<grid_short, 256, 0, s>>>(p);
+                else if (epi_short == EPI_GATE) spmm_short_kernel<RB, MAXE, EPI_GATE, 2><<<grid_short, 256, 0, s>>>(p);
+                else spmm_short_kernel<RB, MAXE, EPI_ANY, 2><<<grid_short, 256, 0, s>>>(p);
             } else {
                 dispatch(p, q == 0 ? (p.w <= SPMM_FOLD_WMAX ? SPMM_FOLD_MED : 1) : fold, s);
             }
